@@ -1,0 +1,331 @@
+"""CPU oracle for the RepQuant inference hot path (arXiv 2402.05628).
+
+TEST INFRASTRUCTURE ONLY.  This file is the slow, plain, fp64 statement of what
+the hot path computes, written from the paper.  It is used by the tests, by the
+smoke check and by the benchmark's CPU-baseline leg; the product path never
+calls it.  It shares no code, tables or constants with the CUDA path and does
+not import it.
+
+Everything is numpy in float64.  Library primitives used as single steps:
+`numpy.matmul` (dense contraction), `numpy.rint` (round half to even),
+`numpy.exp`, `numpy.log`, `scipy.special.erf`.  There is no blocking, fusion or
+reordering beyond what the cited equations state.
+
+The oracle applies the *complex* quantizers of the quantization process
+(channel-wise uniform quantization of LayerNorm activations, log-sqrt2
+quantization of Softmax activations); the CUDA path only ever sees the
+reparameterized, simple quantizers.  Agreement between the two is therefore a
+check of the paper's equivalence claims as well as of the kernels.
+
+Pins (see tests/test_oracle_pins.py): every function below is tied to the
+paper's worked example, a closed form, an algebraic identity of Sec. III-C, a
+library routine for the un-quantized special case, or brute force on tiny
+inputs.  The end-to-end block (`block_forward`) has no external pin beyond the
+composition of its pinned parts: parity unpinned for the composition itself.
+
+Notation follows the paper: s, z quantization scale / zero-point; b bits;
+r1 = s / s~, r2 = z - z~; gamma~, beta~, W~, b~ the reparameterized parameters.
+Weights are stored [out features j, in features c], i.e. the transpose of the
+paper's W in X'W; the paper's "W[:, j]" is row j here.
+"""
+from __future__ import annotations
+
+import math
+from typing import Dict, Optional
+
+import numpy as np
+from scipy.special import erf as _erf
+
+F64 = np.float64
+
+
+# --------------------------------------------------------------------------------------
+# Sec. III-A.2  Efficient quantizers
+# --------------------------------------------------------------------------------------
+
+def uniform_scale_zero(x_low, x_up, bits: int):
+    """Eq. 6: s = (x_up - x_low) / (2^b - 1), z = round(-x_low / s).
+
+    Scales are stored in float32 by every consumer, so s is rounded to float32
+    once and z is computed from the stored value.
+    """
+    x_low = np.asarray(x_low, dtype=F64)
+    x_up = np.asarray(x_up, dtype=F64)
+    s = (x_up - x_low) / F64(2 ** bits - 1)
+    s = s.astype(np.float32).astype(F64)
+    z = np.rint(-x_low / s).astype(np.int64)
+    return s, z
+
+
+def quant_uniform(x, s, z, bits: int):
+    """Eq. 4: x_q = clip(round(x / s) + z, 0, 2^b - 1).  s, z broadcast against x
+    (scalars: layer-wise; length-D vectors: channel-wise, Sec. III-C.1).
+
+    Returns (codes int64, t float64) where t = x / s is the value handed to the
+    round operation (used by the tests to recognise rounding near-ties).
+    """
+    x = np.asarray(x, dtype=F64)
+    t = x / np.asarray(s, dtype=F64)
+    q = np.rint(t) + np.asarray(z, dtype=F64)
+    q = np.clip(q, 0.0, F64(2 ** bits - 1))
+    return q.astype(np.int64), t
+
+
+def dequant_uniform(q, s, z):
+    """Eq. 5: x_hat = s (x_q - z)."""
+    return np.asarray(s, dtype=F64) * (np.asarray(q, dtype=F64) - np.asarray(z, dtype=F64))
+
+
+def quant_log2(x, s, bits: int):
+    """Eq. 7: x_q = clip(round(-log2(x / s)), 0, 2^b - 1); x = 0 clips to the top code."""
+    x = np.asarray(x, dtype=F64)
+    with np.errstate(divide="ignore"):
+        t = -np.log2(x / F64(s))
+    q = np.clip(np.rint(t), 0.0, F64(2 ** bits - 1))
+    return q.astype(np.int64), t
+
+
+def dequant_log2(q, s):
+    """Eq. 8: x_hat = s 2^(-x_q)."""
+    return F64(s) * np.exp2(-np.asarray(q, dtype=F64))
+
+
+# --------------------------------------------------------------------------------------
+# Sec. III-C.1  LayerNorm activations: channel-wise quantization and its reparameterization
+# --------------------------------------------------------------------------------------
+
+def layernorm(X, gamma, beta, eps: float, rms: bool = False):
+    """Eq. 9 per token over the D hidden features: (X - E[X]) / sqrt(Var[X] + eps) * gamma + beta,
+    population variance.  `rms=True` is the mean-free variant (E[X] := 0, Var := E[X^2])."""
+    X = np.asarray(X, dtype=F64)
+    if rms:
+        mu = np.zeros((X.shape[0], 1), dtype=F64)
+    else:
+        mu = X.mean(axis=1, keepdims=True)
+    d = X - mu
+    var = (d * d).mean(axis=1, keepdims=True)
+    return d / np.sqrt(var + F64(eps)) * np.asarray(gamma, dtype=F64) + np.asarray(beta, dtype=F64)
+
+
+def reparam_layernorm(gamma, beta, s, z, W, b) -> Dict[str, np.ndarray]:
+    """Eqs. 10-14.  s~ = E[s]; z~ = E[z] rounded to an integer (the paper declares z~ in Z and
+    pulls r2 out of the round operation in Eq. 10, which needs integer r2); r1 = s / s~;
+    r2 = z - z~; beta~ = (beta + s*r2) / r1; gamma~ = gamma / r1 (Eq. 12);
+    W~[j, c] = r1[c] W[j, c]; b~[j] = b[j] - sum_c s[c] r2[c] W[j, c] (Eq. 14)."""
+    gamma = np.asarray(gamma, dtype=F64)
+    beta = np.asarray(beta, dtype=F64)
+    s = np.asarray(s, dtype=F64)
+    z = np.asarray(z, dtype=np.int64)
+    W = np.asarray(W, dtype=F64)
+    b = np.zeros(W.shape[0], dtype=F64) if b is None else np.asarray(b, dtype=F64)
+    s_t = s.mean()
+    z_t = int(np.rint(z.astype(F64).mean()))
+    r1 = s / s_t
+    r2 = (z - z_t).astype(F64)
+    return dict(s_t=F64(s_t), z_t=z_t, r1=r1, r2=r2,
+                gamma_t=gamma / r1, beta_t=(beta + s * r2) / r1,
+                W_t=W * r1[None, :], b_t=b - W @ (s * r2))
+
+
+def quant_weight_rtn(W, bits: int):
+    """Channel-wise (per output feature) uniform weight quantization, Eqs. 4-6 with round-to-nearest
+    (stand-in for GPTQ, which needs calibration Hessians).  Per row: x_low = min(row, 0),
+    x_up = max(row, 0) so that zero is representable and 0 <= z <= 2^b - 1; an all-zero row gets s = 1.
+    The scale is rounded to float32 (as stored) before the codes are taken."""
+    W = np.asarray(W, dtype=F64)
+    lo = np.minimum(W.min(axis=1), 0.0)
+    hi = np.maximum(W.max(axis=1), 0.0)
+    rng = hi - lo
+    s = np.where(rng > 0.0, rng / F64(2 ** bits - 1), 1.0)
+    s = s.astype(np.float32).astype(F64)
+    z = np.rint(-lo / s).astype(np.int64)
+    q, _ = quant_uniform(W, s[:, None], z[:, None], bits)
+    return q, s, z
+
+
+def int_gemm(q, w):
+    """acc[n, j] = sum_c q[n, c] w[j, c] in int64 (the integer inner loop of the quantized linear layer)."""
+    return np.asarray(q, dtype=np.int64) @ np.asarray(w, dtype=np.int64).T
+
+
+def linear(x_hat, w_codes, s_w, z_w, b):
+    """De-quantized activation times de-quantized weight (Eq. 5 on both operands) plus bias."""
+    W_hat = dequant_uniform(w_codes, np.asarray(s_w, dtype=F64)[:, None], np.asarray(z_w)[:, None])
+    y = np.asarray(x_hat, dtype=F64) @ W_hat.T
+    if b is not None:
+        y = y + np.asarray(b, dtype=F64)
+    return y
+
+
+def linear_after_layernorm(q, s, z, rp: Dict[str, np.ndarray], w_codes, s_w, z_w):
+    """Right-hand side of Eq. 13 applied to the channel-wise de-quantized LayerNorm activation:
+    X^' = s (q - z) per channel (Eq. 5); shifted activation (X^' + s*r2) / r1; times the quantized
+    reparameterized weight W~^ = s_w (w - z_w); plus b~ of Eq. 14 (which the paper forms from the
+    full-precision W before W~ is quantized)."""
+    x_hat = dequant_uniform(q, np.asarray(s, dtype=F64)[None, :], np.asarray(z)[None, :])
+    x_shift = (x_hat + (np.asarray(s, dtype=F64) * rp["r2"])[None, :]) / rp["r1"][None, :]
+    return linear(x_shift, w_codes, s_w, z_w, rp["b_t"])
+
+
+# --------------------------------------------------------------------------------------
+# Sec. III-C.2  Softmax activations: log-sqrt2 quantizer and its base-2 reparameterization
+# --------------------------------------------------------------------------------------
+
+def softmax_rows(S, valid_len: Optional[np.ndarray] = None):
+    """Row Softmax of Eq. 3.  `valid_len[i]` (optional) = number of leading keys row i may attend to
+    (causal masking is structural: masked keys take no part); masked outputs are returned as 0."""
+    S = np.asarray(S, dtype=F64)
+    if valid_len is not None:
+        cols = np.arange(S.shape[-1])[None, :]
+        mask = cols < np.asarray(valid_len)[:, None]
+        S = np.where(mask, S, -np.inf)
+    m = S.max(axis=-1, keepdims=True)
+    e = np.exp(S - m)
+    return e / e.sum(axis=-1, keepdims=True)
+
+
+def quant_logsqrt2(A, s, bits: int):
+    """Eq. 15, first line: A_q = clip(round(-log_sqrt2(A / s)), 0, 2^b - 1), the logarithm to base
+    sqrt(2) taken as ln(.) / ln(sqrt 2).  A = 0 gives +inf and clips to the top code."""
+    A = np.asarray(A, dtype=F64)
+    with np.errstate(divide="ignore"):
+        t = -np.log(A / F64(s)) / math.log(math.sqrt(2.0))
+    q = np.clip(np.rint(t), 0.0, F64(2 ** bits - 1))
+    return q.astype(np.int64), t
+
+
+def quant_logsqrt2_base2(A, s, bits: int):
+    """Eq. 15, second line: the same codes through -2 log2(A / s)."""
+    A = np.asarray(A, dtype=F64)
+    with np.errstate(divide="ignore"):
+        t = -2.0 * np.log2(A / F64(s))
+    q = np.clip(np.rint(t), 0.0, F64(2 ** bits - 1))
+    return q.astype(np.int64), t
+
+
+def dequant_logsqrt2(q, s):
+    """Eq. 16, first line: A^ = s sqrt(2)^(-A_q) = s 2^(-A_q / 2) (evaluated in the base-2 form, whose
+    base is exact in binary floating point)."""
+    return F64(s) * np.exp2(-np.asarray(q, dtype=F64) / 2.0)
+
+
+def dequant_log2_reparam(q, s):
+    """Eq. 16, last line, with Eq. 17: A^ = s~ 2^floor(-A_q / 2), s~ = s [1(A_q)(sqrt2 - 1) + 1],
+    1(.) the parity indicator."""
+    q = np.asarray(q, dtype=np.int64)
+    parity = (q % 2).astype(F64)
+    s_t = F64(s) * (parity * (math.sqrt(2.0) - 1.0) + 1.0)
+    return s_t * np.exp2(np.floor(-q.astype(F64) / 2.0))
+
+
+# --------------------------------------------------------------------------------------
+# Sec. III-A.1  Transformer block (Eqs. 1-3)
+# --------------------------------------------------------------------------------------
+
+def gelu(x):
+    """GELU, exact erf form."""
+    x = np.asarray(x, dtype=F64)
+    return 0.5 * x * (1.0 + _erf(x / math.sqrt(2.0)))
+
+
+def round_bf16(x):
+    """Round-to-nearest-even onto the bf16 grid (8 significant bits), straight from float64
+    (models a bf16-stored activation tensor; sub-normal and overflow ranges are not modelled)."""
+    x = np.asarray(x, dtype=F64)
+    m, e = np.frexp(x)                      # x = m 2^e, 0.5 <= |m| < 1
+    return np.ldexp(np.rint(m * 256.0) / 256.0, e)
+
+
+def attention(Qc, Kc, Vc, qp: dict, B: int, L: int, H: int, softmax_s: float, bits_p: int,
+              causal: bool, keep: bool = False):
+    """Eq. 3 per (batch, head) on de-quantized Q, K, V, with the Softmax output passed through the
+    log-sqrt2 quantizer (Eq. 15) and de-quantized by Eq. 16's first line.
+    Qc/Kc/Vc: [B*L, D] integer codes; qp: layer-wise (s, z) of q, k, v.  The scale is 1/sqrt(d_h)
+    (per-head feature size).  Returns O [B*L, D] and, if `keep`, scores / codes per (b, h)."""
+    M, D = Qc.shape
+    dh = D // H
+    Qh = dequant_uniform(Qc, qp["s_q"], qp["z_q"])
+    Kh = dequant_uniform(Kc, qp["s_k"], qp["z_k"])
+    Vh = dequant_uniform(Vc, qp["s_v"], qp["z_v"])
+    O = np.empty((M, D), dtype=F64)
+    kept = dict(S=[], p=[], t=[]) if keep else None
+    valid = (np.arange(L) + 1) if causal else None
+    for bi in range(B):
+        r = slice(bi * L, (bi + 1) * L)
+        for h in range(H):
+            c = slice(h * dh, (h + 1) * dh)
+            S = Qh[r, c] @ Kh[r, c].T / math.sqrt(dh)
+            A = softmax_rows(S, valid)
+            p, t = quant_logsqrt2(A, softmax_s, bits_p)
+            A_hat = dequant_logsqrt2(p, softmax_s)
+            if causal:
+                A_hat = np.where(np.arange(L)[None, :] < valid[:, None], A_hat, 0.0)
+            O[r, c] = A_hat @ Vh[r, c]
+            if keep:
+                kept["S"].append(S)
+                kept["p"].append(p)
+                kept["t"].append(t)
+    return O, kept
+
+
+def block_forward(w, keep: bool = False) -> Dict[str, np.ndarray]:
+    """Eqs. 1-2 with every matrix-multiplication input quantized (Sec. III-A.1, IV-A):
+    X_bar = MSA(LN(X)) + X,  Y = MLP(LN(X_bar)) + X_bar.
+
+    `w` is a workload (workloads.BlockInputs): full-precision parameters plus clipping bounds.
+    LayerNorm activations: channel-wise quantization (s, z per channel from Eq. 6).  Softmax:
+    log-sqrt2.  Every other activation: layer-wise uniform.  Weights: channel-wise RTN; the weights
+    that follow a LayerNorm are the reparameterized W~ (rounded to float32, as stored).
+    With bf16 activations the residual stream X_bar is stored in bf16.
+    """
+    cfg = w.cfg
+    B, L, D, H = cfg["B"], cfg["L"], cfg["D"], cfg["H"]
+    ba, bw, bp = cfg["bits_a"], cfg["bits_w"], cfg["bits_p"]
+    out: Dict[str, np.ndarray] = {}
+    x = np.asarray(w.x, dtype=F64)
+
+    def post_ln_linear(X_in, gamma, beta, lo, hi, W, b, tag):
+        X1 = layernorm(X_in, gamma, beta, cfg["eps"])
+        s, z = uniform_scale_zero(lo, hi, ba)
+        q, t = quant_uniform(X1, s[None, :], z[None, :], ba)            # channel-wise
+        rp = reparam_layernorm(gamma, beta, s, z, W, b)
+        W_t32 = rp["W_t"].astype(np.float32).astype(F64)
+        wc, s_w, z_w = quant_weight_rtn(W_t32, bw)
+        y = linear_after_layernorm(q, s, z, rp, wc, s_w, z_w)
+        if keep:
+            out[tag + "_codes"], out[tag + "_t"] = q, t
+            out[tag + "_s"], out[tag + "_z"] = s, z
+            out[tag + "_rp"], out[tag + "_wcodes"] = rp, wc
+            out[tag + "_sw"], out[tag + "_zw"] = s_w, z_w
+        return y
+
+    def requant(v, name):
+        lo, hi = w.bounds[name]
+        s, z = uniform_scale_zero(lo, hi, ba)
+        q, t = quant_uniform(v, s, z, ba)
+        if keep:
+            out[name + "_codes"], out[name + "_t"] = q, t
+        return q, float(s), int(z)
+
+    qkv = post_ln_linear(x, w.ln1_gamma, w.ln1_beta, w.ln1_lo, w.ln1_hi, w.w_qkv, w.b_qkv, "ln1")
+    Qc, s_q, z_q = requant(qkv[:, :D], "q")
+    Kc, s_k, z_k = requant(qkv[:, D:2 * D], "k")
+    Vc, s_v, z_v = requant(qkv[:, 2 * D:], "v")
+    qp = dict(s_q=s_q, z_q=z_q, s_k=s_k, z_k=z_k, s_v=s_v, z_v=z_v)
+    O, kept = attention(Qc, Kc, Vc, qp, B, L, H, w.softmax_scale, bp, cfg["causal"], keep)
+    if keep:
+        out["scores"], out["p_codes"], out["p_t"] = kept["S"], kept["p"], kept["t"]
+        out["attn_pre"] = O
+    Oc, s_o, z_o = requant(O, "attn")
+    wc, s_w, z_w = quant_weight_rtn(w.w_proj, bw)
+    x_bar = linear(dequant_uniform(Oc, s_o, z_o), wc, s_w, z_w, w.b_proj) + x
+    if cfg["act"] == "bf16":
+        x_bar = round_bf16(x_bar)
+    if keep:
+        out["x_bar"] = x_bar
+
+    h_pre = post_ln_linear(x_bar, w.ln2_gamma, w.ln2_beta, w.ln2_lo, w.ln2_hi, w.w_fc1, w.b_fc1, "ln2")
+    hc, s_h, z_h = requant(gelu(h_pre), "hidden")
+    wc, s_w, z_w = quant_weight_rtn(w.w_fc2, bw)
+    out["y"] = linear(dequant_uniform(hc, s_h, z_h), wc, s_w, z_w, w.b_fc2) + x_bar
+    return out
