@@ -1,0 +1,261 @@
+/*
+ * repq.h — C ABI of the RepQuant (arXiv 2402.05628) reparameterized quantized-inference hot path
+ * for NVIDIA B200 (sm_100a).
+ *
+ * The library evaluates the *inference process* of the paper: after scale reparameterization
+ * (Sec. III-C) every activation quantizer is a simple one — layer-wise uniform (Eqs. 4-5) for
+ * LayerNorm outputs and all other GEMM inputs, log2 with a parity-selected scale (Eqs. 15-17) for
+ * Softmax outputs — and every GEMM runs on integer codes.
+ *
+ * Conventions
+ *  - Every entry point returns a repq_status; 0 is success.  Nothing throws, aborts or prints.
+ *    repq_last_error() returns the message of the calling thread's last failure.
+ *  - Pointers marked [device] are caller-owned CUDA device pointers; [host] are host pointers.
+ *    The device entry points allocate no device memory: scratch comes from the `workspace` argument,
+ *    sized by the matching *_workspace_bytes() call.
+ *  - Device work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = default stream) and
+ *    the call returns without synchronising.
+ *  - Codes are unsigned integers in [0, 2^b - 1] exactly as Eq. 4 produces them.  4-bit codes are
+ *    packed two per byte (even index in the low nibble); 6- and 8-bit codes take one byte each.
+ *    Code tensors are row-major with a row stride in BYTES; float tensors use strides in ELEMENTS.
+ *  - Weights are stored [out features j, in features c] (row j is the paper's column W[:, j]).
+ *  - Zero-points are plain integers of any sign (Eq. 6 does not bound them).
+ */
+#ifndef REPQ_H_
+#define REPQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int repq_status;
+#define REPQ_OK 0
+#define REPQ_INVALID_ARG 1          /* NULL pointer, non-positive size, bits not in {4,6,8}, ... */
+#define REPQ_UNSUPPORTED 2          /* a size or combination the kernels do not cover */
+#define REPQ_ALIGNMENT 3            /* a pointer or stride violates the stated alignment */
+#define REPQ_WORKSPACE_TOO_SMALL 4
+#define REPQ_CUDA_ERROR 5           /* a CUDA runtime / driver call failed (message has the detail) */
+#define REPQ_TIMEOUT 6              /* a bounded device-side wait ran out (see repq_device_status) */
+
+#define REPQ_F32 0
+#define REPQ_BF16 1
+
+#define REPQ_NORM_LAYERNORM 0
+#define REPQ_NORM_RMS 1             /* mean-free variant: E[x] := 0, Var := E[x^2] */
+
+#define REPQ_OUT_F32 0
+#define REPQ_OUT_BF16 1
+#define REPQ_OUT_CODES 2            /* re-quantize with Eq. 4 into `out_bits` codes */
+
+#define REPQ_MAX_OUT_GROUPS 4
+
+/* Copies the calling thread's last error message (NUL-terminated, truncated to n) and returns its
+ * full length. */
+size_t repq_last_error(char* buf, size_t n);
+
+/* Library ABI version (bumped on any signature change). */
+int repq_abi_version(void);
+
+/* ------------------------------------------------------------------------------------------------
+ * One-time host-side preparation (not on the timed path)
+ * ---------------------------------------------------------------------------------------------- */
+
+/* Eq. 6: s = (x_up - x_low) / (2^b - 1) rounded to float32, z = round(-x_low / s), for n independent
+ * quantizers (n = D for channel-wise, n = 1 for layer-wise).  All pointers [host]. */
+repq_status repq_scale_zero_from_bounds(int n, const float* x_low, const float* x_up, int bits,
+                                        float* s, int32_t* z);
+
+/* Scale reparameterization for LayerNorm activations, Eqs. 10-14 (Sec. III-C.1).
+ * In  [host]: gamma, beta, s (float[D]), z (int32[D]) — LayerNorm affine factors and the channel-wise
+ *             quantizer; W (float N x D, row-major, dense), b (float[N] or NULL) — the next layer.
+ * Out [host]: gamma_t, beta_t (float[D]) = gamma / r1, (beta + s*r2) / r1; *s_t = mean(s);
+ *             *z_t = mean(z) rounded half-to-even to an integer (so r2 = z - z_t is integral, as
+ *             Eq. 10 needs); W_t (N x D) = W * r1 per input channel; b_t (float[N]) = b - W (s*r2).
+ * Arithmetic is float64, results rounded once to float32.  W_t may alias W; b_t may alias b. */
+repq_status repq_fold_ln(int D, int N, const float* gamma, const float* beta, const float* s,
+                         const int32_t* z, const float* W, const float* b, float* gamma_t,
+                         float* beta_t, float* s_t, int32_t* z_t, float* W_t, float* b_t);
+
+/* Channel-wise (per output feature) round-to-nearest weight quantization, Eqs. 4-6; bounds per row
+ * are min(row, 0) and max(row, 0) so that 0 <= z_w <= 2^b - 1; an all-zero row gets s_w = 1.
+ * In  [host]: W (float N x K, row-major, dense).
+ * Out [host]: codes (N rows of ld_codes_bytes bytes; ld_codes_bytes >= K*bits/8 rounded up, multiple
+ *             of 16), s_w (float[N]), z_w (int32[N]), w_row_sum (int32[N]) = sum_c codes[j, c]. */
+repq_status repq_pack_weights(int N, int K, int bits_w, const float* W, uint8_t* codes,
+                              int64_t ld_codes_bytes, float* s_w, int32_t* z_w, int32_t* w_row_sum);
+
+/* ------------------------------------------------------------------------------------------------
+ * Hot path, stage by stage
+ * ---------------------------------------------------------------------------------------------- */
+
+/* LayerNorm (Eq. 9) with the reparameterized affine factors (Eq. 12), followed by layer-wise uniform
+ * quantization (Eq. 4) with the scalar (s_t, z_t):
+ *     y = (x - E[x]) / sqrt(Var[x] + eps) * gamma_t + beta_t   per row, population variance
+ *     q = clip(round(y / s_t) + z_t, 0, 2^bits - 1)            round = half to even
+ * x [device]: rows x D, dtype REPQ_F32 or REPQ_BF16, row stride ldx elements; x and ldx must keep every
+ *   row 16-byte aligned.  D must be a multiple of 8 and at most 16384.
+ * gamma_t, beta_t [device] float[D].  codes [device]: rows of ld_codes_bytes bytes (4-bit: multiple of
+ *   4; 6/8-bit: multiple of 8).  row_sum [device] int32[rows] or NULL: sum of the row's codes (the
+ *   activation term of the GEMM's zero-point correction). */
+repq_status repq_ln_quant(const void* x, int x_dtype, int64_t rows, int D, int64_t ldx,
+                          const float* gamma_t, const float* beta_t, float eps, int norm_kind,
+                          float s_t, int z_t, int bits, uint8_t* codes, int64_t ld_codes_bytes,
+                          int32_t* row_sum, void* stream);
+
+/* Quantized linear layer / batched code-by-code product.  Inference form of Sec. III-A (integer
+ * inputs and weights of every matrix multiplication) with the compensation of Eqs. 13-14 already
+ * folded into the weights and bias:
+ *     acc[m, j]  = sum_c a[m, c] w[j, c]                                   (int32, exact)
+ *     corr[m, j] = acc - z_w[j] asum[m] - z_a wsum[j] + K z_a z_w[j]       (= sum (a - z_a)(w - z_w))
+ *     v          = alpha * s_a * s_w[j] * corr + bias[j]                   (float32)
+ *     v          = gelu(v) if `gelu`;  v += residual[m, j] if `residual`
+ *     out        = v (f32 / bf16)   or   clip(round(v / s_o) + z_o, 0, 2^out_bits - 1)
+ * A batch of batch_outer x batch_inner independent products shares every scalar; operand (bo, bi)
+ * starts at base + bo*stride_outer + bi*stride_inner. */
+typedef struct repq_gemm_desc {
+  int32_t M, N, K;
+  int32_t batch_outer, batch_inner;     /* both 1 for a plain GEMM */
+  /* activation codes a: [M, K] */
+  const uint8_t* a_codes;               /* [device] */
+  int32_t bits_a;                       /* 4, 6 or 8 */
+  int64_t lda_bytes, a_stride_outer, a_stride_inner;    /* bytes */
+  float s_a;                            /* layer-wise scale (s~ after a LayerNorm) */
+  int32_t z_a;                          /* layer-wise zero-point (z~) */
+  const int32_t* a_row_sum;             /* [device] int32[M], plain GEMM only; NULL = computed here */
+  /* weight codes w: [N, K] */
+  const uint8_t* w_codes;               /* [device] */
+  int32_t bits_w;
+  int64_t ldw_bytes, w_stride_outer, w_stride_inner;    /* bytes */
+  const float* s_w;                     /* [device] float[N] per output channel; NULL = s_w_scalar */
+  const int32_t* z_w;                   /* [device] int32[N]; NULL = z_w_scalar */
+  float s_w_scalar;
+  int32_t z_w_scalar;
+  const int32_t* w_row_sum;             /* [device] int32[N], plain GEMM only; NULL = computed here */
+  const float* bias;                    /* [device] float[N] (b~ after a LayerNorm) or NULL */
+  float alpha;                          /* e.g. 1/sqrt(d_h) for attention scores; 1 otherwise */
+  /* epilogue */
+  int32_t gelu;                         /* erf-form GELU */
+  const void* residual;                 /* [device] M x N, dtype residual_dtype, or NULL (plain GEMM) */
+  int32_t residual_dtype;
+  int64_t ld_residual;                  /* elements */
+  int32_t out_kind;                     /* REPQ_OUT_* */
+  int32_t out_bits;
+  int32_t out_groups;                   /* 1..4: output columns split into equal ranges, each with its
+                                           own (s_o, z_o) — e.g. 3 for a fused Q|K|V projection */
+  float out_scale[REPQ_MAX_OUT_GROUPS];
+  int32_t out_zero[REPQ_MAX_OUT_GROUPS];
+  void* out;                            /* [device] */
+  int64_t ldo, o_stride_outer, o_stride_inner;          /* elements (float kinds) or bytes (codes) */
+  int32_t* out_row_sum;                 /* [device] int32[M] or NULL: with REPQ_OUT_CODES, the row sums
+                                           of the produced codes are ADDED here (caller zero-fills) */
+  int32_t* acc_debug;                   /* [device] int32 M x N (dense) raw accumulators, or NULL */
+} repq_gemm_desc;
+
+repq_status repq_qgemm_workspace_bytes(const repq_gemm_desc* d, size_t* bytes);
+repq_status repq_qgemm(const repq_gemm_desc* d, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Softmax (Eq. 3) over each row of `scores`, then the log-sqrt2 quantizer in its base-2 form
+ * (Eq. 15, second line):  A = softmax(pre_scale * scores_row);
+ *     p = clip(round(-2 log2(A / s)), 0, 2^bits - 1).
+ * scores [device]: rows x L, REPQ_F32 or REPQ_BF16, row stride ld elements.
+ * Causal masking is structural: if causal_period > 0, row r sees only its first
+ *     min(L, (r mod causal_period) + 1 + causal_offset) keys;
+ * codes of masked keys are written as 2^bits - 1 and must not be read as probabilities.
+ * codes [device]: rows of ld_codes_bytes bytes (multiple of 4).  s > 0 is the log-sqrt2 scale. */
+repq_status repq_softmax_log2(const void* scores, int dtype, int64_t rows, int L, int64_t ld,
+                              float pre_scale, int causal_period, int causal_offset, float s, int bits,
+                              uint8_t* codes, int64_t ld_codes_bytes, void* stream);
+
+/* P.V with Softmax codes de-quantized by the reparameterized log2 rule (Eqs. 16-17):
+ *     A^[i, j] = s * 2^(-ceil(p/2)) * (sqrt2 if p odd else 1)
+ *     O[i, :]  = sum_j A^[i, j] * s_v * (v[j, :] - z_v)          (causal: j <= i + Lk - Lq only)
+ * for batch_outer x batch_inner (batch, head) pairs.  p [device]: per pair an Lq x Lk code matrix,
+ * row stride ldp_bytes, pair (bo, bi) at p + (bo*batch_inner + bi) * p_stride_pair bytes.
+ * v [device]: Lk x d_h codes, row stride ldv_bytes, pair at v + bo*v_stride_outer + bi*v_stride_inner.
+ * The output uses the same epilogue kinds as repq_qgemm (one group).  d_h must be a multiple of 16, at
+ * most 128. */
+typedef struct repq_pv_desc {
+  int32_t batch_outer, batch_inner, Lq, Lk, d_h;
+  const uint8_t* p_codes;
+  int32_t bits_p;
+  int64_t ldp_bytes, p_stride_pair;
+  float s_p;                            /* log-sqrt2 scale s */
+  const uint8_t* v_codes;
+  int32_t bits_v;
+  int64_t ldv_bytes, v_stride_outer, v_stride_inner;
+  float s_v;
+  int32_t z_v;
+  int32_t causal;
+  int32_t out_kind, out_bits;
+  float out_scale;
+  int32_t out_zero;
+  void* out;
+  int64_t ldo, o_stride_outer, o_stride_inner;
+  int32_t* out_row_sum;                 /* as in repq_gemm_desc; rows are indexed bo*Lq + i */
+} repq_pv_desc;
+
+repq_status repq_pv(const repq_pv_desc* d, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Whole block: Eqs. 1-2,  X_bar = MSA(LN(X)) + X,  Y = MLP(LN(X_bar)) + X_bar, all GEMM inputs
+ * quantized (LayerNorm -> QKV -> QK^T -> Softmax/log2 -> P.V -> proj -> LayerNorm -> fc1/GELU -> fc2).
+ * ---------------------------------------------------------------------------------------------- */
+typedef struct repq_linear_params {
+  const uint8_t* w_codes;               /* [device] packed by repq_pack_weights */
+  int64_t ldw_bytes;
+  const float* s_w;                     /* [device] float[N] */
+  const int32_t* z_w;                   /* [device] int32[N] */
+  const int32_t* w_row_sum;             /* [device] int32[N] */
+  const float* bias;                    /* [device] float[N] */
+} repq_linear_params;
+
+typedef struct repq_block_desc {
+  int32_t batch, seq, dim, heads, mlp;
+  int32_t bits_a, bits_w, bits_p;
+  int32_t causal;
+  int32_t norm_kind;
+  float eps;
+  int32_t act_dtype;                    /* dtype of x and of the stored residual stream X_bar */
+  int32_t out_dtype;                    /* dtype of y */
+} repq_block_desc;
+
+typedef struct repq_block_params {
+  const float* ln1_gamma_t;             /* [device] folded LayerNorm-1 factors */
+  const float* ln1_beta_t;
+  float ln1_s;
+  int32_t ln1_z;
+  repq_linear_params qkv;               /* N = 3*dim (q | k | v), K = dim, weights W~ */
+  float s_q, s_k, s_v;
+  int32_t z_q, z_k, z_v;
+  float softmax_s;                      /* log-sqrt2 scale */
+  float s_attn;
+  int32_t z_attn;                       /* quantizer of the attention output (input of proj) */
+  repq_linear_params proj;              /* N = K = dim */
+  const float* ln2_gamma_t;
+  const float* ln2_beta_t;
+  float ln2_s;
+  int32_t ln2_z;
+  repq_linear_params fc1;               /* N = mlp, K = dim, weights W~ */
+  float s_hidden;
+  int32_t z_hidden;                     /* quantizer of the GELU output (input of fc2) */
+  repq_linear_params fc2;               /* N = dim, K = mlp */
+} repq_block_params;
+
+repq_status repq_block_workspace_bytes(const repq_block_desc* d, size_t* bytes);
+
+/* x [device]: (batch*seq) x dim, dense, dtype act_dtype.  y [device]: same shape, dtype out_dtype. */
+repq_status repq_block_forward(const repq_block_desc* d, const repq_block_params* p, const void* x,
+                               void* y, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Device-side health word of the calling thread's current device: 0 = healthy; non-zero = a bounded
+ * wait inside a kernel gave up (the kernel drained and returned; results of that launch are
+ * invalid).  Synchronises the device.  `reset` != 0 clears it. */
+repq_status repq_device_status(int32_t* status, int reset);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* REPQ_H_ */

@@ -1,0 +1,50 @@
+// Shared host-side plumbing of the repq library: error reporting and argument checks.
+#pragma once
+#include <cuda_runtime.h>
+#include <cstdarg>
+#include <cstdint>
+#include <cstdio>
+#include <string>
+
+#include "../../include/repq.h"
+
+namespace repq {
+
+std::string& last_error_ref();
+
+inline repq_status fail(repq_status code, const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof(buf), fmt, ap);
+  va_end(ap);
+  last_error_ref() = buf;
+  return code;
+}
+
+#define REPQ_REQUIRE(cond, code, ...) \
+  do {                                \
+    if (!(cond)) return ::repq::fail((code), __VA_ARGS__); \
+  } while (0)
+
+#define REPQ_CUDA(call)                                                                   \
+  do {                                                                                    \
+    cudaError_t e__ = (call);                                                             \
+    if (e__ != cudaSuccess)                                                               \
+      return ::repq::fail(REPQ_CUDA_ERROR, "%s failed: %s", #call, cudaGetErrorString(e__)); \
+  } while (0)
+
+#define REPQ_TRY(call)                   \
+  do {                                   \
+    repq_status s__ = (call);            \
+    if (s__ != REPQ_OK) return s__;      \
+  } while (0)
+
+inline bool bits_ok(int b) { return b == 4 || b == 6 || b == 8; }
+inline int64_t code_row_bytes(int64_t n, int bits) { return bits == 4 ? (n + 1) / 2 : n; }
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+inline int64_t round_up(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
+
+int sm_count();
+
+}  // namespace repq

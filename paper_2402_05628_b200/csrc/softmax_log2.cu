@@ -1,0 +1,239 @@
+// Fused Softmax -> log2-domain codes of the log-sqrt2 quantizer (Eq. 3's Softmax, then Eq. 15).
+//
+// With m = max_j S_j and Z = sum_j 2^(c (S_j - m)), c = pre_scale * log2(e), the value handed to the
+// round operation of Eq. 15 is
+//     -2 log2(A_i / s) = 2 (log2 Z + log2 s) - 2 c (S_i - m),
+// so the probabilities themselves are never formed: one exp2 per element for Z, one FMA per element
+// for the code, and no underflow (a key whose probability would underflow simply lands on the top
+// code, as the clip in Eq. 15 demands).
+//
+// HBM-bound: each score is read once (128-bit loads, row kept in registers by a group of TPR threads)
+// and leaves as a 4-bit or 8-bit code.
+#include <cuda_bf16.h>
+#include <math_constants.h>
+
+#include "common.h"
+
+namespace repq {
+namespace {
+
+constexpr int kChunk = 8;
+constexpr int kVPT = 4;
+
+// Loads elements [idx, idx + 8) of a row; elements at or beyond `valid` become -inf.  `vec_ok` says
+// the row base is 16-byte aligned; a vector load is used only when it lies inside the row extent `ld`.
+__device__ __forceinline__ void load_scores(const float* row, int idx, int valid, int64_t ld, bool vec_ok,
+                                            float (&v)[kChunk]) {
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const int i0 = idx + 4 * h;
+    if (vec_ok && i0 + 4 <= ld && i0 < valid) {
+      const float4 a = __ldcs(reinterpret_cast<const float4*>(row + i0));
+      v[4 * h + 0] = a.x; v[4 * h + 1] = a.y; v[4 * h + 2] = a.z; v[4 * h + 3] = a.w;
+    } else {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) v[4 * h + e] = (i0 + e < valid) ? __ldcs(row + i0 + e) : -CUDART_INF_F;
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < kChunk; ++e)
+    if (idx + e >= valid) v[e] = -CUDART_INF_F;
+}
+
+__device__ __forceinline__ void load_scores(const __nv_bfloat16* row, int idx, int valid, int64_t ld,
+                                            bool vec_ok, float (&v)[kChunk]) {
+  if (vec_ok && idx + 8 <= ld && idx < valid) {
+    const uint4 a = __ldcs(reinterpret_cast<const uint4*>(row + idx));
+    const uint32_t w[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      v[2 * i] = __uint_as_float(w[i] << 16);
+      v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+  } else {
+#pragma unroll
+    for (int e = 0; e < kChunk; ++e)
+      v[e] = (idx + e < valid) ? __bfloat162float(row[idx + e]) : -CUDART_INF_F;
+  }
+#pragma unroll
+  for (int e = 0; e < kChunk; ++e)
+    if (idx + e >= valid) v[e] = -CUDART_INF_F;
+}
+
+template <int TPR, bool kMax>
+__device__ __forceinline__ float group_reduce(float v, float* red, int group_first_warp) {
+  constexpr int kShfl = TPR < 32 ? TPR : 32;
+#pragma unroll
+  for (int o = kShfl / 2; o > 0; o >>= 1) {
+    const float other = __shfl_xor_sync(0xffffffffu, v, o);
+    v = kMax ? fmaxf(v, other) : v + other;
+  }
+  if constexpr (TPR > 32) {
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    v = kMax ? -CUDART_INF_F : 0.f;
+#pragma unroll
+    for (int w = 0; w < TPR / 32; ++w) {
+      const float other = red[group_first_warp + w];
+      v = kMax ? fmaxf(v, other) : v + other;
+    }
+  }
+  return v;
+}
+
+template <typename T, int TPR, bool kPack4>
+__global__ void __launch_bounds__((TPR > 256 ? TPR : 256))
+softmax_log2_kernel(const T* __restrict__ scores, int64_t rows, int L, int64_t ld, bool vec_ok, float c,
+                    int causal_period, int causal_offset, float log2_s, int qmax,
+                    uint8_t* __restrict__ codes, int64_t ldc) {
+  constexpr int kBlock = TPR > 256 ? TPR : 256;
+  constexpr int kRowsPerBlock = kBlock / TPR;
+  __shared__ float red_a[kBlock / 32];
+  __shared__ float red_b[kBlock / 32];
+
+  const int tig = threadIdx.x % TPR;
+  const int group = threadIdx.x / TPR;
+  const int group_first_warp = (group * TPR) >> 5;
+  const int nchunks = (L + kChunk - 1) / kChunk;
+  const float fq = float(qmax);
+
+  for (int64_t base = int64_t(blockIdx.x) * kRowsPerBlock; base < rows;
+       base += int64_t(gridDim.x) * kRowsPerBlock) {
+    const int64_t row = base + group;
+    const bool live = row < rows;
+    const T* sr = scores + (live ? row : 0) * ld;
+    int valid = L;
+    if (causal_period > 0) {
+      const int64_t v = (row % causal_period) + 1 + causal_offset;
+      valid = v < L ? int(v) : L;
+      if (valid < 1) valid = 1;
+    }
+    if (!live) valid = 0;
+
+    float v[kVPT][kChunk];
+    float m = -CUDART_INF_F;
+#pragma unroll
+    for (int i = 0; i < kVPT; ++i) {
+      const int ch = tig + i * TPR;
+      if (ch < nchunks && ch * kChunk < valid) {
+        load_scores(sr, ch * kChunk, valid, ld, vec_ok, v[i]);
+      } else {
+#pragma unroll
+        for (int e = 0; e < kChunk; ++e) v[i][e] = -CUDART_INF_F;
+      }
+#pragma unroll
+      for (int e = 0; e < kChunk; ++e) m = fmaxf(m, v[i][e]);
+    }
+    m = group_reduce<TPR, true>(m, red_a, group_first_warp);
+    if (!live) m = 0.f;
+
+    float z = 0.f;
+#pragma unroll
+    for (int i = 0; i < kVPT; ++i) {
+#pragma unroll
+      for (int e = 0; e < kChunk; ++e) {
+        v[i][e] -= m;                       // <= 0, -inf for masked keys
+        z += exp2f(v[i][e] * c);
+      }
+    }
+    z = group_reduce<TPR, false>(z, red_b, group_first_warp);
+    const float k0 = 2.f * (log2f(z) + log2_s);
+    const float k1 = -2.f * c;
+
+    if (live) {
+      uint8_t* out = codes + row * ldc;
+#pragma unroll
+      for (int i = 0; i < kVPT; ++i) {
+        const int ch = tig + i * TPR;
+        if (ch < nchunks) {
+          uint32_t q[kChunk];
+#pragma unroll
+          for (int e = 0; e < kChunk; ++e) {
+            float t = fmaf(v[i][e], k1, k0);          // +inf for masked keys
+            t = fminf(fmaxf(t, 0.f), fq);
+            q[e] = uint32_t(__float2int_rn(t));
+          }
+          if constexpr (kPack4) {
+            uint32_t w = 0;
+#pragma unroll
+            for (int e = 0; e < kChunk; ++e) w |= q[e] << (4 * e);
+            reinterpret_cast<uint32_t*>(out)[ch] = w;
+          } else {
+            uint2 w;
+            w.x = q[0] | q[1] << 8 | q[2] << 16 | q[3] << 24;
+            w.y = q[4] | q[5] << 8 | q[6] << 16 | q[7] << 24;
+            reinterpret_cast<uint2*>(out)[ch] = w;
+          }
+        }
+      }
+    }
+  }
+}
+
+template <typename T, int TPR>
+repq_status launch(const T* scores, int64_t rows, int L, int64_t ld, bool vec_ok, float c, int period,
+                   int offset, float log2_s, int bits, uint8_t* codes, int64_t ldc, cudaStream_t st) {
+  constexpr int kBlock = TPR > 256 ? TPR : 256;
+  constexpr int kRowsPerBlock = kBlock / TPR;
+  const int64_t need = (rows + kRowsPerBlock - 1) / kRowsPerBlock;
+  const int64_t cap = int64_t(sm_count()) * 8;
+  const int grid = int(need < cap ? need : cap);
+  const int qmax = (1 << bits) - 1;
+  if (bits == 4)
+    softmax_log2_kernel<T, TPR, true><<<grid, kBlock, 0, st>>>(scores, rows, L, ld, vec_ok, c, period, offset, log2_s, qmax, codes, ldc);
+  else
+    softmax_log2_kernel<T, TPR, false><<<grid, kBlock, 0, st>>>(scores, rows, L, ld, vec_ok, c, period, offset, log2_s, qmax, codes, ldc);
+  REPQ_CUDA(cudaGetLastError());
+  return REPQ_OK;
+}
+
+template <typename T>
+repq_status dispatch(const T* scores, int64_t rows, int L, int64_t ld, bool vec_ok, float c, int period,
+                     int offset, float log2_s, int bits, uint8_t* codes, int64_t ldc, cudaStream_t st) {
+  const int nchunks = (L + kChunk - 1) / kChunk;
+#define REPQ_SM_CASE(TPR) \
+  if (nchunks <= TPR * kVPT) return launch<T, TPR>(scores, rows, L, ld, vec_ok, c, period, offset, log2_s, bits, codes, ldc, st);
+  REPQ_SM_CASE(8)
+  REPQ_SM_CASE(16)
+  REPQ_SM_CASE(32)
+  REPQ_SM_CASE(64)
+  REPQ_SM_CASE(128)
+  REPQ_SM_CASE(256)
+  REPQ_SM_CASE(512)
+#undef REPQ_SM_CASE
+  return fail(REPQ_UNSUPPORTED, "softmax_log2: L = %d exceeds 16384", L);
+}
+
+}  // namespace
+}  // namespace repq
+
+using namespace repq;
+
+extern "C" repq_status repq_softmax_log2(const void* scores, int dtype, int64_t rows, int L, int64_t ld,
+                                         float pre_scale, int causal_period, int causal_offset, float s,
+                                         int bits, uint8_t* codes, int64_t ld_codes_bytes, void* stream) {
+  REPQ_REQUIRE(rows >= 0 && L > 0, REPQ_INVALID_ARG, "softmax_log2: rows must be >= 0 and L > 0");
+  if (rows == 0) return REPQ_OK;
+  REPQ_REQUIRE(scores && codes, REPQ_INVALID_ARG, "softmax_log2: NULL pointer");
+  REPQ_REQUIRE(dtype == REPQ_F32 || dtype == REPQ_BF16, REPQ_INVALID_ARG, "softmax_log2: dtype must be REPQ_F32 or REPQ_BF16");
+  REPQ_REQUIRE(bits_ok(bits), REPQ_INVALID_ARG, "softmax_log2: bits must be 4, 6 or 8");
+  REPQ_REQUIRE(s > 0.f && pre_scale > 0.f, REPQ_INVALID_ARG, "softmax_log2: s and pre_scale must be positive");
+  REPQ_REQUIRE(ld >= L, REPQ_INVALID_ARG, "softmax_log2: ld < L");
+  REPQ_REQUIRE(causal_period >= 0, REPQ_INVALID_ARG, "softmax_log2: causal_period must be >= 0");
+  REPQ_REQUIRE(L <= 16384, REPQ_UNSUPPORTED, "softmax_log2: L = %d exceeds 16384", L);
+  const int64_t unit = bits == 4 ? 4 : 8;
+  const int64_t need = (int64_t(L) + 7) / 8 * unit;
+  REPQ_REQUIRE(ld_codes_bytes >= need, REPQ_INVALID_ARG,
+               "softmax_log2: ld_codes_bytes = %lld, need at least %lld (rows are written in groups of 8 codes)",
+               (long long)ld_codes_bytes, (long long)need);
+  REPQ_REQUIRE(aligned(codes, unit) && ld_codes_bytes % unit == 0, REPQ_ALIGNMENT,
+               "softmax_log2: codes rows must be %d-byte aligned", int(unit));
+  const size_t esz = dtype == REPQ_F32 ? 4 : 2;
+  REPQ_REQUIRE(aligned(scores, esz), REPQ_ALIGNMENT, "softmax_log2: scores pointer is not element-aligned");
+  const bool vec_ok = aligned(scores, 16) && (size_t(ld) * esz) % 16 == 0;
+  const float c = pre_scale * 1.4426950408889634f;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (dtype == REPQ_F32)
+    return dispatch(static_cast<const float*>(scores), rows, L, ld, vec_ok, c, causal_period, causal_offset, log2f(s), bits, codes, ld_codes_bytes, st);
+  return dispatch(static_cast<const __nv_bfloat16*>(scores), rows, L, ld, vec_ok, c, causal_period, causal_offset, log2f(s), bits, codes, ld_codes_bytes, st);
+}
