@@ -1,0 +1,179 @@
+"""Shared helpers of the GPU parity tests and of the smoke check: code unpacking, the near-tie
+protocol, float tolerances, and stage-level comparisons between the CUDA path and the CPU oracle."""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+REL_L2_TOL = 2e-3          # float outputs: relative L2 error
+MAX_ABS_TOL = 1e-2         # float outputs: max abs error as a fraction of max |ref|
+
+
+def unpack_codes(raw: np.ndarray, n: int, bits: int) -> np.ndarray:
+    """raw: uint8 [rows, ld_bytes] -> int64 [rows, n] (4-bit: low nibble = even index)."""
+    raw = np.asarray(raw, dtype=np.uint8)
+    if bits == 4:
+        lo = raw & 0x0F
+        hi = raw >> 4
+        out = np.stack([lo, hi], axis=-1).reshape(raw.shape[0], -1)
+    else:
+        out = raw
+    return out[:, :n].astype(np.int64)
+
+
+def pack_codes(q: np.ndarray, bits: int, ld_bytes: int) -> np.ndarray:
+    """int codes [rows, n] -> uint8 [rows, ld_bytes] in the library's layout (test-side packing)."""
+    q = np.asarray(q, dtype=np.uint8)
+    rows, n = q.shape
+    out = np.zeros((rows, ld_bytes), dtype=np.uint8)
+    if bits == 4:
+        if n % 2:
+            q = np.concatenate([q, np.zeros((rows, 1), dtype=np.uint8)], axis=1)
+        out[:, : q.shape[1] // 2] = q[:, 0::2] | (q[:, 1::2] << 4)
+    else:
+        out[:, :n] = q
+    return out
+
+
+def near_tie_report(q_gpu: np.ndarray, q_ref: np.ndarray, t_ref: np.ndarray, delta) -> dict:
+    """Bit-exactness of integer codes decided in float32 on the GPU and float64 in the oracle.
+
+    A mismatch is excused only if it is +-1 and the oracle's pre-rounding value t lies within `delta`
+    of a rounding tie (x.5).  Returns counts; `bad` must be 0.
+    """
+    q_gpu = np.asarray(q_gpu, dtype=np.int64)
+    q_ref = np.asarray(q_ref, dtype=np.int64)
+    diff = q_gpu != q_ref
+    n_mis = int(diff.sum())
+    if n_mis == 0:
+        return dict(total=q_ref.size, mismatch=0, excused=0, bad=0)
+    t = np.asarray(t_ref, dtype=np.float64)[diff]
+    d = np.broadcast_to(np.asarray(delta, dtype=np.float64), q_ref.shape)[diff]
+    with np.errstate(invalid="ignore"):
+        dist = np.abs(t - np.floor(t) - 0.5)
+    ok = (np.abs(q_gpu[diff] - q_ref[diff]) == 1) & (dist < d)
+    return dict(total=q_ref.size, mismatch=n_mis, excused=int(ok.sum()), bad=int((~ok).sum()))
+
+
+def float_errors(out: np.ndarray, ref: np.ndarray):
+    out = np.asarray(out, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    rel_l2 = float(np.linalg.norm(out - ref) / max(np.linalg.norm(ref), 1e-300))
+    max_abs = float(np.abs(out - ref).max() / max(np.abs(ref).max(), 1e-300))
+    return rel_l2, max_abs
+
+
+def assert_float_close(out, ref, what=""):
+    rel_l2, max_abs = float_errors(out, ref)
+    assert rel_l2 <= REL_L2_TOL and max_abs <= MAX_ABS_TOL, "%s rel_l2=%.3e max_abs/max|ref|=%.3e" % (what, rel_l2, max_abs)
+    return rel_l2, max_abs
+
+
+# ------------------------------------------------------------------------------------------ stages
+
+def ln_case(rows: int, D: int, bf16: bool, seed: int, rms: bool = False, eps: float = 1e-6):
+    from workloads.kernels import affine_params, channel_profile, ln_calibration_bounds, ln_inputs
+    rng = np.random.default_rng(seed)
+    c, shift = channel_profile(rng, D, 1.0, 0.01, 50.0)
+    gamma, beta = affine_params(rng, D)
+    x_cal = ln_inputs(rng, 2048, c, shift, bf16)
+    x = ln_inputs(rng, rows, c, shift, bf16)
+    lo, hi = ln_calibration_bounds(x_cal, gamma, beta, eps, rms)
+    return x, gamma, beta, lo, hi
+
+
+def ln_delta(x, gamma_t, s_t, t_lw, eps, rms):
+    """Near-tie width for the fused LN+quant kernel: float32 rounding of (x - mu) * rstd * gamma~/s~ + beta~/s~.
+    The subtraction carries about 2^-22 |mu| (rounded mean) and the products 2^-23 relative each; the bound
+    below leaves a factor of 8 over that."""
+    x = np.asarray(x, dtype=np.float64)
+    mu = np.zeros((x.shape[0], 1)) if rms else x.mean(axis=1, keepdims=True)
+    d = x - mu
+    rstd = 1.0 / np.sqrt((d * d).mean(axis=1, keepdims=True) + eps)
+    return 2.0 ** -19 * (np.abs(x) + np.abs(mu)) * rstd * np.abs(gamma_t)[None, :] / s_t + 2.0 ** -20 * np.abs(t_lw)
+
+
+def check_ln_quant(rows, D, bits, bf16, seed=0, rms=False, eps=1e-6, pad_cols=0, want_sum=True):
+    """Runs the fused LN+quant kernel and compares its codes with the oracle's channel-wise codes."""
+    import torch
+    from oracle import repq_oracle as orc
+    from paper_2402_05628_b200 import binding as B
+
+    x, gamma, beta, lo, hi = ln_case(rows, D, bf16, seed, rms, eps)
+    # oracle: complex (channel-wise) quantizer
+    X1 = orc.layernorm(x, gamma, beta, eps, rms)
+    s, z = orc.uniform_scale_zero(lo, hi, bits)
+    q_ref, t_cw = orc.quant_uniform(X1, s[None, :], z[None, :], bits)
+    # CUDA path: folded parameters, layer-wise quantizer
+    W = np.zeros((1, D), dtype=np.float32)
+    gamma_t, beta_t, s_t, z_t, _, _ = B.repq_fold_ln(gamma, beta, s.astype(np.float32), z.astype(np.int32), W, None)
+    dev = torch.device("cuda:0")
+    xt = torch.from_numpy(x).to(dev)
+    if bf16:
+        xt = xt.to(torch.bfloat16)
+    if pad_cols:
+        buf = torch.zeros(rows, D + pad_cols, dtype=xt.dtype, device=dev)
+        buf[:, :D] = xt
+        xt = buf[:, :D]
+    ld = B.code_row_bytes(D, bits)
+    codes = torch.full((max(rows, 1), ld), 0xEE, dtype=torch.uint8, device=dev)[:rows]
+    row_sum = torch.full((max(rows, 1),), -1, dtype=torch.int32, device=dev)[:rows] if want_sum else None
+    B.repq_ln_quant(xt, torch.from_numpy(gamma_t).to(dev), torch.from_numpy(beta_t).to(dev), eps, s_t, z_t, bits,
+                    codes, row_sum, B.REPQ_NORM_RMS if rms else B.REPQ_NORM_LAYERNORM)
+    torch.cuda.synchronize()
+    if rows == 0:
+        return dict(total=0, mismatch=0, excused=0, bad=0)
+    q_gpu = unpack_codes(codes.cpu().numpy(), D, bits)
+    t_lw = t_cw + (z - z_t)[None, :]
+    rep = near_tie_report(q_gpu, q_ref, t_cw, ln_delta(x, gamma_t.astype(np.float64), s_t, t_lw, eps, rms))
+    if want_sum:
+        assert np.array_equal(row_sum.cpu().numpy().astype(np.int64), q_gpu.sum(axis=1)), "row sums"
+    # bytes beyond the row's codes are untouched
+    raw = codes.cpu().numpy()
+    used = D // 2 if bits == 4 else D
+    assert np.all(raw[:, used:] == 0xEE)
+    return rep
+
+
+def check_softmax_log2(rows, L, bits, bf16=False, seed=0, s=1.0, causal_period=0, pre_scale=1.0, ld_pad=None):
+    import torch
+    from oracle import repq_oracle as orc
+    from paper_2402_05628_b200 import binding as B
+    from workloads.kernels import softmax_logits, to_bf16_grid
+
+    rng = np.random.default_rng(seed)
+    S = softmax_logits(rng, rows, L)
+    if bf16:
+        S = to_bf16_grid(S)
+    valid = None
+    if causal_period:
+        valid = np.minimum(L, (np.arange(rows) % causal_period) + 1)
+    A = orc.softmax_rows(S.astype(np.float64) * np.float64(np.float32(pre_scale)), valid)
+    q_ref, t_ref = orc.quant_logsqrt2(A, s, bits)
+    dev = torch.device("cuda:0")
+    ld = ld_pad if ld_pad is not None else (L + 3) // 4 * 4
+    buf = torch.zeros(rows, ld, dtype=torch.float32, device=dev)
+    buf[:, :L] = torch.from_numpy(S).to(dev)
+    if bf16:
+        buf = buf.to(torch.bfloat16)
+    unit = 4 if bits == 4 else 8
+    ldc = max(B.code_row_bytes(L, bits), (L + 7) // 8 * unit)
+    codes = torch.full((rows, ldc), 0xEE, dtype=torch.uint8, device=dev)
+    B.repq_softmax_log2(buf, L, s, bits, codes, pre_scale, causal_period, 0)
+    torch.cuda.synchronize()
+    q_gpu = unpack_codes(codes.cpu().numpy(), L, bits)
+    delta = 2.0 ** -18 * np.maximum(1.0, np.abs(np.where(np.isfinite(t_ref), t_ref, 0.0)))
+    if valid is not None:
+        mask = np.arange(L)[None, :] < valid[:, None]
+        assert np.all(q_gpu[~mask] == 2 ** bits - 1)
+        q_gpu = np.where(mask, q_gpu, 0)
+        q_ref = np.where(mask, q_ref, 0)
+    return near_tie_report(q_gpu, q_ref, t_ref, delta)
+
+
+def smoke_check():
+    rep = check_ln_quant(rows=197, D=384, bits=4, bf16=False, seed=0)
+    assert rep["bad"] == 0, rep
+    rep = check_softmax_log2(rows=197 * 6, L=197, bits=4, seed=0)
+    assert rep["bad"] == 0, rep

@@ -1,0 +1,49 @@
+"""Stage-level parity of the CUDA kernels against the CPU oracle (through the C ABI)."""
+import numpy as np
+import pytest
+
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from paper_2402_05628_b200.build import build_library
+    build_library()
+
+
+@pytest.mark.parametrize("rows,D,bits,bf16", [
+    (197, 384, 4, False), (1000, 768, 4, True), (515, 768, 6, True), (333, 1024, 4, True),
+    (130, 4096, 4, True), (67, 8192, 8, True), (9, 16384, 4, False), (1, 8, 4, False), (77, 200, 8, True),
+    (4099, 768, 4, False),
+])
+def test_ln_quant_matches_channelwise_oracle(rows, D, bits, bf16):
+    rep = parity.check_ln_quant(rows, D, bits, bf16, seed=rows + D)
+    assert rep["bad"] == 0, rep
+    assert rep["mismatch"] <= max(2, 2e-4 * rep["total"]), rep
+
+
+def test_ln_quant_rms_strided_and_empty():
+    assert parity.check_ln_quant(300, 4096, 4, True, seed=3, rms=True, eps=1e-5)["bad"] == 0
+    assert parity.check_ln_quant(300, 768, 4, True, seed=4, pad_cols=8)["bad"] == 0
+    assert parity.check_ln_quant(300, 768, 8, False, seed=5, want_sum=False)["bad"] == 0
+    assert parity.check_ln_quant(0, 768, 4, True, seed=6)["total"] == 0
+
+
+@pytest.mark.parametrize("rows,L,bits,bf16", [
+    (1182, 197, 4, False), (700, 577, 4, False), (300, 2048, 8, False), (40, 8192, 4, False),
+    (64, 197, 6, True), (5, 1, 4, False), (33, 7, 8, False), (20, 16384, 4, True),
+])
+def test_softmax_log2_matches_logsqrt2_oracle(rows, L, bits, bf16):
+    rep = parity.check_softmax_log2(rows, L, bits, bf16, seed=rows + L)
+    assert rep["bad"] == 0, rep
+    assert rep["mismatch"] <= max(2, 2e-4 * rep["total"]), rep
+
+
+def test_softmax_log2_variants():
+    assert parity.check_softmax_log2(512, 256, 8, seed=1, causal_period=256)["bad"] == 0
+    assert parity.check_softmax_log2(394, 197, 4, seed=2, causal_period=197)["bad"] == 0
+    assert parity.check_softmax_log2(300, 197, 4, seed=3, s=0.7)["bad"] == 0
+    assert parity.check_softmax_log2(300, 197, 4, seed=4, pre_scale=0.125)["bad"] == 0
+    assert parity.check_softmax_log2(300, 197, 4, seed=5, ld_pad=197)["bad"] == 0      # unaligned rows
