@@ -1,0 +1,88 @@
+// Shared GEMM epilogue: zero-point correction, de-quantization, bias, GELU, residual, and the optional
+// re-quantization of Eq. 4.  Used by both the tensor-memory GEMM and the warp-MMA GEMM so that the two
+// produce identical results.
+#pragma once
+#include <cuda_bf16.h>
+#include <cstdint>
+
+#include "../../include/repq.h"
+
+namespace repq {
+
+struct EpilogueParams {
+  const float* s_w;        // per output channel or nullptr
+  const int32_t* z_w;      // per output channel or nullptr
+  float s_w_scalar;
+  int32_t z_w_scalar;
+  const float* bias;       // or nullptr
+  float scale_a;           // alpha * s_a
+  int32_t z_a;
+  int32_t K;
+  int32_t N;
+  int32_t gelu;
+  const void* residual;    // or nullptr
+  int32_t residual_bf16;
+  int64_t ld_residual;
+  int32_t out_kind;
+  int32_t qmax;            // 2^out_bits - 1
+  int32_t pack4;           // out_bits == 4
+  int32_t group_width;     // N / out_groups
+  float inv_out_scale[REPQ_MAX_OUT_GROUPS];
+  int32_t out_zero[REPQ_MAX_OUT_GROUPS];
+  void* out;
+  int64_t ldo;
+  int32_t* out_row_sum;    // or nullptr
+  int32_t* acc_debug;      // or nullptr, dense M x N
+};
+
+// Per-column constants of the epilogue, gathered once per output column.
+struct ColumnTerms {
+  float scale;    // alpha * s_a * s_w[j]
+  float bias;
+  int32_t z_w;
+  int32_t kzz;    // K * z_a * z_w[j] - z_a * wsum[j]
+  float inv_so;
+  float zo_lo, zo_hi;
+  int32_t zo;
+};
+
+__device__ __forceinline__ ColumnTerms column_terms(const EpilogueParams& p, int j, int32_t wsum_j) {
+  ColumnTerms c;
+  const float sw = p.s_w ? __ldg(p.s_w + j) : p.s_w_scalar;
+  c.z_w = p.z_w ? __ldg(p.z_w + j) : p.z_w_scalar;
+  c.scale = p.scale_a * sw;
+  c.bias = p.bias ? __ldg(p.bias + j) : 0.f;
+  // wrap-around integer arithmetic: only the final correction has to fit 32 bits
+  c.kzz = int32_t(uint32_t(p.K) * uint32_t(p.z_a) * uint32_t(c.z_w) - uint32_t(p.z_a) * uint32_t(wsum_j));
+  const int g = p.out_kind == REPQ_OUT_CODES ? j / p.group_width : 0;
+  c.inv_so = p.inv_out_scale[g];
+  c.zo = p.out_zero[g];
+  c.zo_lo = float(-c.zo);
+  c.zo_hi = float(p.qmax - c.zo);
+  return c;
+}
+
+__device__ __forceinline__ float gelu_erf(float v) { return 0.5f * v * (1.f + erff(v * 0.70710678118654752f)); }
+
+// acc -> corrected integer -> float value before the output conversion.
+__device__ __forceinline__ float epilogue_value(const EpilogueParams& p, const ColumnTerms& c, int32_t acc,
+                                                int32_t asum_m, int64_t m, int j) {
+  const int32_t corr = int32_t(uint32_t(acc) - uint32_t(c.z_w) * uint32_t(asum_m) + uint32_t(c.kzz));
+  float v = fmaf(c.scale, float(corr), c.bias);
+  if (p.gelu) v = gelu_erf(v);
+  if (p.residual) {
+    const int64_t off = m * p.ld_residual + j;
+    v += p.residual_bf16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(p.residual)[off])
+                         : static_cast<const float*>(p.residual)[off];
+  }
+  return v;
+}
+
+// Eq. 4 with the output quantizer: clip(round(v / s_o) + z_o, 0, qmax).
+__device__ __forceinline__ int32_t requantize(const ColumnTerms& c, float v) {
+  float t = v * c.inv_so;
+  t = fminf(fmaxf(t, c.zo_lo), c.zo_hi);
+  return __float2int_rn(t) + c.zo;
+}
+
+}  // namespace repq

@@ -1,0 +1,28 @@
+// Internal launchers shared between translation units of the repq library.
+#pragma once
+#include "common.h"
+#include "epilogue.cuh"
+
+namespace repq {
+
+// Row sums of a code matrix: out[r] = sum_c codes[r, c] (zero-point correction terms).
+repq_status launch_row_sum(const uint8_t* codes, int bits, int64_t rows, int64_t n, int64_t ld_bytes,
+                           int32_t* out, cudaStream_t st);
+
+// 4-bit packed codes -> one code per byte (dst rows of ld_dst bytes, zero-padded up to n_pad codes).
+repq_status launch_expand4(const uint8_t* src, int64_t rows, int64_t n, int64_t ld_src, uint8_t* dst,
+                           int64_t ld_dst, int64_t n_pad, cudaStream_t st);
+
+// Warp-MMA integer GEMM (any shape, batched).
+repq_status qgemm_mma(const repq_gemm_desc& d, const EpilogueParams& ep, cudaStream_t st);
+
+// Tensor-memory (tcgen05) integer GEMM: plain (unbatched) products with TMA-compatible operands.
+bool qgemm_tc_supported(const repq_gemm_desc& d);
+size_t qgemm_tc_workspace(const repq_gemm_desc& d);
+repq_status qgemm_tc(const repq_gemm_desc& d, const EpilogueParams& ep, void* ws, size_t ws_bytes,
+                     cudaStream_t st);
+
+// Device-side health word (bounded waits report here instead of trapping); nullptr on failure.
+int32_t* device_status_word();
+
+}  // namespace repq

@@ -177,3 +177,100 @@ def smoke_check():
     assert rep["bad"] == 0, rep
     rep = check_softmax_log2(rows=197 * 6, L=197, bits=4, seed=0)
     assert rep["bad"] == 0, rep
+
+
+def check_qgemm(M, N, K, bits_a, bits_w, out_kind="f32", gelu=False, residual=None, groups=1, out_bits=4, seed=0,
+                want_acc=True, want_out_sum=False, give_sums=False):
+    """repq_qgemm against the oracle: int32 accumulators bit-exact vs the int64 brute force, float outputs within
+    tolerance, re-quantized codes bit-exact up to counted near-ties."""
+    import torch
+    from oracle import repq_oracle as orc
+    from paper_2402_05628_b200 import binding as B
+    from workloads.kernels import gemm_codes, to_bf16_grid
+
+    rng = np.random.default_rng(seed)
+    a, w, s_a, z_a, s_w, z_w, bias = gemm_codes(rng, M, N, K, bits_a, bits_w)
+    res = None
+    if residual is not None:
+        res = rng.normal(0, 1.0, size=(M, N)).astype(np.float32)
+        if residual == "bf16":
+            res = to_bf16_grid(res)
+    # ---- oracle
+    acc_ref = orc.int_gemm(a, w)
+    v_pre = orc.linear(orc.dequant_uniform(a, s_a, z_a), w, s_w, z_w, bias)
+    v_ref = orc.gelu(v_pre) if gelu else v_pre
+    if res is not None:
+        v_ref = v_ref + res
+    # ---- CUDA path
+    dev = torch.device("cuda:0")
+    lda, ldw = B.code_row_bytes(K, bits_a), B.code_row_bytes(K, bits_w)
+    a_t = torch.from_numpy(pack_codes(a, bits_a, lda)).to(dev)
+    w_t = torch.from_numpy(pack_codes(w, bits_w, ldw)).to(dev)
+    kw = {}
+    if out_kind == "codes":
+        gw = N // groups
+        lo = [np.percentile(v_ref[:, g * gw:(g + 1) * gw], 1) for g in range(groups)]
+        hi = [np.percentile(v_ref[:, g * gw:(g + 1) * gw], 99) for g in range(groups)]
+        s_o, z_o = orc.uniform_scale_zero(np.array(lo), np.array(hi), out_bits)
+        ldo = B.code_row_bytes(N, out_bits)
+        out = torch.full((M, ldo), 0xEE, dtype=torch.uint8, device=dev)
+        kw = dict(out_kind=B.REPQ_OUT_CODES, out_bits=out_bits, out_scale=[float(v) for v in s_o],
+                  out_zero=[int(v) for v in z_o])
+        if want_out_sum:
+            kw["out_row_sum"] = torch.zeros(M, dtype=torch.int32, device=dev)
+    elif out_kind == "bf16":
+        out = torch.zeros(M, N, dtype=torch.bfloat16, device=dev)
+        kw = dict(out_kind=B.REPQ_OUT_BF16)
+    else:
+        out = torch.zeros(M, N, dtype=torch.float32, device=dev)
+    acc = torch.zeros(M, N, dtype=torch.int32, device=dev) if want_acc else None
+    res_t = None
+    if res is not None:
+        res_t = torch.from_numpy(res).to(dev)
+        if residual == "bf16":
+            res_t = res_t.to(torch.bfloat16)
+    if give_sums:
+        kw["a_row_sum"] = torch.from_numpy(a.sum(axis=1).astype(np.int32)).to(dev)
+        kw["w_row_sum"] = torch.from_numpy(w.sum(axis=1).astype(np.int32)).to(dev)
+    d = B.gemm_desc(M, N, K, a_t, bits_a, float(s_a), int(z_a), w_t, bits_w, out,
+                    s_w=torch.from_numpy(s_w).to(dev), z_w=torch.from_numpy(z_w).to(dev),
+                    bias=torch.from_numpy(bias).to(dev), gelu=gelu, residual=res_t, acc_debug=acc, **kw)
+    nws = B.repq_qgemm_workspace_bytes(d)
+    ws = torch.empty(max(nws, 16), dtype=torch.uint8, device=dev)
+    B.repq_qgemm(d, ws)
+    torch.cuda.synchronize()
+    assert B.repq_device_status() == 0
+    result = {}
+    if want_acc:
+        assert np.array_equal(acc.cpu().numpy().astype(np.int64), acc_ref), "int32 accumulators differ from brute force"
+    if out_kind == "codes":
+        gw = N // groups
+        q_gpu = unpack_codes(out.cpu().numpy(), N, out_bits)
+        rep = dict(total=0, mismatch=0, excused=0, bad=0)
+        for g in range(groups):
+            sl = slice(g * gw, (g + 1) * gw)
+            q_ref, t_ref = orc.quant_uniform(v_ref[:, sl], s_o[g], z_o[g], out_bits)
+            mag = np.abs(v_pre[:, sl] - bias[None, sl]) + np.abs(bias[None, sl]) + np.abs(v_ref[:, sl])
+            if res is not None:
+                mag = mag + np.abs(res[:, sl])
+            delta = 2.0 ** -19 * mag / s_o[g] + 2.0 ** -20 * np.abs(t_ref)
+            r = near_tie_report(q_gpu[:, sl], q_ref, t_ref, delta)
+            for k in rep:
+                rep[k] += r[k]
+        assert rep["bad"] == 0, rep
+        if want_out_sum:
+            assert np.array_equal(kw["out_row_sum"].cpu().numpy().astype(np.int64), q_gpu.sum(axis=1))
+        result = rep
+    else:
+        got = out.float().cpu().numpy()
+        if out_kind == "bf16":
+            # bf16 output = RNE(float32 value): compare against the oracle rounded the same way, 1 bf16 ulp
+            ref16 = orc.round_bf16(v_ref)
+            assert np.all(np.abs(got - ref16) <= np.abs(ref16) * 2.0 ** -7 + 1e-30)
+            rel, mx = float_errors(got, v_ref)
+            assert rel < 4e-3
+        else:
+            rel, mx = assert_float_close(got, v_ref, "qgemm")
+            assert rel < 1e-5, rel          # float32 epilogue on exact integers: far inside the tolerance
+        result = dict(rel_l2=rel, max_abs=mx)
+    return result

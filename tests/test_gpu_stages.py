@@ -47,3 +47,20 @@ def test_softmax_log2_variants():
     assert parity.check_softmax_log2(300, 197, 4, seed=3, s=0.7)["bad"] == 0
     assert parity.check_softmax_log2(300, 197, 4, seed=4, pre_scale=0.125)["bad"] == 0
     assert parity.check_softmax_log2(300, 197, 4, seed=5, ld_pad=197)["bad"] == 0      # unaligned rows
+
+
+@pytest.mark.parametrize("M,N,K,ba,bw", [
+    (64, 64, 64, 8, 8), (197, 1152, 384, 4, 4), (130, 72, 100, 4, 4), (33, 17, 50, 8, 8), (257, 200, 333, 6, 6),
+    (1, 8, 16, 4, 8), (300, 96, 11008, 4, 4), (64, 64, 4000, 8, 8),
+])
+def test_qgemm_accumulators_and_float_output(M, N, K, ba, bw):
+    parity.check_qgemm(M, N, K, ba, bw, seed=M + N + K)
+
+
+def test_qgemm_epilogues():
+    parity.check_qgemm(300, 192, 256, 4, 4, out_kind="bf16", seed=1)
+    parity.check_qgemm(300, 192, 256, 4, 4, out_kind="f32", residual="bf16", seed=2)
+    parity.check_qgemm(300, 192, 256, 4, 4, out_kind="bf16", residual="f32", gelu=True, seed=3)
+    parity.check_qgemm(300, 192, 256, 4, 4, out_kind="codes", groups=3, out_bits=4, seed=4)
+    parity.check_qgemm(300, 192, 256, 8, 8, out_kind="codes", gelu=True, out_bits=8, want_out_sum=True, seed=5)
+    parity.check_qgemm(300, 192, 256, 6, 6, out_kind="codes", out_bits=6, want_out_sum=True, give_sums=True, seed=6)
