@@ -177,6 +177,7 @@ def smoke_check():
     assert rep["bad"] == 0, rep
     rep = check_softmax_log2(rows=197 * 6, L=197, bits=4, seed=0)
     assert rep["bad"] == 0, rep
+    check_block("c1_vit_s", batch=1)
 
 
 def check_qgemm(M, N, K, bits_a, bits_w, out_kind="f32", gelu=False, residual=None, groups=1, out_bits=4, seed=0,
@@ -274,3 +275,115 @@ def check_qgemm(M, N, K, bits_a, bits_w, out_kind="f32", gelu=False, residual=No
             assert rel < 1e-5, rel          # float32 epilogue on exact integers: far inside the tolerance
         result = dict(rel_l2=rel, max_abs=mx)
     return result
+
+
+def check_pv(B_, H, Lq, Lk, dh, bits_p, bits_v, causal=False, out_kind="f32", out_bits=4, seed=0, s_p=1.0,
+             want_out_sum=False):
+    """repq_pv against the oracle: log-sqrt2 de-quantization (Eq. 16, first line) times de-quantized V."""
+    import torch
+    from oracle import repq_oracle as orc
+    from paper_2402_05628_b200 import binding as B
+    from workloads.kernels import softmax_logits
+
+    rng = np.random.default_rng(seed)
+    pairs = B_ * H
+    shift = Lk - Lq
+    valid = np.minimum(Lk, np.arange(Lq) + 1 + shift) if causal else None
+    S = softmax_logits(rng, pairs * Lq, Lk)
+    A = orc.softmax_rows(S, None if valid is None else np.tile(valid, pairs))
+    p, _ = orc.quant_logsqrt2(A, s_p, bits_p)                        # [pairs*Lq, Lk]
+    D = H * dh
+    Vc = rng.integers(0, 1 << bits_v, size=(B_ * Lk, D))
+    s_v = 0.05
+    z_v = int(rng.integers(0, 1 << bits_v))
+    A_hat = orc.dequant_logsqrt2(p, s_p)
+    if causal:
+        A_hat = np.where(np.arange(Lk)[None, :] < np.tile(valid, pairs)[:, None], A_hat, 0.0)
+    V_hat = orc.dequant_uniform(Vc, s_v, z_v)
+    O_ref = np.empty((B_ * Lq, D))
+    for b in range(B_):
+        for h in range(H):
+            pr = (b * H + h) * Lq
+            O_ref[b * Lq:(b + 1) * Lq, h * dh:(h + 1) * dh] = A_hat[pr:pr + Lq] @ V_hat[b * Lk:(b + 1) * Lk, h * dh:(h + 1) * dh]
+    dev = torch.device("cuda:0")
+    ldp = B.code_row_bytes(Lk, bits_p)
+    ldv = B.code_row_bytes(D, bits_v)
+    p_t = torch.from_numpy(pack_codes(p, bits_p, ldp)).to(dev)
+    v_t = torch.from_numpy(pack_codes(Vc, bits_v, ldv)).to(dev)
+    d = B.PvDesc()
+    d.batch_outer, d.batch_inner, d.Lq, d.Lk, d.d_h = B_, H, Lq, Lk, dh
+    d.p_codes, d.bits_p, d.ldp_bytes, d.p_stride_pair, d.s_p = p_t.data_ptr(), bits_p, ldp, Lq * ldp, s_p
+    d.v_codes, d.bits_v, d.ldv_bytes = v_t.data_ptr(), bits_v, ldv
+    d.v_stride_outer, d.v_stride_inner = Lk * ldv, (dh // 2 if bits_v == 4 else dh)
+    d.s_v, d.z_v, d.causal = s_v, z_v, int(causal)
+    row_sum = None
+    if out_kind == "codes":
+        s_o, z_o = orc.uniform_scale_zero(np.percentile(O_ref, 1), np.percentile(O_ref, 99), out_bits)
+        ldo = B.code_row_bytes(D, out_bits)
+        out = torch.full((B_ * Lq, ldo), 0xEE, dtype=torch.uint8, device=dev)
+        d.out_kind, d.out_bits, d.out_scale, d.out_zero = B.REPQ_OUT_CODES, out_bits, float(s_o), int(z_o)
+        d.ldo, d.o_stride_outer, d.o_stride_inner = ldo, Lq * ldo, (dh // 2 if out_bits == 4 else dh)
+        if want_out_sum:
+            row_sum = torch.zeros(B_ * Lq, dtype=torch.int32, device=dev)
+            d.out_row_sum = row_sum.data_ptr()
+    else:
+        dt = torch.float32 if out_kind == "f32" else torch.bfloat16
+        out = torch.zeros(B_ * Lq, D, dtype=dt, device=dev)
+        d.out_kind = B.REPQ_OUT_F32 if out_kind == "f32" else B.REPQ_OUT_BF16
+        d.ldo, d.o_stride_outer, d.o_stride_inner = D, Lq * D, dh
+    d.out = out.data_ptr()
+    B.repq_pv(d)
+    torch.cuda.synchronize()
+    if out_kind == "codes":
+        q_gpu = unpack_codes(out.cpu().numpy(), D, out_bits)
+        q_ref, t_ref = orc.quant_uniform(O_ref, s_o, z_o, out_bits)
+        absO = np.empty_like(O_ref)
+        for b in range(B_):
+            for h in range(H):
+                pr = (b * H + h) * Lq
+                absO[b * Lq:(b + 1) * Lq, h * dh:(h + 1) * dh] = A_hat[pr:pr + Lq] @ np.abs(V_hat[b * Lk:(b + 1) * Lk, h * dh:(h + 1) * dh])
+        delta = 2.0 ** -18 * absO / s_o + 2.0 ** -20 * np.abs(t_ref)
+        rep = near_tie_report(q_gpu, q_ref, t_ref, delta)
+        assert rep["bad"] == 0, rep
+        if want_out_sum:
+            assert np.array_equal(row_sum.cpu().numpy().astype(np.int64), q_gpu.sum(axis=1))
+        return rep
+    got = out.float().cpu().numpy()
+    if out_kind == "bf16":
+        ref16 = orc.round_bf16(O_ref)
+        assert np.all(np.abs(got - ref16) <= np.abs(ref16) * 2.0 ** -7 + 1e-30)
+        return dict(rel_l2=float_errors(got, O_ref)[0])
+    rel, mx = assert_float_close(got, O_ref, "pv")
+    assert rel < 1e-5, rel
+    return dict(rel_l2=rel, max_abs=mx)
+
+
+def check_block(name, batch, sample_items=None, out_dtype="f32", **overrides):
+    """Free-running block: the CUDA path (folded parameters, simple quantizers) against the oracle (complex
+    quantizers) on the block output, for the sampled batch items (items are independent, Eqs. 1-3)."""
+    import dataclasses
+    import torch
+    from oracle import repq_oracle as orc
+    from paper_2402_05628_b200.engine import QuantBlock
+    from workloads import make_block_inputs
+
+    w = make_block_inputs(name, batch=batch, **overrides)
+    L = w.cfg["L"]
+    blk = QuantBlock(w, out_dtype=torch.float32 if out_dtype == "f32" else torch.bfloat16)
+    x = torch.from_numpy(w.x).to(blk.device).to(blk.act_dtype)
+    y = blk.forward(x)
+    torch.cuda.synchronize()
+    y = y.float().cpu().numpy()
+    assert np.all(np.isfinite(y))
+    items = list(range(batch)) if sample_items is None else list(sample_items)
+    rows = np.concatenate([np.arange(i * L, (i + 1) * L) for i in items])
+    cfg = dict(w.cfg)
+    cfg["B"] = len(items)
+    w_s = dataclasses.replace(w, cfg=cfg, x=w.x[rows])
+    ref = orc.block_forward(w_s)["y"]
+    got = y[rows]
+    if out_dtype == "bf16":
+        rel, mx = float_errors(got, ref)
+        assert rel < 6e-3, rel
+        return rel, mx
+    return assert_float_close(got, ref, "block %s" % name)

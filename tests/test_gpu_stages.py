@@ -64,3 +64,18 @@ def test_qgemm_epilogues():
     parity.check_qgemm(300, 192, 256, 4, 4, out_kind="codes", groups=3, out_bits=4, seed=4)
     parity.check_qgemm(300, 192, 256, 8, 8, out_kind="codes", gelu=True, out_bits=8, want_out_sum=True, seed=5)
     parity.check_qgemm(300, 192, 256, 6, 6, out_kind="codes", out_bits=6, want_out_sum=True, give_sums=True, seed=6)
+
+
+@pytest.mark.parametrize("Bn,H,Lq,Lk,dh,bp,bv,causal", [
+    (2, 3, 197, 197, 64, 4, 4, False), (1, 2, 577, 577, 64, 4, 4, False), (1, 2, 300, 300, 128, 8, 4, True),
+    (2, 2, 64, 64, 32, 6, 6, False), (1, 1, 1, 130, 16, 8, 8, False), (1, 2, 100, 260, 64, 4, 8, True),
+    (1, 1, 70, 70, 96, 8, 8, True),
+])
+def test_pv_matches_oracle(Bn, H, Lq, Lk, dh, bp, bv, causal):
+    parity.check_pv(Bn, H, Lq, Lk, dh, bp, bv, causal, seed=Lq + dh)
+
+
+def test_pv_epilogues():
+    parity.check_pv(2, 2, 197, 197, 64, 4, 4, out_kind="bf16", seed=1)
+    parity.check_pv(2, 2, 197, 197, 64, 4, 4, out_kind="codes", out_bits=4, want_out_sum=True, seed=2)
+    parity.check_pv(1, 2, 130, 130, 128, 8, 4, causal=True, out_kind="codes", out_bits=8, want_out_sum=True, seed=3, s_p=0.7)
