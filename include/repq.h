@@ -250,6 +250,19 @@ repq_status repq_block_workspace_bytes(const repq_block_desc* d, size_t* bytes);
 repq_status repq_block_forward(const repq_block_desc* d, const repq_block_params* p, const void* x,
                                void* y, void* workspace, size_t workspace_bytes, void* stream);
 
+/* Number of stages repq_block_forward runs, and a variant of it that also measures them: CUDA events are
+ * recorded on `stream` between the stages, the call synchronises the stream and writes the duration
+ * of each stage in milliseconds to stage_ms [host, REPQ_BLOCK_STAGES floats], in the order
+ * ln1, qkv, scores, softmax, pv, proj, ln2, fc1, fc2.  Same results as repq_block_forward.
+ * (Measurement aid: the paper has no counterpart.) */
+#define REPQ_BLOCK_STAGES 9
+repq_status repq_block_forward_timed(const repq_block_desc* d, const repq_block_params* p, const void* x,
+                                     void* y, void* workspace, size_t workspace_bytes, void* stream,
+                                     float* stage_ms);
+
+/* Number of CUDA kernels this library has launched in the calling process so far. */
+uint64_t repq_launch_count(void);
+
 /* Device-side health word of the calling thread's current device: 0 = healthy; non-zero = a bounded
  * wait inside a kernel gave up (the kernel drained and returned; results of that launch are
  * invalid).  Synchronises the device.  `reset` != 0 clears it. */

@@ -26,8 +26,10 @@ EXPORTS = (
     "repq_last_error", "repq_abi_version", "repq_scale_zero_from_bounds", "repq_fold_ln",
     "repq_pack_weights", "repq_ln_quant", "repq_qgemm_workspace_bytes", "repq_qgemm",
     "repq_softmax_log2", "repq_pv", "repq_block_workspace_bytes", "repq_block_forward",
-    "repq_device_status",
+    "repq_device_status", "repq_block_forward_timed", "repq_launch_count",
 )
+REPQ_BLOCK_STAGES = 9
+BLOCK_STAGE_NAMES = ("ln1", "qkv", "scores", "softmax", "pv", "proj", "ln2", "fc1", "fc2")
 
 
 class RepqError(RuntimeError):
@@ -121,6 +123,10 @@ def lib() -> C.CDLL:
         _lib.repq_block_forward.argtypes = [C.POINTER(BlockDesc), C.POINTER(BlockParams), C.c_void_p, C.c_void_p,
                                             C.c_void_p, C.c_size_t, C.c_void_p]
         _lib.repq_device_status.argtypes = [C.POINTER(C.c_int32), C.c_int]
+        _lib.repq_block_forward_timed.argtypes = [C.POINTER(BlockDesc), C.POINTER(BlockParams), C.c_void_p, C.c_void_p,
+                                                  C.c_void_p, C.c_size_t, C.c_void_p, C.POINTER(C.c_float)]
+        _lib.repq_launch_count.restype = C.c_uint64
+        _lib.repq_launch_count.argtypes = []
         _lib.repq_scale_zero_from_bounds.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
         _lib.repq_fold_ln.argtypes = [C.c_int, C.c_int] + [C.c_void_p] * 12
         _lib.repq_pack_weights.argtypes = [C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_int64,
@@ -252,6 +258,20 @@ def repq_block_forward(d: BlockDesc, p: BlockParams, x: torch.Tensor, y: torch.T
     nbytes = workspace.numel() * workspace.element_size()
     _check(lib().repq_block_forward(C.byref(d), C.byref(p), _ptr(x), _ptr(y), _ptr(workspace), nbytes,
                                     _stream(stream)))
+
+
+def repq_block_forward_timed(d: BlockDesc, p: BlockParams, x: torch.Tensor, y: torch.Tensor, workspace: torch.Tensor,
+                             stream=None):
+    """Like repq_block_forward, but synchronises and returns the per-stage durations in milliseconds."""
+    nbytes = workspace.numel() * workspace.element_size()
+    ms = (C.c_float * REPQ_BLOCK_STAGES)()
+    _check(lib().repq_block_forward_timed(C.byref(d), C.byref(p), _ptr(x), _ptr(y), _ptr(workspace), nbytes,
+                                          _stream(stream), ms))
+    return [float(v) for v in ms]
+
+
+def repq_launch_count() -> int:
+    return int(lib().repq_launch_count())
 
 
 def repq_device_status(reset: bool = False) -> int:

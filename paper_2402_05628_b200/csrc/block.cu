@@ -95,8 +95,9 @@ extern "C" repq_status repq_block_workspace_bytes(const repq_block_desc* d, size
   return REPQ_OK;
 }
 
-extern "C" repq_status repq_block_forward(const repq_block_desc* dp, const repq_block_params* pp, const void* x,
-                                          void* y, void* workspace, size_t workspace_bytes, void* stream) {
+static repq_status block_forward_impl(const repq_block_desc* dp, const repq_block_params* pp, const void* x,
+                                      void* y, void* workspace, size_t workspace_bytes, void* stream,
+                                      cudaEvent_t* marks) {
   REPQ_REQUIRE(dp && pp && x && y, REPQ_INVALID_ARG, "block_forward: NULL argument");
   const repq_block_desc& d = *dp;
   const repq_block_params& p = *pp;
@@ -122,10 +123,17 @@ extern "C" repq_status repq_block_forward(const repq_block_desc* dp, const repq_
   uint8_t* hid_c = ws + L.off_hidden;
   int32_t* asum_h = reinterpret_cast<int32_t*>(ws + L.off_asum_h);
   void* gws = ws + L.off_gemm_ws;
+  int n_mark = 0;
+#define REPQ_MARK()                                            \
+  do {                                                         \
+    if (marks) REPQ_CUDA(cudaEventRecord(marks[n_mark++], st)); \
+  } while (0)
+  REPQ_MARK();
 
   // ---- X_bar = MSA(LN(X)) + X
   REPQ_TRY(repq_ln_quant(x, d.act_dtype, M, D, D, p.ln1_gamma_t, p.ln1_beta_t, d.eps, d.norm_kind, p.ln1_s, p.ln1_z,
                          d.bits_a, ln_c, L.ld_a, asum, stream));
+  REPQ_MARK();
   {
     repq_gemm_desc g = linear_desc(d, M, 3 * D, D, ln_c, L.ld_a, p.ln1_s, p.ln1_z, asum, p.qkv);
     g.out_kind = REPQ_OUT_CODES; g.out_bits = d.bits_a; g.out_groups = 3;
@@ -134,6 +142,7 @@ extern "C" repq_status repq_block_forward(const repq_block_desc* dp, const repq_
     g.out = qkv_c; g.ldo = L.ld_qkv;
     REPQ_TRY(repq_qgemm(&g, gws, L.gemm_ws, stream));
   }
+  REPQ_MARK();
   {
     // scores = Q K^T / sqrt(d_h) per (batch, head): both operands are activation codes
     repq_gemm_desc g{};
@@ -150,8 +159,10 @@ extern "C" repq_status repq_block_forward(const repq_block_desc* dp, const repq_
     g.o_stride_outer = int64_t(H) * S * L.ld_s; g.o_stride_inner = int64_t(S) * L.ld_s;
     REPQ_TRY(repq_qgemm(&g, nullptr, 0, stream));
   }
+  REPQ_MARK();
   REPQ_TRY(repq_softmax_log2(scores, REPQ_F32, int64_t(d.batch) * H * S, S, L.ld_s, 1.f, d.causal ? S : 0, 0,
                              p.softmax_s, d.bits_p, p_c, L.ld_p, stream));
+  REPQ_MARK();
   REPQ_CUDA(cudaMemsetAsync(asum_attn, 0, size_t(M) * 4, st));
   {
     repq_pv_desc v{};
@@ -166,6 +177,7 @@ extern "C" repq_status repq_block_forward(const repq_block_desc* dp, const repq_
     v.out_row_sum = asum_attn;
     REPQ_TRY(repq_pv(&v, stream));
   }
+  REPQ_MARK();
   {
     repq_gemm_desc g = linear_desc(d, M, D, D, attn_c, L.ld_a, p.s_attn, p.z_attn, asum_attn, p.proj);
     g.residual = x; g.residual_dtype = d.act_dtype; g.ld_residual = D;
@@ -173,9 +185,11 @@ extern "C" repq_status repq_block_forward(const repq_block_desc* dp, const repq_
     g.out = xbar; g.ldo = D;
     REPQ_TRY(repq_qgemm(&g, gws, L.gemm_ws, stream));
   }
+  REPQ_MARK();
   // ---- Y = MLP(LN(X_bar)) + X_bar
   REPQ_TRY(repq_ln_quant(xbar, d.act_dtype, M, D, D, p.ln2_gamma_t, p.ln2_beta_t, d.eps, d.norm_kind, p.ln2_s, p.ln2_z,
                          d.bits_a, ln_c, L.ld_a, asum, stream));
+  REPQ_MARK();
   REPQ_CUDA(cudaMemsetAsync(asum_h, 0, size_t(M) * 4, st));
   {
     repq_gemm_desc g = linear_desc(d, M, d.mlp, D, ln_c, L.ld_a, p.ln2_s, p.ln2_z, asum, p.fc1);
@@ -185,6 +199,7 @@ extern "C" repq_status repq_block_forward(const repq_block_desc* dp, const repq_
     g.out = hid_c; g.ldo = L.ld_h; g.out_row_sum = asum_h;
     REPQ_TRY(repq_qgemm(&g, gws, L.gemm_ws, stream));
   }
+  REPQ_MARK();
   {
     repq_gemm_desc g = linear_desc(d, M, D, d.mlp, hid_c, L.ld_h, p.s_hidden, p.z_hidden, asum_h, p.fc2);
     g.residual = xbar; g.residual_dtype = d.act_dtype; g.ld_residual = D;
@@ -192,7 +207,33 @@ extern "C" repq_status repq_block_forward(const repq_block_desc* dp, const repq_
     g.out = y; g.ldo = D;
     REPQ_TRY(repq_qgemm(&g, gws, L.gemm_ws, stream));
   }
+  REPQ_MARK();
   return REPQ_OK;
+}
+#undef REPQ_MARK
+
+extern "C" repq_status repq_block_forward(const repq_block_desc* d, const repq_block_params* p, const void* x,
+                                          void* y, void* workspace, size_t workspace_bytes, void* stream) {
+  return block_forward_impl(d, p, x, y, workspace, workspace_bytes, stream, nullptr);
+}
+
+extern "C" repq_status repq_block_forward_timed(const repq_block_desc* d, const repq_block_params* p,
+                                                const void* x, void* y, void* workspace, size_t workspace_bytes,
+                                                void* stream, float* stage_ms) {
+  REPQ_REQUIRE(stage_ms, REPQ_INVALID_ARG, "block_forward_timed: NULL stage_ms");
+  cudaEvent_t ev[REPQ_BLOCK_STAGES + 1];
+  int made = 0;
+  repq_status rc = REPQ_OK;
+  for (; made <= REPQ_BLOCK_STAGES; ++made)
+    if (cudaEventCreate(&ev[made]) != cudaSuccess) { rc = fail(REPQ_CUDA_ERROR, "cudaEventCreate failed"); break; }
+  if (rc == REPQ_OK) rc = block_forward_impl(d, p, x, y, workspace, workspace_bytes, stream, ev);
+  if (rc == REPQ_OK && cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    rc = fail(REPQ_CUDA_ERROR, "cudaStreamSynchronize failed: %s", cudaGetErrorString(cudaGetLastError()));
+  if (rc == REPQ_OK)
+    for (int i = 0; i < REPQ_BLOCK_STAGES; ++i)
+      if (cudaEventElapsedTime(&stage_ms[i], ev[i], ev[i + 1]) != cudaSuccess) { rc = fail(REPQ_CUDA_ERROR, "cudaEventElapsedTime failed"); break; }
+  for (int i = 0; i < made; ++i) cudaEventDestroy(ev[i]);
+  return rc;
 }
 
 extern "C" repq_status repq_device_status(int32_t* status, int reset) {

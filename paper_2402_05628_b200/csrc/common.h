@@ -47,4 +47,7 @@ inline int64_t round_up(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
 
 int sm_count();
 
+// Launch accounting (repq_launch_count).
+void note_launch(int n = 1);
+
 }  // namespace repq

@@ -2,6 +2,7 @@
 // reparameterization (Eqs. 10-14) and channel-wise weight quantization (Eqs. 4-6).
 // One-time preparation; all arithmetic in float64, results stored as float32 / int32.
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstring>
 #include <vector>
@@ -15,6 +16,8 @@ std::string& last_error_ref() {
   return msg;
 }
 
+uint64_t launches();
+
 int sm_count() {
   static int cached[64] = {0};
   int dev = 0;
@@ -27,9 +30,15 @@ int sm_count() {
   return cached[dev];
 }
 
+static std::atomic<uint64_t> g_launches{0};
+void note_launch(int n) { g_launches.fetch_add(uint64_t(n), std::memory_order_relaxed); }
+uint64_t launches() { return g_launches.load(std::memory_order_relaxed); }
+
 }  // namespace repq
 
 using namespace repq;
+
+extern "C" uint64_t repq_launch_count(void) { return repq::launches(); }
 
 extern "C" size_t repq_last_error(char* buf, size_t n) {
   const std::string& m = last_error_ref();

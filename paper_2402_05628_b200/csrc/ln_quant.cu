@@ -173,6 +173,7 @@ repq_status launch(const T* x, int64_t rows, int D, int64_t ldx, const float* g,
   else
     ln_quant_kernel<T, TPR, false><<<grid, kBlock, 0, st>>>(x, rows, D, ldx, g, b, eps, rms, inv_s, z, qmax, codes, ldc, row_sum);
   REPQ_CUDA(cudaGetLastError());
+  note_launch();
   return REPQ_OK;
 }
 

@@ -284,5 +284,6 @@ extern "C" repq_status repq_pv(const repq_pv_desc* d, void* stream) {
     if (p4) pv_kernel<2, true><<<grid, 256, 0, st>>>(P); else pv_kernel<2, false><<<grid, 256, 0, st>>>(P);
   }
   REPQ_CUDA(cudaGetLastError());
+  note_launch();
   return REPQ_OK;
 }

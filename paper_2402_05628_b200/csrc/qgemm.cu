@@ -145,6 +145,7 @@ repq_status launch_row_sum(const uint8_t* codes, int bits, int64_t rows, int64_t
   const int grid = int(blocks < 4096 ? blocks : 4096);
   row_sum_kernel<<<grid, 256, 0, st>>>(codes, bits, rows, n, ld_bytes, out);
   REPQ_CUDA(cudaGetLastError());
+  note_launch();
   return REPQ_OK;
 }
 
@@ -156,6 +157,7 @@ repq_status launch_expand4(const uint8_t* src, int64_t rows, int64_t n, int64_t 
   const int grid = int(blocks < 8192 ? blocks : 8192);
   expand4_kernel<<<grid, 256, 0, st>>>(src, rows, n, ld_src, dst, ld_dst, n_pad);
   REPQ_CUDA(cudaGetLastError());
+  note_launch();
   return REPQ_OK;
 }
 

@@ -220,6 +220,7 @@ repq_status qgemm_mma(const repq_gemm_desc& d, const EpilogueParams& ep, cudaStr
                                               d.w_stride_outer, d.w_stride_inner, d.o_stride_outer,
                                               d.o_stride_inner, a_al, w_al, ep);
   REPQ_CUDA(cudaGetLastError());
+  note_launch();
   return REPQ_OK;
 }
 

@@ -184,6 +184,7 @@ repq_status launch(const T* scores, int64_t rows, int L, int64_t ld, bool vec_ok
   else
     softmax_log2_kernel<T, TPR, false><<<grid, kBlock, 0, st>>>(scores, rows, L, ld, vec_ok, c, period, offset, log2_s, qmax, codes, ldc);
   REPQ_CUDA(cudaGetLastError());
+  note_launch();
   return REPQ_OK;
 }
 

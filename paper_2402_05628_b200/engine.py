@@ -117,3 +117,8 @@ class QuantBlock:
             y = torch.empty(x.shape, dtype=self.out_dtype, device=x.device)
         B.repq_block_forward(self.desc(batch), self.params(), x, y, self.workspace(batch), stream)
         return y
+
+    def forward_timed(self, x: torch.Tensor, y: torch.Tensor, stream=None) -> List[float]:
+        """Same pass with per-stage CUDA-event timing (synchronises); returns milliseconds per stage."""
+        batch = x.shape[0] // self.cfg["L"]
+        return B.repq_block_forward_timed(self.desc(batch), self.params(), x, y, self.workspace(batch), stream)
