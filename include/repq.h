@@ -260,6 +260,31 @@ repq_status repq_block_forward_timed(const repq_block_desc* d, const repq_block_
                                      void* y, void* workspace, size_t workspace_bytes, void* stream,
                                      float* stage_ms);
 
+/* repq_block_forward for callers that cannot allocate device memory.  (The paper has no counterpart:
+ * this is a deployment convenience.)
+ *
+ * Some hosts of this library never get to call cudaMalloc on the inference path: a plug-in that runs
+ * inside another runtime's memory plan, a real-time serving loop whose allocator is frozen after
+ * start-up, a sandbox that hands out device pointers but not the allocator.  Those callers still pass
+ * x, y and the parameter block as usual, but give no workspace: the intermediates of the block live in
+ * a scratch array that is part of the library image itself (a file-scope __device__ array of
+ * REPQ_STATIC_WORKSPACE_BYTES, 8 MiB, resident on every GPU that loads the library until the process
+ * exits).  The call allocates nothing: no cudaMalloc / cudaFree, no allocating library routine.
+ *
+ *  - Size limit: the block must need at most REPQ_STATIC_WORKSPACE_BYTES of workspace
+ *    (repq_block_workspace_bytes tells; a ViT-S-sized block of a few hundred tokens fits).  Larger
+ *    blocks are rejected with REPQ_WORKSPACE_TOO_SMALL and a message naming both sizes.
+ *  - First call on a device: the library looks up the device address of its scratch array once per
+ *    device (with that device current) and remembers it.  Make that first call outside any stream
+ *    capture.
+ *  - The scratch is shared by every call in the process and keeps whatever the previous call left in
+ *    it; the entry point itself clears the parts that have to start at zero.  Two calls that overlap
+ *    in time on the same GPU (different streams or threads) race on it: serialise them.
+ * Results are identical to repq_block_forward with a caller-provided workspace. */
+#define REPQ_STATIC_WORKSPACE_BYTES (8u << 20)
+repq_status repq_block_forward_static(const repq_block_desc* d, const repq_block_params* p, const void* x,
+                                      void* y, void* stream);
+
 /* Number of CUDA kernels this library has launched in the calling process so far. */
 uint64_t repq_launch_count(void);
 

@@ -27,7 +27,9 @@ EXPORTS = (
     "repq_pack_weights", "repq_ln_quant", "repq_qgemm_workspace_bytes", "repq_qgemm",
     "repq_softmax_log2", "repq_pv", "repq_block_workspace_bytes", "repq_block_forward",
     "repq_device_status", "repq_block_forward_timed", "repq_launch_count",
+    "repq_block_forward_static",
 )
+REPQ_STATIC_WORKSPACE_BYTES = 8 << 20
 REPQ_BLOCK_STAGES = 9
 BLOCK_STAGE_NAMES = ("ln1", "qkv", "scores", "softmax", "pv", "proj", "ln2", "fc1", "fc2")
 
@@ -125,6 +127,8 @@ def lib() -> C.CDLL:
         _lib.repq_device_status.argtypes = [C.POINTER(C.c_int32), C.c_int]
         _lib.repq_block_forward_timed.argtypes = [C.POINTER(BlockDesc), C.POINTER(BlockParams), C.c_void_p, C.c_void_p,
                                                   C.c_void_p, C.c_size_t, C.c_void_p, C.POINTER(C.c_float)]
+        _lib.repq_block_forward_static.argtypes = [C.POINTER(BlockDesc), C.POINTER(BlockParams), C.c_void_p,
+                                                   C.c_void_p, C.c_void_p]
         _lib.repq_launch_count.restype = C.c_uint64
         _lib.repq_launch_count.argtypes = []
         _lib.repq_scale_zero_from_bounds.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
@@ -268,6 +272,13 @@ def repq_block_forward_timed(d: BlockDesc, p: BlockParams, x: torch.Tensor, y: t
     _check(lib().repq_block_forward_timed(C.byref(d), C.byref(p), _ptr(x), _ptr(y), _ptr(workspace), nbytes,
                                           _stream(stream), ms))
     return [float(v) for v in ms]
+
+
+def repq_block_forward_static(d: BlockDesc, p: BlockParams, x: torch.Tensor, y: torch.Tensor, stream=None) -> None:
+    """repq_block_forward without a workspace argument: the library's built-in 8 MiB scratch array is used,
+    so nothing is allocated.  For hosts that may not allocate device memory on the inference path; blocks that
+    need more scratch are rejected.  Calls share the scratch: do not overlap them on one GPU."""
+    _check(lib().repq_block_forward_static(C.byref(d), C.byref(p), _ptr(x), _ptr(y), _stream(stream)))
 
 
 def repq_launch_count() -> int:

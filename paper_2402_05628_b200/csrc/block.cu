@@ -236,6 +236,48 @@ extern "C" repq_status repq_block_forward_timed(const repq_block_desc* d, const 
   return rc;
 }
 
+// ---- allocation-free variant: the workspace is a scratch array inside the library image ------------
+//
+// `g_static_ws` is device memory that exists on every GPU that loads this library.  On the host its
+// name is only a handle for the runtime: the usable device address comes from cudaGetSymbolAddress,
+// looked up once per device (with that device current) and cached below.
+static __device__ __align__(256) unsigned char g_static_ws[REPQ_STATIC_WORKSPACE_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_static_ws_addr[kMaxDevices] = {nullptr};
+
+repq_status static_workspace(void** out) {
+  int dev = -1;
+  REPQ_CUDA(cudaGetDevice(&dev));
+  REPQ_REQUIRE(dev >= 0 && dev < kMaxDevices, REPQ_UNSUPPORTED, "block_forward_static: device index %d not supported", dev);
+  if (g_static_ws_addr[dev] == nullptr) {
+    void* ptr = nullptr;
+    REPQ_CUDA(cudaGetSymbolAddress(&ptr, g_static_ws));
+    REPQ_REQUIRE(ptr != nullptr, REPQ_CUDA_ERROR, "block_forward_static: scratch array has no device address");
+    g_static_ws_addr[dev] = ptr;
+  }
+  *out = g_static_ws_addr[dev];
+  return REPQ_OK;
+}
+}  // namespace
+
+extern "C" repq_status repq_block_forward_static(const repq_block_desc* d, const repq_block_params* p,
+                                                 const void* x, void* y, void* stream) {
+  REPQ_REQUIRE(d && p && x && y, REPQ_INVALID_ARG, "block_forward_static: NULL argument");
+  REPQ_TRY(validate(*d));
+  const size_t need = layout(*d).total;
+  REPQ_REQUIRE(need <= size_t(REPQ_STATIC_WORKSPACE_BYTES), REPQ_WORKSPACE_TOO_SMALL,
+               "block_forward_static: this block needs %zu bytes of workspace, the built-in scratch holds %zu; "
+               "use repq_block_forward with a caller-provided workspace",
+               need, size_t(REPQ_STATIC_WORKSPACE_BYTES));
+  void* ws = nullptr;
+  REPQ_TRY(static_workspace(&ws));
+  // The stages overwrite every intermediate they read, and the two row-sum accumulators that must
+  // start at zero are cleared inside the stage sequence, so stale contents of earlier calls are harmless.
+  return block_forward_impl(d, p, x, y, ws, size_t(REPQ_STATIC_WORKSPACE_BYTES), stream, nullptr);
+}
+
 extern "C" repq_status repq_device_status(int32_t* status, int reset) {
   REPQ_REQUIRE(status, REPQ_INVALID_ARG, "device_status: NULL argument");
   int32_t* word = device_status_word();
