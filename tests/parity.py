@@ -233,9 +233,10 @@ def check_qgemm(M, N, K, bits_a, bits_w, out_kind="f32", gelu=False, residual=No
     if give_sums:
         kw["a_row_sum"] = torch.from_numpy(a.sum(axis=1).astype(np.int32)).to(dev)
         kw["w_row_sum"] = torch.from_numpy(w.sum(axis=1).astype(np.int32)).to(dev)
+    # the descriptor holds raw pointers: keep every tensor alive until the call has run
+    s_w_t, z_w_t, bias_t = (torch.from_numpy(v).to(dev) for v in (s_w, z_w, bias))
     d = B.gemm_desc(M, N, K, a_t, bits_a, float(s_a), int(z_a), w_t, bits_w, out,
-                    s_w=torch.from_numpy(s_w).to(dev), z_w=torch.from_numpy(z_w).to(dev),
-                    bias=torch.from_numpy(bias).to(dev), gelu=gelu, residual=res_t, acc_debug=acc, **kw)
+                    s_w=s_w_t, z_w=z_w_t, bias=bias_t, gelu=gelu, residual=res_t, acc_debug=acc, **kw)
     nws = B.repq_qgemm_workspace_bytes(d)
     ws = torch.empty(max(nws, 16), dtype=torch.uint8, device=dev)
     B.repq_qgemm(d, ws)
