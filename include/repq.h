@@ -57,7 +57,7 @@ typedef int repq_status;
 size_t repq_last_error(char* buf, size_t n);
 
 /* Library ABI version (bumped on any signature change). */
-int repq_abi_version(void);
+int repq_abi_version(void);   /* currently 2 */
 
 /* ------------------------------------------------------------------------------------------------
  * One-time host-side preparation (not on the timed path)
@@ -152,6 +152,8 @@ typedef struct repq_gemm_desc {
   int32_t* out_row_sum;                 /* [device] int32[M] or NULL: with REPQ_OUT_CODES, the row sums
                                            of the produced codes are ADDED here (caller zero-fills) */
   int32_t* acc_debug;                   /* [device] int32 M x N (dense) raw accumulators, or NULL */
+  int32_t causal;                       /* != 0: outputs with n > m + (N - M) are never read by the caller
+                                           and may be left unwritten (attention scores under a causal mask) */
 } repq_gemm_desc;
 
 repq_status repq_qgemm_workspace_bytes(const repq_gemm_desc* d, size_t* bytes);

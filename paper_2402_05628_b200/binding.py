@@ -56,7 +56,7 @@ class GemmDesc(C.Structure):
         ("out_kind", C.c_int32), ("out_bits", C.c_int32), ("out_groups", C.c_int32),
         ("out_scale", C.c_float * REPQ_MAX_OUT_GROUPS), ("out_zero", C.c_int32 * REPQ_MAX_OUT_GROUPS),
         ("out", C.c_void_p), ("ldo", C.c_int64), ("o_stride_outer", C.c_int64), ("o_stride_inner", C.c_int64),
-        ("out_row_sum", C.c_void_p), ("acc_debug", C.c_void_p),
+        ("out_row_sum", C.c_void_p), ("acc_debug", C.c_void_p), ("causal", C.c_int32),
     ]
 
 
@@ -298,7 +298,7 @@ def gemm_desc(M: int, N: int, K: int, a_codes: torch.Tensor, bits_a: int, s_a: f
               z_w_scalar=0, a_row_sum=None, w_row_sum=None, bias=None, alpha=1.0, gelu=False, residual=None,
               out_kind=REPQ_OUT_F32, out_bits=8, out_scale: Sequence[float] = (1.0,), out_zero: Sequence[int] = (0,),
               out_row_sum=None, acc_debug=None, batch=(1, 1), a_strides=(0, 0), w_strides=(0, 0), o_strides=(0, 0),
-              lda_bytes=None, ldw_bytes=None, ldo=None) -> GemmDesc:
+              lda_bytes=None, ldw_bytes=None, ldo=None, causal=False) -> GemmDesc:
     """Fills a GemmDesc from torch tensors (pointer and stride marshalling only)."""
     d = GemmDesc()
     d.M, d.N, d.K = M, N, K
@@ -323,4 +323,5 @@ def gemm_desc(M: int, N: int, K: int, a_codes: torch.Tensor, bits_a: int, s_a: f
     d.ldo = out.stride(0) if ldo is None else ldo
     d.o_stride_outer, d.o_stride_inner = o_strides
     d.out_row_sum, d.acc_debug = _ptr(out_row_sum), _ptr(acc_debug)
+    d.causal = int(causal)
     return d

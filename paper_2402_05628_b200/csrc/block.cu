@@ -154,6 +154,7 @@ static repq_status block_forward_impl(const repq_block_desc* dp, const repq_bloc
     g.w_stride_outer = g.a_stride_outer; g.w_stride_inner = head_bytes;
     g.s_w_scalar = p.s_k; g.z_w_scalar = p.z_k;
     g.alpha = 1.f / sqrtf(float(dh));
+    g.causal = d.causal;
     g.out_kind = REPQ_OUT_F32; g.out_groups = 1; g.out_scale[0] = 1.f;
     g.out = scores; g.ldo = L.ld_s;
     g.o_stride_outer = int64_t(H) * S * L.ld_s; g.o_stride_inner = int64_t(S) * L.ld_s;

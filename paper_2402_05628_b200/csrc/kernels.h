@@ -16,6 +16,10 @@ repq_status launch_expand4(const uint8_t* src, int64_t rows, int64_t n, int64_t 
 // Warp-MMA integer GEMM (any shape, batched).
 repq_status qgemm_mma(const repq_gemm_desc& d, const EpilogueParams& ep, cudaStream_t st);
 
+// Attention-score kernel: batched code-by-code products with scalar quantizers, K <= 128, float32 output.
+bool scores_supported(const repq_gemm_desc& d);
+repq_status launch_scores(const repq_gemm_desc& d, cudaStream_t st);
+
 // Tensor-memory (tcgen05) integer GEMM: plain (unbatched) products with TMA-compatible operands.
 bool qgemm_tc_supported(const repq_gemm_desc& d);
 size_t qgemm_tc_workspace(const repq_gemm_desc& d);

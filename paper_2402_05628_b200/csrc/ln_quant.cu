@@ -2,10 +2,15 @@
 // Eq. 12, then Eq. 4 with the scalar (s~, z~)).
 //
 // HBM-bound: every input element is read once with 128-bit loads and leaves as a 4-bit (or 8-bit)
-// code.  A row is owned by a group of TPR threads; each thread keeps its slice of the row in
-// registers, so mean and centred variance are two register passes with shuffle reductions.  The
-// per-channel factors gamma~/s~ and beta~/s~ are loaded once per thread and reused for every row the
-// thread processes (persistent grid-stride loop over rows).
+// code.  A row is owned by a group of TPR threads which keeps its slice of the row in registers, so mean
+// and centred variance are two register passes with shuffle reductions.  Each group works on kRows rows
+// at a time (all their loads are issued before the first reduction) to keep enough bytes in flight.
+// The per-channel factors gamma~/s~ and beta~/s~ are staged once per CTA in shared memory.
+//
+// Rounding: round_half_even(clamp(t, -z, qmax - z)) is taken with one float add of 1.5 * 2^23 (the float
+// adder rounds to nearest-even at integer granularity there, with the tie decided by the parity of the
+// rounded t itself, as Eq. 4 has it); the integer then sits in the low mantissa bits and z is added while
+// the codes are packed.
 #include <cuda_bf16.h>
 
 #include "common.h"
@@ -15,6 +20,8 @@ namespace {
 
 constexpr int kChunk = 8;   // elements per 128-bit bf16 load
 constexpr int kVPT = 4;     // chunks per thread (upper bound)
+constexpr int kRows = 2;    // rows in flight per thread group
+constexpr uint32_t kMagicBits = 0x4B400000u;   // 1.5 * 2^23
 
 __device__ __forceinline__ void load_chunk(const float* p, float (&v)[kChunk]) {
   const float4 a = __ldcs(reinterpret_cast<const float4*>(p));
@@ -33,19 +40,27 @@ __device__ __forceinline__ void load_chunk(const __nv_bfloat16* p, float (&v)[kC
   }
 }
 
+// Sum over the TPR threads of a group, for kRows values at once.
 template <int TPR, typename V>
-__device__ __forceinline__ V group_reduce(V v, V* red, int group_first_warp) {
+__device__ __forceinline__ void group_reduce(V (&v)[kRows], V* red, int group_first_warp) {
   constexpr int kShfl = TPR < 32 ? TPR : 32;
 #pragma unroll
-  for (int o = kShfl / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  if constexpr (TPR > 32) {
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
-    __syncthreads();
-    v = V(0);
+  for (int o = kShfl / 2; o > 0; o >>= 1)
 #pragma unroll
-    for (int w = 0; w < TPR / 32; ++w) v += red[group_first_warp + w];
+    for (int r = 0; r < kRows; ++r) v[r] += __shfl_xor_sync(0xffffffffu, v[r], o);
+  if constexpr (TPR > 32) {
+    if ((threadIdx.x & 31) == 0)
+#pragma unroll
+      for (int r = 0; r < kRows; ++r) red[(threadIdx.x >> 5) * kRows + r] = v[r];
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < kRows; ++r) {
+      V acc = V(0);
+#pragma unroll
+      for (int w = 0; w < TPR / 32; ++w) acc += red[(group_first_warp + w) * kRows + r];
+      v[r] = acc;
+    }
   }
-  return v;
 }
 
 template <typename T, int TPR, bool kPack4>
@@ -55,104 +70,148 @@ ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
                 float inv_s, int z, int qmax, uint8_t* __restrict__ codes, int64_t ldc,
                 int32_t* __restrict__ row_sum) {
   constexpr int kBlock = TPR > 256 ? TPR : 256;
-  constexpr int kRowsPerBlock = kBlock / TPR;
-  // one array per reduction of a row: a thread can only overwrite an array after every thread of the
-  // block has passed the barrier of a later reduction, hence has finished reading it
-  __shared__ float red_a[kBlock / 32];
-  __shared__ float red_b[kBlock / 32];
-  __shared__ int red_c[kBlock / 32];
+  constexpr int kGroups = kBlock / TPR;
+  constexpr int kRowsPerBlock = kGroups * kRows;
+  extern __shared__ __align__(16) float s_gb[];          // g[D] then b[D]: gamma~/s~ and beta~/s~
+  // one array per reduction of a row: it can only be overwritten after every thread of the block has
+  // passed the barrier of a later reduction, hence has finished reading it
+  __shared__ float red_a[kBlock / 32 * kRows];
+  __shared__ float red_b[kBlock / 32 * kRows];
+  __shared__ int red_c[kBlock / 32 * kRows];
+
+  float* s_g = s_gb;
+  float* s_b = s_gb + D;
+  for (int i = threadIdx.x; i < D; i += kBlock) {
+    s_g[i] = __ldg(gamma_t + i) * inv_s;
+    s_b[i] = __ldg(beta_t + i) * inv_s;
+  }
+  __syncthreads();
 
   const int tig = threadIdx.x % TPR;             // thread in group
   const int group = threadIdx.x / TPR;
   const int group_first_warp = (group * TPR) >> 5;
   const int nchunks = D / kChunk;
-
-  // per-channel factors, pre-divided by the layer-wise scale: t = xhat * g + b = y / s~
-  float g[kVPT][kChunk], b[kVPT][kChunk];
-#pragma unroll
-  for (int i = 0; i < kVPT; ++i) {
-    const int c = tig + i * TPR;
-    if (c < nchunks) {
-#pragma unroll
-      for (int e = 0; e < kChunk; ++e) {
-        g[i][e] = __ldg(gamma_t + c * kChunk + e) * inv_s;
-        b[i][e] = __ldg(beta_t + c * kChunk + e) * inv_s;
-      }
-    }
-  }
   const float t_lo = float(-z), t_hi = float(qmax - z);
+  const float magic = __uint_as_float(kMagicBits);
   const float inv_d = 1.f / float(D);
 
   for (int64_t base = int64_t(blockIdx.x) * kRowsPerBlock; base < rows;
        base += int64_t(gridDim.x) * kRowsPerBlock) {
-    const int64_t row = base + group;
-    const bool live = row < rows;
-    const T* xr = x + (live ? row : 0) * ldx;
+    const int64_t row0 = base + group * kRows;
 
-    float v[kVPT][kChunk];
-    float sum = 0.f;
+    float v[kRows][kVPT][kChunk];
+    float sum[kRows];
 #pragma unroll
-    for (int i = 0; i < kVPT; ++i) {
-      const int c = tig + i * TPR;
-      if (c < nchunks && live) {
-        load_chunk(xr + c * kChunk, v[i]);
+    for (int r = 0; r < kRows; ++r) {
+      const bool live = row0 + r < rows;
+      const T* xr = x + (live ? row0 + r : 0) * ldx;
+      sum[r] = 0.f;
 #pragma unroll
-        for (int e = 0; e < kChunk; ++e) sum += v[i][e];
-      } else {
+      for (int i = 0; i < kVPT; ++i) {
+        const int c = tig + i * TPR;
+        if (c < nchunks && live) {
+          load_chunk(xr + c * kChunk, v[r][i]);
+        } else {
 #pragma unroll
-        for (int e = 0; e < kChunk; ++e) v[i][e] = 0.f;
+          for (int e = 0; e < kChunk; ++e) v[r][i][e] = 0.f;
+        }
       }
     }
-    float mu = 0.f;
-    if (!rms) mu = group_reduce<TPR, float>(sum, red_a, group_first_warp) * inv_d;
+#pragma unroll
+    for (int r = 0; r < kRows; ++r)
+#pragma unroll
+      for (int i = 0; i < kVPT; ++i)
+#pragma unroll
+        for (int e = 0; e < kChunk; ++e) sum[r] += v[r][i][e];
 
-    float ss = 0.f;
+    float mu[kRows];
+    if (!rms) {
+      group_reduce<TPR, float>(sum, red_a, group_first_warp);
+#pragma unroll
+      for (int r = 0; r < kRows; ++r) mu[r] = sum[r] * inv_d;
+    } else {
+#pragma unroll
+      for (int r = 0; r < kRows; ++r) mu[r] = 0.f;
+    }
+
+    float ss[kRows];
+#pragma unroll
+    for (int r = 0; r < kRows; ++r) {
+      ss[r] = 0.f;
+#pragma unroll
+      for (int i = 0; i < kVPT; ++i) {
+        if (tig + i * TPR < nchunks) {
+#pragma unroll
+          for (int e = 0; e < kChunk; ++e) {
+            v[r][i][e] -= mu[r];
+            ss[r] = fmaf(v[r][i][e], v[r][i][e], ss[r]);
+          }
+        }
+      }
+    }
+    group_reduce<TPR, float>(ss, red_b, group_first_warp);
+    float rstd[kRows];
+#pragma unroll
+    for (int r = 0; r < kRows; ++r) rstd[r] = rsqrtf(ss[r] * inv_d + eps);
+
+    int csum[kRows];
+#pragma unroll
+    for (int r = 0; r < kRows; ++r) csum[r] = 0;
 #pragma unroll
     for (int i = 0; i < kVPT; ++i) {
       const int c = tig + i * TPR;
       if (c < nchunks) {
-#pragma unroll
-        for (int e = 0; e < kChunk; ++e) {
-          v[i][e] -= mu;
-          ss = fmaf(v[i][e], v[i][e], ss);
+        float g[kChunk], b[kChunk];
+        {
+          const float4 g0 = *reinterpret_cast<const float4*>(s_g + c * kChunk);
+          const float4 g1 = *reinterpret_cast<const float4*>(s_g + c * kChunk + 4);
+          const float4 b0 = *reinterpret_cast<const float4*>(s_b + c * kChunk);
+          const float4 b1 = *reinterpret_cast<const float4*>(s_b + c * kChunk + 4);
+          g[0] = g0.x; g[1] = g0.y; g[2] = g0.z; g[3] = g0.w; g[4] = g1.x; g[5] = g1.y; g[6] = g1.z; g[7] = g1.w;
+          b[0] = b0.x; b[1] = b0.y; b[2] = b0.z; b[3] = b0.w; b[4] = b1.x; b[5] = b1.y; b[6] = b1.z; b[7] = b1.w;
         }
-      }
-    }
-    const float var = group_reduce<TPR, float>(ss, red_b, group_first_warp) * inv_d;
-    const float rstd = rsqrtf(var + eps);
-
-    int csum = 0;
 #pragma unroll
-    for (int i = 0; i < kVPT; ++i) {
-      const int c = tig + i * TPR;
-      if (c < nchunks) {
-        int q[kChunk];
+        for (int r = 0; r < kRows; ++r) {
+          uint32_t u[kChunk];
 #pragma unroll
-        for (int e = 0; e < kChunk; ++e) {
-          float t = fmaf(v[i][e] * rstd, g[i][e], b[i][e]);
-          t = fminf(fmaxf(t, t_lo), t_hi);        // clip(round(t) + z, 0, qmax) == round(clamp(t)) + z
-          q[e] = __float2int_rn(t) + z;
-          csum += q[e];
-        }
-        if (live) {
-          uint8_t* out = codes + row * ldc;
-          if constexpr (kPack4) {
-            uint32_t w = 0;
+          for (int e = 0; e < kChunk; ++e) {
+            float t = fmaf(v[r][i][e] * rstd[r], g[e], b[e]);
+            t = fminf(fmaxf(t, t_lo), t_hi);       // clip(round(t) + z, 0, qmax) == round(clamp(t)) + z
+            u[e] = __float_as_uint(t + magic);     // = magic_bits + round_half_even(t), as integers
+          }
+          if (row0 + r < rows) {
+            uint8_t* out = codes + (row0 + r) * ldc;
+            if constexpr (kPack4) {
+              // sum_e (magic_bits + round(t_e)) << 4e  -  sum_e (magic_bits - z) << 4e  =  sum_e code_e << 4e
+              uint32_t w = 0;
 #pragma unroll
-            for (int e = 0; e < kChunk; ++e) w |= uint32_t(q[e]) << (4 * e);
-            reinterpret_cast<uint32_t*>(out)[c] = w;
-          } else {
-            uint2 w;
-            w.x = uint32_t(q[0]) | uint32_t(q[1]) << 8 | uint32_t(q[2]) << 16 | uint32_t(q[3]) << 24;
-            w.y = uint32_t(q[4]) | uint32_t(q[5]) << 8 | uint32_t(q[6]) << 16 | uint32_t(q[7]) << 24;
-            reinterpret_cast<uint2*>(out)[c] = w;
+              for (int e = 0; e < kChunk; ++e) w += u[e] << (4 * e);
+              uint32_t k = 0;
+#pragma unroll
+              for (int e = 0; e < kChunk; ++e) k += (kMagicBits - uint32_t(z)) << (4 * e);
+              w -= k;
+              reinterpret_cast<uint32_t*>(out)[c] = w;
+              csum[r] += __dp4a(w & 0x0F0F0F0Fu, 0x01010101u, 0u) + __dp4a((w >> 4) & 0x0F0F0F0Fu, 0x01010101u, 0u);
+            } else {
+              uint2 w;
+              // low bytes hold round(t_e) mod 256; a per-byte add of z gives the codes (all in [0, 255])
+              const uint32_t z4 = (uint32_t(z) & 0xFFu) * 0x01010101u;
+              w.x = __vadd4(__byte_perm(__byte_perm(u[0], u[1], 0x0040), __byte_perm(u[2], u[3], 0x0040), 0x5410), z4);
+              w.y = __vadd4(__byte_perm(__byte_perm(u[4], u[5], 0x0040), __byte_perm(u[6], u[7], 0x0040), 0x5410), z4);
+              reinterpret_cast<uint2*>(out)[c] = w;
+              csum[r] += __dp4a(w.x, 0x01010101u, 0u) + __dp4a(w.y, 0x01010101u, 0u);
+            }
           }
         }
       }
     }
     if (row_sum != nullptr) {
-      csum = group_reduce<TPR, int>(csum, red_c, group_first_warp);
-      if (live && tig == 0) row_sum[row] = csum;
+      group_reduce<TPR, int>(csum, red_c, group_first_warp);
+      if (tig == 0) {
+#pragma unroll
+        for (int r = 0; r < kRows; ++r)
+          if (row0 + r < rows) row_sum[row0 + r] = csum[r];
+      }
     }
   }
 }
@@ -162,16 +221,16 @@ repq_status launch(const T* x, int64_t rows, int D, int64_t ldx, const float* g,
                    int rms, float s_t, int z, int bits, uint8_t* codes, int64_t ldc, int32_t* row_sum,
                    cudaStream_t st) {
   constexpr int kBlock = TPR > 256 ? TPR : 256;
-  constexpr int kRowsPerBlock = kBlock / TPR;
+  constexpr int kRowsPerBlock = kBlock / TPR * kRows;
   const int64_t need = (rows + kRowsPerBlock - 1) / kRowsPerBlock;
   const int64_t cap = int64_t(sm_count()) * 8;
   const int grid = int(need < cap ? need : cap);
   const float inv_s = 1.f / s_t;
   const int qmax = (1 << bits) - 1;
-  if (bits == 4)
-    ln_quant_kernel<T, TPR, true><<<grid, kBlock, 0, st>>>(x, rows, D, ldx, g, b, eps, rms, inv_s, z, qmax, codes, ldc, row_sum);
-  else
-    ln_quant_kernel<T, TPR, false><<<grid, kBlock, 0, st>>>(x, rows, D, ldx, g, b, eps, rms, inv_s, z, qmax, codes, ldc, row_sum);
+  const size_t smem = size_t(D) * 2 * sizeof(float);
+  auto kern = bits == 4 ? ln_quant_kernel<T, TPR, true> : ln_quant_kernel<T, TPR, false>;
+  if (smem > 48 * 1024) REPQ_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+  kern<<<grid, kBlock, smem, st>>>(x, rows, D, ldx, g, b, eps, rms, inv_s, z, qmax, codes, ldc, row_sum);
   REPQ_CUDA(cudaGetLastError());
   note_launch();
   return REPQ_OK;

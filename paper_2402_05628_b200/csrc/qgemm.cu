@@ -168,7 +168,7 @@ using namespace repq;
 extern "C" repq_status repq_qgemm_workspace_bytes(const repq_gemm_desc* d, size_t* bytes) {
   REPQ_REQUIRE(d && bytes, REPQ_INVALID_ARG, "qgemm_workspace_bytes: NULL argument");
   REPQ_TRY(validate(*d));
-  *bytes = (d->M > 0 && qgemm_tc_supported(*d)) ? qgemm_tc_workspace(*d) : 0;
+  *bytes = (d->M > 0 && !scores_supported(*d) && qgemm_tc_supported(*d)) ? qgemm_tc_workspace(*d) : 0;
   return REPQ_OK;
 }
 
@@ -177,6 +177,7 @@ extern "C" repq_status repq_qgemm(const repq_gemm_desc* d, void* workspace, size
   REPQ_TRY(validate(*d));
   if (d->M == 0) return REPQ_OK;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (scores_supported(*d)) return launch_scores(*d, st);
   const EpilogueParams ep = make_epilogue(*d);
   if (qgemm_tc_supported(*d)) {
     const size_t need = qgemm_tc_workspace(*d);

@@ -388,3 +388,46 @@ def check_block(name, batch, sample_items=None, out_dtype="f32", **overrides):
         assert rel < 6e-3, rel
         return rel, mx
     return assert_float_close(got, ref, "block %s" % name)
+
+
+def check_scores(B_, H, Lq, Lk, dh, bits, causal=False, seed=0):
+    """Batched code-by-code product (attention scores) against the oracle: de-quantized Q times de-quantized
+    K^T over the head dimension, scaled by 1/sqrt(d_h)."""
+    import torch
+    from oracle import repq_oracle as orc
+    from paper_2402_05628_b200 import binding as B
+
+    rng = np.random.default_rng(seed)
+    D = H * dh
+    Qc = rng.integers(0, 1 << bits, size=(B_ * Lq, D))
+    Kc = rng.integers(0, 1 << bits, size=(B_ * Lk, D))
+    s_q, s_k = 0.37, 0.21
+    z_q, z_k = int(rng.integers(0, 1 << bits)), int(rng.integers(0, 1 << bits))
+    Qh, Kh = orc.dequant_uniform(Qc, s_q, z_q), orc.dequant_uniform(Kc, s_k, z_k)
+    dev = torch.device("cuda:0")
+    ld = B.code_row_bytes(D, bits)
+    q_t = torch.from_numpy(pack_codes(Qc, bits, ld)).to(dev)
+    k_t = torch.from_numpy(pack_codes(Kc, bits, ld)).to(dev)
+    ld_s = (Lk + 3) // 4 * 4
+    out = torch.full((B_ * H * Lq, ld_s), float("nan"), dtype=torch.float32, device=dev)
+    hb = dh // 2 if bits == 4 else dh
+    d = B.gemm_desc(Lq, Lk, dh, q_t, bits, s_q, z_q, k_t, bits, out, s_w_scalar=s_k, z_w_scalar=z_k,
+                    alpha=1.0 / math.sqrt(dh), batch=(B_, H), a_strides=(Lq * ld, hb), w_strides=(Lk * ld, hb),
+                    o_strides=(H * Lq * ld_s, Lq * ld_s), causal=causal)
+    assert B.repq_qgemm_workspace_bytes(d) == 0
+    B.repq_qgemm(d, None)
+    torch.cuda.synchronize()
+    got = out.cpu().numpy()
+    worst = 0.0
+    for b in range(B_):
+        for h in range(H):
+            ref = Qh[b * Lq:(b + 1) * Lq, h * dh:(h + 1) * dh] @ Kh[b * Lk:(b + 1) * Lk, h * dh:(h + 1) * dh].T / math.sqrt(dh)
+            g = got[(b * H + h) * Lq:(b * H + h + 1) * Lq, :Lk]
+            if causal:
+                mask = np.arange(Lk)[None, :] <= (np.arange(Lq)[:, None] + Lk - Lq)
+                g, ref = np.where(mask, g, 0.0), np.where(mask, ref, 0.0)
+            assert np.all(np.isfinite(g))
+            rel, _ = assert_float_close(g, ref, "scores")
+            worst = max(worst, rel)
+    assert worst < 1e-5
+    return worst

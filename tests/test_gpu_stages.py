@@ -79,3 +79,12 @@ def test_pv_epilogues():
     parity.check_pv(2, 2, 197, 197, 64, 4, 4, out_kind="bf16", seed=1)
     parity.check_pv(2, 2, 197, 197, 64, 4, 4, out_kind="codes", out_bits=4, want_out_sum=True, seed=2)
     parity.check_pv(1, 2, 130, 130, 128, 8, 4, causal=True, out_kind="codes", out_bits=8, want_out_sum=True, seed=3, s_p=0.7)
+
+
+@pytest.mark.parametrize("Bn,H,Lq,Lk,dh,bits,causal", [
+    (2, 3, 197, 197, 64, 4, False), (1, 2, 577, 577, 64, 4, False), (1, 2, 300, 300, 128, 4, True),
+    (2, 2, 70, 70, 32, 8, False), (1, 1, 1, 130, 16, 6, False), (1, 2, 100, 260, 48, 4, True),
+    (1, 2, 50, 50, 24, 4, False),      # head size not a multiple of 16: generic warp-MMA kernel
+])
+def test_scores_match_oracle(Bn, H, Lq, Lk, dh, bits, causal):
+    parity.check_scores(Bn, H, Lq, Lk, dh, bits, causal, seed=Lq + dh)
