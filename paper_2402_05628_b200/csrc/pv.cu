@@ -1,13 +1,19 @@
 // P.V with log2-domain Softmax codes (Eqs. 16-17): A^ = s 2^(-ceil(p/2)) (sqrt2 if p odd else 1).
 //
-// Codes are expanded in registers to exact bf16 powers of two and fed to warp-level bf16 MMA with fp32
-// accumulation.  Even and odd codes go to two separate accumulators, so both MMA operands are exact
-// (powers of two; small integers v - z_v) and the irrational factor sqrt2 of Eq. 17 is applied once, in
-// float32, to the odd accumulator:  O = s s_v (acc_even + sqrt2 acc_odd).
+// Codes are turned into exact bf16 powers of two and fed to warp-level bf16 MMA with fp32 accumulation.
+// Even and odd codes go to two separate accumulators, so both MMA operands are exact (powers of two; small
+// integers v - z_v) and the irrational factor sqrt2 of Eq. 17 is applied once, in float32, to the odd
+// accumulator:  O = s s_v (acc_even + sqrt2 acc_odd).
 //
-// Key order inside a 64-key chunk is permuted so that every thread owns 16 consecutive codes of its two
-// query rows (one 64-bit or 128-bit load); the V fragments are fetched with ldmatrix.trans using the
-// same permutation of row addresses.
+// The code -> operand map is a 256-entry table in shared memory built once per CTA: for 4-bit codes it is
+// indexed by a whole byte (two codes) and returns the packed bf16 pair for the even and for the odd
+// accumulator; for 6/8-bit codes it is indexed by one code.  A CTA of 8 warps owns 128 query rows (64 when
+// the head is wider than 64) of one (batch, head) pair.  V is staged in shared memory as bf16 (v - z_v), up
+// to 256 keys at a time; the codes of the next 64 keys are fetched into registers while the current 64 are
+// multiplied.  Key order inside a 64-key chunk is permuted so that every thread owns 16 consecutive codes of
+// its two query rows (one 64-bit or 128-bit load); the V fragments are fetched with ldmatrix.trans using the
+// same permutation of row addresses.  Keys beyond Lk need no masking (their V rows are zero); under a
+// causal mask only the chunks that touch the diagonal are masked element by element.
 #include <cuda_bf16.h>
 
 #include "kernels.h"
@@ -15,8 +21,9 @@
 namespace repq {
 namespace {
 
-constexpr int kQRows = 64;     // query rows per CTA (4 warps x 16)
-constexpr int kKeys = 64;      // keys per chunk
+constexpr int kKeys = 64;       // keys per MMA chunk
+constexpr int kVKeys = 256;     // keys of V resident in shared memory
+constexpr int kThreads = 256;
 
 struct PvParams {
   const uint8_t* p; int bits_p; int64_t ldp, p_pair;
@@ -49,25 +56,41 @@ __device__ __forceinline__ uint32_t pow2_bits(uint32_t c) {
   return e <= 126u ? (127u - e) << 7 : 0u;
 }
 
-// Two codes -> packed bf16x2 operands for the even and the odd accumulator.
-__device__ __forceinline__ void expand2(uint32_t c0, uint32_t c1, bool ok0, bool ok1, uint32_t& even, uint32_t& odd) {
-  const uint32_t b0 = ok0 ? pow2_bits(c0) : 0u;
-  const uint32_t b1 = ok1 ? pow2_bits(c1) : 0u;
-  even = ((c0 & 1u) ? 0u : b0) | (((c1 & 1u) ? 0u : b1) << 16);
-  odd = ((c0 & 1u) ? b0 : 0u) | (((c1 & 1u) ? b1 : 0u) << 16);
+// Operands of two consecutive codes: .x = bf16 pair for the even accumulator, .y = for the odd one.
+template <bool kP4>
+__device__ __forceinline__ uint2 lookup_pair(const uint2* lut4, const uint32_t* lut8, uint32_t codes) {
+  if (kP4) return lut4[codes & 0xFFu];
+  const uint32_t l0 = lut8[codes & 0xFFu], l1 = lut8[(codes >> 8) & 0xFFu];
+  return make_uint2(__byte_perm(l0, l1, 0x5410), __byte_perm(l0, l1, 0x7632));
 }
 
-// NG = number of 64-wide column groups of V handled by the CTA (d_h <= 64 * NG); 4 warps per group.
+// NG = number of 64-wide column groups of V handled by the CTA (d_h <= 64 * NG); 8 / NG warps per group.
 template <int NG, bool kP4>
-__global__ void __launch_bounds__(128 * NG)
+__global__ void __launch_bounds__(kThreads)
 pv_kernel(PvParams P) {
   constexpr int kDhp = 64 * NG;
   constexpr int kVStride = kDhp + 8;                     // bf16 elements; conflict-free ldmatrix rows
-  __shared__ __align__(16) __nv_bfloat16 sV[kKeys * kVStride];
+  constexpr int kRowWarps = 8 / NG;
+  constexpr int kQRows = 16 * kRowWarps;
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  __nv_bfloat16* sV = reinterpret_cast<__nv_bfloat16*>(smem_raw);     // [kVKeys][kVStride]
+  __shared__ uint2 lut4[256];
+  uint32_t* lut8 = reinterpret_cast<uint32_t*>(lut4);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int rw = warp & 3;                                // row group of the warp
-  const int cg = warp >> 2;                               // column group of the warp
+  {
+    const uint32_t i = uint32_t(tid);
+    if (kP4) {
+      const uint32_t c0 = i & 15u, c1 = i >> 4, b0 = pow2_bits(c0), b1 = pow2_bits(c1);
+      lut4[i] = make_uint2(((c0 & 1u) ? 0u : b0) | (((c1 & 1u) ? 0u : b1) << 16),
+                           ((c0 & 1u) ? b0 : 0u) | (((c1 & 1u) ? b1 : 0u) << 16));
+    } else {
+      const uint32_t b = pow2_bits(i);
+      lut8[i] = (i & 1u) ? (b << 16) : b;
+    }
+  }
+  const int rw = warp % kRowWarps;                        // row group of the warp
+  const int cg = warp / kRowWarps;                        // column group of the warp
   const int g = lane >> 2, t = lane & 3;
   const int pair = blockIdx.y;
   const int bo = pair / P.batch_inner, bi = pair % P.batch_inner;
@@ -77,10 +100,10 @@ pv_kernel(PvParams P) {
 
   const int row_a = q0 + rw * 16 + g, row_b = row_a + 8;
   const int shift = P.Lk - P.Lq;
-  int valid_a = row_a < P.Lq ? (P.causal ? min(P.Lk, row_a + 1 + shift) : P.Lk) : 0;
-  int valid_b = row_b < P.Lq ? (P.causal ? min(P.Lk, row_b + 1 + shift) : P.Lk) : 0;
-  valid_a = max(valid_a, 0);
-  valid_b = max(valid_b, 0);
+  // keys a row may attend to; rows beyond Lq produce values that are never stored
+  const int valid_a = P.causal ? max(0, min(P.Lk, row_a + 1 + shift)) : P.Lk;
+  const int valid_b = P.causal ? max(0, min(P.Lk, row_b + 1 + shift)) : P.Lk;
+  const int warp_min_valid = P.causal ? max(0, min(P.Lk, q0 + rw * 16 + 1 + shift)) : P.Lk;
   int k_end = P.Lk;
   if (P.causal) k_end = max(0, min(P.Lk, min(q0 + kQRows, P.Lq) + shift));
 
@@ -94,36 +117,43 @@ pv_kernel(PvParams P) {
   const uint8_t* pa = p_base + int64_t(row_a < P.Lq ? row_a : 0) * P.ldp + t * kCodeBytes;
   const uint8_t* pb = p_base + int64_t(row_b < P.Lq ? row_b : 0) * P.ldp + t * kCodeBytes;
 
-  for (int k0 = 0; k0 < k_end; k0 += kKeys) {
-    // ---- this thread's 16 codes of each of its two rows (keys k0 + 16 t .. + 15)
-    uint32_t ca[4] = {0, 0, 0, 0}, cb[4] = {0, 0, 0, 0};   // 8-bit: 4 codes per word; 4-bit: words 0,1 used
-    const int64_t boff = kP4 ? k0 / 2 : k0;                 // bytes from the row start to chunk k0
+  // this thread's 16 codes of each of its two rows for the chunk starting at key k0 (keys k0 + 16 t .. + 15)
+  auto load_codes = [&](int k0, uint32_t (&ca)[4], uint32_t (&cb)[4]) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) ca[i] = cb[i] = 0u;
+    if (k0 >= k_end) return;
+    const int64_t boff = kP4 ? k0 / 2 : k0;               // bytes from the row start to chunk k0
     if (boff + t * kCodeBytes + kCodeBytes <= P.ldp) {
       if (kP4) {
-        if (k0 + 16 * t < valid_a) { const uint2 w = *reinterpret_cast<const uint2*>(pa + boff); ca[0] = w.x; ca[1] = w.y; }
-        if (k0 + 16 * t < valid_b) { const uint2 w = *reinterpret_cast<const uint2*>(pb + boff); cb[0] = w.x; cb[1] = w.y; }
+        const uint2 wa = __ldcs(reinterpret_cast<const uint2*>(pa + boff)); ca[0] = wa.x; ca[1] = wa.y;
+        const uint2 wb = __ldcs(reinterpret_cast<const uint2*>(pb + boff)); cb[0] = wb.x; cb[1] = wb.y;
       } else {
-        if (k0 + 16 * t < valid_a) { const uint4 w = *reinterpret_cast<const uint4*>(pa + boff); ca[0] = w.x; ca[1] = w.y; ca[2] = w.z; ca[3] = w.w; }
-        if (k0 + 16 * t < valid_b) { const uint4 w = *reinterpret_cast<const uint4*>(pb + boff); cb[0] = w.x; cb[1] = w.y; cb[2] = w.z; cb[3] = w.w; }
+        const uint4 wa = __ldcs(reinterpret_cast<const uint4*>(pa + boff)); ca[0] = wa.x; ca[1] = wa.y; ca[2] = wa.z; ca[3] = wa.w;
+        const uint4 wb = __ldcs(reinterpret_cast<const uint4*>(pb + boff)); cb[0] = wb.x; cb[1] = wb.y; cb[2] = wb.z; cb[3] = wb.w;
       }
     } else {
       // ragged end of the row: byte loads inside the row stride
       for (int e = 0; e < kCodeBytes; ++e) {
-        const int64_t o = boff + t * kCodeBytes + e;
-        if (o < P.ldp) {
+        if (boff + t * kCodeBytes + e < P.ldp) {
           ca[e >> 2] |= uint32_t(pa[boff + e]) << (8 * (e & 3));
           cb[e >> 2] |= uint32_t(pb[boff + e]) << (8 * (e & 3));
         }
       }
     }
+  };
 
-    // ---- V chunk -> shared memory as bf16 (v - z_v), zero rows beyond Lk and columns beyond d_h
+  uint32_t ca[4], cb[4];
+  load_codes(0, ca, cb);
+
+  for (int kv0 = 0; kv0 < k_end; kv0 += kVKeys) {
+    // ---- up to 256 keys of V -> shared memory as bf16 (v - z_v); zero rows beyond Lk, zero columns beyond d_h
     __syncthreads();
     {
       constexpr int kGroupsPerRow = kDhp / 8;              // 8 columns per work item
-      for (int w = tid; w < kKeys * kGroupsPerRow; w += 128 * NG) {
+      const int keys_here = min(kVKeys, (k_end - kv0 + kKeys - 1) / kKeys * kKeys);
+      for (int w = tid; w < keys_here * kGroupsPerRow; w += kThreads) {
         const int kr = w / kGroupsPerRow, c0 = (w % kGroupsPerRow) * 8;
-        const int key = k0 + kr;
+        const int key = kv0 + kr;
         uint32_t o[4] = {0, 0, 0, 0};
         if (key < P.Lk && c0 < P.d_h) {
           const uint8_t* vr = v_base + int64_t(key) * P.ldv;
@@ -131,14 +161,14 @@ pv_kernel(PvParams P) {
           if (P.bits_v == 4) {
             uint32_t w4 = 0;
             const uint8_t* s = vr + c0 / 2;
-            if ((reinterpret_cast<uintptr_t>(s) & 3) == 0 && c0 + 8 <= P.d_h) w4 = *reinterpret_cast<const uint32_t*>(s);
+            if ((reinterpret_cast<uintptr_t>(s) & 3) == 0 && c0 + 8 <= P.d_h) w4 = __ldg(reinterpret_cast<const uint32_t*>(s));
             else for (int e = 0; e < 4; ++e) if (c0 + 2 * e < P.d_h) w4 |= uint32_t(s[e]) << (8 * e);
 #pragma unroll
             for (int e = 0; e < 8; ++e) q[e] = int((w4 >> (4 * e)) & 15u);
           } else {
             const uint8_t* s = vr + c0;
             uint2 w8 = make_uint2(0, 0);
-            if ((reinterpret_cast<uintptr_t>(s) & 7) == 0 && c0 + 8 <= P.d_h) w8 = *reinterpret_cast<const uint2*>(s);
+            if ((reinterpret_cast<uintptr_t>(s) & 7) == 0 && c0 + 8 <= P.d_h) w8 = __ldg(reinterpret_cast<const uint2*>(s));
             else for (int e = 0; e < 8; ++e) if (c0 + e < P.d_h) (e < 4 ? w8.x : w8.y) |= uint32_t(s[e]) << (8 * (e & 3));
 #pragma unroll
             for (int e = 0; e < 4; ++e) { q[e] = int((w8.x >> (8 * e)) & 255u); q[4 + e] = int((w8.y >> (8 * e)) & 255u); }
@@ -156,38 +186,54 @@ pv_kernel(PvParams P) {
     }
     __syncthreads();
 
-    // ---- 4 MMA k-steps of 16 keys; step s uses codes 4s..4s+3 of every thread
+    const int kv_end = min(k_end, kv0 + kVKeys);
+    for (int k0 = kv0; k0 < kv_end; k0 += kKeys) {
+      uint32_t na[4], nb[4];
+      load_codes(k0 + kKeys, na, nb);                       // next chunk's codes, in flight during the MMAs
+      const bool need_mask = k0 + kKeys > warp_min_valid;   // warp-uniform: this chunk touches the causal diagonal
+      // ---- 4 MMA k-steps of 16 keys; step s uses codes 4s..4s+3 of every thread
 #pragma unroll
-    for (int s = 0; s < 4; ++s) {
-      uint32_t c[2][4];
-      if (kP4) {
-        const uint32_t ha = (ca[s >> 1] >> (16 * (s & 1))) & 0xffffu, hb = (cb[s >> 1] >> (16 * (s & 1))) & 0xffffu;
+      for (int s = 0; s < 4; ++s) {
+        // the 4 codes of this step, per row: 16 bits (4-bit codes) or 32 bits (byte codes)
+        uint32_t qa, qb;
+        if (kP4) {
+          qa = (ca[s >> 1] >> (16 * (s & 1))) & 0xffffu;
+          qb = (cb[s >> 1] >> (16 * (s & 1))) & 0xffffu;
+        } else {
+          qa = ca[s];
+          qb = cb[s];
+        }
+        constexpr int kPairShift = kP4 ? 8 : 16;            // bits per pair of codes
+        // fragment order: a0 = (row g, k 2t..), a1 = (row g+8, k 2t..), a2 = (row g, k 2t+8..), a3 = (row g+8, k 2t+8..)
+        const uint2 fa0 = lookup_pair<kP4>(lut4, lut8, qa), fa1 = lookup_pair<kP4>(lut4, lut8, qa >> kPairShift);
+        const uint2 fb0 = lookup_pair<kP4>(lut4, lut8, qb), fb1 = lookup_pair<kP4>(lut4, lut8, qb >> kPairShift);
+        uint32_t ae[4] = {fa0.x, fb0.x, fa1.x, fb1.x};
+        uint32_t ao[4] = {fa0.y, fb0.y, fa1.y, fb1.y};
+        if (need_mask) {
+          const int key0 = k0 + 16 * t + 4 * s;
+          const uint32_t ma0 = (key0 + 0 < valid_a ? 0xFFFFu : 0u) | (key0 + 1 < valid_a ? 0xFFFF0000u : 0u);
+          const uint32_t ma1 = (key0 + 2 < valid_a ? 0xFFFFu : 0u) | (key0 + 3 < valid_a ? 0xFFFF0000u : 0u);
+          const uint32_t mb0 = (key0 + 0 < valid_b ? 0xFFFFu : 0u) | (key0 + 1 < valid_b ? 0xFFFF0000u : 0u);
+          const uint32_t mb1 = (key0 + 2 < valid_b ? 0xFFFFu : 0u) | (key0 + 3 < valid_b ? 0xFFFF0000u : 0u);
+          ae[0] &= ma0; ao[0] &= ma0; ae[1] &= mb0; ao[1] &= mb0;
+          ae[2] &= ma1; ao[2] &= ma1; ae[3] &= mb1; ao[3] &= mb1;
+        }
+        // V fragments: lane supplies the row address of matrix (lane / 8), row (lane % 8)
+        const int mi = lane >> 3, r = lane & 7;
+        const int klog = (mi & 1) * 8 + r;                                  // logical k of this address
+        const int kr = (k0 - kv0) + 16 * ((klog & 7) >> 1) + 4 * s + ((klog >> 3) << 1) + (klog & 1);
 #pragma unroll
-        for (int e = 0; e < 4; ++e) { c[0][e] = (ha >> (4 * e)) & 15u; c[1][e] = (hb >> (4 * e)) & 15u; }
-      } else {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) { c[0][e] = (ca[s] >> (8 * e)) & 255u; c[1][e] = (cb[s] >> (8 * e)) & 255u; }
+        for (int jp = 0; jp < 4; ++jp) {                                    // pairs of 8-column blocks
+          uint32_t b[4];
+          ldmatrix_x4_trans(b, &sV[kr * kVStride + cg * 64 + jp * 16 + (mi >> 1) * 8]);
+          mma_bf16(acc_e[2 * jp], ae, b[0], b[1]);
+          mma_bf16(acc_o[2 * jp], ao, b[0], b[1]);
+          mma_bf16(acc_e[2 * jp + 1], ae, b[2], b[3]);
+          mma_bf16(acc_o[2 * jp + 1], ao, b[2], b[3]);
+        }
       }
-      const int key0 = k0 + 16 * t + 4 * s;
-      uint32_t ae[4], ao[4];
-      // fragment order: a0 = (row g, k 2t..), a1 = (row g+8, k 2t..), a2 = (row g, k 2t+8..), a3 = (row g+8, k 2t+8..)
-      expand2(c[0][0], c[0][1], key0 + 0 < valid_a, key0 + 1 < valid_a, ae[0], ao[0]);
-      expand2(c[1][0], c[1][1], key0 + 0 < valid_b, key0 + 1 < valid_b, ae[1], ao[1]);
-      expand2(c[0][2], c[0][3], key0 + 2 < valid_a, key0 + 3 < valid_a, ae[2], ao[2]);
-      expand2(c[1][2], c[1][3], key0 + 2 < valid_b, key0 + 3 < valid_b, ae[3], ao[3]);
-      // V fragments: lane supplies the row address of matrix (lane / 8), row (lane % 8)
-      const int mi = lane >> 3, r = lane & 7;
-      const int klog = (mi & 1) * 8 + r;                                  // logical k of this address
-      const int kr = 16 * ((klog & 7) >> 1) + 4 * s + ((klog >> 3) << 1) + (klog & 1);
 #pragma unroll
-      for (int jp = 0; jp < 4; ++jp) {                                    // pairs of 8-column blocks
-        uint32_t b[4];
-        ldmatrix_x4_trans(b, &sV[kr * kVStride + cg * 64 + jp * 16 + (mi >> 1) * 8]);
-        mma_bf16(acc_e[2 * jp], ae, b[0], b[1]);
-        mma_bf16(acc_o[2 * jp], ao, b[0], b[1]);
-        mma_bf16(acc_e[2 * jp + 1], ae, b[2], b[3]);
-        mma_bf16(acc_o[2 * jp + 1], ao, b[2], b[3]);
-      }
+      for (int i = 0; i < 4; ++i) { ca[i] = na[i]; cb[i] = nb[i]; }
     }
   }
 
@@ -238,6 +284,19 @@ pv_kernel(PvParams P) {
   }
 }
 
+template <int NG, bool kP4>
+repq_status launch_pv(const PvParams& P, int64_t pairs, cudaStream_t st) {
+  constexpr int kQRows = 16 * (8 / NG);
+  constexpr size_t smem = size_t(kVKeys) * (64 * NG + 8) * sizeof(__nv_bfloat16);
+  if (smem + 2048 > 48 * 1024)
+    REPQ_CUDA(cudaFuncSetAttribute(pv_kernel<NG, kP4>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+  dim3 grid((P.Lq + kQRows - 1) / kQRows, unsigned(pairs));
+  pv_kernel<NG, kP4><<<grid, kThreads, smem, st>>>(P);
+  REPQ_CUDA(cudaGetLastError());
+  note_launch();
+  return REPQ_OK;
+}
+
 }  // namespace
 }  // namespace repq
 
@@ -276,14 +335,7 @@ extern "C" repq_status repq_pv(const repq_pv_desc* d, void* stream) {
   P.out = d->out; P.ldo = d->ldo; P.o_so = d->o_stride_outer; P.o_si = d->o_stride_inner;
   P.out_row_sum = d->out_kind == REPQ_OUT_CODES ? d->out_row_sum : nullptr;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  dim3 grid((d->Lq + kQRows - 1) / kQRows, unsigned(pairs));
   const bool p4 = d->bits_p == 4;
-  if (d->d_h <= 64) {
-    if (p4) pv_kernel<1, true><<<grid, 128, 0, st>>>(P); else pv_kernel<1, false><<<grid, 128, 0, st>>>(P);
-  } else {
-    if (p4) pv_kernel<2, true><<<grid, 256, 0, st>>>(P); else pv_kernel<2, false><<<grid, 256, 0, st>>>(P);
-  }
-  REPQ_CUDA(cudaGetLastError());
-  note_launch();
-  return REPQ_OK;
+  if (d->d_h <= 64) return p4 ? launch_pv<1, true>(P, pairs, st) : launch_pv<1, false>(P, pairs, st);
+  return p4 ? launch_pv<2, true>(P, pairs, st) : launch_pv<2, false>(P, pairs, st);
 }

@@ -4,15 +4,23 @@
 // and re-quantization of the quantized linear layer.
 //
 // One persistent CTA per SM; roles by warp:
-//   warp 0      TMA producer (one elected lane): A tile 128 x 128 B, W tile 256 x 128 B per stage, 128-byte
-//               swizzle, zero fill outside the matrices
-//   warp 1      tensor-memory allocation and MMA issue (one elected lane): 4 MMAs of K = 32 per stage,
-//               accumulators double-buffered in TMEM (2 x 256 columns) so the epilogue of tile i overlaps
-//               the main loop of tile i + 1
-//   warps 2..9  epilogue: warp w reads TMEM lanes 32 (w mod 4) .. +31 (one output row per thread) and one
-//               half of the 256 accumulator columns
-// 4-bit operands are expanded to one code per byte by a separate pass into the workspace (there is no
-// 4-bit integer MMA), so the main loop is the same for W4A4 and W8A8.
+//   warp 0       TMA producer (one elected lane): A tile 128 x 128 B, W tile BN x 128 B per stage, 128-byte
+//                swizzle, zero fill outside the matrices
+//   warp 1       tensor-memory allocation and MMA issue (one elected lane): 4 MMAs of K = 32 per stage,
+//                accumulators double-buffered in TMEM (2 x 256 columns) so the epilogue of tile i overlaps
+//                the main loop of tile i + 1
+//   warps 2..17  epilogue: warp w reads TMEM lanes 32 (w mod 4) .. +31 (one output row per thread) and a
+//                64-column slice of the accumulator columns
+// The tile width BN (256, 192 or 128) is chosen per problem so that the last round of tiles over the SMs is
+// as full as possible.  4-bit operands are expanded to one code per byte by a separate pass into the
+// workspace (there is no 4-bit integer MMA), so the main loop is the same for W4A4 and W8A8.
+//
+// For short K the epilogue, not the tensor pipe, sets the pace (K = 768: 3072 tensor-pipe cycles per
+// 128 x 256 tile against 32768 outputs), so it is written for few instructions per output: per-column terms
+// are staged once per tile in shared memory and read as vectors, the output quantizer is folded into them
+// where nothing sits between the GEMM and the re-quantization, rounding uses the float adder (add
+// 1.5 * 2^23), codes are packed by shift-adds with the zero-point folded into one constant, and the residual
+// of a tile is requested before the accumulator is waited for.
 //
 // Every wait on an mbarrier is bounded: when it runs out the kernel records a status code, all roles
 // leave their loops, in-flight copies and MMAs are drained, tensor memory is freed and the kernel returns.
@@ -20,35 +28,40 @@
 #include <cuda_bf16.h>
 
 #include <cstdlib>
-#include <mutex>
 
 #include "kernels.h"
 
 namespace repq {
 namespace {
 
-constexpr int BM = 128, BN = 256, BK = 128;        // BK in bytes (= codes)
+constexpr int BM = 128, BK = 128;                   // BK in bytes (= codes); BN is a template parameter
+constexpr int kMaxBN = 256;
+constexpr int kChunk = 16;                           // accumulator columns per tcgen05.ld / per store
 constexpr int kStages = 4;
-constexpr int kEpiWarps = 8;
+constexpr int kEpiWarps = 16;
+constexpr int kEpiThreads = kEpiWarps * 32;
 constexpr int kThreads = 32 * (2 + kEpiWarps);
 constexpr int kTmemCols = 512;
-constexpr uint32_t kABytes = BM * BK, kBBytes = BN * BK;
-constexpr long long kWaitCycles = 2000000000LL;     // about one second
+constexpr int kAccStride = 256;                      // TMEM columns between the two accumulator buffers
+constexpr int kSliceCols = 64;                       // accumulator columns per epilogue warp
+constexpr int kSliceChunks = kSliceCols / kChunk;
+constexpr uint32_t kABytes = BM * BK;
+constexpr long long kWaitCycles = 2000000000LL;      // about one second
+constexpr uint32_t kMagicBits = 0x4B400000u;         // 1.5 * 2^23
 
 __device__ int32_t g_status_word = 0;
 
-struct alignas(16) ColTerms {                         // per output column, staged once per tile
-  float scale[BN];
-  float bias[BN];
-  int32_t z_w[BN];
-  int32_t kzz[BN];
-  float inv_so[BN];
-  int32_t zo[BN];
+struct alignas(16) ColTerms {                          // per output column, staged once per tile
+  int32_t nzw[kMaxBN];  // -z_w[j]
+  int32_t kw[kMaxBN];   // -z_a * wsum[j]
+  float sc[kMaxBN];     // alpha s_a s_w[j]   (times 1/s_o in direct re-quantization mode)
+  float bi[kMaxBN];     // bias[j]            (times 1/s_o in direct re-quantization mode)
 };
 
+template <int BN>
 struct SharedStorage {
   alignas(1024) uint8_t a[kStages][kABytes];
-  alignas(1024) uint8_t b[kStages][kBBytes];
+  alignas(1024) uint8_t b[kStages][BN * BK];
   ColTerms cols[2];
   alignas(8) uint64_t full[kStages];
   uint64_t empty[kStages];
@@ -109,7 +122,7 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-// D[tmem] (+)= A[smem] * B[smem]^T, 128 x 256 x 32, u8 x u8 -> s32
+// D[tmem] (+)= A[smem] * B[smem]^T, 128 x BN x 32, u8 x u8 -> s32
 __device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
@@ -124,18 +137,17 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
          (uint64_t(2) << 61);
 }
 
-// Instruction descriptor: D = s32, A = B = unsigned 8-bit, both K-major, N = 256, M = 128.
-constexpr uint32_t kIdesc = (2u << 4) | (0u << 7) | (0u << 10) | (uint32_t(BN >> 3) << 17) | (uint32_t(BM >> 4) << 24);
+// Instruction descriptor: D = s32, A = B = unsigned 8-bit, both K-major, N = bn, M = 128.
+constexpr uint32_t idesc_for(int bn) {
+  return (2u << 4) | (0u << 7) | (0u << 10) | (uint32_t(bn >> 3) << 17) | (uint32_t(BM >> 4) << 24);
+}
 
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
@@ -144,13 +156,112 @@ struct TcParams {
   int M, N, K;
   const int32_t* asum;
   const int32_t* wsum;
+  int direct_requant;          // codes out, no GELU, no residual: 1/s_o is folded into the column terms
   EpilogueParams ep;
 };
 
+// One 16-column chunk of one output row: v[e] holds the float value before the output conversion.
+__device__ __forceinline__ void store_chunk(const EpilogueParams& ep, const TcParams& P, float (&v)[kChunk], int64_t m,
+                                            int col0, bool full_chunk, int& code_sum) {
+  if (ep.out_kind == REPQ_OUT_F32) {
+    float* o = static_cast<float*>(ep.out) + m * ep.ldo + col0;
+    if (full_chunk) {
+#pragma unroll
+      for (int q4 = 0; q4 < kChunk / 4; ++q4)
+        reinterpret_cast<float4*>(o)[q4] = make_float4(v[q4 * 4], v[q4 * 4 + 1], v[q4 * 4 + 2], v[q4 * 4 + 3]);
+    } else {
+      for (int e = 0; e < kChunk; ++e) if (col0 + e < P.N) o[e] = v[e];
+    }
+    return;
+  }
+  if (ep.out_kind == REPQ_OUT_BF16) {
+    __nv_bfloat16* o = static_cast<__nv_bfloat16*>(ep.out) + m * ep.ldo + col0;
+    if (full_chunk) {
+#pragma unroll
+      for (int q4 = 0; q4 < kChunk / 8; ++q4) {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const __nv_bfloat162 h = __floats2bfloat162_rn(v[q4 * 8 + 2 * i], v[q4 * 8 + 2 * i + 1]);
+          w[i] = *reinterpret_cast<const uint32_t*>(&h);
+        }
+        reinterpret_cast<uint4*>(o)[q4] = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+    } else {
+      for (int e = 0; e < kChunk; ++e) if (col0 + e < P.N) o[e] = __float2bfloat16_rn(v[e]);
+    }
+    return;
+  }
+  // codes: Eq. 4 with the output quantizer of this chunk's column group
+  const int group = col0 / ep.group_width;
+  const int zo = ep.out_zero[group];
+  const float lo = float(-zo), hi = float(ep.qmax - zo);
+  const float mult = P.direct_requant ? 1.f : ep.inv_out_scale[group];
+  const float magic = __uint_as_float(kMagicBits);
+  uint32_t u[kChunk];
+#pragma unroll
+  for (int e = 0; e < kChunk; ++e) {
+    float t = v[e] * mult;
+    t = fminf(fmaxf(t, lo), hi);
+    u[e] = __float_as_uint(t + magic);             // magic_bits + round_half_even(t)
+  }
+  uint8_t* orow = static_cast<uint8_t*>(ep.out) + m * ep.ldo;
+  if (ep.pack4) {
+    uint32_t k = 0;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) k += (kMagicBits - uint32_t(zo)) << (4 * e);
+    uint32_t w[2];
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      w[i] = 0;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) w[i] += u[i * 8 + e] << (4 * e);
+      w[i] -= k;
+    }
+    if (full_chunk) {
+      *reinterpret_cast<uint2*>(orow + (col0 >> 1)) = make_uint2(w[0], w[1]);
+#pragma unroll
+      for (int i = 0; i < 2; ++i)
+        code_sum += __dp4a(w[i] & 0x0F0F0F0Fu, 0x01010101u, 0u) + __dp4a((w[i] >> 4) & 0x0F0F0F0Fu, 0x01010101u, 0u);
+    } else {
+      for (int e = 0; e < kChunk; e += 2) {
+        if (col0 + e < P.N) {
+          const uint32_t byte = (w[e >> 3] >> (4 * (e & 7))) & (col0 + e + 1 < P.N ? 0xFFu : 0x0Fu);
+          orow[(col0 + e) >> 1] = uint8_t(byte);
+          code_sum += int(byte & 15u) + int(byte >> 4);
+        }
+      }
+    }
+  } else {
+    const uint32_t z4 = (uint32_t(zo) & 0xFFu) * 0x01010101u;
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      w[i] = __vadd4(__byte_perm(__byte_perm(u[4 * i], u[4 * i + 1], 0x0040), __byte_perm(u[4 * i + 2], u[4 * i + 3], 0x0040), 0x5410), z4);
+    if (full_chunk) {
+      *reinterpret_cast<uint4*>(orow + col0) = make_uint4(w[0], w[1], w[2], w[3]);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) code_sum += __dp4a(w[i], 0x01010101u, 0u);
+    } else {
+      for (int e = 0; e < kChunk; ++e) {
+        if (col0 + e < P.N) {
+          const uint32_t byte = (w[e >> 2] >> (8 * (e & 3))) & 0xFFu;
+          orow[col0 + e] = uint8_t(byte);
+          code_sum += int(byte);
+        }
+      }
+    }
+  }
+}
+
+template <int BN>
 __global__ void __launch_bounds__(kThreads, 1)
 qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, TcParams P) {
+  using Storage = SharedStorage<BN>;
+  constexpr uint32_t kBBytes = BN * BK;
+  constexpr uint32_t kIdesc = idesc_for(BN);
   extern __shared__ uint8_t smem_raw[];
-  SharedStorage& S = *reinterpret_cast<SharedStorage*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  Storage& S = *reinterpret_cast<Storage*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m_tiles = (P.M + BM - 1) / BM, n_tiles = (P.N + BN - 1) / BN;
@@ -160,7 +271,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&S.full[s]), 1); mbar_init(smem_u32(&S.empty[s]), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&S.tmem_full[a]), 1); mbar_init(smem_u32(&S.tmem_empty[a]), kEpiWarps); }
-    for (int a = 0; a < 2; ++a) mbar_init(smem_u32(&S.cols_ready[a]), kEpiWarps * 32);
+    for (int a = 0; a < 2; ++a) mbar_init(smem_u32(&S.cols_ready[a]), kEpiThreads);
     mbar_init(smem_u32(&S.done), 1);
     S.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -210,7 +321,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         const uint32_t acc = it & 1, acc_phase = (it >> 1) & 1;
         if (!mbar_wait(smem_u32(&S.tmem_empty[acc]), acc_phase ^ 1, abort, 2)) break;
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + acc * BN;
+        const uint32_t d_tmem = tmem_base + acc * kAccStride;
         bool ok = true;
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!mbar_wait(smem_u32(&S.full[stage]), phase, abort, 3)) { ok = false; break; }
@@ -232,160 +343,124 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     }
   } else {
     // ---------------------------------------------------------------- epilogue
-    const int ew = warp - 2;                     // 0..7
+    const int ew = warp - 2;                     // 0..15
     const int quarter = warp & 3;                // TMEM lane quarter this warp may read
-    const int half = ew >> 2;                    // which 128 accumulator columns
-    const int et = threadIdx.x - 64;             // 0..255 among epilogue threads
+    const int slice = ew >> 2;                   // which 64 accumulator columns
+    const bool slice_on = slice * kSliceCols < BN;
+    const int et = threadIdx.x - 64;             // 0..511 among epilogue threads
     const EpilogueParams& ep = P.ep;
+    const int kza = P.K * ep.z_a;
+    const bool res16 = ep.residual != nullptr && ep.residual_bf16;
     int it = 0;
     for (int tile = blockIdx.x; tile < tiles && !*abort; tile += gridDim.x, ++it) {
       const uint32_t acc = it & 1, acc_phase = (it >> 1) & 1;
       const int m0 = (tile % m_tiles) * BM, n0 = (tile / m_tiles) * BN;
-      // stage the per-column terms of this tile (one column per epilogue thread); the buffer was last
-      // read two tiles ago, before this thread's arrival on tmem_empty of that tile
+      const int64_t m = int64_t(m0) + quarter * 32 + lane;
+      const bool row_ok = m < P.M;
+      const int cl0 = slice * kSliceCols;                    // first column of this warp inside the tile
+      // whole 64-column slice inside the matrix: vector paths everywhere
+      const bool slice_full = slice_on && n0 + cl0 + kSliceCols <= P.N;
+      // bf16 residual of the slice and the row's code sum: requested now, needed only after the main loop
+      uint4 res[kSliceCols / 8];
+      if (res16 && row_ok && slice_full) {
+        const uint4* rp = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(ep.residual) + m * ep.ld_residual + n0 + cl0);
+#pragma unroll
+        for (int i = 0; i < kSliceCols / 8; ++i) res[i] = __ldg(rp + i);
+      }
+      // corr = acc - z_w (asum - K z_a) - z_a wsum
+      const int32_t asum_c = row_ok ? __ldg(P.asum + m) - kza : 0;
+      // stage the per-column terms of this tile (one column per thread, threads 0..BN-1); the buffer was last
+      // read two tiles ago, and every epilogue thread has passed the barrier of the tile in between
       {
         ColTerms& C = S.cols[acc];
-        const int j = n0 + et;
-        if (j < P.N) {
-          const ColumnTerms ct = column_terms(ep, j, __ldg(P.wsum + j));
-          C.scale[et] = ct.scale; C.bias[et] = ct.bias; C.z_w[et] = ct.z_w; C.kzz[et] = ct.kzz;
-          C.inv_so[et] = ct.inv_so; C.zo[et] = ct.zo;
-        } else {
-          C.scale[et] = 0.f; C.bias[et] = 0.f; C.z_w[et] = 0; C.kzz[et] = 0; C.inv_so[et] = 1.f; C.zo[et] = 0;
+        if (et < BN) {
+          const int j = n0 + et;
+          int nzw = 0, kw = 0;
+          float sc = 0.f, bi = 0.f;
+          if (j < P.N) {
+            const int zw = ep.z_w ? __ldg(ep.z_w + j) : ep.z_w_scalar;
+            nzw = -zw;
+            kw = -ep.z_a * __ldg(P.wsum + j);
+            sc = ep.scale_a * (ep.s_w ? __ldg(ep.s_w + j) : ep.s_w_scalar);
+            bi = ep.bias ? __ldg(ep.bias + j) : 0.f;
+            if (P.direct_requant) {
+              const float inv = ep.inv_out_scale[j / ep.group_width];
+              sc *= inv;
+              bi *= inv;
+            }
+          }
+          C.nzw[et] = nzw; C.kw[et] = kw; C.sc[et] = sc; C.bi[et] = bi;
         }
         mbar_arrive(smem_u32(&S.cols_ready[acc]));           // release: orders the writes above
         if (!mbar_wait(smem_u32(&S.cols_ready[acc]), acc_phase, abort, 5)) break;
       }
-      if (!mbar_wait(smem_u32(&S.tmem_full[acc]), acc_phase, abort, 4)) break;
-      tc_fence_after();
-
-      const int64_t m = int64_t(m0) + quarter * 32 + lane;
-      const bool row_ok = m < P.M;
-      const int32_t asum_m = row_ok ? __ldg(P.asum + m) : 0;
       const ColTerms& C = S.cols[acc];
       int code_sum = 0;
-#pragma unroll 1
-      for (int c = 0; c < (BN / 2) / 32; ++c) {
-        const int cl = half * (BN / 2) + c * 32;          // column inside the tile
-        uint32_t r[32];
-        __syncwarp();
-        tmem_ld32(tmem_base + (uint32_t(quarter * 32) << 16) + acc * BN + cl, r);
-        tmem_ld_wait();
-        const int col0 = n0 + cl;
-        if (row_ok && col0 < P.N) {
-        const bool full_chunk = col0 + 32 <= P.N;
-        if (ep.acc_debug) {
-          for (int e = 0; e < 32; ++e)
-            if (col0 + e < P.N) ep.acc_debug[m * P.N + col0 + e] = int32_t(r[e]);
-        }
-        float v[32];
+
+      if (!mbar_wait(smem_u32(&S.tmem_full[acc]), acc_phase, abort, 4)) break;
+      tc_fence_after();
+      if (slice_on) {
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          const int32_t corr = int32_t(r[e] - uint32_t(C.z_w[cl + e]) * uint32_t(asum_m) + uint32_t(C.kzz[cl + e]));
-          v[e] = fmaf(C.scale[cl + e], float(corr), C.bias[cl + e]);
-        }
-        if (ep.gelu) {
+        for (int c = 0; c < kSliceChunks; ++c) {
+          const int cl = cl0 + c * kChunk;                     // column inside the tile
+          const int col0 = n0 + cl;
+          const bool live = row_ok && col0 < P.N;
+          const bool full_chunk = col0 + kChunk <= P.N;
+          uint32_t r[kChunk];
+          __syncwarp();
+          tmem_ld16(tmem_base + (uint32_t(quarter * 32) << 16) + acc * kAccStride + cl, r);
+          tmem_ld_wait();
+          if (live) {
+            if (ep.acc_debug) {
+              for (int e = 0; e < kChunk; ++e)
+                if (col0 + e < P.N) ep.acc_debug[m * P.N + col0 + e] = int32_t(r[e]);
+            }
+            float v[kChunk];
 #pragma unroll
-          for (int e = 0; e < 32; ++e) v[e] = gelu_erf(v[e]);
-        }
-        if (ep.residual) {
-          if (ep.residual_bf16) {
-            const __nv_bfloat16* rp = static_cast<const __nv_bfloat16*>(ep.residual) + m * ep.ld_residual + col0;
-            if (full_chunk) {
+            for (int q4 = 0; q4 < kChunk / 4; ++q4) {
+              const int4 nz = *reinterpret_cast<const int4*>(&C.nzw[cl + 4 * q4]);
+              const int4 kw = *reinterpret_cast<const int4*>(&C.kw[cl + 4 * q4]);
+              const float4 sc = *reinterpret_cast<const float4*>(&C.sc[cl + 4 * q4]);
+              const float4 bi = *reinterpret_cast<const float4*>(&C.bi[cl + 4 * q4]);
+              v[4 * q4 + 0] = fmaf(sc.x, float(int32_t(r[4 * q4 + 0]) + nz.x * asum_c + kw.x), bi.x);
+              v[4 * q4 + 1] = fmaf(sc.y, float(int32_t(r[4 * q4 + 1]) + nz.y * asum_c + kw.y), bi.y);
+              v[4 * q4 + 2] = fmaf(sc.z, float(int32_t(r[4 * q4 + 2]) + nz.z * asum_c + kw.z), bi.z);
+              v[4 * q4 + 3] = fmaf(sc.w, float(int32_t(r[4 * q4 + 3]) + nz.w * asum_c + kw.w), bi.w);
+            }
+            if (ep.gelu) {
 #pragma unroll
-              for (int q4 = 0; q4 < 4; ++q4) {
-                const uint4 w = __ldg(reinterpret_cast<const uint4*>(rp) + q4);
-                const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
+              for (int e = 0; e < kChunk; ++e) v[e] = gelu_erf(v[e]);
+            }
+            if (ep.residual) {
+              if (res16 && slice_full) {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  v[q4 * 8 + 2 * i] += __uint_as_float(ws[i] << 16);
-                  v[q4 * 8 + 2 * i + 1] += __uint_as_float(ws[i] & 0xffff0000u);
+                for (int i = 0; i < kChunk / 8; ++i) {
+                  const uint4 w4 = res[c * (kChunk / 8) + i];
+                  const uint32_t ws[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+                  for (int k = 0; k < 4; ++k) {
+                    v[i * 8 + 2 * k] += __uint_as_float(ws[k] << 16);
+                    v[i * 8 + 2 * k + 1] += __uint_as_float(ws[k] & 0xffff0000u);
+                  }
+                }
+              } else if (ep.residual_bf16) {
+                const __nv_bfloat16* rp = static_cast<const __nv_bfloat16*>(ep.residual) + m * ep.ld_residual + col0;
+                for (int e = 0; e < kChunk; ++e) if (col0 + e < P.N) v[e] += __bfloat162float(rp[e]);
+              } else {
+                const float* rp = static_cast<const float*>(ep.residual) + m * ep.ld_residual + col0;
+                if (full_chunk) {
+#pragma unroll
+                  for (int i = 0; i < kChunk / 4; ++i) {
+                    const float4 w4 = __ldg(reinterpret_cast<const float4*>(rp) + i);
+                    v[i * 4] += w4.x; v[i * 4 + 1] += w4.y; v[i * 4 + 2] += w4.z; v[i * 4 + 3] += w4.w;
+                  }
+                } else {
+                  for (int e = 0; e < kChunk; ++e) if (col0 + e < P.N) v[e] += rp[e];
                 }
               }
-            } else {
-              for (int e = 0; e < 32; ++e) if (col0 + e < P.N) v[e] += __bfloat162float(rp[e]);
             }
-          } else {
-            const float* rp = static_cast<const float*>(ep.residual) + m * ep.ld_residual + col0;
-            if (full_chunk) {
-#pragma unroll
-              for (int q4 = 0; q4 < 8; ++q4) {
-                const float4 w = __ldg(reinterpret_cast<const float4*>(rp) + q4);
-                v[q4 * 4] += w.x; v[q4 * 4 + 1] += w.y; v[q4 * 4 + 2] += w.z; v[q4 * 4 + 3] += w.w;
-              }
-            } else {
-              for (int e = 0; e < 32; ++e) if (col0 + e < P.N) v[e] += rp[e];
-            }
+            store_chunk(ep, P, v, m, col0, full_chunk, code_sum);
           }
-        }
-        if (ep.out_kind == REPQ_OUT_F32) {
-          float* o = static_cast<float*>(ep.out) + m * ep.ldo + col0;
-          if (full_chunk) {
-#pragma unroll
-            for (int q4 = 0; q4 < 8; ++q4)
-              reinterpret_cast<float4*>(o)[q4] = make_float4(v[q4 * 4], v[q4 * 4 + 1], v[q4 * 4 + 2], v[q4 * 4 + 3]);
-          } else {
-            for (int e = 0; e < 32; ++e) if (col0 + e < P.N) o[e] = v[e];
-          }
-        } else if (ep.out_kind == REPQ_OUT_BF16) {
-          __nv_bfloat16* o = static_cast<__nv_bfloat16*>(ep.out) + m * ep.ldo + col0;
-          if (full_chunk) {
-#pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) {
-              uint32_t w[4];
-#pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                const __nv_bfloat162 h = __floats2bfloat162_rn(v[q4 * 8 + 2 * i], v[q4 * 8 + 2 * i + 1]);
-                w[i] = *reinterpret_cast<const uint32_t*>(&h);
-              }
-              reinterpret_cast<uint4*>(o)[q4] = make_uint4(w[0], w[1], w[2], w[3]);
-            }
-          } else {
-            for (int e = 0; e < 32; ++e) if (col0 + e < P.N) o[e] = __float2bfloat16_rn(v[e]);
-          }
-        } else {
-          uint32_t q[32];
-#pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            const int zo = C.zo[cl + e];
-            float t = v[e] * C.inv_so[cl + e];
-            t = fminf(fmaxf(t, float(-zo)), float(ep.qmax - zo));
-            q[e] = uint32_t(__float2int_rn(t) + zo);
-            if (col0 + e >= P.N) q[e] = 0;
-            code_sum += int(q[e]);
-          }
-          uint8_t* orow = static_cast<uint8_t*>(ep.out) + m * ep.ldo;
-          if (ep.pack4) {
-            uint32_t w[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              w[i] = 0;
-#pragma unroll
-              for (int e = 0; e < 8; ++e) w[i] |= q[i * 8 + e] << (4 * e);
-            }
-            if (full_chunk) {
-              *reinterpret_cast<uint4*>(orow + (col0 >> 1)) = make_uint4(w[0], w[1], w[2], w[3]);
-            } else {
-              for (int e = 0; e < 32; e += 2)
-                if (col0 + e < P.N) orow[(col0 + e) >> 1] = uint8_t(q[e] | (q[e + 1] << 4));
-            }
-          } else {
-            if (full_chunk) {
-#pragma unroll
-              for (int h2 = 0; h2 < 2; ++h2) {
-                uint32_t w[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  const int b = h2 * 16 + i * 4;
-                  w[i] = q[b] | q[b + 1] << 8 | q[b + 2] << 16 | q[b + 3] << 24;
-                }
-                reinterpret_cast<uint4*>(orow + col0)[h2] = make_uint4(w[0], w[1], w[2], w[3]);
-              }
-            } else {
-              for (int e = 0; e < 32; ++e) if (col0 + e < P.N) orow[col0 + e] = uint8_t(q[e]);
-            }
-          }
-        }
         }
       }
       // accumulator buffer free again
@@ -412,15 +487,14 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static std::once_flag once;
-  std::call_once(once, [] {
+  static EncodeTiledFn fn = [] {
     void* p = nullptr;
     cudaDriverEntryPointQueryResult q;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
         q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  });
+      return reinterpret_cast<EncodeTiledFn>(p);
+    return static_cast<EncodeTiledFn>(nullptr);
+  }();
   return fn;
 }
 
@@ -457,6 +531,32 @@ TcLayout tc_layout(const repq_gemm_desc& d) {
   return L;
 }
 
+// Tile width with the fullest last round: rounds of tiles over the SMs times a cost that grows with BN.
+int pick_bn(int M, int N, int sms) {
+  const int m_tiles = (M + BM - 1) / BM;
+  int best = 256;
+  long best_cost = -1;
+  for (int bn : {256, 192, 128}) {
+    const long tiles = long(m_tiles) * ((N + bn - 1) / bn);
+    const long rounds = (tiles + sms - 1) / sms;
+    const long cost = rounds * (bn + 32);
+    if (best_cost < 0 || cost < best_cost) { best = bn; best_cost = cost; }
+  }
+  return best;
+}
+
+template <int BN>
+repq_status launch_tc(const CUtensorMap& map_a, const CUtensorMap& map_b, const TcParams& P, int sms, cudaStream_t st) {
+  const size_t smem = sizeof(SharedStorage<BN>) + 1024;
+  REPQ_CUDA(cudaFuncSetAttribute(qgemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+  const int tiles = ((P.M + BM - 1) / BM) * ((P.N + BN - 1) / BN);
+  const int grid = tiles < sms ? tiles : sms;
+  qgemm_tc_kernel<BN><<<grid, kThreads, smem, st>>>(map_a, map_b, P);
+  REPQ_CUDA(cudaGetLastError());
+  note_launch();
+  return REPQ_OK;
+}
+
 }  // namespace
 
 int32_t* device_status_word() {
@@ -480,6 +580,7 @@ bool qgemm_tc_supported(const repq_gemm_desc& d) {
   if (d.bits_w != 4 && !(aligned(d.w_codes, 16) && d.ldw_bytes % 16 == 0)) return false;
   const int64_t obytes = d.out_kind == REPQ_OUT_F32 ? 4 : d.out_kind == REPQ_OUT_BF16 ? 2 : 1;
   if (!aligned(d.out, 16) || (d.ldo * obytes) % 16 != 0) return false;
+  if (d.out_kind == REPQ_OUT_CODES && (d.N / d.out_groups) % kChunk != 0) return false;   // one quantizer per 16-column chunk
   if (d.residual) {
     const int64_t rb = d.residual_dtype == REPQ_F32 ? 4 : 2;
     if (!aligned(d.residual, 16) || (d.ld_residual * rb) % 16 != 0) return false;
@@ -521,21 +622,16 @@ repq_status qgemm_tc(const repq_gemm_desc& d, const EpilogueParams& ep, void* ws
     P.wsum = s;
   }
   P.ep = ep;
+  P.direct_requant = d.out_kind == REPQ_OUT_CODES && !d.gelu && !d.residual;
+  REPQ_REQUIRE(device_status_word() != nullptr, REPQ_CUDA_ERROR, "qgemm: device status word unavailable");
+  const int sms = sm_count();
+  const int bn = pick_bn(d.M, d.N, sms);
   CUtensorMap map_a, map_b;
   REPQ_TRY(make_map(&map_a, a, d.M, d.K, lda, BM));
-  REPQ_TRY(make_map(&map_b, w, d.N, d.K, ldw, BN));
-  REPQ_REQUIRE(device_status_word() != nullptr, REPQ_CUDA_ERROR, "qgemm: device status word unavailable");
-
-  const size_t smem = sizeof(SharedStorage) + 1024;
-  REPQ_CUDA(cudaFuncSetAttribute(qgemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
-  const int m_tiles = (d.M + BM - 1) / BM, n_tiles = (d.N + BN - 1) / BN;
-  const int tiles = m_tiles * n_tiles;
-  const int sms = sm_count();
-  const int grid = tiles < sms ? tiles : sms;
-  qgemm_tc_kernel<<<grid, kThreads, smem, st>>>(map_a, map_b, P);
-  REPQ_CUDA(cudaGetLastError());
-  note_launch();
-  return REPQ_OK;
+  REPQ_TRY(make_map(&map_b, w, d.N, d.K, ldw, bn));
+  if (bn == 256) return launch_tc<256>(map_a, map_b, P, sms, st);
+  if (bn == 192) return launch_tc<192>(map_a, map_b, P, sms, st);
+  return launch_tc<128>(map_a, map_b, P, sms, st);
 }
 
 }  // namespace repq
