@@ -160,108 +160,130 @@ struct TcParams {
   EpilogueParams ep;
 };
 
-// One 16-column chunk of one output row: v[e] holds the float value before the output conversion.
-__device__ __forceinline__ void store_chunk(const EpilogueParams& ep, const TcParams& P, float (&v)[kChunk], int64_t m,
-                                            int col0, bool full_chunk, int& code_sum) {
-  if (ep.out_kind == REPQ_OUT_F32) {
-    float* o = static_cast<float*>(ep.out) + m * ep.ldo + col0;
-    if (full_chunk) {
-#pragma unroll
-      for (int q4 = 0; q4 < kChunk / 4; ++q4)
-        reinterpret_cast<float4*>(o)[q4] = make_float4(v[q4 * 4], v[q4 * 4 + 1], v[q4 * 4 + 2], v[q4 * 4 + 3]);
-    } else {
-      for (int e = 0; e < kChunk; ++e) if (col0 + e < P.N) o[e] = v[e];
-    }
-    return;
-  }
-  if (ep.out_kind == REPQ_OUT_BF16) {
-    __nv_bfloat16* o = static_cast<__nv_bfloat16*>(ep.out) + m * ep.ldo + col0;
-    if (full_chunk) {
-#pragma unroll
-      for (int q4 = 0; q4 < kChunk / 8; ++q4) {
-        uint32_t w[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const __nv_bfloat162 h = __floats2bfloat162_rn(v[q4 * 8 + 2 * i], v[q4 * 8 + 2 * i + 1]);
-          w[i] = *reinterpret_cast<const uint32_t*>(&h);
-        }
-        reinterpret_cast<uint4*>(o)[q4] = make_uint4(w[0], w[1], w[2], w[3]);
-      }
-    } else {
-      for (int e = 0; e < kChunk; ++e) if (col0 + e < P.N) o[e] = __float2bfloat16_rn(v[e]);
-    }
-    return;
-  }
-  // codes: Eq. 4 with the output quantizer of this chunk's column group
-  const int group = col0 / ep.group_width;
+enum : int { kOutF32 = 0, kOutBf16 = 1, kOutC4 = 2, kOutC8 = 3 };   // compile-time output kinds of the fast path
+
+// Output quantizer of one 16-column chunk (Eq. 4 with the chunk's column group).
+struct ChunkQuant {
+  float mult, lo, hi;
+  uint32_t pack_k;     // 4-bit: sum_e (magic_bits - z_o) << 4e
+  uint32_t z4;         // 8-bit: z_o replicated in every byte
+  int zo;
+};
+
+__device__ __forceinline__ ChunkQuant chunk_quant(const EpilogueParams& ep, const TcParams& P, int col0) {
+  const int gw = ep.group_width;
+  const int group = (col0 >= gw) + (col0 >= 2 * gw) + (col0 >= 3 * gw);
   const int zo = ep.out_zero[group];
-  const float lo = float(-zo), hi = float(ep.qmax - zo);
-  const float mult = P.direct_requant ? 1.f : ep.inv_out_scale[group];
-  const float magic = __uint_as_float(kMagicBits);
-  uint32_t u[kChunk];
+  ChunkQuant q;
+  q.mult = P.direct_requant ? 1.f : ep.inv_out_scale[group];
+  q.lo = float(-zo);
+  q.hi = float(ep.qmax - zo);
+  q.pack_k = (kMagicBits - uint32_t(zo)) * 0x11111111u;
+  q.z4 = (uint32_t(zo) & 0xFFu) * 0x01010101u;
+  q.zo = zo;
+  return q;
+}
+
+// Fast path: a full 16-column chunk of a valid row, output kind fixed at compile time.
+template <int OUT>
+__device__ __forceinline__ void store_fast(const EpilogueParams& ep, const ChunkQuant& q, float (&v)[kChunk], int64_t m,
+                                           int col0, int& code_sum) {
+  if constexpr (OUT == kOutF32) {
+    float4* o = reinterpret_cast<float4*>(static_cast<float*>(ep.out) + m * ep.ldo + col0);
 #pragma unroll
-  for (int e = 0; e < kChunk; ++e) {
-    float t = v[e] * mult;
-    t = fminf(fmaxf(t, lo), hi);
-    u[e] = __float_as_uint(t + magic);             // magic_bits + round_half_even(t)
-  }
-  uint8_t* orow = static_cast<uint8_t*>(ep.out) + m * ep.ldo;
-  if (ep.pack4) {
-    uint32_t k = 0;
+    for (int i = 0; i < kChunk / 4; ++i) o[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+  } else if constexpr (OUT == kOutBf16) {
+    uint4* o = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(ep.out) + m * ep.ldo + col0);
 #pragma unroll
-    for (int e = 0; e < 8; ++e) k += (kMagicBits - uint32_t(zo)) << (4 * e);
-    uint32_t w[2];
+    for (int i = 0; i < kChunk / 8; ++i) {
+      uint32_t w[4];
 #pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      w[i] = 0;
-#pragma unroll
-      for (int e = 0; e < 8; ++e) w[i] += u[i * 8 + e] << (4 * e);
-      w[i] -= k;
-    }
-    if (full_chunk) {
-      *reinterpret_cast<uint2*>(orow + (col0 >> 1)) = make_uint2(w[0], w[1]);
-#pragma unroll
-      for (int i = 0; i < 2; ++i)
-        code_sum += __dp4a(w[i] & 0x0F0F0F0Fu, 0x01010101u, 0u) + __dp4a((w[i] >> 4) & 0x0F0F0F0Fu, 0x01010101u, 0u);
-    } else {
-      for (int e = 0; e < kChunk; e += 2) {
-        if (col0 + e < P.N) {
-          const uint32_t byte = (w[e >> 3] >> (4 * (e & 7))) & (col0 + e + 1 < P.N ? 0xFFu : 0x0Fu);
-          orow[(col0 + e) >> 1] = uint8_t(byte);
-          code_sum += int(byte & 15u) + int(byte >> 4);
-        }
+      for (int k = 0; k < 4; ++k) {
+        const __nv_bfloat162 h = __floats2bfloat162_rn(v[8 * i + 2 * k], v[8 * i + 2 * k + 1]);
+        w[k] = *reinterpret_cast<const uint32_t*>(&h);
       }
+      o[i] = make_uint4(w[0], w[1], w[2], w[3]);
     }
   } else {
-    const uint32_t z4 = (uint32_t(zo) & 0xFFu) * 0x01010101u;
-    uint32_t w[4];
+    const float magic = __uint_as_float(kMagicBits);
+    uint32_t u[kChunk];
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
-      w[i] = __vadd4(__byte_perm(__byte_perm(u[4 * i], u[4 * i + 1], 0x0040), __byte_perm(u[4 * i + 2], u[4 * i + 3], 0x0040), 0x5410), z4);
-    if (full_chunk) {
-      *reinterpret_cast<uint4*>(orow + col0) = make_uint4(w[0], w[1], w[2], w[3]);
+    for (int e = 0; e < kChunk; ++e) {
+      const float t = fminf(fmaxf(v[e] * q.mult, q.lo), q.hi);
+      u[e] = __float_as_uint(t + magic);             // magic_bits + round_half_even(t)
+    }
+    uint8_t* orow = static_cast<uint8_t*>(ep.out) + m * ep.ldo;
+    if constexpr (OUT == kOutC4) {
+      uint32_t w[2];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) code_sum += __dp4a(w[i], 0x01010101u, 0u);
+      for (int i = 0; i < 2; ++i) {
+        w[i] = 0;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) w[i] += u[i * 8 + e] << (4 * e);
+        w[i] -= q.pack_k;
+        code_sum += __dp4a(w[i] & 0x0F0F0F0Fu, 0x01010101u, 0u) + __dp4a((w[i] >> 4) & 0x0F0F0F0Fu, 0x01010101u, 0u);
+      }
+      *reinterpret_cast<uint2*>(orow + (col0 >> 1)) = make_uint2(w[0], w[1]);
     } else {
-      for (int e = 0; e < kChunk; ++e) {
-        if (col0 + e < P.N) {
-          const uint32_t byte = (w[e >> 2] >> (8 * (e & 3))) & 0xFFu;
-          orow[col0 + e] = uint8_t(byte);
-          code_sum += int(byte);
-        }
+      uint32_t w[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        w[i] = __vadd4(__byte_perm(__byte_perm(u[4 * i], u[4 * i + 1], 0x0040), __byte_perm(u[4 * i + 2], u[4 * i + 3], 0x0040), 0x5410), q.z4);
+        code_sum += __dp4a(w[i], 0x01010101u, 0u);
+      }
+      *reinterpret_cast<uint4*>(orow + col0) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+  }
+}
+
+// General path for one chunk of one thread (ragged rows / columns, float32 residual, accumulator dump):
+// element by element, kept out of line so that the common path stays small.
+__device__ __noinline__ void slow_chunk(const EpilogueParams& ep, const TcParams& P, const ColTerms& C, const uint32_t* r,
+                                        int cl, int64_t m, int col0, int32_t asum_c, int* code_sum) {
+  const ChunkQuant q = chunk_quant(ep, P, col0);
+  const float magic = __uint_as_float(kMagicBits);
+  uint32_t prev_code = 0;
+  for (int e = 0; e < kChunk; ++e) {
+    const int j = col0 + e;
+    if (j >= P.N) break;
+    if (ep.acc_debug) ep.acc_debug[m * P.N + j] = int32_t(r[e]);
+    float v = fmaf(C.sc[cl + e], float(int32_t(r[e]) + C.nzw[cl + e] * asum_c + C.kw[cl + e]), C.bi[cl + e]);
+    if (ep.gelu) v = gelu_erf(v);
+    if (ep.residual) {
+      const int64_t off = m * ep.ld_residual + j;
+      v += ep.residual_bf16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(ep.residual)[off])
+                            : static_cast<const float*>(ep.residual)[off];
+    }
+    if (ep.out_kind == REPQ_OUT_F32) {
+      static_cast<float*>(ep.out)[m * ep.ldo + j] = v;
+    } else if (ep.out_kind == REPQ_OUT_BF16) {
+      static_cast<__nv_bfloat16*>(ep.out)[m * ep.ldo + j] = __float2bfloat16_rn(v);
+    } else {
+      const float t = fminf(fmaxf(v * q.mult, q.lo), q.hi);
+      const uint32_t code = (__float_as_uint(t + magic) - kMagicBits) + uint32_t(q.zo);
+      *code_sum += int(code);
+      uint8_t* orow = static_cast<uint8_t*>(ep.out) + m * ep.ldo;
+      if (ep.pack4) {
+        if (e & 1) orow[j >> 1] = uint8_t(prev_code | (code << 4));
+        else if (j + 1 >= P.N) orow[j >> 1] = uint8_t(code);
+        prev_code = code;
+      } else {
+        orow[j] = uint8_t(code);
       }
     }
   }
 }
 
-template <int BN>
+template <int BN, int OUT>
 __global__ void __launch_bounds__(kThreads, 1)
 qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, TcParams P) {
   using Storage = SharedStorage<BN>;
   constexpr uint32_t kBBytes = BN * BK;
   constexpr uint32_t kIdesc = idesc_for(BN);
-  extern __shared__ uint8_t smem_raw[];
-  Storage& S = *reinterpret_cast<Storage*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  // 1024-byte alignment (swizzle atoms) is requested from the declaration so that the compiler keeps
+  // treating every access below as a shared-memory access (a hand-aligned generic pointer would not)
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  Storage& S = *reinterpret_cast<Storage*>(smem_raw);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m_tiles = (P.M + BM - 1) / BM, n_tiles = (P.N + BN - 1) / BN;
@@ -274,6 +296,10 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     for (int a = 0; a < 2; ++a) mbar_init(smem_u32(&S.cols_ready[a]), kEpiThreads);
     mbar_init(smem_u32(&S.done), 1);
     S.abort = 0;
+    if (smem_u32(smem_raw) & 1023u) {              // the swizzled tiles need the alignment asked for above
+      atomicCAS(&g_status_word, 0, 9);
+      S.abort = 1;
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -351,6 +377,33 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     const EpilogueParams& ep = P.ep;
     const int kza = P.K * ep.z_a;
     const bool res16 = ep.residual != nullptr && ep.residual_bf16;
+    const bool fast_ok = ep.acc_debug == nullptr && (ep.residual == nullptr || res16);
+    // per-column terms (threads 0..BN-1: column et of the tile) and the row's code sum, fetched one tile ahead
+    int nx_nzw = 0, nx_kw = 0, nx_asum = 0;
+    float nx_sc = 0.f, nx_bi = 0.f;
+    auto fetch_terms = [&](int t) {
+      if (t >= tiles) return;
+      const int tm0 = (t % m_tiles) * BM, tn0 = (t / m_tiles) * BN;
+      const int64_t tm = int64_t(tm0) + quarter * 32 + lane;
+      nx_asum = tm < P.M ? __ldg(P.asum + tm) : 0;
+      if (et < BN) {
+        const int j = tn0 + et;
+        nx_nzw = 0; nx_kw = 0; nx_sc = 0.f; nx_bi = 0.f;
+        if (j < P.N) {
+          nx_nzw = -(ep.z_w ? __ldg(ep.z_w + j) : ep.z_w_scalar);
+          nx_kw = -ep.z_a * __ldg(P.wsum + j);
+          nx_sc = ep.scale_a * (ep.s_w ? __ldg(ep.s_w + j) : ep.s_w_scalar);
+          nx_bi = ep.bias ? __ldg(ep.bias + j) : 0.f;
+          if (P.direct_requant) {
+            const int gw = ep.group_width;
+            const float inv = ep.inv_out_scale[(j >= gw) + (j >= 2 * gw) + (j >= 3 * gw)];
+            nx_sc *= inv;
+            nx_bi *= inv;
+          }
+        }
+      }
+    };
+    fetch_terms(blockIdx.x);
     int it = 0;
     for (int tile = blockIdx.x; tile < tiles && !*abort; tile += gridDim.x, ++it) {
       const uint32_t acc = it & 1, acc_phase = (it >> 1) & 1;
@@ -358,109 +411,82 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       const int64_t m = int64_t(m0) + quarter * 32 + lane;
       const bool row_ok = m < P.M;
       const int cl0 = slice * kSliceCols;                    // first column of this warp inside the tile
-      // whole 64-column slice inside the matrix: vector paths everywhere
-      const bool slice_full = slice_on && n0 + cl0 + kSliceCols <= P.N;
-      // bf16 residual of the slice and the row's code sum: requested now, needed only after the main loop
+      // warp-uniform: every row of the warp valid, whole 64-column slice inside the matrix, common epilogue
+      const bool fast = fast_ok && slice_on && n0 + cl0 + kSliceCols <= P.N && m0 + quarter * 32 + 32 <= P.M;
+      const bool any_row = m0 + quarter * 32 < P.M;          // warp-uniform: at least one valid row
+      // bf16 residual of the slice: requested now, needed only after the main loop of the tile
       uint4 res[kSliceCols / 8];
-      if (res16 && row_ok && slice_full) {
+      if (fast && res16) {
         const uint4* rp = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(ep.residual) + m * ep.ld_residual + n0 + cl0);
 #pragma unroll
         for (int i = 0; i < kSliceCols / 8; ++i) res[i] = __ldg(rp + i);
       }
-      // corr = acc - z_w (asum - K z_a) - z_a wsum
-      const int32_t asum_c = row_ok ? __ldg(P.asum + m) - kza : 0;
+      // corr = acc - z_w (asum - K z_a) - z_a wsum; this tile's terms were fetched during the previous tile
+      const int32_t asum_c = row_ok ? nx_asum - kza : 0;
       // stage the per-column terms of this tile (one column per thread, threads 0..BN-1); the buffer was last
       // read two tiles ago, and every epilogue thread has passed the barrier of the tile in between
       {
         ColTerms& C = S.cols[acc];
-        if (et < BN) {
-          const int j = n0 + et;
-          int nzw = 0, kw = 0;
-          float sc = 0.f, bi = 0.f;
-          if (j < P.N) {
-            const int zw = ep.z_w ? __ldg(ep.z_w + j) : ep.z_w_scalar;
-            nzw = -zw;
-            kw = -ep.z_a * __ldg(P.wsum + j);
-            sc = ep.scale_a * (ep.s_w ? __ldg(ep.s_w + j) : ep.s_w_scalar);
-            bi = ep.bias ? __ldg(ep.bias + j) : 0.f;
-            if (P.direct_requant) {
-              const float inv = ep.inv_out_scale[j / ep.group_width];
-              sc *= inv;
-              bi *= inv;
-            }
-          }
-          C.nzw[et] = nzw; C.kw[et] = kw; C.sc[et] = sc; C.bi[et] = bi;
-        }
+        if (et < BN) { C.nzw[et] = nx_nzw; C.kw[et] = nx_kw; C.sc[et] = nx_sc; C.bi[et] = nx_bi; }
         mbar_arrive(smem_u32(&S.cols_ready[acc]));           // release: orders the writes above
         if (!mbar_wait(smem_u32(&S.cols_ready[acc]), acc_phase, abort, 5)) break;
       }
+      fetch_terms(tile + int(gridDim.x));                    // next tile's terms: in flight during this epilogue
       const ColTerms& C = S.cols[acc];
       int code_sum = 0;
 
       if (!mbar_wait(smem_u32(&S.tmem_full[acc]), acc_phase, abort, 4)) break;
       tc_fence_after();
-      if (slice_on) {
+      const uint32_t taddr0 = tmem_base + (uint32_t(quarter * 32) << 16) + acc * kAccStride + cl0;
+      if (fast) {
 #pragma unroll
         for (int c = 0; c < kSliceChunks; ++c) {
           const int cl = cl0 + c * kChunk;                     // column inside the tile
           const int col0 = n0 + cl;
-          const bool live = row_ok && col0 < P.N;
-          const bool full_chunk = col0 + kChunk <= P.N;
           uint32_t r[kChunk];
-          __syncwarp();
-          tmem_ld16(tmem_base + (uint32_t(quarter * 32) << 16) + acc * kAccStride + cl, r);
+          tmem_ld16(taddr0 + c * kChunk, r);
           tmem_ld_wait();
-          if (live) {
-            if (ep.acc_debug) {
-              for (int e = 0; e < kChunk; ++e)
-                if (col0 + e < P.N) ep.acc_debug[m * P.N + col0 + e] = int32_t(r[e]);
-            }
-            float v[kChunk];
+          float v[kChunk];
 #pragma unroll
-            for (int q4 = 0; q4 < kChunk / 4; ++q4) {
-              const int4 nz = *reinterpret_cast<const int4*>(&C.nzw[cl + 4 * q4]);
-              const int4 kw = *reinterpret_cast<const int4*>(&C.kw[cl + 4 * q4]);
-              const float4 sc = *reinterpret_cast<const float4*>(&C.sc[cl + 4 * q4]);
-              const float4 bi = *reinterpret_cast<const float4*>(&C.bi[cl + 4 * q4]);
-              v[4 * q4 + 0] = fmaf(sc.x, float(int32_t(r[4 * q4 + 0]) + nz.x * asum_c + kw.x), bi.x);
-              v[4 * q4 + 1] = fmaf(sc.y, float(int32_t(r[4 * q4 + 1]) + nz.y * asum_c + kw.y), bi.y);
-              v[4 * q4 + 2] = fmaf(sc.z, float(int32_t(r[4 * q4 + 2]) + nz.z * asum_c + kw.z), bi.z);
-              v[4 * q4 + 3] = fmaf(sc.w, float(int32_t(r[4 * q4 + 3]) + nz.w * asum_c + kw.w), bi.w);
-            }
-            if (ep.gelu) {
+          for (int q4 = 0; q4 < kChunk / 4; ++q4) {
+            const int4 nz = *reinterpret_cast<const int4*>(&C.nzw[cl + 4 * q4]);
+            const int4 kw = *reinterpret_cast<const int4*>(&C.kw[cl + 4 * q4]);
+            const float4 sc = *reinterpret_cast<const float4*>(&C.sc[cl + 4 * q4]);
+            const float4 bi = *reinterpret_cast<const float4*>(&C.bi[cl + 4 * q4]);
+            v[4 * q4 + 0] = fmaf(sc.x, float(int32_t(r[4 * q4 + 0]) + nz.x * asum_c + kw.x), bi.x);
+            v[4 * q4 + 1] = fmaf(sc.y, float(int32_t(r[4 * q4 + 1]) + nz.y * asum_c + kw.y), bi.y);
+            v[4 * q4 + 2] = fmaf(sc.z, float(int32_t(r[4 * q4 + 2]) + nz.z * asum_c + kw.z), bi.z);
+            v[4 * q4 + 3] = fmaf(sc.w, float(int32_t(r[4 * q4 + 3]) + nz.w * asum_c + kw.w), bi.w);
+          }
+          if (ep.gelu) {
 #pragma unroll
-              for (int e = 0; e < kChunk; ++e) v[e] = gelu_erf(v[e]);
-            }
-            if (ep.residual) {
-              if (res16 && slice_full) {
+            for (int e = 0; e < kChunk; ++e) v[e] = gelu_erf(v[e]);
+          }
+          if (res16) {
 #pragma unroll
-                for (int i = 0; i < kChunk / 8; ++i) {
-                  const uint4 w4 = res[c * (kChunk / 8) + i];
-                  const uint32_t ws[4] = {w4.x, w4.y, w4.z, w4.w};
+            for (int i = 0; i < kChunk / 8; ++i) {
+              const uint4 w4 = res[c * (kChunk / 8) + i];
+              const uint32_t ws[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
-                  for (int k = 0; k < 4; ++k) {
-                    v[i * 8 + 2 * k] += __uint_as_float(ws[k] << 16);
-                    v[i * 8 + 2 * k + 1] += __uint_as_float(ws[k] & 0xffff0000u);
-                  }
-                }
-              } else if (ep.residual_bf16) {
-                const __nv_bfloat16* rp = static_cast<const __nv_bfloat16*>(ep.residual) + m * ep.ld_residual + col0;
-                for (int e = 0; e < kChunk; ++e) if (col0 + e < P.N) v[e] += __bfloat162float(rp[e]);
-              } else {
-                const float* rp = static_cast<const float*>(ep.residual) + m * ep.ld_residual + col0;
-                if (full_chunk) {
-#pragma unroll
-                  for (int i = 0; i < kChunk / 4; ++i) {
-                    const float4 w4 = __ldg(reinterpret_cast<const float4*>(rp) + i);
-                    v[i * 4] += w4.x; v[i * 4 + 1] += w4.y; v[i * 4 + 2] += w4.z; v[i * 4 + 3] += w4.w;
-                  }
-                } else {
-                  for (int e = 0; e < kChunk; ++e) if (col0 + e < P.N) v[e] += rp[e];
-                }
+              for (int k = 0; k < 4; ++k) {
+                v[i * 8 + 2 * k] += __uint_as_float(ws[k] << 16);
+                v[i * 8 + 2 * k + 1] += __uint_as_float(ws[k] & 0xffff0000u);
               }
             }
-            store_chunk(ep, P, v, m, col0, full_chunk, code_sum);
           }
+          ChunkQuant q{};
+          if constexpr (OUT == kOutC4 || OUT == kOutC8) q = chunk_quant(ep, P, col0);
+          store_fast<OUT>(ep, q, v, m, col0, code_sum);
+        }
+      } else if (slice_on && any_row && n0 + cl0 < P.N) {
+#pragma unroll 1
+        for (int c = 0; c < kSliceChunks; ++c) {
+          const int cl = cl0 + c * kChunk;
+          uint32_t r[kChunk];
+          __syncwarp();
+          tmem_ld16(taddr0 + c * kChunk, r);
+          tmem_ld_wait();
+          if (row_ok && n0 + cl < P.N) slow_chunk(ep, P, C, r, cl, m, n0 + cl, asum_c, &code_sum);
         }
       }
       // accumulator buffer free again
@@ -545,16 +571,24 @@ int pick_bn(int M, int N, int sms) {
   return best;
 }
 
-template <int BN>
-repq_status launch_tc(const CUtensorMap& map_a, const CUtensorMap& map_b, const TcParams& P, int sms, cudaStream_t st) {
-  const size_t smem = sizeof(SharedStorage<BN>) + 1024;
-  REPQ_CUDA(cudaFuncSetAttribute(qgemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+template <int BN, int OUT>
+repq_status launch_tc_out(const CUtensorMap& map_a, const CUtensorMap& map_b, const TcParams& P, int sms, cudaStream_t st) {
+  const size_t smem = sizeof(SharedStorage<BN>);
+  REPQ_CUDA(cudaFuncSetAttribute(qgemm_tc_kernel<BN, OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
   const int tiles = ((P.M + BM - 1) / BM) * ((P.N + BN - 1) / BN);
   const int grid = tiles < sms ? tiles : sms;
-  qgemm_tc_kernel<BN><<<grid, kThreads, smem, st>>>(map_a, map_b, P);
+  qgemm_tc_kernel<BN, OUT><<<grid, kThreads, smem, st>>>(map_a, map_b, P);
   REPQ_CUDA(cudaGetLastError());
   note_launch();
   return REPQ_OK;
+}
+
+template <int BN>
+repq_status launch_tc(const CUtensorMap& map_a, const CUtensorMap& map_b, const TcParams& P, int sms, cudaStream_t st) {
+  if (P.ep.out_kind == REPQ_OUT_F32) return launch_tc_out<BN, kOutF32>(map_a, map_b, P, sms, st);
+  if (P.ep.out_kind == REPQ_OUT_BF16) return launch_tc_out<BN, kOutBf16>(map_a, map_b, P, sms, st);
+  if (P.ep.pack4) return launch_tc_out<BN, kOutC4>(map_a, map_b, P, sms, st);
+  return launch_tc_out<BN, kOutC8>(map_a, map_b, P, sms, st);
 }
 
 }  // namespace
