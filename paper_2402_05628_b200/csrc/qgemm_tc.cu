@@ -62,6 +62,7 @@ template <int BN>
 struct SharedStorage {
   alignas(1024) uint8_t a[kStages][kABytes];
   alignas(1024) uint8_t b[kStages][BN * BK];
+  alignas(1024) uint8_t epi[kEpiWarps][1024];     // per-warp staging box of the epilogue's bulk stores
   ColTerms cols[2];
   alignas(8) uint64_t full[kStages];
   uint64_t empty[kStages];
@@ -184,26 +185,64 @@ __device__ __forceinline__ ChunkQuant chunk_quant(const EpilogueParams& ep, cons
   return q;
 }
 
-// Fast path: a full 16-column chunk of a valid row, output kind fixed at compile time.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
+}
+
+// The warp's 1 KB staging buffer holds a box of 32 rows x 32 bytes in the 32-byte swizzle of the output tensor
+// map (16-byte slot j of row r sits at r * 32 + ((j ^ ((r >> 2) & 1)) << 4): conflict-free for one row per lane).
+// begin: the previous bulk store must have finished reading the buffer; end: make the generic-proxy writes
+// visible to the bulk-copy engine, then one lane issues the store (rows / columns outside the matrix are clipped).
+__device__ __forceinline__ void box_begin(int lane) {
+  if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+  __syncwarp();
+}
+__device__ __forceinline__ void box_end(const CUtensorMap* map, uint32_t buf, int lane, int x, int y) {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  __syncwarp();
+  if (lane == 0) {
+    tma_store_2d(map, buf, x, y);
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+  }
+}
+__device__ __forceinline__ uint32_t box_slot(uint32_t buf, int lane, int j) {
+  return buf + uint32_t(lane) * 32u + (uint32_t(j ^ ((lane >> 2) & 1)) << 4);
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ void sts64(uint32_t addr, uint32_t a, uint32_t b) {
+  asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(addr), "r"(a), "r"(b) : "memory");
+}
+
+// Fast path: chunk c (16 columns) of the warp's 64-column slice, one row per lane, output kind fixed at compile
+// time.  Values go to the staging buffer and leave through bulk tensor stores: one per chunk (bf16), two per
+// chunk (f32), one per two chunks (byte codes) or one per slice (4-bit codes).
 template <int OUT>
-__device__ __forceinline__ void store_fast(const EpilogueParams& ep, const ChunkQuant& q, float (&v)[kChunk], int64_t m,
-                                           int col0, int& code_sum) {
+__device__ __forceinline__ void emit_chunk(const CUtensorMap* map_out, uint32_t buf, int lane, const ChunkQuant& q,
+                                           float (&v)[kChunk], int c, int col0, int row0, int& code_sum) {
   if constexpr (OUT == kOutF32) {
-    float4* o = reinterpret_cast<float4*>(static_cast<float*>(ep.out) + m * ep.ldo + col0);
 #pragma unroll
-    for (int i = 0; i < kChunk / 4; ++i) o[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-  } else if constexpr (OUT == kOutBf16) {
-    uint4* o = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(ep.out) + m * ep.ldo + col0);
+    for (int h = 0; h < 2; ++h) {
+      box_begin(lane);
 #pragma unroll
-    for (int i = 0; i < kChunk / 8; ++i) {
-      uint32_t w[4];
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const __nv_bfloat162 h = __floats2bfloat162_rn(v[8 * i + 2 * k], v[8 * i + 2 * k + 1]);
-        w[k] = *reinterpret_cast<const uint32_t*>(&h);
-      }
-      o[i] = make_uint4(w[0], w[1], w[2], w[3]);
+      for (int j = 0; j < 2; ++j)
+        sts128(box_slot(buf, lane, j), __float_as_uint(v[8 * h + 4 * j]), __float_as_uint(v[8 * h + 4 * j + 1]),
+               __float_as_uint(v[8 * h + 4 * j + 2]), __float_as_uint(v[8 * h + 4 * j + 3]));
+      box_end(map_out, buf, lane, col0 + 8 * h, row0);
     }
+  } else if constexpr (OUT == kOutBf16) {
+    uint32_t w[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * k], v[2 * k + 1]);
+      w[k] = *reinterpret_cast<const uint32_t*>(&h);
+    }
+    box_begin(lane);
+    sts128(box_slot(buf, lane, 0), w[0], w[1], w[2], w[3]);
+    sts128(box_slot(buf, lane, 1), w[4], w[5], w[6], w[7]);
+    box_end(map_out, buf, lane, col0, row0);
   } else {
     const float magic = __uint_as_float(kMagicBits);
     uint32_t u[kChunk];
@@ -212,7 +251,6 @@ __device__ __forceinline__ void store_fast(const EpilogueParams& ep, const Chunk
       const float t = fminf(fmaxf(v[e] * q.mult, q.lo), q.hi);
       u[e] = __float_as_uint(t + magic);             // magic_bits + round_half_even(t)
     }
-    uint8_t* orow = static_cast<uint8_t*>(ep.out) + m * ep.ldo;
     if constexpr (OUT == kOutC4) {
       uint32_t w[2];
 #pragma unroll
@@ -223,7 +261,9 @@ __device__ __forceinline__ void store_fast(const EpilogueParams& ep, const Chunk
         w[i] -= q.pack_k;
         code_sum += __dp4a(w[i] & 0x0F0F0F0Fu, 0x01010101u, 0u) + __dp4a((w[i] >> 4) & 0x0F0F0F0Fu, 0x01010101u, 0u);
       }
-      *reinterpret_cast<uint2*>(orow + (col0 >> 1)) = make_uint2(w[0], w[1]);
+      if (c == 0) box_begin(lane);
+      sts64(box_slot(buf, lane, c >> 1) + uint32_t(c & 1) * 8u, w[0], w[1]);     // 8 bytes = 16 codes
+      if (c == kSliceChunks - 1) box_end(map_out, buf, lane, (col0 - (kSliceChunks - 1) * kChunk) >> 1, row0);
     } else {
       uint32_t w[4];
 #pragma unroll
@@ -231,7 +271,9 @@ __device__ __forceinline__ void store_fast(const EpilogueParams& ep, const Chunk
         w[i] = __vadd4(__byte_perm(__byte_perm(u[4 * i], u[4 * i + 1], 0x0040), __byte_perm(u[4 * i + 2], u[4 * i + 3], 0x0040), 0x5410), q.z4);
         code_sum += __dp4a(w[i], 0x01010101u, 0u);
       }
-      *reinterpret_cast<uint4*>(orow + col0) = make_uint4(w[0], w[1], w[2], w[3]);
+      if ((c & 1) == 0) box_begin(lane);
+      sts128(box_slot(buf, lane, c & 1), w[0], w[1], w[2], w[3]);
+      if (c & 1) box_end(map_out, buf, lane, col0 - kChunk, row0);
     }
   }
 }
@@ -276,7 +318,8 @@ __device__ __noinline__ void slow_chunk(const EpilogueParams& ep, const TcParams
 
 template <int BN, int OUT>
 __global__ void __launch_bounds__(kThreads, 1)
-qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, TcParams P) {
+qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                const __grid_constant__ CUtensorMap map_out, TcParams P) {
   using Storage = SharedStorage<BN>;
   constexpr uint32_t kBBytes = BN * BK;
   constexpr uint32_t kIdesc = idesc_for(BN);
@@ -411,12 +454,13 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       const int64_t m = int64_t(m0) + quarter * 32 + lane;
       const bool row_ok = m < P.M;
       const int cl0 = slice * kSliceCols;                    // first column of this warp inside the tile
-      // warp-uniform: every row of the warp valid, whole 64-column slice inside the matrix, common epilogue
-      const bool fast = fast_ok && slice_on && n0 + cl0 + kSliceCols <= P.N && m0 + quarter * 32 + 32 <= P.M;
+      // warp-uniform: whole 64-column slice inside the matrix, common epilogue (rows beyond M are clipped by
+      // the bulk store)
       const bool any_row = m0 + quarter * 32 < P.M;          // warp-uniform: at least one valid row
+      const bool fast = fast_ok && slice_on && n0 + cl0 + kSliceCols <= P.N && any_row;
       // bf16 residual of the slice: requested now, needed only after the main loop of the tile
       uint4 res[kSliceCols / 8];
-      if (fast && res16) {
+      if (fast && res16 && row_ok) {
         const uint4* rp = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(ep.residual) + m * ep.ld_residual + n0 + cl0);
 #pragma unroll
         for (int i = 0; i < kSliceCols / 8; ++i) res[i] = __ldg(rp + i);
@@ -462,7 +506,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 #pragma unroll
             for (int e = 0; e < kChunk; ++e) v[e] = gelu_erf(v[e]);
           }
-          if (res16) {
+          if (res16 && row_ok) {
 #pragma unroll
             for (int i = 0; i < kChunk / 8; ++i) {
               const uint4 w4 = res[c * (kChunk / 8) + i];
@@ -476,7 +520,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
           }
           ChunkQuant q{};
           if constexpr (OUT == kOutC4 || OUT == kOutC8) q = chunk_quant(ep, P, col0);
-          store_fast<OUT>(ep, q, v, m, col0, code_sum);
+          emit_chunk<OUT>(&map_out, smem_u32(S.epi[ew]), lane, q, v, c, col0, m0 + quarter * 32, code_sum);
         }
       } else if (slice_on && any_row && n0 + cl0 < P.N) {
 #pragma unroll 1
@@ -495,6 +539,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       if (lane == 0) mbar_arrive(smem_u32(&S.tmem_empty[acc]));
       if (ep.out_row_sum != nullptr && row_ok && code_sum != 0) atomicAdd(ep.out_row_sum + m, code_sum);
     }
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");     // bulk stores complete
   }
 
   // ------------------------------------------------------------------ teardown
@@ -571,13 +616,35 @@ int pick_bn(int M, int N, int sms) {
   return best;
 }
 
+// Tensor map of the output for the epilogue's bulk stores: boxes of 32 rows x 32 bytes, 32-byte swizzle.
+repq_status make_out_map(CUtensorMap* map, const TcParams& P) {
+  EncodeTiledFn fn = encode_fn();
+  REPQ_REQUIRE(fn != nullptr, REPQ_CUDA_ERROR, "qgemm: cuTensorMapEncodeTiled is not available");
+  const EpilogueParams& ep = P.ep;
+  CUtensorMapDataType dt = CU_TENSOR_MAP_DATA_TYPE_UINT8;
+  cuuint64_t inner = cuuint64_t(P.N), esz = 1;
+  if (ep.out_kind == REPQ_OUT_F32) { dt = CU_TENSOR_MAP_DATA_TYPE_FLOAT32; esz = 4; }
+  else if (ep.out_kind == REPQ_OUT_BF16) { dt = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16; esz = 2; }
+  else if (ep.pack4) inner = cuuint64_t(P.N) / 2;
+  const cuuint64_t dims[2] = {inner, cuuint64_t(P.M)};
+  const cuuint64_t strides[1] = {cuuint64_t(ep.ldo) * esz};
+  const cuuint32_t box[2] = {cuuint32_t(32 / esz), 32};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(map, dt, 2, ep.out, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  REPQ_REQUIRE(r == CUDA_SUCCESS, REPQ_CUDA_ERROR, "qgemm: output tensor map failed with code %d", int(r));
+  return REPQ_OK;
+}
+
 template <int BN, int OUT>
 repq_status launch_tc_out(const CUtensorMap& map_a, const CUtensorMap& map_b, const TcParams& P, int sms, cudaStream_t st) {
+  CUtensorMap map_out;
+  REPQ_TRY(make_out_map(&map_out, P));
   const size_t smem = sizeof(SharedStorage<BN>);
   REPQ_CUDA(cudaFuncSetAttribute(qgemm_tc_kernel<BN, OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
   const int tiles = ((P.M + BM - 1) / BM) * ((P.N + BN - 1) / BN);
   const int grid = tiles < sms ? tiles : sms;
-  qgemm_tc_kernel<BN, OUT><<<grid, kThreads, smem, st>>>(map_a, map_b, P);
+  qgemm_tc_kernel<BN, OUT><<<grid, kThreads, smem, st>>>(map_a, map_b, map_out, P);
   REPQ_CUDA(cudaGetLastError());
   note_launch();
   return REPQ_OK;
