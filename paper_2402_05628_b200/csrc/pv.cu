@@ -150,28 +150,45 @@ pv_kernel(PvParams P) {
     __syncthreads();
     {
       constexpr int kGroupsPerRow = kDhp / 8;              // 8 columns per work item
+      constexpr int kItems = kVKeys * kGroupsPerRow / kThreads;
       const int keys_here = min(kVKeys, (k_end - kv0 + kKeys - 1) / kKeys * kKeys);
-      for (int w = tid; w < keys_here * kGroupsPerRow; w += kThreads) {
+      const int n_items = keys_here * kGroupsPerRow;
+      // all loads of the thread are issued before the first conversion
+      uint2 raw[kItems];
+#pragma unroll
+      for (int i = 0; i < kItems; ++i) {
+        const int w = tid + i * kThreads;
+        const int kr = w / kGroupsPerRow, c0 = (w % kGroupsPerRow) * 8;
+        const int key = kv0 + kr;
+        raw[i] = make_uint2(0u, 0u);
+        if (w < n_items && key < P.Lk && c0 < P.d_h) {
+          const uint8_t* vr = v_base + int64_t(key) * P.ldv;
+          if (P.bits_v == 4) {
+            const uint8_t* s = vr + c0 / 2;
+            if ((reinterpret_cast<uintptr_t>(s) & 3) == 0 && c0 + 8 <= P.d_h) raw[i].x = __ldg(reinterpret_cast<const uint32_t*>(s));
+            else for (int e = 0; e < 4; ++e) if (c0 + 2 * e < P.d_h) raw[i].x |= uint32_t(s[e]) << (8 * e);
+          } else {
+            const uint8_t* s = vr + c0;
+            if ((reinterpret_cast<uintptr_t>(s) & 7) == 0 && c0 + 8 <= P.d_h) raw[i] = __ldg(reinterpret_cast<const uint2*>(s));
+            else for (int e = 0; e < 8; ++e) if (c0 + e < P.d_h) (e < 4 ? raw[i].x : raw[i].y) |= uint32_t(s[e]) << (8 * (e & 3));
+          }
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < kItems; ++i) {
+        const int w = tid + i * kThreads;
+        if (w >= n_items) continue;
         const int kr = w / kGroupsPerRow, c0 = (w % kGroupsPerRow) * 8;
         const int key = kv0 + kr;
         uint32_t o[4] = {0, 0, 0, 0};
         if (key < P.Lk && c0 < P.d_h) {
-          const uint8_t* vr = v_base + int64_t(key) * P.ldv;
           int q[8];
           if (P.bits_v == 4) {
-            uint32_t w4 = 0;
-            const uint8_t* s = vr + c0 / 2;
-            if ((reinterpret_cast<uintptr_t>(s) & 3) == 0 && c0 + 8 <= P.d_h) w4 = __ldg(reinterpret_cast<const uint32_t*>(s));
-            else for (int e = 0; e < 4; ++e) if (c0 + 2 * e < P.d_h) w4 |= uint32_t(s[e]) << (8 * e);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) q[e] = int((w4 >> (4 * e)) & 15u);
+            for (int e = 0; e < 8; ++e) q[e] = int((raw[i].x >> (4 * e)) & 15u);
           } else {
-            const uint8_t* s = vr + c0;
-            uint2 w8 = make_uint2(0, 0);
-            if ((reinterpret_cast<uintptr_t>(s) & 7) == 0 && c0 + 8 <= P.d_h) w8 = __ldg(reinterpret_cast<const uint2*>(s));
-            else for (int e = 0; e < 8; ++e) if (c0 + e < P.d_h) (e < 4 ? w8.x : w8.y) |= uint32_t(s[e]) << (8 * (e & 3));
 #pragma unroll
-            for (int e = 0; e < 4; ++e) { q[e] = int((w8.x >> (8 * e)) & 255u); q[4 + e] = int((w8.y >> (8 * e)) & 255u); }
+            for (int e = 0; e < 4; ++e) { q[e] = int((raw[i].x >> (8 * e)) & 255u); q[4 + e] = int((raw[i].y >> (8 * e)) & 255u); }
           }
 #pragma unroll
           for (int e = 0; e < 8; e += 2) {
@@ -194,6 +211,7 @@ pv_kernel(PvParams P) {
       // ---- 4 MMA k-steps of 16 keys; step s uses codes 4s..4s+3 of every thread
 #pragma unroll
       for (int s = 0; s < 4; ++s) {
+        if (k0 + 4 * s >= k_end) break;                     // every key of this step (k0 + 16 t + 4 s + i) is past the end
         // the 4 codes of this step, per row: 16 bits (4-bit codes) or 32 bits (byte codes)
         uint32_t qa, qb;
         if (kP4) {

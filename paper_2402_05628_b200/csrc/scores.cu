@@ -68,7 +68,7 @@ __device__ __forceinline__ void row_terms(const uint8_t* smem, int row_bytes, in
 }
 
 template <bool k4>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 3)
 scores_kernel(ScoresParams P) {
   __shared__ __align__(16) uint8_t sQ[kTile * kMaxRowBytes];
   __shared__ __align__(16) uint8_t sK[kTile * kMaxRowBytes];
