@@ -14,6 +14,7 @@ data path).
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import subprocess
@@ -82,6 +83,24 @@ class ClockSampler:
         sm.sort()
         med = sm[len(sm) // 2] if sm else None
         return dict(sm_mhz=med, sm_max_mhz=mx, reasons=sorted(reasons), samples=len(sm))
+
+
+def shard_rows(world: int, rank: int, batch_per_gpu: int, seq: int):
+    """Rows of the global batch (world * batch_per_gpu items) that rank `rank` owns: the path shards over the
+    batch with no exchange step, so a rank's shard is a contiguous block of whole batch items."""
+    rows = batch_per_gpu * seq
+    return rank * rows, (rank + 1) * rows
+
+
+def max_over_ranks(values, device, world: int):
+    """Element-wise MAX of a list of floats over all ranks (timings are reported as the slowest rank's)."""
+    if world == 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
 
 
 def stage_costs(cfg, batch):
@@ -178,12 +197,18 @@ def main():
     from paper_2402_05628_b200 import binding as B
     from paper_2402_05628_b200.engine import QuantBlock
 
-    w = make_block_inputs(args.workload, batch=args.batch)
-    cfg = w.cfg
-    batch, L = cfg["B"], cfg["L"]
+    from workloads import BLOCK_CONFIGS
+    batch = args.batch if args.batch is not None else BLOCK_CONFIGS[args.workload]["B"]
+    # replicated parameters, batch sharded over the ranks: generate the global batch, keep this rank's rows
+    w = make_block_inputs(args.workload, batch=batch * world)
+    cfg = dict(w.cfg)
+    cfg["B"] = batch
+    L = cfg["L"]
+    r0, r1 = shard_rows(world, rank, batch, L)
+    w = dataclasses.replace(w, cfg=cfg, x=w.x[r0:r1])
     tokens_per_step = batch * L
     blk = QuantBlock(w, device=dev)
-    x_host = torch.from_numpy(w.x).to(blk.act_dtype).pin_memory()
+    x_host = torch.from_numpy(np.ascontiguousarray(w.x)).to(blk.act_dtype).pin_memory()
     x = x_host.to(dev, non_blocking=True)
     y = torch.empty_like(x, dtype=blk.out_dtype)
     y_host = torch.empty(y.shape, dtype=y.dtype).pin_memory()
@@ -241,10 +266,7 @@ def main():
     stage_ms /= n_timed
     assert B.repq_device_status() == 0, "a bounded device-side wait gave up"
 
-    if world > 1:
-        t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, ms_e2e = float(t[0]), float(t[1])
+    ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], dev, world)
 
     if rank == 0:
         peaks = load_peaks()
@@ -285,7 +307,7 @@ def main():
         if world == 1 and not args.no_cpu_baseline:
             from threadpoolctl import threadpool_info
             from oracle import repq_oracle as orc
-            nb = min(batch, 32)
+            nb = max(1, min(batch, 32, 6400 // L))        # bounded sample: roughly 10-30 s of host work
             w_s = make_block_inputs(args.workload, batch=nb)
             orc.block_forward(make_block_inputs(args.workload, batch=1))
             t0 = time.perf_counter()

@@ -40,3 +40,13 @@ def test_block_c3_vit_l_sampled():
 def test_block_causal_8bit_log_codes_small():
     # LLaMA-shaped semantics (causal Softmax, 8-bit log codes, head dim 128) at a CPU-sized width
     parity.check_block("c4_llama7b", batch=2, D=512, H=4, MLP=1408, L=320, massive=2)
+
+
+def test_block_c3_full_batch_sampled_items():
+    parity.check_block("c3_vit_l", batch=32, sample_items=(0, 31))
+
+
+def test_block_c4_llama_shaped_full_size_sampled_item():
+    # full LLaMA-7B-shaped layer (batch 4 x 2048 tokens, dim 4096, MLP 11008, causal, 8-bit log codes);
+    # the oracle recomputes one batch item
+    parity.check_block("c4_llama7b", batch=4, sample_items=(3,))
