@@ -17,6 +17,10 @@
  *    the call returns without synchronising.
  *  - Codes are unsigned integers in [0, 2^b - 1] exactly as Eq. 4 produces them.  4-bit codes are
  *    packed two per byte (even index in the low nibble); 6- and 8-bit codes take one byte each.
+ *    Every `bits` argument or field may carry the flag REPQ_BYTE_CODES (e.g. 4 | REPQ_BYTE_CODES): the
+ *    quantizer is unchanged, but its codes are stored one per byte.  That is the operand format of
+ *    the 8-bit integer tensor-core instruction, so 4-bit tensors kept this way need no expansion pass
+ *    before a GEMM; the packed form is for storage and interchange.
  *    Code tensors are row-major with a row stride in BYTES; float tensors use strides in ELEMENTS.
  *  - Weights are stored [out features j, in features c] (row j is the paper's column W[:, j]).
  *  - Zero-points are plain integers of any sign (Eq. 6 does not bound them).
@@ -52,12 +56,14 @@ typedef int repq_status;
 
 #define REPQ_MAX_OUT_GROUPS 4
 
+#define REPQ_BYTE_CODES 0x100       /* OR into a `bits` value: one code per byte whatever the bit width */
+
 /* Copies the calling thread's last error message (NUL-terminated, truncated to n) and returns its
  * full length. */
 size_t repq_last_error(char* buf, size_t n);
 
 /* Library ABI version (bumped on any signature change). */
-int repq_abi_version(void);   /* currently 2 */
+int repq_abi_version(void);   /* currently 3 */
 
 /* ------------------------------------------------------------------------------------------------
  * One-time host-side preparation (not on the timed path)
@@ -216,7 +222,8 @@ typedef struct repq_linear_params {
 
 typedef struct repq_block_desc {
   int32_t batch, seq, dim, heads, mlp;
-  int32_t bits_a, bits_w, bits_p;
+  int32_t bits_a, bits_w, bits_p;       /* bits_w describes the layout of the w_codes given (it may carry
+                                           REPQ_BYTE_CODES); activation codes are internal and byte-wide */
   int32_t causal;
   int32_t norm_kind;
   float eps;

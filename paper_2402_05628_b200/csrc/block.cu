@@ -35,11 +35,15 @@ repq_status validate(const repq_block_desc& d) {
   return REPQ_OK;
 }
 
+// Activation codes between the stages are internal to the block: they are kept one per byte, the operand
+// format of the integer tensor-core instruction, whatever their bit width.
+inline int act_bits(const repq_block_desc& d) { return d.bits_a | REPQ_BYTE_CODES; }
+
 repq_gemm_desc linear_desc(const repq_block_desc& d, int64_t M, int N, int K, const uint8_t* a, int64_t lda,
                            float s_a, int z_a, const int32_t* asum, const repq_linear_params& w) {
   repq_gemm_desc g{};
   g.M = int32_t(M); g.N = N; g.K = K; g.batch_outer = g.batch_inner = 1;
-  g.a_codes = a; g.bits_a = d.bits_a; g.lda_bytes = lda; g.s_a = s_a; g.z_a = z_a; g.a_row_sum = asum;
+  g.a_codes = a; g.bits_a = act_bits(d); g.lda_bytes = lda; g.s_a = s_a; g.z_a = z_a; g.a_row_sum = asum;
   g.w_codes = w.w_codes; g.bits_w = d.bits_w; g.ldw_bytes = w.ldw_bytes; g.s_w = w.s_w; g.z_w = w.z_w;
   g.w_row_sum = w.w_row_sum; g.bias = w.bias; g.alpha = 1.f;
   g.out_groups = 1; g.out_scale[0] = 1.f;
@@ -49,9 +53,9 @@ repq_gemm_desc linear_desc(const repq_block_desc& d, int64_t M, int N, int K, co
 BlockLayout layout(const repq_block_desc& d) {
   BlockLayout L{};
   L.M = int64_t(d.batch) * d.seq;
-  L.ld_a = round_up(code_row_bytes(d.dim, d.bits_a), 16);
-  L.ld_qkv = round_up(code_row_bytes(3 * int64_t(d.dim), d.bits_a), 16);
-  L.ld_h = round_up(code_row_bytes(d.mlp, d.bits_a), 16);
+  L.ld_a = round_up(code_row_bytes(d.dim, act_bits(d)), 16);
+  L.ld_qkv = round_up(code_row_bytes(3 * int64_t(d.dim), act_bits(d)), 16);
+  L.ld_h = round_up(code_row_bytes(d.mlp, act_bits(d)), 16);
   L.ld_s = round_up(d.seq, 4);
   L.ld_p = round_up((int64_t(d.seq) + 7) / 8 * (d.bits_p == 4 ? 4 : 8), 16);
   const int64_t rows_s = int64_t(d.batch) * d.heads * d.seq;
@@ -72,9 +76,9 @@ BlockLayout layout(const repq_block_desc& d) {
   size_t ws = 0;
   const int shapes[4][2] = {{3 * d.dim, d.dim}, {d.dim, d.dim}, {d.mlp, d.dim}, {d.dim, d.mlp}};
   for (auto& s : shapes) {
-    repq_gemm_desc g = linear_desc(d, L.M, s[0], s[1], nullptr, code_row_bytes(s[1], d.bits_a), 1.f, 0, nullptr, none);
+    repq_gemm_desc g = linear_desc(d, L.M, s[0], s[1], nullptr, code_row_bytes(s[1], act_bits(d)), 1.f, 0, nullptr, none);
     g.ldw_bytes = round_up(code_row_bytes(s[1], d.bits_w), 16);
-    g.lda_bytes = round_up(code_row_bytes(s[1], d.bits_a), 16);
+    g.lda_bytes = round_up(code_row_bytes(s[1], act_bits(d)), 16);
     if (qgemm_tc_supported(g)) ws = ws > qgemm_tc_workspace(g) ? ws : qgemm_tc_workspace(g);
   }
   L.gemm_ws = ws;
@@ -110,7 +114,8 @@ static repq_status block_forward_impl(const repq_block_desc* dp, const repq_bloc
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int D = d.dim, H = d.heads, dh = D / H, S = d.seq;
   const int64_t M = L.M;
-  const int64_t head_bytes = code_row_bytes(dh, d.bits_a);          // bytes of one head's codes in a row
+  const int ab = act_bits(d);
+  const int64_t head_bytes = code_row_bytes(dh, ab);          // bytes of one head's codes in a row
 
   uint8_t* ln_c = ws + L.off_ln;
   int32_t* asum = reinterpret_cast<int32_t*>(ws + L.off_asum);
@@ -132,11 +137,11 @@ static repq_status block_forward_impl(const repq_block_desc* dp, const repq_bloc
 
   // ---- X_bar = MSA(LN(X)) + X
   REPQ_TRY(repq_ln_quant(x, d.act_dtype, M, D, D, p.ln1_gamma_t, p.ln1_beta_t, d.eps, d.norm_kind, p.ln1_s, p.ln1_z,
-                         d.bits_a, ln_c, L.ld_a, asum, stream));
+                         ab, ln_c, L.ld_a, asum, stream));
   REPQ_MARK();
   {
     repq_gemm_desc g = linear_desc(d, M, 3 * D, D, ln_c, L.ld_a, p.ln1_s, p.ln1_z, asum, p.qkv);
-    g.out_kind = REPQ_OUT_CODES; g.out_bits = d.bits_a; g.out_groups = 3;
+    g.out_kind = REPQ_OUT_CODES; g.out_bits = ab; g.out_groups = 3;
     g.out_scale[0] = p.s_q; g.out_scale[1] = p.s_k; g.out_scale[2] = p.s_v;
     g.out_zero[0] = p.z_q; g.out_zero[1] = p.z_k; g.out_zero[2] = p.z_v;
     g.out = qkv_c; g.ldo = L.ld_qkv;
@@ -147,10 +152,10 @@ static repq_status block_forward_impl(const repq_block_desc* dp, const repq_bloc
     // scores = Q K^T / sqrt(d_h) per (batch, head): both operands are activation codes
     repq_gemm_desc g{};
     g.M = S; g.N = S; g.K = dh; g.batch_outer = d.batch; g.batch_inner = H;
-    g.a_codes = qkv_c; g.bits_a = d.bits_a; g.lda_bytes = L.ld_qkv;
+    g.a_codes = qkv_c; g.bits_a = ab; g.lda_bytes = L.ld_qkv;
     g.a_stride_outer = int64_t(S) * L.ld_qkv; g.a_stride_inner = head_bytes;
     g.s_a = p.s_q; g.z_a = p.z_q;
-    g.w_codes = qkv_c + code_row_bytes(D, d.bits_a); g.bits_w = d.bits_a; g.ldw_bytes = L.ld_qkv;
+    g.w_codes = qkv_c + code_row_bytes(D, ab); g.bits_w = ab; g.ldw_bytes = L.ld_qkv;
     g.w_stride_outer = g.a_stride_outer; g.w_stride_inner = head_bytes;
     g.s_w_scalar = p.s_k; g.z_w_scalar = p.z_k;
     g.alpha = 1.f / sqrtf(float(dh));
@@ -170,10 +175,10 @@ static repq_status block_forward_impl(const repq_block_desc* dp, const repq_bloc
     v.batch_outer = d.batch; v.batch_inner = H; v.Lq = S; v.Lk = S; v.d_h = dh;
     v.p_codes = p_c; v.bits_p = d.bits_p; v.ldp_bytes = L.ld_p; v.p_stride_pair = int64_t(S) * L.ld_p;
     v.s_p = p.softmax_s;
-    v.v_codes = qkv_c + 2 * code_row_bytes(D, d.bits_a); v.bits_v = d.bits_a; v.ldv_bytes = L.ld_qkv;
+    v.v_codes = qkv_c + 2 * code_row_bytes(D, ab); v.bits_v = ab; v.ldv_bytes = L.ld_qkv;
     v.v_stride_outer = int64_t(S) * L.ld_qkv; v.v_stride_inner = head_bytes;
     v.s_v = p.s_v; v.z_v = p.z_v; v.causal = d.causal;
-    v.out_kind = REPQ_OUT_CODES; v.out_bits = d.bits_a; v.out_scale = p.s_attn; v.out_zero = p.z_attn;
+    v.out_kind = REPQ_OUT_CODES; v.out_bits = ab; v.out_scale = p.s_attn; v.out_zero = p.z_attn;
     v.out = attn_c; v.ldo = L.ld_a; v.o_stride_outer = int64_t(S) * L.ld_a; v.o_stride_inner = head_bytes;
     v.out_row_sum = asum_attn;
     REPQ_TRY(repq_pv(&v, stream));
@@ -189,13 +194,13 @@ static repq_status block_forward_impl(const repq_block_desc* dp, const repq_bloc
   REPQ_MARK();
   // ---- Y = MLP(LN(X_bar)) + X_bar
   REPQ_TRY(repq_ln_quant(xbar, d.act_dtype, M, D, D, p.ln2_gamma_t, p.ln2_beta_t, d.eps, d.norm_kind, p.ln2_s, p.ln2_z,
-                         d.bits_a, ln_c, L.ld_a, asum, stream));
+                         ab, ln_c, L.ld_a, asum, stream));
   REPQ_MARK();
   REPQ_CUDA(cudaMemsetAsync(asum_h, 0, size_t(M) * 4, st));
   {
     repq_gemm_desc g = linear_desc(d, M, d.mlp, D, ln_c, L.ld_a, p.ln2_s, p.ln2_z, asum, p.fc1);
     g.gelu = 1;
-    g.out_kind = REPQ_OUT_CODES; g.out_bits = d.bits_a; g.out_groups = 1;
+    g.out_kind = REPQ_OUT_CODES; g.out_bits = ab; g.out_groups = 1;
     g.out_scale[0] = p.s_hidden; g.out_zero[0] = p.z_hidden;
     g.out = hid_c; g.ldo = L.ld_h; g.out_row_sum = asum_h;
     REPQ_TRY(repq_qgemm(&g, gws, L.gemm_ws, stream));

@@ -40,8 +40,15 @@ inline repq_status fail(repq_status code, const char* fmt, ...) {
     if (s__ != REPQ_OK) return s__;      \
   } while (0)
 
-inline bool bits_ok(int b) { return b == 4 || b == 6 || b == 8; }
-inline int64_t code_row_bytes(int64_t n, int bits) { return bits == 4 ? (n + 1) / 2 : n; }
+// A `bits` value = quantizer width (4, 6, 8) | optional REPQ_BYTE_CODES.
+inline int quant_bits(int b) { return b & 0xFF; }
+inline bool bits_ok(int b) {
+  const int q = quant_bits(b);
+  return (b & ~(0xFF | REPQ_BYTE_CODES)) == 0 && (q == 4 || q == 6 || q == 8);
+}
+inline bool packed4(int b) { return b == 4; }                        // two codes per byte
+inline int code_max(int b) { return (1 << quant_bits(b)) - 1; }
+inline int64_t code_row_bytes(int64_t n, int bits) { return packed4(bits) ? (n + 1) / 2 : n; }
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 inline int64_t round_up(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
 

@@ -50,13 +50,13 @@ extern "C" size_t repq_last_error(char* buf, size_t n) {
   return m.size();
 }
 
-extern "C" int repq_abi_version(void) { return 2; }
+extern "C" int repq_abi_version(void) { return 3; }
 
 extern "C" repq_status repq_scale_zero_from_bounds(int n, const float* x_low, const float* x_up,
                                                    int bits, float* s, int32_t* z) {
   REPQ_REQUIRE(n > 0 && x_low && x_up && s && z, REPQ_INVALID_ARG, "scale_zero_from_bounds: bad argument");
   REPQ_REQUIRE(bits_ok(bits), REPQ_INVALID_ARG, "scale_zero_from_bounds: bits must be 4, 6 or 8");
-  const double qmax = double((1 << bits) - 1);
+  const double qmax = double(code_max(bits));
   for (int i = 0; i < n; ++i) {
     REPQ_REQUIRE(x_up[i] > x_low[i], REPQ_INVALID_ARG, "scale_zero_from_bounds: x_up <= x_low at %d", i);
     const float sf = float((double(x_up[i]) - double(x_low[i])) / qmax);
@@ -112,7 +112,7 @@ extern "C" repq_status repq_pack_weights(int N, int K, int bits_w, const float* 
   REPQ_REQUIRE(bits_ok(bits_w), REPQ_INVALID_ARG, "pack_weights: bits must be 4, 6 or 8");
   REPQ_REQUIRE(ld_codes_bytes >= code_row_bytes(K, bits_w) && ld_codes_bytes % 16 == 0, REPQ_ALIGNMENT,
                "pack_weights: ld_codes_bytes must cover a row and be a multiple of 16");
-  const int qmax = (1 << bits_w) - 1;
+  const int qmax = code_max(bits_w);
   std::vector<int32_t> row(K);
   for (int j = 0; j < N; ++j) {
     const float* wr = W + size_t(j) * K;
@@ -135,7 +135,7 @@ extern "C" repq_status repq_pack_weights(int N, int K, int bits_w, const float* 
     }
     uint8_t* out = codes + size_t(j) * ld_codes_bytes;
     memset(out, 0, size_t(ld_codes_bytes));
-    if (bits_w == 4) {
+    if (packed4(bits_w)) {
       for (int c = 0; c < K; ++c) out[c >> 1] |= uint8_t(row[c] << ((c & 1) * 4));
     } else {
       for (int c = 0; c < K; ++c) out[c] = uint8_t(row[c]);

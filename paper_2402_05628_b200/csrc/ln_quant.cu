@@ -226,9 +226,9 @@ repq_status launch(const T* x, int64_t rows, int D, int64_t ldx, const float* g,
   const int64_t cap = int64_t(sm_count()) * 8;
   const int grid = int(need < cap ? need : cap);
   const float inv_s = 1.f / s_t;
-  const int qmax = (1 << bits) - 1;
+  const int qmax = code_max(bits);
   const size_t smem = size_t(D) * 2 * sizeof(float);
-  auto kern = bits == 4 ? ln_quant_kernel<T, TPR, true> : ln_quant_kernel<T, TPR, false>;
+  auto kern = packed4(bits) ? ln_quant_kernel<T, TPR, true> : ln_quant_kernel<T, TPR, false>;
   if (smem > 48 * 1024) REPQ_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
   kern<<<grid, kBlock, smem, st>>>(x, rows, D, ldx, g, b, eps, rms, inv_s, z, qmax, codes, ldc, row_sum);
   REPQ_CUDA(cudaGetLastError());
@@ -276,7 +276,7 @@ extern "C" repq_status repq_ln_quant(const void* x, int x_dtype, int64_t rows, i
   REPQ_REQUIRE(ldx >= D, REPQ_INVALID_ARG, "ln_quant: ldx < D");
   const size_t esz = x_dtype == REPQ_F32 ? 4 : 2;
   REPQ_REQUIRE(aligned(x, 16) && (size_t(ldx) * esz) % 16 == 0, REPQ_ALIGNMENT, "ln_quant: x rows must be 16-byte aligned");
-  const int64_t unit = bits == 4 ? 4 : 8;
+  const int64_t unit = packed4(bits) ? 4 : 8;
   REPQ_REQUIRE(ld_codes_bytes >= code_row_bytes(D, bits), REPQ_INVALID_ARG, "ln_quant: ld_codes_bytes shorter than a row");
   REPQ_REQUIRE(aligned(codes, unit) && ld_codes_bytes % unit == 0, REPQ_ALIGNMENT,
                "ln_quant: codes rows must be %d-byte aligned", int(unit));

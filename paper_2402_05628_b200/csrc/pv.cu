@@ -332,7 +332,7 @@ extern "C" repq_status repq_pv(const repq_pv_desc* d, void* stream) {
                "pv: p rows must be 16-byte aligned");
   REPQ_REQUIRE(d->ldp_bytes >= code_row_bytes(d->Lk, d->bits_p), REPQ_INVALID_ARG, "pv: ldp_bytes shorter than a row");
   REPQ_REQUIRE(d->ldv_bytes >= code_row_bytes(d->d_h, d->bits_v), REPQ_INVALID_ARG, "pv: ldv_bytes shorter than a row");
-  const int qmax_v = (1 << d->bits_v) - 1;
+  const int qmax_v = code_max(d->bits_v);
   REPQ_REQUIRE(d->z_v >= qmax_v - 256 && d->z_v <= 256, REPQ_UNSUPPORTED,
                "pv: z_v = %d puts v - z_v outside the exactly representable range [-256, 256]", d->z_v);
   REPQ_REQUIRE(!d->causal || d->Lk >= d->Lq, REPQ_INVALID_ARG, "pv: causal needs Lk >= Lq");
@@ -341,19 +341,19 @@ extern "C" repq_status repq_pv(const repq_pv_desc* d, void* stream) {
   REPQ_REQUIRE(pairs <= 65535, REPQ_UNSUPPORTED, "pv: more than 65535 (batch, head) pairs");
   PvParams P{};
   P.p = d->p_codes; P.bits_p = d->bits_p; P.ldp = d->ldp_bytes; P.p_pair = d->p_stride_pair;
-  P.v = d->v_codes; P.bits_v = d->bits_v; P.ldv = d->ldv_bytes; P.v_so = d->v_stride_outer; P.v_si = d->v_stride_inner;
+  P.v = d->v_codes; P.bits_v = packed4(d->bits_v) ? 4 : 8; P.ldv = d->ldv_bytes; P.v_so = d->v_stride_outer; P.v_si = d->v_stride_inner;
   P.Lq = d->Lq; P.Lk = d->Lk; P.d_h = d->d_h; P.batch_inner = d->batch_inner; P.causal = d->causal;
   P.z_v = d->z_v; P.scale = d->s_p * d->s_v;
   P.out_kind = d->out_kind;
   if (d->out_kind == REPQ_OUT_CODES) {
     REPQ_REQUIRE(bits_ok(d->out_bits) && d->out_scale > 0.f, REPQ_INVALID_ARG, "pv: bad output quantizer");
     REPQ_REQUIRE(d->out_zero > -(1 << 20) && d->out_zero < (1 << 20), REPQ_INVALID_ARG, "pv: |out_zero| must be below 2^20");
-    P.qmax = (1 << d->out_bits) - 1; P.pack4 = d->out_bits == 4; P.inv_so = 1.f / d->out_scale; P.zo = d->out_zero;
+    P.qmax = code_max(d->out_bits); P.pack4 = packed4(d->out_bits); P.inv_so = 1.f / d->out_scale; P.zo = d->out_zero;
   }
   P.out = d->out; P.ldo = d->ldo; P.o_so = d->o_stride_outer; P.o_si = d->o_stride_inner;
   P.out_row_sum = d->out_kind == REPQ_OUT_CODES ? d->out_row_sum : nullptr;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const bool p4 = d->bits_p == 4;
+  const bool p4 = packed4(d->bits_p);
   if (d->d_h <= 64) return p4 ? launch_pv<1, true>(P, pairs, st) : launch_pv<1, false>(P, pairs, st);
   return p4 ? launch_pv<2, true>(P, pairs, st) : launch_pv<2, false>(P, pairs, st);
 }

@@ -99,7 +99,7 @@ repq_status validate(const repq_gemm_desc& d) {
       REPQ_REQUIRE(d.out_zero[g] > -(1 << 20) && d.out_zero[g] < (1 << 20), REPQ_INVALID_ARG, "qgemm: |out_zero| must be below 2^20");
     }
     REPQ_REQUIRE(d.ldo >= code_row_bytes(d.N, d.out_bits), REPQ_INVALID_ARG, "qgemm: ldo shorter than a row of codes");
-    if (d.out_bits == 4) REPQ_REQUIRE((d.N / d.out_groups) % 2 == 0, REPQ_UNSUPPORTED, "qgemm: 4-bit output groups must have even width");
+    if (packed4(d.out_bits)) REPQ_REQUIRE((d.N / d.out_groups) % 2 == 0, REPQ_UNSUPPORTED, "qgemm: 4-bit output groups must have even width");
   } else {
     REPQ_REQUIRE(d.ldo >= d.N, REPQ_INVALID_ARG, "qgemm: ldo < N");
     const size_t esz = d.out_kind == REPQ_OUT_F32 ? 4 : 2;
@@ -122,8 +122,8 @@ EpilogueParams make_epilogue(const repq_gemm_desc& d) {
   ep.residual = d.residual; ep.residual_bf16 = d.residual_dtype == REPQ_BF16; ep.ld_residual = d.ld_residual;
   ep.out_kind = d.out_kind;
   const bool codes = d.out_kind == REPQ_OUT_CODES;
-  ep.qmax = codes ? (1 << d.out_bits) - 1 : 0;
-  ep.pack4 = codes && d.out_bits == 4;
+  ep.qmax = codes ? code_max(d.out_bits) : 0;
+  ep.pack4 = codes && packed4(d.out_bits);
   ep.group_width = codes ? d.N / d.out_groups : d.N;
   for (int g = 0; g < REPQ_MAX_OUT_GROUPS; ++g) {
     const bool on = codes && g < d.out_groups;
@@ -143,7 +143,7 @@ repq_status launch_row_sum(const uint8_t* codes, int bits, int64_t rows, int64_t
   if (rows == 0) return REPQ_OK;
   const int64_t blocks = (rows + 7) / 8;
   const int grid = int(blocks < 4096 ? blocks : 4096);
-  row_sum_kernel<<<grid, 256, 0, st>>>(codes, bits, rows, n, ld_bytes, out);
+  row_sum_kernel<<<grid, 256, 0, st>>>(codes, packed4(bits) ? 4 : 8, rows, n, ld_bytes, out);
   REPQ_CUDA(cudaGetLastError());
   note_launch();
   return REPQ_OK;

@@ -204,10 +204,10 @@ qgemm_mma_kernel(MmaOperand A, MmaOperand W, int K, int batch_inner, int64_t a_s
 }  // namespace
 
 repq_status qgemm_mma(const repq_gemm_desc& d, const EpilogueParams& ep, cudaStream_t st) {
-  MmaOperand A{d.a_codes, d.lda_bytes, d.M, d.bits_a};
-  MmaOperand W{d.w_codes, d.ldw_bytes, d.N, d.bits_w};
+  MmaOperand A{d.a_codes, d.lda_bytes, d.M, packed4(d.bits_a) ? 4 : 8};
+  MmaOperand W{d.w_codes, d.ldw_bytes, d.N, packed4(d.bits_w) ? 4 : 8};
   auto al = [](const uint8_t* p, int64_t ld, int64_t so, int64_t si, int bits) {
-    const int64_t unit = bits == 4 ? 2 : 4;
+    const int64_t unit = packed4(bits) ? 2 : 4;
     return aligned(p, size_t(unit)) && ld % unit == 0 && so % unit == 0 && si % unit == 0;
   };
   const bool a_al = al(d.a_codes, d.lda_bytes, d.a_stride_outer, d.a_stride_inner, d.bits_a);

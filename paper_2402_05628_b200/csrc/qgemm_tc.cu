@@ -594,8 +594,8 @@ TcLayout tc_layout(const repq_gemm_desc& d) {
   auto bump = [&](size_t bytes) { size_t at = cur; cur += (bytes + 255) / 256 * 256; return at; };
   L.ld_a = round_up(d.K, 16);
   L.ld_w = round_up(d.K, 16);
-  L.off_a = d.bits_a == 4 ? bump(size_t(d.M) * L.ld_a) : 0;
-  L.off_w = d.bits_w == 4 ? bump(size_t(d.N) * L.ld_w) : 0;
+  L.off_a = packed4(d.bits_a) ? bump(size_t(d.M) * L.ld_a) : 0;
+  L.off_w = packed4(d.bits_w) ? bump(size_t(d.N) * L.ld_w) : 0;
   L.off_asum = d.a_row_sum ? 0 : bump(size_t(d.M) * 4);
   L.off_wsum = d.w_row_sum ? 0 : bump(size_t(d.N) * 4);
   L.total = cur;
@@ -677,8 +677,8 @@ bool qgemm_tc_supported(const repq_gemm_desc& d) {
   if (disabled) return false;
   if (d.batch_outer != 1 || d.batch_inner != 1) return false;
   if (d.M < 64 || d.N < 64 || d.K < 64) return false;           // tiny problems: the warp-MMA kernel
-  if (d.bits_a != 4 && !(aligned(d.a_codes, 16) && d.lda_bytes % 16 == 0)) return false;
-  if (d.bits_w != 4 && !(aligned(d.w_codes, 16) && d.ldw_bytes % 16 == 0)) return false;
+  if (!packed4(d.bits_a) && !(aligned(d.a_codes, 16) && d.lda_bytes % 16 == 0)) return false;
+  if (!packed4(d.bits_w) && !(aligned(d.w_codes, 16) && d.ldw_bytes % 16 == 0)) return false;
   const int64_t obytes = d.out_kind == REPQ_OUT_F32 ? 4 : d.out_kind == REPQ_OUT_BF16 ? 2 : 1;
   if (!aligned(d.out, 16) || (d.ldo * obytes) % 16 != 0) return false;
   if (d.out_kind == REPQ_OUT_CODES && (d.N / d.out_groups) % kChunk != 0) return false;   // one quantizer per 16-column chunk
@@ -698,13 +698,13 @@ repq_status qgemm_tc(const repq_gemm_desc& d, const EpilogueParams& ep, void* ws
   uint8_t* w8 = static_cast<uint8_t*>(ws);
   const uint8_t* a = d.a_codes;
   int64_t lda = d.lda_bytes;
-  if (d.bits_a == 4) {
+  if (packed4(d.bits_a)) {
     REPQ_TRY(launch_expand4(d.a_codes, d.M, d.K, d.lda_bytes, w8 + L.off_a, L.ld_a, L.ld_a, st));
     a = w8 + L.off_a; lda = L.ld_a;
   }
   const uint8_t* w = d.w_codes;
   int64_t ldw = d.ldw_bytes;
-  if (d.bits_w == 4) {
+  if (packed4(d.bits_w)) {
     REPQ_TRY(launch_expand4(d.w_codes, d.N, d.K, d.ldw_bytes, w8 + L.off_w, L.ld_w, L.ld_w, st));
     w = w8 + L.off_w; ldw = L.ld_w;
   }

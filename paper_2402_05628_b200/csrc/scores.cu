@@ -160,7 +160,7 @@ bool scores_supported(const repq_gemm_desc& d) {
   if (d.s_w || d.z_w || d.bias || d.gelu || d.residual || d.acc_debug || d.out_row_sum) return false;
   if (d.out_kind != REPQ_OUT_F32) return false;
   if (d.K > 128 || d.K % 16 != 0) return false;
-  const bool both4 = d.bits_a == 4 && d.bits_w == 4, both8 = d.bits_a != 4 && d.bits_w != 4;
+  const bool both4 = packed4(d.bits_a) && packed4(d.bits_w), both8 = !packed4(d.bits_a) && !packed4(d.bits_w);
   if (!both4 && !both8) return false;
   const int64_t unit = both4 ? 8 : 16;
   auto ok = [&](const uint8_t* p, int64_t ld, int64_t so, int64_t si) {
@@ -183,7 +183,7 @@ repq_status launch_scores(const repq_gemm_desc& d, cudaStream_t st) {
   P.out = static_cast<float*>(d.out); P.ldo = d.ldo; P.o_so = d.o_stride_outer; P.o_si = d.o_stride_inner;
   P.causal = d.causal;
   dim3 grid((d.M + kTile - 1) / kTile, unsigned(int64_t(d.batch_outer) * d.batch_inner));
-  if (d.bits_a == 4) scores_kernel<true><<<grid, kThreads, 0, st>>>(P);
+  if (packed4(d.bits_a)) scores_kernel<true><<<grid, kThreads, 0, st>>>(P);
   else scores_kernel<false><<<grid, kThreads, 0, st>>>(P);
   REPQ_CUDA(cudaGetLastError());
   note_launch();

@@ -178,8 +178,8 @@ repq_status launch(const T* scores, int64_t rows, int L, int64_t ld, bool vec_ok
   const int64_t need = (rows + kRowsPerBlock - 1) / kRowsPerBlock;
   const int64_t cap = int64_t(sm_count()) * 8;
   const int grid = int(need < cap ? need : cap);
-  const int qmax = (1 << bits) - 1;
-  if (bits == 4)
+  const int qmax = code_max(bits);
+  if (packed4(bits))
     softmax_log2_kernel<T, TPR, true><<<grid, kBlock, 0, st>>>(scores, rows, L, ld, vec_ok, c, period, offset, log2_s, qmax, codes, ldc);
   else
     softmax_log2_kernel<T, TPR, false><<<grid, kBlock, 0, st>>>(scores, rows, L, ld, vec_ok, c, period, offset, log2_s, qmax, codes, ldc);
@@ -222,7 +222,7 @@ extern "C" repq_status repq_softmax_log2(const void* scores, int dtype, int64_t 
   REPQ_REQUIRE(ld >= L, REPQ_INVALID_ARG, "softmax_log2: ld < L");
   REPQ_REQUIRE(causal_period >= 0, REPQ_INVALID_ARG, "softmax_log2: causal_period must be >= 0");
   REPQ_REQUIRE(L <= 16384, REPQ_UNSUPPORTED, "softmax_log2: L = %d exceeds 16384", L);
-  const int64_t unit = bits == 4 ? 4 : 8;
+  const int64_t unit = packed4(bits) ? 4 : 8;
   const int64_t need = (int64_t(L) + 7) / 8 * unit;
   REPQ_REQUIRE(ld_codes_bytes >= need, REPQ_INVALID_ARG,
                "softmax_log2: ld_codes_bytes = %lld, need at least %lld (rows are written in groups of 8 codes)",

@@ -46,7 +46,9 @@ class QuantBlock:
         self.cfg = cfg
         dev = torch.device(device)
         self.device = dev
-        ba, bw = cfg["bits_a"], cfg["bits_w"]
+        ba = cfg["bits_a"]
+        # weights live on the device one code per byte: the tensor-core operand format, so no per-call expansion
+        bw = self.bits_w = cfg["bits_w"] | B.REPQ_BYTE_CODES
         self.host: Dict[str, object] = {}
 
         def fold(gamma, beta, lo, hi, W, b, tag):
@@ -78,7 +80,7 @@ class QuantBlock:
         c = self.cfg
         d = B.BlockDesc()
         d.batch, d.seq, d.dim, d.heads, d.mlp = batch, c["L"], c["D"], c["H"], c["MLP"]
-        d.bits_a, d.bits_w, d.bits_p = c["bits_a"], c["bits_w"], c["bits_p"]
+        d.bits_a, d.bits_w, d.bits_p = c["bits_a"], self.bits_w, c["bits_p"]
         d.causal, d.norm_kind, d.eps = int(c["causal"]), B.REPQ_NORM_LAYERNORM, c["eps"]
         d.act_dtype = B.REPQ_F32 if self.act_dtype == torch.float32 else B.REPQ_BF16
         d.out_dtype = B.REPQ_F32 if self.out_dtype == torch.float32 else B.REPQ_BF16

@@ -10,6 +10,14 @@ REL_L2_TOL = 2e-3          # float outputs: relative L2 error
 MAX_ABS_TOL = 1e-2         # float outputs: max abs error as a fraction of max |ref|
 
 
+BYTE_CODES = 0x100         # flag of the C ABI: a `bits` value with it set stores one code per byte
+
+
+def qb(bits: int) -> int:
+    """Quantizer width of a `bits` value (the flag only changes the storage)."""
+    return bits & 0xFF
+
+
 def unpack_codes(raw: np.ndarray, n: int, bits: int) -> np.ndarray:
     """raw: uint8 [rows, ld_bytes] -> int64 [rows, n] (4-bit: low nibble = even index)."""
     raw = np.asarray(raw, dtype=np.uint8)
@@ -103,8 +111,8 @@ def check_ln_quant(rows, D, bits, bf16, seed=0, rms=False, eps=1e-6, pad_cols=0,
     x, gamma, beta, lo, hi = ln_case(rows, D, bf16, seed, rms, eps)
     # oracle: complex (channel-wise) quantizer
     X1 = orc.layernorm(x, gamma, beta, eps, rms)
-    s, z = orc.uniform_scale_zero(lo, hi, bits)
-    q_ref, t_cw = orc.quant_uniform(X1, s[None, :], z[None, :], bits)
+    s, z = orc.uniform_scale_zero(lo, hi, qb(bits))
+    q_ref, t_cw = orc.quant_uniform(X1, s[None, :], z[None, :], qb(bits))
     # CUDA path: folded parameters, layer-wise quantizer
     W = np.zeros((1, D), dtype=np.float32)
     gamma_t, beta_t, s_t, z_t, _, _ = B.repq_fold_ln(gamma, beta, s.astype(np.float32), z.astype(np.int32), W, None)
@@ -150,7 +158,7 @@ def check_softmax_log2(rows, L, bits, bf16=False, seed=0, s=1.0, causal_period=0
     if causal_period:
         valid = np.minimum(L, (np.arange(rows) % causal_period) + 1)
     A = orc.softmax_rows(S.astype(np.float64) * np.float64(np.float32(pre_scale)), valid)
-    q_ref, t_ref = orc.quant_logsqrt2(A, s, bits)
+    q_ref, t_ref = orc.quant_logsqrt2(A, s, qb(bits))
     dev = torch.device("cuda:0")
     ld = ld_pad if ld_pad is not None else (L + 3) // 4 * 4
     buf = torch.zeros(rows, ld, dtype=torch.float32, device=dev)
@@ -166,7 +174,7 @@ def check_softmax_log2(rows, L, bits, bf16=False, seed=0, s=1.0, causal_period=0
     delta = 2.0 ** -18 * np.maximum(1.0, np.abs(np.where(np.isfinite(t_ref), t_ref, 0.0)))
     if valid is not None:
         mask = np.arange(L)[None, :] < valid[:, None]
-        assert np.all(q_gpu[~mask] == 2 ** bits - 1)
+        assert np.all(q_gpu[~mask] == 2 ** qb(bits) - 1)
         q_gpu = np.where(mask, q_gpu, 0)
         q_ref = np.where(mask, q_ref, 0)
     return near_tie_report(q_gpu, q_ref, t_ref, delta)
@@ -190,7 +198,7 @@ def check_qgemm(M, N, K, bits_a, bits_w, out_kind="f32", gelu=False, residual=No
     from workloads.kernels import gemm_codes, to_bf16_grid
 
     rng = np.random.default_rng(seed)
-    a, w, s_a, z_a, s_w, z_w, bias = gemm_codes(rng, M, N, K, bits_a, bits_w)
+    a, w, s_a, z_a, s_w, z_w, bias = gemm_codes(rng, M, N, K, qb(bits_a), qb(bits_w))
     res = None
     if residual is not None:
         res = rng.normal(0, 1.0, size=(M, N)).astype(np.float32)
@@ -212,7 +220,7 @@ def check_qgemm(M, N, K, bits_a, bits_w, out_kind="f32", gelu=False, residual=No
         gw = N // groups
         lo = [np.percentile(v_ref[:, g * gw:(g + 1) * gw], 1) for g in range(groups)]
         hi = [np.percentile(v_ref[:, g * gw:(g + 1) * gw], 99) for g in range(groups)]
-        s_o, z_o = orc.uniform_scale_zero(np.array(lo), np.array(hi), out_bits)
+        s_o, z_o = orc.uniform_scale_zero(np.array(lo), np.array(hi), qb(out_bits))
         ldo = B.code_row_bytes(N, out_bits)
         out = torch.full((M, ldo), 0xEE, dtype=torch.uint8, device=dev)
         kw = dict(out_kind=B.REPQ_OUT_CODES, out_bits=out_bits, out_scale=[float(v) for v in s_o],
@@ -251,7 +259,7 @@ def check_qgemm(M, N, K, bits_a, bits_w, out_kind="f32", gelu=False, residual=No
         rep = dict(total=0, mismatch=0, excused=0, bad=0)
         for g in range(groups):
             sl = slice(g * gw, (g + 1) * gw)
-            q_ref, t_ref = orc.quant_uniform(v_ref[:, sl], s_o[g], z_o[g], out_bits)
+            q_ref, t_ref = orc.quant_uniform(v_ref[:, sl], s_o[g], z_o[g], qb(out_bits))
             mag = np.abs(v_pre[:, sl] - bias[None, sl]) + np.abs(bias[None, sl]) + np.abs(v_ref[:, sl])
             if res is not None:
                 mag = mag + np.abs(res[:, sl])
@@ -292,11 +300,11 @@ def check_pv(B_, H, Lq, Lk, dh, bits_p, bits_v, causal=False, out_kind="f32", ou
     valid = np.minimum(Lk, np.arange(Lq) + 1 + shift) if causal else None
     S = softmax_logits(rng, pairs * Lq, Lk)
     A = orc.softmax_rows(S, None if valid is None else np.tile(valid, pairs))
-    p, _ = orc.quant_logsqrt2(A, s_p, bits_p)                        # [pairs*Lq, Lk]
+    p, _ = orc.quant_logsqrt2(A, s_p, qb(bits_p))                        # [pairs*Lq, Lk]
     D = H * dh
-    Vc = rng.integers(0, 1 << bits_v, size=(B_ * Lk, D))
+    Vc = rng.integers(0, 1 << qb(bits_v), size=(B_ * Lk, D))
     s_v = 0.05
-    z_v = int(rng.integers(0, 1 << bits_v))
+    z_v = int(rng.integers(0, 1 << qb(bits_v)))
     A_hat = orc.dequant_logsqrt2(p, s_p)
     if causal:
         A_hat = np.where(np.arange(Lk)[None, :] < np.tile(valid, pairs)[:, None], A_hat, 0.0)
@@ -319,7 +327,7 @@ def check_pv(B_, H, Lq, Lk, dh, bits_p, bits_v, causal=False, out_kind="f32", ou
     d.s_v, d.z_v, d.causal = s_v, z_v, int(causal)
     row_sum = None
     if out_kind == "codes":
-        s_o, z_o = orc.uniform_scale_zero(np.percentile(O_ref, 1), np.percentile(O_ref, 99), out_bits)
+        s_o, z_o = orc.uniform_scale_zero(np.percentile(O_ref, 1), np.percentile(O_ref, 99), qb(out_bits))
         ldo = B.code_row_bytes(D, out_bits)
         out = torch.full((B_ * Lq, ldo), 0xEE, dtype=torch.uint8, device=dev)
         d.out_kind, d.out_bits, d.out_scale, d.out_zero = B.REPQ_OUT_CODES, out_bits, float(s_o), int(z_o)
@@ -337,7 +345,7 @@ def check_pv(B_, H, Lq, Lk, dh, bits_p, bits_v, causal=False, out_kind="f32", ou
     torch.cuda.synchronize()
     if out_kind == "codes":
         q_gpu = unpack_codes(out.cpu().numpy(), D, out_bits)
-        q_ref, t_ref = orc.quant_uniform(O_ref, s_o, z_o, out_bits)
+        q_ref, t_ref = orc.quant_uniform(O_ref, s_o, z_o, qb(out_bits))
         absO = np.empty_like(O_ref)
         for b in range(B_):
             for h in range(H):
@@ -399,10 +407,10 @@ def check_scores(B_, H, Lq, Lk, dh, bits, causal=False, seed=0):
 
     rng = np.random.default_rng(seed)
     D = H * dh
-    Qc = rng.integers(0, 1 << bits, size=(B_ * Lq, D))
-    Kc = rng.integers(0, 1 << bits, size=(B_ * Lk, D))
+    Qc = rng.integers(0, 1 << qb(bits), size=(B_ * Lq, D))
+    Kc = rng.integers(0, 1 << qb(bits), size=(B_ * Lk, D))
     s_q, s_k = 0.37, 0.21
-    z_q, z_k = int(rng.integers(0, 1 << bits)), int(rng.integers(0, 1 << bits))
+    z_q, z_k = int(rng.integers(0, 1 << qb(bits))), int(rng.integers(0, 1 << qb(bits)))
     Qh, Kh = orc.dequant_uniform(Qc, s_q, z_q), orc.dequant_uniform(Kc, s_k, z_k)
     dev = torch.device("cuda:0")
     ld = B.code_row_bytes(D, bits)

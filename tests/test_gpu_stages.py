@@ -88,3 +88,17 @@ def test_pv_epilogues():
 ])
 def test_scores_match_oracle(Bn, H, Lq, Lk, dh, bits, causal):
     parity.check_scores(Bn, H, Lq, Lk, dh, bits, causal, seed=Lq + dh)
+
+
+def test_four_bit_quantizers_stored_one_code_per_byte():
+    """REPQ_BYTE_CODES changes the storage of the codes, not the quantizer: same oracle, byte-wide containers."""
+    b4 = 4 | parity.BYTE_CODES
+    assert parity.check_ln_quant(515, 768, b4, True, seed=11)["bad"] == 0
+    assert parity.check_softmax_log2(300, 197, b4, seed=12)["bad"] == 0
+    parity.check_qgemm(300, 192, 256, b4, b4, out_kind="codes", groups=3, out_bits=b4, seed=13)
+    parity.check_qgemm(197, 1152, 384, b4, 4, out_kind="codes", out_bits=b4, want_out_sum=True, gelu=True, seed=14)
+    parity.check_qgemm(130, 72, 100, 4, b4, seed=15)
+    parity.check_pv(2, 2, 197, 197, 64, 4, b4, out_kind="codes", out_bits=b4, want_out_sum=True, seed=16)
+    parity.check_pv(1, 2, 130, 130, 128, b4, b4, causal=True, seed=17)
+    parity.check_scores(2, 3, 197, 197, 64, b4, seed=18)
+    parity.check_scores(1, 2, 50, 50, 24, b4, seed=19)
