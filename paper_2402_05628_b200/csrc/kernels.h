@@ -26,6 +26,23 @@ size_t qgemm_tc_workspace(const repq_gemm_desc& d);
 repq_status qgemm_tc(const repq_gemm_desc& d, const EpilogueParams& ep, void* ws, size_t ws_bytes,
                      cudaStream_t st);
 
+// P.V (Eqs. 16-17): kernel parameters shared by the two implementations, storage widths already resolved
+// (bits_v is 4 for packed codes, 8 for byte codes).
+struct PvParams {
+  const uint8_t* p; int bits_p; int64_t ldp, p_pair;
+  const uint8_t* v; int bits_v; int64_t ldv, v_so, v_si;
+  int Lq, Lk, d_h, batch_inner, causal;
+  int z_v;
+  float scale;               // s_p * s_v
+  int out_kind, qmax, pack4;
+  float inv_so; int zo;
+  void* out; int64_t ldo, o_so, o_si;
+  int32_t* out_row_sum;
+};
+// Tensor-memory (tcgen05) P.V kernel: needs V rows that allow vector loads; the warp-MMA kernel covers the rest.
+bool pv_tc_supported(const repq_pv_desc& d);
+repq_status launch_pv_tc(const repq_pv_desc& d, const PvParams& P, cudaStream_t st);
+
 // Device-side health word (bounded waits report here instead of trapping); nullptr on failure.
 int32_t* device_status_word();
 

@@ -25,18 +25,6 @@ constexpr int kKeys = 64;       // keys per MMA chunk
 constexpr int kVKeys = 256;     // keys of V resident in shared memory
 constexpr int kThreads = 256;
 
-struct PvParams {
-  const uint8_t* p; int bits_p; int64_t ldp, p_pair;
-  const uint8_t* v; int bits_v; int64_t ldv, v_so, v_si;
-  int Lq, Lk, d_h, batch_inner, causal;
-  int z_v;
-  float scale;               // s_p * s_v
-  int out_kind, qmax, pack4;
-  float inv_so; int zo;
-  void* out; int64_t ldo, o_so, o_si;
-  int32_t* out_row_sum;
-};
-
 __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
   asm volatile(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
@@ -337,6 +325,8 @@ extern "C" repq_status repq_pv(const repq_pv_desc* d, void* stream) {
                "pv: z_v = %d puts v - z_v outside the exactly representable range [-256, 256]", d->z_v);
   REPQ_REQUIRE(!d->causal || d->Lk >= d->Lq, REPQ_INVALID_ARG, "pv: causal needs Lk >= Lq");
   REPQ_REQUIRE(d->out_kind == REPQ_OUT_F32 || d->out_kind == REPQ_OUT_BF16 || d->out_kind == REPQ_OUT_CODES, REPQ_INVALID_ARG, "pv: unknown out_kind");
+  REPQ_REQUIRE(aligned(d->out, d->out_kind == REPQ_OUT_F32 ? 4 : d->out_kind == REPQ_OUT_BF16 ? 2 : 1), REPQ_ALIGNMENT,
+               "pv: out is not element-aligned");
   const int64_t pairs = int64_t(d->batch_outer) * d->batch_inner;
   REPQ_REQUIRE(pairs <= 65535, REPQ_UNSUPPORTED, "pv: more than 65535 (batch, head) pairs");
   PvParams P{};
@@ -353,6 +343,7 @@ extern "C" repq_status repq_pv(const repq_pv_desc* d, void* stream) {
   P.out = d->out; P.ldo = d->ldo; P.o_so = d->o_stride_outer; P.o_si = d->o_stride_inner;
   P.out_row_sum = d->out_kind == REPQ_OUT_CODES ? d->out_row_sum : nullptr;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (pv_tc_supported(*d)) return launch_pv_tc(*d, P, st);
   const bool p4 = packed4(d->bits_p);
   if (d->d_h <= 64) return p4 ? launch_pv<1, true>(P, pairs, st) : launch_pv<1, false>(P, pairs, st);
   return p4 ? launch_pv<2, true>(P, pairs, st) : launch_pv<2, false>(P, pairs, st);

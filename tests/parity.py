@@ -439,3 +439,51 @@ def check_scores(B_, H, Lq, Lk, dh, bits, causal=False, seed=0):
             worst = max(worst, rel)
     assert worst < 1e-5
     return worst
+
+
+def check_pv_uniform_codes(B_, H, L, dh, bits_p, bits_v, runs=10, seed=0):
+    """repq_pv on uniformly random Softmax codes (every key carries weight, so a single misplaced tile row
+    shows), launched `runs` times: every launch must reproduce the oracle and the first launch bit for bit."""
+    import torch
+    from oracle import repq_oracle as orc
+    from paper_2402_05628_b200 import binding as B
+
+    rng = np.random.default_rng(seed)
+    D = H * dh
+    p = rng.integers(0, 1 << qb(bits_p), size=(B_ * H * L, L))
+    Vc = rng.integers(0, 1 << qb(bits_v), size=(B_ * L, D))
+    s_p, s_v = 0.9, 0.05
+    z_v = int(rng.integers(0, 1 << qb(bits_v)))
+    A_hat = orc.dequant_logsqrt2(p, s_p)
+    V_hat = orc.dequant_uniform(Vc, s_v, z_v)
+    O_ref = np.empty((B_ * L, D))
+    for b in range(B_):
+        for h in range(H):
+            pr = (b * H + h) * L
+            O_ref[b * L:(b + 1) * L, h * dh:(h + 1) * dh] = A_hat[pr:pr + L] @ V_hat[b * L:(b + 1) * L, h * dh:(h + 1) * dh]
+    dev = torch.device("cuda:0")
+    ldp, ldv = B.code_row_bytes(L, bits_p), B.code_row_bytes(D, bits_v)
+    p_t = torch.from_numpy(pack_codes(p, bits_p, ldp)).to(dev)
+    v_t = torch.from_numpy(pack_codes(Vc, bits_v, ldv)).to(dev)
+    out = torch.zeros(B_ * L, D, dtype=torch.float32, device=dev)
+    d = B.PvDesc()
+    d.batch_outer, d.batch_inner, d.Lq, d.Lk, d.d_h = B_, H, L, L, dh
+    d.p_codes, d.bits_p, d.ldp_bytes, d.p_stride_pair, d.s_p = p_t.data_ptr(), bits_p, ldp, L * ldp, s_p
+    d.v_codes, d.bits_v, d.ldv_bytes = v_t.data_ptr(), bits_v, ldv
+    d.v_stride_outer, d.v_stride_inner = L * ldv, (dh // 2 if bits_v == 4 else dh)
+    d.s_v, d.z_v, d.causal = s_v, z_v, 0
+    d.out_kind = B.REPQ_OUT_F32
+    d.ldo, d.o_stride_outer, d.o_stride_inner = D, L * D, dh
+    d.out = out.data_ptr()
+    first = None
+    for _ in range(runs):
+        out.zero_()
+        B.repq_pv(d)
+        torch.cuda.synchronize()
+        got = out.cpu().numpy()
+        rel, _ = assert_float_close(got, O_ref, "pv, uniform codes")
+        assert rel < 1e-5, rel
+        if first is None:
+            first = got
+        assert np.array_equal(got, first), "launches differ"
+    assert B.repq_device_status() == 0

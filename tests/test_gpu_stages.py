@@ -102,3 +102,8 @@ def test_four_bit_quantizers_stored_one_code_per_byte():
     parity.check_pv(1, 2, 130, 130, 128, b4, b4, causal=True, seed=17)
     parity.check_scores(2, 3, 197, 197, 64, b4, seed=18)
     parity.check_scores(1, 2, 50, 50, 24, b4, seed=19)
+
+
+@pytest.mark.parametrize("Bn,H,L,dh,bp,bv", [(3, 12, 256, 64, 4, 4 | parity.BYTE_CODES), (1, 4, 600, 128, 8, 4), (2, 3, 197, 32, 6, 6)])
+def test_pv_repeated_launches_reproduce_the_oracle(Bn, H, L, dh, bp, bv):
+    parity.check_pv_uniform_codes(Bn, H, L, dh, bp, bv, runs=12, seed=L)
