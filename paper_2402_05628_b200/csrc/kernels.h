@@ -19,6 +19,9 @@ repq_status qgemm_mma(const repq_gemm_desc& d, const EpilogueParams& ep, cudaStr
 // Attention-score kernel: batched code-by-code products with scalar quantizers, K <= 128, float32 output.
 bool scores_supported(const repq_gemm_desc& d);
 repq_status launch_scores(const repq_gemm_desc& d, cudaStream_t st);
+// The same on tcgen05 (byte codes, 16-byte aligned operand rows and output rows); call only if scores_supported.
+bool scores_tc_supported(const repq_gemm_desc& d);
+repq_status launch_scores_tc(const repq_gemm_desc& d, cudaStream_t st);
 
 // Tensor-memory (tcgen05) integer GEMM: plain (unbatched) products with TMA-compatible operands.
 bool qgemm_tc_supported(const repq_gemm_desc& d);

@@ -177,7 +177,7 @@ extern "C" repq_status repq_qgemm(const repq_gemm_desc* d, void* workspace, size
   REPQ_TRY(validate(*d));
   if (d->M == 0) return REPQ_OK;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (scores_supported(*d)) return launch_scores(*d, st);
+  if (scores_supported(*d)) return scores_tc_supported(*d) ? launch_scores_tc(*d, st) : launch_scores(*d, st);
   const EpilogueParams ep = make_epilogue(*d);
   if (qgemm_tc_supported(*d)) {
     const size_t need = qgemm_tc_workspace(*d);

@@ -107,3 +107,12 @@ def test_four_bit_quantizers_stored_one_code_per_byte():
 @pytest.mark.parametrize("Bn,H,L,dh,bp,bv", [(3, 12, 256, 64, 4, 4 | parity.BYTE_CODES), (1, 4, 600, 128, 8, 4), (2, 3, 197, 32, 6, 6)])
 def test_pv_repeated_launches_reproduce_the_oracle(Bn, H, L, dh, bp, bv):
     parity.check_pv_uniform_codes(Bn, H, L, dh, bp, bv, runs=12, seed=L)
+
+
+@pytest.mark.parametrize("Bn,H,Lq,Lk,dh,bits,causal", [
+    (2, 3, 197, 197, 64, 4 | parity.BYTE_CODES, False), (1, 2, 577, 577, 64, 4 | parity.BYTE_CODES, False),
+    (1, 2, 300, 300, 128, 4 | parity.BYTE_CODES, True), (1, 2, 100, 260, 48, 8, True), (1, 1, 513, 513, 16, 6, False),
+    (1, 3, 130, 700, 96, 4 | parity.BYTE_CODES, True),
+])
+def test_scores_from_byte_codes_match_oracle(Bn, H, Lq, Lk, dh, bits, causal):
+    parity.check_scores(Bn, H, Lq, Lk, dh, bits, causal, seed=Lq + dh + 1)
