@@ -3,45 +3,72 @@
 //
 // HBM-bound: every input element is read once with 128-bit loads and leaves as a 4-bit (or 8-bit)
 // code.  A row is owned by a group of TPR threads which keeps its slice of the row in registers, so mean
-// and centred variance are two register passes with shuffle reductions.  Each group works on kRows rows
-// at a time (all their loads are issued before the first reduction) to keep enough bytes in flight.
+// and centred variance are two register passes with shuffle reductions.  Each group works on one or two rows
+// at a time, and the rows of its next iteration are requested before the current ones are reduced, so that
+// loads stay in flight all the time.
 // The per-channel factors gamma~/s~ and beta~/s~ are staged once per CTA in shared memory.
 //
-// Rounding: round_half_even(clamp(t, -z, qmax - z)) is taken with one float add of 1.5 * 2^23 (the float
-// adder rounds to nearest-even at integer granularity there, with the tie decided by the parity of the
-// rounded t itself, as Eq. 4 has it); the integer then sits in the low mantissa bits and z is added while
-// the codes are packed.
+// The float work runs on packed pairs (two elements per add / mul / fma issue slot).  Rounding is the
+// float -> int conversion (half to even, on t itself, as Eq. 4 has it); z is added as an integer and the
+// clip of Eq. 4 is the saturation of the packing instruction.
 #include <cuda_bf16.h>
 
 #include "common.h"
+#include "f32x2.cuh"
 
 namespace repq {
 namespace {
 
 constexpr int kChunk = 8;   // elements per 128-bit bf16 load
-constexpr int kVPT = 4;     // chunks per thread (upper bound)
-constexpr int kRows = 2;    // rows in flight per thread group
-constexpr uint32_t kMagicBits = 0x4B400000u;   // 1.5 * 2^23
+constexpr int kMaxVPT = 4;  // chunks per thread: 1..4, chosen per row length
 
-__device__ __forceinline__ void load_chunk(const float* p, float (&v)[kChunk]) {
-  const float4 a = __ldcs(reinterpret_cast<const float4*>(p));
-  const float4 b = __ldcs(reinterpret_cast<const float4*>(p) + 1);
-  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
-  v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+// Rows a thread group works on at a time (the loads of the next ones are always in flight as well): two,
+// except where four chunks per thread would cost a resident block (measured: 16 x 3 / 32 x 3 / 256 x 4 threads x
+// chunks run best with two rows, 32 x 4 / 128 x 4 with one).
+__host__ __device__ constexpr int rows_in_flight(int vpt, int tpr) { return vpt >= 4 && tpr < 256 ? 1 : 2; }
+
+// A chunk of 8 elements as it is loaded (kept in this form while the rows before it are processed), and
+// its expansion into 4 packed float pairs.
+template <typename T> struct RawChunk;
+template <> struct RawChunk<float> { float4 a, b; };
+template <> struct RawChunk<__nv_bfloat16> { uint4 a; };
+
+__device__ __forceinline__ void load_raw(const float* p, bool on, RawChunk<float>& r) {
+  r.a = r.b = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (on) {
+    r.a = __ldcs(reinterpret_cast<const float4*>(p));
+    r.b = __ldcs(reinterpret_cast<const float4*>(p) + 1);
+  }
+}
+__device__ __forceinline__ void load_raw(const __nv_bfloat16* p, bool on, RawChunk<__nv_bfloat16>& r) {
+  r.a = make_uint4(0u, 0u, 0u, 0u);
+  if (on) r.a = __ldcs(reinterpret_cast<const uint4*>(p));
+}
+__device__ __forceinline__ void expand(const RawChunk<float>& r, f32x2 (&v)[kChunk / 2]) {
+  v[0] = pack2(r.a.x, r.a.y); v[1] = pack2(r.a.z, r.a.w); v[2] = pack2(r.b.x, r.b.y); v[3] = pack2(r.b.z, r.b.w);
+}
+__device__ __forceinline__ void expand(const RawChunk<__nv_bfloat16>& r, f32x2 (&v)[kChunk / 2]) {
+  const uint32_t w[4] = {r.a.x, r.a.y, r.a.z, r.a.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) v[i] = pack2(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xffff0000u));
 }
 
-__device__ __forceinline__ void load_chunk(const __nv_bfloat16* p, float (&v)[kChunk]) {
-  const uint4 a = __ldcs(reinterpret_cast<const uint4*>(p));
-  const uint32_t w[4] = {a.x, a.y, a.z, a.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    v[2 * i] = __uint_as_float(w[i] << 16);
-    v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-  }
+// Two consecutive codes (even index e0 in the low nibble) pushed into the low byte of a word that already
+// holds the codes of the following pairs: d = (c << 8) | sat4(e1) << 4 | sat4(e0), saturation to [0, 15].
+__device__ __forceinline__ uint32_t push_pair_u4(int e0, int e1, uint32_t c) {
+  uint32_t d;
+  asm("cvt.pack.sat.u4.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(e1), "r"(e0), "r"(c));
+  return d;
+}
+// The same for byte codes: d = (c << 16) | sat8(e1) << 8 | sat8(e0), saturation to [0, 255].
+__device__ __forceinline__ uint32_t push_pair_u8(int e0, int e1, uint32_t c) {
+  uint32_t d;
+  asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(e1), "r"(e0), "r"(c));
+  return d;
 }
 
 // Sum over the TPR threads of a group, for kRows values at once.
-template <int TPR, typename V>
+template <int TPR, int kRows, typename V>
 __device__ __forceinline__ void group_reduce(V (&v)[kRows], V* red, int group_first_warp) {
   constexpr int kShfl = TPR < 32 ? TPR : 32;
 #pragma unroll
@@ -63,12 +90,13 @@ __device__ __forceinline__ void group_reduce(V (&v)[kRows], V* red, int group_fi
   }
 }
 
-template <typename T, int TPR, bool kPack4>
+template <typename T, int TPR, int kVPT, bool kPack4>
 __global__ void __launch_bounds__((TPR > 256 ? TPR : 256))
 ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
                 const float* __restrict__ gamma_t, const float* __restrict__ beta_t, float eps, int rms,
                 float inv_s, int z, int qmax, uint8_t* __restrict__ codes, int64_t ldc,
                 int32_t* __restrict__ row_sum) {
+  constexpr int kRows = rows_in_flight(kVPT, TPR);
   constexpr int kBlock = TPR > 256 ? TPR : 256;
   constexpr int kGroups = kBlock / TPR;
   constexpr int kRowsPerBlock = kGroups * kRows;
@@ -81,52 +109,68 @@ ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
 
   float* s_g = s_gb;
   float* s_b = s_gb + D;
+  // |t| <= sqrt(D) |gamma~/s~| + |beta~/s~|.  Unless that bound is far inside the int32 range, t is clamped
+  // before the conversion so that adding z cannot wrap (a whole-kernel decision, taken here once).
+  const float root_d = sqrtf(float(D));
+  bool wide = false;
   for (int i = threadIdx.x; i < D; i += kBlock) {
-    s_g[i] = __ldg(gamma_t + i) * inv_s;
-    s_b[i] = __ldg(beta_t + i) * inv_s;
+    const float gi = __ldg(gamma_t + i) * inv_s, bi = __ldg(beta_t + i) * inv_s;
+    s_g[i] = gi;
+    s_b[i] = bi;
+    wide = wide || !(fabsf(gi) * root_d < 5.0e8f) || !(fabsf(bi) < 5.0e8f);
   }
-  __syncthreads();
+  const bool guard = __syncthreads_or(wide) != 0;
 
   const int tig = threadIdx.x % TPR;             // thread in group
   const int group = threadIdx.x / TPR;
   const int group_first_warp = (group * TPR) >> 5;
   const int nchunks = D / kChunk;
-  const float t_lo = float(-z), t_hi = float(qmax - z);
-  const float magic = __uint_as_float(kMagicBits);
   const float inv_d = 1.f / float(D);
+  const uint32_t qmax4 = uint32_t(qmax) * 0x01010101u;
 
-  for (int64_t base = int64_t(blockIdx.x) * kRowsPerBlock; base < rows;
-       base += int64_t(gridDim.x) * kRowsPerBlock) {
-    const int64_t row0 = base + group * kRows;
-
-    float v[kRows][kVPT][kChunk];
-    float sum[kRows];
+  // The rows of the next iteration are requested while those of the current one are processed, so that loads
+  // stay in flight through the reductions and the packing.
+  RawChunk<T> raw[kRows][kVPT];
+  auto fetch = [&](int64_t first_row) {
 #pragma unroll
     for (int r = 0; r < kRows; ++r) {
-      const bool live = row0 + r < rows;
-      const T* xr = x + (live ? row0 + r : 0) * ldx;
-      sum[r] = 0.f;
+      const bool live = first_row + r < rows;
+      const T* xr = x + (live ? first_row + r : 0) * ldx;
 #pragma unroll
       for (int i = 0; i < kVPT; ++i) {
         const int c = tig + i * TPR;
-        if (c < nchunks && live) {
-          load_chunk(xr + c * kChunk, v[r][i]);
-        } else {
-#pragma unroll
-          for (int e = 0; e < kChunk; ++e) v[r][i][e] = 0.f;
-        }
+        load_raw(xr + c * kChunk, live && c < nchunks, raw[r][i]);
       }
     }
+  };
+  const int64_t stride = int64_t(gridDim.x) * kRowsPerBlock;
+  fetch(int64_t(blockIdx.x) * kRowsPerBlock + group * kRows);
+
+  for (int64_t base = int64_t(blockIdx.x) * kRowsPerBlock; base < rows; base += stride) {
+    const int64_t row0 = base + group * kRows;
+
+    f32x2 v[kRows][kVPT][kChunk / 2];
+    float sum[kRows];
 #pragma unroll
     for (int r = 0; r < kRows; ++r)
 #pragma unroll
+      for (int i = 0; i < kVPT; ++i) expand(raw[r][i], v[r][i]);
+    fetch(row0 + stride);
+#pragma unroll
+    for (int r = 0; r < kRows; ++r) {
+      f32x2 acc = 0ull;
+#pragma unroll
       for (int i = 0; i < kVPT; ++i)
 #pragma unroll
-        for (int e = 0; e < kChunk; ++e) sum[r] += v[r][i][e];
+        for (int e = 0; e < kChunk / 2; ++e) acc = add2(acc, v[r][i][e]);
+      float lo, hi;
+      unpack2(acc, lo, hi);
+      sum[r] = lo + hi;
+    }
 
     float mu[kRows];
     if (!rms) {
-      group_reduce<TPR, float>(sum, red_a, group_first_warp);
+      group_reduce<TPR, kRows, float>(sum, red_a, group_first_warp);
 #pragma unroll
       for (int r = 0; r < kRows; ++r) mu[r] = sum[r] * inv_d;
     } else {
@@ -137,22 +181,26 @@ ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
     float ss[kRows];
 #pragma unroll
     for (int r = 0; r < kRows; ++r) {
-      ss[r] = 0.f;
+      const f32x2 neg_mu = splat2(-mu[r]);
+      f32x2 acc = 0ull;
 #pragma unroll
       for (int i = 0; i < kVPT; ++i) {
         if (tig + i * TPR < nchunks) {
 #pragma unroll
-          for (int e = 0; e < kChunk; ++e) {
-            v[r][i][e] -= mu[r];
-            ss[r] = fmaf(v[r][i][e], v[r][i][e], ss[r]);
+          for (int e = 0; e < kChunk / 2; ++e) {
+            v[r][i][e] = add2(v[r][i][e], neg_mu);
+            acc = fma2(v[r][i][e], v[r][i][e], acc);
           }
         }
       }
+      float lo, hi;
+      unpack2(acc, lo, hi);
+      ss[r] = lo + hi;
     }
-    group_reduce<TPR, float>(ss, red_b, group_first_warp);
-    float rstd[kRows];
+    group_reduce<TPR, kRows, float>(ss, red_b, group_first_warp);
+    f32x2 rstd[kRows];
 #pragma unroll
-    for (int r = 0; r < kRows; ++r) rstd[r] = rsqrtf(ss[r] * inv_d + eps);
+    for (int r = 0; r < kRows; ++r) rstd[r] = splat2(rsqrtf(ss[r] * inv_d + eps));
 
     int csum[kRows];
 #pragma unroll
@@ -161,43 +209,43 @@ ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
     for (int i = 0; i < kVPT; ++i) {
       const int c = tig + i * TPR;
       if (c < nchunks) {
-        float g[kChunk], b[kChunk];
+        f32x2 g[kChunk / 2], b[kChunk / 2];
         {
           const float4 g0 = *reinterpret_cast<const float4*>(s_g + c * kChunk);
           const float4 g1 = *reinterpret_cast<const float4*>(s_g + c * kChunk + 4);
           const float4 b0 = *reinterpret_cast<const float4*>(s_b + c * kChunk);
           const float4 b1 = *reinterpret_cast<const float4*>(s_b + c * kChunk + 4);
-          g[0] = g0.x; g[1] = g0.y; g[2] = g0.z; g[3] = g0.w; g[4] = g1.x; g[5] = g1.y; g[6] = g1.z; g[7] = g1.w;
-          b[0] = b0.x; b[1] = b0.y; b[2] = b0.z; b[3] = b0.w; b[4] = b1.x; b[5] = b1.y; b[6] = b1.z; b[7] = b1.w;
+          g[0] = pack2(g0.x, g0.y); g[1] = pack2(g0.z, g0.w); g[2] = pack2(g1.x, g1.y); g[3] = pack2(g1.z, g1.w);
+          b[0] = pack2(b0.x, b0.y); b[1] = pack2(b0.z, b0.w); b[2] = pack2(b1.x, b1.y); b[3] = pack2(b1.z, b1.w);
         }
 #pragma unroll
         for (int r = 0; r < kRows; ++r) {
-          uint32_t u[kChunk];
+          // Eq. 4: clip(round(t) + z, 0, qmax): round half to even by the float -> int conversion, then the
+          // packing instruction saturates to the container ([0, 15] or [0, 255])
+          float t[kChunk];
 #pragma unroll
-          for (int e = 0; e < kChunk; ++e) {
-            float t = fmaf(v[r][i][e] * rstd[r], g[e], b[e]);
-            t = fminf(fmaxf(t, t_lo), t_hi);       // clip(round(t) + z, 0, qmax) == round(clamp(t)) + z
-            u[e] = __float_as_uint(t + magic);     // = magic_bits + round_half_even(t), as integers
+          for (int e = 0; e < kChunk / 2; ++e) unpack2(fma2(mul2(v[r][i][e], rstd[r]), g[e], b[e]), t[2 * e], t[2 * e + 1]);
+          if (guard) {
+#pragma unroll
+            for (int e = 0; e < kChunk; ++e) t[e] = fminf(fmaxf(t[e], -1.0e9f), 1.0e9f);
           }
+          int q[kChunk];
+#pragma unroll
+          for (int e = 0; e < kChunk; ++e) q[e] = __float2int_rn(t[e]) + z;
           if (row0 + r < rows) {
             uint8_t* out = codes + (row0 + r) * ldc;
             if constexpr (kPack4) {
-              // sum_e (magic_bits + round(t_e)) << 4e  -  sum_e (magic_bits - z) << 4e  =  sum_e code_e << 4e
               uint32_t w = 0;
 #pragma unroll
-              for (int e = 0; e < kChunk; ++e) w += u[e] << (4 * e);
-              uint32_t k = 0;
-#pragma unroll
-              for (int e = 0; e < kChunk; ++e) k += (kMagicBits - uint32_t(z)) << (4 * e);
-              w -= k;
+              for (int e = kChunk - 2; e >= 0; e -= 2) w = push_pair_u4(q[e], q[e + 1], w);
               reinterpret_cast<uint32_t*>(out)[c] = w;
               csum[r] += __dp4a(w & 0x0F0F0F0Fu, 0x01010101u, 0u) + __dp4a((w >> 4) & 0x0F0F0F0Fu, 0x01010101u, 0u);
             } else {
               uint2 w;
-              // low bytes hold round(t_e) mod 256; a per-byte add of z gives the codes (all in [0, 255])
-              const uint32_t z4 = (uint32_t(z) & 0xFFu) * 0x01010101u;
-              w.x = __vadd4(__byte_perm(__byte_perm(u[0], u[1], 0x0040), __byte_perm(u[2], u[3], 0x0040), 0x5410), z4);
-              w.y = __vadd4(__byte_perm(__byte_perm(u[4], u[5], 0x0040), __byte_perm(u[6], u[7], 0x0040), 0x5410), z4);
+              w.x = push_pair_u8(q[0], q[1], push_pair_u8(q[2], q[3], 0u));
+              w.y = push_pair_u8(q[4], q[5], push_pair_u8(q[6], q[7], 0u));
+              w.x = __vminu4(w.x, qmax4);          // 4- and 6-bit quantizers in byte containers
+              w.y = __vminu4(w.y, qmax4);
               reinterpret_cast<uint2*>(out)[c] = w;
               csum[r] += __dp4a(w.x, 0x01010101u, 0u) + __dp4a(w.y, 0x01010101u, 0u);
             }
@@ -206,7 +254,7 @@ ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
       }
     }
     if (row_sum != nullptr) {
-      group_reduce<TPR, int>(csum, red_c, group_first_warp);
+      group_reduce<TPR, kRows, int>(csum, red_c, group_first_warp);
       if (tig == 0) {
 #pragma unroll
         for (int r = 0; r < kRows; ++r)
@@ -216,24 +264,36 @@ ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
   }
 }
 
-template <typename T, int TPR>
+template <typename T, int TPR, int kVPT>
 repq_status launch(const T* x, int64_t rows, int D, int64_t ldx, const float* g, const float* b, float eps,
                    int rms, float s_t, int z, int bits, uint8_t* codes, int64_t ldc, int32_t* row_sum,
                    cudaStream_t st) {
   constexpr int kBlock = TPR > 256 ? TPR : 256;
-  constexpr int kRowsPerBlock = kBlock / TPR * kRows;
+  constexpr int kRowsPerBlock = kBlock / TPR * rows_in_flight(kVPT, TPR);
   const int64_t need = (rows + kRowsPerBlock - 1) / kRowsPerBlock;
   const int64_t cap = int64_t(sm_count()) * 8;
   const int grid = int(need < cap ? need : cap);
   const float inv_s = 1.f / s_t;
   const int qmax = code_max(bits);
   const size_t smem = size_t(D) * 2 * sizeof(float);
-  auto kern = packed4(bits) ? ln_quant_kernel<T, TPR, true> : ln_quant_kernel<T, TPR, false>;
+  auto kern = packed4(bits) ? ln_quant_kernel<T, TPR, kVPT, true> : ln_quant_kernel<T, TPR, kVPT, false>;
   if (smem > 48 * 1024) REPQ_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
   kern<<<grid, kBlock, smem, st>>>(x, rows, D, ldx, g, b, eps, rms, inv_s, z, qmax, codes, ldc, row_sum);
   REPQ_CUDA(cudaGetLastError());
   note_launch();
   return REPQ_OK;
+}
+
+template <typename T, int TPR>
+repq_status launch_vpt(int vpt, const T* x, int64_t rows, int D, int64_t ldx, const float* g, const float* b, float eps,
+                       int rms, float s_t, int z, int bits, uint8_t* codes, int64_t ldc, int32_t* row_sum,
+                       cudaStream_t st) {
+  switch (vpt) {
+    case 1: return launch<T, TPR, 1>(x, rows, D, ldx, g, b, eps, rms, s_t, z, bits, codes, ldc, row_sum, st);
+    case 2: return launch<T, TPR, 2>(x, rows, D, ldx, g, b, eps, rms, s_t, z, bits, codes, ldc, row_sum, st);
+    case 3: return launch<T, TPR, 3>(x, rows, D, ldx, g, b, eps, rms, s_t, z, bits, codes, ldc, row_sum, st);
+    default: return launch<T, TPR, 4>(x, rows, D, ldx, g, b, eps, rms, s_t, z, bits, codes, ldc, row_sum, st);
+  }
 }
 
 template <typename T>
@@ -242,7 +302,7 @@ repq_status dispatch(const T* x, int64_t rows, int D, int64_t ldx, const float* 
                      cudaStream_t st) {
   const int nchunks = D / kChunk;
 #define REPQ_LN_CASE(TPR) \
-  if (nchunks <= TPR * kVPT) return launch<T, TPR>(x, rows, D, ldx, g, b, eps, rms, s_t, z, bits, codes, ldc, row_sum, st);
+  if (nchunks <= TPR * kMaxVPT) return launch_vpt<T, TPR>((nchunks + TPR - 1) / TPR, x, rows, D, ldx, g, b, eps, rms, s_t, z, bits, codes, ldc, row_sum, st);
   REPQ_LN_CASE(8)
   REPQ_LN_CASE(16)
   REPQ_LN_CASE(32)

@@ -13,12 +13,20 @@
 #include <math_constants.h>
 
 #include "common.h"
+#include "f32x2.cuh"
 
 namespace repq {
 namespace {
 
 constexpr int kChunk = 8;
-constexpr int kVPT = 4;
+constexpr int kMaxVPT = 4;   // chunks per thread: 1..4, chosen per row length
+constexpr uint32_t kMagicBits = 0x4B400000u;   // 1.5 * 2^23
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 
 // Loads elements [idx, idx + 8) of a row; elements at or beyond `valid` become -inf.  `vec_ok` says
 // the row base is 16-byte aligned; a vector load is used only when it lies inside the row extent `ld`.
@@ -35,9 +43,11 @@ __device__ __forceinline__ void load_scores(const float* row, int idx, int valid
       for (int e = 0; e < 4; ++e) v[4 * h + e] = (i0 + e < valid) ? __ldcs(row + i0 + e) : -CUDART_INF_F;
     }
   }
+  if (idx + kChunk > valid) {                       // only the chunk that holds the row's last visible key
 #pragma unroll
-  for (int e = 0; e < kChunk; ++e)
-    if (idx + e >= valid) v[e] = -CUDART_INF_F;
+    for (int e = 0; e < kChunk; ++e)
+      if (idx + e >= valid) v[e] = -CUDART_INF_F;
+  }
 }
 
 __device__ __forceinline__ void load_scores(const __nv_bfloat16* row, int idx, int valid, int64_t ld,
@@ -55,9 +65,11 @@ __device__ __forceinline__ void load_scores(const __nv_bfloat16* row, int idx, i
     for (int e = 0; e < kChunk; ++e)
       v[e] = (idx + e < valid) ? __bfloat162float(row[idx + e]) : -CUDART_INF_F;
   }
+  if (idx + kChunk > valid) {                       // only the chunk that holds the row's last visible key
 #pragma unroll
-  for (int e = 0; e < kChunk; ++e)
-    if (idx + e >= valid) v[e] = -CUDART_INF_F;
+    for (int e = 0; e < kChunk; ++e)
+      if (idx + e >= valid) v[e] = -CUDART_INF_F;
+  }
 }
 
 template <int TPR, bool kMax>
@@ -81,7 +93,7 @@ __device__ __forceinline__ float group_reduce(float v, float* red, int group_fir
   return v;
 }
 
-template <typename T, int TPR, bool kPack4>
+template <typename T, int TPR, int kVPT, bool kPack4>
 __global__ void __launch_bounds__((TPR > 256 ? TPR : 256))
 softmax_log2_kernel(const T* __restrict__ scores, int64_t rows, int L, int64_t ld, bool vec_ok, float c,
                     int causal_period, int causal_offset, float log2_s, int qmax,
@@ -96,6 +108,7 @@ softmax_log2_kernel(const T* __restrict__ scores, int64_t rows, int L, int64_t l
   const int group_first_warp = (group * TPR) >> 5;
   const int nchunks = (L + kChunk - 1) / kChunk;
   const float fq = float(qmax);
+  const bool clamp_lo = log2_s < 0.f;
 
   for (int64_t base = int64_t(blockIdx.x) * kRowsPerBlock; base < rows;
        base += int64_t(gridDim.x) * kRowsPerBlock) {
@@ -110,58 +123,82 @@ softmax_log2_kernel(const T* __restrict__ scores, int64_t rows, int L, int64_t l
     }
     if (!live) valid = 0;
 
-    float v[kVPT][kChunk];
+    // the row slice of this thread as packed pairs; masked keys (at or beyond `valid`) are -inf
+    f32x2 v[kVPT][kChunk / 2];
     float m = -CUDART_INF_F;
 #pragma unroll
     for (int i = 0; i < kVPT; ++i) {
       const int ch = tig + i * TPR;
+      float f[kChunk];
       if (ch < nchunks && ch * kChunk < valid) {
-        load_scores(sr, ch * kChunk, valid, ld, vec_ok, v[i]);
+        load_scores(sr, ch * kChunk, valid, ld, vec_ok, f);
       } else {
 #pragma unroll
-        for (int e = 0; e < kChunk; ++e) v[i][e] = -CUDART_INF_F;
+        for (int e = 0; e < kChunk; ++e) f[e] = -CUDART_INF_F;
       }
 #pragma unroll
-      for (int e = 0; e < kChunk; ++e) m = fmaxf(m, v[i][e]);
+      for (int e = 0; e < kChunk; e += 2) {
+        m = fmaxf(m, fmaxf(f[e], f[e + 1]));
+        v[i][e / 2] = pack2(f[e], f[e + 1]);
+      }
     }
     m = group_reduce<TPR, true>(m, red_a, group_first_warp);
     if (!live) m = 0.f;
 
+    // d = S - m (<= 0, -inf for masked keys); Z = sum 2^(c d)
+    const f32x2 neg_m = splat2(-m), c2 = splat2(c);
     float z = 0.f;
 #pragma unroll
     for (int i = 0; i < kVPT; ++i) {
+      if ((tig + i * TPR) * kChunk >= valid) continue;          // chunk fully masked: contributes nothing
 #pragma unroll
-      for (int e = 0; e < kChunk; ++e) {
-        v[i][e] -= m;                       // <= 0, -inf for masked keys
-        z += exp2f(v[i][e] * c);
+      for (int e = 0; e < kChunk / 2; ++e) {
+        v[i][e] = add2(v[i][e], neg_m);
+        float a0, a1;
+        unpack2(mul2(v[i][e], c2), a0, a1);
+        z += ex2(a0) + ex2(a1);
       }
     }
     z = group_reduce<TPR, false>(z, red_b, group_first_warp);
-    const float k0 = 2.f * (log2f(z) + log2_s);
-    const float k1 = -2.f * c;
+    const f32x2 k0 = splat2(2.f * (log2f(z) + log2_s));
+    const f32x2 k1 = splat2(-2.f * c);
+    const f32x2 magic2 = splat2(__uint_as_float(kMagicBits));
 
     if (live) {
       uint8_t* out = codes + row * ldc;
 #pragma unroll
       for (int i = 0; i < kVPT; ++i) {
         const int ch = tig + i * TPR;
-        if (ch < nchunks) {
-          uint32_t q[kChunk];
+        if (ch < nchunks && ch * kChunk >= valid) {
+          // fully masked chunk: top codes, no arithmetic
+          const uint32_t top = uint32_t(qmax) * (kPack4 ? 0x11111111u : 0x01010101u);
+          if constexpr (kPack4) reinterpret_cast<uint32_t*>(out)[ch] = top;
+          else reinterpret_cast<uint2*>(out)[ch] = make_uint2(top, top);
+        } else if (ch < nchunks) {
+          // round_half_even(clamp(t, 0, qmax)) by one float add of 1.5 * 2^23: the code is left in the low
+          // mantissa bits.  t = +inf (masked keys) clamps to the top code; with s >= 1, t cannot be negative
+          // by more than a rounding error, which the add absorbs, so the lower clamp is needed for s < 1 only.
+          uint32_t u[kChunk];
 #pragma unroll
-          for (int e = 0; e < kChunk; ++e) {
-            float t = fmaf(v[i][e], k1, k0);          // +inf for masked keys
-            t = fminf(fmaxf(t, 0.f), fq);
-            q[e] = uint32_t(__float2int_rn(t));
+          for (int e = 0; e < kChunk / 2; ++e) {
+            float t0, t1;
+            unpack2(fma2(v[i][e], k1, k0), t0, t1);
+            t0 = fminf(t0, fq); t1 = fminf(t1, fq);
+            if (clamp_lo) { t0 = fmaxf(t0, 0.f); t1 = fmaxf(t1, 0.f); }
+            float r0, r1;
+            unpack2(add2(pack2(t0, t1), magic2), r0, r1);
+            u[2 * e] = __float_as_uint(r0);
+            u[2 * e + 1] = __float_as_uint(r1);
           }
           if constexpr (kPack4) {
             uint32_t w = 0;
 #pragma unroll
-            for (int e = 0; e < kChunk; ++e) w |= q[e] << (4 * e);
-            reinterpret_cast<uint32_t*>(out)[ch] = w;
+            for (int e = 0; e < kChunk; ++e) w += u[e] << (4 * e);
+            reinterpret_cast<uint32_t*>(out)[ch] = w - kMagicBits * 0x11111111u;
           } else {
             uint2 w;
-            w.x = q[0] | q[1] << 8 | q[2] << 16 | q[3] << 24;
-            w.y = q[4] | q[5] << 8 | q[6] << 16 | q[7] << 24;
+            w.x = __byte_perm(__byte_perm(u[0], u[1], 0x0040), __byte_perm(u[2], u[3], 0x0040), 0x5410);
+            w.y = __byte_perm(__byte_perm(u[4], u[5], 0x0040), __byte_perm(u[6], u[7], 0x0040), 0x5410);
             reinterpret_cast<uint2*>(out)[ch] = w;
           }
         }
@@ -170,7 +207,7 @@ softmax_log2_kernel(const T* __restrict__ scores, int64_t rows, int L, int64_t l
   }
 }
 
-template <typename T, int TPR>
+template <typename T, int TPR, int kVPT>
 repq_status launch(const T* scores, int64_t rows, int L, int64_t ld, bool vec_ok, float c, int period,
                    int offset, float log2_s, int bits, uint8_t* codes, int64_t ldc, cudaStream_t st) {
   constexpr int kBlock = TPR > 256 ? TPR : 256;
@@ -180,12 +217,23 @@ repq_status launch(const T* scores, int64_t rows, int L, int64_t ld, bool vec_ok
   const int grid = int(need < cap ? need : cap);
   const int qmax = code_max(bits);
   if (packed4(bits))
-    softmax_log2_kernel<T, TPR, true><<<grid, kBlock, 0, st>>>(scores, rows, L, ld, vec_ok, c, period, offset, log2_s, qmax, codes, ldc);
+    softmax_log2_kernel<T, TPR, kVPT, true><<<grid, kBlock, 0, st>>>(scores, rows, L, ld, vec_ok, c, period, offset, log2_s, qmax, codes, ldc);
   else
-    softmax_log2_kernel<T, TPR, false><<<grid, kBlock, 0, st>>>(scores, rows, L, ld, vec_ok, c, period, offset, log2_s, qmax, codes, ldc);
+    softmax_log2_kernel<T, TPR, kVPT, false><<<grid, kBlock, 0, st>>>(scores, rows, L, ld, vec_ok, c, period, offset, log2_s, qmax, codes, ldc);
   REPQ_CUDA(cudaGetLastError());
   note_launch();
   return REPQ_OK;
+}
+
+template <typename T, int TPR>
+repq_status launch_vpt(int vpt, const T* scores, int64_t rows, int L, int64_t ld, bool vec_ok, float c, int period,
+                       int offset, float log2_s, int bits, uint8_t* codes, int64_t ldc, cudaStream_t st) {
+  switch (vpt) {
+    case 1: return launch<T, TPR, 1>(scores, rows, L, ld, vec_ok, c, period, offset, log2_s, bits, codes, ldc, st);
+    case 2: return launch<T, TPR, 2>(scores, rows, L, ld, vec_ok, c, period, offset, log2_s, bits, codes, ldc, st);
+    case 3: return launch<T, TPR, 3>(scores, rows, L, ld, vec_ok, c, period, offset, log2_s, bits, codes, ldc, st);
+    default: return launch<T, TPR, 4>(scores, rows, L, ld, vec_ok, c, period, offset, log2_s, bits, codes, ldc, st);
+  }
 }
 
 template <typename T>
@@ -193,7 +241,7 @@ repq_status dispatch(const T* scores, int64_t rows, int L, int64_t ld, bool vec_
                      int offset, float log2_s, int bits, uint8_t* codes, int64_t ldc, cudaStream_t st) {
   const int nchunks = (L + kChunk - 1) / kChunk;
 #define REPQ_SM_CASE(TPR) \
-  if (nchunks <= TPR * kVPT) return launch<T, TPR>(scores, rows, L, ld, vec_ok, c, period, offset, log2_s, bits, codes, ldc, st);
+  if (nchunks <= TPR * kMaxVPT) return launch_vpt<T, TPR>((nchunks + TPR - 1) / TPR, scores, rows, L, ld, vec_ok, c, period, offset, log2_s, bits, codes, ldc, st);
   REPQ_SM_CASE(8)
   REPQ_SM_CASE(16)
   REPQ_SM_CASE(32)
