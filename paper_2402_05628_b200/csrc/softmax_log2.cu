@@ -28,48 +28,51 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-// Loads elements [idx, idx + 8) of a row; elements at or beyond `valid` become -inf.  `vec_ok` says
-// the row base is 16-byte aligned; a vector load is used only when it lies inside the row extent `ld`.
-__device__ __forceinline__ void load_scores(const float* row, int idx, int valid, int64_t ld, bool vec_ok,
-                                            float (&v)[kChunk]) {
+// Elements [idx, idx + 8) of a row.  Fast form: the whole chunk is visible and one or two 128-bit loads cover
+// it; it is requested one row ahead, kept as loaded, and expanded into 4 packed pairs when its row's turn comes.
+template <typename T> struct RawChunk;
+template <> struct RawChunk<float> { float4 a, b; };
+template <> struct RawChunk<__nv_bfloat16> { uint4 a; };
+__device__ __forceinline__ void load_raw(const float* p, RawChunk<float>& r) {
+  r.a = __ldcs(reinterpret_cast<const float4*>(p));
+  r.b = __ldcs(reinterpret_cast<const float4*>(p) + 1);
+}
+__device__ __forceinline__ void load_raw(const __nv_bfloat16* p, RawChunk<__nv_bfloat16>& r) {
+  r.a = __ldcs(reinterpret_cast<const uint4*>(p));
+}
+__device__ __forceinline__ void expand(const RawChunk<float>& r, f32x2 (&v)[kChunk / 2]) {
+  v[0] = pack2(r.a.x, r.a.y); v[1] = pack2(r.a.z, r.a.w); v[2] = pack2(r.b.x, r.b.y); v[3] = pack2(r.b.z, r.b.w);
+}
+__device__ __forceinline__ void expand(const RawChunk<__nv_bfloat16>& r, f32x2 (&v)[kChunk / 2]) {
+  const uint32_t w[4] = {r.a.x, r.a.y, r.a.z, r.a.w};
 #pragma unroll
-  for (int h = 0; h < 2; ++h) {
-    const int i0 = idx + 4 * h;
-    if (vec_ok && i0 + 4 <= ld && i0 < valid) {
-      const float4 a = __ldcs(reinterpret_cast<const float4*>(row + i0));
-      v[4 * h + 0] = a.x; v[4 * h + 1] = a.y; v[4 * h + 2] = a.z; v[4 * h + 3] = a.w;
-    } else {
-#pragma unroll
-      for (int e = 0; e < 4; ++e) v[4 * h + e] = (i0 + e < valid) ? __ldcs(row + i0 + e) : -CUDART_INF_F;
-    }
-  }
-  if (idx + kChunk > valid) {                       // only the chunk that holds the row's last visible key
-#pragma unroll
-    for (int e = 0; e < kChunk; ++e)
-      if (idx + e >= valid) v[e] = -CUDART_INF_F;
-  }
+  for (int i = 0; i < 4; ++i) v[i] = pack2(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xffff0000u));
+}
+// General form (kept out of line: it runs for rows that are not 16-byte aligned and for a chunk that would
+// cross the row stride): element loads, -inf at or beyond `valid`.
+struct ChunkPairs { f32x2 p0, p1, p2, p3; };
+__device__ __noinline__ ChunkPairs load_ragged(const float* row, int idx, int valid) {
+  float f[kChunk];
+  for (int e = 0; e < kChunk; ++e) f[e] = (idx + e < valid) ? __ldcs(row + idx + e) : -CUDART_INF_F;
+  return ChunkPairs{pack2(f[0], f[1]), pack2(f[2], f[3]), pack2(f[4], f[5]), pack2(f[6], f[7])};
+}
+__device__ __noinline__ ChunkPairs load_ragged(const __nv_bfloat16* row, int idx, int valid) {
+  float f[kChunk];
+  for (int e = 0; e < kChunk; ++e) f[e] = (idx + e < valid) ? __bfloat162float(row[idx + e]) : -CUDART_INF_F;
+  return ChunkPairs{pack2(f[0], f[1]), pack2(f[2], f[3]), pack2(f[4], f[5]), pack2(f[6], f[7])};
 }
 
-__device__ __forceinline__ void load_scores(const __nv_bfloat16* row, int idx, int valid, int64_t ld,
-                                            bool vec_ok, float (&v)[kChunk]) {
-  if (vec_ok && idx + 8 <= ld && idx < valid) {
-    const uint4 a = __ldcs(reinterpret_cast<const uint4*>(row + idx));
-    const uint32_t w[4] = {a.x, a.y, a.z, a.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      v[2 * i] = __uint_as_float(w[i] << 16);
-      v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-    }
-  } else {
-#pragma unroll
-    for (int e = 0; e < kChunk; ++e)
-      v[e] = (idx + e < valid) ? __bfloat162float(row[idx + e]) : -CUDART_INF_F;
-  }
-  if (idx + kChunk > valid) {                       // only the chunk that holds the row's last visible key
-#pragma unroll
-    for (int e = 0; e < kChunk; ++e)
-      if (idx + e >= valid) v[e] = -CUDART_INF_F;
-  }
+// Two consecutive codes (even index first) pushed into the low byte / low half of a word that already holds the
+// codes after them, with saturation to [0, 15] / [0, 255] (cvt.pack.sat: d = c << 8 | sat(e1) << 4 | sat(e0)).
+__device__ __forceinline__ uint32_t push_pair_u4(int e0, int e1, uint32_t c) {
+  uint32_t d;
+  asm("cvt.pack.sat.u4.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(e1), "r"(e0), "r"(c));
+  return d;
+}
+__device__ __forceinline__ uint32_t push_pair_u8(int e0, int e1, uint32_t c) {
+  uint32_t d;
+  asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(e1), "r"(e0), "r"(c));
+  return d;
 }
 
 template <int TPR, bool kMax>
@@ -108,40 +111,70 @@ softmax_log2_kernel(const T* __restrict__ scores, int64_t rows, int L, int64_t l
   const int group_first_warp = (group * TPR) >> 5;
   const int nchunks = (L + kChunk - 1) / kChunk;
   const float fq = float(qmax);
-  const bool clamp_lo = log2_s < 0.f;
 
-  for (int64_t base = int64_t(blockIdx.x) * kRowsPerBlock; base < rows;
-       base += int64_t(gridDim.x) * kRowsPerBlock) {
+  // keys a row may see (0 for rows past the end)
+  auto visible = [&](int64_t row) {
+    if (row >= rows) return 0;
+    if (causal_period <= 0) return L;
+    const int64_t v = (row % causal_period) + 1 + causal_offset;
+    return v < 1 ? 1 : (v < L ? int(v) : L);
+  };
+  // The vector-loadable chunks (16-byte aligned rows, chunk inside the row stride) of the next row of this group are requested while the current row
+  // is processed, so that loads stay in flight through the reductions.
+  RawChunk<T> raw[kVPT];
+  auto fetch = [&](int64_t row) {
+    const int valid = visible(row);
+    const T* sr = scores + (row < rows ? row : 0) * ld;
+#pragma unroll
+    for (int i = 0; i < kVPT; ++i) {
+      const int idx = (tig + i * TPR) * kChunk;
+      if (vec_ok && idx < valid && idx + kChunk <= ld) load_raw(sr + idx, raw[i]);
+    }
+  };
+  const int64_t stride = int64_t(gridDim.x) * kRowsPerBlock;
+  fetch(int64_t(blockIdx.x) * kRowsPerBlock + group);
+
+  for (int64_t base = int64_t(blockIdx.x) * kRowsPerBlock; base < rows; base += stride) {
     const int64_t row = base + group;
     const bool live = row < rows;
     const T* sr = scores + (live ? row : 0) * ld;
-    int valid = L;
-    if (causal_period > 0) {
-      const int64_t v = (row % causal_period) + 1 + causal_offset;
-      valid = v < L ? int(v) : L;
-      if (valid < 1) valid = 1;
-    }
-    if (!live) valid = 0;
+    const int valid = visible(row);
 
     // the row slice of this thread as packed pairs; masked keys (at or beyond `valid`) are -inf
     f32x2 v[kVPT][kChunk / 2];
     float m = -CUDART_INF_F;
+    const f32x2 ninf2 = splat2(-CUDART_INF_F);
 #pragma unroll
     for (int i = 0; i < kVPT; ++i) {
       const int ch = tig + i * TPR;
-      float f[kChunk];
-      if (ch < nchunks && ch * kChunk < valid) {
-        load_scores(sr, ch * kChunk, valid, ld, vec_ok, f);
-      } else {
+      const int idx = ch * kChunk;
+      if (idx >= valid) {                                    // (also: chunks past the row, rows past the end)
 #pragma unroll
-        for (int e = 0; e < kChunk; ++e) f[e] = -CUDART_INF_F;
+        for (int e = 0; e < kChunk / 2; ++e) v[i][e] = ninf2;
+        continue;
+      }
+      if (vec_ok && idx + kChunk <= ld) {
+        expand(raw[i], v[i]);
+        if (idx + kChunk > valid) {                          // the chunk that holds the row's last visible key
+#pragma unroll
+          for (int e = 0; e < kChunk / 2; ++e) {
+            float lo, hi;
+            unpack2(v[i][e], lo, hi);
+            v[i][e] = pack2(idx + 2 * e < valid ? lo : -CUDART_INF_F, idx + 2 * e + 1 < valid ? hi : -CUDART_INF_F);
+          }
+        }
+      } else {
+        const ChunkPairs r = load_ragged(sr, idx, valid);
+        v[i][0] = r.p0; v[i][1] = r.p1; v[i][2] = r.p2; v[i][3] = r.p3;
       }
 #pragma unroll
-      for (int e = 0; e < kChunk; e += 2) {
-        m = fmaxf(m, fmaxf(f[e], f[e + 1]));
-        v[i][e / 2] = pack2(f[e], f[e + 1]);
+      for (int e = 0; e < kChunk / 2; ++e) {
+        float lo, hi;
+        unpack2(v[i][e], lo, hi);
+        m = fmaxf(m, fmaxf(lo, hi));
       }
     }
+    fetch(row + stride);
     m = group_reduce<TPR, true>(m, red_a, group_first_warp);
     if (!live) m = 0.f;
 
@@ -175,30 +208,29 @@ softmax_log2_kernel(const T* __restrict__ scores, int64_t rows, int L, int64_t l
           if constexpr (kPack4) reinterpret_cast<uint32_t*>(out)[ch] = top;
           else reinterpret_cast<uint2*>(out)[ch] = make_uint2(top, top);
         } else if (ch < nchunks) {
-          // round_half_even(clamp(t, 0, qmax)) by one float add of 1.5 * 2^23: the code is left in the low
-          // mantissa bits.  t = +inf (masked keys) clamps to the top code; with s >= 1, t cannot be negative
-          // by more than a rounding error, which the add absorbs, so the lower clamp is needed for s < 1 only.
-          uint32_t u[kChunk];
+          // Eq. 15: clip(round(t), 0, qmax).  The upper clip is a float min (t = +inf for masked keys and
+          // underflowed probabilities lands on the top code); rounding half to even is one packed float add of
+          // 1.5 * 2^23, which leaves the code in the low mantissa bits; negative t (possible for s < 1 only) would
+          // leave a negative integer there, which the saturating pack turns into code 0.
+          int q[kChunk];
 #pragma unroll
           for (int e = 0; e < kChunk / 2; ++e) {
             float t0, t1;
             unpack2(fma2(v[i][e], k1, k0), t0, t1);
-            t0 = fminf(t0, fq); t1 = fminf(t1, fq);
-            if (clamp_lo) { t0 = fmaxf(t0, 0.f); t1 = fmaxf(t1, 0.f); }
             float r0, r1;
-            unpack2(add2(pack2(t0, t1), magic2), r0, r1);
-            u[2 * e] = __float_as_uint(r0);
-            u[2 * e + 1] = __float_as_uint(r1);
+            unpack2(add2(pack2(fminf(t0, fq), fminf(t1, fq)), magic2), r0, r1);
+            q[2 * e] = __float_as_int(r0) - int(kMagicBits);
+            q[2 * e + 1] = __float_as_int(r1) - int(kMagicBits);
           }
           if constexpr (kPack4) {
             uint32_t w = 0;
 #pragma unroll
-            for (int e = 0; e < kChunk; ++e) w += u[e] << (4 * e);
-            reinterpret_cast<uint32_t*>(out)[ch] = w - kMagicBits * 0x11111111u;
+            for (int e = kChunk - 2; e >= 0; e -= 2) w = push_pair_u4(q[e], q[e + 1], w);
+            reinterpret_cast<uint32_t*>(out)[ch] = w;
           } else {
             uint2 w;
-            w.x = __byte_perm(__byte_perm(u[0], u[1], 0x0040), __byte_perm(u[2], u[3], 0x0040), 0x5410);
-            w.y = __byte_perm(__byte_perm(u[4], u[5], 0x0040), __byte_perm(u[6], u[7], 0x0040), 0x5410);
+            w.x = push_pair_u8(q[0], q[1], push_pair_u8(q[2], q[3], 0u));
+            w.y = push_pair_u8(q[4], q[5], push_pair_u8(q[6], q[7], 0u));
             reinterpret_cast<uint2*>(out)[ch] = w;
           }
         }

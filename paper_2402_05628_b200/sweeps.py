@@ -6,7 +6,7 @@ uses of the same buffer exceed the L2 capacity.  Reports achieved GB/s or TOP/s 
 bytes / operations of the case.  Inputs are seeded torch tensors with the value ranges of the workloads
 (the arithmetic does not depend on the values; parity is checked elsewhere).
 
-    python -m paper_2402_05628_b200.sweeps ln softmax gemm pv scores [--quick]
+    python -m paper_2402_05628_b200.sweeps ln softmax gemm [--quick] [--dim D] [--rows R]
 """
 from __future__ import annotations
 
@@ -39,14 +39,14 @@ def _nbuf(bytes_per_call):
     return max(2, min(64, int(2 * L2_BYTES / max(bytes_per_call, 1)) + 1))
 
 
-def sweep_ln(quick):
+def sweep_ln(quick, only_dim=None, only_rows=None):
     dev = torch.device("cuda:0")
     g = torch.Generator(device=dev).manual_seed(4)
     out = []
     rows_list = [1024, 16384, 262144] if quick else [1024, 4096, 16384, 65536, 262144, 1048576]
     for D in (384, 768, 1024, 4096, 8192):
         for rows in rows_list:
-            if rows * D * 2 > (8 << 30):
+            if rows * D * 2 > (8 << 30) or (only_dim and D != only_dim) or (only_rows and rows != only_rows):
                 continue
             for bits in ((4,) if quick else (4, 6, 8)):
                 for dt in (torch.bfloat16,):
@@ -67,11 +67,13 @@ def sweep_ln(quick):
     return out
 
 
-def sweep_softmax(quick):
+def sweep_softmax(quick, only_dim=None, only_rows=None):
     dev = torch.device("cuda:0")
     g = torch.Generator(device=dev).manual_seed(4)
     out = []
     for L in (197, 577, 2048, 8192):
+        if only_dim and L != only_dim:
+            continue
         for rows in ((151296,) if quick else (4096, 32768, 151296)):
             if L >= 2048:
                 rows = min(rows, 32768)
@@ -90,7 +92,7 @@ def sweep_softmax(quick):
     return out
 
 
-def sweep_gemm(quick):
+def sweep_gemm(quick, only_dim=None, only_rows=None):
     dev = torch.device("cuda:0")
     out = []
     shapes = [(12608, 2304, 768), (12608, 768, 768), (12608, 3072, 768), (12608, 768, 3072),
@@ -131,10 +133,12 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("which", nargs="+", choices=["ln", "softmax", "gemm"])
     ap.add_argument("--quick", action="store_true")
+    ap.add_argument("--dim", type=int, default=None, help="only this feature size (ln) / row length (softmax)")
+    ap.add_argument("--rows", type=int, default=None, help="only this row count (ln)")
     args = ap.parse_args()
     B.lib()
     for name in args.which:
-        for row in {"ln": sweep_ln, "softmax": sweep_softmax, "gemm": sweep_gemm}[name](args.quick):
+        for row in {"ln": sweep_ln, "softmax": sweep_softmax, "gemm": sweep_gemm}[name](args.quick, args.dim, args.rows):
             print(json.dumps(row))
             sys.stdout.flush()
 
