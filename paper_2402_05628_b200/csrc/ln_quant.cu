@@ -271,13 +271,17 @@ repq_status launch(const T* x, int64_t rows, int D, int64_t ldx, const float* g,
   constexpr int kBlock = TPR > 256 ? TPR : 256;
   constexpr int kRowsPerBlock = kBlock / TPR * rows_in_flight(kVPT, TPR);
   const int64_t need = (rows + kRowsPerBlock - 1) / kRowsPerBlock;
-  const int64_t cap = int64_t(sm_count()) * 8;
-  const int grid = int(need < cap ? need : cap);
   const float inv_s = 1.f / s_t;
   const int qmax = code_max(bits);
   const size_t smem = size_t(D) * 2 * sizeof(float);
   auto kern = packed4(bits) ? ln_quant_kernel<T, TPR, kVPT, true> : ln_quant_kernel<T, TPR, kVPT, false>;
   if (smem > 48 * 1024) REPQ_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+  // persistent grid: exactly the blocks that are resident at once, so that every block keeps its load pipeline
+  // running over all of its rows
+  int resident = 0;
+  REPQ_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, kern, kBlock, smem));
+  const int64_t cap = int64_t(sm_count()) * (resident > 0 ? resident : 1);
+  const int grid = int(need < cap ? need : cap);
   kern<<<grid, kBlock, smem, st>>>(x, rows, D, ldx, g, b, eps, rms, inv_s, z, qmax, codes, ldc, row_sum);
   REPQ_CUDA(cudaGetLastError());
   note_launch();

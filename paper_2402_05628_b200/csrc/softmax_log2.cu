@@ -245,13 +245,14 @@ repq_status launch(const T* scores, int64_t rows, int L, int64_t ld, bool vec_ok
   constexpr int kBlock = TPR > 256 ? TPR : 256;
   constexpr int kRowsPerBlock = kBlock / TPR;
   const int64_t need = (rows + kRowsPerBlock - 1) / kRowsPerBlock;
-  const int64_t cap = int64_t(sm_count()) * 8;
-  const int grid = int(need < cap ? need : cap);
   const int qmax = code_max(bits);
-  if (packed4(bits))
-    softmax_log2_kernel<T, TPR, kVPT, true><<<grid, kBlock, 0, st>>>(scores, rows, L, ld, vec_ok, c, period, offset, log2_s, qmax, codes, ldc);
-  else
-    softmax_log2_kernel<T, TPR, kVPT, false><<<grid, kBlock, 0, st>>>(scores, rows, L, ld, vec_ok, c, period, offset, log2_s, qmax, codes, ldc);
+  auto kern = packed4(bits) ? softmax_log2_kernel<T, TPR, kVPT, true> : softmax_log2_kernel<T, TPR, kVPT, false>;
+  // persistent grid: exactly the blocks that are resident at once (every block keeps its load pipeline running)
+  int resident = 0;
+  REPQ_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, kern, kBlock, 0));
+  const int64_t cap = int64_t(sm_count()) * (resident > 0 ? resident : 1);
+  const int grid = int(need < cap ? need : cap);
+  kern<<<grid, kBlock, 0, st>>>(scores, rows, L, ld, vec_ok, c, period, offset, log2_s, qmax, codes, ldc);
   REPQ_CUDA(cudaGetLastError());
   note_launch();
   return REPQ_OK;
