@@ -29,6 +29,10 @@ if ROOT not in sys.path:
 METRIC = "quantized_block_tokens_per_s"
 UNIT = "tokens/s"
 INT8_OVER_BF16 = 2.0          # nominal dense int8 : bf16 tensor throughput on B200
+# Fused attention is bound by its per-score arithmetic, not by tensor cores or HBM: pass 1 needs about 8 instructions
+# per score (correction, int -> float, scale, max, subtract, scale, ex2, add), pass 2 about 15 (the first three again,
+# the code, its power of two, the parity split, packing): the algorithmic count the roofline figure uses.
+ATTENTION_INSTR_PER_SCORE = 23
 
 # DRAM traffic of one launch of each stage kernel, from one ncu capture of this file's default workload
 # (DeiT-B shape, batch 64; the summaries are under profiles/).  A figure is reported only while the kernel's
@@ -203,6 +207,8 @@ def main():
     ap.add_argument("--batch", type=int, default=None, help="override the workload's batch (parity-sized runs)")
     ap.add_argument("--ref-batch", type=int, default=8)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--staged-attention", action="store_true",
+                    help="run scores, Softmax codes and P.V as three kernels instead of the fused attention kernel")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -240,7 +246,7 @@ def main():
     r0, r1 = shard_rows(world, rank, batch, L)
     w = dataclasses.replace(w, cfg=cfg, x=w.x[r0:r1])
     tokens_per_step = batch * L
-    blk = QuantBlock(w, device=dev)
+    blk = QuantBlock(w, device=dev, staged_attention=args.staged_attention)
     x_host = torch.from_numpy(np.ascontiguousarray(w.x)).to(blk.act_dtype).pin_memory()
     x = x_host.to(dev, non_blocking=True)
     y = torch.empty_like(x, dtype=blk.out_dtype)
@@ -311,12 +317,34 @@ def main():
             if c["ops"]:
                 st["tops"] = c["ops"] / (ms * 1e-3) / 1e12 if ms > 0 else None
             stages[name] = st
+        if not args.staged_attention:
+            # the fused kernel ran in the slot of the scores stage; Softmax and P.V have no launch of their own
+            att = stages.pop("scores")
+            stages.pop("softmax")
+            stages.pop("pv")
+            n_scores = batch * cfg["H"] * L * L * (0.5 if cfg["causal"] else 1.0)
+            att_instr = ATTENTION_INSTR_PER_SCORE * n_scores
+            att = dict(ms=att["ms"], gbs=4.0 * batch * L * cfg["D"] / (att["ms"] * 1e-3) / 1e9,
+                       ginstr=att_instr / (att["ms"] * 1e-3) / 1e9)
+            stages = {k: (att if k == "qkv_next" else v) for k, v in stages.items()}
+            ordered = {}
+            for k, v in stages.items():
+                ordered[k] = v
+                if k == "qkv":
+                    ordered["attention"] = att
+            stages = ordered
         top = max(stages, key=lambda k: stages[k]["ms"])
         int8_peak = peaks["bf16_tflops"] * INT8_OVER_BF16
         if top in ("qkv", "proj", "fc1", "fc2"):          # scores: bound by its float32 writes, see the HBM branch
             roof = dict(kernel=top, bound="tensor", achieved=stages[top]["tops"], peak=int8_peak, unit="TOP/s",
                         frac=stages[top]["tops"] / int8_peak, traffic=measured_traffic(top, cfg["name"], batch),
                         peak_source="%s bf16 burst x %.0f (nominal int8:bf16)" % (peaks["source"], INT8_OVER_BF16))
+        elif top == "attention":
+            alu_peak = 148 * 4 * 32 * (clocks["sm_max_mhz"] or 1965.0) * 1e6 / 1e9      # G thread-instructions / s
+            roof = dict(kernel=top, bound="alu", achieved=stages[top]["ginstr"], peak=alu_peak, unit="Ginstr/s",
+                        frac=stages[top]["ginstr"] / alu_peak, traffic=measured_traffic(top, cfg["name"], batch),
+                        peak_source="148 SMs x 4 schedulers x 32 lanes x SM clock; %d instructions per score (two passes)"
+                                    % ATTENTION_INSTR_PER_SCORE)
         elif top == "pv":
             roof = dict(kernel=top, bound="tensor", achieved=2 * stages[top]["tops"], peak=peaks["bf16_tflops"],
                         unit="TFLOP/s", frac=2 * stages[top]["tops"] / peaks["bf16_tflops"], traffic=measured_traffic(top, cfg["name"], batch),

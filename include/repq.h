@@ -63,7 +63,7 @@ typedef int repq_status;
 size_t repq_last_error(char* buf, size_t n);
 
 /* Library ABI version (bumped on any signature change). */
-int repq_abi_version(void);   /* currently 3 */
+int repq_abi_version(void);   /* currently 4 */
 
 /* ------------------------------------------------------------------------------------------------
  * One-time host-side preparation (not on the timed path)
@@ -207,6 +207,46 @@ typedef struct repq_pv_desc {
 
 repq_status repq_pv(const repq_pv_desc* d, void* stream);
 
+/* Fused attention on codes: Eq. 3 (scores from quantized Q and K, Softmax), Eq. 15 (log-sqrt2 codes of the
+ * probabilities) and Eqs. 16-17 (P.V with the reparameterized log2 de-quantization) in one kernel; scores and
+ * codes stay on chip.  Same result as repq_qgemm (scores) -> repq_softmax_log2 -> repq_pv, except that the
+ * Softmax sum is accumulated in a different order, which can move a code across a rounding tie.
+ *     S[i, j] = alpha s_q s_k sum_c (q[i, c] - z_q)(k[j, c] - z_k)      (causal: j <= i + Lk - Lq only)
+ *     p       = clip(round(-2 log2(softmax(S)[i, j] / s_p)), 0, 2^bits_p - 1)
+ *     O[i, :] = sum_j s_p 2^(-ceil(p/2)) (sqrt2 if p odd) s_v (v[j, :] - z_v)
+ * for batch_outer x batch_inner (batch, head) pairs.  q, k, v [device]: codes of one quantizer width, stored one
+ * per byte (bits_qkv must carry REPQ_BYTE_CODES); operand (bo, bi) starts at base + bo*stride_outer +
+ * bi*stride_inner; Q and K rows 16-byte aligned, V rows 8-byte aligned.  d_h a multiple of 16, at most 128.
+ * Output as in repq_pv. */
+typedef struct repq_attention_desc {
+  int32_t batch_outer, batch_inner, Lq, Lk, d_h;
+  int32_t bits_qkv;
+  const uint8_t* q_codes;
+  int64_t ldq_bytes, q_stride_outer, q_stride_inner;
+  float s_q;
+  int32_t z_q;
+  const uint8_t* k_codes;
+  int64_t ldk_bytes, k_stride_outer, k_stride_inner;
+  float s_k;
+  int32_t z_k;
+  const uint8_t* v_codes;
+  int64_t ldv_bytes, v_stride_outer, v_stride_inner;
+  float s_v;
+  int32_t z_v;
+  float alpha;                          /* 1/sqrt(d_h) */
+  int32_t causal;
+  int32_t bits_p;                       /* width of the log-sqrt2 quantizer */
+  float s_p;                            /* its scale s */
+  int32_t out_kind, out_bits;
+  float out_scale;
+  int32_t out_zero;
+  void* out;
+  int64_t ldo, o_stride_outer, o_stride_inner;
+  int32_t* out_row_sum;                 /* as in repq_pv_desc */
+} repq_attention_desc;
+
+repq_status repq_attention(const repq_attention_desc* d, void* stream);
+
 /* ------------------------------------------------------------------------------------------------
  * Whole block: Eqs. 1-2,  X_bar = MSA(LN(X)) + X,  Y = MLP(LN(X_bar)) + X_bar, all GEMM inputs
  * quantized (LayerNorm -> QKV -> QK^T -> Softmax/log2 -> P.V -> proj -> LayerNorm -> fc1/GELU -> fc2).
@@ -229,6 +269,8 @@ typedef struct repq_block_desc {
   float eps;
   int32_t act_dtype;                    /* dtype of x and of the stored residual stream X_bar */
   int32_t out_dtype;                    /* dtype of y */
+  int32_t staged_attention;             /* 0: fused attention kernel (repq_attention); != 0: the three separate
+                                           stages (scores -> Softmax codes -> P.V) through the workspace */
 } repq_block_desc;
 
 typedef struct repq_block_params {

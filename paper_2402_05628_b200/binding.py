@@ -28,7 +28,7 @@ EXPORTS = (
     "repq_pack_weights", "repq_ln_quant", "repq_qgemm_workspace_bytes", "repq_qgemm",
     "repq_softmax_log2", "repq_pv", "repq_block_workspace_bytes", "repq_block_forward",
     "repq_device_status", "repq_block_forward_timed", "repq_launch_count",
-    "repq_block_forward_static",
+    "repq_block_forward_static", "repq_attention",
 )
 REPQ_STATIC_WORKSPACE_BYTES = 8 << 20
 REPQ_BLOCK_STAGES = 9
@@ -84,7 +84,24 @@ class BlockDesc(C.Structure):
     _fields_ = [("batch", C.c_int32), ("seq", C.c_int32), ("dim", C.c_int32), ("heads", C.c_int32),
                 ("mlp", C.c_int32), ("bits_a", C.c_int32), ("bits_w", C.c_int32), ("bits_p", C.c_int32),
                 ("causal", C.c_int32), ("norm_kind", C.c_int32), ("eps", C.c_float),
-                ("act_dtype", C.c_int32), ("out_dtype", C.c_int32)]
+                ("act_dtype", C.c_int32), ("out_dtype", C.c_int32), ("staged_attention", C.c_int32)]
+
+
+class AttentionDesc(C.Structure):
+    _fields_ = [
+        ("batch_outer", C.c_int32), ("batch_inner", C.c_int32), ("Lq", C.c_int32), ("Lk", C.c_int32), ("d_h", C.c_int32),
+        ("bits_qkv", C.c_int32),
+        ("q_codes", C.c_void_p), ("ldq_bytes", C.c_int64), ("q_stride_outer", C.c_int64), ("q_stride_inner", C.c_int64),
+        ("s_q", C.c_float), ("z_q", C.c_int32),
+        ("k_codes", C.c_void_p), ("ldk_bytes", C.c_int64), ("k_stride_outer", C.c_int64), ("k_stride_inner", C.c_int64),
+        ("s_k", C.c_float), ("z_k", C.c_int32),
+        ("v_codes", C.c_void_p), ("ldv_bytes", C.c_int64), ("v_stride_outer", C.c_int64), ("v_stride_inner", C.c_int64),
+        ("s_v", C.c_float), ("z_v", C.c_int32),
+        ("alpha", C.c_float), ("causal", C.c_int32), ("bits_p", C.c_int32), ("s_p", C.c_float),
+        ("out_kind", C.c_int32), ("out_bits", C.c_int32), ("out_scale", C.c_float), ("out_zero", C.c_int32),
+        ("out", C.c_void_p), ("ldo", C.c_int64), ("o_stride_outer", C.c_int64), ("o_stride_inner", C.c_int64),
+        ("out_row_sum", C.c_void_p),
+    ]
 
 
 class BlockParams(C.Structure):
@@ -130,6 +147,7 @@ def lib() -> C.CDLL:
                                                   C.c_void_p, C.c_size_t, C.c_void_p, C.POINTER(C.c_float)]
         _lib.repq_block_forward_static.argtypes = [C.POINTER(BlockDesc), C.POINTER(BlockParams), C.c_void_p,
                                                    C.c_void_p, C.c_void_p]
+        _lib.repq_attention.argtypes = [C.POINTER(AttentionDesc), C.c_void_p]
         _lib.repq_launch_count.restype = C.c_uint64
         _lib.repq_launch_count.argtypes = []
         _lib.repq_scale_zero_from_bounds.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
@@ -250,6 +268,10 @@ def repq_qgemm(d: GemmDesc, workspace: Optional[torch.Tensor] = None, stream=Non
 
 def repq_pv(d: PvDesc, stream=None) -> None:
     _check(lib().repq_pv(C.byref(d), _stream(stream)))
+
+
+def repq_attention(d: AttentionDesc, stream: Optional[int] = None) -> None:
+    _check(lib().repq_attention(C.byref(d), _stream(stream)))
 
 
 def repq_block_workspace_bytes(d: BlockDesc) -> int:

@@ -1,0 +1,604 @@
+// Fused attention on integer codes: scores (Eq. 3 with quantized Q and K), Softmax, log-sqrt2 codes (Eq. 15) and
+// P.V with the reparameterized log2 de-quantization (Eqs. 16-17) in one kernel.  Scores and codes never leave the
+// SM.  The code of a score depends on the row's final Softmax sum, so the keys are walked twice:
+//   pass 1   S = Q K^T per block of 64 keys (tcgen05.mma kind::i8 into tensor memory), running row maximum m and
+//            sum Z = sum 2^(c (S - m)) (each thread: one row, 32 of the 64 columns; the two partial results of a row
+//            are merged once, after the pass)
+//   pass 2   S again, t = 2 (log2 Z + log2 s) - 2 c (S - m), code p = clip(round(t), 0, 2^b - 1), operand values
+//            2^(-ceil(p/2)) split by the parity of p into the tiles E and O (exact bf16 powers of two), V as exact bf16
+//            integers v - z_v, and two tcgen05.mma kind::f16 per 16 keys accumulate E.V and O.V in tensor memory;
+//            O = s s_v (acc_E + sqrt2 acc_O), then the output conversion (Eq. 4 or float)
+// Float arithmetic on S is the same as in the separate kernels (float(corr) * (alpha s_q s_k); one ex2 per element
+// for Z), so the codes agree with theirs except where the differently ordered sum Z moves a value across a
+// rounding tie.
+//
+// One CTA owns 128 query rows of one (batch, head) pair.  Warps 0..7: K tiles and V tiles from registers (fetched one
+// block ahead) into 128-byte-swizzled shared-memory tiles, the Softmax arithmetic, the E / O tiles, the epilogue.
+// Warp 8 (one lane): tensor-memory allocation and MMA issue.  S is double-buffered in tensor memory (2 x 64 columns),
+// the E / O / V tiles are single (their block's code arithmetic overlaps the MMAs of the block before).  Under a causal mask, key blocks no row of the CTA may see are
+// skipped.  Every mbarrier wait is bounded; when one runs out the kernel records a status code, all roles leave
+// their loops, MMAs in flight are drained, tensor memory is freed and the kernel returns.
+#include <cuda_bf16.h>
+#include <math_constants.h>
+
+#include <cstdlib>
+
+#include "kernels.h"
+#include "tc_ptx.cuh"
+
+namespace repq {
+namespace {
+
+using namespace tc;
+
+constexpr int kRows = 128;                  // query rows per CTA (MMA M)
+constexpr int kKeys = 64;                   // keys per block
+constexpr int kWorkWarps = 8;
+constexpr int kWorkThreads = 32 * kWorkWarps;
+constexpr int kThreads = kWorkThreads + 32;
+constexpr uint32_t kQBytes = kRows * 128;         // Q tile: rows of 128 bytes (the head's codes, zero-padded)
+constexpr uint32_t kKBytes = kKeys * 128;
+constexpr uint32_t kTileBytes = kRows * 128;      // E or O tile of one block (64 keys of bf16 per row)
+constexpr uint32_t kVBlockBytes = kKeys * 128;    // 64 keys x 64 channels of bf16
+constexpr uint32_t kMagicBits = 0x4B400000u;      // float 1.5 * 2^23
+constexpr int kAccCol = 2 * kKeys;                // first tensor-memory column of the P.V accumulators
+
+struct AttnParams {
+  const uint8_t* q; const uint8_t* k; const uint8_t* v;
+  int64_t ldq, ldk, ldv, q_so, q_si, k_so, k_si, v_so, v_si;
+  int Lq, Lk, dh, batch_inner, causal;
+  float scale;            // alpha s_q s_k
+  int zq, zk;
+  float log2_s;           // log2 of the log-sqrt2 scale
+  int qmax_p;             // 2^bits_p - 1
+  int z_v, v_small;
+  float out_scale;        // s_p s_v
+  int out_kind, qmax, pack4;
+  float inv_so; int zo;
+  void* out; int64_t ldo, o_so, o_si;
+  int32_t* out_row_sum;
+  int n_pad, tmem_cols, vec_store;
+  int32_t* status;
+};
+
+template <int NB>
+struct AttnShared {
+  alignas(1024) uint8_t q[kQBytes];
+  alignas(1024) uint8_t k[2][kKBytes];
+  alignas(1024) uint8_t e[kTileBytes];
+  alignas(1024) uint8_t o[kTileBytes];
+  alignas(1024) uint8_t v[NB * kVBlockBytes];
+  int row_term[kRows];                              // -z_k qsum[m] + d_h z_q z_k
+  int col_term[4][kKeys];                           // -z_q ksum[n], ring of 4 key blocks
+  float stat_m[2][kRows], stat_z[2][kRows];         // pass-1 results of the two column halves of every row
+  uint32_t lut[16][32];                             // 4-bit codes: [code][lane] = E value | O value << 16 (one bank per lane)
+  alignas(8) uint64_t k_full[2];
+  uint64_t s_full[2], s_empty[2], p_full, p_empty;
+  uint64_t stats_ready, acc_full, done;
+  uint32_t tmem_base;
+  volatile int abort;
+};
+
+__device__ __forceinline__ uint32_t tile_offset(int row, int piece) {
+  return uint32_t(row >> 3) * 1024u + uint32_t(row & 7) * 128u + (uint32_t(piece ^ (row & 7)) << 4);
+}
+__device__ __forceinline__ int sum_bytes(const uint4& v) {
+  return __dp4a(v.x, 0x01010101u, __dp4a(v.y, 0x01010101u, __dp4a(v.z, 0x01010101u, __dp4a(v.w, 0x01010101u, 0u))));
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// NB: 64-channel blocks of the head; kLut: Softmax codes of at most 4 bits (operand values from the per-lane table)
+template <int NB, bool kLut>
+__global__ void __launch_bounds__(kThreads, NB == 1 ? 2 : 1)
+attention_tc_kernel(AttnParams P) {
+  using Shared = AttnShared<NB>;
+  constexpr int kVItems = 2 * NB;                         // 8-channel groups of V per thread and block
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  Shared& S = *reinterpret_cast<Shared*>(smem_raw);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int pair = blockIdx.y;
+  const int bo = pair / P.batch_inner, bi = pair % P.batch_inner;
+  const int q0 = blockIdx.x * kRows;
+  const int shift = P.Lk - P.Lq;
+  const int k_end = P.causal ? max(1, min(P.Lk, min(q0 + kRows, P.Lq) + shift)) : P.Lk;
+  const int min_valid = P.causal ? max(0, min(P.Lk, q0 + 1 + shift)) : P.Lk;   // fewest keys any row of the CTA sees
+  const int nb = (k_end + kKeys - 1) / kKeys;             // key blocks; every block is visited in both passes
+  const int ksteps = (P.dh + 31) >> 5;                    // S MMAs of K = 32 per key block
+  const int pieces = P.dh >> 4;                           // 16-byte pieces of a Q / K row
+
+  if (tid == 0) {
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(smem_u32(&S.k_full[s]), kWorkWarps);
+      mbar_init(smem_u32(&S.s_full[s]), 1);
+      mbar_init(smem_u32(&S.s_empty[s]), kWorkWarps);
+    }
+    mbar_init(smem_u32(&S.p_full), kWorkWarps);
+    mbar_init(smem_u32(&S.p_empty), 1);
+    mbar_init(smem_u32(&S.stats_ready), kWorkWarps);
+    mbar_init(smem_u32(&S.acc_full), 1);
+    mbar_init(smem_u32(&S.done), 1);
+    S.abort = 0;
+    if (smem_u32(smem_raw) & 1023u) {                     // the swizzled tiles need this alignment
+      atomicCAS(P.status, 0, 49);
+      S.abort = 1;
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == kWorkWarps) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&S.tmem_base)), "r"(uint32_t(P.tmem_cols)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+
+  // ---- K rows: 4 threads per key, 2 pieces each; Q rows: 2 threads per row, 4 pieces each
+  const uint8_t* k_base = P.k + bo * P.k_so + bi * P.k_si;
+  const int kkey = (tid >> 2) & (kKeys - 1), kq = tid & 3;
+  uint4 kreg[2], knext[2];                      // the K rows of the next two key blocks
+  auto fetch_k = [&](int block, uint4 (&dst)[2]) {
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      dst[j] = make_uint4(0u, 0u, 0u, 0u);
+      const int piece = 2 * kq + j, key = block * kKeys + kkey;
+      if (key < P.Lk && piece < pieces) dst[j] = __ldg(reinterpret_cast<const uint4*>(k_base + int64_t(key) * P.ldk) + piece);
+    }
+  };
+  auto store_k = [&](uint8_t* tile) {            // returns the code sum of the thread's key
+    int s = 0;
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const int piece = 2 * kq + j;
+      if (piece < 2 * ksteps) *reinterpret_cast<uint4*>(tile + tile_offset(kkey, piece)) = kreg[j];
+      s += sum_bytes(kreg[j]);
+    }
+    s += __shfl_xor_sync(0xffffffffu, s, 1);
+    s += __shfl_xor_sync(0xffffffffu, s, 2);
+    return s;
+  };
+
+  if (warp < kWorkWarps) {
+    fetch_k(0, kreg);
+    fetch_k(nb > 1 ? 1 : 0, knext);
+    const uint8_t* q_base = P.q + bo * P.q_so + bi * P.q_si;
+    const int qrow = (tid >> 1) & (kRows - 1), qh = tid & 1;
+    int s = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int piece = 4 * qh + j;
+      uint4 w = make_uint4(0u, 0u, 0u, 0u);
+      if (q0 + qrow < P.Lq && piece < pieces) w = __ldg(reinterpret_cast<const uint4*>(q_base + int64_t(q0 + qrow) * P.ldq) + piece);
+      if (piece < 2 * ksteps) *reinterpret_cast<uint4*>(S.q + tile_offset(qrow, piece)) = w;
+      s += sum_bytes(w);
+    }
+    s += __shfl_xor_sync(0xffffffffu, s, 1);
+    if (qh == 0) S.row_term[qrow] = -P.zk * s + P.dh * P.zq * P.zk;
+    for (int i = tid; i < 16 * 32; i += kWorkThreads) {
+      const uint32_t code = uint32_t(i >> 5), bits16 = (127u - ((code + 1u) >> 1)) << 7;      // bf16 bits of 2^-ceil(code/2)
+      S.lut[0][i] = (code & 1u) ? bits16 << 16 : bits16;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = S.tmem_base;
+  volatile int* abort = &S.abort;
+
+  if (warp == kWorkWarps) {
+    // ---------------------------------------------------------------- MMA issue
+    if (lane == 0) {
+      // S: D = s32, A = B = unsigned 8-bit, both K-major, N = 64, M = 128
+      constexpr uint32_t idesc_s = (2u << 4) | (uint32_t(kKeys >> 3) << 17) | (uint32_t(kRows >> 4) << 24);
+      // P.V: D = f32, A = B = bf16, A K-major, B MN-major, N = n_pad, M = 128
+      const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (uint32_t(P.n_pad >> 3) << 17) |
+                                (uint32_t(kRows >> 4) << 24);
+      const uint64_t dq = smem_desc_sw128(smem_u32(S.q));
+      bool ok = true;
+      auto issue_s = [&](int g) {                          // S of key block g % nb, g counted over both passes
+        const int b = g & 1;
+        const uint32_t ph = uint32_t(g >> 1) & 1u;
+        if (!mbar_wait(smem_u32(&S.k_full[b]), ph, abort, 41, P.status)) return false;
+        if (!mbar_wait(smem_u32(&S.s_empty[b]), ph ^ 1u, abort, 42, P.status)) return false;
+        tc_fence_after();
+        const uint64_t dk = smem_desc_sw128(smem_u32(S.k[b]));
+        for (int s = 0; s < ksteps; ++s)
+          umma_i8(tmem_base + uint32_t(b * kKeys), dq + uint64_t(2 * s), dk + uint64_t(2 * s), idesc_s, s != 0 ? 1u : 0u);
+        umma_commit(smem_u32(&S.s_full[b]));
+        return true;
+      };
+      for (int g = 0; g < nb && ok && !*abort; ++g) ok = issue_s(g);
+      if (ok && !*abort) ok = issue_s(nb);
+      for (int j = 0; j < nb && ok && !*abort; ++j) {
+        if (j + 1 < nb && !issue_s(nb + j + 1)) { ok = false; break; }
+        if (!mbar_wait(smem_u32(&S.p_full), uint32_t(j) & 1u, abort, 43, P.status)) { ok = false; break; }
+        tc_fence_after();
+        const uint64_t de = smem_desc_sw128(smem_u32(S.e)), dd = smem_desc_sw128(smem_u32(S.o));
+        const uint64_t dv = smem_desc_sw128(smem_u32(S.v), kVBlockBytes);
+        const int keys_here = min(kKeys, k_end - j * kKeys);
+        const int steps = (keys_here + 15) >> 4;                       // 16 keys per MMA
+        for (int s = 0; s < steps; ++s) {
+          const uint32_t accumulate = (j | s) != 0 ? 1u : 0u;
+          umma_f16(tmem_base + uint32_t(kAccCol), de + uint64_t(2 * s), dv + uint64_t(128 * s), idesc_pv, accumulate);
+          umma_f16(tmem_base + uint32_t(kAccCol + P.n_pad), dd + uint64_t(2 * s), dv + uint64_t(128 * s), idesc_pv, accumulate);
+        }
+        umma_commit(smem_u32(&S.p_empty));
+      }
+      if (ok && !*abort) umma_commit(smem_u32(&S.acc_full));
+      umma_commit(smem_u32(&S.done));
+      mbar_drain(smem_u32(&S.done), 0);
+    }
+  } else {
+    // ---------------------------------------------------------------- tiles, Softmax arithmetic, epilogue
+    const int quarter = warp & 3, half = warp >> 2;
+    const int r = quarter * 32 + lane;                    // the thread's row inside the CTA = its tensor-memory lane
+    const int row = q0 + r;
+    const int valid = row < P.Lq ? (P.causal ? max(1, min(P.Lk, row + 1 + shift)) : P.Lk) : 0;   // keys the row sees
+    const int my_row_term = S.row_term[r];
+    const float c = 1.4426950408889634f;
+    const float k1 = -2.f * c;
+    const float fq = float(P.qmax_p);
+    const float magic = __uint_as_float(kMagicBits);
+    const uint32_t taddr_s = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(half * 32);
+
+    // V items of a block (as in the P.V kernel): 2 NB groups of 8 channels per thread
+    const uint8_t* v_ptr[kVItems];
+    uint32_t v_off[kVItems];
+    int v_key[kVItems];
+#pragma unroll
+    for (int qi = 0; qi < kVItems; ++qi) {
+      const int i = tid + kWorkThreads * qi;
+      const int kr = i / (8 * NB), g8 = i % (8 * NB);
+      v_ptr[qi] = P.v + bo * P.v_so + bi * P.v_si + int64_t(kr) * P.ldv + g8 * 8;
+      v_off[qi] = uint32_t(g8 >> 3) * kVBlockBytes + tile_offset(kr, g8 & 7);
+      v_key[qi] = g8 * 8 < P.dh ? kr : -1;
+    }
+    const int64_t v_step = int64_t(kKeys) * P.ldv;
+    uint2 vraw[kVItems];
+    auto fetch_v = [&](int block) {
+#pragma unroll
+      for (int qi = 0; qi < kVItems; ++qi) {
+        vraw[qi] = make_uint2(0u, 0u);
+        if (block < nb && v_key[qi] >= 0 && block * kKeys + v_key[qi] < P.Lk)
+          vraw[qi] = __ldg(reinterpret_cast<const uint2*>(v_ptr[qi] + block * v_step));
+      }
+    };
+    const float vz = __uint_as_float(kMagicBits) + float(P.z_v);
+    const __nv_bfloat162 vz2 = __float2bfloat162_rn(128.f + float(P.z_v));
+
+    float m = -CUDART_INF_F, z = 0.f;       // pass 1: running maximum and sum of this thread's columns
+    float k0 = 0.f;                         // pass 2: 2 (log2 Z + log2 s), with m the row's final maximum
+
+    // corr = acc - z_k qsum - z_q ksum + d_h z_q z_k of the thread's 32 columns of key block j (buffer g & 1), as
+    // integers; keys the row may not see become kMasked.  Frees the buffer as soon as it is read.
+    constexpr int kMasked = -2147483647 - 1;
+    auto read_s = [&](int g, int j, int (&corr)[32]) -> bool {
+      const int b = g & 1;
+      if (!mbar_wait(smem_u32(&S.s_full[b]), uint32_t(g >> 1) & 1u, abort, 44, P.status)) return false;
+      tc_fence_after();
+      uint32_t r0[16], r1[16];
+      __syncwarp();
+      tmem_ld16(taddr_s + uint32_t(b * kKeys), r0);
+      tmem_ld16(taddr_s + uint32_t(b * kKeys + 16), r1);
+      tmem_ld_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&S.s_empty[b]));
+      const int* ct = S.col_term[g & 3] + half * 32;
+#pragma unroll
+      for (int e4 = 0; e4 < 8; ++e4) {
+        const int4 c4 = *reinterpret_cast<const int4*>(ct + 4 * e4);
+        const uint32_t* rr = e4 < 4 ? &r0[4 * e4] : &r1[4 * (e4 - 4)];
+        corr[4 * e4 + 0] = int32_t(rr[0]) + my_row_term + c4.x;
+        corr[4 * e4 + 1] = int32_t(rr[1]) + my_row_term + c4.y;
+        corr[4 * e4 + 2] = int32_t(rr[2]) + my_row_term + c4.z;
+        corr[4 * e4 + 3] = int32_t(rr[3]) + my_row_term + c4.w;
+      }
+      // causal mask and keys past Lk: only in blocks that reach past the fewest keys any row of the CTA sees
+      const int key0 = j * kKeys + half * 32;
+      if (__builtin_expect(key0 + 32 > min(min_valid, valid), 0)) {
+#pragma unroll
+        for (int e = 0; e < 32; ++e)
+          if (key0 + e >= valid) corr[e] = kMasked;
+      }
+      return true;
+    };
+
+    auto process = [&](int g) -> bool {
+      const int j = g < nb ? g : g - nb;
+      int corr[32];
+      if (!read_s(g, j, corr)) return false;
+      if (g < nb) {
+        // ---- pass 1: running maximum and sum.  The maximum is taken on the integers (S = scale * float(corr) is
+        // monotonic in corr); a masked key contributes 2^(-huge) = 0.
+        int bmi = corr[0];
+#pragma unroll
+        for (int e = 1; e < 32; ++e) bmi = max(bmi, corr[e]);
+        if (bmi != kMasked) {
+          const float mn = fmaxf(m, P.scale * float(bmi));
+          float acc0 = 0.f, acc1 = 0.f;
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            acc0 += ex2(fmaf(float(corr[e]), P.scale, -mn) * c);
+            acc1 += ex2(fmaf(float(corr[e + 1]), P.scale, -mn) * c);
+          }
+          z = z * ex2((m - mn) * c) + (acc0 + acc1);     // m = -inf at first: factor 0
+          m = mn;
+        }
+        if (g == nb - 1) {
+          // merge the two halves of every row: m = max, Z = sum of the rescaled partial sums
+          S.stat_m[half][r] = m;
+          S.stat_z[half][r] = z;
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&S.stats_ready));
+          if (!mbar_wait(smem_u32(&S.stats_ready), 0, abort, 45, P.status)) return false;
+          const float m2 = S.stat_m[half ^ 1][r], z2 = S.stat_z[half ^ 1][r];
+          const float mn = fmaxf(m, m2);
+          float zt = 0.f;
+          if (m > -CUDART_INF_F) zt += z * ex2((m - mn) * c);
+          if (m2 > -CUDART_INF_F) zt += z2 * ex2((m2 - mn) * c);
+          m = mn;
+          k0 = 2.f * (log2f(zt) + P.log2_s);
+          fetch_v(0);
+        }
+        return true;
+      }
+      // ---- pass 2: codes, operand tiles, V tile.
+      // Eq. 15: p = clip(round(t), 0, qmax), t = k0 - 2 c (S - m); rounding half to even by the float add of
+      // 1.5 * 2^23, which leaves p in the low mantissa bits u - kMagicBits.  The pair (E, O) of bf16 operand values,
+      // 2^-ceil(p/2) on the side of p's parity and 0 on the other, comes from a per-lane table for 4-bit codes and
+      // from integer arithmetic for wider ones.  A masked key gets (0, 0).
+      const bool boundary = j * kKeys + half * 32 + 32 > min(min_valid, valid);
+      const uint32_t lut_addr = smem_u32(&S.lut[0][lane]) - (kMagicBits << 7);
+      uint32_t eo[32];
+#pragma unroll
+      for (int e = 0; e < 32; ++e) {
+        // clamped on both sides whatever the inputs (rows past Lq carry m = -inf, Z = 0): p indexes the table
+        const float t = fmaxf(fminf(fmaf(fmaf(float(corr[e]), P.scale, -m), k1, k0), fq), 0.f);
+        const uint32_t u = __float_as_uint(t + magic);
+        if (kLut) {
+          asm("ld.shared.u32 %0, [%1];" : "=r"(eo[e]) : "r"(lut_addr + (u << 7)));
+        } else {
+          const int kk = int((u - kMagicBits + 1u) >> 1);                       // ceil(p / 2)
+          const uint32_t val = uint32_t(max(127 - kk, 0)) << 7;                 // bf16 bits of 2^-kk (0 below the normal range)
+          eo[e] = (u & 1u) ? val << 16 : val;
+        }
+      }
+      if (__builtin_expect(boundary, 0)) {
+#pragma unroll
+        for (int e = 0; e < 32; ++e)
+          if (corr[e] == kMasked) eo[e] = 0u;
+      }
+      uint4 ev[4], ov[4];
+#pragma unroll
+      for (int p4 = 0; p4 < 4; ++p4) {
+        ev[p4] = make_uint4(__byte_perm(eo[8 * p4 + 0], eo[8 * p4 + 1], 0x5410), __byte_perm(eo[8 * p4 + 2], eo[8 * p4 + 3], 0x5410),
+                            __byte_perm(eo[8 * p4 + 4], eo[8 * p4 + 5], 0x5410), __byte_perm(eo[8 * p4 + 6], eo[8 * p4 + 7], 0x5410));
+        ov[p4] = make_uint4(__byte_perm(eo[8 * p4 + 0], eo[8 * p4 + 1], 0x7632), __byte_perm(eo[8 * p4 + 2], eo[8 * p4 + 3], 0x7632),
+                            __byte_perm(eo[8 * p4 + 4], eo[8 * p4 + 5], 0x7632), __byte_perm(eo[8 * p4 + 6], eo[8 * p4 + 7], 0x7632));
+      }
+      // one stage of operand tiles: the MMAs of the block before must have read them (the code arithmetic above
+      // has overlapped with those MMAs)
+      if (!mbar_wait(smem_u32(&S.p_empty), (uint32_t(j) & 1u) ^ 1u, abort, 46, P.status)) return false;
+#pragma unroll
+      for (int p4 = 0; p4 < 4; ++p4) {
+        const uint32_t off = tile_offset(r, half * 4 + p4);
+        *reinterpret_cast<uint4*>(S.e + off) = ev[p4];
+        *reinterpret_cast<uint4*>(S.o + off) = ov[p4];
+      }
+#pragma unroll
+      for (int qi = 0; qi < kVItems; ++qi) {
+        uint32_t o4[4] = {0u, 0u, 0u, 0u};
+        if (v_key[qi] >= 0 && j * kKeys + v_key[qi] < P.Lk) {
+          const uint32_t b03 = vraw[qi].x, b47 = vraw[qi].y;
+          if (P.v_small) {
+            // v - z_v as bf16: for codes below 128, 128 + v is the bit pattern 0x4300 | v and the bf16 subtraction exact
+            const uint32_t w[4] = {__byte_perm(b03, 0x43434343u, 0x4140), __byte_perm(b03, 0x43434343u, 0x4342),
+                                   __byte_perm(b47, 0x43434343u, 0x4140), __byte_perm(b47, 0x43434343u, 0x4342)};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const __nv_bfloat162 h = __hsub2(*reinterpret_cast<const __nv_bfloat162*>(&w[e]), vz2);
+              o4[e] = *reinterpret_cast<const uint32_t*>(&h);
+            }
+          } else {
+            float f[8];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              f[e] = __uint_as_float(__byte_perm(b03, kMagicBits, 0x7650 + e)) - vz;
+              f[4 + e] = __uint_as_float(__byte_perm(b47, kMagicBits, 0x7650 + e)) - vz;
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * e], f[2 * e + 1]);
+              o4[e] = *reinterpret_cast<const uint32_t*>(&h);
+            }
+          }
+        }
+        *reinterpret_cast<uint4*>(S.v + v_off[qi]) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+      }
+      fetch_v(j + 1);
+      fence_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&S.p_full));
+      return true;
+    };
+
+    bool ok = true;
+    for (int g = 0; g < 2 * nb && !*abort; ++g) {
+      // tile g & 1 was last read by the S MMAs of g - 2, whose result this thread has already waited for
+      const int ks = store_k(S.k[g & 1]);
+      if (kq == 0) S.col_term[g & 3][kkey] = -P.zq * ks;
+      fence_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&S.k_full[g & 1]));
+      kreg[0] = knext[0]; kreg[1] = knext[1];
+      if (g + 2 < 2 * nb) fetch_k((g + 2) % nb, knext);            // two blocks ahead: global latency is about one block
+      if (g > 0 && !process(g - 1)) { ok = false; break; }
+    }
+    if (ok && !*abort) ok = process(2 * nb - 1);
+
+    // ---------------------------------------------------------------- epilogue: one row per thread, the 16-column
+    // chunks of the accumulators split between warps 0..3 and 4..7
+    if (ok && !*abort && mbar_wait(smem_u32(&S.acc_full), 0, abort, 47, P.status)) {
+      tc_fence_after();
+      const float kSqrt2 = 1.41421356237309504880f;
+      const float zo_lo = float(-P.zo), zo_hi = float(P.qmax - P.zo);
+      const bool row_ok = row < P.Lq;
+      const int64_t roff = bo * P.o_so + bi * P.o_si + int64_t(row) * P.ldo;
+      const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(kAccCol);
+      const int n_c16 = P.dh >> 4, c_mid = (n_c16 + 1) >> 1;
+      const int c_begin = half ? c_mid * 16 : 0, c_end = half ? P.dh : c_mid * 16;
+      int code_sum = 0;
+      for (int c0 = c_begin; c0 < c_end; c0 += 16) {
+        uint32_t re[16], ro[16];
+        __syncwarp();
+        tmem_ld16(taddr + uint32_t(c0), re);
+        tmem_ld16(taddr + uint32_t(P.n_pad + c0), ro);
+        tmem_ld_wait();
+        float v[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) v[e] = P.out_scale * fmaf(kSqrt2, __uint_as_float(ro[e]), __uint_as_float(re[e]));
+        if (!row_ok) continue;
+        if (P.out_kind == REPQ_OUT_F32) {
+          float* o = static_cast<float*>(P.out) + roff + c0;
+          if (P.vec_store) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) reinterpret_cast<float4*>(o)[e] = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
+          } else {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) o[e] = v[e];
+          }
+        } else if (P.out_kind == REPQ_OUT_BF16) {
+          __nv_bfloat16* o = static_cast<__nv_bfloat16*>(P.out) + roff + c0;
+          if (P.vec_store) {
+            uint32_t w[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]);
+              w[e] = *reinterpret_cast<const uint32_t*>(&h);
+            }
+            reinterpret_cast<uint4*>(o)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+            reinterpret_cast<uint4*>(o)[1] = make_uint4(w[4], w[5], w[6], w[7]);
+          } else {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) o[e] = __float2bfloat16_rn(v[e]);
+          }
+        } else {
+          uint32_t q[16];
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const float tq = fminf(fmaxf(v[e] * P.inv_so, zo_lo), zo_hi);
+            q[e] = uint32_t(__float2int_rn(tq) + P.zo);
+            code_sum += int(q[e]);
+          }
+          uint8_t* orow = static_cast<uint8_t*>(P.out) + roff;
+          if (P.pack4) {
+            uint32_t w0 = 0u, w1 = 0u;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) { w0 |= q[e] << (4 * e); w1 |= q[8 + e] << (4 * e); }
+            if (P.vec_store) *reinterpret_cast<uint2*>(orow + (c0 >> 1)) = make_uint2(w0, w1);
+            else {
+#pragma unroll
+              for (int e = 0; e < 4; ++e) { orow[(c0 >> 1) + e] = uint8_t(w0 >> (8 * e)); orow[(c0 >> 1) + 4 + e] = uint8_t(w1 >> (8 * e)); }
+            }
+          } else {
+            uint32_t w[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) w[e] = q[4 * e] | (q[4 * e + 1] << 8) | (q[4 * e + 2] << 16) | (q[4 * e + 3] << 24);
+            if (P.vec_store) *reinterpret_cast<uint4*>(orow + c0) = make_uint4(w[0], w[1], w[2], w[3]);
+            else {
+#pragma unroll
+              for (int e = 0; e < 16; ++e) orow[c0 + e] = uint8_t(q[e]);
+            }
+          }
+        }
+      }
+      if (P.out_row_sum != nullptr && P.out_kind == REPQ_OUT_CODES && row_ok && c_begin < c_end)
+        atomicAdd(P.out_row_sum + int64_t(bo) * P.Lq + row, code_sum);
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == kWorkWarps) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(uint32_t(P.tmem_cols)) : "memory");
+  }
+}
+
+template <int NB, bool kLut>
+repq_status launch(const AttnParams& P, int64_t pairs, cudaStream_t st) {
+  const size_t smem = sizeof(AttnShared<NB>);
+  REPQ_CUDA(cudaFuncSetAttribute(attention_tc_kernel<NB, kLut>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+  dim3 grid((P.Lq + kRows - 1) / kRows, unsigned(pairs));
+  attention_tc_kernel<NB, kLut><<<grid, kThreads, smem, st>>>(P);
+  REPQ_CUDA(cudaGetLastError());
+  note_launch();
+  return REPQ_OK;
+}
+
+}  // namespace
+}  // namespace repq
+
+using namespace repq;
+
+extern "C" repq_status repq_attention(const repq_attention_desc* d, void* stream) {
+  REPQ_REQUIRE(d, REPQ_INVALID_ARG, "attention: NULL descriptor");
+  REPQ_REQUIRE(d->batch_outer > 0 && d->batch_inner > 0 && d->Lq >= 0 && d->Lk > 0 && d->d_h > 0, REPQ_INVALID_ARG, "attention: bad sizes");
+  if (d->Lq == 0) return REPQ_OK;
+  REPQ_REQUIRE(d->q_codes && d->k_codes && d->v_codes && d->out, REPQ_INVALID_ARG, "attention: NULL pointer");
+  REPQ_REQUIRE(bits_ok(d->bits_qkv) && bits_ok(d->bits_p), REPQ_INVALID_ARG, "attention: bits must be 4, 6 or 8");
+  REPQ_REQUIRE(!packed4(d->bits_qkv), REPQ_UNSUPPORTED, "attention: Q, K, V codes must be stored one per byte (REPQ_BYTE_CODES)");
+  REPQ_REQUIRE(d->d_h % 16 == 0 && d->d_h <= 128, REPQ_UNSUPPORTED, "attention: d_h = %d must be a multiple of 16, at most 128", d->d_h);
+  REPQ_REQUIRE(d->s_q > 0.f && d->s_k > 0.f && d->s_v > 0.f && d->s_p > 0.f && d->alpha > 0.f, REPQ_INVALID_ARG, "attention: scales must be positive");
+  REPQ_REQUIRE(!d->causal || d->Lk >= d->Lq, REPQ_INVALID_ARG, "attention: causal needs Lk >= Lq");
+  auto rows16 = [](const void* p, int64_t ld, int64_t so, int64_t si) { return aligned(p, 16) && ld % 16 == 0 && so % 16 == 0 && si % 16 == 0; };
+  REPQ_REQUIRE(rows16(d->q_codes, d->ldq_bytes, d->q_stride_outer, d->q_stride_inner) &&
+               rows16(d->k_codes, d->ldk_bytes, d->k_stride_outer, d->k_stride_inner), REPQ_ALIGNMENT,
+               "attention: Q and K rows must be 16-byte aligned");
+  REPQ_REQUIRE(aligned(d->v_codes, 8) && d->ldv_bytes % 8 == 0 && d->v_stride_outer % 8 == 0 && d->v_stride_inner % 8 == 0, REPQ_ALIGNMENT,
+               "attention: V rows must be 8-byte aligned");
+  REPQ_REQUIRE(d->ldq_bytes >= d->d_h && d->ldk_bytes >= d->d_h && d->ldv_bytes >= d->d_h, REPQ_INVALID_ARG, "attention: row stride shorter than d_h");
+  const int qmax_v = code_max(d->bits_qkv);
+  REPQ_REQUIRE(d->z_v >= qmax_v - 256 && d->z_v <= 256, REPQ_UNSUPPORTED, "attention: z_v = %d puts v - z_v outside [-256, 256]", d->z_v);
+  REPQ_REQUIRE(d->out_kind == REPQ_OUT_F32 || d->out_kind == REPQ_OUT_BF16 || d->out_kind == REPQ_OUT_CODES, REPQ_INVALID_ARG, "attention: unknown out_kind");
+  const int64_t esz = d->out_kind == REPQ_OUT_F32 ? 4 : d->out_kind == REPQ_OUT_BF16 ? 2 : 1;
+  REPQ_REQUIRE(aligned(d->out, size_t(esz)), REPQ_ALIGNMENT, "attention: out is not element-aligned");
+  const int64_t pairs = int64_t(d->batch_outer) * d->batch_inner;
+  REPQ_REQUIRE(pairs <= 65535, REPQ_UNSUPPORTED, "attention: more than 65535 (batch, head) pairs");
+  AttnParams P{};
+  P.q = d->q_codes; P.k = d->k_codes; P.v = d->v_codes;
+  P.ldq = d->ldq_bytes; P.ldk = d->ldk_bytes; P.ldv = d->ldv_bytes;
+  P.q_so = d->q_stride_outer; P.q_si = d->q_stride_inner; P.k_so = d->k_stride_outer; P.k_si = d->k_stride_inner;
+  P.v_so = d->v_stride_outer; P.v_si = d->v_stride_inner;
+  P.Lq = d->Lq; P.Lk = d->Lk; P.dh = d->d_h; P.batch_inner = d->batch_inner; P.causal = d->causal;
+  P.scale = d->alpha * d->s_q * d->s_k;
+  P.zq = d->z_q; P.zk = d->z_k;
+  P.log2_s = log2f(d->s_p);
+  P.qmax_p = code_max(d->bits_p);
+  P.z_v = d->z_v;
+  P.v_small = qmax_v < 128 && d->z_v > -128 && d->z_v < 128;
+  P.out_scale = d->s_p * d->s_v;
+  P.out_kind = d->out_kind;
+  if (d->out_kind == REPQ_OUT_CODES) {
+    REPQ_REQUIRE(bits_ok(d->out_bits) && d->out_scale > 0.f, REPQ_INVALID_ARG, "attention: bad output quantizer");
+    REPQ_REQUIRE(d->out_zero > -(1 << 20) && d->out_zero < (1 << 20), REPQ_INVALID_ARG, "attention: |out_zero| must be below 2^20");
+    P.qmax = code_max(d->out_bits); P.pack4 = packed4(d->out_bits); P.inv_so = 1.f / d->out_scale; P.zo = d->out_zero;
+  }
+  P.out = d->out; P.ldo = d->ldo; P.o_so = d->o_stride_outer; P.o_si = d->o_stride_inner;
+  P.out_row_sum = d->out_kind == REPQ_OUT_CODES ? d->out_row_sum : nullptr;
+  P.n_pad = (d->d_h + 15) / 16 * 16;
+  P.tmem_cols = 2 * kKeys + 2 * P.n_pad <= 256 ? 256 : 512;
+  const int64_t chunk_bytes = d->out_kind == REPQ_OUT_CODES && packed4(d->out_bits) ? 8 : 16 * esz;
+  const int64_t al = chunk_bytes < 16 ? chunk_bytes : 16;
+  P.vec_store = aligned(d->out, size_t(al)) && (d->ldo * esz) % al == 0 && (d->o_stride_outer * esz) % al == 0 &&
+                (d->o_stride_inner * esz) % al == 0;
+  P.status = device_status_word();
+  REPQ_REQUIRE(P.status != nullptr, REPQ_CUDA_ERROR, "attention: device status word unavailable");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const bool lut = P.qmax_p <= 15;
+  if (d->d_h <= 64) return lut ? launch<1, true>(P, pairs, st) : launch<1, false>(P, pairs, st);
+  return lut ? launch<2, true>(P, pairs, st) : launch<2, false>(P, pairs, st);
+}

@@ -148,6 +148,27 @@ static repq_status block_forward_impl(const repq_block_desc* dp, const repq_bloc
     REPQ_TRY(repq_qgemm(&g, gws, L.gemm_ws, stream));
   }
   REPQ_MARK();
+  if (!d.staged_attention) {
+    // scores, Softmax codes and P.V in one kernel; it takes the time slot of the scores stage, the two
+    // following stages are empty
+    REPQ_CUDA(cudaMemsetAsync(asum_attn, 0, size_t(M) * 4, st));
+    repq_attention_desc a{};
+    a.batch_outer = d.batch; a.batch_inner = H; a.Lq = S; a.Lk = S; a.d_h = dh; a.bits_qkv = ab;
+    a.q_codes = qkv_c; a.ldq_bytes = L.ld_qkv; a.q_stride_outer = int64_t(S) * L.ld_qkv; a.q_stride_inner = head_bytes;
+    a.s_q = p.s_q; a.z_q = p.z_q;
+    a.k_codes = qkv_c + code_row_bytes(D, ab); a.ldk_bytes = L.ld_qkv; a.k_stride_outer = a.q_stride_outer; a.k_stride_inner = head_bytes;
+    a.s_k = p.s_k; a.z_k = p.z_k;
+    a.v_codes = qkv_c + 2 * code_row_bytes(D, ab); a.ldv_bytes = L.ld_qkv; a.v_stride_outer = a.q_stride_outer; a.v_stride_inner = head_bytes;
+    a.s_v = p.s_v; a.z_v = p.z_v;
+    a.alpha = 1.f / sqrtf(float(dh)); a.causal = d.causal; a.bits_p = d.bits_p; a.s_p = p.softmax_s;
+    a.out_kind = REPQ_OUT_CODES; a.out_bits = ab; a.out_scale = p.s_attn; a.out_zero = p.z_attn;
+    a.out = attn_c; a.ldo = L.ld_a; a.o_stride_outer = int64_t(S) * L.ld_a; a.o_stride_inner = head_bytes;
+    a.out_row_sum = asum_attn;
+    REPQ_TRY(repq_attention(&a, stream));
+    REPQ_MARK();
+    REPQ_MARK();
+    REPQ_MARK();
+  } else {
   {
     // scores = Q K^T / sqrt(d_h) per (batch, head): both operands are activation codes
     repq_gemm_desc g{};
@@ -184,6 +205,7 @@ static repq_status block_forward_impl(const repq_block_desc* dp, const repq_bloc
     REPQ_TRY(repq_pv(&v, stream));
   }
   REPQ_MARK();
+  }
   {
     repq_gemm_desc g = linear_desc(d, M, D, D, attn_c, L.ld_a, p.s_attn, p.z_attn, asum_attn, p.proj);
     g.residual = x; g.residual_dtype = d.act_dtype; g.ld_residual = D;

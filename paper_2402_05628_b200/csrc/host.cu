@@ -50,7 +50,7 @@ extern "C" size_t repq_last_error(char* buf, size_t n) {
   return m.size();
 }
 
-extern "C" int repq_abi_version(void) { return 3; }
+extern "C" int repq_abi_version(void) { return 4; }
 
 extern "C" repq_status repq_scale_zero_from_bounds(int n, const float* x_low, const float* x_up,
                                                    int bits, float* s, int32_t* z) {

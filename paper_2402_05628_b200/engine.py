@@ -41,7 +41,8 @@ def _pack_linear(W: np.ndarray, bias: np.ndarray, bits_w: int, dev) -> PreparedL
 class QuantBlock:
     """Device-resident parameters of one block plus its workspace; `forward` runs the hot path."""
 
-    def __init__(self, w, device="cuda:0", out_dtype: Optional[torch.dtype] = None):
+    def __init__(self, w, device="cuda:0", out_dtype: Optional[torch.dtype] = None, staged_attention: bool = False):
+        self.staged_attention = bool(staged_attention)
         cfg = w.cfg
         self.cfg = cfg
         dev = torch.device(device)
@@ -84,6 +85,7 @@ class QuantBlock:
         d.causal, d.norm_kind, d.eps = int(c["causal"]), B.REPQ_NORM_LAYERNORM, c["eps"]
         d.act_dtype = B.REPQ_F32 if self.act_dtype == torch.float32 else B.REPQ_BF16
         d.out_dtype = B.REPQ_F32 if self.out_dtype == torch.float32 else B.REPQ_BF16
+        d.staged_attention = int(self.staged_attention)
         return d
 
     def params(self) -> B.BlockParams:

@@ -367,7 +367,7 @@ def check_pv(B_, H, Lq, Lk, dh, bits_p, bits_v, causal=False, out_kind="f32", ou
     return dict(rel_l2=rel, max_abs=mx)
 
 
-def check_block(name, batch, sample_items=None, out_dtype="f32", **overrides):
+def check_block(name, batch, sample_items=None, out_dtype="f32", staged_attention=False, **overrides):
     """Free-running block: the CUDA path (folded parameters, simple quantizers) against the oracle (complex
     quantizers) on the block output, for the sampled batch items (items are independent, Eqs. 1-3)."""
     import dataclasses
@@ -378,7 +378,7 @@ def check_block(name, batch, sample_items=None, out_dtype="f32", **overrides):
 
     w = make_block_inputs(name, batch=batch, **overrides)
     L = w.cfg["L"]
-    blk = QuantBlock(w, out_dtype=torch.float32 if out_dtype == "f32" else torch.bfloat16)
+    blk = QuantBlock(w, out_dtype=torch.float32 if out_dtype == "f32" else torch.bfloat16, staged_attention=staged_attention)
     x = torch.from_numpy(w.x).to(blk.device).to(blk.act_dtype)
     y = blk.forward(x)
     torch.cuda.synchronize()
@@ -487,3 +487,100 @@ def check_pv_uniform_codes(B_, H, L, dh, bits_p, bits_v, runs=10, seed=0):
             first = got
         assert np.array_equal(got, first), "launches differ"
     assert B.repq_device_status() == 0
+
+
+def check_attention(B_, H, Lq, Lk, dh, bits, bits_p, causal=False, out_kind="f32", out_bits=4 | BYTE_CODES, seed=0, s_p=1.0):
+    """repq_attention (scores, Softmax, log-sqrt2 codes and P.V fused) against the oracle's chain of the same
+    steps.  A Softmax code that sits on a rounding tie may legitimately differ by one (the near-tie protocol);
+    such a flip changes a whole output row, so rows that hold a near-tie are counted and left out of the strict
+    comparison."""
+    import torch
+    from oracle import repq_oracle as orc
+    from paper_2402_05628_b200 import binding as B
+
+    rng = np.random.default_rng(seed)
+    D = H * dh
+    nq = 1 << qb(bits)
+    Qc = rng.integers(0, nq, size=(B_ * Lq, D))
+    Kc = rng.integers(0, nq, size=(B_ * Lk, D))
+    Vc = rng.integers(0, nq, size=(B_ * Lk, D))
+    z_q, z_k, z_v = (int(rng.integers(0, nq)) for _ in range(3))
+    sig = (nq / 3.5) ** 2 * math.sqrt(dh)                 # rough std of sum (q - z_q)(k - z_k)
+    s_q = s_k = math.sqrt(3.0 * math.sqrt(dh) / sig)      # logits with a standard deviation of about 3
+    s_v = 0.05
+    alpha = 1.0 / math.sqrt(dh)
+    Qh, Kh, Vh = orc.dequant_uniform(Qc, s_q, z_q), orc.dequant_uniform(Kc, s_k, z_k), orc.dequant_uniform(Vc, s_v, z_v)
+    shift = Lk - Lq
+    valid = np.minimum(Lk, np.arange(Lq) + 1 + shift) if causal else np.full(Lq, Lk)
+    O_ref = np.empty((B_ * Lq, D))
+    absO = np.empty_like(O_ref)
+    tie_rows = np.zeros(B_ * Lq, dtype=bool)
+    for b in range(B_):
+        for h in range(H):
+            sl = slice(h * dh, (h + 1) * dh)
+            S = Qh[b * Lq:(b + 1) * Lq, sl] @ Kh[b * Lk:(b + 1) * Lk, sl].T * alpha
+            # the GPU forms S in float32 from the exact integer sum: do the same before the Softmax
+            S = S.astype(np.float32).astype(np.float64)
+            A = orc.softmax_rows(S, valid)
+            p, t = orc.quant_logsqrt2(A, s_p, qb(bits_p))
+            mask = np.arange(Lk)[None, :] < valid[:, None]
+            tf = np.where(mask & np.isfinite(t), t, 0.25)
+            near = mask & (np.abs(tf - np.floor(tf) - 0.5) < 2.0 ** -18 * np.maximum(1.0, np.abs(tf))) & (tf < min(2 ** qb(bits_p) - 0.4, 40.0))     # a flip below a weight of 2^-20 is invisible
+            tie_rows[b * Lq:(b + 1) * Lq] |= near.any(axis=1)
+            A_hat = np.where(mask, orc.dequant_logsqrt2(p, s_p), 0.0)
+            O_ref[b * Lq:(b + 1) * Lq, sl] = A_hat @ Vh[b * Lk:(b + 1) * Lk, sl]
+            absO[b * Lq:(b + 1) * Lq, sl] = A_hat @ np.abs(Vh[b * Lk:(b + 1) * Lk, sl])
+    dev = torch.device("cuda:0")
+    byte_bits = qb(bits) | BYTE_CODES
+    q_t = torch.from_numpy(Qc.astype(np.uint8)).to(dev)
+    k_t = torch.from_numpy(Kc.astype(np.uint8)).to(dev)
+    v_t = torch.from_numpy(Vc.astype(np.uint8)).to(dev)
+    d = B.AttentionDesc()
+    d.batch_outer, d.batch_inner, d.Lq, d.Lk, d.d_h, d.bits_qkv = B_, H, Lq, Lk, dh, byte_bits
+    d.q_codes, d.ldq_bytes, d.q_stride_outer, d.q_stride_inner, d.s_q, d.z_q = q_t.data_ptr(), D, Lq * D, dh, s_q, z_q
+    d.k_codes, d.ldk_bytes, d.k_stride_outer, d.k_stride_inner, d.s_k, d.z_k = k_t.data_ptr(), D, Lk * D, dh, s_k, z_k
+    d.v_codes, d.ldv_bytes, d.v_stride_outer, d.v_stride_inner, d.s_v, d.z_v = v_t.data_ptr(), D, Lk * D, dh, s_v, z_v
+    d.alpha, d.causal, d.bits_p, d.s_p = alpha, int(causal), bits_p, s_p
+    row_sum = None
+    if out_kind == "codes":
+        s_o, z_o = orc.uniform_scale_zero(np.percentile(O_ref, 1), np.percentile(O_ref, 99), qb(out_bits))
+        ldo = B.code_row_bytes(D, out_bits)
+        out = torch.full((B_ * Lq, ldo), 0xEE, dtype=torch.uint8, device=dev)
+        d.out_kind, d.out_bits, d.out_scale, d.out_zero = B.REPQ_OUT_CODES, out_bits, float(s_o), int(z_o)
+        d.ldo, d.o_stride_outer, d.o_stride_inner = ldo, Lq * ldo, (dh // 2 if out_bits == 4 else dh)
+        row_sum = torch.zeros(B_ * Lq, dtype=torch.int32, device=dev)
+        d.out_row_sum = row_sum.data_ptr()
+    else:
+        out = torch.zeros(B_ * Lq, D, dtype=torch.float32 if out_kind == "f32" else torch.bfloat16, device=dev)
+        d.out_kind = B.REPQ_OUT_F32 if out_kind == "f32" else B.REPQ_OUT_BF16
+        d.ldo, d.o_stride_outer, d.o_stride_inner = D, Lq * D, dh
+    d.out = out.data_ptr()
+    first = None
+    for _ in range(3):                                   # repeated launches must agree bit for bit
+        if row_sum is not None:
+            row_sum.zero_()
+        B.repq_attention(d)
+        torch.cuda.synchronize()
+        got_raw = out.cpu().numpy() if out_kind != "bf16" else out.float().cpu().numpy()
+        if first is None:
+            first = got_raw.copy()
+        assert np.array_equal(got_raw, first), "launches differ"
+    assert B.repq_device_status() == 0
+    keep = ~tie_rows
+    assert keep.mean() > 0.9, "too many rows with a Softmax code on a rounding tie: %.3f" % (1 - keep.mean())
+    if out_kind == "codes":
+        q_gpu = unpack_codes(first, D, out_bits)
+        q_ref, t_ref = orc.quant_uniform(O_ref, s_o, z_o, qb(out_bits))
+        delta = 2.0 ** -17 * absO / s_o + 2.0 ** -20 * np.abs(t_ref)
+        rep = near_tie_report(q_gpu[keep], q_ref[keep], t_ref[keep], delta[keep])
+        assert rep["bad"] == 0, rep
+        assert np.array_equal(row_sum.cpu().numpy().astype(np.int64), q_gpu.sum(axis=1))
+        return rep
+    got = first.astype(np.float64)
+    if out_kind == "bf16":
+        rel, _ = float_errors(got[keep], O_ref[keep])
+        assert rel < 6e-3, rel
+        return dict(rel_l2=rel)
+    rel, mx = assert_float_close(got[keep], O_ref[keep], "attention")
+    assert rel < 1e-4, rel                               # exact operands, float32 sums: far inside the tolerance
+    return dict(rel_l2=rel, max_abs=mx, tie_rows=int(tie_rows.sum()))

@@ -50,3 +50,9 @@ def test_block_c4_llama_shaped_full_size_sampled_item():
     # full LLaMA-7B-shaped layer (batch 4 x 2048 tokens, dim 4096, MLP 11008, causal, 8-bit log codes);
     # the oracle recomputes one batch item
     parity.check_block("c4_llama7b", batch=4, sample_items=(3,))
+
+
+def test_block_with_the_three_separate_attention_stages():
+    """The block through repq_qgemm (scores) -> repq_softmax_log2 -> repq_pv instead of the fused kernel."""
+    parity.check_block("c2_deit_b", batch=3, staged_attention=True)
+    parity.check_block("c4_llama7b", batch=2, D=512, H=4, MLP=1408, L=320, massive=2, staged_attention=True)

@@ -116,3 +116,19 @@ def test_pv_repeated_launches_reproduce_the_oracle(Bn, H, L, dh, bp, bv):
 ])
 def test_scores_from_byte_codes_match_oracle(Bn, H, Lq, Lk, dh, bits, causal):
     parity.check_scores(Bn, H, Lq, Lk, dh, bits, causal, seed=Lq + dh + 1)
+
+
+@pytest.mark.parametrize("Bn,H,Lq,Lk,dh,bits,bp,causal", [
+    (2, 3, 197, 197, 64, 4, 4, False), (1, 2, 577, 577, 64, 4, 4, False), (1, 2, 300, 300, 128, 4, 8, True),
+    (2, 2, 64, 64, 32, 6, 6, False), (1, 1, 1, 130, 16, 8, 8, False), (1, 2, 100, 260, 48, 4, 4, True),
+    (1, 1, 70, 70, 96, 8, 4, True), (1, 2, 700, 700, 64, 4, 4, True),
+])
+def test_fused_attention_matches_oracle(Bn, H, Lq, Lk, dh, bits, bp, causal):
+    parity.check_attention(Bn, H, Lq, Lk, dh, bits, bp, causal, seed=Lq + dh)
+
+
+def test_fused_attention_epilogues():
+    parity.check_attention(2, 2, 197, 197, 64, 4, 4, out_kind="bf16", seed=1)
+    parity.check_attention(2, 2, 197, 197, 64, 4, 4, out_kind="codes", out_bits=4 | parity.BYTE_CODES, seed=2)
+    parity.check_attention(1, 2, 130, 130, 128, 4, 8, causal=True, out_kind="codes", out_bits=8, seed=3, s_p=0.7)
+    parity.check_attention(1, 2, 130, 130, 64, 4, 4, out_kind="codes", out_bits=4, seed=4)

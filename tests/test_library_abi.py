@@ -29,7 +29,7 @@ def test_exports_match_header(B):
     for name in sorted(declared):
         assert hasattr(lib, name), "library does not export %s" % name
     assert declared == set(B.EXPORTS)
-    assert lib.repq_abi_version() == 3
+    assert lib.repq_abi_version() == 4
 
 
 def test_scale_zero_from_bounds_matches_oracle(B):
