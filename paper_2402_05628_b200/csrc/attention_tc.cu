@@ -2,7 +2,7 @@
 // P.V with the reparameterized log2 de-quantization (Eqs. 16-17) in one kernel.  Scores and codes never leave the
 // SM.  The code of a score depends on the row's final Softmax sum, so the keys are walked twice:
 //   pass 1   S = Q K^T per block of 64 keys (tcgen05.mma kind::i8 into tensor memory), running row maximum m and
-//            sum Z = sum 2^(c (S - m)) (each thread: one row, 32 of the 64 columns; the two partial results of a row
+//            sum Z = sum 2^(c (S - m)) (each thread: one row, 16 of the 64 columns; the four partial results of a row
 //            are merged once, after the pass)
 //   pass 2   S again, t = 2 (log2 Z + log2 s) - 2 c (S - m), code p = clip(round(t), 0, 2^b - 1), operand values
 //            2^(-ceil(p/2)) split by the parity of p into the tiles E and O (exact bf16 powers of two), V as exact bf16
@@ -12,9 +12,10 @@
 // for Z), so the codes agree with theirs except where the differently ordered sum Z moves a value across a
 // rounding tie.
 //
-// One CTA owns 128 query rows of one (batch, head) pair.  Warps 0..7: K tiles and V tiles from registers (fetched one
+// One CTA owns 128 query rows of one (batch, head) pair.  Warps 0..15 (four per tensor-memory lane quarter: a thread
+// has one row and 16 of the 64 columns of a key block): K tiles and V tiles from registers (fetched one
 // block ahead) into 128-byte-swizzled shared-memory tiles, the Softmax arithmetic, the E / O tiles, the epilogue.
-// Warp 8 (one lane): tensor-memory allocation and MMA issue.  S is double-buffered in tensor memory (2 x 64 columns),
+// Warp 16 (one lane): tensor-memory allocation and MMA issue.  S is double-buffered in tensor memory (2 x 64 columns),
 // the E / O / V tiles are single (their block's code arithmetic overlaps the MMAs of the block before).  Under a causal mask, key blocks no row of the CTA may see are
 // skipped.  Every mbarrier wait is bounded; when one runs out the kernel records a status code, all roles leave
 // their loops, MMAs in flight are drained, tensor memory is freed and the kernel returns.
@@ -33,7 +34,9 @@ using namespace tc;
 
 constexpr int kRows = 128;                  // query rows per CTA (MMA M)
 constexpr int kKeys = 64;                   // keys per block
-constexpr int kWorkWarps = 8;
+constexpr int kWorkWarps = 16;                // 4 per tensor-memory lane quarter: a row's 64 columns are split 4 ways
+constexpr int kParts = kWorkWarps / 4;
+constexpr int kCols = kKeys / kParts;         // S columns per thread and key block
 constexpr int kWorkThreads = 32 * kWorkWarps;
 constexpr int kThreads = kWorkThreads + 32;
 constexpr uint32_t kQBytes = kRows * 128;         // Q tile: rows of 128 bytes (the head's codes, zero-padded)
@@ -70,7 +73,7 @@ struct AttnShared {
   alignas(1024) uint8_t v[NB * kVBlockBytes];
   int row_term[kRows];                              // -z_k qsum[m] + d_h z_q z_k
   int col_term[4][kKeys];                           // -z_q ksum[n], ring of 4 key blocks
-  float stat_m[2][kRows], stat_z[2][kRows];         // pass-1 results of the two column halves of every row
+  float stat_m[kParts][kRows], stat_z[kParts][kRows];   // pass-1 results of the column parts of every row
   uint32_t lut[16][32];                             // 4-bit codes: [code][lane] = E value | O value << 16 (one bank per lane)
   alignas(8) uint64_t k_full[2];
   uint64_t s_full[2], s_empty[2], p_full, p_empty;
@@ -96,7 +99,7 @@ template <int NB, bool kLut>
 __global__ void __launch_bounds__(kThreads, NB == 1 ? 2 : 1)
 attention_tc_kernel(AttnParams P) {
   using Shared = AttnShared<NB>;
-  constexpr int kVItems = 2 * NB;                         // 8-channel groups of V per thread and block
+  constexpr int kVItems = NB;                             // 8-channel groups of V per thread and block
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   Shared& S = *reinterpret_cast<Shared*>(smem_raw);
 
@@ -134,28 +137,21 @@ attention_tc_kernel(AttnParams P) {
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
 
-  // ---- K rows: 4 threads per key, 2 pieces each; Q rows: 2 threads per row, 4 pieces each
+  // ---- K rows: 8 threads per key, one 16-byte piece each; Q rows: 4 threads per row, 2 pieces each
   const uint8_t* k_base = P.k + bo * P.k_so + bi * P.k_si;
-  const int kkey = (tid >> 2) & (kKeys - 1), kq = tid & 3;
-  uint4 kreg[2], knext[2];                      // the K rows of the next two key blocks
-  auto fetch_k = [&](int block, uint4 (&dst)[2]) {
-#pragma unroll
-    for (int j = 0; j < 2; ++j) {
-      dst[j] = make_uint4(0u, 0u, 0u, 0u);
-      const int piece = 2 * kq + j, key = block * kKeys + kkey;
-      if (key < P.Lk && piece < pieces) dst[j] = __ldg(reinterpret_cast<const uint4*>(k_base + int64_t(key) * P.ldk) + piece);
-    }
+  const int kkey = (tid >> 3) & (kKeys - 1), kq = tid & 7;
+  uint4 kreg, knext;                            // the thread's piece of the K rows of the next two key blocks
+  auto fetch_k = [&](int block, uint4& dst) {
+    dst = make_uint4(0u, 0u, 0u, 0u);
+    const int key = block * kKeys + kkey;
+    if (key < P.Lk && kq < pieces) dst = __ldg(reinterpret_cast<const uint4*>(k_base + int64_t(key) * P.ldk) + kq);
   };
   auto store_k = [&](uint8_t* tile) {            // returns the code sum of the thread's key
-    int s = 0;
-#pragma unroll
-    for (int j = 0; j < 2; ++j) {
-      const int piece = 2 * kq + j;
-      if (piece < 2 * ksteps) *reinterpret_cast<uint4*>(tile + tile_offset(kkey, piece)) = kreg[j];
-      s += sum_bytes(kreg[j]);
-    }
+    if (kq < 2 * ksteps) *reinterpret_cast<uint4*>(tile + tile_offset(kkey, kq)) = kreg;
+    int s = sum_bytes(kreg);
     s += __shfl_xor_sync(0xffffffffu, s, 1);
     s += __shfl_xor_sync(0xffffffffu, s, 2);
+    s += __shfl_xor_sync(0xffffffffu, s, 4);
     return s;
   };
 
@@ -163,17 +159,18 @@ attention_tc_kernel(AttnParams P) {
     fetch_k(0, kreg);
     fetch_k(nb > 1 ? 1 : 0, knext);
     const uint8_t* q_base = P.q + bo * P.q_so + bi * P.q_si;
-    const int qrow = (tid >> 1) & (kRows - 1), qh = tid & 1;
+    const int qrow = (tid >> 2) & (kRows - 1), qh = tid & 3;
     int s = 0;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int piece = 4 * qh + j;
+    for (int j = 0; j < 2; ++j) {
+      const int piece = 2 * qh + j;
       uint4 w = make_uint4(0u, 0u, 0u, 0u);
       if (q0 + qrow < P.Lq && piece < pieces) w = __ldg(reinterpret_cast<const uint4*>(q_base + int64_t(q0 + qrow) * P.ldq) + piece);
       if (piece < 2 * ksteps) *reinterpret_cast<uint4*>(S.q + tile_offset(qrow, piece)) = w;
       s += sum_bytes(w);
     }
     s += __shfl_xor_sync(0xffffffffu, s, 1);
+    s += __shfl_xor_sync(0xffffffffu, s, 2);
     if (qh == 0) S.row_term[qrow] = -P.zk * s + P.dh * P.zq * P.zk;
     for (int i = tid; i < 16 * 32; i += kWorkThreads) {
       const uint32_t code = uint32_t(i >> 5), bits16 = (127u - ((code + 1u) >> 1)) << 7;      // bf16 bits of 2^-ceil(code/2)
@@ -231,7 +228,7 @@ attention_tc_kernel(AttnParams P) {
     }
   } else {
     // ---------------------------------------------------------------- tiles, Softmax arithmetic, epilogue
-    const int quarter = warp & 3, half = warp >> 2;
+    const int quarter = warp & 3, part = warp >> 2;       // lane quarter of tensor memory, column part of the row
     const int r = quarter * 32 + lane;                    // the thread's row inside the CTA = its tensor-memory lane
     const int row = q0 + r;
     const int valid = row < P.Lq ? (P.causal ? max(1, min(P.Lk, row + 1 + shift)) : P.Lk) : 0;   // keys the row sees
@@ -240,7 +237,7 @@ attention_tc_kernel(AttnParams P) {
     const float k1 = -2.f * c;
     const float fq = float(P.qmax_p);
     const float magic = __uint_as_float(kMagicBits);
-    const uint32_t taddr_s = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(half * 32);
+    const uint32_t taddr_s = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(part * kCols);
 
     // V items of a block (as in the P.V kernel): 2 NB groups of 8 channels per thread
     const uint8_t* v_ptr[kVItems];
@@ -270,36 +267,34 @@ attention_tc_kernel(AttnParams P) {
     float m = -CUDART_INF_F, z = 0.f;       // pass 1: running maximum and sum of this thread's columns
     float k0 = 0.f;                         // pass 2: 2 (log2 Z + log2 s), with m the row's final maximum
 
-    // corr = acc - z_k qsum - z_q ksum + d_h z_q z_k of the thread's 32 columns of key block j (buffer g & 1), as
+    // corr = acc - z_k qsum - z_q ksum + d_h z_q z_k of the thread's 16 columns of key block j (buffer g & 1), as
     // integers; keys the row may not see become kMasked.  Frees the buffer as soon as it is read.
     constexpr int kMasked = -2147483647 - 1;
-    auto read_s = [&](int g, int j, int (&corr)[32]) -> bool {
+    auto read_s = [&](int g, int j, int (&corr)[kCols]) -> bool {
       const int b = g & 1;
       if (!mbar_wait(smem_u32(&S.s_full[b]), uint32_t(g >> 1) & 1u, abort, 44, P.status)) return false;
       tc_fence_after();
-      uint32_t r0[16], r1[16];
+      uint32_t r0[16];
       __syncwarp();
       tmem_ld16(taddr_s + uint32_t(b * kKeys), r0);
-      tmem_ld16(taddr_s + uint32_t(b * kKeys + 16), r1);
       tmem_ld_wait();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&S.s_empty[b]));
-      const int* ct = S.col_term[g & 3] + half * 32;
+      const int* ct = S.col_term[g & 3] + part * kCols;
 #pragma unroll
-      for (int e4 = 0; e4 < 8; ++e4) {
+      for (int e4 = 0; e4 < kCols / 4; ++e4) {
         const int4 c4 = *reinterpret_cast<const int4*>(ct + 4 * e4);
-        const uint32_t* rr = e4 < 4 ? &r0[4 * e4] : &r1[4 * (e4 - 4)];
-        corr[4 * e4 + 0] = int32_t(rr[0]) + my_row_term + c4.x;
-        corr[4 * e4 + 1] = int32_t(rr[1]) + my_row_term + c4.y;
-        corr[4 * e4 + 2] = int32_t(rr[2]) + my_row_term + c4.z;
-        corr[4 * e4 + 3] = int32_t(rr[3]) + my_row_term + c4.w;
+        corr[4 * e4 + 0] = int32_t(r0[4 * e4 + 0]) + my_row_term + c4.x;
+        corr[4 * e4 + 1] = int32_t(r0[4 * e4 + 1]) + my_row_term + c4.y;
+        corr[4 * e4 + 2] = int32_t(r0[4 * e4 + 2]) + my_row_term + c4.z;
+        corr[4 * e4 + 3] = int32_t(r0[4 * e4 + 3]) + my_row_term + c4.w;
       }
       // causal mask and keys past Lk: only in blocks that reach past the fewest keys any row of the CTA sees
-      const int key0 = j * kKeys + half * 32;
-      if (__builtin_expect(key0 + 32 > min(min_valid, valid), 0)) {
+      const int key0 = j * kKeys + part * kCols;
+      if (__builtin_expect(key0 + kCols > min(min_valid, valid), 0)) {
 #pragma unroll
-        for (int e = 0; e < 32; ++e)
+        for (int e = 0; e < kCols; ++e)
           if (key0 + e >= valid) corr[e] = kMasked;
       }
       return true;
@@ -307,19 +302,19 @@ attention_tc_kernel(AttnParams P) {
 
     auto process = [&](int g) -> bool {
       const int j = g < nb ? g : g - nb;
-      int corr[32];
+      int corr[kCols];
       if (!read_s(g, j, corr)) return false;
       if (g < nb) {
         // ---- pass 1: running maximum and sum.  The maximum is taken on the integers (S = scale * float(corr) is
         // monotonic in corr); a masked key contributes 2^(-huge) = 0.
         int bmi = corr[0];
 #pragma unroll
-        for (int e = 1; e < 32; ++e) bmi = max(bmi, corr[e]);
+        for (int e = 1; e < kCols; ++e) bmi = max(bmi, corr[e]);
         if (bmi != kMasked) {
           const float mn = fmaxf(m, P.scale * float(bmi));
           float acc0 = 0.f, acc1 = 0.f;
 #pragma unroll
-          for (int e = 0; e < 32; e += 2) {
+          for (int e = 0; e < kCols; e += 2) {
             acc0 += ex2(fmaf(float(corr[e]), P.scale, -mn) * c);
             acc1 += ex2(fmaf(float(corr[e + 1]), P.scale, -mn) * c);
           }
@@ -327,17 +322,22 @@ attention_tc_kernel(AttnParams P) {
           m = mn;
         }
         if (g == nb - 1) {
-          // merge the two halves of every row: m = max, Z = sum of the rescaled partial sums
-          S.stat_m[half][r] = m;
-          S.stat_z[half][r] = z;
+          // merge the column parts of every row: m = max, Z = sum of the rescaled partial sums (same order in
+          // every thread of the row, so that all of them hold the same Z)
+          S.stat_m[part][r] = m;
+          S.stat_z[part][r] = z;
           __syncwarp();
           if (lane == 0) mbar_arrive(smem_u32(&S.stats_ready));
           if (!mbar_wait(smem_u32(&S.stats_ready), 0, abort, 45, P.status)) return false;
-          const float m2 = S.stat_m[half ^ 1][r], z2 = S.stat_z[half ^ 1][r];
-          const float mn = fmaxf(m, m2);
+          float mn = -CUDART_INF_F;
+#pragma unroll
+          for (int q = 0; q < kParts; ++q) mn = fmaxf(mn, S.stat_m[q][r]);
           float zt = 0.f;
-          if (m > -CUDART_INF_F) zt += z * ex2((m - mn) * c);
-          if (m2 > -CUDART_INF_F) zt += z2 * ex2((m2 - mn) * c);
+#pragma unroll
+          for (int q = 0; q < kParts; ++q) {
+            const float mq = S.stat_m[q][r];
+            if (mq > -CUDART_INF_F) zt += S.stat_z[q][r] * ex2((mq - mn) * c);
+          }
           m = mn;
           k0 = 2.f * (log2f(zt) + P.log2_s);
           fetch_v(0);
@@ -349,11 +349,11 @@ attention_tc_kernel(AttnParams P) {
       // 1.5 * 2^23, which leaves p in the low mantissa bits u - kMagicBits.  The pair (E, O) of bf16 operand values,
       // 2^-ceil(p/2) on the side of p's parity and 0 on the other, comes from a per-lane table for 4-bit codes and
       // from integer arithmetic for wider ones.  A masked key gets (0, 0).
-      const bool boundary = j * kKeys + half * 32 + 32 > min(min_valid, valid);
+      const bool boundary = j * kKeys + part * kCols + kCols > min(min_valid, valid);
       const uint32_t lut_addr = smem_u32(&S.lut[0][lane]) - (kMagicBits << 7);
-      uint32_t eo[32];
+      uint32_t eo[kCols];
 #pragma unroll
-      for (int e = 0; e < 32; ++e) {
+      for (int e = 0; e < kCols; ++e) {
         // clamped on both sides whatever the inputs (rows past Lq carry m = -inf, Z = 0): p indexes the table
         const float t = fmaxf(fminf(fmaf(fmaf(float(corr[e]), P.scale, -m), k1, k0), fq), 0.f);
         const uint32_t u = __float_as_uint(t + magic);
@@ -367,12 +367,12 @@ attention_tc_kernel(AttnParams P) {
       }
       if (__builtin_expect(boundary, 0)) {
 #pragma unroll
-        for (int e = 0; e < 32; ++e)
+        for (int e = 0; e < kCols; ++e)
           if (corr[e] == kMasked) eo[e] = 0u;
       }
-      uint4 ev[4], ov[4];
+      uint4 ev[kCols / 8], ov[kCols / 8];
 #pragma unroll
-      for (int p4 = 0; p4 < 4; ++p4) {
+      for (int p4 = 0; p4 < kCols / 8; ++p4) {
         ev[p4] = make_uint4(__byte_perm(eo[8 * p4 + 0], eo[8 * p4 + 1], 0x5410), __byte_perm(eo[8 * p4 + 2], eo[8 * p4 + 3], 0x5410),
                             __byte_perm(eo[8 * p4 + 4], eo[8 * p4 + 5], 0x5410), __byte_perm(eo[8 * p4 + 6], eo[8 * p4 + 7], 0x5410));
         ov[p4] = make_uint4(__byte_perm(eo[8 * p4 + 0], eo[8 * p4 + 1], 0x7632), __byte_perm(eo[8 * p4 + 2], eo[8 * p4 + 3], 0x7632),
@@ -382,8 +382,8 @@ attention_tc_kernel(AttnParams P) {
       // has overlapped with those MMAs)
       if (!mbar_wait(smem_u32(&S.p_empty), (uint32_t(j) & 1u) ^ 1u, abort, 46, P.status)) return false;
 #pragma unroll
-      for (int p4 = 0; p4 < 4; ++p4) {
-        const uint32_t off = tile_offset(r, half * 4 + p4);
+      for (int p4 = 0; p4 < kCols / 8; ++p4) {
+        const uint32_t off = tile_offset(r, part * (kCols / 8) + p4);
         *reinterpret_cast<uint4*>(S.e + off) = ev[p4];
         *reinterpret_cast<uint4*>(S.o + off) = ov[p4];
       }
@@ -432,14 +432,14 @@ attention_tc_kernel(AttnParams P) {
       fence_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&S.k_full[g & 1]));
-      kreg[0] = knext[0]; kreg[1] = knext[1];
+      kreg = knext;
       if (g + 2 < 2 * nb) fetch_k((g + 2) % nb, knext);            // two blocks ahead: global latency is about one block
       if (g > 0 && !process(g - 1)) { ok = false; break; }
     }
     if (ok && !*abort) ok = process(2 * nb - 1);
 
     // ---------------------------------------------------------------- epilogue: one row per thread, the 16-column
-    // chunks of the accumulators split between warps 0..3 and 4..7
+    // chunks of the accumulators dealt to the four warps of a lane quarter
     if (ok && !*abort && mbar_wait(smem_u32(&S.acc_full), 0, abort, 47, P.status)) {
       tc_fence_after();
       const float kSqrt2 = 1.41421356237309504880f;
@@ -447,10 +447,8 @@ attention_tc_kernel(AttnParams P) {
       const bool row_ok = row < P.Lq;
       const int64_t roff = bo * P.o_so + bi * P.o_si + int64_t(row) * P.ldo;
       const uint32_t taddr = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(kAccCol);
-      const int n_c16 = P.dh >> 4, c_mid = (n_c16 + 1) >> 1;
-      const int c_begin = half ? c_mid * 16 : 0, c_end = half ? P.dh : c_mid * 16;
       int code_sum = 0;
-      for (int c0 = c_begin; c0 < c_end; c0 += 16) {
+      for (int c0 = part * 16; c0 < P.dh; c0 += kParts * 16) {      // the 16-column chunks of the accumulators, dealt to the parts
         uint32_t re[16], ro[16];
         __syncwarp();
         tmem_ld16(taddr + uint32_t(c0), re);
@@ -514,7 +512,7 @@ attention_tc_kernel(AttnParams P) {
           }
         }
       }
-      if (P.out_row_sum != nullptr && P.out_kind == REPQ_OUT_CODES && row_ok && c_begin < c_end)
+      if (P.out_row_sum != nullptr && P.out_kind == REPQ_OUT_CODES && row_ok && part * 16 < P.dh)
         atomicAdd(P.out_row_sum + int64_t(bo) * P.Lq + row, code_sum);
     }
   }
