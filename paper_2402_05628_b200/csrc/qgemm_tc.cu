@@ -355,7 +355,8 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     const EpilogueParams& ep = P.ep;
     const int kza = P.K * ep.z_a;
     const bool res16 = ep.residual != nullptr && ep.residual_bf16;
-    const bool fast_ok = ep.acc_debug == nullptr && (ep.residual == nullptr || res16);
+    const bool res32 = ep.residual != nullptr && !ep.residual_bf16;
+    const bool fast_ok = ep.acc_debug == nullptr;
     // per-column terms (threads 0..BN-1: column et of the tile) and the row's code sum, fetched one tile ahead
     int nx_nzw = 0, nx_kw = 0, nx_asum = 0;
     float nx_sc = 0.f, nx_bi = 0.f;
@@ -440,6 +441,15 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
           if (ep.gelu) {
 #pragma unroll
             for (int e = 0; e < kChunk; ++e) v[e] = gelu_erf(v[e]);
+          }
+          if (res32 && row_ok) {
+            // float32 residual: read where it is used (16 columns = four 16-byte loads of this thread's row)
+            const float4* rp = reinterpret_cast<const float4*>(static_cast<const float*>(ep.residual) + m * ep.ld_residual + col0);
+#pragma unroll
+            for (int i = 0; i < kChunk / 4; ++i) {
+              const float4 r4 = __ldg(rp + i);
+              v[4 * i] += r4.x; v[4 * i + 1] += r4.y; v[4 * i + 2] += r4.z; v[4 * i + 3] += r4.w;
+            }
           }
           if (res16 && row_ok) {
 #pragma unroll
