@@ -39,15 +39,16 @@ ATTENTION_INSTR_PER_SCORE = 23
 # sources still hash to what was captured; otherwise `traffic` is null.
 NCU_TRAFFIC_WORKLOAD = ("c2_deit_b", 64)
 NCU_TRAFFIC = {   # stage: (DRAM bytes read + written per launch, kernel sources, their sha1 when captured)
-    'ln1': (19390000, ['ln_quant.cu', 'f32x2.cuh'], 'f7a75aeecd3f'),
-    'ln2': (19390000, ['ln_quant.cu', 'f32x2.cuh'], 'f7a75aeecd3f'),
-    'qkv': (14150000, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '288dde775815'),
-    'scores': (88310000, ['scores_tc.cu', 'tc_ptx.cuh'], '6d7463c0b75f'),
-    'softmax': (129705000, ['softmax_log2.cu', 'f32x2.cuh'], '56dfe4bea2f6'),
-    'pv': (26712048, ['pv_tc.cu', 'tc_ptx.cuh'], '32a9d7c4307a'),
-    'proj': (33901000, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '288dde775815'),
-    'fc1': (20387000, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '288dde775815'),
-    'fc2': (82620000, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '288dde775815'),
+    'ln1': (19392768, ['ln_quant.cu', 'f32x2.cuh'], '9869074ea6b9'),
+    'ln2': (19392768, ['ln_quant.cu', 'f32x2.cuh'], '9869074ea6b9'),
+    'qkv': (14875648, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '470d458babdd'),
+    'attention': (29183744, ['attention_tc.cu', 'tc_ptx.cuh'], 'eda123b891cd'),
+    'scores': (85920512, ['scores_tc.cu', 'tc_ptx.cuh'], '56c4b8afa690'),
+    'softmax': (130385920, ['softmax_log2.cu', 'f32x2.cuh'], '45f5e16c2857'),
+    'pv': (26710528, ['pv_tc.cu', 'tc_ptx.cuh'], '7d458ef14cde'),
+    'proj': (33147392, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '470d458babdd'),
+    'fc1': (21291008, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '470d458babdd'),
+    'fc2': (83022592, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '470d458babdd'),
 }
 
 
