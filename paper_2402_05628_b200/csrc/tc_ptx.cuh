@@ -35,11 +35,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 
 // Bounded wait: false if the wait ran out (status word := code, abort flag raised) or another role of the
-// CTA already gave up.
+// CTA already gave up.  The retry loop is kept to the try_wait and its branch; the clock and the abort flag are
+// looked at once every kTriesPerCheck failed tries (waiting warps share issue slots with working ones).
+constexpr int kTriesPerCheck = 32;
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort, int code, int32_t* status) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
-  while (!mbar_try_wait(bar, parity)) {
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < kTriesPerCheck; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
     if (*abort) return false;
     if (clock64() - t0 > kWaitCycles) {
       atomicCAS(status, 0, code);
@@ -47,7 +52,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       return false;
     }
   }
-  return true;
 }
 
 // Wait without side effects, for draining copies or MMAs that are still in flight before the CTA exits.
