@@ -51,11 +51,11 @@ constexpr uint32_t kMagicBits = 0x4B400000u;         // 1.5 * 2^23
 
 __device__ int32_t g_status_word = 0;
 
-struct alignas(16) ColTerms {                          // per output column, staged once per tile
-  int32_t nzw[kMaxBN];  // -z_w[j]
-  int32_t kw[kMaxBN];   // -z_a * wsum[j]
-  float sc[kMaxBN];     // alpha s_a s_w[j]   (times 1/s_o in direct re-quantization mode)
-  float bi[kMaxBN];     // bias[j]            (times 1/s_o in direct re-quantization mode)
+struct alignas(16) ColTerms {                          // per output column of a warp's slice, staged once per tile
+  int32_t nzw[kSliceCols];  // -z_w[j]
+  int32_t kw[kSliceCols];   // -z_a * wsum[j]
+  float sc[kSliceCols];     // alpha s_a s_w[j]   (times 1/s_o in direct re-quantization mode)
+  float bi[kSliceCols];     // bias[j]            (times 1/s_o in direct re-quantization mode)
 };
 
 template <int BN>
@@ -63,12 +63,11 @@ struct SharedStorage {
   alignas(1024) uint8_t a[kStages][kABytes];
   alignas(1024) uint8_t b[kStages][BN * BK];
   alignas(1024) uint8_t epi[kEpiWarps][1024];     // per-warp staging box of the epilogue's bulk stores
-  ColTerms cols[2];
+  ColTerms cols[kEpiWarps];                       // each epilogue warp stages the terms of its own slice: no barrier
   alignas(8) uint64_t full[kStages];
   uint64_t empty[kStages];
   uint64_t tmem_full[2];
   uint64_t tmem_empty[2];
-  uint64_t cols_ready[2];
   uint64_t done;
   uint32_t tmem_base;
   volatile int abort;
@@ -104,6 +103,8 @@ struct ChunkQuant {
   uint32_t pack_k;     // 4-bit: sum_e (magic_bits - z_o) << 4e
   uint32_t z4;         // 8-bit: z_o replicated in every byte
   int zo;
+  float inv_qs, qs, csat;   // byte codes of at most 7 bits: 1 / 2^bits, 2^bits, (z_o - magic) / 2^bits
+  int qs_shift;             //   bits
 };
 
 __device__ __forceinline__ ChunkQuant chunk_quant(const EpilogueParams& ep, const TcParams& P, int col0) {
@@ -117,6 +118,10 @@ __device__ __forceinline__ ChunkQuant chunk_quant(const EpilogueParams& ep, cons
   q.pack_k = (kMagicBits - uint32_t(zo)) * 0x11111111u;
   q.z4 = (uint32_t(zo) & 0xFFu) * 0x01010101u;
   q.zo = zo;
+  q.qs_shift = 32 - __clz(ep.qmax);                      // qmax = 2^bits - 1
+  q.qs = __uint_as_float(uint32_t(127 + q.qs_shift) << 23);         // 2^bits
+  q.inv_qs = __uint_as_float(uint32_t(127 - q.qs_shift) << 23);     // 2^-bits
+  q.csat = (float(zo) - __uint_as_float(kMagicBits)) * q.inv_qs;    // exact: an integer below 2^24 times a power of two
   return q;
 }
 
@@ -147,6 +152,11 @@ __device__ __forceinline__ uint32_t box_slot(uint32_t buf, int lane, int j) {
 __device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
+__device__ __forceinline__ float fma_sat(float a, float b, float c) {       // fma clamped to [0, 1]
+  float d;
+  asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 __device__ __forceinline__ void sts64(uint32_t addr, uint32_t a, uint32_t b) {
   asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(addr), "r"(a), "r"(b) : "memory");
 }
@@ -156,7 +166,7 @@ __device__ __forceinline__ void sts64(uint32_t addr, uint32_t a, uint32_t b) {
 // chunk (f32), one per two chunks (byte codes) or one per slice (4-bit codes).
 template <int OUT>
 __device__ __forceinline__ void emit_chunk(const CUtensorMap* map_out, uint32_t buf, int lane, const ChunkQuant& q,
-                                           float (&v)[kChunk], int c, int col0, int row0, int& code_sum) {
+                                           float (&v)[kChunk], int c, int col0, int row0, int& code_sum, bool direct, bool sat) {
   if constexpr (OUT == kOutF32) {
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
@@ -181,6 +191,30 @@ __device__ __forceinline__ void emit_chunk(const CUtensorMap* map_out, uint32_t 
   } else {
     const float magic = __uint_as_float(kMagicBits);
     uint32_t u[kChunk];
+    if (OUT == kOutC8 && sat) {
+      // Byte codes of at most 7 bits, no comparisons: r = magic + round_half_even(t) by the float adder (one fma
+      // from the value when the scale is still to be applied), w = clamp((r - magic + z_o) / 2^bits, 0, 1) by a
+      // saturating fma whose unclamped result is exact, u = magic + 2^bits w.  The low byte of u is the code,
+      // except that 2^bits stands for the top code 2^bits - 1; that bit is subtracted after packing.
+      uint32_t w[4];
+      if (direct) {
+#pragma unroll
+        for (int e = 0; e < kChunk; ++e) u[e] = __float_as_uint(fmaf(fma_sat(v[e] + magic, q.inv_qs, q.csat), q.qs, magic));
+      } else {
+#pragma unroll
+        for (int e = 0; e < kChunk; ++e) u[e] = __float_as_uint(fmaf(fma_sat(fmaf(v[e], q.mult, magic), q.inv_qs, q.csat), q.qs, magic));
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t p = __byte_perm(__byte_perm(u[4 * i], u[4 * i + 1], 0x0040), __byte_perm(u[4 * i + 2], u[4 * i + 3], 0x0040), 0x5410);
+        w[i] = p - ((p >> q.qs_shift) & 0x01010101u);
+        code_sum += __dp4a(w[i], 0x01010101u, 0u);
+      }
+      if ((c & 1) == 0) box_begin(lane);
+      sts128(box_slot(buf, lane, c & 1), w[0], w[1], w[2], w[3]);
+      if (c & 1) box_end(map_out, buf, lane, col0 - kChunk, row0);
+      return;
+    }
 #pragma unroll
     for (int e = 0; e < kChunk; ++e) {
       const float t = fminf(fmaxf(v[e] * q.mult, q.lo), q.hi);
@@ -271,7 +305,6 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&S.full[s]), 1); mbar_init(smem_u32(&S.empty[s]), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&S.tmem_full[a]), 1); mbar_init(smem_u32(&S.tmem_empty[a]), kEpiWarps); }
-    for (int a = 0; a < 2; ++a) mbar_init(smem_u32(&S.cols_ready[a]), kEpiThreads);
     mbar_init(smem_u32(&S.done), 1);
     S.abort = 0;
     if (smem_u32(smem_raw) & 1023u) {              // the swizzled tiles need the alignment asked for above
@@ -351,35 +384,34 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     const int quarter = warp & 3;                // TMEM lane quarter this warp may read
     const int slice = ew >> 2;                   // which 64 accumulator columns
     const bool slice_on = slice * kSliceCols < BN;
-    const int et = threadIdx.x - 64;             // 0..511 among epilogue threads
     const EpilogueParams& ep = P.ep;
     const int kza = P.K * ep.z_a;
     const bool res16 = ep.residual != nullptr && ep.residual_bf16;
     const bool res32 = ep.residual != nullptr && !ep.residual_bf16;
     const bool fast_ok = ep.acc_debug == nullptr;
-    // per-column terms (threads 0..BN-1: column et of the tile) and the row's code sum, fetched one tile ahead
-    int nx_nzw = 0, nx_kw = 0, nx_asum = 0;
-    float nx_sc = 0.f, nx_bi = 0.f;
+    const bool sat = ep.qmax <= 127;             // byte codes narrow enough for the comparison-free quantizer
+    const bool direct = P.direct_requant != 0;
+    const int cl0 = slice * kSliceCols;          // first column of this warp inside the tile
+    ColTerms& C = S.cols[ew];
+    // Raw per-column inputs of the warp's slice (lane: columns lane and lane + 32 of the slice) and the row's code
+    // sum, fetched one tile ahead; nothing is computed from them before the next tile starts, so the loads stay in
+    // flight behind this tile's epilogue.
+    int nx_zw[2] = {0, 0}, nx_ws[2] = {0, 0}, nx_asum = 0;
+    float nx_sw[2] = {0.f, 0.f}, nx_bs[2] = {0.f, 0.f};
     auto fetch_terms = [&](int t) {
-      if (t >= tiles) return;
+      if (t >= tiles || !slice_on) return;
       const int tm0 = (t % m_tiles) * BM, tn0 = (t / m_tiles) * BN;
-      const int64_t tm = int64_t(tm0) + quarter * 32 + lane;
-      nx_asum = tm < P.M ? __ldg(P.asum + tm) : 0;
-      if (et < BN) {
-        const int j = tn0 + et;
-        nx_nzw = 0; nx_kw = 0; nx_sc = 0.f; nx_bi = 0.f;
-        if (j < P.N) {
-          nx_nzw = -(ep.z_w ? __ldg(ep.z_w + j) : ep.z_w_scalar);
-          nx_kw = -ep.z_a * __ldg(P.wsum + j);
-          nx_sc = ep.scale_a * (ep.s_w ? __ldg(ep.s_w + j) : ep.s_w_scalar);
-          nx_bi = ep.bias ? __ldg(ep.bias + j) : 0.f;
-          if (P.direct_requant) {
-            const int gw = ep.group_width;
-            const float inv = ep.inv_out_scale[(j >= gw) + (j >= 2 * gw) + (j >= 3 * gw)];
-            nx_sc *= inv;
-            nx_bi *= inv;
-          }
-        }
+      // plain loads from clamped indices: nothing here may consume a loaded value (a select on it would hold the
+      // warp until the load returns); rows and columns outside the matrix are dealt with where the values are used
+      const int64_t tm = min(int64_t(tm0) + quarter * 32 + lane, int64_t(P.M) - 1);
+      nx_asum = __ldg(P.asum + tm);
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int j = min(tn0 + cl0 + lane + 32 * h, P.N - 1);
+        if (ep.z_w) nx_zw[h] = __ldg(ep.z_w + j);
+        nx_ws[h] = __ldg(P.wsum + j);
+        if (ep.s_w) nx_sw[h] = __ldg(ep.s_w + j);
+        if (ep.bias) nx_bs[h] = __ldg(ep.bias + j);
       }
     };
     fetch_terms(blockIdx.x);
@@ -389,7 +421,6 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       const int m0 = (tile % m_tiles) * BM, n0 = (tile / m_tiles) * BN;
       const int64_t m = int64_t(m0) + quarter * 32 + lane;
       const bool row_ok = m < P.M;
-      const int cl0 = slice * kSliceCols;                    // first column of this warp inside the tile
       // warp-uniform: whole 64-column slice inside the matrix, common epilogue (rows beyond M are clipped by
       // the bulk store)
       const bool any_row = m0 + quarter * 32 < P.M;          // warp-uniform: at least one valid row
@@ -401,18 +432,30 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 #pragma unroll
         for (int i = 0; i < kSliceCols / 8; ++i) res[i] = __ldg(rp + i);
       }
-      // corr = acc - z_w (asum - K z_a) - z_a wsum; this tile's terms were fetched during the previous tile
+      // corr = acc - z_w (asum - K z_a) - z_a wsum; this tile's inputs were fetched during the previous tile
       const int32_t asum_c = row_ok ? nx_asum - kza : 0;
-      // stage the per-column terms of this tile (one column per thread, threads 0..BN-1); the buffer was last
-      // read two tiles ago, and every epilogue thread has passed the barrier of the tile in between
-      {
-        ColTerms& C = S.cols[acc];
-        if (et < BN) { C.nzw[et] = nx_nzw; C.kw[et] = nx_kw; C.sc[et] = nx_sc; C.bi[et] = nx_bi; }
-        mbar_arrive(smem_u32(&S.cols_ready[acc]));           // release: orders the writes above
-        if (!mbar_wait(smem_u32(&S.cols_ready[acc]), acc_phase, abort, 5)) break;
+      // stage the per-column terms of the warp's slice in the warp's own buffer (read by this warp alone)
+      if (slice_on) {
+        __syncwarp();                                          // the previous tile's reads of the buffer are done
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int cs = lane + 32 * h, j = n0 + cl0 + cs;
+          const bool in = j < P.N;                             // columns outside the matrix: all terms 0
+          float sc = in ? ep.scale_a * (ep.s_w ? nx_sw[h] : ep.s_w_scalar) : 0.f, bi = in && ep.bias ? nx_bs[h] : 0.f;
+          if (direct) {
+            const int gw = ep.group_width;
+            const float inv = ep.inv_out_scale[(j >= gw) + (j >= 2 * gw) + (j >= 3 * gw)];
+            sc *= inv;
+            bi *= inv;
+          }
+          C.nzw[cs] = in ? -(ep.z_w ? nx_zw[h] : ep.z_w_scalar) : 0;
+          C.kw[cs] = in ? -ep.z_a * nx_ws[h] : 0;
+          C.sc[cs] = sc;
+          C.bi[cs] = bi;
+        }
+        __syncwarp();
       }
-      fetch_terms(tile + int(gridDim.x));                    // next tile's terms: in flight during this epilogue
-      const ColTerms& C = S.cols[acc];
+      fetch_terms(tile + int(gridDim.x));                    // next tile's inputs: in flight during this epilogue
       int code_sum = 0;
 
       if (!mbar_wait(smem_u32(&S.tmem_full[acc]), acc_phase, abort, 4)) break;
@@ -429,10 +472,10 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
           float v[kChunk];
 #pragma unroll
           for (int q4 = 0; q4 < kChunk / 4; ++q4) {
-            const int4 nz = *reinterpret_cast<const int4*>(&C.nzw[cl + 4 * q4]);
-            const int4 kw = *reinterpret_cast<const int4*>(&C.kw[cl + 4 * q4]);
-            const float4 sc = *reinterpret_cast<const float4*>(&C.sc[cl + 4 * q4]);
-            const float4 bi = *reinterpret_cast<const float4*>(&C.bi[cl + 4 * q4]);
+            const int4 nz = *reinterpret_cast<const int4*>(&C.nzw[c * kChunk + 4 * q4]);
+            const int4 kw = *reinterpret_cast<const int4*>(&C.kw[c * kChunk + 4 * q4]);
+            const float4 sc = *reinterpret_cast<const float4*>(&C.sc[c * kChunk + 4 * q4]);
+            const float4 bi = *reinterpret_cast<const float4*>(&C.bi[c * kChunk + 4 * q4]);
             v[4 * q4 + 0] = fmaf(sc.x, float(int32_t(r[4 * q4 + 0]) + nz.x * asum_c + kw.x), bi.x);
             v[4 * q4 + 1] = fmaf(sc.y, float(int32_t(r[4 * q4 + 1]) + nz.y * asum_c + kw.y), bi.y);
             v[4 * q4 + 2] = fmaf(sc.z, float(int32_t(r[4 * q4 + 2]) + nz.z * asum_c + kw.z), bi.z);
@@ -465,7 +508,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
           }
           ChunkQuant q{};
           if constexpr (OUT == kOutC4 || OUT == kOutC8) q = chunk_quant(ep, P, col0);
-          emit_chunk<OUT>(&map_out, smem_u32(S.epi[ew]), lane, q, v, c, col0, m0 + quarter * 32, code_sum);
+          emit_chunk<OUT>(&map_out, smem_u32(S.epi[ew]), lane, q, v, c, col0, m0 + quarter * 32, code_sum, direct, sat);
         }
       } else if (slice_on && any_row && n0 + cl0 < P.N) {
 #pragma unroll 1
@@ -475,7 +518,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
           __syncwarp();
           tmem_ld16(taddr0 + c * kChunk, r);
           tmem_ld_wait();
-          if (row_ok && n0 + cl < P.N) slow_chunk(ep, P, C, r, cl, m, n0 + cl, asum_c, &code_sum);
+          if (row_ok && n0 + cl < P.N) slow_chunk(ep, P, C, r, c * kChunk, m, n0 + cl, asum_c, &code_sum);
         }
       }
       // accumulator buffer free again
@@ -531,7 +574,9 @@ TcLayout tc_layout(const repq_gemm_desc& d) {
   return L;
 }
 
-// Tile width with the fullest last round: rounds of tiles over the SMs times a cost that grows with BN.
+// Tile width: rounds of tiles over the SMs times the time of one round, which has a part that does not depend on the
+// width (per-tile waits, staging and bulk-store latencies of the epilogue warps) and a part proportional to it
+// (measured: about 160 columns' worth of fixed time for K = 768).
 int pick_bn(int M, int N, int sms) {
   const int m_tiles = (M + BM - 1) / BM;
   int best = 256;
@@ -539,7 +584,7 @@ int pick_bn(int M, int N, int sms) {
   for (int bn : {256, 192, 128}) {
     const long tiles = long(m_tiles) * ((N + bn - 1) / bn);
     const long rounds = (tiles + sms - 1) / sms;
-    const long cost = rounds * (bn + 32);
+    const long cost = rounds * (bn + 160);
     if (best_cost < 0 || cost < best_cost) { best = bn; best_cost = cost; }
   }
   return best;
