@@ -26,7 +26,6 @@
 
 #include "kernels.h"
 #include "tc_ptx.cuh"
-#include "f32x2.cuh"
 
 namespace repq {
 namespace {
@@ -74,8 +73,7 @@ struct AttnShared {
   alignas(1024) uint8_t v[NB * kVBlockBytes];
   int row_term[kRows];                              // -z_k qsum[m] + d_h z_q z_k
   int col_term[4][kKeys];                           // -z_q ksum[n], ring of 4 key blocks
-  int stat_m[kParts][kRows];                        // pass-1 results of the column parts of every row: maximum (integer)
-  float stat_z[kParts][kRows];                      //   and sum relative to it
+  float stat_m[kParts][kRows], stat_z[kParts][kRows];   // pass-1 results of the column parts of every row
   uint32_t lut[16][32];                             // 4-bit codes: [code][lane] = E value | O value << 16 (one bank per lane)
   alignas(8) uint64_t k_full[2];
   uint64_t s_full[2], s_empty[2], p_full, p_empty;
@@ -234,11 +232,9 @@ attention_tc_kernel(AttnParams P) {
     const int r = quarter * 32 + lane;                    // the thread's row inside the CTA = its tensor-memory lane
     const int row = q0 + r;
     const int valid = row < P.Lq ? (P.causal ? max(1, min(P.Lk, row + 1 + shift)) : P.Lk) : 0;   // keys the row sees
-    // the most keys any row of this warp sees: a 16-column part that starts at or past it holds masked keys only
-    // (all of them, in a warp whose rows lie past Lq), and its arithmetic is skipped
-    const int warp_valid = __reduce_max_sync(0xffffffffu, valid);
     const int my_row_term = S.row_term[r];
-    const float sc = P.scale * 1.4426950408889634f;       // log2(e) s_q s_k alpha: 2^(sc * corr) = e^S
+    const float c = 1.4426950408889634f;
+    const float k1 = -2.f * c;
     const float fq = float(P.qmax_p);
     const float magic = __uint_as_float(kMagicBits);
     const uint32_t taddr_s = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(part * kCols);
@@ -268,25 +264,15 @@ attention_tc_kernel(AttnParams P) {
     const float vz = __uint_as_float(kMagicBits) + float(P.z_v);
     const __nv_bfloat162 vz2 = __float2bfloat162_rn(128.f + float(P.z_v));
 
-    // Every S of a row is taken relative to the row's maximum as an integer difference of corrected accumulators
-    // (exact), so that pass 2 rounds t once: t = k0 - 2 sc (corr - max).
-    constexpr int kMasked = -(1 << 30);     // below every corrected accumulator (|corr| < 2^24); differences cannot overflow
-    int mi = kMasked;                       // pass 1: running maximum of this thread's columns,
-    float z = 0.f;                          //   sum of 2^(sc (corr - mi))
-    int row_term = my_row_term;             // pass 2: the row's maximum subtracted as well
-    float k0 = 0.f, a_row = 0.f;            // pass 2: t = k0 + a_row * (corr - max); k0 = 2 (log2 Z + log2 s), a_row = -2 sc
-    bool clamp_low = false;                 // pass 2: some row of the warp has k0 < -1/2, so that t can round below 0
+    float m = -CUDART_INF_F, z = 0.f;       // pass 1: running maximum and sum of this thread's columns
+    float k0 = 0.f;                         // pass 2: 2 (log2 Z + log2 s), with m the row's final maximum
 
     // corr = acc - z_k qsum - z_q ksum + d_h z_q z_k of the thread's 16 columns of key block j (buffer g & 1), as
     // integers; keys the row may not see become kMasked.  Frees the buffer as soon as it is read.
-    auto read_s = [&](int g, int j, bool dead, int (&corr)[kCols]) -> bool {
+    constexpr int kMasked = -2147483647 - 1;
+    auto read_s = [&](int g, int j, int (&corr)[kCols]) -> bool {
       const int b = g & 1;
       if (!mbar_wait(smem_u32(&S.s_full[b]), uint32_t(g >> 1) & 1u, abort, 44, P.status)) return false;
-      if (dead) {                                  // nothing to read, but the buffer is freed in step with the others
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&S.s_empty[b]));
-        return true;
-      }
       tc_fence_after();
       uint32_t r0[16];
       __syncwarp();
@@ -299,10 +285,10 @@ attention_tc_kernel(AttnParams P) {
 #pragma unroll
       for (int e4 = 0; e4 < kCols / 4; ++e4) {
         const int4 c4 = *reinterpret_cast<const int4*>(ct + 4 * e4);
-        corr[4 * e4 + 0] = int32_t(r0[4 * e4 + 0]) + row_term + c4.x;
-        corr[4 * e4 + 1] = int32_t(r0[4 * e4 + 1]) + row_term + c4.y;
-        corr[4 * e4 + 2] = int32_t(r0[4 * e4 + 2]) + row_term + c4.z;
-        corr[4 * e4 + 3] = int32_t(r0[4 * e4 + 3]) + row_term + c4.w;
+        corr[4 * e4 + 0] = int32_t(r0[4 * e4 + 0]) + my_row_term + c4.x;
+        corr[4 * e4 + 1] = int32_t(r0[4 * e4 + 1]) + my_row_term + c4.y;
+        corr[4 * e4 + 2] = int32_t(r0[4 * e4 + 2]) + my_row_term + c4.z;
+        corr[4 * e4 + 3] = int32_t(r0[4 * e4 + 3]) + my_row_term + c4.w;
       }
       // causal mask and keys past Lk: only in blocks that reach past the fewest keys any row of the CTA sees
       const int key0 = j * kKeys + part * kCols;
@@ -316,109 +302,70 @@ attention_tc_kernel(AttnParams P) {
 
     auto process = [&](int g) -> bool {
       const int j = g < nb ? g : g - nb;
-      const bool dead = j * kKeys + part * kCols >= warp_valid;
       int corr[kCols];
-      if (!read_s(g, j, dead, corr)) return false;
+      if (!read_s(g, j, corr)) return false;
       if (g < nb) {
-        // ---- pass 1: running maximum and sum, both relative to integers: a masked key is left out
-        const bool boundary = j * kKeys + part * kCols + kCols > min(min_valid, valid);
-        int bmi = kMasked;
-        if (!dead) {
+        // ---- pass 1: running maximum and sum.  The maximum is taken on the integers (S = scale * float(corr) is
+        // monotonic in corr); a masked key contributes 2^(-huge) = 0.
+        int bmi = corr[0];
 #pragma unroll
-          for (int e = 0; e < kCols; ++e) bmi = max(bmi, corr[e]);
-        }
+        for (int e = 1; e < kCols; ++e) bmi = max(bmi, corr[e]);
         if (bmi != kMasked) {
-          const int mn = max(mi, bmi);
-          float zs = 0.f;
-          if (__builtin_expect(boundary, 0)) {
+          const float mn = fmaxf(m, P.scale * float(bmi));
+          float acc0 = 0.f, acc1 = 0.f;
 #pragma unroll
-            for (int e = 0; e < kCols; ++e)
-              if (corr[e] != kMasked) zs += ex2(sc * float(corr[e] - mn));
-          } else {
-            const f32x2 sc2 = splat2(sc);
-            f32x2 acc = pack2(0.f, 0.f);
-#pragma unroll
-            for (int e = 0; e < kCols; e += 2) {
-              float y0, y1;
-              unpack2(mul2(pack2(float(corr[e] - mn), float(corr[e + 1] - mn)), sc2), y0, y1);
-              acc = add2(acc, pack2(ex2(y0), ex2(y1)));
-            }
-            float a0, a1;
-            unpack2(acc, a0, a1);
-            zs = a0 + a1;
+          for (int e = 0; e < kCols; e += 2) {
+            acc0 += ex2(fmaf(float(corr[e]), P.scale, -mn) * c);
+            acc1 += ex2(fmaf(float(corr[e + 1]), P.scale, -mn) * c);
           }
-          z = z * ex2(sc * float(mi - mn)) + zs;          // z = 0 at first
-          mi = mn;
+          z = z * ex2((m - mn) * c) + (acc0 + acc1);     // m = -inf at first: factor 0
+          m = mn;
         }
         if (g == nb - 1) {
-          // merge the column parts of every row: maximum, and Z = sum of the rescaled partial sums (same order in
+          // merge the column parts of every row: m = max, Z = sum of the rescaled partial sums (same order in
           // every thread of the row, so that all of them hold the same Z)
-          S.stat_m[part][r] = mi;
+          S.stat_m[part][r] = m;
           S.stat_z[part][r] = z;
           __syncwarp();
           if (lane == 0) mbar_arrive(smem_u32(&S.stats_ready));
           if (!mbar_wait(smem_u32(&S.stats_ready), 0, abort, 45, P.status)) return false;
-          int mrow = kMasked;
+          float mn = -CUDART_INF_F;
 #pragma unroll
-          for (int q = 0; q < kParts; ++q) mrow = max(mrow, S.stat_m[q][r]);
+          for (int q = 0; q < kParts; ++q) mn = fmaxf(mn, S.stat_m[q][r]);
           float zt = 0.f;
 #pragma unroll
           for (int q = 0; q < kParts; ++q) {
-            const int mq = S.stat_m[q][r];
-            if (mq != kMasked) zt += S.stat_z[q][r] * ex2(sc * float(mq - mrow));
+            const float mq = S.stat_m[q][r];
+            if (mq > -CUDART_INF_F) zt += S.stat_z[q][r] * ex2((mq - mn) * c);
           }
-          if (mrow != kMasked) {                           // a row past Lq keeps t = 0
-            row_term = my_row_term - mrow;
-            k0 = 2.f * (log2f(zt) + P.log2_s);
-            a_row = -2.f * sc;
-          }
-          clamp_low = __any_sync(0xffffffffu, !(k0 >= -0.5f));
+          m = mn;
+          k0 = 2.f * (log2f(zt) + P.log2_s);
           fetch_v(0);
         }
         return true;
       }
       // ---- pass 2: codes, operand tiles, V tile.
-      // Eq. 15: p = clip(round(t), 0, qmax), t = k0 - 2 log2(e) (S - max) = k0 + a_row * corr; rounding half to even
-      // by the float add of 1.5 * 2^23, which leaves p in the low mantissa bits u - kMagicBits.  t >= k0 for every key
-      // the row sees (corr <= 0), so the clamp at 0 is needed only where k0 < -1/2; the clamp at qmax is then taken on
-      // the integer u (a masked key has a huge t and is zeroed below).  The pair (E, O) of bf16 operand values,
+      // Eq. 15: p = clip(round(t), 0, qmax), t = k0 - 2 c (S - m); rounding half to even by the float add of
+      // 1.5 * 2^23, which leaves p in the low mantissa bits u - kMagicBits.  The pair (E, O) of bf16 operand values,
       // 2^-ceil(p/2) on the side of p's parity and 0 on the other, comes from a per-lane table for 4-bit codes and
-      // from integer arithmetic for wider ones.
+      // from integer arithmetic for wider ones.  A masked key gets (0, 0).
       const bool boundary = j * kKeys + part * kCols + kCols > min(min_valid, valid);
       const uint32_t lut_addr = smem_u32(&S.lut[0][lane]) - (kMagicBits << 7);
-      auto operand_pair = [&](uint32_t u) -> uint32_t {
-        if (kLut) {
-          uint32_t w;
-          asm("ld.shared.u32 %0, [%1];" : "=r"(w) : "r"(lut_addr + (u << 7)));
-          return w;
-        }
-        const int kk = int((u - kMagicBits + 1u) >> 1);                       // ceil(p / 2)
-        const uint32_t val = uint32_t(max(127 - kk, 0)) << 7;                 // bf16 bits of 2^-kk (0 below the normal range)
-        return (u & 1u) ? val << 16 : val;
-      };
       uint32_t eo[kCols];
 #pragma unroll
-      for (int e = 0; e < kCols; ++e) eo[e] = 0u;
-      if (!dead) {
-        if (__builtin_expect(!clamp_low, 1)) {
-          const f32x2 a2 = splat2(a_row), k2 = splat2(k0), magic2 = splat2(magic);
-          const int u_top = int(kMagicBits) + P.qmax_p;
-#pragma unroll
-          for (int e = 0; e < kCols; e += 2) {
-            float y0, y1;
-            unpack2(add2(fma2(pack2(float(corr[e]), float(corr[e + 1])), a2, k2), magic2), y0, y1);
-            eo[e] = operand_pair(uint32_t(min(__float_as_int(y0), u_top)));
-            eo[e + 1] = operand_pair(uint32_t(min(__float_as_int(y1), u_top)));
-          }
+      for (int e = 0; e < kCols; ++e) {
+        // clamped on both sides whatever the inputs (rows past Lq carry m = -inf, Z = 0): p indexes the table
+        const float t = fmaxf(fminf(fmaf(fmaf(float(corr[e]), P.scale, -m), k1, k0), fq), 0.f);
+        const uint32_t u = __float_as_uint(t + magic);
+        if (kLut) {
+          asm("ld.shared.u32 %0, [%1];" : "=r"(eo[e]) : "r"(lut_addr + (u << 7)));
         } else {
-#pragma unroll
-          for (int e = 0; e < kCols; ++e) {
-            const float t = fmaxf(fminf(fmaf(float(corr[e]), a_row, k0), fq), 0.f);
-            eo[e] = operand_pair(__float_as_uint(t + magic));
-          }
+          const int kk = int((u - kMagicBits + 1u) >> 1);                       // ceil(p / 2)
+          const uint32_t val = uint32_t(max(127 - kk, 0)) << 7;                 // bf16 bits of 2^-kk (0 below the normal range)
+          eo[e] = (u & 1u) ? val << 16 : val;
         }
       }
-      if (__builtin_expect(boundary && !dead, 0)) {
+      if (__builtin_expect(boundary, 0)) {
 #pragma unroll
         for (int e = 0; e < kCols; ++e)
           if (corr[e] == kMasked) eo[e] = 0u;
