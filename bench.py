@@ -283,16 +283,15 @@ def main():
     ms_total = sum(s.elapsed_time(e) for s, e in zip(starts, ends))
     clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
 
-    # ---- end to end through the public API: pinned host input -> device -> block -> host output
-    for _ in range(2):
-        x.copy_(x_host, non_blocking=True); blk.forward(x, y); y_host.copy_(y, non_blocking=True)
+    # ---- end to end through the host-buffer entry point: every step's input is copied from pinned host memory
+    # and its output copied back inside the timed region; the library overlaps the copies of neighbouring steps
+    # with the kernels (two device staging buffers per direction)
+    y_hosts = [y_host, torch.empty(y.shape, dtype=y.dtype).pin_memory()]
+    blk.forward_host([x_host] * 2, y_hosts)
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
-    for i in range(args.steps):
-        x.copy_(x_host, non_blocking=True)
-        blk.forward(x, y)
-        y_host.copy_(y, non_blocking=True)
+    blk.forward_host([x_host] * args.steps, [y_hosts[i & 1] for i in range(args.steps)])
     e1.record(stream)
     barrier()
     ms_e2e = e0.elapsed_time(e1)

@@ -336,6 +336,33 @@ repq_status repq_block_forward_timed(const repq_block_desc* d, const repq_block_
 repq_status repq_block_forward_static(const repq_block_desc* d, const repq_block_params* p, const void* x,
                                       void* y, void* stream);
 
+/* repq_block_forward for a sequence of n_batches independent batches whose inputs and outputs are in HOST
+ * memory: batch i is read from x_host[i] and its result written to y_host[i] (each (batch*seq) x dim, dense,
+ * act_dtype / out_dtype).  The library copies through the caller's device staging buffers and overlaps the
+ * copies with the block's kernels: batch i + 1 is copied in and batch i - 1 copied out while batch i is
+ * computed (two helper streams per device, created on first use and kept).  The same x_host or y_host pointer
+ * may be given for several batches.  (Plumbing around Eqs. 1-3 of the block; the paper has no counterpart.)
+ *
+ *  - x_dev[2], y_dev[2] [device]: staging buffers of one batch each; workspace as for repq_block_forward
+ *    (one suffices: the blocks themselves run one after the other on `stream`).  Owned by the caller, who
+ *    may not touch them until `stream` has completed.
+ *  - Host buffers should be page-locked: with pageable memory the copies are correct but do not overlap.
+ *  - Ordering: everything is queued after the work already on `stream`; the call returns when the work is
+ *    queued, and `stream` completes after the last copy out, so synchronising `stream` (or an event recorded
+ *    on it) makes every y_host[i] valid.  Two calls that overlap in time on the same device must use
+ *    different staging buffers and are serialised on the helper streams.
+ *  - Errors: REPQ_INVALID_ARG for NULL pointers or staging buffers that alias; errors of repq_block_forward
+ *    are passed on (work queued before the error still runs). */
+typedef struct repq_host_staging {
+  void* x_dev[2];
+  void* y_dev[2];
+  void* workspace;
+  size_t workspace_bytes;
+} repq_host_staging;
+repq_status repq_block_forward_host(const repq_block_desc* d, const repq_block_params* p,
+                                    const void* const* x_host, void* const* y_host, int n_batches,
+                                    const repq_host_staging* s, void* stream);
+
 /* Number of CUDA kernels this library has launched in the calling process so far. */
 uint64_t repq_launch_count(void);
 

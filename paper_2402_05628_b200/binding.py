@@ -28,7 +28,7 @@ EXPORTS = (
     "repq_pack_weights", "repq_ln_quant", "repq_qgemm_workspace_bytes", "repq_qgemm",
     "repq_softmax_log2", "repq_pv", "repq_block_workspace_bytes", "repq_block_forward",
     "repq_device_status", "repq_block_forward_timed", "repq_launch_count",
-    "repq_block_forward_static", "repq_attention",
+    "repq_block_forward_static", "repq_attention", "repq_block_forward_host",
 )
 REPQ_STATIC_WORKSPACE_BYTES = 8 << 20
 REPQ_BLOCK_STAGES = 9
@@ -148,6 +148,8 @@ def lib() -> C.CDLL:
         _lib.repq_block_forward_static.argtypes = [C.POINTER(BlockDesc), C.POINTER(BlockParams), C.c_void_p,
                                                    C.c_void_p, C.c_void_p]
         _lib.repq_attention.argtypes = [C.POINTER(AttentionDesc), C.c_void_p]
+        _lib.repq_block_forward_host.argtypes = [C.POINTER(BlockDesc), C.POINTER(BlockParams), C.POINTER(C.c_void_p),
+                                                 C.POINTER(C.c_void_p), C.c_int, C.POINTER(HostStaging), C.c_void_p]
         _lib.repq_launch_count.restype = C.c_uint64
         _lib.repq_launch_count.argtypes = []
         _lib.repq_scale_zero_from_bounds.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
@@ -302,6 +304,29 @@ def repq_block_forward_static(d: BlockDesc, p: BlockParams, x: torch.Tensor, y: 
     so nothing is allocated.  For hosts that may not allocate device memory on the inference path; blocks that
     need more scratch are rejected.  Calls share the scratch: do not overlap them on one GPU."""
     _check(lib().repq_block_forward_static(C.byref(d), C.byref(p), _ptr(x), _ptr(y), _stream(stream)))
+
+
+class HostStaging(C.Structure):
+    _fields_ = [("x_dev", C.c_void_p * 2), ("y_dev", C.c_void_p * 2), ("workspace", C.c_void_p),
+                ("workspace_bytes", C.c_size_t)]
+
+
+def repq_block_forward_host(d: BlockDesc, p: BlockParams, x_host, y_host, x_dev, y_dev, workspace: torch.Tensor,
+                            stream=None) -> None:
+    """Block over a sequence of batches held in host memory: x_host / y_host are lists of (pinned) CPU tensors,
+    x_dev / y_dev pairs of device staging tensors.  Copies and kernels of neighbouring batches overlap; the
+    results are valid once `stream` has completed."""
+    n = len(x_host)
+    assert len(y_host) == n and len(x_dev) == 2 and len(y_dev) == 2
+    xs = (C.c_void_p * max(n, 1))(*[t.data_ptr() for t in x_host])
+    ys = (C.c_void_p * max(n, 1))(*[t.data_ptr() for t in y_host])
+    st = HostStaging()
+    for k in range(2):
+        st.x_dev[k] = _ptr(x_dev[k])
+        st.y_dev[k] = _ptr(y_dev[k])
+    st.workspace = _ptr(workspace)
+    st.workspace_bytes = workspace.numel() * workspace.element_size()
+    _check(lib().repq_block_forward_host(C.byref(d), C.byref(p), xs, ys, n, C.byref(st), _stream(stream)))
 
 
 def repq_launch_count() -> int:

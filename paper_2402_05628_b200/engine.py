@@ -75,6 +75,7 @@ class QuantBlock:
         self.out_dtype = out_dtype or self.act_dtype
         self.softmax_s = float(w.softmax_scale)
         self._ws: Optional[torch.Tensor] = None
+        self._staging = None
         self._batch = None
 
     def desc(self, batch: int) -> B.BlockDesc:
@@ -121,6 +122,25 @@ class QuantBlock:
             y = torch.empty(x.shape, dtype=self.out_dtype, device=x.device)
         B.repq_block_forward(self.desc(batch), self.params(), x, y, self.workspace(batch), stream)
         return y
+
+    def forward_host(self, x_host: List[torch.Tensor], y_host: List[torch.Tensor], stream=None) -> None:
+        """The block over batches held in (pinned) host memory: x_host[i] -> y_host[i], every tensor
+        [batch * seq, dim].  Copies in, kernels and copies out of neighbouring batches overlap; y_host is valid
+        once `stream` (default: the current stream) has completed."""
+        c = self.cfg
+        if not x_host:
+            return
+        rows = x_host[0].shape[0]
+        batch = rows // c["L"]
+        for t in x_host:
+            assert t.dtype == self.act_dtype and t.is_contiguous() and tuple(t.shape) == (rows, c["D"]) and not t.is_cuda
+        for t in y_host:
+            assert t.dtype == self.out_dtype and t.is_contiguous() and tuple(t.shape) == (rows, c["D"]) and not t.is_cuda
+        if self._staging is None or self._staging[0][0].shape[0] != rows:
+            self._staging = ([torch.empty((rows, c["D"]), dtype=self.act_dtype, device=self.device) for _ in range(2)],
+                             [torch.empty((rows, c["D"]), dtype=self.out_dtype, device=self.device) for _ in range(2)])
+        B.repq_block_forward_host(self.desc(batch), self.params(), x_host, y_host, self._staging[0], self._staging[1],
+                                  self.workspace(batch), stream)
 
     def forward_timed(self, x: torch.Tensor, y: torch.Tensor, stream=None) -> List[float]:
         """Same pass with per-stage CUDA-event timing (synchronises); returns milliseconds per stage."""

@@ -56,3 +56,38 @@ def test_block_with_the_three_separate_attention_stages():
     """The block through repq_qgemm (scores) -> repq_softmax_log2 -> repq_pv instead of the fused kernel."""
     parity.check_block("c2_deit_b", batch=3, staged_attention=True)
     parity.check_block("c4_llama7b", batch=2, D=512, H=4, MLP=1408, L=320, massive=2, staged_attention=True)
+
+
+def test_block_forward_host_matches_the_device_path():
+    """Host-buffer entry point: five batches (two of them from the same host buffer) pipelined through two
+    staging buffers give, batch by batch, the bits that repq_block_forward gives on device buffers; the device
+    path itself is checked against the oracle above."""
+    import numpy as np
+    import torch
+    from paper_2402_05628_b200.engine import QuantBlock
+    from paper_2402_05628_b200 import binding as B
+    from workloads import make_block_inputs
+
+    w = make_block_inputs("c2_deit_b", batch=2)
+    blk = QuantBlock(w)
+    rng = np.random.default_rng(5)
+    xs = [torch.from_numpy(np.ascontiguousarray(w.x * s)).to(blk.act_dtype).pin_memory()
+          for s in (1.0, 0.5, 1.5, float(rng.uniform(0.7, 1.3)))]
+    x_host = [xs[0], xs[1], xs[2], xs[1], xs[3]]
+    y_host = [torch.zeros(xs[0].shape, dtype=blk.out_dtype).pin_memory() for _ in x_host]
+    blk.forward_host(x_host, y_host)
+    torch.cuda.synchronize()
+    assert B.repq_device_status() == 0
+    for xh, yh in zip(x_host, y_host):
+        y_dev = blk.forward(xh.to(blk.device))
+        torch.cuda.synchronize()
+        assert torch.equal(y_dev.cpu(), yh)
+    assert not torch.equal(y_host[0], y_host[1])
+    # nothing to do, and arguments that cannot work
+    d, p = blk.desc(2), blk.params()
+    ws = blk.workspace(2)
+    B.repq_block_forward_host(d, p, [], [], blk._staging[0], blk._staging[1], ws)
+    same = blk._staging[0][0]
+    with pytest.raises(B.RepqError):
+        B.repq_block_forward_host(d, p, x_host[:1], y_host[:1], [same, same], blk._staging[1], ws)
+    torch.cuda.synchronize()
