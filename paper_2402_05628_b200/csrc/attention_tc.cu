@@ -137,6 +137,10 @@ attention_tc_kernel(AttnParams P) {
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
 
+  // everything above touched no global memory of the kernel chain
+  grid_dependency_wait();
+  grid_dependency_trigger();
+
   // ---- K rows: 8 threads per key, one 16-byte piece each; Q rows: 4 threads per row, 2 pieces each
   const uint8_t* k_base = P.k + bo * P.k_so + bi * P.k_si;
   const int kkey = (tid >> 3) & (kKeys - 1), kq = tid & 7;
@@ -531,8 +535,7 @@ repq_status launch(const AttnParams& P, int64_t pairs, cudaStream_t st) {
   const size_t smem = sizeof(AttnShared<NB>);
   REPQ_CUDA(cudaFuncSetAttribute(attention_tc_kernel<NB, kLut>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
   dim3 grid((P.Lq + kRows - 1) / kRows, unsigned(pairs));
-  attention_tc_kernel<NB, kLut><<<grid, kThreads, smem, st>>>(P);
-  REPQ_CUDA(cudaGetLastError());
+  REPQ_CUDA(launch_chained(attention_tc_kernel<NB, kLut>, grid, dim3(kThreads), smem, st, P));
   note_launch();
   return REPQ_OK;
 }

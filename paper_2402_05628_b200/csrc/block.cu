@@ -128,6 +128,10 @@ static repq_status block_forward_impl(const repq_block_desc* dp, const repq_bloc
   uint8_t* hid_c = ws + L.off_hidden;
   int32_t* asum_h = reinterpret_cast<int32_t*>(ws + L.off_asum_h);
   void* gws = ws + L.off_gemm_ws;
+  // the two row-sum accumulators that kernels add into start at zero; cleared here, ahead of the first kernel,
+  // so that the kernels of the block follow one another in the stream without anything in between
+  REPQ_CUDA(cudaMemsetAsync(asum_attn, 0, size_t(M) * 4, st));
+  REPQ_CUDA(cudaMemsetAsync(asum_h, 0, size_t(M) * 4, st));
   int n_mark = 0;
 #define REPQ_MARK()                                            \
   do {                                                         \
@@ -151,7 +155,6 @@ static repq_status block_forward_impl(const repq_block_desc* dp, const repq_bloc
   if (!d.staged_attention) {
     // scores, Softmax codes and P.V in one kernel; it takes the time slot of the scores stage, the two
     // following stages are empty
-    REPQ_CUDA(cudaMemsetAsync(asum_attn, 0, size_t(M) * 4, st));
     repq_attention_desc a{};
     a.batch_outer = d.batch; a.batch_inner = H; a.Lq = S; a.Lk = S; a.d_h = dh; a.bits_qkv = ab;
     a.q_codes = qkv_c; a.ldq_bytes = L.ld_qkv; a.q_stride_outer = int64_t(S) * L.ld_qkv; a.q_stride_inner = head_bytes;
@@ -190,7 +193,6 @@ static repq_status block_forward_impl(const repq_block_desc* dp, const repq_bloc
   REPQ_TRY(repq_softmax_log2(scores, REPQ_F32, int64_t(d.batch) * H * S, S, L.ld_s, 1.f, d.causal ? S : 0, 0,
                              p.softmax_s, d.bits_p, p_c, L.ld_p, stream));
   REPQ_MARK();
-  REPQ_CUDA(cudaMemsetAsync(asum_attn, 0, size_t(M) * 4, st));
   {
     repq_pv_desc v{};
     v.batch_outer = d.batch; v.batch_inner = H; v.Lq = S; v.Lk = S; v.d_h = dh;
@@ -218,7 +220,6 @@ static repq_status block_forward_impl(const repq_block_desc* dp, const repq_bloc
   REPQ_TRY(repq_ln_quant(xbar, d.act_dtype, M, D, D, p.ln2_gamma_t, p.ln2_beta_t, d.eps, d.norm_kind, p.ln2_s, p.ln2_z,
                          ab, ln_c, L.ld_a, asum, stream));
   REPQ_MARK();
-  REPQ_CUDA(cudaMemsetAsync(asum_h, 0, size_t(M) * 4, st));
   {
     repq_gemm_desc g = linear_desc(d, M, d.mlp, D, ln_c, L.ld_a, p.ln2_s, p.ln2_z, asum, p.fc1);
     g.gelu = 1;

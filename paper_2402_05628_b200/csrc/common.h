@@ -57,4 +57,29 @@ int sm_count();
 // Launch accounting (repq_launch_count).
 void note_launch(int n = 1);
 
+// Kernels of one stream that follow each other are launched with programmatic stream serialization: the next
+// kernel may be scheduled, and run its prologue (barrier setup, tensor-memory allocation, parameter staging), as
+// SMs drain from the one before.  Such a kernel calls grid_dependency_wait() before its first access to global
+// memory that an earlier kernel may have written or may still read, and grid_dependency_trigger() once it has
+// started (both are no-ops in a kernel launched the plain way).
+#ifdef __CUDACC__
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 }  // namespace repq

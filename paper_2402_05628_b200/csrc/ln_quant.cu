@@ -120,6 +120,9 @@ ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
     wide = wide || !(fabsf(gi) * root_d < 5.0e8f) || !(fabsf(bi) < 5.0e8f);
   }
   const bool guard = __syncthreads_or(wide) != 0;
+  // gamma~ and beta~ are parameters; x and the outputs belong to the chain of kernels
+  grid_dependency_wait();
+  grid_dependency_trigger();
 
   const int tig = threadIdx.x % TPR;             // thread in group
   const int group = threadIdx.x / TPR;
@@ -282,8 +285,7 @@ repq_status launch(const T* x, int64_t rows, int D, int64_t ldx, const float* g,
   REPQ_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, kern, kBlock, smem));
   const int64_t cap = int64_t(sm_count()) * (resident > 0 ? resident : 1);
   const int grid = int(need < cap ? need : cap);
-  kern<<<grid, kBlock, smem, st>>>(x, rows, D, ldx, g, b, eps, rms, inv_s, z, qmax, codes, ldc, row_sum);
-  REPQ_CUDA(cudaGetLastError());
+  REPQ_CUDA(launch_chained(kern, dim3(grid), dim3(kBlock), smem, st, x, rows, D, ldx, g, b, eps, rms, inv_s, z, qmax, codes, ldc, row_sum));
   note_launch();
   return REPQ_OK;
 }

@@ -322,6 +322,9 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   tc_fence_after();
   const uint32_t tmem_base = S.tmem_base;
   volatile int* abort = &S.abort;
+  // everything above touched no global memory of the kernel chain
+  grid_dependency_wait();
+  grid_dependency_trigger();
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer
@@ -618,8 +621,7 @@ repq_status launch_tc_out(const CUtensorMap& map_a, const CUtensorMap& map_b, co
   REPQ_CUDA(cudaFuncSetAttribute(qgemm_tc_kernel<BN, OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
   const int tiles = ((P.M + BM - 1) / BM) * ((P.N + BN - 1) / BN);
   const int grid = tiles < sms ? tiles : sms;
-  qgemm_tc_kernel<BN, OUT><<<grid, kThreads, smem, st>>>(map_a, map_b, map_out, P);
-  REPQ_CUDA(cudaGetLastError());
+  REPQ_CUDA(launch_chained(qgemm_tc_kernel<BN, OUT>, dim3(grid), dim3(kThreads), smem, st, map_a, map_b, map_out, P));
   note_launch();
   return REPQ_OK;
 }
