@@ -39,16 +39,16 @@ ATTENTION_INSTR_PER_SCORE = 23
 # sources still hash to what was captured; otherwise `traffic` is null.
 NCU_TRAFFIC_WORKLOAD = ("c2_deit_b", 64)
 NCU_TRAFFIC = {   # stage: (DRAM bytes read + written per launch, kernel sources, their sha1 when captured)
-    'ln1': (19392768, ['ln_quant.cu', 'f32x2.cuh'], '9869074ea6b9'),
-    'ln2': (19392768, ['ln_quant.cu', 'f32x2.cuh'], '9869074ea6b9'),
-    'qkv': (14875648, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '470d458babdd'),
-    'attention': (29183744, ['attention_tc.cu', 'tc_ptx.cuh'], 'eda123b891cd'),
-    'scores': (85920512, ['scores_tc.cu', 'tc_ptx.cuh'], '56c4b8afa690'),
-    'softmax': (130385920, ['softmax_log2.cu', 'f32x2.cuh'], '45f5e16c2857'),
-    'pv': (26710528, ['pv_tc.cu', 'tc_ptx.cuh'], '7d458ef14cde'),
-    'proj': (33147392, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '470d458babdd'),
-    'fc1': (21291008, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '470d458babdd'),
-    'fc2': (83022592, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '470d458babdd'),
+    'ln1': (19393024, ['ln_quant.cu', 'f32x2.cuh'], '38b79e2bac15'),
+    'ln2': (19393024, ['ln_quant.cu', 'f32x2.cuh'], '38b79e2bac15'),
+    'qkv': (14141696, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '422fd03dd4de'),
+    'attention': (29182720, ['attention_tc.cu', 'tc_ptx.cuh'], '287296f40928'),
+    'scores': (85649408, ['scores_tc.cu', 'tc_ptx.cuh'], '0ec10eb039ae'),
+    'softmax': (132519680, ['softmax_log2.cu', 'f32x2.cuh'], '45f5e16c2857'),
+    'pv': (26712320, ['pv_tc.cu', 'tc_ptx.cuh'], '44d2a2d061d5'),
+    'proj': (32784384, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '422fd03dd4de'),
+    'fc1': (19791104, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '422fd03dd4de'),
+    'fc2': (81971968, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '422fd03dd4de'),
 }
 
 
