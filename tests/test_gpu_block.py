@@ -91,3 +91,27 @@ def test_block_forward_host_matches_the_device_path():
     with pytest.raises(B.RepqError):
         B.repq_block_forward_host(d, p, x_host[:1], y_host[:1], [same, same], blk._staging[1], ws)
     torch.cuda.synchronize()
+
+
+def test_block_back_to_back_passes_are_identical():
+    """Twenty passes queued without a synchronisation in between (each kernel's prologue overlaps the tail of the
+    kernel before) write the same bits as a pass that runs alone."""
+    import numpy as np
+    import torch
+    from paper_2402_05628_b200.engine import QuantBlock
+    from paper_2402_05628_b200 import binding as B
+    from workloads import make_block_inputs
+
+    for name, batch in (("c2_deit_b", 8), ("c1_vit_s", 1)):
+        w = make_block_inputs(name, batch=batch)
+        blk = QuantBlock(w)
+        x = torch.from_numpy(np.ascontiguousarray(w.x)).to(blk.device).to(blk.act_dtype)
+        alone = blk.forward(x).clone()
+        torch.cuda.synchronize()
+        outs = [torch.empty_like(alone) for _ in range(20)]
+        for y in outs:
+            blk.forward(x, y)
+        torch.cuda.synchronize()
+        assert B.repq_device_status() == 0
+        for y in outs:
+            assert torch.equal(y, alone)

@@ -132,3 +132,24 @@ def test_fused_attention_epilogues():
     parity.check_attention(2, 2, 197, 197, 64, 4, 4, out_kind="codes", out_bits=4 | parity.BYTE_CODES, seed=2)
     parity.check_attention(1, 2, 130, 130, 128, 4, 8, causal=True, out_kind="codes", out_bits=8, seed=3, s_p=0.7)
     parity.check_attention(1, 2, 130, 130, 64, 4, 4, out_kind="codes", out_bits=4, seed=4)
+
+
+@pytest.mark.parametrize("M,N,K,bits,out_bits,groups,gelu,residual,out_kind", [
+    # byte codes of 4 and 6 bits through the comparison-free quantizer: one and three column groups (group edges on
+    # and off the 64-column slices), GELU in front of it, rows that end inside a tile
+    (700, 768, 256, 4, 4, 1, False, None, "codes"), (700, 768, 256, 4, 4, 3, False, None, "codes"),
+    (389, 576, 384, 4, 4, 3, False, None, "codes"), (700, 512, 256, 6, 6, 1, True, None, "codes"),
+    (260, 1024, 128, 4, 6, 1, True, None, "codes"),
+    # 8-bit byte codes and packed 4-bit codes keep the clamping quantizer
+    (700, 512, 256, 8, 8, 2, False, None, "codes"), (300, 256, 256, 4, -4, 1, False, None, "codes"),
+    # float outputs with both residual types, ragged last column tile
+    (700, 768, 256, 4, 4, 1, False, "bf16", "bf16"), (389, 448, 768, 6, 4, 1, False, "f32", "f32"),
+    (513, 200, 256, 4, 4, 1, True, "bf16", "bf16"),
+])
+def test_qgemm_common_epilogue_path(M, N, K, bits, out_bits, groups, gelu, residual, out_kind):
+    """The epilogue the block runs (no accumulator dump, so the per-warp column terms, the bulk stores and the
+    comparison-free quantizer are what is checked), output against the oracle."""
+    b = bits | parity.BYTE_CODES
+    ob = -out_bits if out_bits < 0 else (out_bits | parity.BYTE_CODES)              # negative: packed 4-bit output
+    parity.check_qgemm(M, N, K, b, b, out_kind=out_kind, gelu=gelu, residual=residual, groups=groups, out_bits=ob,
+                       want_acc=False, want_out_sum=(out_kind == "codes"), seed=M + N + K + groups)
