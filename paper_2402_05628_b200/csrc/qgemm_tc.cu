@@ -38,7 +38,6 @@ namespace {
 constexpr int BM = 128, BK = 128;                   // BK in bytes (= codes); BN is a template parameter
 constexpr int kMaxBN = 256;
 constexpr int kChunk = 16;                           // accumulator columns per tcgen05.ld / per store
-constexpr int kStages = 4;
 constexpr int kEpiWarps = 16;
 constexpr int kEpiThreads = kEpiWarps * 32;
 constexpr int kThreads = 32 * (2 + kEpiWarps);
@@ -58,10 +57,17 @@ struct alignas(16) ColTerms {                          // per output column of a
   float bi[kSliceCols];     // bias[j]            (times 1/s_o in direct re-quantization mode)
 };
 
-template <int BN>
+constexpr uint32_t kResBytes = 32 * 128;            // bf16 residual of one warp and tile: 32 rows x 64 columns
+
+// RES: the bf16 residual of a tile comes in by bulk tensor copies, one 32 x 64 box per epilogue warp, asked for one
+// tile ahead (the operand ring gives up a stage for the boxes)
+template <int BN, bool RES>
 struct SharedStorage {
+  static constexpr int kStages = RES ? 3 : 4;
   alignas(1024) uint8_t a[kStages][kABytes];
   alignas(1024) uint8_t b[kStages][BN * BK];
+  alignas(1024) uint8_t res[RES ? kEpiWarps * kResBytes : 1024];
+  uint64_t res_full[kEpiWarps];
   alignas(1024) uint8_t epi[kEpiWarps][1024];     // per-warp staging box of the epilogue's bulk stores
   ColTerms cols[kEpiWarps];                       // each epilogue warp stages the terms of its own slice: no barrier
   alignas(8) uint64_t full[kStages];
@@ -285,11 +291,12 @@ __device__ __noinline__ void slow_chunk(const EpilogueParams& ep, const TcParams
   }
 }
 
-template <int BN, int OUT>
+template <int BN, int OUT, bool RES>
 __global__ void __launch_bounds__(kThreads, 1)
 qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                const __grid_constant__ CUtensorMap map_out, TcParams P) {
-  using Storage = SharedStorage<BN>;
+                const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_res, TcParams P) {
+  using Storage = SharedStorage<BN, RES>;
+  constexpr int kStages = Storage::kStages;
   constexpr uint32_t kBBytes = BN * BK;
   constexpr uint32_t kIdesc = idesc_for(BN);
   // 1024-byte alignment (swizzle atoms) is requested from the declaration so that the compiler keeps
@@ -305,6 +312,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&S.full[s]), 1); mbar_init(smem_u32(&S.empty[s]), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&S.tmem_full[a]), 1); mbar_init(smem_u32(&S.tmem_empty[a]), kEpiWarps); }
+    for (int w = 0; w < kEpiWarps; ++w) mbar_init(smem_u32(&S.res_full[w]), 1);
     mbar_init(smem_u32(&S.done), 1);
     S.abort = 0;
     if (smem_u32(smem_raw) & 1023u) {              // the swizzled tiles need the alignment asked for above
@@ -417,6 +425,20 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         if (ep.bias) nx_bs[h] = __ldg(ep.bias + j);
       }
     };
+    // bulk copy of the residual box of tile t (rows and columns outside the matrix are zero-filled)
+    const uint32_t res_buf = smem_u32(S.res) + uint32_t(RES ? ew : 0) * kResBytes;
+    const uint32_t res_bar = smem_u32(&S.res_full[ew]);
+    bool res_pending = false;
+    auto fetch_residual = [&](int t) {
+      if (!RES || t >= tiles || !slice_on) return;
+      const int tm0 = (t % m_tiles) * BM, tn0 = (t / m_tiles) * BN;
+      if (lane == 0) {
+        mbar_expect_tx(res_bar, kResBytes);
+        tma_load_2d(res_buf, &map_res, res_bar, tn0 + cl0, tm0 + quarter * 32);
+      }
+      res_pending = true;
+    };
+    fetch_residual(blockIdx.x);
     fetch_terms(blockIdx.x);
     int it = 0;
     for (int tile = blockIdx.x; tile < tiles && !*abort; tile += gridDim.x, ++it) {
@@ -430,7 +452,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       const bool fast = fast_ok && slice_on && n0 + cl0 + kSliceCols <= P.N && any_row;
       // bf16 residual of the slice: requested now, needed only after the main loop of the tile
       uint4 res[kSliceCols / 8];
-      if (fast && res16 && row_ok) {
+      if (!RES && fast && res16 && row_ok) {
         const uint4* rp = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(ep.residual) + m * ep.ld_residual + n0 + cl0);
 #pragma unroll
         for (int i = 0; i < kSliceCols / 8; ++i) res[i] = __ldg(rp + i);
@@ -464,6 +486,10 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       if (!mbar_wait(smem_u32(&S.tmem_full[acc]), acc_phase, abort, 4)) break;
       tc_fence_after();
       const uint32_t taddr0 = tmem_base + (uint32_t(quarter * 32) << 16) + acc * kAccStride + cl0;
+      if (RES && res_pending) {
+        if (!mbar_wait(res_bar, uint32_t(it) & 1u, abort, 6)) break;
+        res_pending = false;
+      }
       if (fast) {
 #pragma unroll
         for (int c = 0; c < kSliceChunks; ++c) {
@@ -500,7 +526,15 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
           if (res16 && row_ok) {
 #pragma unroll
             for (int i = 0; i < kChunk / 8; ++i) {
-              const uint4 w4 = res[c * (kChunk / 8) + i];
+              uint4 w4;
+              if (RES) {
+                // the thread's row of the box: 16-byte piece p sits at (p ^ (row & 7)) inside the 128-byte row
+                const uint32_t piece = uint32_t(c * (kChunk / 8) + i);
+                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w4.x), "=r"(w4.y), "=r"(w4.z), "=r"(w4.w)
+                             : "r"(res_buf + uint32_t(lane) * 128u + ((piece ^ uint32_t(lane & 7)) << 4)));
+              } else {
+                w4 = res[c * (kChunk / 8) + i];
+              }
               const uint32_t ws[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
               for (int k = 0; k < 4; ++k) {
@@ -528,8 +562,10 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&S.tmem_empty[acc]));
+      fetch_residual(tile + int(gridDim.x));               // every lane has read this tile's box (the __syncwarp above)
       if (ep.out_row_sum != nullptr && row_ok && code_sum != 0) atomicAdd(ep.out_row_sum + m, code_sum);
     }
+    if (RES && res_pending) mbar_drain(res_bar, uint32_t(it) & 1u);              // left the loop early: the copy must land
     if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");     // bulk stores complete
   }
 
@@ -613,17 +649,46 @@ repq_status make_out_map(CUtensorMap* map, const TcParams& P) {
   return REPQ_OK;
 }
 
-template <int BN, int OUT>
-repq_status launch_tc_out(const CUtensorMap& map_a, const CUtensorMap& map_b, const TcParams& P, int sms, cudaStream_t st) {
-  CUtensorMap map_out;
+// Tensor map of a bf16 residual for the epilogue warps' boxes: 32 rows x 64 columns, 128-byte swizzle.
+repq_status make_res_map(CUtensorMap* map, const TcParams& P) {
+  EncodeTiledFn fn = encode_fn();
+  REPQ_REQUIRE(fn != nullptr, REPQ_CUDA_ERROR, "qgemm: cuTensorMapEncodeTiled is not available");
+  const cuuint64_t dims[2] = {cuuint64_t(P.N), cuuint64_t(P.M)};
+  const cuuint64_t strides[1] = {cuuint64_t(P.ep.ld_residual) * 2};
+  const cuuint32_t box[2] = {kSliceCols, 32};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(P.ep.residual), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  REPQ_REQUIRE(r == CUDA_SUCCESS, REPQ_CUDA_ERROR, "qgemm: residual tensor map failed with code %d", int(r));
+  return REPQ_OK;
+}
+
+template <int BN, int OUT, bool RES>
+repq_status launch_tc_res(const CUtensorMap& map_a, const CUtensorMap& map_b, const TcParams& P, int sms, cudaStream_t st) {
+  CUtensorMap map_out, map_res;
   REPQ_TRY(make_out_map(&map_out, P));
-  const size_t smem = sizeof(SharedStorage<BN>);
-  REPQ_CUDA(cudaFuncSetAttribute(qgemm_tc_kernel<BN, OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+  if (RES) REPQ_TRY(make_res_map(&map_res, P));
+  else map_res = map_out;                                  // not read
+  const size_t smem = sizeof(SharedStorage<BN, RES>);
+  REPQ_CUDA(cudaFuncSetAttribute(qgemm_tc_kernel<BN, OUT, RES>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
   const int tiles = ((P.M + BM - 1) / BM) * ((P.N + BN - 1) / BN);
   const int grid = tiles < sms ? tiles : sms;
-  REPQ_CUDA(launch_chained(qgemm_tc_kernel<BN, OUT>, dim3(grid), dim3(kThreads), smem, st, map_a, map_b, map_out, P));
+  REPQ_CUDA(launch_chained(qgemm_tc_kernel<BN, OUT, RES>, dim3(grid), dim3(kThreads), smem, st, map_a, map_b, map_out, map_res, P));
   note_launch();
   return REPQ_OK;
+}
+
+template <int BN, int OUT>
+repq_status launch_tc_out(const CUtensorMap& map_a, const CUtensorMap& map_b, const TcParams& P, int sms, cudaStream_t st) {
+  // float outputs with a bf16 residual on tiles of at most 192 columns: the residual boxes fit beside three stages.
+  // Taken for short K, where the epilogue sets the pace (measured at 12608 x 768: K = 768 24 us against 27 us with
+  // row-per-lane residual loads; K = 3072 46 us against 39 us, the main loop missing its fourth stage).
+  if constexpr (BN <= 192 && (OUT == kOutF32 || OUT == kOutBf16)) {
+    if (P.ep.residual != nullptr && P.ep.residual_bf16 && P.ep.acc_debug == nullptr && P.K <= 1536)
+      return launch_tc_res<BN, OUT, true>(map_a, map_b, P, sms, st);
+  }
+  return launch_tc_res<BN, OUT, false>(map_a, map_b, P, sms, st);
 }
 
 template <int BN>
