@@ -41,14 +41,14 @@ NCU_TRAFFIC_WORKLOAD = ("c2_deit_b", 64)
 NCU_TRAFFIC = {   # stage: (DRAM bytes read + written per launch, kernel sources, their sha1 when captured)
     'ln1': (19393024, ['ln_quant.cu', 'f32x2.cuh'], '38b79e2bac15'),
     'ln2': (19393024, ['ln_quant.cu', 'f32x2.cuh'], '38b79e2bac15'),
-    'qkv': (14228736, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '32a19e0cdb0c'),
+    'qkv': (14292480, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '04dc33d1b726'),
     'attention': (29182720, ['attention_tc.cu', 'tc_ptx.cuh'], '287296f40928'),
     'scores': (85649408, ['scores_tc.cu', 'tc_ptx.cuh'], '0ec10eb039ae'),
     'softmax': (132519680, ['softmax_log2.cu', 'f32x2.cuh'], '45f5e16c2857'),
     'pv': (26712320, ['pv_tc.cu', 'tc_ptx.cuh'], '44d2a2d061d5'),
-    'proj': (33320960, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '32a19e0cdb0c'),
-    'fc1': (19666432, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '32a19e0cdb0c'),
-    'fc2': (79708672, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '32a19e0cdb0c'),
+    'proj': (33026560, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '04dc33d1b726'),
+    'fc1': (20006400, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '04dc33d1b726'),
+    'fc2': (80646912, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '04dc33d1b726'),
 }
 
 

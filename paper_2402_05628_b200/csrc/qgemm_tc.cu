@@ -11,16 +11,18 @@
 //                the main loop of tile i + 1
 //   warps 2..17  epilogue: warp w reads TMEM lanes 32 (w mod 4) .. +31 (one output row per thread) and a
 //                64-column slice of the accumulator columns
-// The tile width BN (256, 192 or 128) is chosen per problem so that the last round of tiles over the SMs is
-// as full as possible.  4-bit operands are expanded to one code per byte by a separate pass into the
+// The tile width BN (256, 192 or 128) is chosen per problem: rounds of tiles over the SMs times a per-round time
+// with a fixed part.  4-bit operands are expanded to one code per byte by a separate pass into the
 // workspace (there is no 4-bit integer MMA), so the main loop is the same for W4A4 and W8A8.
 //
 // For short K the epilogue, not the tensor pipe, sets the pace (K = 768: 3072 tensor-pipe cycles per
-// 128 x 256 tile against 32768 outputs), so it is written for few instructions per output: per-column terms
-// are staged once per tile in shared memory and read as vectors, the output quantizer is folded into them
-// where nothing sits between the GEMM and the re-quantization, rounding uses the float adder (add
-// 1.5 * 2^23), codes are packed by shift-adds with the zero-point folded into one constant, and the residual
-// of a tile is requested before the accumulator is waited for.
+// 128 x 256 tile against 32768 outputs), so it is written for few instructions per output and few waits per
+// tile: every epilogue warp stages the per-column terms of its own 64 columns in its own shared-memory buffer
+// (no barrier between warps) from plain loads issued one tile ahead and reads them as vectors, the output
+// quantizer is folded into them where nothing sits between the GEMM and the re-quantization, rounding uses
+// the float adder (add 1.5 * 2^23), byte codes of at most 7 bits are clamped by one saturating fma instead of
+// comparisons, and a bf16 residual comes in either by row-per-lane loads requested before the accumulator is
+// waited for or, for short K, by bulk tensor copies (one 32 x 64 box per epilogue warp, one tile ahead).
 //
 // Every wait on an mbarrier is bounded: when it runs out the kernel records a status code, all roles
 // leave their loops, in-flight copies and MMAs are drained, tensor memory is freed and the kernel returns.
