@@ -83,6 +83,12 @@ def test_block_forward_host_matches_the_device_path():
         torch.cuda.synchronize()
         assert torch.equal(y_dev.cpu(), yh)
     assert not torch.equal(y_host[0], y_host[1])
+    # pageable host memory: the copies no longer overlap, the results are the same
+    xp = [xs[2].clone(), xs[0].clone(), xs[3].clone()]
+    yp = [torch.zeros(xs[0].shape, dtype=blk.out_dtype) for _ in xp]
+    blk.forward_host(xp, yp)
+    torch.cuda.synchronize()
+    assert torch.equal(yp[0], y_host[2]) and torch.equal(yp[1], y_host[0]) and torch.equal(yp[2], y_host[4])
     # nothing to do, and arguments that cannot work
     d, p = blk.desc(2), blk.params()
     ws = blk.workspace(2)
