@@ -74,7 +74,8 @@ struct AttnShared {
   int row_term[kRows];                              // -z_k qsum[m] + d_h z_q z_k
   int col_term[4][kKeys];                           // -z_q ksum[n], ring of 4 key blocks
   float stat_m[kParts][kRows], stat_z[kParts][kRows];   // pass-1 results of the column parts of every row
-  uint32_t lut[16][32];                             // 4-bit codes: [code][lane] = E value | O value << 16 (one bank per lane)
+  uint32_t lut[17][32];                             // 4-bit codes: [code][lane] = E value | O value << 16 (one bank per lane);
+                                                    // entry 16 repeats 15 (a clamp at 16 that rounds up lands there)
   alignas(8) uint64_t k_full[2];
   uint64_t s_full[2], s_empty[2], p_full, p_empty;
   uint64_t stats_ready, acc_full, done;
@@ -176,8 +177,8 @@ attention_tc_kernel(AttnParams P) {
     s += __shfl_xor_sync(0xffffffffu, s, 1);
     s += __shfl_xor_sync(0xffffffffu, s, 2);
     if (qh == 0) S.row_term[qrow] = -P.zk * s + P.dh * P.zq * P.zk;
-    for (int i = tid; i < 16 * 32; i += kWorkThreads) {
-      const uint32_t code = uint32_t(i >> 5), bits16 = (127u - ((code + 1u) >> 1)) << 7;      // bf16 bits of 2^-ceil(code/2)
+    for (int i = tid; i < 17 * 32; i += kWorkThreads) {
+      const uint32_t code = min(uint32_t(i >> 5), 15u), bits16 = (127u - ((code + 1u) >> 1)) << 7;   // bf16 bits of 2^-ceil(code/2)
       S.lut[0][i] = (code & 1u) ? bits16 << 16 : bits16;
     }
   }
@@ -359,11 +360,16 @@ attention_tc_kernel(AttnParams P) {
 #pragma unroll
       for (int e = 0; e < kCols; ++e) {
         // clamped on both sides whatever the inputs (rows past Lq carry m = -inf, Z = 0): p indexes the table
-        const float t = fmaxf(fminf(fmaf(fmaf(float(corr[e]), P.scale, -m), k1, k0), fq), 0.f);
-        const uint32_t u = __float_as_uint(t + magic);
         if (kLut) {
+          // 4-bit codes: the clamp to [0, 16] is a saturating multiply by 1/16 (exact), the scaling back and the
+          // rounding one fma; 16 (t in [15.5, 16]) reads the table's copy of entry 15
+          float w;
+          asm("mul.rn.sat.f32 %0, %1, %2;" : "=f"(w) : "f"(fmaf(fmaf(float(corr[e]), P.scale, -m), k1, k0)), "f"(0.0625f));
+          const uint32_t u = __float_as_uint(fmaf(w, 16.f, magic));
           asm("ld.shared.u32 %0, [%1];" : "=r"(eo[e]) : "r"(lut_addr + (u << 7)));
         } else {
+          const float t = fmaxf(fminf(fmaf(fmaf(float(corr[e]), P.scale, -m), k1, k0), fq), 0.f);
+          const uint32_t u = __float_as_uint(t + magic);
           const int kk = int((u - kMagicBits + 1u) >> 1);                       // ceil(p / 2)
           const uint32_t val = uint32_t(max(127 - kk, 0)) << 7;                 // bf16 bits of 2^-kk (0 below the normal range)
           eo[e] = (u & 1u) ? val << 16 : val;
