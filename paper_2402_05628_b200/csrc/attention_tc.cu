@@ -240,7 +240,8 @@ attention_tc_kernel(AttnParams P) {
     const int my_row_term = S.row_term[r];
     const float c = 1.4426950408889634f;
     const float k1 = -2.f * c;
-    const float fq = float(P.qmax_p);
+    const float qs = float(P.qmax_p + 1), inv_qs = 1.f / qs;      // 2^bits and its reciprocal (exact)
+    const uint32_t u_top = kMagicBits + uint32_t(P.qmax_p);
     const float magic = __uint_as_float(kMagicBits);
     const uint32_t taddr_s = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(part * kCols);
 
@@ -368,8 +369,10 @@ attention_tc_kernel(AttnParams P) {
           const uint32_t u = __float_as_uint(fmaf(w, 16.f, magic));
           asm("ld.shared.u32 %0, [%1];" : "=r"(eo[e]) : "r"(lut_addr + (u << 7)));
         } else {
-          const float t = fmaxf(fminf(fmaf(fmaf(float(corr[e]), P.scale, -m), k1, k0), fq), 0.f);
-          const uint32_t u = __float_as_uint(t + magic);
+          // wider codes: the same clamp to [0, 2^bits], then the top code by one integer minimum
+          float w;
+          asm("mul.rn.sat.f32 %0, %1, %2;" : "=f"(w) : "f"(fmaf(fmaf(float(corr[e]), P.scale, -m), k1, k0)), "f"(inv_qs));
+          const uint32_t u = min(__float_as_uint(fmaf(w, qs, magic)), u_top);
           const int kk = int((u - kMagicBits + 1u) >> 1);                       // ceil(p / 2)
           const uint32_t val = uint32_t(max(127 - kk, 0)) << 7;                 // bf16 bits of 2^-kk (0 below the normal range)
           eo[e] = (u & 1u) ? val << 16 : val;
