@@ -89,6 +89,12 @@ __device__ __forceinline__ uint32_t tile_offset(int row, int piece) {
 __device__ __forceinline__ int sum_bytes(const uint4& v) {
   return __dp4a(v.x, 0x01010101u, __dp4a(v.y, 0x01010101u, __dp4a(v.z, 0x01010101u, __dp4a(v.w, 0x01010101u, 0u))));
 }
+// Bytewise c - z (two's complement) for codes and zero points below 128: with the top bit of every byte of c set
+// no borrow crosses a byte, and flipping that bit back leaves c - z mod 256.
+__device__ __forceinline__ uint32_t sub_bytes(uint32_t c, uint32_t z4) { return ((c | 0x80808080u) - z4) ^ 0x80808080u; }
+__device__ __forceinline__ uint4 sub_bytes(const uint4& c, uint32_t z4) {
+  return make_uint4(sub_bytes(c.x, z4), sub_bytes(c.y, z4), sub_bytes(c.z, z4), sub_bytes(c.w, z4));
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -96,7 +102,9 @@ __device__ __forceinline__ float ex2(float x) {
 }
 
 // NB: 64-channel blocks of the head; kLut: Softmax codes of at most 4 bits (operand values from the per-lane table)
-template <int NB, bool kLut>
+// kCentered: Q and K codes minus their zero points fit a signed byte (quantizers of at most 7 bits); the tiles then
+// hold q - z_q and k - z_k, the S MMAs run signed x signed and their accumulators need no zero-point correction.
+template <int NB, bool kLut, bool kCentered>
 __global__ void __launch_bounds__(kThreads, NB == 1 ? 2 : 1)
 attention_tc_kernel(AttnParams P) {
   using Shared = AttnShared<NB>;
@@ -146,12 +154,20 @@ attention_tc_kernel(AttnParams P) {
   const uint8_t* k_base = P.k + bo * P.k_so + bi * P.k_si;
   const int kkey = (tid >> 3) & (kKeys - 1), kq = tid & 7;
   uint4 kreg, knext;                            // the thread's piece of the K rows of the next two key blocks
-  auto fetch_k = [&](int block, uint4& dst) {
+  bool k_live = false, k_live_next = false;     // whether that piece holds codes (key below Lk, piece below d_h)
+  auto fetch_k = [&](int block, uint4& dst, bool& live) {
     dst = make_uint4(0u, 0u, 0u, 0u);
     const int key = block * kKeys + kkey;
-    if (key < P.Lk && kq < pieces) dst = __ldg(reinterpret_cast<const uint4*>(k_base + int64_t(key) * P.ldk) + kq);
+    live = key < P.Lk && kq < pieces;
+    if (live) dst = __ldg(reinterpret_cast<const uint4*>(k_base + int64_t(key) * P.ldk) + kq);
   };
-  auto store_k = [&](uint8_t* tile) {            // returns the code sum of the thread's key
+  const uint32_t zk4 = uint32_t(P.zk) * 0x01010101u, zq4 = uint32_t(P.zq) * 0x01010101u;
+  auto store_k = [&](uint8_t* tile) {            // returns the code sum of the thread's key (not needed when centred)
+    if (kCentered) {
+      // keys past Lk and pieces past d_h stay 0, so that they add nothing to S
+      if (kq < 2 * ksteps) *reinterpret_cast<uint4*>(tile + tile_offset(kkey, kq)) = k_live ? sub_bytes(kreg, zk4) : kreg;
+      return 0;
+    }
     if (kq < 2 * ksteps) *reinterpret_cast<uint4*>(tile + tile_offset(kkey, kq)) = kreg;
     int s = sum_bytes(kreg);
     s += __shfl_xor_sync(0xffffffffu, s, 1);
@@ -161,8 +177,8 @@ attention_tc_kernel(AttnParams P) {
   };
 
   if (warp < kWorkWarps) {
-    fetch_k(0, kreg);
-    fetch_k(nb > 1 ? 1 : 0, knext);
+    fetch_k(0, kreg, k_live);
+    fetch_k(nb > 1 ? 1 : 0, knext, k_live_next);
     const uint8_t* q_base = P.q + bo * P.q_so + bi * P.q_si;
     const int qrow = (tid >> 2) & (kRows - 1), qh = tid & 3;
     int s = 0;
@@ -170,7 +186,10 @@ attention_tc_kernel(AttnParams P) {
     for (int j = 0; j < 2; ++j) {
       const int piece = 2 * qh + j;
       uint4 w = make_uint4(0u, 0u, 0u, 0u);
-      if (q0 + qrow < P.Lq && piece < pieces) w = __ldg(reinterpret_cast<const uint4*>(q_base + int64_t(q0 + qrow) * P.ldq) + piece);
+      if (q0 + qrow < P.Lq && piece < pieces) {
+        w = __ldg(reinterpret_cast<const uint4*>(q_base + int64_t(q0 + qrow) * P.ldq) + piece);
+        if (kCentered) w = sub_bytes(w, zq4);
+      }
       if (piece < 2 * ksteps) *reinterpret_cast<uint4*>(S.q + tile_offset(qrow, piece)) = w;
       s += sum_bytes(w);
     }
@@ -192,7 +211,9 @@ attention_tc_kernel(AttnParams P) {
     // ---------------------------------------------------------------- MMA issue
     if (lane == 0) {
       // S: D = s32, A = B = unsigned 8-bit, both K-major, N = 64, M = 128
-      constexpr uint32_t idesc_s = (2u << 4) | (uint32_t(kKeys >> 3) << 17) | (uint32_t(kRows >> 4) << 24);
+      // (operand formats: 0 = unsigned, 1 = signed bytes)
+      constexpr uint32_t idesc_s = (2u << 4) | (uint32_t(kCentered) << 7) | (uint32_t(kCentered) << 10) | (uint32_t(kKeys >> 3) << 17) |
+                                   (uint32_t(kRows >> 4) << 24);
       // P.V: D = f32, A = B = bf16, A K-major, B MN-major, N = n_pad, M = 128
       const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (uint32_t(P.n_pad >> 3) << 17) |
                                 (uint32_t(kRows >> 4) << 24);
@@ -287,14 +308,19 @@ attention_tc_kernel(AttnParams P) {
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&S.s_empty[b]));
-      const int* ct = S.col_term[g & 3] + part * kCols;
+      if (kCentered) {
 #pragma unroll
-      for (int e4 = 0; e4 < kCols / 4; ++e4) {
-        const int4 c4 = *reinterpret_cast<const int4*>(ct + 4 * e4);
-        corr[4 * e4 + 0] = int32_t(r0[4 * e4 + 0]) + my_row_term + c4.x;
-        corr[4 * e4 + 1] = int32_t(r0[4 * e4 + 1]) + my_row_term + c4.y;
-        corr[4 * e4 + 2] = int32_t(r0[4 * e4 + 2]) + my_row_term + c4.z;
-        corr[4 * e4 + 3] = int32_t(r0[4 * e4 + 3]) + my_row_term + c4.w;
+        for (int e = 0; e < kCols; ++e) corr[e] = int32_t(r0[e]);
+      } else {
+        const int* ct = S.col_term[g & 3] + part * kCols;
+#pragma unroll
+        for (int e4 = 0; e4 < kCols / 4; ++e4) {
+          const int4 c4 = *reinterpret_cast<const int4*>(ct + 4 * e4);
+          corr[4 * e4 + 0] = int32_t(r0[4 * e4 + 0]) + my_row_term + c4.x;
+          corr[4 * e4 + 1] = int32_t(r0[4 * e4 + 1]) + my_row_term + c4.y;
+          corr[4 * e4 + 2] = int32_t(r0[4 * e4 + 2]) + my_row_term + c4.z;
+          corr[4 * e4 + 3] = int32_t(r0[4 * e4 + 3]) + my_row_term + c4.w;
+        }
       }
       // causal mask and keys past Lk: only in blocks that reach past the fewest keys any row of the CTA sees
       const int key0 = j * kKeys + part * kCols;
@@ -441,12 +467,13 @@ attention_tc_kernel(AttnParams P) {
     for (int g = 0; g < 2 * nb && !*abort; ++g) {
       // tile g & 1 was last read by the S MMAs of g - 2, whose result this thread has already waited for
       const int ks = store_k(S.k[g & 1]);
-      if (kq == 0) S.col_term[g & 3][kkey] = -P.zq * ks;
+      if (!kCentered && kq == 0) S.col_term[g & 3][kkey] = -P.zq * ks;
       fence_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&S.k_full[g & 1]));
       kreg = knext;
-      if (g + 2 < 2 * nb) fetch_k((g + 2) % nb, knext);            // two blocks ahead: global latency is about one block
+      k_live = k_live_next;
+      if (g + 2 < 2 * nb) fetch_k((g + 2) % nb, knext, k_live_next);            // two blocks ahead: global latency is about one block
       if (g > 0 && !process(g - 1)) { ok = false; break; }
     }
     if (ok && !*abort) ok = process(2 * nb - 1);
@@ -539,14 +566,21 @@ attention_tc_kernel(AttnParams P) {
   }
 }
 
-template <int NB, bool kLut>
-repq_status launch(const AttnParams& P, int64_t pairs, cudaStream_t st) {
+template <int NB, bool kLut, bool kCentered>
+repq_status launch_kernel(const AttnParams& P, int64_t pairs, cudaStream_t st) {
   const size_t smem = sizeof(AttnShared<NB>);
-  REPQ_CUDA(cudaFuncSetAttribute(attention_tc_kernel<NB, kLut>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+  REPQ_CUDA(cudaFuncSetAttribute(attention_tc_kernel<NB, kLut, kCentered>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
   dim3 grid((P.Lq + kRows - 1) / kRows, unsigned(pairs));
-  REPQ_CUDA(launch_chained(attention_tc_kernel<NB, kLut>, grid, dim3(kThreads), smem, st, P));
+  REPQ_CUDA(launch_chained(attention_tc_kernel<NB, kLut, kCentered>, grid, dim3(kThreads), smem, st, P));
   note_launch();
   return REPQ_OK;
+}
+
+template <int NB, bool kLut>
+repq_status launch(const AttnParams& P, int64_t pairs, int qmax_qk, cudaStream_t st) {
+  // q - z_q and k - z_k as signed bytes: codes and zero points below 128 and differences within [-128, 127]
+  const bool centred = qmax_qk < 128 && P.zq >= 0 && P.zq < 128 && P.zk >= 0 && P.zk < 128;
+  return centred ? launch_kernel<NB, kLut, true>(P, pairs, st) : launch_kernel<NB, kLut, false>(P, pairs, st);
 }
 
 }  // namespace
@@ -609,6 +643,6 @@ extern "C" repq_status repq_attention(const repq_attention_desc* d, void* stream
   REPQ_REQUIRE(P.status != nullptr, REPQ_CUDA_ERROR, "attention: device status word unavailable");
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool lut = P.qmax_p <= 15;
-  if (d->d_h <= 64) return lut ? launch<1, true>(P, pairs, st) : launch<1, false>(P, pairs, st);
-  return lut ? launch<2, true>(P, pairs, st) : launch<2, false>(P, pairs, st);
+  if (d->d_h <= 64) return lut ? launch<1, true>(P, pairs, qmax_v, st) : launch<1, false>(P, pairs, qmax_v, st);
+  return lut ? launch<2, true>(P, pairs, qmax_v, st) : launch<2, false>(P, pairs, qmax_v, st);
 }
