@@ -42,7 +42,7 @@ NCU_TRAFFIC = {   # stage: (DRAM bytes read + written per launch, kernel sources
     'ln1': (19393024, ['ln_quant.cu', 'f32x2.cuh'], '38b79e2bac15'),
     'ln2': (19393024, ['ln_quant.cu', 'f32x2.cuh'], '38b79e2bac15'),
     'qkv': (14292480, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '04dc33d1b726'),
-    'attention': (29182720, ['attention_tc.cu', 'tc_ptx.cuh'], '287296f40928'),
+    'attention': (29182464, ['attention_tc.cu', 'tc_ptx.cuh'], '09a7ba52cc05'),
     'scores': (85649408, ['scores_tc.cu', 'tc_ptx.cuh'], '0ec10eb039ae'),
     'softmax': (132519680, ['softmax_log2.cu', 'f32x2.cuh'], '45f5e16c2857'),
     'pv': (26712320, ['pv_tc.cu', 'tc_ptx.cuh'], '44d2a2d061d5'),
