@@ -90,7 +90,7 @@ __device__ __forceinline__ void group_reduce(V (&v)[kRows], V* red, int group_fi
   }
 }
 
-template <typename T, int TPR, int kVPT, bool kPack4>
+template <typename T, int TPR, int kVPT, bool kPack4, bool kFull>
 __global__ void __launch_bounds__((TPR > 256 ? TPR : 256))
 ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
                 const float* __restrict__ gamma_t, const float* __restrict__ beta_t, float eps, int rms,
@@ -137,12 +137,14 @@ ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
   auto fetch = [&](int64_t first_row) {
 #pragma unroll
     for (int r = 0; r < kRows; ++r) {
-      const bool live = first_row + r < rows;
-      const T* xr = x + (live ? first_row + r : 0) * ldx;
+      // rows past the end re-read the last row (their codes are never stored); when the row fills the group
+      // exactly (kFull) no load is predicated
+      const int64_t row = first_row + r < rows ? first_row + r : rows - 1;
+      const T* xr = x + row * ldx;
 #pragma unroll
       for (int i = 0; i < kVPT; ++i) {
         const int c = tig + i * TPR;
-        load_raw(xr + c * kChunk, live && c < nchunks, raw[r][i]);
+        load_raw(xr + c * kChunk, kFull || c < nchunks, raw[r][i]);
       }
     }
   };
@@ -188,7 +190,7 @@ ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
       f32x2 acc = 0ull;
 #pragma unroll
       for (int i = 0; i < kVPT; ++i) {
-        if (tig + i * TPR < nchunks) {
+        if (kFull || tig + i * TPR < nchunks) {
 #pragma unroll
           for (int e = 0; e < kChunk / 2; ++e) {
             v[r][i][e] = add2(v[r][i][e], neg_mu);
@@ -206,12 +208,18 @@ ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
     for (int r = 0; r < kRows; ++r) rstd[r] = splat2(rsqrtf(ss[r] * inv_d + eps));
 
     int csum[kRows];
+    bool live[kRows];
+    uint8_t* out[kRows];
 #pragma unroll
-    for (int r = 0; r < kRows; ++r) csum[r] = 0;
+    for (int r = 0; r < kRows; ++r) {
+      csum[r] = 0;
+      live[r] = row0 + r < rows;
+      out[r] = codes + (row0 + r) * ldc;
+    }
 #pragma unroll
     for (int i = 0; i < kVPT; ++i) {
       const int c = tig + i * TPR;
-      if (c < nchunks) {
+      if (kFull || c < nchunks) {
         f32x2 g[kChunk / 2], b[kChunk / 2];
         {
           const float4 g0 = *reinterpret_cast<const float4*>(s_g + c * kChunk);
@@ -235,23 +243,21 @@ ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
           int q[kChunk];
 #pragma unroll
           for (int e = 0; e < kChunk; ++e) q[e] = __float2int_rn(t[e]) + z;
-          if (row0 + r < rows) {
-            uint8_t* out = codes + (row0 + r) * ldc;
-            if constexpr (kPack4) {
-              uint32_t w = 0;
+          // rows past the end compute on a copy of the last row; only the stores are predicated
+          if constexpr (kPack4) {
+            uint32_t w = 0;
 #pragma unroll
-              for (int e = kChunk - 2; e >= 0; e -= 2) w = push_pair_u4(q[e], q[e + 1], w);
-              reinterpret_cast<uint32_t*>(out)[c] = w;
-              csum[r] += __dp4a(w & 0x0F0F0F0Fu, 0x01010101u, 0u) + __dp4a((w >> 4) & 0x0F0F0F0Fu, 0x01010101u, 0u);
-            } else {
-              uint2 w;
-              w.x = push_pair_u8(q[0], q[1], push_pair_u8(q[2], q[3], 0u));
-              w.y = push_pair_u8(q[4], q[5], push_pair_u8(q[6], q[7], 0u));
-              w.x = __vminu4(w.x, qmax4);          // 4- and 6-bit quantizers in byte containers
-              w.y = __vminu4(w.y, qmax4);
-              reinterpret_cast<uint2*>(out)[c] = w;
-              csum[r] += __dp4a(w.x, 0x01010101u, 0u) + __dp4a(w.y, 0x01010101u, 0u);
-            }
+            for (int e = kChunk - 2; e >= 0; e -= 2) w = push_pair_u4(q[e], q[e + 1], w);
+            if (live[r]) reinterpret_cast<uint32_t*>(out[r])[c] = w;
+            csum[r] = int(__dp4a(w & 0x0F0F0F0Fu, 0x01010101u, __dp4a((w >> 4) & 0x0F0F0F0Fu, 0x01010101u, uint32_t(csum[r]))));
+          } else {
+            uint2 w;
+            w.x = push_pair_u8(q[0], q[1], push_pair_u8(q[2], q[3], 0u));
+            w.y = push_pair_u8(q[4], q[5], push_pair_u8(q[6], q[7], 0u));
+            w.x = __vminu4(w.x, qmax4);          // 4- and 6-bit quantizers in byte containers
+            w.y = __vminu4(w.y, qmax4);
+            if (live[r]) reinterpret_cast<uint2*>(out[r])[c] = w;
+            csum[r] = int(__dp4a(w.x, 0x01010101u, __dp4a(w.y, 0x01010101u, uint32_t(csum[r]))));
           }
         }
       }
@@ -277,7 +283,9 @@ repq_status launch(const T* x, int64_t rows, int D, int64_t ldx, const float* g,
   const float inv_s = 1.f / s_t;
   const int qmax = code_max(bits);
   const size_t smem = size_t(D) * 2 * sizeof(float);
-  auto kern = packed4(bits) ? ln_quant_kernel<T, TPR, kVPT, true> : ln_quant_kernel<T, TPR, kVPT, false>;
+  const bool full = D == TPR * kVPT * kChunk;   // the row fills the group exactly: no chunk is predicated
+  auto kern = packed4(bits) ? (full ? ln_quant_kernel<T, TPR, kVPT, true, true> : ln_quant_kernel<T, TPR, kVPT, true, false>)
+                            : (full ? ln_quant_kernel<T, TPR, kVPT, false, true> : ln_quant_kernel<T, TPR, kVPT, false, false>);
   if (smem > 48 * 1024) REPQ_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
   // persistent grid: exactly the blocks that are resident at once, so that every block keeps its load pipeline
   // running over all of its rows
