@@ -91,7 +91,7 @@ __device__ __forceinline__ void group_reduce(V (&v)[kRows], V* red, int group_fi
 }
 
 template <typename T, int TPR, int kVPT, bool kPack4, bool kFull>
-__global__ void __launch_bounds__((TPR > 256 ? TPR : 256))
+__global__ void __launch_bounds__((TPR > 256 ? TPR : 256), (kVPT <= 2 && TPR == 256 ? 3 : 0))
 ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
                 const float* __restrict__ gamma_t, const float* __restrict__ beta_t, float eps, int rms,
                 float inv_s, int z, int qmax, uint8_t* __restrict__ codes, int64_t ldc,
@@ -109,15 +109,16 @@ ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
 
   float* s_g = s_gb;
   float* s_b = s_gb + D;
-  // |t| <= sqrt(D) |gamma~/s~| + |beta~/s~|.  Unless that bound is far inside the int32 range, t is clamped
-  // before the conversion so that adding z cannot wrap (a whole-kernel decision, taken here once).
+  // |t| <= sqrt(D) |gamma~/s~| + |beta~/s~|.  While that bound stays below 2^22 the round operation is one packed
+  // float add of 1.5 * 2^23 (round half to even by the adder, rint(t) left in the low mantissa bits); otherwise t
+  // is clamped and converted, so that adding z cannot wrap (a whole-kernel decision, taken here once).
   const float root_d = sqrtf(float(D));
   bool wide = false;
   for (int i = threadIdx.x; i < D; i += kBlock) {
     const float gi = __ldg(gamma_t + i) * inv_s, bi = __ldg(beta_t + i) * inv_s;
     s_g[i] = gi;
     s_b[i] = bi;
-    wide = wide || !(fabsf(gi) * root_d < 5.0e8f) || !(fabsf(bi) < 5.0e8f);
+    wide = wide || !(fabsf(gi) * root_d + fabsf(bi) < 4.0e6f);
   }
   const bool guard = __syncthreads_or(wide) != 0;
   // gamma~ and beta~ are parameters; x and the outputs belong to the chain of kernels
@@ -130,6 +131,9 @@ ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
   const int nchunks = D / kChunk;
   const float inv_d = 1.f / float(D);
   const uint32_t qmax4 = uint32_t(qmax) * 0x01010101u;
+  constexpr uint32_t kMagicBits = 0x4B400000u;   // 1.5 * 2^23
+  const f32x2 magic2 = splat2(__uint_as_float(kMagicBits));
+  const int z_less_magic = z - int(kMagicBits);
 
   // The rows of the next iteration are requested while those of the current one are processed, so that loads
   // stay in flight through the reductions and the packing.
@@ -233,16 +237,22 @@ ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
         for (int r = 0; r < kRows; ++r) {
           // Eq. 4: clip(round(t) + z, 0, qmax): round half to even by the float -> int conversion, then the
           // packing instruction saturates to the container ([0, 15] or [0, 255])
-          float t[kChunk];
-#pragma unroll
-          for (int e = 0; e < kChunk / 2; ++e) unpack2(fma2(mul2(v[r][i][e], rstd[r]), g[e], b[e]), t[2 * e], t[2 * e + 1]);
-          if (guard) {
-#pragma unroll
-            for (int e = 0; e < kChunk; ++e) t[e] = fminf(fmaxf(t[e], -1.0e9f), 1.0e9f);
-          }
           int q[kChunk];
+          if (!guard) {
 #pragma unroll
-          for (int e = 0; e < kChunk; ++e) q[e] = __float2int_rn(t[e]) + z;
+            for (int e = 0; e < kChunk / 2; ++e) {
+              float u0, u1;
+              unpack2(add2(fma2(mul2(v[r][i][e], rstd[r]), g[e], b[e]), magic2), u0, u1);
+              q[2 * e] = __float_as_int(u0) + z_less_magic;
+              q[2 * e + 1] = __float_as_int(u1) + z_less_magic;
+            }
+          } else {
+            float t[kChunk];
+#pragma unroll
+            for (int e = 0; e < kChunk / 2; ++e) unpack2(fma2(mul2(v[r][i][e], rstd[r]), g[e], b[e]), t[2 * e], t[2 * e + 1]);
+#pragma unroll
+            for (int e = 0; e < kChunk; ++e) q[e] = __float2int_rn(fminf(fmaxf(t[e], -1.0e9f), 1.0e9f)) + z;
+          }
           // rows past the end compute on a copy of the last row; only the stores are predicated
           if constexpr (kPack4) {
             uint32_t w = 0;
@@ -315,8 +325,10 @@ repq_status dispatch(const T* x, int64_t rows, int D, int64_t ldx, const float* 
                      int rms, float s_t, int z, int bits, uint8_t* codes, int64_t ldc, int32_t* row_sum,
                      cudaStream_t st) {
   const int nchunks = D / kChunk;
+  // a row that would take four chunks per thread in a group of 128 goes to a whole block with two (measured:
+  // D = 4096 runs 9 % faster as 256 x 2 with three resident blocks than as 128 x 4 with one)
 #define REPQ_LN_CASE(TPR) \
-  if (nchunks <= TPR * kMaxVPT) return launch_vpt<T, TPR>((nchunks + TPR - 1) / TPR, x, rows, D, ldx, g, b, eps, rms, s_t, z, bits, codes, ldc, row_sum, st);
+  if (nchunks <= TPR * (TPR == 128 ? 3 : kMaxVPT)) return launch_vpt<T, TPR>((nchunks + TPR - 1) / TPR, x, rows, D, ldx, g, b, eps, rms, s_t, z, bits, codes, ldc, row_sum, st);
   REPQ_LN_CASE(8)
   REPQ_LN_CASE(16)
   REPQ_LN_CASE(32)
