@@ -40,6 +40,14 @@ __device__ __forceinline__ void load_raw(const float* p, RawChunk<float>& r) {
 __device__ __forceinline__ void load_raw(const __nv_bfloat16* p, RawChunk<__nv_bfloat16>& r) {
   r.a = __ldcs(reinterpret_cast<const uint4*>(p));
 }
+// The same with the second 16 bytes of a float chunk optional (a row stride that ends inside the last chunk).
+__device__ __forceinline__ void load_raw_part(const float* p, bool second, RawChunk<float>& r) {
+  r.a = __ldcs(reinterpret_cast<const float4*>(p));
+  if (second) r.b = __ldcs(reinterpret_cast<const float4*>(p) + 1);
+}
+__device__ __forceinline__ void load_raw_part(const __nv_bfloat16* p, bool, RawChunk<__nv_bfloat16>& r) {
+  r.a = __ldcs(reinterpret_cast<const uint4*>(p));
+}
 __device__ __forceinline__ void expand(const RawChunk<float>& r, f32x2 (&v)[kChunk / 2]) {
   v[0] = pack2(r.a.x, r.a.y); v[1] = pack2(r.a.z, r.a.w); v[2] = pack2(r.b.x, r.b.y); v[3] = pack2(r.b.z, r.b.w);
 }
@@ -239,6 +247,128 @@ softmax_log2_kernel(const T* __restrict__ scores, int64_t rows, int L, int64_t l
   }
 }
 
+// The same computation for the common case: no causal mask, 16-byte aligned rows, and a row stride that covers
+// the last chunk of 8 (or, for float32 scores, its first half when the row ends there).  Which of a thread's chunks are whole, partial or past the row is then the same for every
+// row, so it is decided once; chunk slots that are whole for every thread of a group run without predicates, rows
+// past the end re-read the last row (nothing of them is stored), and the upper clip of Eq. 15 is left to the
+// saturating pack (t = +inf or beyond 2^22 leaves a large positive integer after the magic-number subtraction).
+template <typename T, int TPR, int kVPT, bool kPack4>
+__global__ void __launch_bounds__((TPR > 256 ? TPR : 256), (TPR <= 32 ? 3 : 0))
+softmax_log2_plain_kernel(const T* __restrict__ scores, int64_t rows, int L, int64_t ld, bool tail_half, float c,
+                          float log2_s, int qmax, uint8_t* __restrict__ codes, int64_t ldc) {
+  constexpr int kBlock = TPR > 256 ? TPR : 256;
+  constexpr int kRowsPerBlock = kBlock / TPR;
+  __shared__ float red_a[kBlock / 32];
+  __shared__ float red_b[kBlock / 32];
+
+  const int tig = threadIdx.x % TPR;
+  const int group = threadIdx.x / TPR;
+  const int group_first_warp = (group * TPR) >> 5;
+  const int n_full = (L / kChunk) / TPR;        // chunk slots below this are whole for every thread of a group
+  int cnt[kVPT];                                // visible elements of this thread's chunk i (0..8), any row
+#pragma unroll
+  for (int i = 0; i < kVPT; ++i) {
+    const int left = L - (tig + i * TPR) * kChunk;
+    cnt[i] = left < 0 ? 0 : (left > kChunk ? kChunk : left);
+  }
+  const uint32_t qmax4 = uint32_t(qmax) * 0x01010101u;
+
+  RawChunk<T> raw[kVPT];
+#pragma unroll
+  for (int i = 0; i < kVPT; ++i) raw[i] = RawChunk<T>{};
+  auto fetch = [&](int64_t row) {
+    const T* sr = scores + (row < rows ? row : rows - 1) * ld;
+#pragma unroll
+    for (int i = 0; i < kVPT; ++i)
+      if (i < n_full || cnt[i] > 0)   // tail_half: the row's last chunk holds at most 4 keys and the stride ends after them
+        load_raw_part(sr + (tig + i * TPR) * kChunk, i < n_full || !tail_half || cnt[i] > 4, raw[i]);
+  };
+  const int64_t stride = int64_t(gridDim.x) * kRowsPerBlock;
+  fetch(int64_t(blockIdx.x) * kRowsPerBlock + group);
+
+  const f32x2 c2 = splat2(c);
+  const f32x2 k1 = splat2(-2.f * c);
+  const f32x2 magic2 = splat2(__uint_as_float(kMagicBits));
+  for (int64_t base = int64_t(blockIdx.x) * kRowsPerBlock; base < rows; base += stride) {
+    const int64_t row = base + group;
+    const bool live = row < rows;
+
+    f32x2 v[kVPT][kChunk / 2];
+    float m = -CUDART_INF_F;
+#pragma unroll
+    for (int i = 0; i < kVPT; ++i) {
+      expand(raw[i], v[i]);
+      if (i >= n_full) {                         // a slot that holds the row's ragged end for some thread
+#pragma unroll
+        for (int e = 0; e < kChunk / 2; ++e) {
+          float lo, hi;
+          unpack2(v[i][e], lo, hi);
+          v[i][e] = pack2(2 * e < cnt[i] ? lo : -CUDART_INF_F, 2 * e + 1 < cnt[i] ? hi : -CUDART_INF_F);
+        }
+      }
+#pragma unroll
+      for (int e = 0; e < kChunk / 2; ++e) {
+        float lo, hi;
+        unpack2(v[i][e], lo, hi);
+        m = fmaxf(m, fmaxf(lo, hi));
+      }
+    }
+    fetch(row + stride);
+    m = group_reduce<TPR, true>(m, red_a, group_first_warp);
+
+    // d = S - m (<= 0, -inf for keys past the row); Z = sum 2^(c d)
+    const f32x2 neg_m = splat2(-m);
+    f32x2 zz = 0ull;
+#pragma unroll
+    for (int i = 0; i < kVPT; ++i) {
+      if (i < n_full || cnt[i] > 0) {
+#pragma unroll
+        for (int e = 0; e < kChunk / 2; ++e) {
+          v[i][e] = add2(v[i][e], neg_m);
+          float a0, a1;
+          unpack2(mul2(v[i][e], c2), a0, a1);
+          zz = add2(zz, pack2(ex2(a0), ex2(a1)));
+        }
+      }
+    }
+    float z0, z1;
+    unpack2(zz, z0, z1);
+    const float z = group_reduce<TPR, false>(z0 + z1, red_b, group_first_warp);
+    const f32x2 k0 = splat2(2.f * (log2f(z) + log2_s));
+
+    uint8_t* out = codes + row * ldc;
+#pragma unroll
+    for (int i = 0; i < kVPT; ++i) {
+      const int ch = tig + i * TPR;
+      if (i < n_full || cnt[i] > 0) {
+        // Eq. 15: clip(round(t), 0, qmax); rounding half to even is one packed float add of 1.5 * 2^23, which
+        // leaves the code in the low mantissa bits; both clips are the saturation of the pack (negative t,
+        // possible for s < 1 only, leaves a negative integer; t = +inf for keys past the row and underflowed
+        // probabilities leaves a large positive one)
+        int q[kChunk];
+#pragma unroll
+        for (int e = 0; e < kChunk / 2; ++e) {
+          float r0, r1;
+          unpack2(add2(fma2(v[i][e], k1, k0), magic2), r0, r1);
+          q[2 * e] = __float_as_int(r0) - int(kMagicBits);
+          q[2 * e + 1] = __float_as_int(r1) - int(kMagicBits);
+        }
+        if constexpr (kPack4) {
+          uint32_t w = 0;
+#pragma unroll
+          for (int e = kChunk - 2; e >= 0; e -= 2) w = push_pair_u4(q[e], q[e + 1], w);
+          if (live) reinterpret_cast<uint32_t*>(out)[ch] = w;
+        } else {
+          uint2 w;
+          w.x = __vminu4(push_pair_u8(q[0], q[1], push_pair_u8(q[2], q[3], 0u)), qmax4);   // 6-bit codes in bytes
+          w.y = __vminu4(push_pair_u8(q[4], q[5], push_pair_u8(q[6], q[7], 0u)), qmax4);
+          if (live) reinterpret_cast<uint2*>(out)[ch] = w;
+        }
+      }
+    }
+  }
+}
+
 template <typename T, int TPR, int kVPT>
 repq_status launch(const T* scores, int64_t rows, int L, int64_t ld, bool vec_ok, float c, int period,
                    int offset, float log2_s, int bits, uint8_t* codes, int64_t ldc, cudaStream_t st) {
@@ -246,6 +376,18 @@ repq_status launch(const T* scores, int64_t rows, int L, int64_t ld, bool vec_ok
   constexpr int kRowsPerBlock = kBlock / TPR;
   const int64_t need = (rows + kRowsPerBlock - 1) / kRowsPerBlock;
   const int qmax = code_max(bits);
+  const int64_t chunks8 = (int64_t(L) + kChunk - 1) / kChunk * kChunk;
+  const bool tail_half = chunks8 > ld && sizeof(T) == 4 && L % kChunk >= 1 && L % kChunk <= 4 && chunks8 - 4 <= ld;
+  if (vec_ok && period <= 0 && (chunks8 <= ld || tail_half)) {
+    auto plain = packed4(bits) ? softmax_log2_plain_kernel<T, TPR, kVPT, true> : softmax_log2_plain_kernel<T, TPR, kVPT, false>;
+    int fit = 0;
+    REPQ_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&fit, plain, kBlock, 0));
+    const int64_t most = int64_t(sm_count()) * (fit > 0 ? fit : 1);
+    plain<<<int(need < most ? need : most), kBlock, 0, st>>>(scores, rows, L, ld, tail_half, c, log2_s, qmax, codes, ldc);
+    REPQ_CUDA(cudaGetLastError());
+    note_launch();
+    return REPQ_OK;
+  }
   auto kern = packed4(bits) ? softmax_log2_kernel<T, TPR, kVPT, true> : softmax_log2_kernel<T, TPR, kVPT, false>;
   // persistent grid: exactly the blocks that are resident at once (every block keeps its load pipeline running)
   int resident = 0;

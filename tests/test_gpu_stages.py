@@ -47,6 +47,9 @@ def test_softmax_log2_variants():
     assert parity.check_softmax_log2(300, 197, 4, seed=3, s=0.7)["bad"] == 0
     assert parity.check_softmax_log2(300, 197, 4, seed=4, pre_scale=0.125)["bad"] == 0
     assert parity.check_softmax_log2(300, 197, 4, seed=5, ld_pad=197)["bad"] == 0      # unaligned rows
+    assert parity.check_softmax_log2(300, 197, 8, seed=6, ld_pad=208)["bad"] == 0      # stride beyond the last chunk
+    assert parity.check_softmax_log2(70, 577, 6, seed=7, ld_pad=584)["bad"] == 0       # whole last chunk in the stride
+    assert parity.check_softmax_log2(70, 581, 4, seed=8, ld_pad=584)["bad"] == 0       # stride ends inside the last chunk
 
 
 @pytest.mark.parametrize("M,N,K,ba,bw", [
