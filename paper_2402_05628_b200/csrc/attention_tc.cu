@@ -259,6 +259,18 @@ attention_tc_kernel(AttnParams P) {
     const int row = q0 + r;
     const int valid = row < P.Lq ? (P.causal ? max(1, min(P.Lk, row + 1 + shift)) : P.Lk) : 0;   // keys the row sees
     const int my_row_term = S.row_term[r];
+    // a warp whose 32 rows all lie past Lq (the tail of the last query tile): its rows of the E / O tiles are
+    // cleared once here and never written again, and it skips the code arithmetic of pass 2; it still stages K
+    // and V and arrives on every barrier
+    const bool dead_warp = __all_sync(0xffffffffu, valid == 0);
+    if (dead_warp) {
+#pragma unroll
+      for (int p4 = 0; p4 < kCols / 8; ++p4) {
+        const uint32_t off = tile_offset(r, part * (kCols / 8) + p4);
+        *reinterpret_cast<uint4*>(S.e + off) = make_uint4(0u, 0u, 0u, 0u);
+        *reinterpret_cast<uint4*>(S.o + off) = make_uint4(0u, 0u, 0u, 0u);
+      }
+    }
     const float c = 1.4426950408889634f;
     const float k1 = -2.f * c;
     const float qs = float(P.qmax_p + 1), inv_qs = 1.f / qs;      // 2^bits and its reciprocal (exact)
@@ -383,6 +395,8 @@ attention_tc_kernel(AttnParams P) {
       // from integer arithmetic for wider ones.  A masked key gets (0, 0).
       const bool boundary = j * kKeys + part * kCols + kCols > min(min_valid, valid);
       const uint32_t lut_addr = smem_u32(&S.lut[0][lane]) - (kMagicBits << 7);
+      uint4 ev[kCols / 8], ov[kCols / 8];
+      if (!dead_warp) {
       uint32_t eo[kCols];
 #pragma unroll
       for (int e = 0; e < kCols; ++e) {
@@ -409,7 +423,6 @@ attention_tc_kernel(AttnParams P) {
         for (int e = 0; e < kCols; ++e)
           if (corr[e] == kMasked) eo[e] = 0u;
       }
-      uint4 ev[kCols / 8], ov[kCols / 8];
 #pragma unroll
       for (int p4 = 0; p4 < kCols / 8; ++p4) {
         ev[p4] = make_uint4(__byte_perm(eo[8 * p4 + 0], eo[8 * p4 + 1], 0x5410), __byte_perm(eo[8 * p4 + 2], eo[8 * p4 + 3], 0x5410),
@@ -417,14 +430,17 @@ attention_tc_kernel(AttnParams P) {
         ov[p4] = make_uint4(__byte_perm(eo[8 * p4 + 0], eo[8 * p4 + 1], 0x7632), __byte_perm(eo[8 * p4 + 2], eo[8 * p4 + 3], 0x7632),
                             __byte_perm(eo[8 * p4 + 4], eo[8 * p4 + 5], 0x7632), __byte_perm(eo[8 * p4 + 6], eo[8 * p4 + 7], 0x7632));
       }
+      }
       // one stage of operand tiles: the MMAs of the block before must have read them (the code arithmetic above
       // has overlapped with those MMAs)
       if (!mbar_wait(smem_u32(&S.p_empty), (uint32_t(j) & 1u) ^ 1u, abort, 46, P.status)) return false;
+      if (!dead_warp) {
 #pragma unroll
-      for (int p4 = 0; p4 < kCols / 8; ++p4) {
-        const uint32_t off = tile_offset(r, part * (kCols / 8) + p4);
-        *reinterpret_cast<uint4*>(S.e + off) = ev[p4];
-        *reinterpret_cast<uint4*>(S.o + off) = ov[p4];
+        for (int p4 = 0; p4 < kCols / 8; ++p4) {
+          const uint32_t off = tile_offset(r, part * (kCols / 8) + p4);
+          *reinterpret_cast<uint4*>(S.e + off) = ev[p4];
+          *reinterpret_cast<uint4*>(S.o + off) = ov[p4];
+        }
       }
 #pragma unroll
       for (int qi = 0; qi < kVItems; ++qi) {
