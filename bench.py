@@ -44,7 +44,7 @@ NCU_TRAFFIC = {   # stage: (DRAM bytes read + written per launch, kernel sources
     'qkv': (14292480, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '04dc33d1b726'),
     'attention': (29795840, ['attention_tc.cu', 'tc_ptx.cuh'], 'cd1889cc1260'),
     'scores': (85649408, ['scores_tc.cu', 'tc_ptx.cuh'], '0ec10eb039ae'),
-    'softmax': (129887232, ['softmax_log2.cu', 'f32x2.cuh'], 'c4e0c2ebf28f'),
+    'softmax': (129327104, ['softmax_log2.cu', 'f32x2.cuh'], '9685eb0f7366'),
     'pv': (26712320, ['pv_tc.cu', 'tc_ptx.cuh'], '44d2a2d061d5'),
     'proj': (33026560, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '04dc33d1b726'),
     'fc1': (20006400, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '04dc33d1b726'),
