@@ -64,7 +64,7 @@ struct AttnParams {
   int32_t* status;
 };
 
-template <int NB>
+template <int NB, int kLutBits>
 struct AttnShared {
   alignas(1024) uint8_t q[kQBytes];
   alignas(1024) uint8_t k[2][kKBytes];
@@ -74,8 +74,10 @@ struct AttnShared {
   int row_term[kRows];                              // -z_k qsum[m] + d_h z_q z_k
   int col_term[4][kKeys];                           // -z_q ksum[n], ring of 4 key blocks
   float stat_m[kParts][kRows], stat_z[kParts][kRows];   // pass-1 results of the column parts of every row
-  uint32_t lut[17][32];                             // 4-bit codes: [code][lane] = E value | O value << 16 (one bank per lane);
-                                                    // entry 16 repeats 15 (a clamp at 16 that rounds up lands there)
+  static constexpr int kLutEntries = kLutBits ? (1 << kLutBits) + 1 : 1;
+  uint32_t lut[kLutEntries][32];                    // table-driven codes: [code][lane] = E value | O value << 16 (one bank per
+                                                    // lane); the last entry repeats the top code (a clamp at 2^bits that
+                                                    // rounds up lands there)
   alignas(8) uint64_t k_full[2];
   uint64_t s_full[2], s_empty[2], p_full, p_empty;
   uint64_t stats_ready, acc_full, done;
@@ -101,13 +103,15 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-// NB: 64-channel blocks of the head; kLut: Softmax codes of at most 4 bits (operand values from the per-lane table)
+// NB: 64-channel blocks of the head; kLutBits: width of the Softmax codes when their operand values come from the
+// per-lane table (4, 6, or 8 where one CTA per SM leaves room for 257 entries), 0: integer arithmetic
 // kCentered: Q and K codes minus their zero points fit a signed byte (quantizers of at most 7 bits); the tiles then
 // hold q - z_q and k - z_k, the S MMAs run signed x signed and their accumulators need no zero-point correction.
-template <int NB, bool kLut, bool kCentered>
+template <int NB, int kLutBits, bool kCentered>
 __global__ void __launch_bounds__(kThreads, NB == 1 ? 2 : 1)
 attention_tc_kernel(AttnParams P) {
-  using Shared = AttnShared<NB>;
+  using Shared = AttnShared<NB, kLutBits>;
+  constexpr bool kLut = kLutBits != 0;
   constexpr int kVItems = NB;                             // 8-channel groups of V per thread and block
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   Shared& S = *reinterpret_cast<Shared*>(smem_raw);
@@ -196,9 +200,12 @@ attention_tc_kernel(AttnParams P) {
     s += __shfl_xor_sync(0xffffffffu, s, 1);
     s += __shfl_xor_sync(0xffffffffu, s, 2);
     if (qh == 0) S.row_term[qrow] = -P.zk * s + P.dh * P.zq * P.zk;
-    for (int i = tid; i < 17 * 32; i += kWorkThreads) {
-      const uint32_t code = min(uint32_t(i >> 5), 15u), bits16 = (127u - ((code + 1u) >> 1)) << 7;   // bf16 bits of 2^-ceil(code/2)
-      S.lut[0][i] = (code & 1u) ? bits16 << 16 : bits16;
+    if (kLut) {
+      for (int i = tid; i < Shared::kLutEntries * 32; i += kWorkThreads) {
+        const uint32_t code = min(uint32_t(i >> 5), uint32_t(Shared::kLutEntries - 2)), kk = (code + 1u) >> 1;
+        const uint32_t bits16 = kk > 126u ? 0u : (127u - kk) << 7;   // bf16 bits of 2^-ceil(code/2) (0 below the normal range)
+        S.lut[0][i] = (code & 1u) ? bits16 << 16 : bits16;
+      }
     }
   }
   tc_fence_before();
@@ -402,11 +409,12 @@ attention_tc_kernel(AttnParams P) {
       for (int e = 0; e < kCols; ++e) {
         // clamped on both sides whatever the inputs (rows past Lq carry m = -inf, Z = 0): p indexes the table
         if (kLut) {
-          // 4-bit codes: the clamp to [0, 16] is a saturating multiply by 1/16 (exact), the scaling back and the
-          // rounding one fma; 16 (t in [15.5, 16]) reads the table's copy of entry 15
+          // table-driven codes: the clamp to [0, 2^bits] is a saturating multiply by 2^-bits (exact), the scaling back
+          // and the rounding one fma; 2^bits (t within half a code of it) reads the table's copy of the top entry
           float w;
-          asm("mul.rn.sat.f32 %0, %1, %2;" : "=f"(w) : "f"(fmaf(fmaf(float(corr[e]), P.scale, -m), k1, k0)), "f"(0.0625f));
-          const uint32_t u = __float_as_uint(fmaf(w, 16.f, magic));
+          constexpr float kSteps = float(1 << kLutBits), kInvSteps = 1.f / kSteps;      // 2^bits and its reciprocal (exact)
+          asm("mul.rn.sat.f32 %0, %1, %2;" : "=f"(w) : "f"(fmaf(fmaf(float(corr[e]), P.scale, -m), k1, k0)), "f"(kInvSteps));
+          const uint32_t u = __float_as_uint(fmaf(w, kSteps, magic));
           asm("ld.shared.u32 %0, [%1];" : "=r"(eo[e]) : "r"(lut_addr + (u << 7)));
         } else {
           // wider codes: the same clamp to [0, 2^bits], then the top code by one integer minimum
@@ -582,21 +590,21 @@ attention_tc_kernel(AttnParams P) {
   }
 }
 
-template <int NB, bool kLut, bool kCentered>
+template <int NB, int kLutBits, bool kCentered>
 repq_status launch_kernel(const AttnParams& P, int64_t pairs, cudaStream_t st) {
-  const size_t smem = sizeof(AttnShared<NB>);
-  REPQ_CUDA(cudaFuncSetAttribute(attention_tc_kernel<NB, kLut, kCentered>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+  const size_t smem = sizeof(AttnShared<NB, kLutBits>);
+  REPQ_CUDA(cudaFuncSetAttribute(attention_tc_kernel<NB, kLutBits, kCentered>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
   dim3 grid((P.Lq + kRows - 1) / kRows, unsigned(pairs));
-  REPQ_CUDA(launch_chained(attention_tc_kernel<NB, kLut, kCentered>, grid, dim3(kThreads), smem, st, P));
+  REPQ_CUDA(launch_chained(attention_tc_kernel<NB, kLutBits, kCentered>, grid, dim3(kThreads), smem, st, P));
   note_launch();
   return REPQ_OK;
 }
 
-template <int NB, bool kLut>
+template <int NB, int kLutBits>
 repq_status launch(const AttnParams& P, int64_t pairs, int qmax_qk, cudaStream_t st) {
   // q - z_q and k - z_k as signed bytes: codes and zero points below 128 and differences within [-128, 127]
   const bool centred = qmax_qk < 128 && P.zq >= 0 && P.zq < 128 && P.zk >= 0 && P.zk < 128;
-  return centred ? launch_kernel<NB, kLut, true>(P, pairs, st) : launch_kernel<NB, kLut, false>(P, pairs, st);
+  return centred ? launch_kernel<NB, kLutBits, true>(P, pairs, st) : launch_kernel<NB, kLutBits, false>(P, pairs, st);
 }
 
 }  // namespace
@@ -658,7 +666,14 @@ extern "C" repq_status repq_attention(const repq_attention_desc* d, void* stream
   P.status = device_status_word();
   REPQ_REQUIRE(P.status != nullptr, REPQ_CUDA_ERROR, "attention: device status word unavailable");
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const bool lut = P.qmax_p <= 15;
-  if (d->d_h <= 64) return lut ? launch<1, true>(P, pairs, qmax_v, st) : launch<1, false>(P, pairs, qmax_v, st);
-  return lut ? launch<2, true>(P, pairs, qmax_v, st) : launch<2, false>(P, pairs, qmax_v, st);
+  // the per-lane table of the Softmax codes' operand values: 17 / 65 entries everywhere; the 257 entries of 8-bit codes
+  // (33 KB) only where the head already limits the SM to one CTA
+  if (d->d_h <= 64) {
+    if (P.qmax_p <= 15) return launch<1, 4>(P, pairs, qmax_v, st);
+    if (P.qmax_p <= 63) return launch<1, 6>(P, pairs, qmax_v, st);
+    return launch<1, 0>(P, pairs, qmax_v, st);
+  }
+  if (P.qmax_p <= 15) return launch<2, 4>(P, pairs, qmax_v, st);
+  if (P.qmax_p <= 63) return launch<2, 6>(P, pairs, qmax_v, st);
+  return launch<2, 8>(P, pairs, qmax_v, st);
 }

@@ -124,7 +124,8 @@ def test_scores_from_byte_codes_match_oracle(Bn, H, Lq, Lk, dh, bits, causal):
 @pytest.mark.parametrize("Bn,H,Lq,Lk,dh,bits,bp,causal", [
     (2, 3, 197, 197, 64, 4, 4, False), (1, 2, 577, 577, 64, 4, 4, False), (1, 2, 300, 300, 128, 4, 8, True),
     (2, 2, 64, 64, 32, 6, 6, False), (1, 1, 1, 130, 16, 8, 8, False), (1, 2, 100, 260, 48, 4, 4, True),
-    (1, 1, 70, 70, 96, 8, 4, True), (1, 2, 700, 700, 64, 4, 4, True),
+    (1, 1, 70, 70, 96, 8, 4, True), (1, 2, 700, 700, 64, 4, 4, True), (1, 2, 150, 150, 128, 6, 6, False),
+    (1, 2, 300, 300, 64, 4, 6, True),
 ])
 def test_fused_attention_matches_oracle(Bn, H, Lq, Lk, dh, bits, bp, causal):
     parity.check_attention(Bn, H, Lq, Lk, dh, bits, bp, causal, seed=Lq + dh)
