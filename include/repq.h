@@ -168,7 +168,9 @@ repq_status repq_qgemm(const repq_gemm_desc* d, void* workspace, size_t workspac
 /* Softmax (Eq. 3) over each row of `scores`, then the log-sqrt2 quantizer in its base-2 form
  * (Eq. 15, second line):  A = softmax(pre_scale * scores_row);
  *     p = clip(round(-2 log2(A / s)), 0, 2^bits - 1).
- * scores [device]: rows x L, REPQ_F32 or REPQ_BF16, row stride ld elements.
+ * scores [device]: rows x L, REPQ_F32 or REPQ_BF16, row stride ld elements; the buffer holds rows x ld elements
+ * and the padding [L, ld) of a row may be read (its values are ignored).  Rows that start on a 16-byte boundary
+ * with a 16-byte multiple stride take the fast kernels.
  * Causal masking is structural: if causal_period > 0, row r sees only its first
  *     min(L, (r mod causal_period) + 1 + causal_offset) keys;
  * codes of masked keys are written as 2^bits - 1 and must not be read as probabilities.
