@@ -42,7 +42,7 @@ NCU_TRAFFIC = {   # stage: (DRAM bytes read + written per launch, kernel sources
     'ln1': (19393280, ['ln_quant.cu', 'f32x2.cuh'], '49b01de9f539'),
     'ln2': (19393280, ['ln_quant.cu', 'f32x2.cuh'], '49b01de9f539'),
     'qkv': (14292480, ['qgemm_tc.cu', 'tc_ptx.cuh', 'epilogue.cuh'], '04dc33d1b726'),
-    'attention': (29788928, ['attention_tc.cu', 'tc_ptx.cuh'], '95b157b7408b'),
+    'attention': (30422016, ['attention_tc.cu', 'tc_ptx.cuh'], 'fbb5e4d22f81'),
     'scores': (85649408, ['scores_tc.cu', 'tc_ptx.cuh'], '0ec10eb039ae'),
     'softmax': (129327104, ['softmax_log2.cu', 'f32x2.cuh'], '9685eb0f7366'),
     'pv': (26712320, ['pv_tc.cu', 'tc_ptx.cuh'], '44d2a2d061d5'),
