@@ -20,8 +20,11 @@ check of the paper's equivalence claims as well as of the kernels.
 Pins (see tests/test_oracle_pins.py): every function below is tied to the
 paper's worked example, a closed form, an algebraic identity of Sec. III-C, a
 library routine for the un-quantized special case, or brute force on tiny
-inputs.  The end-to-end block (`block_forward`) has no external pin beyond the
-composition of its pinned parts: parity unpinned for the composition itself.
+inputs.  The block composition (`block_forward`, both block forms) is pinned by
+a second statement of Eqs. 1-3 and of the quantizer placement written as
+explicit per-token / per-head / per-channel loops on tiny blocks, which shares
+only the pinned leaf quantizers with it, and is compared with it on the
+output, the residual stream and every intermediate code tensor.
 
 Notation follows the paper: s, z quantization scale / zero-point; b bits;
 r1 = s / s~, r2 = z - z~; gamma~, beta~, W~, b~ the reparameterized parameters.
@@ -236,6 +239,33 @@ def round_bf16(x):
     return np.ldexp(np.rint(m * 256.0) / 256.0, e)
 
 
+def silu(x):
+    """SiLU, x sigmoid(x): the gate non-linearity of the LLaMA-style MLP (not in the paper's block; see
+    `block_forward`)."""
+    x = np.asarray(x, dtype=F64)
+    return x / (1.0 + np.exp(-x))
+
+
+def rope(X, B: int, L: int, H: int, base: float = 10000.0):
+    """Rotary position embedding on a [B*L, D] matrix of H heads (not in the paper's block; the LLaMA models of
+    Sec. IV-A apply it to Q and K).  Within a head of d_h channels, the consecutive pair (2i, 2i+1) of the token
+    at position m is one complex number, multiplied by exp(j m theta_i), theta_i = base^(-2i / d_h):
+        x'[2i]   = x[2i] cos(m theta_i) - x[2i+1] sin(m theta_i)
+        x'[2i+1] = x[2i] sin(m theta_i) + x[2i+1] cos(m theta_i)."""
+    X = np.asarray(X, dtype=F64)
+    M, D = X.shape
+    dh = D // H
+    theta = F64(base) ** (-np.arange(0, dh, 2, dtype=F64) / F64(dh))       # [dh/2]
+    ang = np.arange(L, dtype=F64)[:, None] * theta[None, :]                 # [L, dh/2]
+    cos = np.tile(np.cos(ang), (B, H))                                      # [B*L, D/2]
+    sin = np.tile(np.sin(ang), (B, H))
+    even, odd = X[:, 0::2], X[:, 1::2]
+    out = np.empty_like(X)
+    out[:, 0::2] = even * cos - odd * sin
+    out[:, 1::2] = even * sin + odd * cos
+    return out
+
+
 def attention(Qc, Kc, Vc, qp: dict, B: int, L: int, H: int, softmax_s: float, bits_p: int,
               causal: bool, keep: bool = False):
     """Eq. 3 per (batch, head) on de-quantized Q, K, V, with the Softmax output passed through the
@@ -277,6 +307,15 @@ def block_forward(w, keep: bool = False) -> Dict[str, np.ndarray]:
     log-sqrt2.  Every other activation: layer-wise uniform.  Weights: channel-wise RTN; the weights
     that follow a LayerNorm are the reparameterized W~ (rounded to float32, as stored).
     With bf16 activations the residual stream X_bar is stored in bf16.
+
+    Two block forms.  The default is the paper's own block (LayerNorm, MLP = fc2(GELU(fc1(.)))).  The paper also
+    evaluates LLaMA models (Sec. IV-A) but never writes their block down; `cfg["arch"] == "llama"` selects that
+    form, with the same quantizer placement (every matrix-multiplication input quantized): the normalisation is
+    the mean-free one (RMSNorm: Eq. 9 with E[X] := 0, Var := E[X^2]; its channel-wise quantizer is reparameterized
+    by Eqs. 10-14 all the same, beta being whatever the workload holds, zero for RMSNorm), rotary position
+    embedding is applied to the full-precision Q and K of the projection before their quantizers, and the MLP is
+    down(SiLU(gate(.)) * up(.)) with `w_fc1` = [gate; up] stacked on the output axis, the product being the
+    quantized input of the down projection `w_fc2`.
     """
     cfg = w.cfg
     B, L, D, H = cfg["B"], cfg["L"], cfg["D"], cfg["H"]
@@ -284,8 +323,10 @@ def block_forward(w, keep: bool = False) -> Dict[str, np.ndarray]:
     out: Dict[str, np.ndarray] = {}
     x = np.asarray(w.x, dtype=F64)
 
+    llama = cfg.get("arch", "vit") == "llama"
+
     def post_ln_linear(X_in, gamma, beta, lo, hi, W, b, tag):
-        X1 = layernorm(X_in, gamma, beta, cfg["eps"])
+        X1 = layernorm(X_in, gamma, beta, cfg["eps"], rms=llama)
         s, z = uniform_scale_zero(lo, hi, ba)
         q, t = quant_uniform(X1, s[None, :], z[None, :], ba)            # channel-wise
         rp = reparam_layernorm(gamma, beta, s, z, W, b)
@@ -308,8 +349,12 @@ def block_forward(w, keep: bool = False) -> Dict[str, np.ndarray]:
         return q, float(s), int(z)
 
     qkv = post_ln_linear(x, w.ln1_gamma, w.ln1_beta, w.ln1_lo, w.ln1_hi, w.w_qkv, w.b_qkv, "ln1")
-    Qc, s_q, z_q = requant(qkv[:, :D], "q")
-    Kc, s_k, z_k = requant(qkv[:, D:2 * D], "k")
+    Q_fp, K_fp = qkv[:, :D], qkv[:, D:2 * D]
+    if llama:
+        Q_fp = rope(Q_fp, B, L, H, cfg.get("rope_base", 10000.0))
+        K_fp = rope(K_fp, B, L, H, cfg.get("rope_base", 10000.0))
+    Qc, s_q, z_q = requant(Q_fp, "q")
+    Kc, s_k, z_k = requant(K_fp, "k")
     Vc, s_v, z_v = requant(qkv[:, 2 * D:], "v")
     qp = dict(s_q=s_q, z_q=z_q, s_k=s_k, z_k=z_k, s_v=s_v, z_v=z_v)
     O, kept = attention(Qc, Kc, Vc, qp, B, L, H, w.softmax_scale, bp, cfg["causal"], keep)
@@ -325,7 +370,12 @@ def block_forward(w, keep: bool = False) -> Dict[str, np.ndarray]:
         out["x_bar"] = x_bar
 
     h_pre = post_ln_linear(x_bar, w.ln2_gamma, w.ln2_beta, w.ln2_lo, w.ln2_hi, w.w_fc1, w.b_fc1, "ln2")
-    hc, s_h, z_h = requant(gelu(h_pre), "hidden")
+    if llama:
+        n_mlp = cfg["MLP"]
+        h_act = silu(h_pre[:, :n_mlp]) * h_pre[:, n_mlp:]
+    else:
+        h_act = gelu(h_pre)
+    hc, s_h, z_h = requant(h_act, "hidden")
     wc, s_w, z_w = quant_weight_rtn(w.w_fc2, bw)
     out["y"] = linear(dequant_uniform(hc, s_h, z_h), wc, s_w, z_w, w.b_fc2) + x_bar
     return out

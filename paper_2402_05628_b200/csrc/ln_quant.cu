@@ -8,9 +8,10 @@
 // loads stay in flight all the time.
 // The per-channel factors gamma~/s~ and beta~/s~ are staged once per CTA in shared memory.
 //
-// The float work runs on packed pairs (two elements per add / mul / fma issue slot).  Rounding is the
-// float -> int conversion (half to even, on t itself, as Eq. 4 has it); z is added as an integer and the
-// clip of Eq. 4 is the saturation of the packing instruction.
+// The float work runs on packed pairs (two elements per add / mul / fma issue slot).  Rounding is done by the
+// float adder: t + 1.5 * 2^23 leaves rint(t) (half to even, on t itself, as Eq. 4 has it) in the low mantissa
+// bits while |t| < 2^22; inputs that cannot guarantee that bound are clamped and converted with cvt.rni
+// instead.  z is added as an integer and the clip of Eq. 4 is the saturation of the packing instruction.
 #include <cuda_bf16.h>
 
 #include "common.h"
@@ -101,10 +102,13 @@ ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
   constexpr int kGroups = kBlock / TPR;
   constexpr int kRowsPerBlock = kGroups * kRows;
   extern __shared__ __align__(16) float s_gb[];          // g[D] then b[D]: gamma~/s~ and beta~/s~
-  // one array per reduction of a row: it can only be overwritten after every thread of the block has
-  // passed the barrier of a later reduction, hence has finished reading it
+  // One array per reduction of a row.  A slot may be overwritten only after every thread of the block has passed
+  // a barrier that follows its reads of the slot.  With two or three reductions per iteration the barrier of the
+  // next reduction is that barrier; the mean-free form without row sums has the variance reduction alone (one
+  // barrier per iteration), so red_b alternates between two halves by iteration parity: the write of iteration
+  // k + 2 follows the barrier of iteration k + 1, which every thread reaches after its reads of iteration k.
   __shared__ float red_a[kBlock / 32 * kRows];
-  __shared__ float red_b[kBlock / 32 * kRows];
+  __shared__ float red_b[2][kBlock / 32 * kRows];
   __shared__ int red_c[kBlock / 32 * kRows];
 
   float* s_g = s_gb;
@@ -155,7 +159,8 @@ ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
   const int64_t stride = int64_t(gridDim.x) * kRowsPerBlock;
   fetch(int64_t(blockIdx.x) * kRowsPerBlock + group * kRows);
 
-  for (int64_t base = int64_t(blockIdx.x) * kRowsPerBlock; base < rows; base += stride) {
+  int parity = 0;
+  for (int64_t base = int64_t(blockIdx.x) * kRowsPerBlock; base < rows; base += stride, parity ^= 1) {
     const int64_t row0 = base + group * kRows;
 
     f32x2 v[kRows][kVPT][kChunk / 2];
@@ -206,7 +211,7 @@ ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
       unpack2(acc, lo, hi);
       ss[r] = lo + hi;
     }
-    group_reduce<TPR, kRows, float>(ss, red_b, group_first_warp);
+    group_reduce<TPR, kRows, float>(ss, red_b[parity], group_first_warp);
     f32x2 rstd[kRows];
 #pragma unroll
     for (int r = 0; r < kRows; ++r) rstd[r] = splat2(rsqrtf(ss[r] * inv_d + eps));

@@ -351,3 +351,264 @@ def test_block_error_shrinks_with_bits():
         errs.append(np.linalg.norm(y - ref) / np.linalg.norm(ref))
     assert errs[0] > errs[1] > errs[2]
     assert errs[2] < 0.05
+
+
+# ------------------------------------------------------------------ block composition (pin)
+
+def _loop_block(w):
+    """Eqs. 1-3 and the quantizer placement of Sec. III-A / IV-A written out a second time, token by token, head
+    by head and channel by channel, for tiny blocks.  It shares only the leaf quantizers (pinned above) with
+    `block_forward`: the normalisation, the reparameterization (Eqs. 10-14), the shifted linear layer (Eq. 13,
+    right-hand side), the Softmax, the rotary embedding, the non-linearities and every index are restated here
+    with Python scalars."""
+    import cmath
+    cfg = w.cfg
+    B, L, D, H, MLP = cfg["B"], cfg["L"], cfg["D"], cfg["H"], cfg["MLP"]
+    ba, bw, bp = cfg["bits_a"], cfg["bits_w"], cfg["bits_p"]
+    dh = D // H
+    M = B * L
+    llama = cfg.get("arch", "vit") == "llama"
+    kept = {}
+
+    def normalise(row, gamma, beta):
+        row = [float(v) for v in row]
+        mu = 0.0 if llama else sum(row) / D
+        var = sum((v - mu) ** 2 for v in row) / D
+        return [(v - mu) / math.sqrt(var + cfg["eps"]) * float(gamma[c]) + float(beta[c]) for c, v in enumerate(row)]
+
+    def rtn_rows(Wm):
+        q, s_w, z_w = orc.quant_weight_rtn(Wm, bw)
+        return [[float(s_w[j]) * (int(q[j, c]) - int(z_w[j])) for c in range(Wm.shape[1])] for j in range(Wm.shape[0])]
+
+    def after_norm(X_in, gamma, beta, lo, hi, W, b, tag):
+        N = W.shape[0]
+        s, z = orc.uniform_scale_zero(lo, hi, ba)
+        s_t = sum(float(v) for v in s) / D
+        z_mean = sum(int(v) for v in z) / D
+        z_t = int(np.rint(z_mean))
+        r1 = [float(s[c]) / s_t for c in range(D)]
+        r2 = [int(z[c]) - z_t for c in range(D)]
+        # W~ (stored in float32) and its channel-wise RTN de-quantization; b~ from the full-precision W
+        W_t = np.array([[np.float32(r1[c] * float(W[j, c])) for c in range(D)] for j in range(N)], dtype=np.float64)
+        W_hat = rtn_rows(W_t)
+        b_t = [float(b[j]) - sum(float(s[c]) * r2[c] * float(W[j, c]) for c in range(D)) for j in range(N)]
+        codes = np.zeros((M, D), dtype=np.int64)
+        Y = np.zeros((M, N))
+        for n in range(M):
+            x1 = normalise(X_in[n], gamma, beta)
+            for c in range(D):
+                codes[n, c] = int(orc.quant_uniform(x1[c], float(s[c]), int(z[c]), ba)[0])
+            x_hat = [float(s[c]) * (int(codes[n, c]) - int(z[c])) for c in range(D)]
+            shifted = [(x_hat[c] + float(s[c]) * r2[c]) / r1[c] for c in range(D)]
+            for j in range(N):
+                Y[n, j] = sum(shifted[c] * W_hat[j][c] for c in range(D)) + b_t[j]
+        kept[tag + "_codes"] = codes
+        return Y
+
+    def layerwise(V, name):
+        lo, hi = w.bounds[name]
+        s, z = orc.uniform_scale_zero(lo, hi, ba)
+        q = np.zeros(V.shape, dtype=np.int64)
+        for i in range(V.shape[0]):
+            for j in range(V.shape[1]):
+                q[i, j] = int(orc.quant_uniform(float(V[i, j]), float(s), int(z), ba)[0])
+        kept[name + "_codes"] = q
+        return q, float(s) * (q.astype(np.float64) - int(z))
+
+    def plain_linear(X_hat, W, b):
+        W_hat = rtn_rows(np.asarray(W, dtype=np.float64))
+        N = W.shape[0]
+        out = np.zeros((X_hat.shape[0], N))
+        for n in range(X_hat.shape[0]):
+            for j in range(N):
+                out[n, j] = sum(float(X_hat[n, c]) * W_hat[j][c] for c in range(X_hat.shape[1])) + float(b[j])
+        return out
+
+    x = np.asarray(w.x, dtype=np.float64)
+    qkv = after_norm(x, w.ln1_gamma, w.ln1_beta, w.ln1_lo, w.ln1_hi, w.w_qkv, w.b_qkv, "ln1")
+    Q, K, V = qkv[:, :D].copy(), qkv[:, D:2 * D].copy(), qkv[:, 2 * D:].copy()
+    if llama:
+        base = cfg.get("rope_base", 10000.0)
+        for T in (Q, K):
+            for n in range(M):
+                pos = n % L
+                for h in range(H):
+                    for i in range(dh // 2):
+                        c0 = h * dh + 2 * i
+                        zc = complex(T[n, c0], T[n, c0 + 1]) * cmath.exp(1j * pos * base ** (-2.0 * i / dh))
+                        T[n, c0], T[n, c0 + 1] = zc.real, zc.imag
+    _, Qh = layerwise(Q, "q")
+    _, Kh = layerwise(K, "k")
+    _, Vh = layerwise(V, "v")
+    O = np.zeros((M, D))
+    p_codes = []
+    for b_ in range(B):
+        for h in range(H):
+            pc = np.zeros((L, L), dtype=np.int64)
+            for i in range(L):
+                n_keys = i + 1 if cfg["causal"] else L
+                sc = [sum(Qh[b_ * L + i, h * dh + d] * Kh[b_ * L + j, h * dh + d] for d in range(dh)) / math.sqrt(dh)
+                      for j in range(n_keys)]
+                mx = max(sc)
+                e = [math.exp(v - mx) for v in sc]
+                tot = sum(e)
+                for j in range(n_keys):
+                    code = int(orc.quant_logsqrt2(e[j] / tot, w.softmax_scale, bp)[0])
+                    pc[i, j] = code
+                    a_hat = float(orc.dequant_logsqrt2(code, w.softmax_scale))
+                    for d in range(dh):
+                        O[b_ * L + i, h * dh + d] += a_hat * Vh[b_ * L + j, h * dh + d]
+            p_codes.append(pc)
+    kept["p_codes"] = p_codes
+    _, Oh = layerwise(O, "attn")
+    x_bar = plain_linear(Oh, w.w_proj, w.b_proj) + x
+    if cfg["act"] == "bf16":
+        x_bar = orc.round_bf16(x_bar)
+    kept["x_bar"] = x_bar
+    pre = after_norm(x_bar, w.ln2_gamma, w.ln2_beta, w.ln2_lo, w.ln2_hi, w.w_fc1, w.b_fc1, "ln2")
+    if llama:
+        act = np.array([[pre[n, j] / (1.0 + math.exp(-pre[n, j])) * pre[n, MLP + j] for j in range(MLP)] for n in range(M)])
+    else:
+        act = np.array([[0.5 * pre[n, j] * (1.0 + math.erf(pre[n, j] / math.sqrt(2.0))) for j in range(MLP)] for n in range(M)])
+    _, Hh = layerwise(act, "hidden")
+    kept["y"] = plain_linear(Hh, w.w_fc2, w.b_fc2) + x_bar
+    return kept
+
+
+def _soft_attention(w, k=7e-4):
+    """The generator's attention temperature gives nearly one-hot Softmax rows at 5 tokens; scale the query
+    projection (and its clipping bounds) down so that the tiny block's Softmax codes take many values."""
+    import dataclasses
+    D = w.cfg["D"]
+    w_qkv, b_qkv = w.w_qkv.copy(), w.b_qkv.copy()
+    w_qkv[:D] *= np.float32(k)
+    b_qkv[:D] *= np.float32(k)
+    bounds = dict(w.bounds)
+    bounds["q"] = (np.float32(w.bounds["q"][0] * k), np.float32(w.bounds["q"][1] * k))
+    return dataclasses.replace(w, w_qkv=w_qkv, b_qkv=b_qkv, bounds=bounds)
+
+
+@pytest.mark.parametrize("name,causal,act", [
+    ("c1_vit_s", False, "f32"), ("c1_vit_s", True, "bf16"), ("c4_llama7b_arch", True, "bf16"),
+    ("c4_llama7b_arch", False, "f32"),
+])
+def test_block_forward_against_loop_written_block(name, causal, act):
+    """`block_forward` against the loop-written block: the output, the residual stream and every code tensor."""
+    w = _soft_attention(make_block_inputs(name, batch=2, D=8, H=2, MLP=16, L=5, causal=causal, act=act, bits_p=4,
+                                          massive=1, calib_samples=32))
+    got = orc.block_forward(w, keep=True)
+    ref = _loop_block(w)
+    L, causal_ = w.cfg["L"], w.cfg["causal"]
+    checked = 0
+    for key in ("ln1_codes", "q_codes", "k_codes", "v_codes", "attn_codes", "ln2_codes", "hidden_codes"):
+        a, b = np.asarray(got[key]), np.asarray(ref[key])
+        assert a.shape == b.shape
+        if not np.array_equal(a, b):
+            # the two statements round the same real number computed in two orders: a code may differ only where
+            # the value handed to the round operation is a tie up to float64 round-off
+            t = np.asarray(got[key[:-6] + "_t"])
+            bad = (a != b) & ~((np.abs(a - b) == 1) & (np.abs(t - np.floor(t) - 0.5) < 1e-9))
+            assert not bad.any(), key
+        checked += a.size
+    for pair, (pa, pb) in enumerate(zip(got["p_codes"], ref["p_codes"])):
+        mask = np.tril(np.ones((L, L), dtype=bool)) if causal_ else np.ones((L, L), dtype=bool)
+        assert np.array_equal(np.asarray(pa)[mask], pb[mask]), pair
+        checked += int(mask.sum())
+    assert checked > 500
+    assert np.abs(got["x_bar"] - ref["x_bar"]).max() <= 1e-11 * np.abs(ref["x_bar"]).max()
+    assert np.abs(got["y"] - ref["y"]).max() <= 1e-11 * np.abs(ref["y"]).max()
+    # the codes are not degenerate: several distinct values per tensor, Softmax codes included
+    assert len(np.unique(got["ln1_codes"])) > 4 and len(np.unique(got["hidden_codes"])) > 2
+    assert len(np.unique(np.concatenate([np.asarray(p).ravel() for p in got["p_codes"]]))) > 3
+
+
+def _mutated(fn_name, replacement):
+    class _Swap:
+        def __enter__(self):
+            self.old = getattr(orc, fn_name)
+            setattr(orc, fn_name, replacement)
+        def __exit__(self, *a):
+            setattr(orc, fn_name, self.old)
+    return _Swap()
+
+
+def test_loop_written_block_catches_planted_mistakes():
+    """Mistakes planted in the oracle's composition (on the CPU) make the comparison above fail: a dropped bias
+    compensation (Eq. 14), a missing bf16 rounding of the residual stream, swapped K / V bounds, GELU after the
+    hidden quantizer instead of before it."""
+    w = _soft_attention(make_block_inputs("c1_vit_s", batch=1, D=8, H=2, MLP=16, L=5, act="bf16", calib_samples=32))
+    ref = _loop_block(w)
+    base = orc.block_forward(w)["y"]
+    assert np.abs(base - ref["y"]).max() <= 1e-11 * np.abs(ref["y"]).max()
+
+    def differs(y):
+        return np.abs(y - ref["y"]).max() > 1e-6 * np.abs(ref["y"]).max()
+
+    real_reparam = orc.reparam_layernorm
+    def no_bias_compensation(gamma, beta, s, z, W, b):
+        rp = dict(real_reparam(gamma, beta, s, z, W, b))
+        rp["b_t"] = np.zeros(W.shape[0]) if b is None else np.asarray(b, dtype=np.float64)
+        return rp
+    with _mutated("reparam_layernorm", no_bias_compensation):
+        assert differs(orc.block_forward(w)["y"])
+    with _mutated("round_bf16", lambda v: np.asarray(v, dtype=np.float64)):
+        assert differs(orc.block_forward(w)["y"])
+    import dataclasses
+    swapped = dict(w.bounds)
+    swapped["k"], swapped["v"] = w.bounds["v"], w.bounds["k"]
+    assert differs(orc.block_forward(dataclasses.replace(w, bounds=swapped))["y"])
+    real_gelu = orc.gelu
+    with _mutated("gelu", lambda v: np.asarray(v, dtype=np.float64)):
+        y_no_gelu = orc.block_forward(w)["y"]
+    assert differs(y_no_gelu)
+
+
+# ------------------------------------------------------------------ rotary embedding and SiLU (LLaMA block form)
+
+def test_rope_against_complex_rotation_and_its_invariants():
+    import cmath
+    rng = np.random.default_rng(21)
+    B, L, H, dh = 2, 7, 3, 8
+    X = rng.normal(size=(B * L, H * dh))
+    Y = orc.rope(X, B, L, H, base=10000.0)
+    for n in range(B * L):
+        m = n % L
+        for h in range(H):
+            for i in range(dh // 2):
+                c0 = h * dh + 2 * i
+                zc = complex(X[n, c0], X[n, c0 + 1]) * cmath.exp(1j * m * 10000.0 ** (-2.0 * i / dh))
+                assert abs(Y[n, c0] - zc.real) < 1e-13 and abs(Y[n, c0 + 1] - zc.imag) < 1e-13
+    # position 0 is the identity; a rotation keeps every pair's length
+    assert np.array_equal(Y[0], X[0]) and np.array_equal(Y[L], X[L])
+    assert np.allclose((Y.reshape(-1, 2) ** 2).sum(1), (X.reshape(-1, 2) ** 2).sum(1), rtol=1e-13)
+    # relative-position property: <rope(q)_m, rope(k)_n> depends on m - n only
+    q, k = rng.normal(size=(1, dh)), rng.normal(size=(1, dh))
+    Qr = orc.rope(np.repeat(q, L, axis=0), 1, L, 1)
+    Kr = orc.rope(np.repeat(k, L, axis=0), 1, L, 1)
+    G = Qr @ Kr.T
+    for d in range(-(L - 1), L):
+        diag = np.diagonal(G, offset=-d)
+        assert np.allclose(diag, diag[0], atol=1e-12)
+    # the first pair rotates by one radian per position (theta_0 = 1)
+    e0 = np.zeros((L, dh)); e0[:, 0] = 1.0
+    R = orc.rope(e0, 1, L, 1)
+    assert np.allclose(R[:, 0], np.cos(np.arange(L))) and np.allclose(R[:, 1], np.sin(np.arange(L)))
+
+
+def test_silu_matches_library():
+    x = np.linspace(-12, 12, 2401)
+    ref = torch.nn.functional.silu(torch.from_numpy(x)).numpy()
+    assert np.abs(orc.silu(x) - ref).max() < 1e-15
+    assert orc.silu(np.array([0.0]))[0] == 0.0
+
+
+def test_llama_form_reduces_to_paper_form_pieces():
+    """RMS normalisation of a zero-mean row equals LayerNorm of it; rotary embedding with every token at
+    position 0 (L = 1) leaves the block's attention unchanged."""
+    rng = np.random.default_rng(5)
+    X = rng.normal(size=(6, 16))
+    X -= X.mean(axis=1, keepdims=True)
+    g, b = rng.normal(size=16), rng.normal(size=16)
+    assert np.allclose(orc.layernorm(X, g, b, 1e-6, rms=True), orc.layernorm(X, g, b, 1e-6), rtol=1e-12, atol=1e-12)
+    ref = torch.nn.functional.rms_norm(torch.from_numpy(X + 0.3), (16,), weight=torch.from_numpy(g), eps=1e-6).numpy() + b
+    assert np.allclose(orc.layernorm(X + 0.3, g, b, 1e-6, rms=True), ref, rtol=1e-12, atol=1e-12)

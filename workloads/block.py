@@ -39,6 +39,11 @@ BLOCK_CONFIGS: Dict[str, dict] = {
     "c4_llama7b": dict(B=4, L=2048, D=4096, H=32, MLP=11008, bits_a=4, bits_w=4, bits_p=8, act="bf16",
                        sigma_c=1.0, outlier_frac=0.0, outlier_mul=1.0, massive=4, eps=1e-5,
                        causal=True, calib_samples=1, seed=3),
+    # the same shapes in the LLaMA block form: RMSNorm (no shift), rotary embedding on Q and K, gated MLP
+    # (w_fc1 = [gate; up] stacked on the output axis, w_fc2 = down), no biases
+    "c4_llama7b_arch": dict(B=4, L=2048, D=4096, H=32, MLP=11008, bits_a=4, bits_w=4, bits_p=8, act="bf16",
+                            sigma_c=1.0, outlier_frac=0.0, outlier_mul=1.0, massive=4, eps=1e-5,
+                            causal=True, calib_samples=1, seed=3, arch="llama", rope_base=10000.0),
 }
 
 
@@ -65,12 +70,22 @@ class BlockInputs:
     ln2_beta: np.ndarray
     ln2_lo: np.ndarray
     ln2_hi: np.ndarray
-    w_fc1: np.ndarray            # [MLP, D]
+    w_fc1: np.ndarray            # [MLP, D]; LLaMA block form: [2 MLP, D] = gate rows, then up rows
     b_fc1: np.ndarray
     w_fc2: np.ndarray            # [D, MLP]
     b_fc2: np.ndarray
     bounds: Dict[str, tuple]     # 'q','k','v','attn','hidden' -> (lo, hi) float32 scalars
     softmax_scale: float         # scale s of the log-sqrt2 quantizer
+
+
+def _rotary(t, n, L, H, dh, base):
+    """Rotary position embedding through torch's complex multiply: consecutive channel pairs of a head are one
+    complex number, rotated by position * base^(-2i/d_h)."""
+    theta = torch.pow(torch.tensor(base, dtype=torch.float64), -torch.arange(0, dh, 2, dtype=torch.float64) / dh)
+    ang = torch.arange(L, dtype=torch.float64)[:, None] * theta[None, :]
+    rot = torch.polar(torch.ones_like(ang), ang)                       # [L, dh/2]
+    tc = torch.view_as_complex(t.double().reshape(n, L, H, dh // 2, 2).contiguous())
+    return torch.view_as_real(tc * rot[None, :, None, :]).reshape(n, L, H * dh).to(t.dtype)
 
 
 def _fp_forward(x, p, cfg, want_attn_stats: bool = False):
@@ -79,9 +94,19 @@ def _fp_forward(x, p, cfg, want_attn_stats: bool = False):
     D, H = cfg["D"], cfg["H"]
     dh = D // H
     n, L, _ = x.shape
-    x1 = F.layer_norm(x, (D,), p["ln1_gamma"], p["ln1_beta"], cfg["eps"])
+    llama = cfg.get("arch", "vit") == "llama"
+
+    def norm(t, g, b):
+        if llama:
+            return F.rms_norm(t, (D,), weight=g, eps=cfg["eps"]) + b
+        return F.layer_norm(t, (D,), g, b, cfg["eps"])
+
+    x1 = norm(x, p["ln1_gamma"], p["ln1_beta"])
     qkv = F.linear(x1, p["w_qkv"], p["b_qkv"])
     q, k, v = qkv.split(D, dim=-1)
+    if llama:
+        q = _rotary(q, n, L, H, dh, cfg.get("rope_base", 10000.0))
+        k = _rotary(k, n, L, H, dh, cfg.get("rope_base", 10000.0))
     qh = q.reshape(n, L, H, dh).transpose(1, 2)
     kh = k.reshape(n, L, H, dh).transpose(1, 2)
     vh = v.reshape(n, L, H, dh).transpose(1, 2)
@@ -94,8 +119,13 @@ def _fp_forward(x, p, cfg, want_attn_stats: bool = False):
         return a.amax(dim=-1)
     o = torch.matmul(a, vh).transpose(1, 2).reshape(n, L, D)
     xbar = F.linear(o, p["w_proj"], p["b_proj"]) + x
-    x2 = F.layer_norm(xbar, (D,), p["ln2_gamma"], p["ln2_beta"], cfg["eps"])
-    h = F.gelu(F.linear(x2, p["w_fc1"], p["b_fc1"]))
+    x2 = norm(xbar, p["ln2_gamma"], p["ln2_beta"])
+    h = F.linear(x2, p["w_fc1"], p["b_fc1"])
+    if llama:
+        gate, up = h.split(cfg["MLP"], dim=-1)
+        h = F.silu(gate) * up
+    else:
+        h = F.gelu(h)
     return dict(x1=x1, q=q, k=k, v=v, attn=o, x2=x2, hidden=h)
 
 
@@ -112,6 +142,8 @@ def make_block_inputs(name: str, batch: Optional[int] = None, **overrides) -> Bl
                                cfg["massive"])
     g1, b1 = affine_params(rng, D)
     g2, b2 = affine_params(rng, D)
+    llama = cfg.get("arch", "vit") == "llama"
+    n_fc1 = 2 * MLP if llama else MLP           # gated MLP: gate and up projections stacked
 
     def weight(n_out, n_in):
         w = rng.standard_normal(size=(n_out, n_in), dtype=np.float32)
@@ -122,10 +154,13 @@ def make_block_inputs(name: str, batch: Optional[int] = None, **overrides) -> Bl
     b_qkv = rng.normal(0.0, 0.02, size=3 * D).astype(np.float32)
     w_proj = weight(D, D)
     b_proj = rng.normal(0.0, 0.02, size=D).astype(np.float32)
-    w_fc1 = weight(MLP, D)
-    b_fc1 = rng.normal(0.0, 0.02, size=MLP).astype(np.float32)
+    w_fc1 = weight(n_fc1, D)
+    b_fc1 = rng.normal(0.0, 0.02, size=n_fc1).astype(np.float32)
     w_fc2 = weight(D, MLP)
     b_fc2 = rng.normal(0.0, 0.02, size=D).astype(np.float32)
+    if llama:                                    # RMSNorm has no shift, the linear layers no bias
+        for a in (b1, b2, b_qkv, b_proj, b_fc1, b_fc2):
+            a[...] = 0.0
 
     # calibration batch first (fixed size), then the benchmark batch: changing B never changes parameters
     n_cal = cfg["calib_samples"]
