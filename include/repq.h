@@ -63,7 +63,7 @@ typedef int repq_status;
 size_t repq_last_error(char* buf, size_t n);
 
 /* Library ABI version (bumped on any signature change). */
-int repq_abi_version(void);   /* currently 4 */
+int repq_abi_version(void);   /* currently 5 */
 
 /* ------------------------------------------------------------------------------------------------
  * One-time host-side preparation (not on the timed path)
@@ -92,6 +92,26 @@ repq_status repq_fold_ln(int D, int N, const float* gamma, const float* beta, co
  *             of 16), s_w (float[N]), z_w (int32[N]), w_row_sum (int32[N]) = sum_c codes[j, c]. */
 repq_status repq_pack_weights(int N, int K, int bits_w, const float* W, uint8_t* codes,
                               int64_t ld_codes_bytes, float* s_w, int32_t* z_w, int32_t* w_row_sum);
+
+/* Per-channel dual clipping (Sec. III-D, Eqs. 18-20): the clipping bounds of the channel-wise quantizer of a
+ * LayerNorm activation, learned on a calibration batch just before the scale reparameterization
+ * (repq_scale_zero_from_bounds -> repq_fold_ln take them from here).  For every channel d
+ *     x_up[d] = max_d sigmoid(alpha1_d),   x_low[d] = min_d sigmoid(alpha2_d)                   (Eqs. 18-19)
+ * with the factors found by `iters` Adam steps of size `lr` (Sec. IV-A: 100 steps of 0.01; decay rates 0.9 / 0.999,
+ * epsilon 1e-8) on || X'_{:,d} - X^'_{:,d} ||^2 (Eq. 20), X^' = Eq. 5 of Eq. 4 with the (s, z) of Eq. 6 on those
+ * bounds; the round operations pass the gradient straight through, the clip passes it on [0, 2^bits - 1].
+ * `alpha0` is the factors' starting value (the paper gives none; 0 starts at half of the extremes).
+ * x [device]: n x D float32 activations, row stride ldx elements.  x_low, x_up [device] float[D].
+ * loss [device] double[2 D] or NULL: the objective per channel before the first step and with the returned
+ * bounds.  Runs in float64 on `stream`, one kernel, no scratch memory; channels are independent. */
+repq_status repq_dual_clip(const float* x, int64_t n, int D, int64_t ldx, int bits, int iters, float lr,
+                           float alpha0, float* x_low, float* x_up, double* loss, void* stream);
+
+/* Rotation table of the rotary position embedding for repq_gemm_desc.rope_cos_sin.  (The paper's block,
+ * Eqs. 1-3, has no position embedding inside; the LLaMA models it evaluates in Sec. IV-A rotate Q and K.)
+ * table [host]: seq x (d_h / 2) pairs of floats, table[(m * d_h / 2 + i) * 2 + {0, 1}] = cos, sin of
+ * m * base^(-2 i / d_h), evaluated in float64 and rounded once.  d_h must be even. */
+repq_status repq_rope_table(int seq, int d_h, double base, float* table);
 
 /* ------------------------------------------------------------------------------------------------
  * Hot path, stage by stage
@@ -160,6 +180,22 @@ typedef struct repq_gemm_desc {
   int32_t* acc_debug;                   /* [device] int32 M x N (dense) raw accumulators, or NULL */
   int32_t causal;                       /* != 0: outputs with n > m + (N - M) are never read by the caller
                                            and may be left unwritten (attention scores under a causal mask) */
+  /* Two optional steps between v and the output conversion, on pairs of neighbouring output columns (plain GEMM
+   * only, not together with gelu or residual).  Neither is part of the paper's block (Eqs. 1-3); they serve the
+   * LLaMA block form of the models in Sec. IV-A, where the quantizer of Eq. 4 follows them.
+   *  - rope_cos_sin != NULL: rotary position embedding.  [device] table of repq_rope_table for rope_period
+   *    positions and heads of rope_dim channels (16-byte aligned).  Row m has position m mod rope_period; inside
+   *    the first rope_groups of the out_groups equal column ranges (out_groups delimits the ranges in every output
+   *    kind; with float outputs it has no other effect), the pair
+   *    (v[2i], v[2i+1]) of every head is rotated by the angle of (position, i):
+   *        v'[2i] = v[2i] cos - v[2i+1] sin,   v'[2i+1] = v[2i] sin + v[2i+1] cos.
+   *    rope_dim must be a multiple of 16 and divide N / out_groups.
+   *  - glu != 0: gated linear unit.  Weight rows (2i, 2i+1) are (gate_i, up_i); the output has N / 2 columns,
+   *    out[m, i] = silu(v[m, 2i]) * v[m, 2i+1], silu(x) = x / (1 + exp(-x)); ldo, out_groups and the output
+   *    quantizer refer to those N / 2 columns.  N must be even. */
+  const float* rope_cos_sin;
+  int32_t rope_period, rope_dim, rope_groups;
+  int32_t glu;
 } repq_gemm_desc;
 
 repq_status repq_qgemm_workspace_bytes(const repq_gemm_desc* d, size_t* bytes);
@@ -252,7 +288,17 @@ repq_status repq_attention(const repq_attention_desc* d, void* stream);
 /* ------------------------------------------------------------------------------------------------
  * Whole block: Eqs. 1-2,  X_bar = MSA(LN(X)) + X,  Y = MLP(LN(X_bar)) + X_bar, all GEMM inputs
  * quantized (LayerNorm -> QKV -> QK^T -> Softmax/log2 -> P.V -> proj -> LayerNorm -> fc1/GELU -> fc2).
+ *
+ * Besides the paper's own block form, the LLaMA form of the models of Sec. IV-A (which the paper evaluates
+ * but does not write down) is selected by three independent fields: norm_kind = REPQ_NORM_RMS (mean-free
+ * normalisation; its channel-wise quantizer is reparameterized by Eqs. 10-14 like LayerNorm's, so gamma_t
+ * and beta_t are both used), rope != 0 (Q and K of the projection are rotated by the table in
+ * repq_block_params.rope_cos_sin before their quantizers) and mlp_kind = REPQ_MLP_SWIGLU
+ * (Y = down(silu(gate(.)) * up(.)) + X_bar: `fc1` then holds 2*mlp weight rows, gate_i and up_i
+ * interleaved as rows 2i and 2i+1, and `fc2` is the down projection).
  * ---------------------------------------------------------------------------------------------- */
+#define REPQ_MLP_GELU 0
+#define REPQ_MLP_SWIGLU 1
 typedef struct repq_linear_params {
   const uint8_t* w_codes;               /* [device] packed by repq_pack_weights */
   int64_t ldw_bytes;
@@ -273,6 +319,8 @@ typedef struct repq_block_desc {
   int32_t out_dtype;                    /* dtype of y */
   int32_t staged_attention;             /* 0: fused attention kernel (repq_attention); != 0: the three separate
                                            stages (scores -> Softmax codes -> P.V) through the workspace */
+  int32_t rope;                         /* != 0: rotary position embedding on Q and K (position = token index) */
+  int32_t mlp_kind;                     /* REPQ_MLP_GELU (the paper's block) or REPQ_MLP_SWIGLU */
 } repq_block_desc;
 
 typedef struct repq_block_params {
@@ -291,10 +339,11 @@ typedef struct repq_block_params {
   const float* ln2_beta_t;
   float ln2_s;
   int32_t ln2_z;
-  repq_linear_params fc1;               /* N = mlp, K = dim, weights W~ */
+  repq_linear_params fc1;               /* N = mlp (REPQ_MLP_SWIGLU: 2*mlp, gate / up interleaved), K = dim, weights W~ */
   float s_hidden;
   int32_t z_hidden;                     /* quantizer of the GELU output (input of fc2) */
   repq_linear_params fc2;               /* N = dim, K = mlp */
+  const float* rope_cos_sin;            /* [device] repq_rope_table(seq, dim / heads, base), or NULL if !rope */
 } repq_block_params;
 
 repq_status repq_block_workspace_bytes(const repq_block_desc* d, size_t* bytes);
@@ -328,8 +377,8 @@ repq_status repq_block_forward_timed(const repq_block_desc* d, const repq_block_
  *    (repq_block_workspace_bytes tells; a ViT-S-sized block of a few hundred tokens fits).  Larger
  *    blocks are rejected with REPQ_WORKSPACE_TOO_SMALL and a message naming both sizes.
  *  - First call on a device: the library looks up the device address of its scratch array once per
- *    device (with that device current) and remembers it.  Make that first call outside any stream
- *    capture.
+ *    device (with that device current) and remembers it (threads that race on that first call both
+ *    look it up and store the same address).  Make that first call outside any stream capture.
  *  - The scratch is shared by every call in the process and keeps whatever the previous call left in
  *    it; the entry point itself clears the parts that have to start at zero.  Two calls that overlap
  *    in time on the same GPU (different streams or threads) race on it: serialise them.
@@ -370,8 +419,17 @@ uint64_t repq_launch_count(void);
 
 /* Device-side health word of the calling thread's current device: 0 = healthy; non-zero = a bounded
  * wait inside a kernel gave up (the kernel drained and returned; results of that launch are
- * invalid).  Synchronises the device.  `reset` != 0 clears it. */
+ * invalid).  Synchronises the device and writes the word to *status; returns REPQ_OK if it is 0 and
+ * REPQ_TIMEOUT otherwise.  `reset` != 0 clears it. */
 repq_status repq_device_status(int32_t* status, int reset);
+
+/* Self-test of the failure path of the bounded device-side waits.  (Every mbarrier wait of the
+ * tensor-core kernels gives up after about a second, records a code in the health word and lets the kernel
+ * drain and return instead of hanging; the paper has no counterpart.)  Launches, on `stream`, a one-thread
+ * kernel whose barrier is never completed and whose wait uses the same routine with a limit of
+ * limit_cycles SM clock cycles (1 .. 2e9): the kernel returns after that long, repq_device_status then
+ * reports REPQ_TIMEOUT with code 77 until it is reset, and the context stays usable. */
+repq_status repq_bounded_wait_selftest(int64_t limit_cycles, void* stream);
 
 #ifdef __cplusplus
 }

@@ -222,6 +222,84 @@ def dequant_log2_reparam(q, s):
 
 
 # --------------------------------------------------------------------------------------
+# Sec. III-D  Per-channel dual clipping (Eqs. 18-20)
+# --------------------------------------------------------------------------------------
+
+def dual_clip_bounds(x_max, x_min, alpha1, alpha2):
+    """Eqs. 18-19: X'_up = max_d * Sigmoid(alpha1), X'_low = min_d * Sigmoid(alpha2), per channel."""
+    sig = lambda a: 1.0 / (1.0 + np.exp(-np.asarray(a, dtype=F64)))
+    return np.asarray(x_max, dtype=F64) * sig(alpha1), np.asarray(x_min, dtype=F64) * sig(alpha2)
+
+
+def dual_clip_loss_grad(X, alpha1, alpha2, bits: int):
+    """Objective of Eq. 20 per channel, ||X'_{:,d} - X^'_{:,d}||^2 with the channel-wise quantizer of Eqs. 4-6 built
+    on the bounds of Eqs. 18-19, and its gradient with respect to (alpha1, alpha2).
+
+    The round operations (of x/s in Eq. 4 and of -x_low/s in Eq. 6) are passed straight through in the backward
+    direction (derivative 1), the clip passes the gradient on [0, 2^b - 1] inclusive and blocks it outside; the
+    paper learns the factors by gradient descent (Sec. IV-A) without printing these conventions, which are the
+    usual ones for learned quantizer bounds.  With u = x/s, zc = -x_low/s, r = round(u), z = round(zc),
+    q = clip(r + z, 0, Q), Q = 2^b - 1 and x^ = s (q - z):
+        inside the clip   dx^/ds = r - u            dx^/dx_low (s fixed) = 0
+        clipped           dx^/ds = q - z + zc       dx^/dx_low (s fixed) = 1
+    and s = (x_up - x_low) / Q, x_up = max * sig(alpha1), x_low = min * sig(alpha2).
+    Returns (loss[D], dloss/dalpha1[D], dloss/dalpha2[D])."""
+    X = np.asarray(X, dtype=F64)
+    Q = F64(2 ** bits - 1)
+    x_max, x_min = X.max(axis=0), X.min(axis=0)
+    sg1 = 1.0 / (1.0 + np.exp(-np.asarray(alpha1, dtype=F64)))
+    sg2 = 1.0 / (1.0 + np.exp(-np.asarray(alpha2, dtype=F64)))
+    up, low = x_max * sg1, x_min * sg2
+    s = (up - low) / Q
+    u = X / s
+    zc = -low / s
+    r, z = np.rint(u), np.rint(zc)
+    pre = r + z
+    q = np.clip(pre, 0.0, Q)
+    x_hat = s * (q - z)
+    inside = (pre >= 0.0) & (pre <= Q)
+    g = 2.0 * (x_hat - X)                                   # dL/dx^
+    dxh_ds = np.where(inside, r - u, q - z + zc)
+    dxh_dlow = np.where(inside, 0.0, 1.0)
+    dL_ds = (g * dxh_ds).sum(axis=0)
+    dL_dlow_direct = (g * dxh_dlow).sum(axis=0)
+    dL_dup = dL_ds / Q
+    dL_dlow = dL_dlow_direct - dL_ds / Q
+    loss = ((x_hat - X) ** 2).sum(axis=0)
+    return loss, dL_dup * x_max * sg1 * (1.0 - sg1), dL_dlow * x_min * sg2 * (1.0 - sg2)
+
+
+def dual_clip(X, bits: int, iters: int = 100, lr: float = 0.01, alpha0: float = 0.0,
+              beta1: float = 0.9, beta2: float = 0.999, adam_eps: float = 1e-8):
+    """Per-channel dual clipping (Sec. III-D): Adam (Sec. IV-A: 100 iterations, learning rate 0.01; the moment
+    decay rates and epsilon are the optimizer's customary defaults, which the paper does not restate) on the
+    clipping factors of every channel of the LayerNorm activations X [tokens, D], objective of Eq. 20.
+    `alpha0` is the factors' initial value, which the paper does not give (0: the bounds start at half of each
+    channel's extremes; 2: at 0.88 of them, from where 100 steps of 0.01 reach contractions of 0.73 to 0.95).  Returns dict(x_low, x_up, alpha1, alpha2, loss0, loss) with loss0 / loss the per-channel
+    objective before the first and after the last update."""
+    X = np.asarray(X, dtype=F64)
+    D = X.shape[1]
+    a1 = np.full(D, alpha0, dtype=F64)
+    a2 = np.full(D, alpha0, dtype=F64)
+    m1, v1, m2, v2 = (np.zeros(D, dtype=F64) for _ in range(4))
+    loss0 = None
+    for t in range(1, iters + 1):
+        loss, g1, g2 = dual_clip_loss_grad(X, a1, a2, bits)
+        if loss0 is None:
+            loss0 = loss
+        m1 = beta1 * m1 + (1.0 - beta1) * g1
+        v1 = beta2 * v1 + (1.0 - beta2) * g1 * g1
+        m2 = beta1 * m2 + (1.0 - beta1) * g2
+        v2 = beta2 * v2 + (1.0 - beta2) * g2 * g2
+        c1, c2 = 1.0 - beta1 ** t, 1.0 - beta2 ** t
+        a1 = a1 - lr * (m1 / c1) / (np.sqrt(v1 / c2) + adam_eps)
+        a2 = a2 - lr * (m2 / c1) / (np.sqrt(v2 / c2) + adam_eps)
+    loss, _, _ = dual_clip_loss_grad(X, a1, a2, bits)
+    up, low = dual_clip_bounds(X.max(axis=0), X.min(axis=0), a1, a2)
+    return dict(x_low=low, x_up=up, alpha1=a1, alpha2=a2, loss0=loss if loss0 is None else loss0, loss=loss)
+
+
+# --------------------------------------------------------------------------------------
 # Sec. III-A.1  Transformer block (Eqs. 1-3)
 # --------------------------------------------------------------------------------------
 

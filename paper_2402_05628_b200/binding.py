@@ -28,8 +28,10 @@ EXPORTS = (
     "repq_pack_weights", "repq_ln_quant", "repq_qgemm_workspace_bytes", "repq_qgemm",
     "repq_softmax_log2", "repq_pv", "repq_block_workspace_bytes", "repq_block_forward",
     "repq_device_status", "repq_block_forward_timed", "repq_launch_count",
-    "repq_block_forward_static", "repq_attention", "repq_block_forward_host",
+    "repq_block_forward_static", "repq_attention", "repq_block_forward_host", "repq_rope_table",
+    "repq_bounded_wait_selftest", "repq_dual_clip",
 )
+REPQ_MLP_GELU, REPQ_MLP_SWIGLU = 0, 1
 REPQ_STATIC_WORKSPACE_BYTES = 8 << 20
 REPQ_BLOCK_STAGES = 9
 BLOCK_STAGE_NAMES = ("ln1", "qkv", "scores", "softmax", "pv", "proj", "ln2", "fc1", "fc2")
@@ -58,6 +60,8 @@ class GemmDesc(C.Structure):
         ("out_scale", C.c_float * REPQ_MAX_OUT_GROUPS), ("out_zero", C.c_int32 * REPQ_MAX_OUT_GROUPS),
         ("out", C.c_void_p), ("ldo", C.c_int64), ("o_stride_outer", C.c_int64), ("o_stride_inner", C.c_int64),
         ("out_row_sum", C.c_void_p), ("acc_debug", C.c_void_p), ("causal", C.c_int32),
+        ("rope_cos_sin", C.c_void_p), ("rope_period", C.c_int32), ("rope_dim", C.c_int32), ("rope_groups", C.c_int32),
+        ("glu", C.c_int32),
     ]
 
 
@@ -84,7 +88,8 @@ class BlockDesc(C.Structure):
     _fields_ = [("batch", C.c_int32), ("seq", C.c_int32), ("dim", C.c_int32), ("heads", C.c_int32),
                 ("mlp", C.c_int32), ("bits_a", C.c_int32), ("bits_w", C.c_int32), ("bits_p", C.c_int32),
                 ("causal", C.c_int32), ("norm_kind", C.c_int32), ("eps", C.c_float),
-                ("act_dtype", C.c_int32), ("out_dtype", C.c_int32), ("staged_attention", C.c_int32)]
+                ("act_dtype", C.c_int32), ("out_dtype", C.c_int32), ("staged_attention", C.c_int32),
+                ("rope", C.c_int32), ("mlp_kind", C.c_int32)]
 
 
 class AttentionDesc(C.Structure):
@@ -115,6 +120,7 @@ class BlockParams(C.Structure):
         ("ln2_gamma_t", C.c_void_p), ("ln2_beta_t", C.c_void_p), ("ln2_s", C.c_float), ("ln2_z", C.c_int32),
         ("fc1", LinearParams), ("s_hidden", C.c_float), ("z_hidden", C.c_int32),
         ("fc2", LinearParams),
+        ("rope_cos_sin", C.c_void_p),
     ]
 
 
@@ -156,6 +162,10 @@ def lib() -> C.CDLL:
         _lib.repq_fold_ln.argtypes = [C.c_int, C.c_int] + [C.c_void_p] * 12
         _lib.repq_pack_weights.argtypes = [C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_int64,
                                            C.c_void_p, C.c_void_p, C.c_void_p]
+        _lib.repq_rope_table.argtypes = [C.c_int, C.c_int, C.c_double, C.c_void_p]
+        _lib.repq_dual_clip.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_int64, C.c_int, C.c_int, C.c_float, C.c_float,
+                                        C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        _lib.repq_bounded_wait_selftest.argtypes = [C.c_int64, C.c_void_p]
     return _lib
 
 
@@ -334,9 +344,32 @@ def repq_launch_count() -> int:
 
 
 def repq_device_status(reset: bool = False) -> int:
+    """The device's health word (0 = healthy).  REPQ_TIMEOUT from the library is the non-zero word, not an error
+    of this call."""
     v = C.c_int32()
-    _check(lib().repq_device_status(C.byref(v), int(reset)))
+    st = lib().repq_device_status(C.byref(v), int(reset))
+    if st != REPQ_TIMEOUT:
+        _check(st)
     return int(v.value)
+
+
+def repq_bounded_wait_selftest(limit_cycles: int, stream=None) -> None:
+    _check(lib().repq_bounded_wait_selftest(int(limit_cycles), _stream(stream)))
+
+
+def repq_dual_clip(x: torch.Tensor, bits: int, x_low: torch.Tensor, x_up: torch.Tensor, loss: Optional[torch.Tensor] = None,
+                   iters: int = 100, lr: float = 0.01, alpha0: float = 0.0, stream=None) -> None:
+    """Per-channel dual clipping on device activations x [n, D] float32: learned bounds into x_low / x_up [D]."""
+    n, D = x.shape
+    _check(lib().repq_dual_clip(_ptr(x), n, D, x.stride(0), bits, iters, lr, alpha0, _ptr(x_low), _ptr(x_up), _ptr(loss),
+                                _stream(stream)))
+
+
+def repq_rope_table(seq: int, d_h: int, base: float = 10000.0) -> np.ndarray:
+    """(cos, sin) table of the rotary embedding, float32 [seq, d_h / 2, 2]."""
+    t = np.empty((seq, d_h // 2, 2), dtype=np.float32)
+    _check(lib().repq_rope_table(seq, d_h, float(base), _ptr(t)))
+    return t
 
 
 # ---------------------------------------------------------------------------------- descriptor helpers
@@ -346,7 +379,8 @@ def gemm_desc(M: int, N: int, K: int, a_codes: torch.Tensor, bits_a: int, s_a: f
               z_w_scalar=0, a_row_sum=None, w_row_sum=None, bias=None, alpha=1.0, gelu=False, residual=None,
               out_kind=REPQ_OUT_F32, out_bits=8, out_scale: Sequence[float] = (1.0,), out_zero: Sequence[int] = (0,),
               out_row_sum=None, acc_debug=None, batch=(1, 1), a_strides=(0, 0), w_strides=(0, 0), o_strides=(0, 0),
-              lda_bytes=None, ldw_bytes=None, ldo=None, causal=False) -> GemmDesc:
+              lda_bytes=None, ldw_bytes=None, ldo=None, causal=False, rope=None, rope_period=0, rope_dim=0,
+              rope_groups=0, glu=False) -> GemmDesc:
     """Fills a GemmDesc from torch tensors (pointer and stride marshalling only)."""
     d = GemmDesc()
     d.M, d.N, d.K = M, N, K
@@ -372,4 +406,6 @@ def gemm_desc(M: int, N: int, K: int, a_codes: torch.Tensor, bits_a: int, s_a: f
     d.o_stride_outer, d.o_stride_inner = o_strides
     d.out_row_sum, d.acc_debug = _ptr(out_row_sum), _ptr(acc_debug)
     d.causal = int(causal)
+    d.rope_cos_sin, d.rope_period, d.rope_dim, d.rope_groups = _ptr(rope), rope_period, rope_dim, rope_groups
+    d.glu = int(glu)
     return d

@@ -1,6 +1,7 @@
 // repq_block_forward: one quantized transformer block (Eqs. 1-3) as a stream-ordered sequence of the
 // stage kernels.  No host synchronisation, no allocation: every intermediate lives in the caller's
 // workspace.
+#include <atomic>
 #include <cmath>
 
 #include "kernels.h"
@@ -32,6 +33,9 @@ repq_status validate(const repq_block_desc& d) {
                REPQ_INVALID_ARG, "block: dtypes must be REPQ_F32 or REPQ_BF16");
   REPQ_REQUIRE(d.norm_kind == REPQ_NORM_LAYERNORM || d.norm_kind == REPQ_NORM_RMS, REPQ_INVALID_ARG, "block: unknown norm_kind");
   REPQ_REQUIRE(int64_t(d.batch) * d.heads <= 65535, REPQ_UNSUPPORTED, "block: batch * heads exceeds 65535");
+  REPQ_REQUIRE(int64_t(d.batch) * d.seq <= 2147483647LL, REPQ_UNSUPPORTED, "block: batch * seq exceeds 2^31 - 1");
+  REPQ_REQUIRE(d.mlp_kind == REPQ_MLP_GELU || d.mlp_kind == REPQ_MLP_SWIGLU, REPQ_INVALID_ARG, "block: unknown mlp_kind");
+  REPQ_REQUIRE(!d.rope || dh % 16 == 0, REPQ_UNSUPPORTED, "block: rope needs a head dim that is a multiple of 16");
   return REPQ_OK;
 }
 
@@ -64,8 +68,9 @@ BlockLayout layout(const repq_block_desc& d) {
   L.off_ln = bump(cur, size_t(L.M * L.ld_a));
   L.off_asum = bump(cur, size_t(L.M) * 4);
   L.off_qkv = bump(cur, size_t(L.M * L.ld_qkv));
-  L.off_scores = bump(cur, size_t(rows_s * L.ld_s) * 4);
-  L.off_p = bump(cur, size_t(rows_s * L.ld_p));
+  // float32 scores and Softmax codes exist only when the three attention stages run as separate kernels
+  L.off_scores = bump(cur, d.staged_attention ? size_t(rows_s * L.ld_s) * 4 : 0);
+  L.off_p = bump(cur, d.staged_attention ? size_t(rows_s * L.ld_p) : 0);
   L.off_attn = bump(cur, size_t(L.M * L.ld_a));
   L.off_asum_attn = bump(cur, size_t(L.M) * 4);
   L.off_xbar = bump(cur, size_t(L.M) * d.dim * act);
@@ -74,7 +79,8 @@ BlockLayout layout(const repq_block_desc& d) {
   // scratch of the largest GEMM of the block
   repq_linear_params none{};
   size_t ws = 0;
-  const int shapes[4][2] = {{3 * d.dim, d.dim}, {d.dim, d.dim}, {d.mlp, d.dim}, {d.dim, d.mlp}};
+  const int n_fc1 = d.mlp_kind == REPQ_MLP_SWIGLU ? 2 * d.mlp : d.mlp;
+  const int shapes[4][2] = {{3 * d.dim, d.dim}, {d.dim, d.dim}, {n_fc1, d.dim}, {d.dim, d.mlp}};
   for (auto& s : shapes) {
     repq_gemm_desc g = linear_desc(d, L.M, s[0], s[1], nullptr, code_row_bytes(s[1], act_bits(d)), 1.f, 0, nullptr, none);
     g.ldw_bytes = round_up(code_row_bytes(s[1], d.bits_w), 16);
@@ -106,6 +112,7 @@ static repq_status block_forward_impl(const repq_block_desc* dp, const repq_bloc
   const repq_block_desc& d = *dp;
   const repq_block_params& p = *pp;
   REPQ_TRY(validate(d));
+  REPQ_REQUIRE(!d.rope || p.rope_cos_sin != nullptr, REPQ_INVALID_ARG, "block_forward: rope is set but rope_cos_sin is NULL");
   const BlockLayout L = layout(d);
   REPQ_REQUIRE(workspace && workspace_bytes >= L.total, REPQ_WORKSPACE_TOO_SMALL,
                "block_forward: workspace of %zu bytes given, %zu needed", workspace_bytes, L.total);
@@ -149,6 +156,9 @@ static repq_status block_forward_impl(const repq_block_desc* dp, const repq_bloc
     g.out_scale[0] = p.s_q; g.out_scale[1] = p.s_k; g.out_scale[2] = p.s_v;
     g.out_zero[0] = p.z_q; g.out_zero[1] = p.z_k; g.out_zero[2] = p.z_v;
     g.out = qkv_c; g.ldo = L.ld_qkv;
+    if (d.rope) {                       // Q and K ranges rotated ahead of their quantizers, V left alone
+      g.rope_cos_sin = p.rope_cos_sin; g.rope_period = S; g.rope_dim = dh; g.rope_groups = 2;
+    }
     REPQ_TRY(repq_qgemm(&g, gws, L.gemm_ws, stream));
   }
   REPQ_MARK();
@@ -221,8 +231,10 @@ static repq_status block_forward_impl(const repq_block_desc* dp, const repq_bloc
                          ab, ln_c, L.ld_a, asum, stream));
   REPQ_MARK();
   {
-    repq_gemm_desc g = linear_desc(d, M, d.mlp, D, ln_c, L.ld_a, p.ln2_s, p.ln2_z, asum, p.fc1);
-    g.gelu = 1;
+    const bool swiglu = d.mlp_kind == REPQ_MLP_SWIGLU;
+    repq_gemm_desc g = linear_desc(d, M, swiglu ? 2 * d.mlp : d.mlp, D, ln_c, L.ld_a, p.ln2_s, p.ln2_z, asum, p.fc1);
+    g.gelu = !swiglu;
+    g.glu = swiglu;                     // weight rows (2i, 2i+1) = (gate_i, up_i): d.mlp codes per row leave
     g.out_kind = REPQ_OUT_CODES; g.out_bits = ab; g.out_groups = 1;
     g.out_scale[0] = p.s_hidden; g.out_zero[0] = p.z_hidden;
     g.out = hid_c; g.ldo = L.ld_h; g.out_row_sum = asum_h;
@@ -274,19 +286,20 @@ static __device__ __align__(256) unsigned char g_static_ws[REPQ_STATIC_WORKSPACE
 
 namespace {
 constexpr int kMaxDevices = 64;
-void* g_static_ws_addr[kMaxDevices] = {nullptr};
+// one slot per device; concurrent first calls may both look the address up, and store the same value
+std::atomic<void*> g_static_ws_addr[kMaxDevices];
 
 repq_status static_workspace(void** out) {
   int dev = -1;
   REPQ_CUDA(cudaGetDevice(&dev));
   REPQ_REQUIRE(dev >= 0 && dev < kMaxDevices, REPQ_UNSUPPORTED, "block_forward_static: device index %d not supported", dev);
-  if (g_static_ws_addr[dev] == nullptr) {
-    void* ptr = nullptr;
+  void* ptr = g_static_ws_addr[dev].load(std::memory_order_acquire);
+  if (ptr == nullptr) {
     REPQ_CUDA(cudaGetSymbolAddress(&ptr, g_static_ws));
     REPQ_REQUIRE(ptr != nullptr, REPQ_CUDA_ERROR, "block_forward_static: scratch array has no device address");
-    g_static_ws_addr[dev] = ptr;
+    g_static_ws_addr[dev].store(ptr, std::memory_order_release);
   }
-  *out = g_static_ws_addr[dev];
+  *out = ptr;
   return REPQ_OK;
 }
 }  // namespace
@@ -307,6 +320,12 @@ extern "C" repq_status repq_block_forward_static(const repq_block_desc* d, const
   return block_forward_impl(d, p, x, y, ws, size_t(REPQ_STATIC_WORKSPACE_BYTES), stream, nullptr);
 }
 
+extern "C" repq_status repq_bounded_wait_selftest(int64_t limit_cycles, void* stream) {
+  REPQ_REQUIRE(limit_cycles > 0 && limit_cycles <= 2000000000LL, REPQ_INVALID_ARG,
+               "bounded_wait_selftest: limit must be between 1 and 2e9 cycles");
+  return launch_wait_selftest(limit_cycles, static_cast<cudaStream_t>(stream));
+}
+
 extern "C" repq_status repq_device_status(int32_t* status, int reset) {
   REPQ_REQUIRE(status, REPQ_INVALID_ARG, "device_status: NULL argument");
   int32_t* word = device_status_word();
@@ -317,5 +336,6 @@ extern "C" repq_status repq_device_status(int32_t* status, int reset) {
   REPQ_CUDA(cudaDeviceSynchronize());
   REPQ_CUDA(cudaMemcpy(status, word, sizeof(int32_t), cudaMemcpyDeviceToHost));
   if (reset) REPQ_CUDA(cudaMemset(word, 0, sizeof(int32_t)));
+  REPQ_REQUIRE(*status == 0, REPQ_TIMEOUT, "a bounded device-side wait ran out (code %d): results of that launch are invalid", int(*status));
   return REPQ_OK;
 }

@@ -33,6 +33,12 @@ struct EpilogueParams {
   int64_t ldo;
   int32_t* out_row_sum;    // or nullptr
   int32_t* acc_debug;      // or nullptr, dense M x N
+  // steps on pairs of neighbouring columns (LLaMA block form), applied to v before the output conversion
+  const float2* rope;      // (cos, sin) table [rope_period][rope_dim / 2], or nullptr
+  int32_t rope_period;
+  int32_t rope_dim;
+  int32_t rope_cols;       // columns below this bound are rotated
+  int32_t glu;             // columns (2i, 2i+1) = (gate, up): output column i = silu(gate) * up
 };
 
 // Per-column constants of the epilogue, gathered once per output column.
@@ -94,6 +100,17 @@ __device__ __forceinline__ float epilogue_value(const EpilogueParams& p, const C
   }
   return v;
 }
+
+// Rotary position embedding of one pair: (a, b) at column pair index `pair` of its head, row position `pos`.
+__device__ __forceinline__ void rope_rotate(const float2 cs, float& a, float& b) {
+  const float ra = fmaf(a, cs.x, -(b * cs.y));
+  const float rb = fmaf(a, cs.y, b * cs.x);
+  a = ra;
+  b = rb;
+}
+
+// silu(g) * u, silu(x) = x / (1 + exp(-x)); exp(-x) = +inf for very negative x gives -0 * u.
+__device__ __forceinline__ float silu_mul(float g, float u) { return __fdividef(g, 1.f + __expf(-g)) * u; }
 
 // Eq. 4 with the output quantizer: clip(round(v / s_o) + z_o, 0, qmax).
 __device__ __forceinline__ int32_t requantize(const ColumnTerms& c, float v) {

@@ -50,7 +50,21 @@ extern "C" size_t repq_last_error(char* buf, size_t n) {
   return m.size();
 }
 
-extern "C" int repq_abi_version(void) { return 4; }
+extern "C" int repq_abi_version(void) { return 5; }
+
+extern "C" repq_status repq_rope_table(int seq, int d_h, double base, float* table) {
+  REPQ_REQUIRE(seq > 0 && d_h > 0 && d_h % 2 == 0 && base > 0.0 && table, REPQ_INVALID_ARG, "rope_table: bad argument");
+  const int half = d_h / 2;
+  for (int i = 0; i < half; ++i) {
+    const double theta = std::pow(base, -2.0 * double(i) / double(d_h));
+    for (int m = 0; m < seq; ++m) {
+      const double ang = double(m) * theta;
+      table[(size_t(m) * half + i) * 2 + 0] = float(std::cos(ang));
+      table[(size_t(m) * half + i) * 2 + 1] = float(std::sin(ang));
+    }
+  }
+  return REPQ_OK;
+}
 
 extern "C" repq_status repq_scale_zero_from_bounds(int n, const float* x_low, const float* x_up,
                                                    int bits, float* s, int32_t* z) {

@@ -46,6 +46,9 @@ struct PvParams {
 bool pv_tc_supported(const repq_pv_desc& d);
 repq_status launch_pv_tc(const repq_pv_desc& d, const PvParams& P, cudaStream_t st);
 
+// One-thread kernel whose mbarrier wait can only run out (see repq_bounded_wait_selftest).
+repq_status launch_wait_selftest(long long limit_cycles, cudaStream_t st);
+
 // Device-side health word (bounded waits report here instead of trapping); nullptr on failure.
 int32_t* device_status_word();
 

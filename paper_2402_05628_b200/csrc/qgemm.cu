@@ -90,6 +90,12 @@ repq_status validate(const repq_gemm_desc& d) {
   if (batched)
     REPQ_REQUIRE(!d.residual && !d.acc_debug && !d.out_row_sum && !d.a_row_sum && !d.w_row_sum, REPQ_UNSUPPORTED,
                  "qgemm: residual / row sums / acc_debug are for plain (unbatched) products");
+  const int n_out = d.glu ? d.N / 2 : d.N;        // output columns
+  if (d.glu) {
+    REPQ_REQUIRE(d.out_groups <= 1, REPQ_UNSUPPORTED, "qgemm: glu takes one output group");
+    REPQ_REQUIRE(!(d.out_kind == REPQ_OUT_CODES && packed4(d.out_bits)), REPQ_UNSUPPORTED,
+                 "qgemm: glu writes float outputs or codes stored one per byte");
+  }
   if (d.out_kind == REPQ_OUT_CODES) {
     REPQ_REQUIRE(bits_ok(d.out_bits), REPQ_INVALID_ARG, "qgemm: out_bits must be 4, 6 or 8");
     REPQ_REQUIRE(d.out_groups >= 1 && d.out_groups <= REPQ_MAX_OUT_GROUPS && d.N % d.out_groups == 0,
@@ -98,16 +104,30 @@ repq_status validate(const repq_gemm_desc& d) {
       REPQ_REQUIRE(d.out_scale[g] > 0.f, REPQ_INVALID_ARG, "qgemm: out_scale[%d] must be positive", g);
       REPQ_REQUIRE(d.out_zero[g] > -(1 << 20) && d.out_zero[g] < (1 << 20), REPQ_INVALID_ARG, "qgemm: |out_zero| must be below 2^20");
     }
-    REPQ_REQUIRE(d.ldo >= code_row_bytes(d.N, d.out_bits), REPQ_INVALID_ARG, "qgemm: ldo shorter than a row of codes");
-    if (packed4(d.out_bits)) REPQ_REQUIRE((d.N / d.out_groups) % 2 == 0, REPQ_UNSUPPORTED, "qgemm: 4-bit output groups must have even width");
+    REPQ_REQUIRE(d.ldo >= code_row_bytes(n_out, d.out_bits), REPQ_INVALID_ARG, "qgemm: ldo shorter than a row of codes");
+    if (packed4(d.out_bits)) REPQ_REQUIRE((n_out / d.out_groups) % 2 == 0, REPQ_UNSUPPORTED, "qgemm: 4-bit output groups must have even width");
   } else {
-    REPQ_REQUIRE(d.ldo >= d.N, REPQ_INVALID_ARG, "qgemm: ldo < N");
+    REPQ_REQUIRE(d.ldo >= n_out, REPQ_INVALID_ARG, "qgemm: ldo < output columns");
     const size_t esz = d.out_kind == REPQ_OUT_F32 ? 4 : 2;
     REPQ_REQUIRE(aligned(d.out, esz), REPQ_ALIGNMENT, "qgemm: out is not element-aligned");
   }
   if (d.residual) {
     REPQ_REQUIRE(d.residual_dtype == REPQ_F32 || d.residual_dtype == REPQ_BF16, REPQ_INVALID_ARG, "qgemm: residual_dtype");
     REPQ_REQUIRE(d.ld_residual >= d.N, REPQ_INVALID_ARG, "qgemm: ld_residual < N");
+  }
+  if (d.rope_cos_sin || d.glu) {
+    REPQ_REQUIRE(!batched && !d.gelu && !d.residual, REPQ_UNSUPPORTED,
+                 "qgemm: rope / glu are for plain products without gelu or residual");
+    REPQ_REQUIRE(!(d.rope_cos_sin && d.glu), REPQ_UNSUPPORTED, "qgemm: rope and glu exclude each other");
+    REPQ_REQUIRE(d.N % 2 == 0, REPQ_INVALID_ARG, "qgemm: rope / glu need an even N");
+  }
+  if (d.rope_cos_sin) {
+    const int groups = d.out_groups >= 1 ? d.out_groups : 1;
+    REPQ_REQUIRE(groups <= REPQ_MAX_OUT_GROUPS && d.N % groups == 0, REPQ_INVALID_ARG, "qgemm: out_groups must be 1..4 and divide N");
+    REPQ_REQUIRE(d.rope_period > 0 && d.rope_dim > 0 && d.rope_dim % 16 == 0 && (d.N / groups) % d.rope_dim == 0,
+                 REPQ_INVALID_ARG, "qgemm: rope_dim must be a multiple of 16 that divides N / out_groups, rope_period positive");
+    REPQ_REQUIRE(d.rope_groups >= 1 && d.rope_groups <= groups, REPQ_INVALID_ARG, "qgemm: rope_groups must be 1..out_groups");
+    REPQ_REQUIRE(aligned(d.rope_cos_sin, 16), REPQ_ALIGNMENT, "qgemm: rope_cos_sin must be 16-byte aligned");
   }
   return REPQ_OK;
 }
@@ -133,6 +153,11 @@ EpilogueParams make_epilogue(const repq_gemm_desc& d) {
   ep.out = d.out; ep.ldo = d.ldo;
   ep.out_row_sum = codes ? d.out_row_sum : nullptr;
   ep.acc_debug = d.acc_debug;
+  ep.rope = reinterpret_cast<const float2*>(d.rope_cos_sin);
+  ep.rope_period = d.rope_period;
+  ep.rope_dim = d.rope_dim;
+  ep.rope_cols = d.rope_cos_sin ? d.rope_groups * (d.N / (d.out_groups >= 1 ? d.out_groups : 1)) : 0;
+  ep.glu = d.glu;
   return ep;
 }
 

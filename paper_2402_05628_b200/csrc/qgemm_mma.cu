@@ -159,19 +159,43 @@ qgemm_mma_kernel(MmaOperand A, MmaOperand W, int K, int batch_inner, int64_t a_s
         const int col = n0 + cl;
         int q[2] = {0, 0};
         float v[2] = {0.f, 0.f};
+        ColumnTerms ct[2];
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
           const int jcol = col + e;
           if (row_ok && jcol < ep.N) {
-            const ColumnTerms ct = column_terms(ep, jcol, s_wsum[cl + e]);
+            ct[e] = column_terms(ep, jcol, s_wsum[cl + e]);
             const int a = acc[i][j][2 * h + e];
             if (ep.acc_debug) ep.acc_debug[m * ep.N + jcol] = a;
-            v[e] = epilogue_value(ep, ct, a, asum_m, m, jcol);
-            if (ep.out_kind == REPQ_OUT_CODES) {
-              q[e] = requantize(ct, v[e]);
-              code_sum += q[e];
+            v[e] = epilogue_value(ep, ct[e], a, asum_m, m, jcol);
+          }
+        }
+        // steps on the column pair (col is even, N is even when they are on)
+        if (ep.rope != nullptr && row_ok && col < ep.rope_cols)
+          rope_rotate(ep.rope[int64_t(m % ep.rope_period) * (ep.rope_dim >> 1) + ((col % ep.rope_dim) >> 1)], v[0], v[1]);
+        if (ep.glu) {
+          if (row_ok && col < ep.N) {
+            const float hv = silu_mul(v[0], v[1]);
+            const int oc = col >> 1;
+            if (ep.out_kind == REPQ_OUT_F32) {
+              static_cast<float*>(ep.out)[m * ep.ldo + oc] = hv;
+            } else if (ep.out_kind == REPQ_OUT_BF16) {
+              static_cast<__nv_bfloat16*>(ep.out)[m * ep.ldo + oc] = __float2bfloat16_rn(hv);
+            } else {
+              const int code = requantize(column_terms(ep, 0, 0), hv);     // one output group: its quantizer
+              code_sum += code;
+              static_cast<uint8_t*>(ep.out)[m * ep.ldo + oc] = uint8_t(code);
             }
           }
+          continue;
+        }
+        if (ep.out_kind == REPQ_OUT_CODES) {
+#pragma unroll
+          for (int e = 0; e < 2; ++e)
+            if (row_ok && col + e < ep.N) {
+              q[e] = requantize(ct[e], v[e]);
+              code_sum += q[e];
+            }
         }
         if (row_ok && col < ep.N) {
           const bool two = col + 1 < ep.N;

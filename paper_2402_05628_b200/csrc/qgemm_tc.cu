@@ -261,39 +261,69 @@ __device__ __noinline__ void slow_chunk(const EpilogueParams& ep, const TcParams
                                         int cl, int64_t m, int col0, int32_t asum_c, int* code_sum) {
   const ChunkQuant q = chunk_quant(ep, P, col0);
   const float magic = __uint_as_float(kMagicBits);
-  uint32_t prev_code = 0;
-  for (int e = 0; e < kChunk; ++e) {
+  auto code_of = [&](float v) {
+    const float t = fminf(fmaxf(v * q.mult, q.lo), q.hi);
+    return (__float_as_uint(t + magic) - kMagicBits) + uint32_t(q.zo);
+  };
+  for (int e = 0; e < kChunk; e += 2) {                // column pairs (the chunk starts at an even column)
     const int j = col0 + e;
     if (j >= P.N) break;
-    if (ep.acc_debug) ep.acc_debug[m * P.N + j] = int32_t(r[e]);
-    float v = fmaf(C.sc[cl + e], float(int32_t(r[e]) + C.nzw[cl + e] * asum_c + C.kw[cl + e]), C.bi[cl + e]);
-    if (ep.gelu) v = gelu_erf(v);
-    if (ep.residual) {
-      const int64_t off = m * ep.ld_residual + j;
-      v += ep.residual_bf16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(ep.residual)[off])
-                            : static_cast<const float*>(ep.residual)[off];
+    const bool two = j + 1 < P.N;
+    float v[2] = {0.f, 0.f};
+    for (int h = 0; h < (two ? 2 : 1); ++h) {
+      if (ep.acc_debug) ep.acc_debug[m * P.N + j + h] = int32_t(r[e + h]);
+      float x = fmaf(C.sc[cl + e + h], float(int32_t(r[e + h]) + C.nzw[cl + e + h] * asum_c + C.kw[cl + e + h]), C.bi[cl + e + h]);
+      if (ep.gelu) x = gelu_erf(x);
+      if (ep.residual) {
+        const int64_t off = m * ep.ld_residual + j + h;
+        x += ep.residual_bf16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(ep.residual)[off])
+                              : static_cast<const float*>(ep.residual)[off];
+      }
+      v[h] = x;
+    }
+    if (ep.rope != nullptr && j < ep.rope_cols)
+      rope_rotate(ep.rope[int64_t(m % ep.rope_period) * (ep.rope_dim >> 1) + ((j % ep.rope_dim) >> 1)], v[0], v[1]);
+    if (ep.glu) {
+      const float hv = silu_mul(v[0], v[1]);
+      const int oc = j >> 1;
+      if (ep.out_kind == REPQ_OUT_F32) {
+        static_cast<float*>(ep.out)[m * ep.ldo + oc] = hv;
+      } else if (ep.out_kind == REPQ_OUT_BF16) {
+        static_cast<__nv_bfloat16*>(ep.out)[m * ep.ldo + oc] = __float2bfloat16_rn(hv);
+      } else {
+        const uint32_t code = code_of(hv);
+        *code_sum += int(code);
+        static_cast<uint8_t*>(ep.out)[m * ep.ldo + oc] = uint8_t(code);
+      }
+      continue;
     }
     if (ep.out_kind == REPQ_OUT_F32) {
-      static_cast<float*>(ep.out)[m * ep.ldo + j] = v;
+      float* o = static_cast<float*>(ep.out) + m * ep.ldo + j;
+      o[0] = v[0];
+      if (two) o[1] = v[1];
     } else if (ep.out_kind == REPQ_OUT_BF16) {
-      static_cast<__nv_bfloat16*>(ep.out)[m * ep.ldo + j] = __float2bfloat16_rn(v);
+      __nv_bfloat16* o = static_cast<__nv_bfloat16*>(ep.out) + m * ep.ldo + j;
+      o[0] = __float2bfloat16_rn(v[0]);
+      if (two) o[1] = __float2bfloat16_rn(v[1]);
     } else {
-      const float t = fminf(fmaxf(v * q.mult, q.lo), q.hi);
-      const uint32_t code = (__float_as_uint(t + magic) - kMagicBits) + uint32_t(q.zo);
-      *code_sum += int(code);
+      const uint32_t c0 = code_of(v[0]), c1 = two ? code_of(v[1]) : 0u;
+      *code_sum += int(c0 + c1);
       uint8_t* orow = static_cast<uint8_t*>(ep.out) + m * ep.ldo;
       if (ep.pack4) {
-        if (e & 1) orow[j >> 1] = uint8_t(prev_code | (code << 4));
-        else if (j + 1 >= P.N) orow[j >> 1] = uint8_t(code);
-        prev_code = code;
+        orow[j >> 1] = uint8_t(c0 | (c1 << 4));
       } else {
-        orow[j] = uint8_t(code);
+        orow[j] = uint8_t(c0);
+        if (two) orow[j + 1] = uint8_t(c1);
       }
     }
   }
 }
 
-template <int BN, int OUT, bool RES>
+// PAIR: step on neighbouring column pairs ahead of the output conversion, compiled into the common epilogue only
+// where asked for: kPairNone, kPairRope (rotary embedding), kPairGlu (gated product; byte codes out)
+enum : int { kPairNone = 0, kPairRope = 1, kPairGlu = 2 };
+
+template <int BN, int OUT, bool RES, int PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_res, TcParams P) {
@@ -401,7 +431,8 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     const int kza = P.K * ep.z_a;
     const bool res16 = ep.residual != nullptr && ep.residual_bf16;
     const bool res32 = ep.residual != nullptr && !ep.residual_bf16;
-    const bool fast_ok = ep.acc_debug == nullptr;
+    // the common epilogue applies the pair step it was compiled with; any other combination goes chunk by chunk
+    const bool fast_ok = ep.acc_debug == nullptr && (ep.rope != nullptr) == (PAIR == kPairRope) && (ep.glu != 0) == (PAIR == kPairGlu);
     const bool sat = ep.qmax <= 127;             // byte codes narrow enough for the comparison-free quantizer
     const bool direct = P.direct_requant != 0;
     const int cl0 = slice * kSliceCols;          // first column of this warp inside the tile
@@ -484,6 +515,13 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       }
       fetch_terms(tile + int(gridDim.x));                    // next tile's inputs: in flight during this epilogue
       int code_sum = 0;
+      // rotary embedding: this row's line of the (cos, sin) table and the slice's first column inside its head
+      const float2* rope_row = nullptr;
+      int rope_hb = 0;
+      if (PAIR == kPairRope && n0 + cl0 < ep.rope_cols) {
+        rope_row = ep.rope + int64_t(m % ep.rope_period) * (ep.rope_dim >> 1);
+        rope_hb = (n0 + cl0) % ep.rope_dim;
+      }
 
       if (!mbar_wait(smem_u32(&S.tmem_full[acc]), acc_phase, abort, 4)) break;
       tc_fence_after();
@@ -545,8 +583,43 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
               }
             }
           }
+          if (PAIR == kPairRope && rope_row != nullptr && col0 < ep.rope_cols) {       // warp-uniform: range edges fall on chunk edges
+            int hx = rope_hb + c * kChunk;
+            while (hx >= ep.rope_dim) hx -= ep.rope_dim;
+            const float4* cs = reinterpret_cast<const float4*>(rope_row + (hx >> 1));
+#pragma unroll
+            for (int i = 0; i < kChunk / 4; ++i) {
+              const float4 t4 = __ldg(cs + i);
+              rope_rotate(make_float2(t4.x, t4.y), v[4 * i], v[4 * i + 1]);
+              rope_rotate(make_float2(t4.z, t4.w), v[4 * i + 2], v[4 * i + 3]);
+            }
+          }
           ChunkQuant q{};
           if constexpr (OUT == kOutC4 || OUT == kOutC8) q = chunk_quant(ep, P, col0);
+          if constexpr (OUT == kOutC8 && PAIR == kPairGlu) {
+            {
+              // gated product: 16 accumulator columns (gate, up interleaved) give 8 byte codes; the slice's 32 codes
+              // fill one box row
+              const float magic = __uint_as_float(kMagicBits);
+              uint32_t u[kChunk / 2];
+#pragma unroll
+              for (int i = 0; i < kChunk / 2; ++i) {
+                const float t = fminf(fmaxf(silu_mul(v[2 * i], v[2 * i + 1]) * q.mult, q.lo), q.hi);
+                u[i] = __float_as_uint(t + magic);
+              }
+              uint32_t w[2];
+#pragma unroll
+              for (int i = 0; i < 2; ++i) {
+                w[i] = __vadd4(__byte_perm(__byte_perm(u[4 * i], u[4 * i + 1], 0x0040), __byte_perm(u[4 * i + 2], u[4 * i + 3], 0x0040), 0x5410), q.z4);
+                code_sum += __dp4a(w[i], 0x01010101u, 0u);
+              }
+              const uint32_t buf = smem_u32(S.epi[ew]);
+              if (c == 0) box_begin(lane);
+              sts64(box_slot(buf, lane, c >> 1) + uint32_t(c & 1) * 8u, w[0], w[1]);
+              if (c == kSliceChunks - 1) box_end(&map_out, buf, lane, (col0 - (kSliceChunks - 1) * kChunk) >> 1, m0 + quarter * 32);
+              continue;
+            }
+          }
           emit_chunk<OUT>(&map_out, smem_u32(S.epi[ew]), lane, q, v, c, col0, m0 + quarter * 32, code_sum, direct, sat);
         }
       } else if (slice_on && any_row && n0 + cl0 < P.N) {
@@ -637,10 +710,10 @@ repq_status make_out_map(CUtensorMap* map, const TcParams& P) {
   REPQ_REQUIRE(fn != nullptr, REPQ_CUDA_ERROR, "qgemm: cuTensorMapEncodeTiled is not available");
   const EpilogueParams& ep = P.ep;
   CUtensorMapDataType dt = CU_TENSOR_MAP_DATA_TYPE_UINT8;
-  cuuint64_t inner = cuuint64_t(P.N), esz = 1;
+  cuuint64_t inner = cuuint64_t(ep.glu ? P.N / 2 : P.N), esz = 1;     // output columns
   if (ep.out_kind == REPQ_OUT_F32) { dt = CU_TENSOR_MAP_DATA_TYPE_FLOAT32; esz = 4; }
   else if (ep.out_kind == REPQ_OUT_BF16) { dt = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16; esz = 2; }
-  else if (ep.pack4) inner = cuuint64_t(P.N) / 2;
+  else if (ep.pack4) inner /= 2;
   const cuuint64_t dims[2] = {inner, cuuint64_t(P.M)};
   const cuuint64_t strides[1] = {cuuint64_t(ep.ldo) * esz};
   const cuuint32_t box[2] = {cuuint32_t(32 / esz), 32};
@@ -666,17 +739,17 @@ repq_status make_res_map(CUtensorMap* map, const TcParams& P) {
   return REPQ_OK;
 }
 
-template <int BN, int OUT, bool RES>
+template <int BN, int OUT, bool RES, int PAIR = kPairNone>
 repq_status launch_tc_res(const CUtensorMap& map_a, const CUtensorMap& map_b, const TcParams& P, int sms, cudaStream_t st) {
   CUtensorMap map_out, map_res;
   REPQ_TRY(make_out_map(&map_out, P));
   if (RES) REPQ_TRY(make_res_map(&map_res, P));
   else map_res = map_out;                                  // not read
   const size_t smem = sizeof(SharedStorage<BN, RES>);
-  REPQ_CUDA(cudaFuncSetAttribute(qgemm_tc_kernel<BN, OUT, RES>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+  REPQ_CUDA(cudaFuncSetAttribute(qgemm_tc_kernel<BN, OUT, RES, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
   const int tiles = ((P.M + BM - 1) / BM) * ((P.N + BN - 1) / BN);
   const int grid = tiles < sms ? tiles : sms;
-  REPQ_CUDA(launch_chained(qgemm_tc_kernel<BN, OUT, RES>, dim3(grid), dim3(kThreads), smem, st, map_a, map_b, map_out, map_res, P));
+  REPQ_CUDA(launch_chained(qgemm_tc_kernel<BN, OUT, RES, PAIR>, dim3(grid), dim3(kThreads), smem, st, map_a, map_b, map_out, map_res, P));
   note_launch();
   return REPQ_OK;
 }
@@ -698,10 +771,34 @@ repq_status launch_tc(const CUtensorMap& map_a, const CUtensorMap& map_b, const 
   if (P.ep.out_kind == REPQ_OUT_F32) return launch_tc_out<BN, kOutF32>(map_a, map_b, P, sms, st);
   if (P.ep.out_kind == REPQ_OUT_BF16) return launch_tc_out<BN, kOutBf16>(map_a, map_b, P, sms, st);
   if (P.ep.pack4) return launch_tc_out<BN, kOutC4>(map_a, map_b, P, sms, st);
+  if (P.ep.rope != nullptr) return launch_tc_res<BN, kOutC8, false, kPairRope>(map_a, map_b, P, sms, st);
+  if (P.ep.glu) return launch_tc_res<BN, kOutC8, false, kPairGlu>(map_a, map_b, P, sms, st);
   return launch_tc_out<BN, kOutC8>(map_a, map_b, P, sms, st);
 }
 
+// A wait that nothing ends: one thread sets up an mbarrier that never receives its arrival and waits on it through the
+// same bounded-wait routine as the tensor-core kernels, with the caller's limit.  The wait runs out, the status word
+// takes the code, the kernel returns.
+__global__ void wait_selftest_kernel(long long limit_cycles, int code) {
+  __shared__ alignas(8) uint64_t bar;
+  __shared__ volatile int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    tc::mbar_wait(smem_u32(&bar), 0, &abort_flag, code, &g_status_word, limit_cycles);
+  }
+}
+
 }  // namespace
+
+repq_status launch_wait_selftest(long long limit_cycles, cudaStream_t st) {
+  REPQ_REQUIRE(device_status_word() != nullptr, REPQ_CUDA_ERROR, "wait_selftest: device status word unavailable");
+  wait_selftest_kernel<<<1, 32, 0, st>>>(limit_cycles, 77);
+  REPQ_CUDA(cudaGetLastError());
+  note_launch();
+  return REPQ_OK;
+}
 
 int32_t* device_status_word() {
   static int32_t* addr[64] = {nullptr};
@@ -766,7 +863,7 @@ repq_status qgemm_tc(const repq_gemm_desc& d, const EpilogueParams& ep, void* ws
     P.wsum = s;
   }
   P.ep = ep;
-  P.direct_requant = d.out_kind == REPQ_OUT_CODES && !d.gelu && !d.residual;
+  P.direct_requant = d.out_kind == REPQ_OUT_CODES && !d.gelu && !d.residual && !d.glu;
   REPQ_REQUIRE(device_status_word() != nullptr, REPQ_CUDA_ERROR, "qgemm: device status word unavailable");
   const int sms = sm_count();
   const int bn = pick_bn(d.M, d.N, sms);

@@ -59,10 +59,20 @@ class QuantBlock:
             return (torch.from_numpy(g_t).to(dev), torch.from_numpy(b_t).to(dev), s_t, z_t,
                     _pack_linear(W_t, bias_t, bw, dev))
 
+        self.llama = cfg.get("arch", "vit") == "llama"
+        w_fc1, b_fc1 = w.w_fc1, w.b_fc1
+        if self.llama:
+            # gated MLP: the library takes gate_i and up_i as neighbouring weight rows (2i, 2i+1)
+            mlp = cfg["MLP"]
+            order = np.stack([np.arange(mlp), mlp + np.arange(mlp)], axis=1).reshape(-1)
+            w_fc1, b_fc1 = w.w_fc1[order], w.b_fc1[order]
         self.ln1_g, self.ln1_b, self.ln1_s, self.ln1_z, self.qkv = fold(
             w.ln1_gamma, w.ln1_beta, w.ln1_lo, w.ln1_hi, w.w_qkv, w.b_qkv, "ln1")
         self.ln2_g, self.ln2_b, self.ln2_s, self.ln2_z, self.fc1 = fold(
-            w.ln2_gamma, w.ln2_beta, w.ln2_lo, w.ln2_hi, w.w_fc1, w.b_fc1, "ln2")
+            w.ln2_gamma, w.ln2_beta, w.ln2_lo, w.ln2_hi, w_fc1, b_fc1, "ln2")
+        self.rope = None
+        if self.llama:
+            self.rope = torch.from_numpy(B.repq_rope_table(cfg["L"], cfg["D"] // cfg["H"], cfg.get("rope_base", 10000.0))).to(dev)
         self.proj = _pack_linear(w.w_proj, w.b_proj, bw, dev)
         self.fc2 = _pack_linear(w.w_fc2, w.b_fc2, bw, dev)
         self.act_q = {}
@@ -83,7 +93,10 @@ class QuantBlock:
         d = B.BlockDesc()
         d.batch, d.seq, d.dim, d.heads, d.mlp = batch, c["L"], c["D"], c["H"], c["MLP"]
         d.bits_a, d.bits_w, d.bits_p = c["bits_a"], self.bits_w, c["bits_p"]
-        d.causal, d.norm_kind, d.eps = int(c["causal"]), B.REPQ_NORM_LAYERNORM, c["eps"]
+        d.causal, d.eps = int(c["causal"]), c["eps"]
+        d.norm_kind = B.REPQ_NORM_RMS if self.llama else B.REPQ_NORM_LAYERNORM
+        d.rope = int(self.llama)
+        d.mlp_kind = B.REPQ_MLP_SWIGLU if self.llama else B.REPQ_MLP_GELU
         d.act_dtype = B.REPQ_F32 if self.act_dtype == torch.float32 else B.REPQ_BF16
         d.out_dtype = B.REPQ_F32 if self.out_dtype == torch.float32 else B.REPQ_BF16
         d.staged_attention = int(self.staged_attention)
@@ -101,6 +114,7 @@ class QuantBlock:
         p.fc1 = self.fc1.params()
         p.s_hidden, p.z_hidden = self.act_q["hidden"]
         p.fc2 = self.fc2.params()
+        p.rope_cos_sin = self.rope.data_ptr() if self.rope is not None else None
         return p
 
     def workspace(self, batch: int) -> torch.Tensor:

@@ -102,13 +102,15 @@ def ln_delta(x, gamma_t, s_t, t_lw, eps, rms):
     return 2.0 ** -19 * (np.abs(x) + np.abs(mu)) * rstd * np.abs(gamma_t)[None, :] / s_t + 2.0 ** -20 * np.abs(t_lw)
 
 
-def check_ln_quant(rows, D, bits, bf16, seed=0, rms=False, eps=1e-6, pad_cols=0, want_sum=True):
-    """Runs the fused LN+quant kernel and compares its codes with the oracle's channel-wise codes."""
+def check_ln_quant(rows, D, bits, bf16, seed=0, rms=False, eps=1e-6, pad_cols=0, want_sum=True, runs=1, inputs=None):
+    """Runs the fused LN+quant kernel and compares its codes with the oracle's channel-wise codes.  With
+    `runs` > 1 the launch is repeated and every launch has to write the bits of the first.  `inputs`, if given,
+    is (x, gamma, beta, lo, hi) of a real workload instead of the stage-level generator's."""
     import torch
     from oracle import repq_oracle as orc
     from paper_2402_05628_b200 import binding as B
 
-    x, gamma, beta, lo, hi = ln_case(rows, D, bf16, seed, rms, eps)
+    x, gamma, beta, lo, hi = ln_case(rows, D, bf16, seed, rms, eps) if inputs is None else inputs
     # oracle: complex (channel-wise) quantizer
     X1 = orc.layernorm(x, gamma, beta, eps, rms)
     s, z = orc.uniform_scale_zero(lo, hi, qb(bits))
@@ -127,9 +129,16 @@ def check_ln_quant(rows, D, bits, bf16, seed=0, rms=False, eps=1e-6, pad_cols=0,
     ld = B.code_row_bytes(D, bits)
     codes = torch.full((max(rows, 1), ld), 0xEE, dtype=torch.uint8, device=dev)[:rows]
     row_sum = torch.full((max(rows, 1),), -1, dtype=torch.int32, device=dev)[:rows] if want_sum else None
-    B.repq_ln_quant(xt, torch.from_numpy(gamma_t).to(dev), torch.from_numpy(beta_t).to(dev), eps, s_t, z_t, bits,
-                    codes, row_sum, B.REPQ_NORM_RMS if rms else B.REPQ_NORM_LAYERNORM)
-    torch.cuda.synchronize()
+    g_dev, b_dev = torch.from_numpy(gamma_t).to(dev), torch.from_numpy(beta_t).to(dev)
+    first = None
+    for _ in range(runs):
+        codes.fill_(0xEE)
+        B.repq_ln_quant(xt, g_dev, b_dev, eps, s_t, z_t, bits, codes, row_sum,
+                        B.REPQ_NORM_RMS if rms else B.REPQ_NORM_LAYERNORM)
+        torch.cuda.synchronize()
+        if first is None:
+            first = codes.clone()
+        assert torch.equal(codes, first), "launches differ"
     if rows == 0:
         return dict(total=0, mismatch=0, excused=0, bad=0)
     q_gpu = unpack_codes(codes.cpu().numpy(), D, bits)
@@ -250,6 +259,16 @@ def check_qgemm(M, N, K, bits_a, bits_w, out_kind="f32", gelu=False, residual=No
     B.repq_qgemm(d, ws)
     torch.cuda.synchronize()
     assert B.repq_device_status() == 0
+    out32 = None
+    if out_kind == "bf16":
+        # the same product with float32 output: the bf16 output has to be its round-to-nearest-even, bit for bit
+        out32 = torch.zeros(M, N, dtype=torch.float32, device=dev)
+        d32 = B.gemm_desc(M, N, K, a_t, bits_a, float(s_a), int(z_a), w_t, bits_w, out32, s_w=s_w_t, z_w=z_w_t,
+                          bias=bias_t, gelu=gelu, residual=res_t, acc_debug=None,
+                          **{k: v for k, v in kw.items() if k not in ("out_kind",)})
+        B.repq_qgemm(d32, ws)
+        torch.cuda.synchronize()
+        assert torch.equal(out32.to(torch.bfloat16), out), "bf16 output is not RNE(float32 output)"
     result = {}
     if want_acc:
         assert np.array_equal(acc.cpu().numpy().astype(np.int64), acc_ref), "int32 accumulators differ from brute force"
@@ -280,8 +299,8 @@ def check_qgemm(M, N, K, bits_a, bits_w, out_kind="f32", gelu=False, residual=No
             ref16 = orc.round_bf16(v_ref)
             addends = np.abs(v_ref - res) + np.abs(res) if res is not None else 0.0
             assert np.all(np.abs(got - ref16) <= np.abs(ref16) * 2.0 ** -7 + addends * 2.0 ** -22 + 1e-30)
-            rel, mx = float_errors(got, v_ref)
-            assert rel < 4e-3
+            rel, mx = assert_float_close(out32.cpu().numpy(), v_ref, "qgemm (float32 value behind the bf16 output)")
+            assert rel < 1e-5, rel
         else:
             rel, mx = assert_float_close(got, v_ref, "qgemm")
             assert rel < 1e-5, rel          # float32 epilogue on exact integers: far inside the tolerance
@@ -346,6 +365,14 @@ def check_pv(B_, H, Lq, Lk, dh, bits_p, bits_v, causal=False, out_kind="f32", ou
     d.out = out.data_ptr()
     B.repq_pv(d)
     torch.cuda.synchronize()
+    if out_kind == "bf16":
+        out32 = torch.zeros(B_ * Lq, D, dtype=torch.float32, device=dev)
+        d.out_kind, d.out = B.REPQ_OUT_F32, out32.data_ptr()
+        B.repq_pv(d)
+        torch.cuda.synchronize()
+        assert torch.equal(out32.to(torch.bfloat16), out), "bf16 output is not RNE(float32 output)"
+        rel, _ = assert_float_close(out32.cpu().numpy(), O_ref, "pv (float32 value behind the bf16 output)")
+        assert rel < 1e-5, rel
     if out_kind == "codes":
         q_gpu = unpack_codes(out.cpu().numpy(), D, out_bits)
         q_ref, t_ref = orc.quant_uniform(O_ref, s_o, z_o, qb(out_bits))
@@ -383,9 +410,9 @@ def check_block(name, batch, sample_items=None, out_dtype="f32", staged_attentio
     L = w.cfg["L"]
     blk = QuantBlock(w, out_dtype=torch.float32 if out_dtype == "f32" else torch.bfloat16, staged_attention=staged_attention)
     x = torch.from_numpy(w.x).to(blk.device).to(blk.act_dtype)
-    y = blk.forward(x)
+    y_dev = blk.forward(x)
     torch.cuda.synchronize()
-    y = y.float().cpu().numpy()
+    y = y_dev.float().cpu().numpy()
     assert np.all(np.isfinite(y))
     items = list(range(batch)) if sample_items is None else list(sample_items)
     rows = np.concatenate([np.arange(i * L, (i + 1) * L) for i in items])
@@ -395,9 +422,13 @@ def check_block(name, batch, sample_items=None, out_dtype="f32", staged_attentio
     ref = orc.block_forward(w_s)["y"]
     got = y[rows]
     if out_dtype == "bf16":
-        rel, mx = float_errors(got, ref)
-        assert rel < 6e-3, rel
-        return rel, mx
+        # the bf16 output is the float32 output rounded to nearest even, bit for bit (rounding to bf16 alone costs
+        # about 1.5e-3 of relative L2: the tolerance is spent on the float32 value)
+        blk32 = QuantBlock(w, out_dtype=torch.float32, staged_attention=staged_attention)
+        y32 = blk32.forward(x)
+        torch.cuda.synchronize()
+        assert torch.equal(y32.to(torch.bfloat16), y_dev), "bf16 block output is not RNE(float32 block output)"
+        got = y32.cpu().numpy()[rows]
     return assert_float_close(got, ref, "block %s" % name)
 
 
@@ -492,11 +523,18 @@ def check_pv_uniform_codes(B_, H, L, dh, bits_p, bits_v, runs=10, seed=0):
     assert B.repq_device_status() == 0
 
 
-def check_attention(B_, H, Lq, Lk, dh, bits, bits_p, causal=False, out_kind="f32", out_bits=4 | BYTE_CODES, seed=0, s_p=1.0):
+def check_attention(B_, H, Lq, Lk, dh, bits, bits_p, causal=False, out_kind="f32", out_bits=4 | BYTE_CODES, seed=0, s_p=1.0,
+                    inputs=None, out_quant=None):
     """repq_attention (scores, Softmax, log-sqrt2 codes and P.V fused) against the oracle's chain of the same
-    steps.  A Softmax code that sits on a rounding tie may legitimately differ by one (the near-tie protocol);
-    such a flip changes a whole output row, so rows that hold a near-tie are counted and left out of the strict
-    comparison."""
+    steps, all in float64 on the oracle's side.  A Softmax code whose pre-rounding value t sits on a rounding tie
+    may legitimately differ by one (the near-tie protocol); such a flip changes the whole output row, so a row
+    that holds near-ties is compared with every output the oracle gives with any subset of its tied codes moved
+    to the other neighbour, and has to match one of them as strictly as an ordinary row matches its only one.
+
+    `inputs`, if given, is (Qc, Kc, Vc, (s_q, z_q, s_k, z_k, s_v, z_v)): codes and quantizers of a real workload
+    instead of the uniformly random ones; `out_quant` = (s_o, z_o) likewise replaces the output quantizer that is
+    otherwise drawn from the output's percentiles."""
+    import itertools
     import torch
     from oracle import repq_oracle as orc
     from paper_2402_05628_b200 import binding as B
@@ -504,86 +542,475 @@ def check_attention(B_, H, Lq, Lk, dh, bits, bits_p, causal=False, out_kind="f32
     rng = np.random.default_rng(seed)
     D = H * dh
     nq = 1 << qb(bits)
-    Qc = rng.integers(0, nq, size=(B_ * Lq, D))
-    Kc = rng.integers(0, nq, size=(B_ * Lk, D))
-    Vc = rng.integers(0, nq, size=(B_ * Lk, D))
-    z_q, z_k, z_v = (int(rng.integers(0, nq)) for _ in range(3))
-    sig = (nq / 3.5) ** 2 * math.sqrt(dh)                 # rough std of sum (q - z_q)(k - z_k)
-    s_q = s_k = math.sqrt(3.0 * math.sqrt(dh) / sig)      # logits with a standard deviation of about 3
-    s_v = 0.05
-    alpha = 1.0 / math.sqrt(dh)
+    if inputs is None:
+        Qc = rng.integers(0, nq, size=(B_ * Lq, D))
+        Kc = rng.integers(0, nq, size=(B_ * Lk, D))
+        Vc = rng.integers(0, nq, size=(B_ * Lk, D))
+        z_q, z_k, z_v = (int(rng.integers(0, nq)) for _ in range(3))
+        sig = (nq / 3.5) ** 2 * math.sqrt(dh)                 # rough std of sum (q - z_q)(k - z_k)
+        s_q = s_k = math.sqrt(3.0 * math.sqrt(dh) / sig)      # logits with a standard deviation of about 3
+        s_v = 0.05
+    else:
+        Qc, Kc, Vc, (s_q, z_q, s_k, z_k, s_v, z_v) = inputs
+    # what the library is handed are float32 scales: the oracle takes the same numbers
+    s_q, s_k, s_v, s_p = (float(np.float32(v)) for v in (s_q, s_k, s_v, s_p))
+    alpha = float(np.float32(1.0 / math.sqrt(dh)))
     Qh, Kh, Vh = orc.dequant_uniform(Qc, s_q, z_q), orc.dequant_uniform(Kc, s_k, z_k), orc.dequant_uniform(Vc, s_v, z_v)
     shift = Lk - Lq
     valid = np.minimum(Lk, np.arange(Lq) + 1 + shift) if causal else np.full(Lq, Lk)
     O_ref = np.empty((B_ * Lq, D))
     absO = np.empty_like(O_ref)
-    tie_rows = np.zeros(B_ * Lq, dtype=bool)
+    tie_rows = {}                                    # (b, h, i) -> list of (key j, the other neighbour of t)
+    top = 2 ** qb(bits_p) - 1
     for b in range(B_):
         for h in range(H):
             sl = slice(h * dh, (h + 1) * dh)
             S = Qh[b * Lq:(b + 1) * Lq, sl] @ Kh[b * Lk:(b + 1) * Lk, sl].T * alpha
-            # the GPU forms S in float32 from the exact integer sum: do the same before the Softmax
-            S = S.astype(np.float32).astype(np.float64)
             A = orc.softmax_rows(S, valid)
             p, t = orc.quant_logsqrt2(A, s_p, qb(bits_p))
             mask = np.arange(Lk)[None, :] < valid[:, None]
             tf = np.where(mask & np.isfinite(t), t, 0.25)
-            near = mask & (np.abs(tf - np.floor(tf) - 0.5) < 2.0 ** -18 * np.maximum(1.0, np.abs(tf))) & (tf < min(2 ** qb(bits_p) - 0.4, 40.0))     # a flip below a weight of 2^-20 is invisible
-            tie_rows[b * Lq:(b + 1) * Lq] |= near.any(axis=1)
+            m_row = np.where(mask, S, -np.inf).max(axis=1, keepdims=True)
+            # width of a tie: float32 evaluation of t = 2 (log2 Z + log2 s) - 2 log2(e) (S - m) (2^-18 max(1, |t|), as
+            # for the separate Softmax kernel) plus what the float32 scores carry into it.  S = float(integer sum) *
+            # float(alpha s_q s_k): the rounding of the scale is common to S_i and m, so it is relative to S_i - m
+            # (part of the |t| term); the rounding of m itself, 2^-24 |m|, enters t through 2 log2(e) = 2.9
+            delta = 2.0 ** -18 * np.maximum(1.0, np.abs(tf)) + 2.0 ** -22 * np.abs(m_row)
+            near = mask & (np.abs(tf - np.floor(tf) - 0.5) < delta) & (tf < min(top + 0.6, 40.0))   # a flip below a weight of 2^-20 is invisible
+            for i, j in zip(*np.nonzero(near)):
+                alt = int(np.clip(np.floor(tf[i, j]) + np.ceil(tf[i, j]) - np.rint(tf[i, j]), 0, top))
+                if alt != int(p[i, j]):
+                    tie_rows.setdefault((b, h, int(i)), []).append((int(j), alt))
             A_hat = np.where(mask, orc.dequant_logsqrt2(p, s_p), 0.0)
             O_ref[b * Lq:(b + 1) * Lq, sl] = A_hat @ Vh[b * Lk:(b + 1) * Lk, sl]
             absO[b * Lq:(b + 1) * Lq, sl] = A_hat @ np.abs(Vh[b * Lk:(b + 1) * Lk, sl])
+            for (bb, hh, i), ties in tie_rows.items():
+                if (bb, hh) == (b, h) and isinstance(ties, list):
+                    # per tied key: what moving its code adds to the row's output
+                    tie_rows[(bb, hh, i)] = [(j, (float(orc.dequant_logsqrt2(alt, s_p)) - A_hat[i, j]) * Vh[b * Lk + j, sl],
+                                              abs(float(orc.dequant_logsqrt2(alt, s_p)) - A_hat[i, j]) * np.abs(Vh[b * Lk + j, sl]))
+                                             for j, alt in ties]
+                    tie_rows[(bb, hh, i)] = tuple(tie_rows[(bb, hh, i)])
     dev = torch.device("cuda:0")
     byte_bits = qb(bits) | BYTE_CODES
-    q_t = torch.from_numpy(Qc.astype(np.uint8)).to(dev)
-    k_t = torch.from_numpy(Kc.astype(np.uint8)).to(dev)
-    v_t = torch.from_numpy(Vc.astype(np.uint8)).to(dev)
+    q_t = torch.from_numpy(np.ascontiguousarray(Qc).astype(np.uint8)).to(dev)
+    k_t = torch.from_numpy(np.ascontiguousarray(Kc).astype(np.uint8)).to(dev)
+    v_t = torch.from_numpy(np.ascontiguousarray(Vc).astype(np.uint8)).to(dev)
     d = B.AttentionDesc()
     d.batch_outer, d.batch_inner, d.Lq, d.Lk, d.d_h, d.bits_qkv = B_, H, Lq, Lk, dh, byte_bits
     d.q_codes, d.ldq_bytes, d.q_stride_outer, d.q_stride_inner, d.s_q, d.z_q = q_t.data_ptr(), D, Lq * D, dh, s_q, z_q
     d.k_codes, d.ldk_bytes, d.k_stride_outer, d.k_stride_inner, d.s_k, d.z_k = k_t.data_ptr(), D, Lk * D, dh, s_k, z_k
     d.v_codes, d.ldv_bytes, d.v_stride_outer, d.v_stride_inner, d.s_v, d.z_v = v_t.data_ptr(), D, Lk * D, dh, s_v, z_v
     d.alpha, d.causal, d.bits_p, d.s_p = alpha, int(causal), bits_p, s_p
-    row_sum = None
+
+    def run(kind):
+        row_sum = None
+        if kind == "codes":
+            ldo = B.code_row_bytes(D, out_bits)
+            out = torch.full((B_ * Lq, ldo), 0xEE, dtype=torch.uint8, device=dev)
+            d.out_kind, d.out_bits, d.out_scale, d.out_zero = B.REPQ_OUT_CODES, out_bits, float(s_o), int(z_o)
+            d.ldo, d.o_stride_outer, d.o_stride_inner = ldo, Lq * ldo, (dh // 2 if out_bits == 4 else dh)
+            row_sum = torch.zeros(B_ * Lq, dtype=torch.int32, device=dev)
+            d.out_row_sum = row_sum.data_ptr()
+        else:
+            out = torch.zeros(B_ * Lq, D, dtype=torch.float32 if kind == "f32" else torch.bfloat16, device=dev)
+            d.out_kind = B.REPQ_OUT_F32 if kind == "f32" else B.REPQ_OUT_BF16
+            d.ldo, d.o_stride_outer, d.o_stride_inner = D, Lq * D, dh
+            d.out_row_sum = None
+        d.out = out.data_ptr()
+        first = None
+        for _ in range(3):                                   # repeated launches must agree bit for bit
+            if row_sum is not None:
+                row_sum.zero_()
+            B.repq_attention(d)
+            torch.cuda.synchronize()
+            if first is None:
+                first = out.clone()
+            assert torch.equal(out, first), "launches differ"
+        assert B.repq_device_status() == 0
+        return first, row_sum
+
     if out_kind == "codes":
-        s_o, z_o = orc.uniform_scale_zero(np.percentile(O_ref, 1), np.percentile(O_ref, 99), qb(out_bits))
-        ldo = B.code_row_bytes(D, out_bits)
-        out = torch.full((B_ * Lq, ldo), 0xEE, dtype=torch.uint8, device=dev)
-        d.out_kind, d.out_bits, d.out_scale, d.out_zero = B.REPQ_OUT_CODES, out_bits, float(s_o), int(z_o)
-        d.ldo, d.o_stride_outer, d.o_stride_inner = ldo, Lq * ldo, (dh // 2 if out_bits == 4 else dh)
-        row_sum = torch.zeros(B_ * Lq, dtype=torch.int32, device=dev)
-        d.out_row_sum = row_sum.data_ptr()
-    else:
-        out = torch.zeros(B_ * Lq, D, dtype=torch.float32 if out_kind == "f32" else torch.bfloat16, device=dev)
-        d.out_kind = B.REPQ_OUT_F32 if out_kind == "f32" else B.REPQ_OUT_BF16
-        d.ldo, d.o_stride_outer, d.o_stride_inner = D, Lq * D, dh
-    d.out = out.data_ptr()
-    first = None
-    for _ in range(3):                                   # repeated launches must agree bit for bit
-        if row_sum is not None:
-            row_sum.zero_()
-        B.repq_attention(d)
-        torch.cuda.synchronize()
-        got_raw = out.cpu().numpy() if out_kind != "bf16" else out.float().cpu().numpy()
-        if first is None:
-            first = got_raw.copy()
-        assert np.array_equal(got_raw, first), "launches differ"
-    assert B.repq_device_status() == 0
-    keep = ~tie_rows
-    assert keep.mean() > 0.9, "too many rows with a Softmax code on a rounding tie: %.3f" % (1 - keep.mean())
-    if out_kind == "codes":
-        q_gpu = unpack_codes(first, D, out_bits)
-        q_ref, t_ref = orc.quant_uniform(O_ref, s_o, z_o, qb(out_bits))
-        delta = 2.0 ** -17 * absO / s_o + 2.0 ** -20 * np.abs(t_ref)
-        rep = near_tie_report(q_gpu[keep], q_ref[keep], t_ref[keep], delta[keep])
-        assert rep["bad"] == 0, rep
-        assert np.array_equal(row_sum.cpu().numpy().astype(np.int64), q_gpu.sum(axis=1))
-        return rep
-    got = first.astype(np.float64)
+        if out_quant is None:
+            s_o, z_o = orc.uniform_scale_zero(np.percentile(O_ref, 1), np.percentile(O_ref, 99), qb(out_bits))
+        else:
+            s_o, z_o = out_quant
+    out_t, row_sum = run(out_kind)
     if out_kind == "bf16":
-        rel, _ = float_errors(got[keep], O_ref[keep])
-        assert rel < 6e-3, rel
-        return dict(rel_l2=rel)
+        # the bf16 output is the float32 output rounded to nearest even, bit for bit; the float32 output is what
+        # is compared with the oracle
+        out32, _ = run("f32")
+        assert torch.equal(out32.to(torch.bfloat16), out_t), "bf16 output is not RNE(float32 output)"
+        out_t = out32
+
+    def candidates(key):
+        """Outputs of a row that holds near-ties: the oracle's, plus any subset of the tied codes moved."""
+        b, h, i = key
+        ties = tie_rows[key]
+        base = O_ref[b * Lq + i, h * dh:(h + 1) * dh]
+        base_abs = absO[b * Lq + i, h * dh:(h + 1) * dh]
+        assert len(ties) <= 10, "a row with %d near-ties" % len(ties)
+        for n in range(len(ties) + 1):
+            for sub in itertools.combinations(ties, n):
+                yield base + sum((dv for _, dv, _ in sub), np.zeros(dh)), base_abs + sum((da for _, _, da in sub), np.zeros(dh))
+
+    tie_mask = np.zeros(B_ * Lq, dtype=bool)
+    for (b, h, i) in tie_rows:
+        tie_mask[b * Lq + i] = True
+    keep = ~tie_mask
+    n_tie = len(tie_rows)
+    if out_kind == "codes":
+        q_gpu = unpack_codes(out_t.cpu().numpy(), D, out_bits)
+
+        def code_report(got, ref_rows, abs_rows):
+            q_ref, t_ref = orc.quant_uniform(ref_rows, s_o, z_o, qb(out_bits))
+            delta = 2.0 ** -17 * abs_rows / s_o + 2.0 ** -20 * np.abs(t_ref)
+            return near_tie_report(got, q_ref, t_ref, delta)
+
+        rep = code_report(q_gpu[keep], O_ref[keep], absO[keep])
+        assert rep["bad"] == 0, rep
+        for key in tie_rows:
+            b, h, i = key
+            got = q_gpu[b * Lq + i, h * dh:(h + 1) * dh]
+            assert any(code_report(got, c, a)["bad"] == 0 for c, a in candidates(key)), ("tie row", key)
+        # untied heads of a tied row
+        for (b, h, i) in tie_rows:
+            for h2 in range(H):
+                if (b, h2, i) not in tie_rows:
+                    s2 = slice(h2 * dh, (h2 + 1) * dh)
+                    r = code_report(q_gpu[b * Lq + i, s2], O_ref[b * Lq + i, s2], absO[b * Lq + i, s2])
+                    assert r["bad"] == 0, r
+        assert np.array_equal(row_sum.cpu().numpy().astype(np.int64), q_gpu.sum(axis=1))
+        rep["tie_rows"] = n_tie
+        return rep
+    got = out_t.double().cpu().numpy()
     rel, mx = assert_float_close(got[keep], O_ref[keep], "attention")
     assert rel < 1e-4, rel                               # exact operands, float32 sums: far inside the tolerance
-    return dict(rel_l2=rel, max_abs=mx, tie_rows=int(tie_rows.sum()))
+    scale_all = np.abs(O_ref).max()
+    for key in tie_rows:
+        b, h, i = key
+        g = got[b * Lq + i, h * dh:(h + 1) * dh]
+        err = min(np.abs(g - c).max() / max(np.abs(c).max(), 1e-3 * scale_all) for c, _ in candidates(key))
+        assert err < 1e-4, ("tie row", key, err)
+    for (b, h, i) in tie_rows:
+        for h2 in range(H):
+            if (b, h2, i) not in tie_rows:
+                s2 = slice(h2 * dh, (h2 + 1) * dh)
+                ref = O_ref[b * Lq + i, s2]
+                assert np.abs(got[b * Lq + i, s2] - ref).max() <= 1e-4 * max(np.abs(ref).max(), 1e-3 * scale_all)
+    return dict(rel_l2=rel, max_abs=mx, tie_rows=n_tie)
+
+
+def check_block_teacher_forced(name, **overrides):
+    """Every stage of the block on the workload's own tensors, each fed the ORACLE's output of the stage before
+    (`block_forward(keep=True)`), with the engine's folded parameters: LayerNorm codes, Q / K / V codes, attention
+    codes, the residual stream, hidden codes and the block output are compared tensor by tensor, integer codes
+    under the near-tie protocol.  One batch item."""
+    import torch
+    from oracle import repq_oracle as orc
+    from paper_2402_05628_b200 import binding as B
+    from paper_2402_05628_b200.engine import QuantBlock
+    from workloads import make_block_inputs
+
+    w = make_block_inputs(name, batch=1, **overrides)
+    cfg = w.cfg
+    L, D, H, MLP = cfg["L"], cfg["D"], cfg["H"], cfg["MLP"]
+    dh, M = D // H, cfg["L"]
+    ba = cfg["bits_a"]
+    ab = ba | BYTE_CODES
+    llama = cfg.get("arch", "vit") == "llama"
+    ref = orc.block_forward(w, keep=True)
+    blk = QuantBlock(w, out_dtype=torch.float32)
+    dev = blk.device
+    norm_kind = B.REPQ_NORM_RMS if llama else B.REPQ_NORM_LAYERNORM
+    rep = {}
+
+    def dev_codes(q):
+        return torch.from_numpy(np.ascontiguousarray(q).astype(np.uint8)).to(dev)
+
+    def ln_stage(x_np, tag, g_dev, b_dev, s_t, z_t):
+        x_t = torch.from_numpy(np.ascontiguousarray(x_np, dtype=np.float32)).to(dev).to(blk.act_dtype)
+        codes = torch.full((M, D), 0xEE, dtype=torch.uint8, device=dev)
+        rs = torch.zeros(M, dtype=torch.int32, device=dev)
+        B.repq_ln_quant(x_t, g_dev, b_dev, cfg["eps"], s_t, z_t, ab, codes, rs, norm_kind)
+        torch.cuda.synchronize()
+        got = codes.cpu().numpy().astype(np.int64)
+        h = blk.host[tag]
+        t_cw = ref[tag + "_t"]
+        t_lw = t_cw + (h["z"].astype(np.int64) - z_t)[None, :]
+        r = near_tie_report(got, ref[tag + "_codes"], t_cw,
+                            ln_delta(x_np, h["gamma_t"].astype(np.float64), s_t, t_lw, cfg["eps"], llama))
+        assert r["bad"] == 0, (tag, r)
+        assert r["mismatch"] <= max(2, 2e-4 * r["total"]), (tag, r)
+        assert np.array_equal(rs.cpu().numpy().astype(np.int64), got.sum(axis=1))
+        rep[tag] = r
+
+    def linear_stage(a_codes, s_a, z_a, lin, N, **kw):
+        a_t = dev_codes(a_codes)
+        asum = torch.from_numpy(np.asarray(a_codes).sum(axis=1).astype(np.int32)).to(dev)
+        return a_t, asum, dict(s_w=lin.s_w, z_w=lin.z_w, w_row_sum=lin.w_row_sum, bias=lin.bias, a_row_sum=asum, **kw)
+
+    def run_gemm(d):
+        ws = torch.empty(max(B.repq_qgemm_workspace_bytes(d), 16), dtype=torch.uint8, device=dev)
+        B.repq_qgemm(d, ws)
+        torch.cuda.synchronize()
+        assert B.repq_device_status() == 0
+
+    def requant_report(got, name, mag):
+        """Codes of a layer-wise quantizer against the oracle's; `mag` bounds the float32 terms behind the value."""
+        lo, hi = w.bounds[name]
+        s_o, _ = orc.uniform_scale_zero(lo, hi, ba)
+        t = ref[name + "_t"]
+        r = near_tie_report(got, ref[name + "_codes"], t, 2.0 ** -19 * mag / float(s_o) + 2.0 ** -20 * np.abs(t))
+        assert r["bad"] == 0, (name, r)
+        assert r["mismatch"] <= max(2, 2e-4 * r["total"]), (name, r)
+        rep[name] = r
+
+    # ---- LayerNorm 1 on x
+    ln_stage(w.x, "ln1", blk.ln1_g, blk.ln1_b, blk.ln1_s, blk.ln1_z)
+
+    # ---- QKV projection on the oracle's LayerNorm codes (rotary embedding in the epilogue for the LLaMA form)
+    a_t, asum, kw = linear_stage(ref["ln1_codes"], blk.ln1_s, blk.ln1_z, blk.qkv, 3 * D)
+    qkv = torch.full((M, 3 * D), 0xEE, dtype=torch.uint8, device=dev)
+    quant = [blk.act_q[k] for k in ("q", "k", "v")]
+    if llama:
+        kw.update(rope=blk.rope, rope_period=L, rope_dim=dh, rope_groups=2)
+    d = B.gemm_desc(M, 3 * D, D, a_t, ab, blk.ln1_s, blk.ln1_z, blk.qkv.codes, blk.bits_w, qkv, out_kind=B.REPQ_OUT_CODES,
+                    out_bits=ab, out_scale=[q[0] for q in quant], out_zero=[q[1] for q in quant], **kw)
+    run_gemm(d)
+    got = qkv.cpu().numpy().astype(np.int64)
+    b_t = blk.qkv.bias.cpu().numpy().astype(np.float64)
+    for g, name in enumerate(("q", "k", "v")):
+        s_o, _ = orc.uniform_scale_zero(*w.bounds[name], ba)
+        v = ref[name + "_t"] * float(s_o)                           # the value the quantizer saw
+        if llama and name != "v":                                   # a rotation keeps the length of a pair
+            pair = np.sqrt(v[:, 0::2] ** 2 + v[:, 1::2] ** 2)
+            v = np.repeat(pair, 2, axis=1)
+            bias = np.abs(b_t[g * D:(g + 1) * D])
+            bias = np.repeat(np.maximum(bias[0::2], bias[1::2]), 2)
+            mag = 2.0 * (np.abs(v) + bias[None, :])
+        else:
+            mag = np.abs(v) + np.abs(b_t[g * D:(g + 1) * D])[None, :]
+        requant_report(got[:, g * D:(g + 1) * D], name, 2.0 * mag)
+
+    # ---- fused attention on the oracle's Q, K, V codes
+    quants = []
+    for name in ("q", "k", "v"):
+        s_, z_ = orc.uniform_scale_zero(*w.bounds[name], ba)
+        quants += [float(s_), int(z_)]
+    s_at, z_at = orc.uniform_scale_zero(*w.bounds["attn"], ba)
+    rep["attn"] = check_attention(1, H, L, L, dh, ab, cfg["bits_p"], causal=cfg["causal"], out_kind="codes", out_bits=ab,
+                                  s_p=w.softmax_scale, inputs=(ref["q_codes"], ref["k_codes"], ref["v_codes"], tuple(quants)),
+                                  out_quant=(float(s_at), int(z_at)))
+
+    # ---- output projection on the oracle's attention codes, residual x: the residual stream X_bar
+    s_a, z_a = blk.act_q["attn"]
+    a_t, asum, kw = linear_stage(ref["attn_codes"], s_a, z_a, blk.proj, D)
+    x_t = torch.from_numpy(np.ascontiguousarray(w.x)).to(dev).to(blk.act_dtype)
+    xbar = torch.zeros(M, D, dtype=blk.act_dtype, device=dev)
+    d = B.gemm_desc(M, D, D, a_t, ab, s_a, z_a, blk.proj.codes, blk.bits_w, xbar, residual=x_t,
+                    out_kind=B.REPQ_OUT_BF16 if blk.act_dtype == torch.bfloat16 else B.REPQ_OUT_F32, **kw)
+    run_gemm(d)
+    got = xbar.float().cpu().numpy().astype(np.float64)
+    xb = ref["x_bar"]
+    if blk.act_dtype == torch.bfloat16:
+        # RNE(float32 value) within one bf16 ulp of the oracle's rounded value; where the residual cancels the GEMM
+        # value the float32 rounding of the two addends (2^-23 of each) remains in the small sum
+        addends = np.abs(xb - w.x) + np.abs(w.x)
+        assert np.all(np.abs(got - xb) <= np.abs(xb) * 2.0 ** -7 + addends * 2.0 ** -22 + 1e-30), "x_bar"
+        rep["x_bar"] = float(np.mean(got != xb))
+    else:
+        rel, _ = assert_float_close(got, xb, "x_bar")
+        assert rel < 1e-5, rel
+        rep["x_bar"] = rel
+
+    # ---- LayerNorm 2 on the oracle's residual stream
+    ln_stage(xb, "ln2", blk.ln2_g, blk.ln2_b, blk.ln2_s, blk.ln2_z)
+
+    # ---- fc1 on the oracle's LayerNorm-2 codes: GELU, or the gated product of the LLaMA form
+    n_fc1 = 2 * MLP if llama else MLP
+    a_t, asum, kw = linear_stage(ref["ln2_codes"], blk.ln2_s, blk.ln2_z, blk.fc1, n_fc1)
+    hid = torch.full((M, MLP), 0xEE, dtype=torch.uint8, device=dev)
+    s_h, z_h = blk.act_q["hidden"]
+    d = B.gemm_desc(M, n_fc1, D, a_t, ab, blk.ln2_s, blk.ln2_z, blk.fc1.codes, blk.bits_w, hid, out_kind=B.REPQ_OUT_CODES,
+                    out_bits=ab, out_scale=[s_h], out_zero=[z_h], gelu=not llama, glu=llama, **kw)
+    run_gemm(d)
+    pre = orc.linear_after_layernorm(ref["ln2_codes"], ref["ln2_s"], ref["ln2_z"], ref["ln2_rp"], ref["ln2_wcodes"],
+                                     ref["ln2_sw"], ref["ln2_zw"])
+    b_t = np.abs(ref["ln2_rp"]["b_t"])
+    if llama:
+        g_, u_ = pre[:, :MLP], pre[:, MLP:]
+        dg = np.abs(g_) + b_t[None, :MLP]                  # float32 terms behind gate and up
+        du = np.abs(u_) + b_t[None, MLP:]
+        mag = 1.2 * dg * np.abs(u_) + np.abs(orc.silu(g_)) * du + 2.0 * np.abs(orc.silu(g_) * u_)      # ex2 / division approximations: 2^-20 of the product
+    else:
+        mag = 1.2 * (np.abs(pre) + b_t[None, :]) + np.abs(orc.gelu(pre))
+    requant_report(hid.cpu().numpy().astype(np.int64), "hidden", 2.0 * mag)
+
+    # ---- fc2 on the oracle's hidden codes, residual X_bar: the block output
+    a_t, asum, kw = linear_stage(ref["hidden_codes"], s_h, z_h, blk.fc2, D)
+    xb_t = torch.from_numpy(np.ascontiguousarray(xb, dtype=np.float32)).to(dev).to(blk.act_dtype)
+    y = torch.zeros(M, D, dtype=torch.float32, device=dev)
+    d = B.gemm_desc(M, D, MLP, a_t, ab, s_h, z_h, blk.fc2.codes, blk.bits_w, y, residual=xb_t, out_kind=B.REPQ_OUT_F32, **kw)
+    run_gemm(d)
+    rel, _ = assert_float_close(y.cpu().numpy(), ref["y"], "y")
+    assert rel < 1e-5, rel
+    rep["y"] = rel
+    return rep
+
+
+def check_qgemm_pair_step(M, N, K, bits, mode, out_kind="codes", seed=0, L=50, dh=32):
+    """repq_qgemm with one of the two steps on neighbouring column pairs (LLaMA block form) against the oracle:
+    mode "rope": the first two of three column ranges rotated by position m mod L (then Eq. 4 per range);
+    mode "glu": columns (2i, 2i+1) = (gate, up), output silu(gate) * up (then Eq. 4)."""
+    import torch
+    from oracle import repq_oracle as orc
+    from paper_2402_05628_b200 import binding as B
+    from workloads.kernels import gemm_codes
+
+    rng = np.random.default_rng(seed)
+    a, wq, s_a, z_a, s_w, z_w, bias = gemm_codes(rng, M, N, K, qb(bits), qb(bits))
+    v_lin = orc.linear(orc.dequant_uniform(a, s_a, z_a), wq, s_w, z_w, bias)
+    lin_mag = np.abs(v_lin - bias[None, :]) + np.abs(bias)[None, :]
+    dev = torch.device("cuda:0")
+    lda = B.code_row_bytes(K, bits)
+    a_t = torch.from_numpy(pack_codes(a, bits, lda)).to(dev)
+    w_t = torch.from_numpy(pack_codes(wq, bits, lda)).to(dev)
+    s_w_t, z_w_t, bias_t = (torch.from_numpy(v).to(dev) for v in (s_w, z_w, bias))
+    kw = dict(s_w=s_w_t, z_w=z_w_t, bias=bias_t)
+    if mode == "rope":
+        gw = N // 3
+        H = gw // dh
+        assert H * dh == gw and M % L == 0
+        table = torch.from_numpy(B.repq_rope_table(L, dh, 10000.0)).to(dev)
+        v_ref = v_lin.copy()
+        mag = lin_mag.copy()
+        for g in range(2):
+            sl = slice(g * gw, (g + 1) * gw)
+            v_ref[:, sl] = orc.rope(v_lin[:, sl], M // L, L, H, 10000.0)
+            pm = np.sqrt(lin_mag[:, sl][:, 0::2] ** 2 + lin_mag[:, sl][:, 1::2] ** 2)
+            mag[:, sl] = 2.0 * np.repeat(pm, 2, axis=1)
+        kw.update(rope=table, rope_period=L, rope_dim=dh, rope_groups=2)
+        n_out, groups = N, 3
+    else:
+        g_, u_ = v_lin[:, 0::2], v_lin[:, 1::2]
+        v_ref = orc.silu(g_) * u_
+        mag = 1.2 * lin_mag[:, 0::2] * np.abs(u_) + np.abs(orc.silu(g_)) * lin_mag[:, 1::2] + 2.0 * np.abs(v_ref)
+        kw.update(glu=True)
+        n_out, groups = N // 2, 1
+    if out_kind == "codes":
+        ob = qb(bits) | BYTE_CODES
+        gw_o = n_out // groups
+        lo = [np.percentile(v_ref[:, g * gw_o:(g + 1) * gw_o], 1) for g in range(groups)]
+        hi = [np.percentile(v_ref[:, g * gw_o:(g + 1) * gw_o], 99) for g in range(groups)]
+        s_o, z_o = orc.uniform_scale_zero(np.array(lo), np.array(hi), qb(bits))
+        out = torch.full((M, B.code_row_bytes(n_out, ob)), 0xEE, dtype=torch.uint8, device=dev)
+        rs = torch.zeros(M, dtype=torch.int32, device=dev)
+        kw.update(out_kind=B.REPQ_OUT_CODES, out_bits=ob, out_scale=[float(v) for v in s_o], out_zero=[int(v) for v in z_o],
+                  out_row_sum=rs)
+    else:
+        out = torch.zeros(M, n_out, dtype=torch.float32, device=dev)
+        if mode == "rope":
+            kw.update(out_scale=[1.0, 1.0, 1.0], out_zero=[0, 0, 0])          # three ranges: the first two are rotated
+    d = B.gemm_desc(M, N, K, a_t, bits, float(s_a), int(z_a), w_t, bits, out, **kw)
+    ws = torch.empty(max(B.repq_qgemm_workspace_bytes(d), 16), dtype=torch.uint8, device=dev)
+    B.repq_qgemm(d, ws)
+    torch.cuda.synchronize()
+    assert B.repq_device_status() == 0
+    if out_kind != "codes":
+        rel, mx = assert_float_close(out.cpu().numpy(), v_ref, "qgemm " + mode)
+        assert rel < 2e-6, rel
+        return dict(rel_l2=rel)
+    q_gpu = out.cpu().numpy()[:, :n_out].astype(np.int64)
+    rep = dict(total=0, mismatch=0, excused=0, bad=0)
+    for g in range(groups):
+        sl = slice(g * gw_o, (g + 1) * gw_o)
+        q_ref, t_ref = orc.quant_uniform(v_ref[:, sl], s_o[g], z_o[g], qb(bits))
+        r = near_tie_report(q_gpu[:, sl], q_ref, t_ref, 2.0 ** -19 * mag[:, sl] / s_o[g] + 2.0 ** -20 * np.abs(t_ref))
+        for k in rep:
+            rep[k] += r[k]
+    assert rep["bad"] == 0, rep
+    assert rep["mismatch"] <= max(2, 2e-4 * rep["total"]), rep
+    assert np.array_equal(rs.cpu().numpy().astype(np.int64), q_gpu.sum(axis=1))
+    return rep
+
+
+def check_qgemm_repeated(M, N, K, bits, residual, out_kind, runs=12, seed=0):
+    """A GEMM with a residual on dense random data, launched `runs` times: every launch reproduces the oracle and
+    the first launch bit for bit (the residual boxes are refilled by bulk copies right after they are read)."""
+    import torch
+    from oracle import repq_oracle as orc
+    from paper_2402_05628_b200 import binding as B
+    from workloads.kernels import gemm_codes, to_bf16_grid
+
+    rng = np.random.default_rng(seed)
+    b = bits | BYTE_CODES
+    a, wq, s_a, z_a, s_w, z_w, bias = gemm_codes(rng, M, N, K, bits, bits)
+    res = rng.normal(0, 1.0, size=(M, N)).astype(np.float32)
+    if residual == "bf16":
+        res = to_bf16_grid(res)
+    v_ref = orc.linear(orc.dequant_uniform(a, s_a, z_a), wq, s_w, z_w, bias) + res
+    dev = torch.device("cuda:0")
+    a_t = torch.from_numpy(a.astype(np.uint8)).to(dev)
+    w_t = torch.from_numpy(wq.astype(np.uint8)).to(dev)
+    res_t = torch.from_numpy(res).to(dev)
+    if residual == "bf16":
+        res_t = res_t.to(torch.bfloat16)
+    s_w_t, z_w_t, bias_t = (torch.from_numpy(v).to(dev) for v in (s_w, z_w, bias))
+    out = torch.zeros(M, N, dtype=torch.float32 if out_kind == "f32" else torch.bfloat16, device=dev)
+    d = B.gemm_desc(M, N, K, a_t, b, float(s_a), int(z_a), w_t, b, out, s_w=s_w_t, z_w=z_w_t, bias=bias_t, residual=res_t,
+                    out_kind=B.REPQ_OUT_F32 if out_kind == "f32" else B.REPQ_OUT_BF16)
+    ws = torch.empty(max(B.repq_qgemm_workspace_bytes(d), 16), dtype=torch.uint8, device=dev)
+    first = None
+    for _ in range(runs):
+        out.zero_()
+        B.repq_qgemm(d, ws)
+        torch.cuda.synchronize()
+        if first is None:
+            first = out.clone()
+            got = out.float().cpu().numpy()
+            if out_kind == "f32":
+                rel, _ = assert_float_close(got, v_ref, "qgemm + residual")
+                assert rel < 1e-5, rel
+            else:
+                ref16 = orc.round_bf16(v_ref)
+                addends = np.abs(v_ref - res) + np.abs(res)
+                assert np.all(np.abs(got - ref16) <= np.abs(ref16) * 2.0 ** -7 + addends * 2.0 ** -22 + 1e-30)
+        assert torch.equal(out, first), "launches differ"
+    assert B.repq_device_status() == 0
+
+
+def check_dual_clip(n, D, bits, seed=0, iters=100, alpha0=2.0, strided=False):
+    """repq_dual_clip against the oracle's per-channel dual clipping on LayerNorm activations of the stage-level
+    generator: learned bounds and the objective before / after.  Both sides work in float64; they differ in the
+    order of the sums over tokens, so a value that sits on a rounding tie to within round-off may steer one step of
+    one channel differently: the bounds are compared to 1e-6 of the channel's range."""
+    import torch
+    from oracle import repq_oracle as orc
+    from paper_2402_05628_b200 import binding as B
+    from workloads.kernels import affine_params, channel_profile, ln_inputs
+
+    rng = np.random.default_rng(seed)
+    c, shift = channel_profile(rng, D, 1.0, 0.02, 20.0)
+    gamma, beta = affine_params(rng, D)
+    X1 = orc.layernorm(ln_inputs(rng, n, c, shift, False), gamma, beta, 1e-6).astype(np.float32)
+    ref = orc.dual_clip(X1, bits, iters=iters, lr=0.01, alpha0=alpha0)
+    dev = torch.device("cuda:0")
+    if strided:
+        buf = torch.zeros(n, D + 5, dtype=torch.float32, device=dev)
+        buf[:, :D] = torch.from_numpy(X1).to(dev)
+        x_t = buf[:, :D]
+    else:
+        x_t = torch.from_numpy(X1).to(dev)
+    lo = torch.full((D,), float("nan"), device=dev)
+    hi = torch.full((D,), float("nan"), device=dev)
+    loss = torch.zeros(2 * D, dtype=torch.float64, device=dev)
+    B.repq_dual_clip(x_t, bits, lo, hi, loss, iters=iters, lr=0.01, alpha0=alpha0)
+    torch.cuda.synchronize()
+    rng_ch = X1.max(axis=0).astype(np.float64) - X1.min(axis=0)
+    assert np.all(np.abs(lo.cpu().numpy() - ref["x_low"]) <= 1e-6 * rng_ch + 1e-7 * np.abs(ref["x_low"])), "x_low"
+    assert np.all(np.abs(hi.cpu().numpy() - ref["x_up"]) <= 1e-6 * rng_ch + 1e-7 * np.abs(ref["x_up"])), "x_up"
+    got = loss.cpu().numpy()
+    assert np.allclose(got[:D], ref["loss0"], rtol=1e-9), "objective before the first step"
+    assert np.allclose(got[D:], ref["loss"], rtol=1e-5), "objective with the learned bounds"
+    return dict(loss0=float(ref["loss0"].sum()), loss=float(ref["loss"].sum()))

@@ -52,6 +52,36 @@ def test_block_c4_llama_shaped_full_size_sampled_item():
     parity.check_block("c4_llama7b", batch=4, sample_items=(3,))
 
 
+def test_block_llama_form_small():
+    # RMS normalisation, rotary embedding on Q / K, gated SiLU MLP, causal Softmax with 8-bit log codes
+    parity.check_block("c4_llama7b_arch", batch=2, D=512, H=4, MLP=1408, L=320, massive=2)
+    parity.check_block("c4_llama7b_arch", batch=2, D=512, H=8, MLP=1408, L=200, massive=2, out_dtype="bf16")
+
+
+def test_block_c4_llama_form_full_size_sampled_item():
+    parity.check_block("c4_llama7b_arch", batch=4, sample_items=(1,))
+
+
+@pytest.mark.parametrize("name,overrides", [
+    ("c2_deit_b", {}), ("c2_deit_b_w6a6", {}), ("c3_vit_l", {}),
+    ("c4_llama7b", dict(D=1024, H=8, MLP=2816, L=640, massive=4)),
+    ("c4_llama7b_arch", dict(D=1024, H=8, MLP=2816, L=640, massive=4)),
+])
+def test_block_stages_teacher_forced_on_workload_tensors(name, overrides):
+    """Each stage of the block on the workload's own distributions, fed the oracle's output of the stage before:
+    every in-block code tensor against the oracle's."""
+    rep = parity.check_block_teacher_forced(name, **overrides)
+    print(name, rep)
+
+
+def test_block_stages_teacher_forced_c4_full_size():
+    parity.check_block_teacher_forced("c4_llama7b")
+
+
+def test_block_stages_teacher_forced_c4_llama_form_full_size():
+    parity.check_block_teacher_forced("c4_llama7b_arch")
+
+
 def test_block_with_the_three_separate_attention_stages():
     """The block through repq_qgemm (scores) -> repq_softmax_log2 -> repq_pv instead of the fused kernel."""
     parity.check_block("c2_deit_b", batch=3, staged_attention=True)

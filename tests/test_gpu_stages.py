@@ -24,6 +24,15 @@ def test_ln_quant_matches_channelwise_oracle(rows, D, bits, bf16):
     assert rep["mismatch"] <= max(2, 2e-4 * rep["total"]), rep
 
 
+@pytest.mark.parametrize("D", [4096, 8192, 768])
+def test_ln_quant_mean_free_without_row_sums_repeated(D):
+    """Mean-free normalisation without row sums runs one reduction per row (one barrier per iteration of a thread
+    group wider than a warp): repeated launches over many rows per block agree with the oracle and one another."""
+    rep = parity.check_ln_quant(20000, D, 4, True, seed=D, rms=True, eps=1e-5, want_sum=False, runs=6)
+    assert rep["bad"] == 0, rep
+    assert rep["mismatch"] <= max(2, 2e-4 * rep["total"]), rep
+
+
 def test_ln_quant_rms_strided_and_empty():
     assert parity.check_ln_quant(300, 4096, 4, True, seed=3, rms=True, eps=1e-5)["bad"] == 0
     assert parity.check_ln_quant(300, 768, 4, True, seed=4, pad_cols=8)["bad"] == 0
@@ -157,3 +166,57 @@ def test_qgemm_common_epilogue_path(M, N, K, bits, out_bits, groups, gelu, resid
     ob = -out_bits if out_bits < 0 else (out_bits | parity.BYTE_CODES)              # negative: packed 4-bit output
     parity.check_qgemm(M, N, K, b, b, out_kind=out_kind, gelu=gelu, residual=residual, groups=groups, out_bits=ob,
                        want_acc=False, want_out_sum=(out_kind == "codes"), seed=M + N + K + groups)
+
+
+@pytest.mark.parametrize("M,N,K,bits,out_kind", [
+    (300, 768, 256, 4, "codes"), (400, 1536, 384, 4, "codes"), (150, 192, 128, 8, "codes"), (300, 768, 256, 4, "f32"),
+    (50, 96, 64, 4, "codes"),                 # small: the warp-MMA kernel
+])
+def test_qgemm_rotary_embedding_in_the_epilogue(M, N, K, bits, out_kind):
+    dh = 32 if N % 96 == 0 else 64
+    parity.check_qgemm_pair_step(M, N, K, bits | parity.BYTE_CODES, "rope", out_kind=out_kind, seed=M + N, L=50, dh=dh)
+
+
+@pytest.mark.parametrize("M,N,K,bits,out_kind", [
+    (300, 1024, 256, 4, "codes"), (389, 2816, 512, 4, "codes"), (260, 640, 128, 8, "codes"), (300, 512, 256, 6, "f32"),
+    (40, 96, 64, 4, "codes"),
+])
+def test_qgemm_gated_product_in_the_epilogue(M, N, K, bits, out_kind):
+    parity.check_qgemm_pair_step(M, N, K, bits | parity.BYTE_CODES, "glu", out_kind=out_kind, seed=M + N)
+
+
+@pytest.mark.parametrize("M,N,K,residual,out_kind", [
+    (12608, 768, 768, "bf16", "bf16"),        # residual boxes by bulk tensor copies (short K)
+    (4000, 768, 3072, "bf16", "bf16"),        # row-per-lane residual loads
+    (3000, 512, 256, "f32", "f32"),
+])
+def test_qgemm_with_residual_repeated_launches(M, N, K, residual, out_kind):
+    parity.check_qgemm_repeated(M, N, K, 4, residual, out_kind, runs=12, seed=K)
+
+
+def test_bounded_wait_runs_out_and_the_context_survives():
+    """A device-side wait that nothing ends returns after its limit, reports through the health word, and the
+    next launches are correct."""
+    import torch
+    from paper_2402_05628_b200 import binding as B
+    torch.cuda.synchronize()
+    assert B.repq_device_status(reset=True) == 0
+    B.repq_bounded_wait_selftest(2_000_000)               # about a millisecond of SM clock
+    torch.cuda.synchronize()
+    assert B.repq_device_status() == 77                    # the self-test's code; the library call says REPQ_TIMEOUT
+    v = __import__("ctypes").c_int32()
+    assert B.lib().repq_device_status(__import__("ctypes").byref(v), 1) == B.REPQ_TIMEOUT and v.value == 77
+    assert B.repq_device_status() == 0                     # cleared by the reset above
+    parity.check_qgemm(300, 192, 256, 4, 4, out_kind="bf16", seed=1)
+    assert parity.check_ln_quant(300, 768, 4, True, seed=4)["bad"] == 0
+    with pytest.raises(B.RepqError):
+        B.repq_bounded_wait_selftest(0)
+
+
+@pytest.mark.parametrize("n,D,bits,iters,strided", [
+    (1500, 48, 4, 100, False), (6304, 384, 4, 100, False), (700, 100, 8, 30, True), (33, 7, 6, 10, False), (900, 64, 4, 0, False),
+])
+def test_dual_clip_matches_oracle(n, D, bits, iters, strided):
+    rep = parity.check_dual_clip(n, D, bits, seed=n + D, iters=iters, strided=strided)
+    if iters:
+        assert rep["loss"] < rep["loss0"]

@@ -29,7 +29,7 @@ def test_exports_match_header(B):
     for name in sorted(declared):
         assert hasattr(lib, name), "library does not export %s" % name
     assert declared == set(B.EXPORTS)
-    assert lib.repq_abi_version() == 4
+    assert lib.repq_abi_version() == 5
 
 
 def test_scale_zero_from_bounds_matches_oracle(B):
@@ -99,3 +99,22 @@ def test_device_entry_points_validate_arguments_without_gpu(B):
     assert lib.repq_softmax_log2(16, 0, 4, 64, 64, 1.0, 0, 0, 1.0, 5, 16, 32, None) == B.REPQ_INVALID_ARG
     assert lib.repq_ln_quant(16, 0, 4, 60, 64, 16, 16, 1e-6, 0, 1.0, 0, 4, 16, 32, None, None) == B.REPQ_UNSUPPORTED
     assert lib.repq_ln_quant(16, 0, 4, 64, 64, 16, 16, 1e-6, 0, 1.0, 0, 4, 18, 32, None, None) == B.REPQ_ALIGNMENT
+
+
+def test_rope_table_rotates_like_the_oracle(B):
+    """The library's (cos, sin) table applied to a matrix gives the oracle's rotary embedding (float32 table against
+    float64 angles: a few units of 2^-24 per entry)."""
+    rng = np.random.default_rng(9)
+    L, H, dh = 37, 2, 32
+    t = B.repq_rope_table(L, dh, 10000.0).astype(np.float64)          # [L, dh/2, 2]
+    X = rng.normal(size=(2 * L, H * dh))
+    ref = orc.rope(X, 2, L, H, 10000.0)
+    cos = np.tile(t[:, :, 0], (2, H))
+    sin = np.tile(t[:, :, 1], (2, H))
+    got = np.empty_like(X)
+    got[:, 0::2] = X[:, 0::2] * cos - X[:, 1::2] * sin
+    got[:, 1::2] = X[:, 0::2] * sin + X[:, 1::2] * cos
+    assert np.abs(got - ref).max() < 4e-7 * np.abs(X).max()
+    assert t[0, :, 0].tolist() == [1.0] * (dh // 2) and t[0, :, 1].tolist() == [0.0] * (dh // 2)
+    with pytest.raises(B.RepqError):
+        B.repq_rope_table(L, 7, 10000.0)

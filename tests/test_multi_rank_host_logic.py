@@ -39,3 +39,15 @@ def test_two_ranks_shard_the_batch_and_take_the_slowest_timing():
         assert p.exitcode == 0
     assert spans == [(0, 3 * 197), (3 * 197, 6 * 197)]          # disjoint, contiguous, whole batch items
     assert slowest == [11.0, 5.0]
+
+
+def test_bench_starts_its_own_ranks_when_not_launched_as_ranks():
+    """`bench.py --gpus N` without a launcher's environment hands over to N ranks on this node (one per GPU,
+    rendezvous on 127.0.0.1); the command line it builds is checked here, nothing is started."""
+    sys.path.insert(0, ROOT)
+    import bench
+    cmd = bench.spawn_command(4, ["--gpus", "4", "--steps", "20"], 29555)
+    assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"]
+    assert cmd[cmd.index("--nproc-per-node") + 1] == "4"
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[cmd.index("--master-port") + 1] == "29555"
+    assert cmd[-4:] == ["--gpus", "4", "--steps", "20"] and cmd[-5].endswith("bench.py")

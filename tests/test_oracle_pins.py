@@ -612,3 +612,90 @@ def test_llama_form_reduces_to_paper_form_pieces():
     assert np.allclose(orc.layernorm(X, g, b, 1e-6, rms=True), orc.layernorm(X, g, b, 1e-6), rtol=1e-12, atol=1e-12)
     ref = torch.nn.functional.rms_norm(torch.from_numpy(X + 0.3), (16,), weight=torch.from_numpy(g), eps=1e-6).numpy() + b
     assert np.allclose(orc.layernorm(X + 0.3, g, b, 1e-6, rms=True), ref, rtol=1e-12, atol=1e-12)
+
+
+# ------------------------------------------------------------------ per-channel dual clipping (Eqs. 18-20)
+
+def _torch_dual_clip_loss(Xt, a1, a2, bits):
+    """Eq. 20 through torch autograd: quantizer of Eqs. 4-6 on the bounds of Eqs. 18-19, round passed straight
+    through (library routines: sigmoid, round, clamp, autograd)."""
+    Q = 2 ** bits - 1
+    up = Xt.max(0).values * torch.sigmoid(a1)
+    low = Xt.min(0).values * torch.sigmoid(a2)
+    s = (up - low) / Q
+    ste = lambda v: (torch.round(v) - v).detach() + v
+    z = ste(-low / s)
+    q = torch.clamp(ste(Xt / s) + z, 0, Q)
+    return ((s * (q - z) - Xt) ** 2).sum(0)
+
+
+def _clip_case(seed=0, n=600, D=7):
+    rng = np.random.default_rng(seed)
+    X = rng.normal(size=(n, D)) * np.exp(rng.normal(0, 1, D)) + rng.normal(0, 1, D)
+    X[::40, 2] *= 5.0            # one-sided outliers in one channel, two-sided in another
+    X[7::55, 4] -= 6.0
+    X[3::70, 4] += 9.0
+    return X
+
+
+@pytest.mark.parametrize("bits", [4, 6, 8])
+def test_dual_clip_loss_and_gradient_match_autograd(bits):
+    X = _clip_case()
+    D = X.shape[1]
+    rng = np.random.default_rng(bits)
+    a1n, a2n = rng.normal(0, 1.5, D), rng.normal(0, 1.5, D)
+    a1 = torch.tensor(a1n, requires_grad=True)
+    a2 = torch.tensor(a2n, requires_grad=True)
+    L = _torch_dual_clip_loss(torch.from_numpy(X), a1, a2, bits)
+    L.sum().backward()
+    loss, g1, g2 = orc.dual_clip_loss_grad(X, a1n, a2n, bits)
+    assert np.allclose(loss, L.detach().numpy(), rtol=1e-12)
+    assert np.allclose(g1, a1.grad.numpy(), rtol=1e-9, atol=1e-9 * np.abs(g1).max())
+    assert np.allclose(g2, a2.grad.numpy(), rtol=1e-9, atol=1e-9 * np.abs(g2).max())
+    # the loss is the quantization error of the channel-wise quantizer built on the same bounds
+    up, low = orc.dual_clip_bounds(X.max(0), X.min(0), a1n, a2n)
+    s = (up - low) / (2 ** bits - 1)
+    z = np.rint(-low / s)
+    q, _ = orc.quant_uniform(X, s[None, :], z[None, :], bits)
+    assert np.allclose(loss, ((orc.dequant_uniform(q, s[None, :], z[None, :]) - X) ** 2).sum(0), rtol=1e-12)
+
+
+def test_dual_clip_follows_the_library_optimizer_and_lowers_the_objective():
+    X = _clip_case(seed=1)
+    D = X.shape[1]
+    a1 = torch.zeros(D, dtype=torch.float64, requires_grad=True)
+    a2 = torch.zeros(D, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.Adam([a1, a2], lr=0.01)
+    Xt = torch.from_numpy(X)
+    for _ in range(100):
+        opt.zero_grad()
+        _torch_dual_clip_loss(Xt, a1, a2, 4).sum().backward()
+        opt.step()
+    r = orc.dual_clip(X, 4, iters=100, lr=0.01, alpha0=0.0)
+    assert np.abs(r["alpha1"] - a1.detach().numpy()).max() < 1e-9
+    assert np.abs(r["alpha2"] - a2.detach().numpy()).max() < 1e-9
+    assert np.all(r["loss"] < r["loss0"])
+    up, low = orc.dual_clip_bounds(X.max(0), X.min(0), r["alpha1"], r["alpha2"])
+    assert np.array_equal(up, r["x_up"]) and np.array_equal(low, r["x_low"])
+    assert np.all(r["x_up"] <= X.max(0)) and np.all(r["x_low"] >= X.min(0))        # a contraction of the extremes
+    # zero iterations: the initial contraction itself
+    r0 = orc.dual_clip(X, 4, iters=0, alpha0=0.0)
+    assert np.allclose(r0["x_up"], 0.5 * X.max(0)) and np.allclose(r0["x_low"], 0.5 * X.min(0))
+
+
+def test_dual_clip_beats_the_percentile_stand_in_on_layernorm_activations():
+    """On the LayerNorm activations of a seeded calibration batch, the learned per-channel bounds give a smaller
+    objective (Eq. 20) than the 0.1 / 99.9 percentile bounds the workloads use in their place."""
+    from workloads.kernels import affine_params, channel_profile, ln_inputs, percentile_bounds
+    rng = np.random.default_rng(11)
+    D = 48
+    c, shift = channel_profile(rng, D, 1.0, 0.04, 20.0)
+    gamma, beta = affine_params(rng, D)
+    X1 = orc.layernorm(ln_inputs(rng, 1500, c, shift, False), gamma, beta, 1e-6)
+    lo, hi = percentile_bounds(X1, axis=0)
+    s, z = orc.uniform_scale_zero(lo, hi, 4)
+    q, _ = orc.quant_uniform(X1, s[None, :], z[None, :], 4)
+    err_pct = ((orc.dequant_uniform(q, s[None, :], z[None, :]) - X1) ** 2).sum()
+    r = orc.dual_clip(X1, 4, alpha0=2.0)            # start at 0.88 of the extremes
+    assert r["loss"].sum() < err_pct
+    assert r["loss"].sum() < r["loss0"].sum()

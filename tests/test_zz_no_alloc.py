@@ -36,12 +36,21 @@ def test_static_workspace_block_matches_regular_block_twice():
     ref2 = blk.forward(x2).cpu().numpy()
 
     d, p = blk.desc(2), blk.params()
-    for xin, expect in ((x, ref), (x2, ref2)):
-        y = torch.full_like(y_ref, float("nan"))
+    # one call first, so that the library's one-time work (module load, the look-up of its scratch array's
+    # address) is behind us; the two calls that are checked must then leave the device's free memory as it was,
+    # by the driver's own count (torch's allocator statistics would not see a cudaMalloc inside the library)
+    warm = torch.empty_like(y_ref)
+    B.repq_block_forward_static(d, p, x, warm)
+    torch.cuda.synchronize()
+    ys = [torch.full_like(y_ref, float("nan")) for _ in range(2)]
+    free_before = torch.cuda.mem_get_info()[0]
+    for (xin, expect), y in zip(((x, ref), (x2, ref2)), ys):
         before = torch.cuda.memory_allocated()
         B.repq_block_forward_static(d, p, xin, y)
         torch.cuda.synchronize()
         assert torch.cuda.memory_allocated() == before
+        assert torch.cuda.mem_get_info()[0] == free_before, "the call changed the device's free memory"
+        assert B.repq_device_status() == 0
         got = y.cpu().numpy()
         # same kernels, same inputs: the two entry points agree to the tolerance of the block tests
         rel = np.linalg.norm(got - expect) / np.linalg.norm(expect)
