@@ -11,9 +11,12 @@
 //                the main loop of tile i + 1
 //   warps 2..17  epilogue: warp w reads TMEM lanes 32 (w mod 4) .. +31 (one output row per thread) and a
 //                64-column slice of the accumulator columns
+//   warps 18..19 (packed 4-bit weights only) converters: the weight tile arrives packed, two codes per byte, and is
+//                expanded into the 128-byte-swizzled byte tile the MMA descriptor expects (there is no 4-bit integer
+//                MMA); one more barrier hop between the copy and the MMA, weights stay packed in HBM
 // The tile width BN (256, 192 or 128) is chosen per problem: rounds of tiles over the SMs times a per-round time
-// with a fixed part.  4-bit operands are expanded to one code per byte by a separate pass into the
-// workspace (there is no 4-bit integer MMA), so the main loop is the same for W4A4 and W8A8.
+// with a fixed part.  Packed 4-bit activations are expanded to one code per byte by a separate pass into the
+// workspace (inside the block the producers write byte codes, so that pass does not run there).
 //
 // For short K the epilogue, not the tensor pipe, sets the pace (K = 768: 3072 tensor-pipe cycles per
 // 128 x 256 tile against 32768 outputs), so it is written for few instructions per output and few waits per
@@ -43,6 +46,9 @@ constexpr int kChunk = 16;                           // accumulator columns per 
 constexpr int kEpiWarps = 16;
 constexpr int kEpiThreads = kEpiWarps * 32;
 constexpr int kThreads = 32 * (2 + kEpiWarps);
+constexpr int kConvWarps = 2;                        // converter warps of the packed-weight variant
+constexpr int kConvThreads = 32 * kConvWarps;
+constexpr int kThreadsW4 = kThreads + kConvThreads;  // 20 warps: five per scheduler, the same register budget as 18
 constexpr int kTmemCols = 512;
 constexpr int kAccStride = 256;                      // TMEM columns between the two accumulator buffers
 constexpr int kSliceCols = 64;                       // accumulator columns per epilogue warp
@@ -63,23 +69,28 @@ constexpr uint32_t kResBytes = 32 * 128;            // bf16 residual of one warp
 
 // RES: the bf16 residual of a tile comes in by bulk tensor copies, one 32 x 64 box per epilogue warp, asked for one
 // tile ahead (the operand ring gives up a stage for the boxes)
-template <int BN, bool RES>
+template <int BN, bool RES, bool W4>
 struct SharedStorage {
-  static constexpr int kStages = RES ? 3 : 4;
+  static constexpr int kStages = (RES || W4) ? 3 : 4;
   alignas(1024) uint8_t a[kStages][kABytes];
   alignas(1024) uint8_t b[kStages][BN * BK];
   alignas(1024) uint8_t res[RES ? kEpiWarps * kResBytes : 1024];
   uint64_t res_full[kEpiWarps];
   alignas(1024) uint8_t epi[kEpiWarps][1024];     // per-warp staging box of the epilogue's bulk stores
   ColTerms cols[kEpiWarps];                       // each epilogue warp stages the terms of its own slice: no barrier
+  alignas(128) uint8_t bp[W4 ? kStages : 1][W4 ? BN * BK / 2 : 128];   // packed weight tiles: rows of 64 bytes, unswizzled
   alignas(8) uint64_t full[kStages];
   uint64_t empty[kStages];
+  uint64_t ready[kStages];                          // weight tile expanded (packed variant)
   uint64_t tmem_full[2];
   uint64_t tmem_empty[2];
   uint64_t done;
   uint32_t tmem_base;
   volatile int abort;
 };
+
+static_assert(sizeof(SharedStorage<kMaxBN, false, false>) <= 227 * 1024 && sizeof(SharedStorage<kMaxBN, false, true>) <= 227 * 1024 &&
+              sizeof(SharedStorage<192, true, false>) <= 227 * 1024, "shared storage exceeds the 227 KB a CTA may use");
 
 using namespace tc;
 
@@ -100,6 +111,7 @@ struct TcParams {
   const int32_t* asum;
   const int32_t* wsum;
   int direct_requant;          // codes out, no GELU, no residual: 1/s_o is folded into the column terms
+  int w_packed4;               // weight tiles arrive packed (two codes per byte) and are expanded in shared memory
   EpilogueParams ep;
 };
 
@@ -323,11 +335,11 @@ __device__ __noinline__ void slow_chunk(const EpilogueParams& ep, const TcParams
 // where asked for: kPairNone, kPairRope (rotary embedding), kPairGlu (gated product; byte codes out)
 enum : int { kPairNone = 0, kPairRope = 1, kPairGlu = 2 };
 
-template <int BN, int OUT, bool RES, int PAIR>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int BN, int OUT, bool RES, int PAIR, bool W4>
+__global__ void __launch_bounds__(W4 ? kThreadsW4 : kThreads, 1)
 qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_res, TcParams P) {
-  using Storage = SharedStorage<BN, RES>;
+  using Storage = SharedStorage<BN, RES, W4>;
   constexpr int kStages = Storage::kStages;
   constexpr uint32_t kBBytes = BN * BK;
   constexpr uint32_t kIdesc = idesc_for(BN);
@@ -342,7 +354,11 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   const int kblocks = (P.K + BK - 1) / BK;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&S.full[s]), 1); mbar_init(smem_u32(&S.empty[s]), 1); }
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(smem_u32(&S.full[s]), 1);
+      mbar_init(smem_u32(&S.empty[s]), 1);
+      mbar_init(smem_u32(&S.ready[s]), kConvWarps);
+    }
     for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&S.tmem_full[a]), 1); mbar_init(smem_u32(&S.tmem_empty[a]), kEpiWarps); }
     for (int w = 0; w < kEpiWarps; ++w) mbar_init(smem_u32(&S.res_full[w]), 1);
     mbar_init(smem_u32(&S.done), 1);
@@ -376,9 +392,10 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!mbar_wait(smem_u32(&S.empty[stage]), phase ^ 1, abort, 1)) break;
           const uint32_t bar = smem_u32(&S.full[stage]);
-          mbar_expect_tx(bar, kABytes + kBBytes);
+          mbar_expect_tx(bar, kABytes + (W4 ? kBBytes / 2 : kBBytes));
           tma_load_2d(smem_u32(S.a[stage]), &map_a, bar, kb * BK, m0);
-          tma_load_2d(smem_u32(S.b[stage]), &map_b, bar, kb * BK, n0);
+          if constexpr (W4) tma_load_2d(smem_u32(S.bp[stage]), &map_b, bar, kb * (BK / 2), n0);
+          else tma_load_2d(smem_u32(S.b[stage]), &map_b, bar, kb * BK, n0);
           ++issued;
           if (++stage == kStages) { stage = 0; phase ^= 1; }
         }
@@ -404,7 +421,9 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         const uint32_t d_tmem = tmem_base + acc * kAccStride;
         bool ok = true;
         for (int kb = 0; kb < kblocks; ++kb) {
-          if (!mbar_wait(smem_u32(&S.full[stage]), phase, abort, 3)) { ok = false; break; }
+          // packed weights: the converters release the stage once the byte tile is written (they have waited for the
+          // copies themselves, so the activation tile has landed as well)
+          if (!mbar_wait(smem_u32(W4 ? &S.ready[stage] : &S.full[stage]), phase, abort, 3)) { ok = false; break; }
           tc_fence_after();
           const uint64_t da = smem_desc(smem_u32(S.a[stage])), db = smem_desc(smem_u32(S.b[stage]));
 #pragma unroll
@@ -420,6 +439,41 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       umma_commit(smem_u32(&S.done));
       const long long t0 = clock64();
       while (!mbar_try_wait(smem_u32(&S.done), 0) && clock64() - t0 < kWaitCycles) {}
+    }
+  } else if (W4 && warp >= 2 + kEpiWarps) {
+    // ---------------------------------------------------------------- converters (packed 4-bit weights)
+    // A packed tile holds BN rows of 64 bytes (128 codes, even index in the low nibble).  Thread ct takes 16-byte
+    // pieces ct, ct + 64, ...: piece g = (row g / 4, codes 32 (g % 4) ..) becomes the two 16-byte pieces 2 (g % 4) and
+    // 2 (g % 4) + 1 of the row's 128 bytes, stored where the 128-byte swizzle puts them.  Reads are consecutive
+    // across the warp; the stores of eight neighbouring threads cover two rows and all eight swizzled positions.
+    const int ct = int(threadIdx.x) - 32 * (2 + kEpiWarps);
+    uint32_t stage = 0, phase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < tiles && ok && !*abort; tile += gridDim.x) {
+      for (int kb = 0; kb < kblocks; ++kb) {
+        if (!mbar_wait(smem_u32(&S.full[stage]), phase, abort, 7)) { ok = false; break; }
+        const uint32_t src = smem_u32(S.bp[stage]), dst = smem_u32(S.b[stage]);
+#pragma unroll 4
+        for (int g = ct; g < BN * 4; g += kConvThreads) {
+          const int n = g >> 2, pp = g & 3;
+          uint32_t w[4];
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(src + uint32_t(g) * 16u));
+          uint32_t o[8];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const uint32_t lo = w[i] & 0x0F0F0F0Fu, hi = (w[i] >> 4) & 0x0F0F0F0Fu;
+            o[2 * i] = __byte_perm(lo, hi, 0x5140);
+            o[2 * i + 1] = __byte_perm(lo, hi, 0x7362);
+          }
+          const uint32_t row = dst + uint32_t(n >> 3) * 1024u + uint32_t(n & 7) * 128u;
+          sts128(row + (uint32_t((2 * pp) ^ (n & 7)) << 4), o[0], o[1], o[2], o[3]);
+          sts128(row + (uint32_t((2 * pp + 1) ^ (n & 7)) << 4), o[4], o[5], o[6], o[7]);
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&S.ready[stage]));
+        if (++stage == kStages) { stage = 0; phase ^= 1; }
+      }
     }
   } else {
     // ---------------------------------------------------------------- epilogue
@@ -655,16 +709,19 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 
 // ---- host side -------------------------------------------------------------------------------------
 
-repq_status make_map(CUtensorMap* map, const uint8_t* base, int64_t rows, int64_t K, int64_t ld, int box_rows) {
+// Operand tensor map: rows of `row_bytes` bytes, boxes of `box_bytes` x box_rows; byte tiles take the 128-byte swizzle
+// of the MMA descriptor, packed tiles (expanded by the converter warps) stay unswizzled.
+repq_status make_map(CUtensorMap* map, const uint8_t* base, int64_t rows, int64_t row_bytes, int64_t ld, int box_rows,
+                     int box_bytes = BK, bool swizzle = true) {
   EncodeTiledFn fn = encode_fn();
   REPQ_REQUIRE(fn != nullptr, REPQ_CUDA_ERROR, "qgemm: cuTensorMapEncodeTiled is not available");
-  const cuuint64_t dims[2] = {cuuint64_t(K), cuuint64_t(rows)};
+  const cuuint64_t dims[2] = {cuuint64_t(row_bytes), cuuint64_t(rows)};
   const cuuint64_t strides[1] = {cuuint64_t(ld)};
-  const cuuint32_t box[2] = {cuuint32_t(BK), cuuint32_t(box_rows)};
+  const cuuint32_t box[2] = {cuuint32_t(box_bytes), cuuint32_t(box_rows)};
   const cuuint32_t estr[2] = {1, 1};
   const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(base), dims, strides, box, estr,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   REPQ_REQUIRE(r == CUDA_SUCCESS, REPQ_CUDA_ERROR, "qgemm: cuTensorMapEncodeTiled failed with code %d", int(r));
   return REPQ_OK;
 }
@@ -681,7 +738,7 @@ TcLayout tc_layout(const repq_gemm_desc& d) {
   L.ld_a = round_up(d.K, 16);
   L.ld_w = round_up(d.K, 16);
   L.off_a = packed4(d.bits_a) ? bump(size_t(d.M) * L.ld_a) : 0;
-  L.off_w = packed4(d.bits_w) ? bump(size_t(d.N) * L.ld_w) : 0;
+  L.off_w = 0;                                  // packed weights are expanded inside the kernel
   L.off_asum = d.a_row_sum ? 0 : bump(size_t(d.M) * 4);
   L.off_wsum = d.w_row_sum ? 0 : bump(size_t(d.N) * 4);
   L.total = cur;
@@ -739,19 +796,27 @@ repq_status make_res_map(CUtensorMap* map, const TcParams& P) {
   return REPQ_OK;
 }
 
-template <int BN, int OUT, bool RES, int PAIR = kPairNone>
-repq_status launch_tc_res(const CUtensorMap& map_a, const CUtensorMap& map_b, const TcParams& P, int sms, cudaStream_t st) {
+template <int BN, int OUT, bool RES, int PAIR, bool W4>
+repq_status launch_tc_w(const CUtensorMap& map_a, const CUtensorMap& map_b, const TcParams& P, int sms, cudaStream_t st) {
   CUtensorMap map_out, map_res;
   REPQ_TRY(make_out_map(&map_out, P));
   if (RES) REPQ_TRY(make_res_map(&map_res, P));
   else map_res = map_out;                                  // not read
-  const size_t smem = sizeof(SharedStorage<BN, RES>);
-  REPQ_CUDA(cudaFuncSetAttribute(qgemm_tc_kernel<BN, OUT, RES, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+  const size_t smem = sizeof(SharedStorage<BN, RES, W4>);
+  REPQ_CUDA(cudaFuncSetAttribute(qgemm_tc_kernel<BN, OUT, RES, PAIR, W4>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
   const int tiles = ((P.M + BM - 1) / BM) * ((P.N + BN - 1) / BN);
   const int grid = tiles < sms ? tiles : sms;
-  REPQ_CUDA(launch_chained(qgemm_tc_kernel<BN, OUT, RES, PAIR>, dim3(grid), dim3(kThreads), smem, st, map_a, map_b, map_out, map_res, P));
+  REPQ_CUDA(launch_chained(qgemm_tc_kernel<BN, OUT, RES, PAIR, W4>, dim3(grid), dim3(W4 ? kThreadsW4 : kThreads), smem, st, map_a, map_b, map_out, map_res, P));
   note_launch();
   return REPQ_OK;
+}
+
+template <int BN, int OUT, bool RES, int PAIR = kPairNone>
+repq_status launch_tc_res(const CUtensorMap& map_a, const CUtensorMap& map_b, const TcParams& P, int sms, cudaStream_t st) {
+  if constexpr (!RES) {
+    if (P.w_packed4) return launch_tc_w<BN, OUT, false, PAIR, true>(map_a, map_b, P, sms, st);
+  }
+  return launch_tc_w<BN, OUT, RES, PAIR, false>(map_a, map_b, P, sms, st);
 }
 
 template <int BN, int OUT>
@@ -760,7 +825,7 @@ repq_status launch_tc_out(const CUtensorMap& map_a, const CUtensorMap& map_b, co
   // Taken for short K, where the epilogue sets the pace (measured at 12608 x 768: K = 768 24 us against 27 us with
   // row-per-lane residual loads; K = 3072 46 us against 39 us, the main loop missing its fourth stage).
   if constexpr (BN <= 192 && (OUT == kOutF32 || OUT == kOutBf16)) {
-    if (P.ep.residual != nullptr && P.ep.residual_bf16 && P.ep.acc_debug == nullptr && P.K <= 1536)
+    if (P.ep.residual != nullptr && P.ep.residual_bf16 && P.ep.acc_debug == nullptr && P.K <= 1536 && !P.w_packed4)
       return launch_tc_res<BN, OUT, true>(map_a, map_b, P, sms, st);
   }
   return launch_tc_res<BN, OUT, false>(map_a, map_b, P, sms, st);
@@ -818,7 +883,7 @@ bool qgemm_tc_supported(const repq_gemm_desc& d) {
   if (d.batch_outer != 1 || d.batch_inner != 1) return false;
   if (d.M < 64 || d.N < 64 || d.K < 64) return false;           // tiny problems: the warp-MMA kernel
   if (!packed4(d.bits_a) && !(aligned(d.a_codes, 16) && d.lda_bytes % 16 == 0)) return false;
-  if (!packed4(d.bits_w) && !(aligned(d.w_codes, 16) && d.ldw_bytes % 16 == 0)) return false;
+  if (!(aligned(d.w_codes, 16) && d.ldw_bytes % 16 == 0)) return false;      // byte or packed: the tiles come by TMA
   const int64_t obytes = d.out_kind == REPQ_OUT_F32 ? 4 : d.out_kind == REPQ_OUT_BF16 ? 2 : 1;
   if (!aligned(d.out, 16) || (d.ldo * obytes) % 16 != 0) return false;
   if (d.out_kind == REPQ_OUT_CODES && (d.N / d.out_groups) % kChunk != 0) return false;   // one quantizer per 16-column chunk
@@ -842,13 +907,8 @@ repq_status qgemm_tc(const repq_gemm_desc& d, const EpilogueParams& ep, void* ws
     REPQ_TRY(launch_expand4(d.a_codes, d.M, d.K, d.lda_bytes, w8 + L.off_a, L.ld_a, L.ld_a, st));
     a = w8 + L.off_a; lda = L.ld_a;
   }
-  const uint8_t* w = d.w_codes;
-  int64_t ldw = d.ldw_bytes;
-  if (packed4(d.bits_w)) {
-    REPQ_TRY(launch_expand4(d.w_codes, d.N, d.K, d.ldw_bytes, w8 + L.off_w, L.ld_w, L.ld_w, st));
-    w = w8 + L.off_w; ldw = L.ld_w;
-  }
   TcParams P{};
+  P.w_packed4 = packed4(d.bits_w);
   P.M = d.M; P.N = d.N; P.K = d.K;
   P.asum = d.a_row_sum;
   if (!P.asum) {
@@ -869,7 +929,8 @@ repq_status qgemm_tc(const repq_gemm_desc& d, const EpilogueParams& ep, void* ws
   const int bn = pick_bn(d.M, d.N, sms);
   CUtensorMap map_a, map_b;
   REPQ_TRY(make_map(&map_a, a, d.M, d.K, lda, BM));
-  REPQ_TRY(make_map(&map_b, w, d.N, d.K, ldw, bn));
+  if (P.w_packed4) REPQ_TRY(make_map(&map_b, d.w_codes, d.N, (int64_t(d.K) + 1) / 2, d.ldw_bytes, bn, BK / 2, false));
+  else REPQ_TRY(make_map(&map_b, d.w_codes, d.N, d.K, d.ldw_bytes, bn));
   if (bn == 256) return launch_tc<256>(map_a, map_b, P, sms, st);
   if (bn == 192) return launch_tc<192>(map_a, map_b, P, sms, st);
   return launch_tc<128>(map_a, map_b, P, sms, st);

@@ -41,15 +41,19 @@ def _pack_linear(W: np.ndarray, bias: np.ndarray, bits_w: int, dev) -> PreparedL
 class QuantBlock:
     """Device-resident parameters of one block plus its workspace; `forward` runs the hot path."""
 
-    def __init__(self, w, device="cuda:0", out_dtype: Optional[torch.dtype] = None, staged_attention: bool = False):
+    def __init__(self, w, device="cuda:0", out_dtype: Optional[torch.dtype] = None, staged_attention: bool = False,
+                 weight_storage: str = "packed"):
+        """weight_storage: "packed" keeps 4-bit weight codes two per byte in device memory (the GEMM expands the
+        tiles in shared memory); "bytes" keeps one code per byte, the tensor-core operand format."""
+        assert weight_storage in ("packed", "bytes")
+        self.weight_storage = weight_storage
         self.staged_attention = bool(staged_attention)
         cfg = w.cfg
         self.cfg = cfg
         dev = torch.device(device)
         self.device = dev
         ba = cfg["bits_a"]
-        # weights live on the device one code per byte: the tensor-core operand format, so no per-call expansion
-        bw = self.bits_w = cfg["bits_w"] | B.REPQ_BYTE_CODES
+        bw = self.bits_w = cfg["bits_w"] if weight_storage == "packed" else cfg["bits_w"] | B.REPQ_BYTE_CODES
         self.host: Dict[str, object] = {}
 
         def fold(gamma, beta, lo, hi, W, b, tag):
