@@ -217,7 +217,7 @@ def measure_block(name, batch, args, dev, rank, world, peaks, headline, sampler=
     r0, r1 = shard_rows(world, rank, batch, L)
     w = dataclasses.replace(w, cfg=cfg, x=w.x[r0:r1])
     tokens_per_step = batch * L
-    blk = QuantBlock(w, device=dev, staged_attention=args.staged_attention)
+    blk = QuantBlock(w, device=dev, staged_attention=args.staged_attention, weight_storage=args.weights)
     x_host = torch.from_numpy(np.ascontiguousarray(w.x)).to(blk.act_dtype).pin_memory()
     x = x_host.to(dev, non_blocking=True)
     y = torch.empty_like(x, dtype=blk.out_dtype)
@@ -291,7 +291,8 @@ def measure_block(name, batch, args, dev, rank, world, peaks, headline, sampler=
                e2e=dict(value=world * tokens_per_step * steps / (ms_e2e * 1e-3), unit=UNIT,
                         h2d_bytes_per_step=x_host.numel() * x_host.element_size(),
                         d2h_bytes_per_step=y_hosts[0].numel() * y_hosts[0].element_size()),
-               stages=stages, gpu_launches=int(launches), clocks=clocks, cfg=cfg)
+               stages=stages, gpu_launches=int(launches), clocks=clocks, cfg=cfg,
+               weight_bytes=int(sum(l.codes.numel() for l in (blk.qkv, blk.proj, blk.fc1, blk.fc2))))
     if headline:
         rec["_blk"], rec["_x"], rec["_y"] = blk, x, y
     return rec
@@ -485,6 +486,8 @@ def main():
     ap.add_argument("--sweep-only", default=None, choices=["ln", "softmax", "gemm"],
                     help="run only the single-kernel sweep points of this kernel and print them (profiling aid)")
     ap.add_argument("--sweep-dim", type=int, default=None, help="with --sweep-only: only this D (ln), L (softmax) or N (gemm)")
+    ap.add_argument("--weights", default="bytes", choices=["packed", "bytes"],
+                    help="4-bit weight codes in device memory: two per byte (expanded in shared memory by the GEMM) or one per byte")
     ap.add_argument("--staged-attention", action="store_true",
                     help="run scores, Softmax codes and P.V as three kernels instead of the fused attention kernel")
     args = ap.parse_args()
@@ -576,7 +579,8 @@ def main():
                     dtype="u8" if cfg["bits_a"] != 4 else "u4/u8->s32", data="synthetic",
                     config=dict(workload=cfg["name"], batch_per_gpu=batch, seq=cfg["L"], dim=cfg["D"], heads=cfg["H"],
                                 mlp=cfg["MLP"], bits="W%dA%d" % (cfg["bits_w"], cfg["bits_a"]), bits_p=cfg["bits_p"],
-                                act=cfg["act"], causal=bool(cfg["causal"]), parallelism="batch-sharded replicas x%d" % world,
+                                act=cfg["act"], causal=bool(cfg["causal"]), weights=args.weights,
+                                weight_code_bytes=head["weight_bytes"], parallelism="batch-sharded replicas x%d" % world,
                                 l2="256 MiB written between timed steps",
                                 stage_times="CUDA events between the stages: kernels serialised, so their sum exceeds ms_per_step"),
                     clocks=head["clocks"], gpu_launches=head["gpu_launches"], e2e=head["e2e"], roofline=roof, stages=stages,

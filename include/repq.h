@@ -93,6 +93,13 @@ repq_status repq_fold_ln(int D, int N, const float* gamma, const float* beta, co
 repq_status repq_pack_weights(int N, int K, int bits_w, const float* W, uint8_t* codes,
                               int64_t ld_codes_bytes, float* s_w, int32_t* z_w, int32_t* w_row_sum);
 
+/* Full-precision normalisation (Eq. 9; REPQ_NORM_RMS: the mean-free variant) of a calibration batch, float32 out:
+ * the activations X' that repq_dual_clip learns its clipping factors on.  Calibration-time only; the inference
+ * path (repq_ln_quant) never forms X'.  x [device]: rows x D, REPQ_F32 or REPQ_BF16, row stride ldx elements;
+ * gamma, beta [device] float[D] (the un-reparameterized affine factors); y [device]: rows x D float32, row stride ldy. */
+repq_status repq_layernorm(const void* x, int x_dtype, int64_t rows, int D, int64_t ldx, const float* gamma,
+                           const float* beta, float eps, int norm_kind, float* y, int64_t ldy, void* stream);
+
 /* Per-channel dual clipping (Sec. III-D, Eqs. 18-20): the clipping bounds of the channel-wise quantizer of a
  * LayerNorm activation, learned on a calibration batch just before the scale reparameterization
  * (repq_scale_zero_from_bounds -> repq_fold_ln take them from here).  For every channel d

@@ -376,7 +376,14 @@ def attention(Qc, Kc, Vc, qp: dict, B: int, L: int, H: int, softmax_s: float, bi
     return O, kept
 
 
-def block_forward(w, keep: bool = False) -> Dict[str, np.ndarray]:
+def percentile_bounds(v, lo_pct: float = 0.1, hi_pct: float = 99.9):
+    """Percentile calibration of a layer-wise quantizer (Sec. IV-A names the strategy, not the percentiles; the
+    workloads fix 0.1 / 99.9): the bounds handed to Eq. 6, rounded to float32 as they are stored."""
+    lo, hi = np.percentile(np.asarray(v, dtype=F64), [lo_pct, hi_pct])
+    return np.float32(lo), np.float32(hi)
+
+
+def block_forward(w, keep: bool = False, calibrate: Optional[dict] = None) -> Dict[str, np.ndarray]:
     """Eqs. 1-2 with every matrix-multiplication input quantized (Sec. III-A.1, IV-A):
     X_bar = MSA(LN(X)) + X,  Y = MLP(LN(X_bar)) + X_bar.
 
@@ -394,6 +401,13 @@ def block_forward(w, keep: bool = False) -> Dict[str, np.ndarray]:
     embedding is applied to the full-precision Q and K of the projection before their quantizers, and the MLP is
     down(SiLU(gate(.)) * up(.)) with `w_fc1` = [gate; up] stacked on the output axis, the product being the
     quantized input of the down projection `w_fc2`.
+
+    `calibrate` (a dict, possibly empty) turns the pass into the sequential pipeline of Algorithm 1 on a
+    calibration batch `w.x`, with round-to-nearest in GPTQ's place: every quantizer's bounds are found on the input
+    that reaches it through the layers already quantized (Algorithm 1 collects each layer's input in one
+    traversal) instead of being taken from `w`: per-channel dual clipping (Eqs. 18-20; keys `alpha0`, `iters`,
+    `lr`) for the two LayerNorm activations, percentile calibration (keys `lo_pct`, `hi_pct`) for the layer-wise
+    quantizers.  The bounds found are returned under "bounds", "ln1_lo", "ln1_hi", "ln2_lo", "ln2_hi".
     """
     cfg = w.cfg
     B, L, D, H = cfg["B"], cfg["L"], cfg["D"], cfg["H"]
@@ -402,9 +416,17 @@ def block_forward(w, keep: bool = False) -> Dict[str, np.ndarray]:
     x = np.asarray(w.x, dtype=F64)
 
     llama = cfg.get("arch", "vit") == "llama"
+    cal = calibrate
+    found: Dict[str, tuple] = {}
 
     def post_ln_linear(X_in, gamma, beta, lo, hi, W, b, tag):
         X1 = layernorm(X_in, gamma, beta, cfg["eps"], rms=llama)
+        if cal is not None:
+            # the activations as the calibration tool holds them (float32), then Eqs. 18-20
+            X1_32 = X1.astype(np.float32).astype(F64)
+            r = dual_clip(X1_32, ba, iters=cal.get("iters", 100), lr=cal.get("lr", 0.01), alpha0=cal.get("alpha0", 0.0))
+            lo, hi = r["x_low"].astype(np.float32), r["x_up"].astype(np.float32)
+            out[tag + "_lo"], out[tag + "_hi"] = lo, hi
         s, z = uniform_scale_zero(lo, hi, ba)
         q, t = quant_uniform(X1, s[None, :], z[None, :], ba)            # channel-wise
         rp = reparam_layernorm(gamma, beta, s, z, W, b)
@@ -419,7 +441,11 @@ def block_forward(w, keep: bool = False) -> Dict[str, np.ndarray]:
         return y
 
     def requant(v, name):
-        lo, hi = w.bounds[name]
+        if cal is not None:
+            found[name] = percentile_bounds(v, cal.get("lo_pct", 0.1), cal.get("hi_pct", 99.9))
+            lo, hi = found[name]
+        else:
+            lo, hi = w.bounds[name]
         s, z = uniform_scale_zero(lo, hi, ba)
         q, t = quant_uniform(v, s, z, ba)
         if keep:
@@ -456,4 +482,6 @@ def block_forward(w, keep: bool = False) -> Dict[str, np.ndarray]:
     hc, s_h, z_h = requant(h_act, "hidden")
     wc, s_w, z_w = quant_weight_rtn(w.w_fc2, bw)
     out["y"] = linear(dequant_uniform(hc, s_h, z_h), wc, s_w, z_w, w.b_fc2) + x_bar
+    if cal is not None:
+        out["bounds"] = found
     return out

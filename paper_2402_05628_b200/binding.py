@@ -29,7 +29,7 @@ EXPORTS = (
     "repq_softmax_log2", "repq_pv", "repq_block_workspace_bytes", "repq_block_forward",
     "repq_device_status", "repq_block_forward_timed", "repq_launch_count",
     "repq_block_forward_static", "repq_attention", "repq_block_forward_host", "repq_rope_table",
-    "repq_bounded_wait_selftest", "repq_dual_clip",
+    "repq_bounded_wait_selftest", "repq_dual_clip", "repq_layernorm",
 )
 REPQ_MLP_GELU, REPQ_MLP_SWIGLU = 0, 1
 REPQ_STATIC_WORKSPACE_BYTES = 8 << 20
@@ -163,6 +163,8 @@ def lib() -> C.CDLL:
         _lib.repq_pack_weights.argtypes = [C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_int64,
                                            C.c_void_p, C.c_void_p, C.c_void_p]
         _lib.repq_rope_table.argtypes = [C.c_int, C.c_int, C.c_double, C.c_void_p]
+        _lib.repq_layernorm.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int, C.c_int64, C.c_void_p, C.c_void_p, C.c_float,
+                                        C.c_int, C.c_void_p, C.c_int64, C.c_void_p]
         _lib.repq_dual_clip.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_int64, C.c_int, C.c_int, C.c_float, C.c_float,
                                         C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         _lib.repq_bounded_wait_selftest.argtypes = [C.c_int64, C.c_void_p]
@@ -355,6 +357,14 @@ def repq_device_status(reset: bool = False) -> int:
 
 def repq_bounded_wait_selftest(limit_cycles: int, stream=None) -> None:
     _check(lib().repq_bounded_wait_selftest(int(limit_cycles), _stream(stream)))
+
+
+def repq_layernorm(x: torch.Tensor, gamma: torch.Tensor, beta: torch.Tensor, eps: float, y: torch.Tensor,
+                   norm_kind: int = REPQ_NORM_LAYERNORM, stream=None) -> None:
+    """Full-precision normalisation of a calibration batch (float32 out), the input of repq_dual_clip."""
+    rows, D = x.shape
+    _check(lib().repq_layernorm(_ptr(x), _dtype_code(x), rows, D, x.stride(0), _ptr(gamma), _ptr(beta), eps, norm_kind,
+                                _ptr(y), y.stride(0), _stream(stream)))
 
 
 def repq_dual_clip(x: torch.Tensor, bits: int, x_low: torch.Tensor, x_up: torch.Tensor, loss: Optional[torch.Tensor] = None,

@@ -13,6 +13,8 @@
 // the activations (L2-resident for calibration-sized inputs), a shared-memory reduction of three sums per channel,
 // and the Adam update by the channel's first thread.  Arithmetic is float64 throughout (the decisions of the two
 // round operations steer the gradient).  No scratch memory, no atomics, no inter-CTA traffic.
+#include <cuda_bf16.h>
+
 #include <cmath>
 
 #include "common.h"
@@ -128,10 +130,74 @@ __global__ void __launch_bounds__(kThreads) dual_clip_kernel(ClipParams P) {
   }
 }
 
+// Full-precision normalisation of the calibration batch (Eq. 9; mean-free variant for RMS): the activations the
+// clipping factors are learned on.  One CTA per row at a time, mean and centred variance in float32 with a
+// float64 block reduction, float32 output.  Calibration-time only: the inference path never forms X'.
+template <typename T>
+__global__ void __launch_bounds__(256) layernorm_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
+                                                        const float* __restrict__ gamma, const float* __restrict__ beta,
+                                                        float eps, int rms, float* __restrict__ y, int64_t ldy) {
+  __shared__ double red[8];
+  __shared__ float bc;
+  auto block_sum = [&](double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    __syncthreads();                               // the previous use of red / bc is over
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      double t = 0.0;
+      for (int i = 0; i < 8; ++i) t += red[i];
+      bc = float(t / double(D));
+    }
+    __syncthreads();
+    return bc;
+  };
+  auto ld = [](const T* p) {
+    if constexpr (sizeof(T) == 2) return __bfloat162float(*p);
+    else return float(*p);
+  };
+  for (int64_t r = blockIdx.x; r < rows; r += gridDim.x) {
+    const T* xr = x + r * ldx;
+    double acc = 0.0;
+    if (!rms)
+      for (int c = threadIdx.x; c < D; c += 256) acc += double(ld(xr + c));
+    const float mu = rms ? 0.f : block_sum(acc);
+    acc = 0.0;
+    for (int c = threadIdx.x; c < D; c += 256) {
+      const float dlt = ld(xr + c) - mu;
+      acc += double(dlt) * double(dlt);
+    }
+    const float rstd = rsqrtf(block_sum(acc) + eps);
+    for (int c = threadIdx.x; c < D; c += 256)
+      y[r * ldy + c] = fmaf((ld(xr + c) - mu) * rstd, __ldg(gamma + c), __ldg(beta + c));
+  }
+}
+
 }  // namespace
 }  // namespace repq
 
 using namespace repq;
+
+extern "C" repq_status repq_layernorm(const void* x, int x_dtype, int64_t rows, int D, int64_t ldx, const float* gamma,
+                                      const float* beta, float eps, int norm_kind, float* y, int64_t ldy, void* stream) {
+  REPQ_REQUIRE(rows >= 0 && D > 0 && ldx >= D && ldy >= D, REPQ_INVALID_ARG, "layernorm: bad sizes");
+  if (rows == 0) return REPQ_OK;
+  REPQ_REQUIRE(x && gamma && beta && y, REPQ_INVALID_ARG, "layernorm: NULL pointer");
+  REPQ_REQUIRE(x_dtype == REPQ_F32 || x_dtype == REPQ_BF16, REPQ_INVALID_ARG, "layernorm: x_dtype must be REPQ_F32 or REPQ_BF16");
+  REPQ_REQUIRE(norm_kind == REPQ_NORM_LAYERNORM || norm_kind == REPQ_NORM_RMS, REPQ_INVALID_ARG, "layernorm: unknown norm_kind");
+  REPQ_REQUIRE(eps >= 0.f, REPQ_INVALID_ARG, "layernorm: eps must be non-negative");
+  const int grid = int(rows < 4096 ? rows : 4096);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int rms = norm_kind == REPQ_NORM_RMS;
+  if (x_dtype == REPQ_F32)
+    layernorm_kernel<float><<<grid, 256, 0, st>>>(static_cast<const float*>(x), rows, D, ldx, gamma, beta, eps, rms, y, ldy);
+  else
+    layernorm_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(x), rows, D, ldx, gamma, beta, eps, rms, y, ldy);
+  REPQ_CUDA(cudaGetLastError());
+  note_launch();
+  return REPQ_OK;
+}
 
 extern "C" repq_status repq_dual_clip(const float* x, int64_t n, int D, int64_t ldx, int bits, int iters, float lr,
                                       float alpha0, float* x_low, float* x_up, double* loss, void* stream) {

@@ -452,22 +452,34 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     for (int tile = blockIdx.x; tile < tiles && ok && !*abort; tile += gridDim.x) {
       for (int kb = 0; kb < kblocks; ++kb) {
         if (!mbar_wait(smem_u32(&S.full[stage]), phase, abort, 7)) { ok = false; break; }
-        const uint32_t src = smem_u32(S.bp[stage]), dst = smem_u32(S.b[stage]);
-#pragma unroll 4
-        for (int g = ct; g < BN * 4; g += kConvThreads) {
-          const int n = g >> 2, pp = g & 3;
-          uint32_t w[4];
-          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(src + uint32_t(g) * 16u));
-          uint32_t o[8];
+        // pieces ct, ct + 64, ...: the row advances by 16 per step, so the row's position inside its group of eight
+        // (hence the swizzle) is the thread's own; four pieces are loaded before any is expanded, so that the loads
+        // of a batch overlap the arithmetic of the one before
+        const uint4* src = reinterpret_cast<const uint4*>(S.bp[stage]) + ct;
+        const int n_lo = (ct >> 2) & 7, pp = ct & 3;
+        uint8_t* row = S.b[stage] + uint32_t(ct >> 5) * 1024u + uint32_t(n_lo) * 128u;
+        uint8_t* d0 = row + (uint32_t((2 * pp) ^ n_lo) << 4);
+        uint8_t* d1 = row + (uint32_t((2 * pp + 1) ^ n_lo) << 4);
+        constexpr int kBatch = 4, kSteps = BN * 4 / kConvThreads;          // 16-row steps per thread
+        static_assert(kSteps % kBatch == 0, "converter batches must divide the tile");
+#pragma unroll 1
+        for (int i0 = 0; i0 < kSteps; i0 += kBatch) {
+          uint4 w[kBatch];
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const uint32_t lo = w[i] & 0x0F0F0F0Fu, hi = (w[i] >> 4) & 0x0F0F0F0Fu;
-            o[2 * i] = __byte_perm(lo, hi, 0x5140);
-            o[2 * i + 1] = __byte_perm(lo, hi, 0x7362);
+          for (int u = 0; u < kBatch; ++u) w[u] = src[(i0 + u) * kConvThreads];
+#pragma unroll
+          for (int u = 0; u < kBatch; ++u) {
+            const uint32_t in[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
+            uint32_t o[8];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const uint32_t lo = in[i] & 0x0F0F0F0Fu, hi = (in[i] >> 4) & 0x0F0F0F0Fu;
+              o[2 * i] = __byte_perm(lo, hi, 0x5140);
+              o[2 * i + 1] = __byte_perm(lo, hi, 0x7362);
+            }
+            *reinterpret_cast<uint4*>(d0 + (i0 + u) * 2048) = make_uint4(o[0], o[1], o[2], o[3]);
+            *reinterpret_cast<uint4*>(d1 + (i0 + u) * 2048) = make_uint4(o[4], o[5], o[6], o[7]);
           }
-          const uint32_t row = dst + uint32_t(n >> 3) * 1024u + uint32_t(n & 7) * 128u;
-          sts128(row + (uint32_t((2 * pp) ^ (n & 7)) << 4), o[0], o[1], o[2], o[3]);
-          sts128(row + (uint32_t((2 * pp + 1) ^ (n & 7)) << 4), o[4], o[5], o[6], o[7]);
         }
         fence_async_smem();
         __syncwarp();

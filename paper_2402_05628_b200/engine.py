@@ -42,7 +42,7 @@ class QuantBlock:
     """Device-resident parameters of one block plus its workspace; `forward` runs the hot path."""
 
     def __init__(self, w, device="cuda:0", out_dtype: Optional[torch.dtype] = None, staged_attention: bool = False,
-                 weight_storage: str = "packed"):
+                 weight_storage: str = "bytes"):
         """weight_storage: "packed" keeps 4-bit weight codes two per byte in device memory (the GEMM expands the
         tiles in shared memory); "bytes" keeps one code per byte, the tensor-core operand format."""
         assert weight_storage in ("packed", "bytes")
@@ -164,3 +164,125 @@ class QuantBlock:
         """Same pass with per-stage CUDA-event timing (synchronises); returns milliseconds per stage."""
         batch = x.shape[0] // self.cfg["L"]
         return B.repq_block_forward_timed(self.desc(batch), self.params(), x, y, self.workspace(batch), stream)
+
+
+def _percentile(t: torch.Tensor, pct: float) -> float:
+    """Percentile with linear interpolation between order statistics (a sort: library call, host-side calibration)."""
+    v, _ = torch.sort(t.reshape(-1).float())
+    pos = (v.numel() - 1) * pct / 100.0
+    i = int(pos)
+    frac = pos - i
+    lo = float(v[i])
+    hi = float(v[min(i + 1, v.numel() - 1)])
+    return lo + (hi - lo) * frac
+
+
+def calibrate_block(w, device="cuda:0", alpha0: float = 0.0, iters: int = 100, lr: float = 0.01,
+                    lo_pct: float = 0.1, hi_pct: float = 99.9):
+    """Sequential pipeline of Algorithm 1 for one block on the calibration batch `w.x`, round-to-nearest weight
+    quantization in GPTQ's place: every quantizer's bounds are found on the input that reaches it through the layers
+    already quantized.  LayerNorm activations: full-precision normalisation (repq_layernorm), per-channel dual
+    clipping (repq_dual_clip, Eqs. 18-20), scale reparameterization (repq_fold_ln).  Every other activation:
+    percentile calibration on the float32 output of the quantized layer before it (repq_qgemm / repq_attention with
+    float outputs).  Returns a copy of `w` whose clipping bounds are the calibrated ones; `QuantBlock` of that copy
+    is the calibrated block.  This function only sequences library calls and sorts for the percentiles."""
+    import dataclasses
+    cfg = w.cfg
+    dev = torch.device(device)
+    L, D, H, MLP = cfg["L"], cfg["D"], cfg["H"], cfg["MLP"]
+    dh = D // H
+    ba = cfg["bits_a"]
+    ab = ba | B.REPQ_BYTE_CODES
+    bw = cfg["bits_w"]
+    llama = cfg.get("arch", "vit") == "llama"
+    norm_kind = B.REPQ_NORM_RMS if llama else B.REPQ_NORM_LAYERNORM
+    act_dtype = torch.float32 if cfg["act"] == "f32" else torch.bfloat16
+    x = torch.from_numpy(np.ascontiguousarray(w.x)).to(dev).to(act_dtype)
+    M = x.shape[0]
+    batch = M // L
+    t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+    bounds = {}
+
+    def quantizer(name, values):
+        lo, hi = np.float32(_percentile(values, lo_pct)), np.float32(_percentile(values, hi_pct))
+        bounds[name] = (lo, hi)
+        s, z = B.repq_scale_zero_from_bounds(lo, hi, ba)
+        return float(s[0]), int(z[0])
+
+    def after_norm(x_in, gamma, beta, W, b):
+        """Dual clipping on the normalised calibration batch, fold, pack, and the LayerNorm codes of the batch."""
+        X1 = torch.empty(M, D, dtype=torch.float32, device=dev)
+        B.repq_layernorm(x_in, t(gamma), t(beta), cfg["eps"], X1, norm_kind)
+        lo, hi = torch.empty(D, device=dev), torch.empty(D, device=dev)
+        B.repq_dual_clip(X1, ba, lo, hi, None, iters=iters, lr=lr, alpha0=alpha0)
+        lo, hi = lo.cpu().numpy(), hi.cpu().numpy()
+        s, z = B.repq_scale_zero_from_bounds(lo, hi, ba)
+        g_t, b_t, s_t, z_t, W_t, bias_t = B.repq_fold_ln(gamma, beta, s, z, W, b)
+        lin = _pack_linear(W_t, bias_t, bw, dev)
+        codes = torch.empty(M, D, dtype=torch.uint8, device=dev)
+        rs = torch.empty(M, dtype=torch.int32, device=dev)
+        B.repq_ln_quant(x_in, t(g_t), t(b_t), cfg["eps"], s_t, z_t, ab, codes, rs, norm_kind)
+        return lo, hi, lin, codes, rs, s_t, z_t
+
+    def gemm(a, s_a, z_a, asum, lin, N, K, out, **kw):
+        d = B.gemm_desc(M, N, K, a, ab, s_a, z_a, lin.codes, bw, out, s_w=lin.s_w, z_w=lin.z_w, w_row_sum=lin.w_row_sum,
+                        bias=lin.bias, a_row_sum=asum, **kw)
+        ws = torch.empty(max(B.repq_qgemm_workspace_bytes(d), 16), dtype=torch.uint8, device=dev)
+        B.repq_qgemm(d, ws)
+        torch.cuda.synchronize()
+
+    # ---- LayerNorm 1 -> QKV
+    ln1_lo, ln1_hi, qkv, c1, rs1, s1, z1 = after_norm(x, w.ln1_gamma, w.ln1_beta, w.w_qkv, w.b_qkv)
+    rope = None
+    kw = {}
+    if llama:
+        rope = t(B.repq_rope_table(L, dh, cfg.get("rope_base", 10000.0)))
+        kw = dict(rope=rope, rope_period=L, rope_dim=dh, rope_groups=2)
+    qkv_f = torch.empty(M, 3 * D, dtype=torch.float32, device=dev)
+    gemm(c1, s1, z1, rs1, qkv, 3 * D, D, qkv_f, out_scale=[1.0] * 3, out_zero=[0] * 3, **kw)
+    quant = [quantizer(n, qkv_f[:, i * D:(i + 1) * D]) for i, n in enumerate(("q", "k", "v"))]
+    qkv_c = torch.empty(M, 3 * D, dtype=torch.uint8, device=dev)
+    gemm(c1, s1, z1, rs1, qkv, 3 * D, D, qkv_c, out_kind=B.REPQ_OUT_CODES, out_bits=ab, out_scale=[q[0] for q in quant],
+         out_zero=[q[1] for q in quant], **kw)
+    del qkv_f
+
+    # ---- attention (float output for the calibration of its quantizer, then codes)
+    a = B.AttentionDesc()
+    a.batch_outer, a.batch_inner, a.Lq, a.Lk, a.d_h, a.bits_qkv = batch, H, L, L, dh, ab
+    for i, n in enumerate("qkv"):
+        setattr(a, n + "_codes", qkv_c.data_ptr() + i * D)
+        setattr(a, "ld%s_bytes" % n, 3 * D)
+        setattr(a, n + "_stride_outer", L * 3 * D)
+        setattr(a, n + "_stride_inner", dh)
+        setattr(a, "s_" + n, quant[i][0])
+        setattr(a, "z_" + n, quant[i][1])
+    a.alpha, a.causal, a.bits_p, a.s_p = 1.0 / float(np.sqrt(dh)), int(cfg["causal"]), cfg["bits_p"], float(w.softmax_scale)
+    o_f = torch.empty(M, D, dtype=torch.float32, device=dev)
+    a.out_kind, a.out, a.ldo, a.o_stride_outer, a.o_stride_inner = B.REPQ_OUT_F32, o_f.data_ptr(), D, L * D, dh
+    B.repq_attention(a)
+    torch.cuda.synchronize()
+    s_at, z_at = quantizer("attn", o_f)
+    o_c = torch.empty(M, D, dtype=torch.uint8, device=dev)
+    rs_o = torch.zeros(M, dtype=torch.int32, device=dev)
+    a.out_kind, a.out_bits, a.out_scale, a.out_zero = B.REPQ_OUT_CODES, ab, s_at, z_at
+    a.out, a.out_row_sum = o_c.data_ptr(), rs_o.data_ptr()
+    B.repq_attention(a)
+    torch.cuda.synchronize()
+
+    # ---- output projection + residual: the residual stream
+    proj = _pack_linear(w.w_proj, w.b_proj, bw, dev)
+    xbar = torch.empty(M, D, dtype=act_dtype, device=dev)
+    gemm(o_c, s_at, z_at, rs_o, proj, D, D, xbar, residual=x,
+         out_kind=B.REPQ_OUT_F32 if act_dtype == torch.float32 else B.REPQ_OUT_BF16)
+
+    # ---- LayerNorm 2 -> fc1 -> activation
+    w_fc1, b_fc1 = w.w_fc1, w.b_fc1
+    if llama:
+        order = np.stack([np.arange(MLP), MLP + np.arange(MLP)], axis=1).reshape(-1)
+        w_fc1, b_fc1 = w.w_fc1[order], w.b_fc1[order]
+    ln2_lo, ln2_hi, fc1, c2, rs2, s2, z2 = after_norm(xbar, w.ln2_gamma, w.ln2_beta, w_fc1, b_fc1)
+    h_f = torch.empty(M, MLP, dtype=torch.float32, device=dev)
+    gemm(c2, s2, z2, rs2, fc1, 2 * MLP if llama else MLP, D, h_f, gelu=not llama, glu=llama)
+    quantizer("hidden", h_f)
+    assert B.repq_device_status() == 0
+    return dataclasses.replace(w, ln1_lo=ln1_lo, ln1_hi=ln1_hi, ln2_lo=ln2_lo, ln2_hi=ln2_hi, bounds=bounds)

@@ -1014,3 +1014,35 @@ def check_dual_clip(n, D, bits, seed=0, iters=100, alpha0=2.0, strided=False):
     assert np.allclose(got[:D], ref["loss0"], rtol=1e-9), "objective before the first step"
     assert np.allclose(got[D:], ref["loss"], rtol=1e-5), "objective with the learned bounds"
     return dict(loss0=float(ref["loss0"].sum()), loss=float(ref["loss"].sum()))
+
+
+def check_calibration(name, batch, alpha0=2.0, **overrides):
+    """The calibration pipeline on the GPU path (dual clipping, percentile calibration, every layer's input taken
+    behind the layers already quantized) against the oracle's: the bounds found, then the block run with the
+    GPU-calibrated bounds against the oracle block on the same bounds."""
+    import torch
+    from oracle import repq_oracle as orc
+    from paper_2402_05628_b200.engine import QuantBlock, calibrate_block
+    from workloads import make_block_inputs
+
+    w = make_block_inputs(name, batch=batch, **overrides)
+    ref = orc.block_forward(w, calibrate=dict(alpha0=alpha0))
+    w_cal = calibrate_block(w, alpha0=alpha0)
+    # LayerNorm bounds: to 1e-4 of the channel's range (float32 activations against float64, sums in another order)
+    for tag in ("ln1", "ln2"):
+        lo_r, hi_r = ref[tag + "_lo"].astype(np.float64), ref[tag + "_hi"].astype(np.float64)
+        lo_g, hi_g = getattr(w_cal, tag + "_lo").astype(np.float64), getattr(w_cal, tag + "_hi").astype(np.float64)
+        rng_ch = hi_r - lo_r
+        frac_ok = np.mean((np.abs(lo_g - lo_r) <= 1e-4 * rng_ch) & (np.abs(hi_g - hi_r) <= 1e-4 * rng_ch))
+        assert frac_ok >= 0.99, (tag, frac_ok)          # a rounding decision on a tie may steer one channel's steps apart
+        assert np.all(np.abs(lo_g - lo_r) <= 2e-2 * rng_ch) and np.all(np.abs(hi_g - hi_r) <= 2e-2 * rng_ch), tag
+    for key, (lo_r, hi_r) in ref["bounds"].items():
+        lo_g, hi_g = w_cal.bounds[key]
+        width = float(hi_r) - float(lo_r)
+        assert abs(float(lo_g) - float(lo_r)) <= 2e-3 * width and abs(float(hi_g) - float(hi_r)) <= 2e-3 * width, (key, lo_g, lo_r, hi_g, hi_r)
+    # the calibrated block: CUDA path against the oracle, both on the bounds the GPU pipeline found
+    blk = QuantBlock(w_cal, out_dtype=torch.float32)
+    x = torch.from_numpy(w.x).to(blk.device).to(blk.act_dtype)
+    y = blk.forward(x)
+    torch.cuda.synchronize()
+    return assert_float_close(y.cpu().numpy(), orc.block_forward(w_cal)["y"], "calibrated block %s" % name)

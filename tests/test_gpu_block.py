@@ -82,6 +82,30 @@ def test_block_stages_teacher_forced_c4_llama_form_full_size():
     parity.check_block_teacher_forced("c4_llama7b_arch")
 
 
+@pytest.mark.parametrize("name,batch,overrides", [
+    ("c1_vit_s", 4, {}), ("c4_llama7b_arch", 2, dict(D=512, H=4, MLP=1408, L=320, massive=2)),
+])
+def test_calibration_pipeline_matches_oracle(name, batch, overrides):
+    """Algorithm 1 for one block (dual clipping for the LayerNorm activations, percentile calibration elsewhere,
+    round-to-nearest weights) through the library against the oracle's pipeline."""
+    parity.check_calibration(name, batch, **overrides)
+
+
+def test_block_with_byte_wide_weight_storage():
+    """4-bit weights kept one code per byte in device memory instead of packed: same block."""
+    import numpy as np
+    import torch
+    from paper_2402_05628_b200.engine import QuantBlock
+    from workloads import make_block_inputs
+    w = make_block_inputs("c2_deit_b", batch=3)
+    a, b = QuantBlock(w, weight_storage="packed"), QuantBlock(w, weight_storage="bytes")
+    assert a.qkv.codes.shape[1] * 2 == b.qkv.codes.shape[1]
+    x = torch.from_numpy(np.ascontiguousarray(w.x)).to(a.device).to(a.act_dtype)
+    ya, yb = a.forward(x), b.forward(x)
+    torch.cuda.synchronize()
+    assert torch.equal(ya, yb)
+
+
 def test_block_with_the_three_separate_attention_stages():
     """The block through repq_qgemm (scores) -> repq_softmax_log2 -> repq_pv instead of the fused kernel."""
     parity.check_block("c2_deit_b", batch=3, staged_attention=True)
