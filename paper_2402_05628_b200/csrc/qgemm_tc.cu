@@ -11,9 +11,10 @@
 //                the main loop of tile i + 1
 //   warps 2..17  epilogue: warp w reads TMEM lanes 32 (w mod 4) .. +31 (one output row per thread) and a
 //                64-column slice of the accumulator columns
-//   warps 18..19 (packed 4-bit weights only) converters: the weight tile arrives packed, two codes per byte, and is
-//                expanded into the 128-byte-swizzled byte tile the MMA descriptor expects (there is no 4-bit integer
-//                MMA); one more barrier hop between the copy and the MMA, weights stay packed in HBM
+//   packed 4-bit weights: 12 epilogue warps (tiles of at most 192 columns) and 4 converter warps.  The weight tile
+//                arrives packed, two codes per byte, and the converters expand it into the 128-byte-swizzled byte tile
+//                the MMA descriptor expects (there is no 4-bit integer MMA); one more barrier hop between the copy
+//                and the MMA, weights stay packed in HBM
 // The tile width BN (256, 192 or 128) is chosen per problem: rounds of tiles over the SMs times a per-round time
 // with a fixed part.  Packed 4-bit activations are expanded to one code per byte by a separate pass into the
 // workspace (inside the block the producers write byte codes, so that pass does not run there).
@@ -46,13 +47,14 @@ constexpr int kChunk = 16;                           // accumulator columns per 
 constexpr int kEpiWarps = 16;
 constexpr int kEpiThreads = kEpiWarps * 32;
 constexpr int kThreads = 32 * (2 + kEpiWarps);
-constexpr int kConvWarps = 2;                        // converter warps of the packed-weight variant
-constexpr int kConvThreads = 32 * kConvWarps;
-constexpr int kThreadsW4 = kThreads + kConvThreads;  // 20 warps: five per scheduler, the same register budget as 18
 constexpr int kTmemCols = 512;
 constexpr int kAccStride = 256;                      // TMEM columns between the two accumulator buffers
 constexpr int kSliceCols = 64;                       // accumulator columns per epilogue warp
 constexpr int kSliceChunks = kSliceCols / kChunk;
+constexpr int kConvWarps = 4;                        // converter warps of the packed-weight variant, which gives up four
+constexpr int kConvThreads = 32 * kConvWarps;        // epilogue warps for them (same CTA size, same register budget)
+constexpr int kEpiWarpsW4 = kEpiWarps - kConvWarps;
+constexpr int kMaxBNW4 = kEpiWarpsW4 / 4 * kSliceCols;   // 192: one 64-column slice per epilogue warp of a lane quarter
 constexpr uint32_t kABytes = BM * BK;
 constexpr uint32_t kMagicBits = 0x4B400000u;         // 1.5 * 2^23
 
@@ -71,17 +73,23 @@ constexpr uint32_t kResBytes = 32 * 128;            // bf16 residual of one warp
 // tile ahead (the operand ring gives up a stage for the boxes)
 template <int BN, bool RES, bool W4>
 struct SharedStorage {
-  static constexpr int kStages = (RES || W4) ? 3 : 4;
+  // kStages: ring of the bulk copies (activation tile + weight tile as it arrives).  kStagesB: ring of byte weight
+  // tiles the MMA reads: the same ring when the weights arrive as bytes; with packed weights a short ring of its own
+  // (the hop from converter to MMA is short), which leaves room for a deeper copy ring ahead of the converters.
+  static constexpr int kStages = W4 ? 5 : (RES ? 3 : 4);
+  static constexpr int kStagesB = W4 ? 2 : kStages;
+  static constexpr int kEpi = W4 ? kEpiWarpsW4 : kEpiWarps;
   alignas(1024) uint8_t a[kStages][kABytes];
-  alignas(1024) uint8_t b[kStages][BN * BK];
+  alignas(1024) uint8_t b[kStagesB][BN * BK];
   alignas(1024) uint8_t res[RES ? kEpiWarps * kResBytes : 1024];
   uint64_t res_full[kEpiWarps];
-  alignas(1024) uint8_t epi[kEpiWarps][1024];     // per-warp staging box of the epilogue's bulk stores
-  ColTerms cols[kEpiWarps];                       // each epilogue warp stages the terms of its own slice: no barrier
+  alignas(1024) uint8_t epi[kEpi][1024];          // per-warp staging box of the epilogue's bulk stores
+  ColTerms cols[kEpi];                            // each epilogue warp stages the terms of its own slice: no barrier
   alignas(128) uint8_t bp[W4 ? kStages : 1][W4 ? BN * BK / 2 : 128];   // packed weight tiles: rows of 64 bytes, unswizzled
   alignas(8) uint64_t full[kStages];
   uint64_t empty[kStages];
-  uint64_t ready[kStages];                          // weight tile expanded (packed variant)
+  uint64_t ready[kStagesB];                         // packed variant: byte weight tile written by the converters
+  uint64_t bfree[kStagesB];                         //                 ... and read by the MMAs
   uint64_t tmem_full[2];
   uint64_t tmem_empty[2];
   uint64_t done;
@@ -89,7 +97,7 @@ struct SharedStorage {
   volatile int abort;
 };
 
-static_assert(sizeof(SharedStorage<kMaxBN, false, false>) <= 227 * 1024 && sizeof(SharedStorage<kMaxBN, false, true>) <= 227 * 1024 &&
+static_assert(sizeof(SharedStorage<kMaxBN, false, false>) <= 227 * 1024 && sizeof(SharedStorage<kMaxBNW4, false, true>) <= 227 * 1024 &&
               sizeof(SharedStorage<192, true, false>) <= 227 * 1024, "shared storage exceeds the 227 KB a CTA may use");
 
 using namespace tc;
@@ -336,11 +344,13 @@ __device__ __noinline__ void slow_chunk(const EpilogueParams& ep, const TcParams
 enum : int { kPairNone = 0, kPairRope = 1, kPairGlu = 2 };
 
 template <int BN, int OUT, bool RES, int PAIR, bool W4>
-__global__ void __launch_bounds__(W4 ? kThreadsW4 : kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 1)
 qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_res, TcParams P) {
   using Storage = SharedStorage<BN, RES, W4>;
   constexpr int kStages = Storage::kStages;
+  constexpr int EW = W4 ? kEpiWarpsW4 : kEpiWarps;       // epilogue warps of this variant
+  static_assert(!W4 || BN <= kMaxBNW4, "the packed-weight variant has three column slices");
   constexpr uint32_t kBBytes = BN * BK;
   constexpr uint32_t kIdesc = idesc_for(BN);
   // 1024-byte alignment (swizzle atoms) is requested from the declaration so that the compiler keeps
@@ -357,9 +367,9 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     for (int s = 0; s < kStages; ++s) {
       mbar_init(smem_u32(&S.full[s]), 1);
       mbar_init(smem_u32(&S.empty[s]), 1);
-      mbar_init(smem_u32(&S.ready[s]), kConvWarps);
     }
-    for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&S.tmem_full[a]), 1); mbar_init(smem_u32(&S.tmem_empty[a]), kEpiWarps); }
+    for (int s = 0; s < Storage::kStagesB; ++s) { mbar_init(smem_u32(&S.ready[s]), kConvWarps); mbar_init(smem_u32(&S.bfree[s]), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&S.tmem_full[a]), 1); mbar_init(smem_u32(&S.tmem_empty[a]), EW); }
     for (int w = 0; w < kEpiWarps; ++w) mbar_init(smem_u32(&S.res_full[w]), 1);
     mbar_init(smem_u32(&S.done), 1);
     S.abort = 0;
@@ -412,7 +422,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issue
     if (lane == 0) {
-      uint32_t stage = 0, phase = 0;
+      uint32_t stage = 0, phase = 0, bstage = 0, bphase = 0;
       int it = 0;
       for (int tile = blockIdx.x; tile < tiles && !*abort; tile += gridDim.x, ++it) {
         const uint32_t acc = it & 1, acc_phase = (it >> 1) & 1;
@@ -421,16 +431,20 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         const uint32_t d_tmem = tmem_base + acc * kAccStride;
         bool ok = true;
         for (int kb = 0; kb < kblocks; ++kb) {
-          // packed weights: the converters release the stage once the byte tile is written (they have waited for the
-          // copies themselves, so the activation tile has landed as well)
-          if (!mbar_wait(smem_u32(W4 ? &S.ready[stage] : &S.full[stage]), phase, abort, 3)) { ok = false; break; }
+          // packed weights: the converters hand over a byte tile (they have waited for the copies themselves, so the
+          // activation tile of the same k-block has landed as well)
+          if (!mbar_wait(smem_u32(W4 ? &S.ready[bstage] : &S.full[stage]), W4 ? bphase : phase, abort, 3)) { ok = false; break; }
           tc_fence_after();
-          const uint64_t da = smem_desc(smem_u32(S.a[stage])), db = smem_desc(smem_u32(S.b[stage]));
+          const uint64_t da = smem_desc(smem_u32(S.a[stage])), db = smem_desc(smem_u32(S.b[W4 ? bstage : stage]));
 #pragma unroll
           for (int k = 0; k < BK / 32; ++k)
             umma_i8(d_tmem, da + uint64_t(k * 2), db + uint64_t(k * 2), kIdesc, (kb | k) != 0 ? 1u : 0u);
           umma_commit(smem_u32(&S.empty[stage]));          // frees the stage once these MMAs have read it
           if (++stage == kStages) { stage = 0; phase ^= 1; }
+          if constexpr (W4) {
+            umma_commit(smem_u32(&S.bfree[bstage]));       // and the byte tile for the converters
+            if (++bstage == Storage::kStagesB) { bstage = 0; bphase ^= 1; }
+          }
         }
         if (!ok) break;
         umma_commit(smem_u32(&S.tmem_full[acc]));           // accumulator complete
@@ -440,27 +454,28 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       const long long t0 = clock64();
       while (!mbar_try_wait(smem_u32(&S.done), 0) && clock64() - t0 < kWaitCycles) {}
     }
-  } else if (W4 && warp >= 2 + kEpiWarps) {
+  } else if (W4 && warp >= 2 + EW) {
     // ---------------------------------------------------------------- converters (packed 4-bit weights)
     // A packed tile holds BN rows of 64 bytes (128 codes, even index in the low nibble).  Thread ct takes 16-byte
-    // pieces ct, ct + 64, ...: piece g = (row g / 4, codes 32 (g % 4) ..) becomes the two 16-byte pieces 2 (g % 4) and
+    // pieces ct, ct + 128, ...: piece g = (row g / 4, codes 32 (g % 4) ..) becomes the two 16-byte pieces 2 (g % 4) and
     // 2 (g % 4) + 1 of the row's 128 bytes, stored where the 128-byte swizzle puts them.  Reads are consecutive
     // across the warp; the stores of eight neighbouring threads cover two rows and all eight swizzled positions.
-    const int ct = int(threadIdx.x) - 32 * (2 + kEpiWarps);
-    uint32_t stage = 0, phase = 0;
+    const int ct = int(threadIdx.x) - 32 * (2 + EW);
+    uint32_t stage = 0, phase = 0, bstage = 0, bphase = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < tiles && ok && !*abort; tile += gridDim.x) {
       for (int kb = 0; kb < kblocks; ++kb) {
+        // the packed tile has landed, and the MMAs that read the byte tile's previous content have completed
         if (!mbar_wait(smem_u32(&S.full[stage]), phase, abort, 7)) { ok = false; break; }
-        // pieces ct, ct + 64, ...: the row advances by 16 per step, so the row's position inside its group of eight
-        // (hence the swizzle) is the thread's own; four pieces are loaded before any is expanded, so that the loads
-        // of a batch overlap the arithmetic of the one before
+        if (!mbar_wait(smem_u32(&S.bfree[bstage]), bphase ^ 1, abort, 8)) { ok = false; break; }
+        // pieces ct, ct + 128, ...: the row advances by 32 per step, so the row's position inside its group of eight
+        // (hence the swizzle) is the thread's own; the pieces of a batch are loaded before any is expanded
         const uint4* src = reinterpret_cast<const uint4*>(S.bp[stage]) + ct;
         const int n_lo = (ct >> 2) & 7, pp = ct & 3;
-        uint8_t* row = S.b[stage] + uint32_t(ct >> 5) * 1024u + uint32_t(n_lo) * 128u;
+        uint8_t* row = S.b[bstage] + uint32_t(ct >> 5) * 1024u + uint32_t(n_lo) * 128u;
         uint8_t* d0 = row + (uint32_t((2 * pp) ^ n_lo) << 4);
         uint8_t* d1 = row + (uint32_t((2 * pp + 1) ^ n_lo) << 4);
-        constexpr int kBatch = 4, kSteps = BN * 4 / kConvThreads;          // 16-row steps per thread
+        constexpr int kBatch = 2, kSteps = BN * 4 / kConvThreads;          // 32-row steps per thread
         static_assert(kSteps % kBatch == 0, "converter batches must divide the tile");
 #pragma unroll 1
         for (int i0 = 0; i0 < kSteps; i0 += kBatch) {
@@ -477,14 +492,15 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
               o[2 * i] = __byte_perm(lo, hi, 0x5140);
               o[2 * i + 1] = __byte_perm(lo, hi, 0x7362);
             }
-            *reinterpret_cast<uint4*>(d0 + (i0 + u) * 2048) = make_uint4(o[0], o[1], o[2], o[3]);
-            *reinterpret_cast<uint4*>(d1 + (i0 + u) * 2048) = make_uint4(o[4], o[5], o[6], o[7]);
+            *reinterpret_cast<uint4*>(d0 + (i0 + u) * 4096) = make_uint4(o[0], o[1], o[2], o[3]);
+            *reinterpret_cast<uint4*>(d1 + (i0 + u) * 4096) = make_uint4(o[4], o[5], o[6], o[7]);
           }
         }
         fence_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&S.ready[stage]));
+        if (lane == 0) mbar_arrive(smem_u32(&S.ready[bstage]));
         if (++stage == kStages) { stage = 0; phase ^= 1; }
+        if (++bstage == Storage::kStagesB) { bstage = 0; bphase ^= 1; }
       }
     }
   } else {
@@ -760,11 +776,12 @@ TcLayout tc_layout(const repq_gemm_desc& d) {
 // Tile width: rounds of tiles over the SMs times the time of one round, which has a part that does not depend on the
 // width (per-tile waits, staging and bulk-store latencies of the epilogue warps) and a part proportional to it
 // (measured: about 160 columns' worth of fixed time for K = 768).
-int pick_bn(int M, int N, int sms) {
+int pick_bn(int M, int N, int sms, bool w_packed4) {
   const int m_tiles = (M + BM - 1) / BM;
   int best = 256;
   long best_cost = -1;
   for (int bn : {256, 192, 128}) {
+    if (w_packed4 && bn > kMaxBNW4) continue;
     const long tiles = long(m_tiles) * ((N + bn - 1) / bn);
     const long rounds = (tiles + sms - 1) / sms;
     const long cost = rounds * (bn + 160);
@@ -818,14 +835,14 @@ repq_status launch_tc_w(const CUtensorMap& map_a, const CUtensorMap& map_b, cons
   REPQ_CUDA(cudaFuncSetAttribute(qgemm_tc_kernel<BN, OUT, RES, PAIR, W4>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
   const int tiles = ((P.M + BM - 1) / BM) * ((P.N + BN - 1) / BN);
   const int grid = tiles < sms ? tiles : sms;
-  REPQ_CUDA(launch_chained(qgemm_tc_kernel<BN, OUT, RES, PAIR, W4>, dim3(grid), dim3(W4 ? kThreadsW4 : kThreads), smem, st, map_a, map_b, map_out, map_res, P));
+  REPQ_CUDA(launch_chained(qgemm_tc_kernel<BN, OUT, RES, PAIR, W4>, dim3(grid), dim3(kThreads), smem, st, map_a, map_b, map_out, map_res, P));
   note_launch();
   return REPQ_OK;
 }
 
 template <int BN, int OUT, bool RES, int PAIR = kPairNone>
 repq_status launch_tc_res(const CUtensorMap& map_a, const CUtensorMap& map_b, const TcParams& P, int sms, cudaStream_t st) {
-  if constexpr (!RES) {
+  if constexpr (!RES && BN <= kMaxBNW4) {
     if (P.w_packed4) return launch_tc_w<BN, OUT, false, PAIR, true>(map_a, map_b, P, sms, st);
   }
   return launch_tc_w<BN, OUT, RES, PAIR, false>(map_a, map_b, P, sms, st);
@@ -938,7 +955,7 @@ repq_status qgemm_tc(const repq_gemm_desc& d, const EpilogueParams& ep, void* ws
   P.direct_requant = d.out_kind == REPQ_OUT_CODES && !d.gelu && !d.residual && !d.glu;
   REPQ_REQUIRE(device_status_word() != nullptr, REPQ_CUDA_ERROR, "qgemm: device status word unavailable");
   const int sms = sm_count();
-  const int bn = pick_bn(d.M, d.N, sms);
+  const int bn = pick_bn(d.M, d.N, sms, P.w_packed4 != 0);
   CUtensorMap map_a, map_b;
   REPQ_TRY(make_map(&map_a, a, d.M, d.K, lda, BM));
   if (P.w_packed4) REPQ_TRY(make_map(&map_b, d.w_codes, d.N, (int64_t(d.K) + 1) / 2, d.ldw_bytes, bn, BK / 2, false));
