@@ -46,6 +46,9 @@ ATTENTION_INSTR_PER_SCORE = 23
 # DRAM traffic of one launch of a stage kernel, from one ncu capture of the same bench command (summaries under
 # profiles/).  A figure is reported only while the kernel's sources still hash to what was captured.
 NCU_TRAFFIC = {   # (workload, batch, stage): (DRAM bytes read + written per launch, kernel sources, their sha1 when captured)
+    ("c4_llama7b", 4, "attention"): (139604224, ["attention_tc.cu", "tc_ptx.cuh"], "190324ee6ef2"),
+    ("c4_llama7b", 4, "ln1"): (71457792, ["ln_quant.cu", "f32x2.cuh"], "8927f8809457"),
+    ("c4_llama7b", 4, "ln2"): (71122432, ["ln_quant.cu", "f32x2.cuh"], "8927f8809457"),
 }
 
 

@@ -120,10 +120,30 @@ struct TcParams {
   const int32_t* wsum;
   int direct_requant;          // codes out, no GELU, no residual: 1/s_o is folded into the column terms
   int w_packed4;               // weight tiles arrive packed (two codes per byte) and are expanded in shared memory
+  int panel;                   // row tiles per panel of the tile order
   EpilogueParams ep;
 };
 
 enum : int { kOutF32 = 0, kOutBf16 = 1, kOutC4 = 2, kOutC8 = 3 };   // compile-time output kinds of the fast path
+
+// Order of the output tiles.  The row tiles are cut into panels of P.panel; a panel is walked column tile by column
+// tile with its row tiles innermost.  The CTAs that run at the same time then share a panel of activations small
+// enough to stay in L2 while the weight tiles stream past it (with long K the activations of all row tiles do not
+// fit, and walking every row tile per column tile read them from DRAM once per wave of CTAs).
+struct TileOrigin { int m0, n0; };
+__device__ __forceinline__ TileOrigin tile_origin(int tile, int m_tiles, int n_tiles, int panel, int bn) {
+  const int full = (m_tiles / panel) * panel * n_tiles;       // tiles inside whole panels
+  int rows = panel, first = 0, t = tile;
+  if (tile >= full) {                                          // the last, shorter panel
+    t = tile - full;
+    rows = m_tiles - (m_tiles / panel) * panel;
+    first = m_tiles - rows;
+  } else {
+    first = (tile / (panel * n_tiles)) * panel;
+    t = tile % (panel * n_tiles);
+  }
+  return TileOrigin{(first + t % rows) * BM, (t / rows) * bn};
+}
 
 // Output quantizer of one 16-column chunk (Eq. 4 with the chunk's column group).
 struct ChunkQuant {
@@ -398,7 +418,8 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       uint32_t stage = 0, phase = 0;
       long long issued = 0;
       for (int tile = blockIdx.x; tile < tiles && !*abort; tile += gridDim.x) {
-        const int m0 = (tile % m_tiles) * BM, n0 = (tile / m_tiles) * BN;
+        const TileOrigin o = tile_origin(tile, m_tiles, n_tiles, P.panel, BN);
+        const int m0 = o.m0, n0 = o.n0;
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!mbar_wait(smem_u32(&S.empty[stage]), phase ^ 1, abort, 1)) break;
           const uint32_t bar = smem_u32(&S.full[stage]);
@@ -526,7 +547,8 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     float nx_sw[2] = {0.f, 0.f}, nx_bs[2] = {0.f, 0.f};
     auto fetch_terms = [&](int t) {
       if (t >= tiles || !slice_on) return;
-      const int tm0 = (t % m_tiles) * BM, tn0 = (t / m_tiles) * BN;
+      const TileOrigin o = tile_origin(t, m_tiles, n_tiles, P.panel, BN);
+      const int tm0 = o.m0, tn0 = o.n0;
       // plain loads from clamped indices: nothing here may consume a loaded value (a select on it would hold the
       // warp until the load returns); rows and columns outside the matrix are dealt with where the values are used
       const int64_t tm = min(int64_t(tm0) + quarter * 32 + lane, int64_t(P.M) - 1);
@@ -546,7 +568,8 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     bool res_pending = false;
     auto fetch_residual = [&](int t) {
       if (!RES || t >= tiles || !slice_on) return;
-      const int tm0 = (t % m_tiles) * BM, tn0 = (t / m_tiles) * BN;
+      const TileOrigin o = tile_origin(t, m_tiles, n_tiles, P.panel, BN);
+      const int tm0 = o.m0, tn0 = o.n0;
       if (lane == 0) {
         mbar_expect_tx(res_bar, kResBytes);
         tma_load_2d(res_buf, &map_res, res_bar, tn0 + cl0, tm0 + quarter * 32);
@@ -558,7 +581,8 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     int it = 0;
     for (int tile = blockIdx.x; tile < tiles && !*abort; tile += gridDim.x, ++it) {
       const uint32_t acc = it & 1, acc_phase = (it >> 1) & 1;
-      const int m0 = (tile % m_tiles) * BM, n0 = (tile / m_tiles) * BN;
+      const TileOrigin o = tile_origin(tile, m_tiles, n_tiles, P.panel, BN);
+      const int m0 = o.m0, n0 = o.n0;
       const int64_t m = int64_t(m0) + quarter * 32 + lane;
       const bool row_ok = m < P.M;
       // warp-uniform: whole 64-column slice inside the matrix, common epilogue (rows beyond M are clipped by
@@ -956,6 +980,13 @@ repq_status qgemm_tc(const repq_gemm_desc& d, const EpilogueParams& ep, void* ws
   REPQ_REQUIRE(device_status_word() != nullptr, REPQ_CUDA_ERROR, "qgemm: device status word unavailable");
   const int sms = sm_count();
   const int bn = pick_bn(d.M, d.N, sms, P.w_packed4 != 0);
+  {
+    // panels of activations of about 40 MB (a third of the L2 capacity), at least 8 row tiles
+    const int m_tiles = (d.M + BM - 1) / BM;
+    const int64_t fit = (int64_t(40) << 20) / (int64_t(BM) * d.K);
+    P.panel = int(fit < 8 ? 8 : fit);
+    if (P.panel > m_tiles) P.panel = m_tiles;
+  }
   CUtensorMap map_a, map_b;
   REPQ_TRY(make_map(&map_a, a, d.M, d.K, lda, BM));
   if (P.w_packed4) REPQ_TRY(make_map(&map_b, d.w_codes, d.N, (int64_t(d.K) + 1) / 2, d.ldw_bytes, bn, BK / 2, false));
