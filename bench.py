@@ -358,7 +358,17 @@ def kernel_sweeps(peaks, dev, quick=True, only=None, dim=None):
     from paper_2402_05628_b200 import binding as B
     g = torch.Generator(device=dev).manual_seed(4)
     int8_peak = peaks["bf16_tflops"] * INT8_OVER_BF16
-    out = dict(ln_quant=[], softmax_log2=[], qgemm=[])
+    out = dict(ln_quant=[], softmax_log2=[], qgemm=[], dual_clip=[])
+    # per-channel dual clipping (calibration-time; Table X of the paper reports 17 s (DeiT-S) and 46 s (LLaMA-13B) per layer
+    # for its PyTorch implementation on an A6000: context, not a target): 100 Adam steps on the activations of a
+    # calibration batch, float64, every step one pass over the L2-resident activations
+    for n, D in ((6304, 384), (16384, 4096)):
+        if only and only != "clip":
+            continue
+        x = torch.randn(n, D, device=dev, generator=g, dtype=torch.float32) * 2.0 + 0.3
+        lo, hi = torch.empty(D, device=dev), torch.empty(D, device=dev)
+        t = _time_launches(lambda i: B.repq_dual_clip(x, 4, lo, hi, None, iters=100, lr=0.01, alpha0=2.0), 1, reps=3, warmup=1)
+        out["dual_clip"].append(dict(tokens=n, D=D, iters=100, ms=t * 1e3, passes_gbs=102 * n * D * 4 / t / 1e9))
     # fused LN + quant: bf16 in, packed 4-bit codes out (2.5 D bytes per token + 4 for the row sum)
     for D in (384, 768, 1024, 4096, 8192):
         if (only and only != "ln") or (dim and dim != D):
@@ -486,7 +496,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="headline workload only: no other workloads, sweeps or sustained run")
     ap.add_argument("--sustained-seconds", type=float, default=3.0)
-    ap.add_argument("--sweep-only", default=None, choices=["ln", "softmax", "gemm"],
+    ap.add_argument("--sweep-only", default=None, choices=["ln", "softmax", "gemm", "clip"],
                     help="run only the single-kernel sweep points of this kernel and print them (profiling aid)")
     ap.add_argument("--sweep-dim", type=int, default=None, help="with --sweep-only: only this D (ln), L (softmax) or N (gemm)")
     ap.add_argument("--weights", default="bytes", choices=["packed", "bytes"],

@@ -1046,3 +1046,114 @@ def check_calibration(name, batch, alpha0=2.0, **overrides):
     y = blk.forward(x)
     torch.cuda.synchronize()
     return assert_float_close(y.cpu().numpy(), orc.block_forward(w_cal)["y"], "calibrated block %s" % name)
+
+
+# ------------------------------------------------------------------------------------------ sweep sizes, sampled
+
+def check_ln_quant_sampled(rows, D, bits, n_sample=96, seed=4):
+    """The fused LN+quant kernel at a sweep size (the launch the benchmark times), the oracle on sampled rows."""
+    import torch
+    from oracle import repq_oracle as orc
+    from paper_2402_05628_b200 import binding as B
+    from workloads.kernels import affine_params, channel_profile, ln_calibration_bounds, ln_inputs
+
+    rng = np.random.default_rng(seed)
+    c, shift = channel_profile(rng, D, 1.0, 0.01, 50.0)
+    gamma, beta = affine_params(rng, D)
+    lo, hi = ln_calibration_bounds(ln_inputs(rng, 2048, c, shift, True), gamma, beta, 1e-6)
+    x = ln_inputs(rng, rows, c, shift, True)
+    s, z = orc.uniform_scale_zero(lo, hi, qb(bits))
+    gamma_t, beta_t, s_t, z_t, _, _ = B.repq_fold_ln(gamma, beta, s.astype(np.float32), z.astype(np.int32),
+                                                     np.zeros((1, D), dtype=np.float32), None)
+    dev = torch.device("cuda:0")
+    xt = torch.from_numpy(x).to(dev).to(torch.bfloat16)
+    codes = torch.empty(rows, B.code_row_bytes(D, bits), dtype=torch.uint8, device=dev)
+    rs = torch.empty(rows, dtype=torch.int32, device=dev)
+    B.repq_ln_quant(xt, torch.from_numpy(gamma_t).to(dev), torch.from_numpy(beta_t).to(dev), 1e-6, s_t, z_t, bits, codes, rs)
+    torch.cuda.synchronize()
+    pick = np.unique(np.concatenate([[0, rows - 1], rng.integers(0, rows, n_sample)]))
+    xs = x[pick]
+    q_ref, t_cw = orc.quant_uniform(orc.layernorm(xs, gamma, beta, 1e-6), s[None, :], z[None, :], qb(bits))
+    q_gpu = unpack_codes(codes[torch.from_numpy(pick).to(dev)].cpu().numpy(), D, bits)
+    rep = near_tie_report(q_gpu, q_ref, t_cw, ln_delta(xs, gamma_t.astype(np.float64), s_t, t_cw + (z - z_t)[None, :], 1e-6, False))
+    assert rep["bad"] == 0, rep
+    assert rep["mismatch"] <= max(2, 2e-4 * rep["total"]), rep
+    assert np.array_equal(rs.cpu().numpy()[pick].astype(np.int64), q_gpu.sum(axis=1))
+    return rep
+
+
+def check_softmax_log2_sampled(rows, L, bits, n_sample=64, seed=4):
+    import torch
+    from oracle import repq_oracle as orc
+    from paper_2402_05628_b200 import binding as B
+    from workloads.kernels import softmax_logits
+
+    rng = np.random.default_rng(seed)
+    # rows of the generator are independent: a block of distinct rows is tiled to the sweep's row count
+    base = softmax_logits(rng, 1024, L)
+    reps = (rows + 1023) // 1024
+    dev = torch.device("cuda:0")
+    ld = (L + 3) // 4 * 4
+    buf = torch.zeros(1024, ld, dtype=torch.float32, device=dev)
+    buf[:, :L] = torch.from_numpy(base).to(dev)
+    S = buf.repeat(reps, 1)[:rows].contiguous()
+    ldc = max(B.code_row_bytes(L, bits), (L + 7) // 8 * (4 if bits == 4 else 8))
+    codes = torch.empty(rows, ldc, dtype=torch.uint8, device=dev)
+    B.repq_softmax_log2(S, L, 1.0, bits, codes)
+    torch.cuda.synchronize()
+    pick = np.unique(np.concatenate([[0, rows - 1], rng.integers(0, rows, n_sample)]))
+    q_ref, t_ref = orc.quant_logsqrt2(orc.softmax_rows(base[pick % 1024].astype(np.float64)), 1.0, qb(bits))
+    q_gpu = unpack_codes(codes[torch.from_numpy(pick).to(dev)].cpu().numpy(), L, bits)
+    delta = 2.0 ** -18 * np.maximum(1.0, np.abs(np.where(np.isfinite(t_ref), t_ref, 0.0)))
+    rep = near_tie_report(q_gpu, q_ref, t_ref, delta)
+    assert rep["bad"] == 0, rep
+    assert rep["mismatch"] <= max(2, 2e-4 * rep["total"]), rep
+    return rep
+
+
+def check_qgemm_sampled(M, N, K, qbits, out_kind, n_sample=24, seed=4, weights="bytes"):
+    """repq_qgemm at a sweep size with the operand formats the benchmark times, the oracle on sampled rows."""
+    import torch
+    from oracle import repq_oracle as orc
+    from paper_2402_05628_b200 import binding as B
+
+    rng = np.random.default_rng(seed)
+    bits = qbits | BYTE_CODES
+    bits_w = qbits if weights == "packed" else bits
+    a = rng.integers(0, 1 << qbits, size=(M, K), dtype=np.uint8)
+    wq = rng.integers(0, 1 << qbits, size=(N, K), dtype=np.uint8)
+    s_a, z_a = np.float32(0.07), int(rng.integers(0, 1 << qbits))
+    s_w = rng.uniform(0.001, 0.01, size=N).astype(np.float32)
+    z_w = rng.integers(0, 1 << qbits, size=N, dtype=np.int32)
+    bias = rng.normal(0.0, 0.02, size=N).astype(np.float32)
+    dev = torch.device("cuda:0")
+    a_t = torch.from_numpy(a).to(dev)
+    w_t = torch.from_numpy(pack_codes(wq, bits_w, B.code_row_bytes(K, bits_w)) if weights == "packed" else wq).to(dev)
+    s_w_t, z_w_t, bias_t = (torch.from_numpy(v).to(dev) for v in (s_w, z_w, bias))
+    pick = np.unique(np.concatenate([[0, M - 1], rng.integers(0, M, n_sample)]))
+    v_ref = orc.linear(orc.dequant_uniform(a[pick], s_a, z_a), wq, s_w, z_w, bias)
+    kw = {}
+    if out_kind == "codes":
+        s_o, z_o = orc.uniform_scale_zero(np.percentile(v_ref, 1), np.percentile(v_ref, 99), qbits)
+        out = torch.empty(M, N, dtype=torch.uint8, device=dev)
+        kw = dict(out_kind=B.REPQ_OUT_CODES, out_bits=bits, out_scale=[float(s_o)], out_zero=[int(z_o)])
+    else:
+        out = torch.empty(M, N, dtype=torch.bfloat16, device=dev)
+        kw = dict(out_kind=B.REPQ_OUT_BF16)
+    d = B.gemm_desc(M, N, K, a_t, bits, float(s_a), z_a, w_t, bits_w, out, s_w=s_w_t, z_w=z_w_t, bias=bias_t, **kw)
+    ws = torch.empty(max(B.repq_qgemm_workspace_bytes(d), 16), dtype=torch.uint8, device=dev)
+    B.repq_qgemm(d, ws)
+    torch.cuda.synchronize()
+    assert B.repq_device_status() == 0
+    got = out[torch.from_numpy(pick).to(dev)]
+    if out_kind == "codes":
+        q_ref, t_ref = orc.quant_uniform(v_ref, s_o, z_o, qbits)
+        mag = np.abs(v_ref - bias[None, :]) + np.abs(bias)[None, :] + np.abs(v_ref)
+        rep = near_tie_report(got.cpu().numpy().astype(np.int64), q_ref, t_ref, 2.0 ** -19 * mag / s_o + 2.0 ** -20 * np.abs(t_ref))
+        assert rep["bad"] == 0, rep
+        assert rep["mismatch"] <= max(2, 2e-4 * rep["total"]), rep
+        return rep
+    ref16 = orc.round_bf16(v_ref)
+    g = got.float().cpu().numpy()
+    assert np.all(np.abs(g - ref16) <= np.abs(ref16) * 2.0 ** -7 + 1e-30)
+    return dict(rel_l2=float_errors(g, v_ref)[0])

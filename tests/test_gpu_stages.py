@@ -220,3 +220,22 @@ def test_dual_clip_matches_oracle(n, D, bits, iters, strided):
     rep = parity.check_dual_clip(n, D, bits, seed=n + D, iters=iters, strided=strided)
     if iters:
         assert rep["loss"] < rep["loss0"]
+
+
+@pytest.mark.parametrize("rows,D,bits", [(262144, 768, 4), (65536, 4096, 4), (1048576, 384, 4 | parity.BYTE_CODES), (32768, 8192, 8)])
+def test_ln_quant_at_sweep_sizes_sampled_rows(rows, D, bits):
+    parity.check_ln_quant_sampled(rows, D, bits)
+
+
+@pytest.mark.parametrize("rows,L,bits", [(151296, 197, 4), (151296, 577, 8), (32768, 2048, 4), (32768, 8192, 4)])
+def test_softmax_log2_at_sweep_sizes_sampled_rows(rows, L, bits):
+    parity.check_softmax_log2_sampled(rows, L, bits)
+
+
+@pytest.mark.parametrize("M,N,K,qbits,out_kind,weights", [
+    (16384, 2304, 768, 4, "codes", "bytes"), (16384, 768, 3072, 8, "bf16", "bytes"), (16384, 12288, 4096, 4, "codes", "bytes"),
+    (16384, 4096, 11008, 4, "bf16", "bytes"), (65536, 768, 768, 4, "codes", "bytes"), (2048, 4096, 4096, 8, "codes", "bytes"),
+    (16384, 11008, 4096, 4, "codes", "packed"), (8192, 4096, 11008, 4, "bf16", "packed"),
+])
+def test_qgemm_at_sweep_sizes_sampled_rows(M, N, K, qbits, out_kind, weights):
+    parity.check_qgemm_sampled(M, N, K, qbits, out_kind, weights=weights)
