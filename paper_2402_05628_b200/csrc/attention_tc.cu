@@ -510,7 +510,8 @@ attention_tc_kernel(AttnParams P) {
       if (lane == 0) mbar_arrive(smem_u32(&S.k_full[g & 1]));
       kreg = knext;
       k_live = k_live_next;
-      if (g + 2 < 2 * nb) fetch_k((g + 2) % nb, knext, k_live_next);            // two blocks ahead: global latency is about one block
+      // two blocks ahead (global latency is about one block); g + 2 < 2 nb, so the block index needs no division
+      if (g + 2 < 2 * nb) fetch_k(g + 2 < nb ? g + 2 : g + 2 - nb, knext, k_live_next);
       if (g > 0 && !process(g - 1)) { ok = false; break; }
     }
     if (ok && !*abort) ok = process(2 * nb - 1);

@@ -41,6 +41,11 @@ constexpr int kTriesPerCheck = 32;
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort, int code, int32_t* status,
                                           long long limit_cycles = kWaitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
+  // a short run of further tries (each may keep the warp suspended for kSuspendNs) before the clock is read at all:
+  // most waits end here
+#pragma unroll 1
+  for (int i = 0; i < 8; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
 #pragma unroll 1
