@@ -327,9 +327,10 @@ attention_tc_kernel(AttnParams P) {
     float k0 = 0.f;                         // pass 2: 2 (log2 Z + log2 s), with m the row's final maximum
 
     // corr = acc - z_k qsum - z_q ksum + d_h z_q z_k of the thread's 16 columns of key block j (buffer g & 1), as
-    // integers; keys the row may not see become kMasked.  Frees the buffer as soon as it is read.
-    constexpr int kMasked = -2147483647 - 1;
-    auto read_s = [&](int g, int j, int (&corr)[kCols]) -> bool {
+    // integers.  Frees the buffer as soon as it is read.  Keys the row may not see are dealt with by the callers, in
+    // the blocks that reach past the keys the thread's row sees (`edge`): the values themselves are left as they
+    // come from tensor memory, so that the common path carries no selects or copies.
+    auto read_s = [&](int g, int j, int (&corr)[kCols], bool& edge) -> bool {
       const int b = g & 1;
       if (!mbar_wait(smem_u32(&S.s_full[b]), uint32_t(g >> 1) & 1u, abort, 44, P.status)) return false;
       tc_fence_after();
@@ -354,35 +355,46 @@ attention_tc_kernel(AttnParams P) {
           corr[4 * e4 + 3] = int32_t(r0[4 * e4 + 3]) + my_row_term + c4.w;
         }
       }
-      // causal mask and keys past Lk: only in blocks that reach past the fewest keys any row of the CTA sees
-      const int key0 = j * kKeys + part * kCols;
-      if (__builtin_expect(key0 + kCols > min(min_valid, valid), 0)) {
-#pragma unroll
-        for (int e = 0; e < kCols; ++e)
-          if (key0 + e >= valid) corr[e] = kMasked;
-      }
+      edge = j * kKeys + part * kCols + kCols > valid;
       return true;
     };
 
     auto process = [&](int g) -> bool {
       const int j = g < nb ? g : g - nb;
       int corr[kCols];
-      if (!read_s(g, j, corr)) return false;
+      bool edge;
+      if (!read_s(g, j, corr, edge)) return false;
+      const int seen = valid - (j * kKeys + part * kCols);       // columns e < seen are keys the row sees
       if (g < nb) {
         // ---- pass 1: running maximum and sum.  The maximum is taken on the integers (S = scale * float(corr) is
-        // monotonic in corr); a masked key contributes 2^(-huge) = 0.
-        int bmi = corr[0];
+        // monotonic in corr); a key the row may not see contributes nothing.
+        const float sc = P.scale * c;                             // exponent of 2 per unit of corr
+        if (__builtin_expect(!edge, 1)) {
+          int bmi = corr[0];
 #pragma unroll
-        for (int e = 1; e < kCols; ++e) bmi = max(bmi, corr[e]);
-        if (bmi != kMasked) {
+          for (int e = 1; e < kCols; ++e) bmi = max(bmi, corr[e]);
           const float mn = fmaxf(m, P.scale * float(bmi));
+          const float mnc = mn * c;
           float acc0 = 0.f, acc1 = 0.f;
 #pragma unroll
           for (int e = 0; e < kCols; e += 2) {
-            acc0 += ex2(fmaf(float(corr[e]), P.scale, -mn) * c);
-            acc1 += ex2(fmaf(float(corr[e + 1]), P.scale, -mn) * c);
+            acc0 += ex2(fmaf(float(corr[e]), sc, -mnc));
+            acc1 += ex2(fmaf(float(corr[e + 1]), sc, -mnc));
           }
           z = z * ex2((m - mn) * c) + (acc0 + acc1);     // m = -inf at first: factor 0
+          m = mn;
+        } else if (seen > 0) {
+          int bmi = corr[0];
+#pragma unroll
+          for (int e = 1; e < kCols; ++e)
+            if (e < seen) bmi = max(bmi, corr[e]);
+          const float mn = fmaxf(m, P.scale * float(bmi));
+          const float mnc = mn * c;
+          float acc = 0.f;
+#pragma unroll
+          for (int e = 0; e < kCols; ++e)
+            if (e < seen) acc += ex2(fmaf(float(corr[e]), sc, -mnc));
+          z = z * ex2((m - mn) * c) + acc;
           m = mn;
         }
         if (g == nb - 1) {
@@ -413,7 +425,6 @@ attention_tc_kernel(AttnParams P) {
       // 1.5 * 2^23, which leaves p in the low mantissa bits u - kMagicBits.  The pair (E, O) of bf16 operand values,
       // 2^-ceil(p/2) on the side of p's parity and 0 on the other, comes from a per-lane table for 4-bit codes and
       // from integer arithmetic for wider ones.  A masked key gets (0, 0).
-      const bool boundary = j * kKeys + part * kCols + kCols > min(min_valid, valid);
       const uint32_t lut_addr = smem_u32(&S.lut[0][lane]) - (kMagicBits << 7);
       uint4 ev[kCols / 8], ov[kCols / 8];
       if (!dead_warp) {
@@ -439,10 +450,10 @@ attention_tc_kernel(AttnParams P) {
           eo[e] = (u & 1u) ? val << 16 : val;
         }
       }
-      if (__builtin_expect(boundary, 0)) {
+      if (__builtin_expect(edge, 0)) {
 #pragma unroll
         for (int e = 0; e < kCols; ++e)
-          if (corr[e] == kMasked) eo[e] = 0u;
+          if (e >= seen) eo[e] = 0u;
       }
 #pragma unroll
       for (int p4 = 0; p4 < kCols / 8; ++p4) {
