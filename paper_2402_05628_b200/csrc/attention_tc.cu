@@ -13,12 +13,17 @@
 // rounding tie.
 //
 // One CTA owns 128 query rows of one (batch, head) pair.  Warps 0..15 (four per tensor-memory lane quarter: a thread
-// has one row and 16 of the 64 columns of a key block): K tiles and V tiles from registers (fetched one
-// block ahead) into 128-byte-swizzled shared-memory tiles, the Softmax arithmetic, the E / O tiles, the epilogue.
-// Warp 16 (one lane): tensor-memory allocation and MMA issue.  S is double-buffered in tensor memory (2 x 64 columns),
+// has one row and 16 of the 64 columns of a key block): V tiles (and, for quantizers wider than 7 bits, K tiles) from
+// registers (fetched one block ahead) into 128-byte-swizzled shared-memory tiles, the Softmax arithmetic, the E / O
+// tiles, the epilogue.  Warp 16 (one lane): tensor-memory allocation and MMA issue.  Warp 17 (one lane, quantizers of
+// at most 7 bits): K tiles by bulk tensor copies, two blocks ahead.  There the Q tile holds q - z_q as signed bytes and
+// the K tile the raw unsigned codes: S' = sum (q - z_q) k differs from the zero-point-corrected sum by
+// -z_k sum (q - z_q), which is the same for every key of a row and drops out of the Softmax (maximum and values are
+// taken on S' alone), so no correction and no pass over the K bytes is needed.  S is double-buffered in tensor memory (2 x 64 columns),
 // the E / O / V tiles are single (their block's code arithmetic overlaps the MMAs of the block before).  Under a causal mask, key blocks no row of the CTA may see are
 // skipped.  Every mbarrier wait is bounded; when one runs out the kernel records a status code, all roles leave
 // their loops, MMAs in flight are drained, tensor memory is freed and the kernel returns.
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <math_constants.h>
 
@@ -38,7 +43,7 @@ constexpr int kWorkWarps = 16;                // 4 per tensor-memory lane quarte
 constexpr int kParts = kWorkWarps / 4;
 constexpr int kCols = kKeys / kParts;         // S columns per thread and key block
 constexpr int kWorkThreads = 32 * kWorkWarps;
-constexpr int kThreads = kWorkThreads + 32;
+constexpr int kThreads = kWorkThreads + 64;        // + MMA warp + K-copy warp
 constexpr uint32_t kQBytes = kRows * 128;         // Q tile: rows of 128 bytes (the head's codes, zero-padded)
 constexpr uint32_t kKBytes = kKeys * 128;
 constexpr uint32_t kTileBytes = kRows * 128;      // E or O tile of one block (64 keys of bf16 per row)
@@ -80,6 +85,7 @@ struct AttnShared {
                                                     // lane); the last entry repeats the top code (a clamp at 2^bits that
                                                     // rounds up lands there)
   alignas(8) uint64_t k_full[2];
+  uint64_t k_empty[2];                              // K tile read by its S MMAs (bulk-copy variant)
   uint64_t s_full[2], s_empty[2], p_full, p_empty;
   uint64_t stats_ready, acc_full, done;
   uint32_t tmem_base;
@@ -110,7 +116,7 @@ __device__ __forceinline__ float ex2(float x) {
 // hold q - z_q and k - z_k, the S MMAs run signed x signed and their accumulators need no zero-point correction.
 template <int NB, int kLutBits, bool kCentered>
 __global__ void __launch_bounds__(kThreads, NB == 1 ? 2 : 1)
-attention_tc_kernel(AttnParams P) {
+attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
   using Shared = AttnShared<NB, kLutBits>;
   constexpr bool kLut = kLutBits != 0;
   constexpr int kVItems = NB;                             // 8-channel groups of V per thread and block
@@ -142,7 +148,8 @@ attention_tc_kernel(AttnParams P) {
 
   if (tid == 0) {
     for (int s = 0; s < 2; ++s) {
-      mbar_init(smem_u32(&S.k_full[s]), kWorkWarps);
+      mbar_init(smem_u32(&S.k_full[s]), kCentered ? 1 : kWorkWarps);
+      mbar_init(smem_u32(&S.k_empty[s]), 1);
       mbar_init(smem_u32(&S.s_full[s]), 1);
       mbar_init(smem_u32(&S.s_empty[s]), kWorkWarps);
     }
@@ -179,12 +186,7 @@ attention_tc_kernel(AttnParams P) {
     if (live) dst = __ldg(reinterpret_cast<const uint4*>(k_base + int64_t(key) * P.ldk) + kq);
   };
   const uint32_t zk4 = uint32_t(P.zk) * 0x01010101u, zq4 = uint32_t(P.zq) * 0x01010101u;
-  auto store_k = [&](uint8_t* tile) {            // returns the code sum of the thread's key (not needed when centred)
-    if (kCentered) {
-      // keys past Lk and pieces past d_h stay 0, so that they add nothing to S
-      if (kq < 2 * ksteps) *reinterpret_cast<uint4*>(tile + tile_offset(kkey, kq)) = k_live ? sub_bytes(kreg, zk4) : kreg;
-      return 0;
-    }
+  auto store_k = [&](uint8_t* tile) {            // returns the code sum of the thread's key
     if (kq < 2 * ksteps) *reinterpret_cast<uint4*>(tile + tile_offset(kkey, kq)) = kreg;
     int s = sum_bytes(kreg);
     s += __shfl_xor_sync(0xffffffffu, s, 1);
@@ -194,8 +196,10 @@ attention_tc_kernel(AttnParams P) {
   };
 
   if (warp < kWorkWarps) {
-    fetch_k(0, kreg, k_live);
-    fetch_k(nb > 1 ? 1 : 0, knext, k_live_next);
+    if (!kCentered) {
+      fetch_k(0, kreg, k_live);
+      fetch_k(nb > 1 ? 1 : 0, knext, k_live_next);
+    }
     const uint8_t* q_base = P.q + bo * P.q_so + bi * P.q_si;
     const int qrow = (tid >> 2) & (kRows - 1), qh = tid & 3;
     int s = 0;
@@ -232,7 +236,7 @@ attention_tc_kernel(AttnParams P) {
     if (lane == 0) {
       // S: D = s32, A = B = unsigned 8-bit, both K-major, N = 64, M = 128
       // (operand formats: 0 = unsigned, 1 = signed bytes)
-      constexpr uint32_t idesc_s = (2u << 4) | (uint32_t(kCentered) << 7) | (uint32_t(kCentered) << 10) | (uint32_t(kKeys >> 3) << 17) |
+      constexpr uint32_t idesc_s = (2u << 4) | (uint32_t(kCentered) << 7) | (0u << 10) | (uint32_t(kKeys >> 3) << 17) |
                                    (uint32_t(kRows >> 4) << 24);
       // P.V: D = f32, A = B = bf16, A K-major, B MN-major, N = n_pad, M = 128
       const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (uint32_t(P.n_pad >> 3) << 17) |
@@ -249,6 +253,7 @@ attention_tc_kernel(AttnParams P) {
         for (int s = 0; s < ksteps; ++s)
           umma_i8(tmem_base + uint32_t(b * kKeys), dq + uint64_t(2 * s), dk + uint64_t(2 * s), idesc_s, s != 0 ? 1u : 0u);
         umma_commit(smem_u32(&S.s_full[b]));
+        if (kCentered) umma_commit(smem_u32(&S.k_empty[b]));      // the K tile may be refilled once these MMAs have read it
         return true;
       };
       for (int g = 0; g < nb && ok && !*abort; ++g) ok = issue_s(g);
@@ -271,6 +276,23 @@ attention_tc_kernel(AttnParams P) {
       if (ok && !*abort) umma_commit(smem_u32(&S.acc_full));
       umma_commit(smem_u32(&S.done));
       mbar_drain(smem_u32(&S.done), 0);
+    }
+  } else if (warp == kWorkWarps + 1) {
+    // ---------------------------------------------------------------- K tiles by bulk tensor copies
+    if (kCentered && lane == 0) {
+      int issued = 0;
+      for (int g = 0; g < 2 * nb && !*abort; ++g) {
+        const int b = g & 1;
+        if (!mbar_wait(smem_u32(&S.k_empty[b]), (uint32_t(g >> 1) & 1u) ^ 1u, abort, 48, P.status)) break;
+        const uint32_t bar = smem_u32(&S.k_full[b]);
+        mbar_expect_tx(bar, kKBytes);
+        // box: 128 bytes of the head's row (bytes past d_h meet zero bytes of the Q tile), 64 keys (rows past Lk are
+        // zero-filled), one batch item
+        tma_load_3d(smem_u32(S.k[b]), &map_k, bar, bi * int(P.k_si), (g < nb ? g : g - nb) * kKeys, bo);
+        ++issued;
+      }
+      // the copies issued last must have landed before this CTA may exit
+      for (int i = issued > 2 ? issued - 2 : 0; i < issued; ++i) mbar_drain(smem_u32(&S.k_full[i & 1]), uint32_t(i >> 1) & 1u);
     }
   } else {
     // ---------------------------------------------------------------- tiles, Softmax arithmetic, epilogue
@@ -513,16 +535,18 @@ attention_tc_kernel(AttnParams P) {
 
     bool ok = true;
     for (int g = 0; g < 2 * nb && !*abort; ++g) {
-      // tile g & 1 was last read by the S MMAs of g - 2, whose result this thread has already waited for
-      const int ks = store_k(S.k[g & 1]);
-      if (!kCentered && kq == 0) S.col_term[g & 3][kkey] = -P.zq * ks;
-      fence_async_smem();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&S.k_full[g & 1]));
-      kreg = knext;
-      k_live = k_live_next;
-      // two blocks ahead (global latency is about one block); g + 2 < 2 nb, so the block index needs no division
-      if (g + 2 < 2 * nb) fetch_k(g + 2 < nb ? g + 2 : g + 2 - nb, knext, k_live_next);
+      if (!kCentered) {
+        // tile g & 1 was last read by the S MMAs of g - 2, whose result this thread has already waited for
+        const int ks = store_k(S.k[g & 1]);
+        if (kq == 0) S.col_term[g & 3][kkey] = -P.zq * ks;
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&S.k_full[g & 1]));
+        kreg = knext;
+        k_live = k_live_next;
+        // two blocks ahead (global latency is about one block); g + 2 < 2 nb, so the block index needs no division
+        if (g + 2 < 2 * nb) fetch_k(g + 2 < nb ? g + 2 : g + 2 - nb, knext, k_live_next);
+      }
       if (g > 0 && !process(g - 1)) { ok = false; break; }
     }
     if (ok && !*abort) ok = process(2 * nb - 1);
@@ -615,6 +639,22 @@ attention_tc_kernel(AttnParams P) {
   }
 }
 
+// Tensor map of the K codes for the bulk-copy variant: (bytes of a row, keys, batch items); a box is 128 bytes x 64 keys.
+repq_status make_k_map(CUtensorMap* map, const AttnParams& P, int batch_outer) {
+  EncodeTiledFn fn = encode_fn();
+  REPQ_REQUIRE(fn != nullptr, REPQ_CUDA_ERROR, "attention: cuTensorMapEncodeTiled is not available");
+  const cuuint64_t span = cuuint64_t(P.batch_inner - 1) * cuuint64_t(P.k_si) + cuuint64_t(P.dh);    // bytes the heads cover
+  const cuuint64_t dims[3] = {span, cuuint64_t(P.Lk), cuuint64_t(batch_outer)};
+  const cuuint64_t strides[2] = {cuuint64_t(P.ldk), cuuint64_t(P.k_so)};
+  const cuuint32_t box[3] = {128, cuuint32_t(kKeys), 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<uint8_t*>(P.k), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  REPQ_REQUIRE(r == CUDA_SUCCESS, REPQ_CUDA_ERROR, "attention: K tensor map failed with code %d", int(r));
+  return REPQ_OK;
+}
+
 template <int NB, int kLutBits, bool kCentered>
 repq_status launch_kernel(const AttnParams& P, int64_t pairs, cudaStream_t st) {
   const size_t smem = sizeof(AttnShared<NB, kLutBits>);
@@ -622,8 +662,10 @@ repq_status launch_kernel(const AttnParams& P, int64_t pairs, cudaStream_t st) {
   AttnParams Q = P;
   Q.pairs = int(pairs);
   Q.tiles = (P.Lq + kRows - 1) / kRows;
+  CUtensorMap map_k{};
+  if (kCentered) REPQ_TRY(make_k_map(&map_k, P, int(pairs / P.batch_inner)));
   dim3 grid(unsigned(Q.tiles) * unsigned(pairs));
-  REPQ_CUDA(launch_chained(attention_tc_kernel<NB, kLutBits, kCentered>, grid, dim3(kThreads), smem, st, Q));
+  REPQ_CUDA(launch_chained(attention_tc_kernel<NB, kLutBits, kCentered>, grid, dim3(kThreads), smem, st, map_k, Q));
   note_launch();
   return REPQ_OK;
 }
@@ -631,7 +673,10 @@ repq_status launch_kernel(const AttnParams& P, int64_t pairs, cudaStream_t st) {
 template <int NB, int kLutBits>
 repq_status launch(const AttnParams& P, int64_t pairs, int qmax_qk, cudaStream_t st) {
   // q - z_q and k - z_k as signed bytes: codes and zero points below 128 and differences within [-128, 127]
-  const bool centred = qmax_qk < 128 && P.zq >= 0 && P.zq < 128 && P.zk >= 0 && P.zk < 128;
+  // (the K tiles of this variant come by bulk tensor copies: row and batch strides must be usable as tensor-map strides)
+  const bool centred = qmax_qk < 128 && P.zq >= 0 && P.zq < 128 && P.zk >= 0 && P.zk < 128 && P.k_so > 0 &&
+                       P.ldk < (int64_t(1) << 40) && P.k_so < (int64_t(1) << 40) &&
+                       int64_t(P.batch_inner - 1) * P.k_si + P.dh <= P.ldk;
   return centred ? launch_kernel<NB, kLutBits, true>(P, pairs, st) : launch_kernel<NB, kLutBits, false>(P, pairs, st);
 }
 

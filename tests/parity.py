@@ -575,7 +575,10 @@ def check_attention(B_, H, Lq, Lk, dh, bits, bits_p, causal=False, out_kind="f32
             # for the separate Softmax kernel) plus what the float32 scores carry into it.  S = float(integer sum) *
             # float(alpha s_q s_k): the rounding of the scale is common to S_i and m, so it is relative to S_i - m
             # (part of the |t| term); the rounding of m itself, 2^-24 |m|, enters t through 2 log2(e) = 2.9
-            delta = 2.0 ** -18 * np.maximum(1.0, np.abs(tf)) + 2.0 ** -22 * np.abs(m_row)
+            # The kernel may take its scores without the zero-point term of K, -z_k sum_c (q - z_q), which is common
+            # to all keys of a row and drops out of the Softmax: its row maximum is then m + |that term| at most
+            shift_row = np.abs(alpha * s_q * s_k * z_k * (Qc[b * Lq:(b + 1) * Lq, sl].astype(np.float64) - z_q).sum(axis=1, keepdims=True))
+            delta = 2.0 ** -18 * np.maximum(1.0, np.abs(tf)) + 2.0 ** -22 * (np.abs(m_row) + shift_row)
             near = mask & (np.abs(tf - np.floor(tf) - 0.5) < delta) & (tf < min(top + 0.6, 40.0))   # a flip below a weight of 2^-20 is invisible
             for i, j in zip(*np.nonzero(near)):
                 alt = int(np.clip(np.floor(tf[i, j]) + np.ceil(tf[i, j]) - np.rint(tf[i, j]), 0, top))
