@@ -455,17 +455,18 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
       for (int e = 0; e < kCols; ++e) {
         // clamped on both sides whatever the inputs (rows past Lq carry m = -inf, Z = 0): p indexes the table
         if (kLut) {
-          // table-driven codes: the clamp to [0, 2^bits] is a saturating multiply by 2^-bits (exact), the scaling back
-          // and the rounding one fma; 2^bits (t within half a code of it) reads the table's copy of the top entry
+          // table-driven codes: t 2^-bits comes out of one saturating fma (k1 and k0 scaled by 2^-bits, exact, so the
+          // value is t rounded as before and clamped to [0, 1]), the scaling back and the rounding are one more fma;
+          // 2^bits (t within half a code of it) reads the table's copy of the top entry
           float w;
           constexpr float kSteps = float(1 << kLutBits), kInvSteps = 1.f / kSteps;      // 2^bits and its reciprocal (exact)
-          asm("mul.rn.sat.f32 %0, %1, %2;" : "=f"(w) : "f"(fmaf(fmaf(float(corr[e]), P.scale, -m), k1, k0)), "f"(kInvSteps));
+          asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(w) : "f"(fmaf(float(corr[e]), P.scale, -m)), "f"(k1 * kInvSteps), "f"(k0 * kInvSteps));
           const uint32_t u = __float_as_uint(fmaf(w, kSteps, magic));
           asm("ld.shared.u32 %0, [%1];" : "=r"(eo[e]) : "r"(lut_addr + (u << 7)));
         } else {
           // wider codes: the same clamp to [0, 2^bits], then the top code by one integer minimum
           float w;
-          asm("mul.rn.sat.f32 %0, %1, %2;" : "=f"(w) : "f"(fmaf(fmaf(float(corr[e]), P.scale, -m), k1, k0)), "f"(inv_qs));
+          asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(w) : "f"(fmaf(float(corr[e]), P.scale, -m)), "f"(k1 * inv_qs), "f"(k0 * inv_qs));
           const uint32_t u = min(__float_as_uint(fmaf(w, qs, magic)), u_top);
           const int kk = int((u - kMagicBits + 1u) >> 1);                       // ceil(p / 2)
           const uint32_t val = uint32_t(max(127 - kk, 0)) << 7;                 // bf16 bits of 2^-kk (0 below the normal range)
