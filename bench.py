@@ -46,9 +46,14 @@ ATTENTION_INSTR_PER_SCORE = 23
 # DRAM traffic of one launch of a stage kernel, from one ncu capture of the same bench command (summaries under
 # profiles/).  A figure is reported only while the kernel's sources still hash to what was captured.
 NCU_TRAFFIC = {   # (workload, batch, stage): (DRAM bytes read + written per launch, kernel sources, their sha1 when captured)
-    ("c4_llama7b", 4, "attention"): (139604224, ["attention_tc.cu", "tc_ptx.cuh"], "190324ee6ef2"),
+    ("c4_llama7b", 4, "attention"): (140183808, ["attention_tc.cu", "tc_ptx.cuh"], "25f127db9567"),
+    ("c4_llama7b", 4, "qkv"): (188480000, ["qgemm_tc.cu", "tc_ptx.cuh", "epilogue.cuh"], "56d623be4aa8"),
+    ("c4_llama7b", 4, "proj"): (209939712, ["qgemm_tc.cu", "tc_ptx.cuh", "epilogue.cuh"], "56d623be4aa8"),
+    ("c4_llama7b", 4, "fc1"): (170638080, ["qgemm_tc.cu", "tc_ptx.cuh", "epilogue.cuh"], "56d623be4aa8"),
+    ("c4_llama7b", 4, "fc2"): (569528064, ["qgemm_tc.cu", "tc_ptx.cuh", "epilogue.cuh"], "56d623be4aa8"),
     ("c4_llama7b", 4, "ln1"): (71457792, ["ln_quant.cu", "f32x2.cuh"], "8927f8809457"),
     ("c4_llama7b", 4, "ln2"): (71122432, ["ln_quant.cu", "f32x2.cuh"], "8927f8809457"),
+    ("c2_deit_b", 64, "attention"): (29162496, ["attention_tc.cu", "tc_ptx.cuh"], "25f127db9567"),
 }
 
 

@@ -110,7 +110,8 @@ repq_status repq_layernorm(const void* x, int x_dtype, int64_t rows, int D, int6
  * `alpha0` is the factors' starting value (the paper gives none; 0 starts at half of the extremes).
  * x [device]: n x D float32 activations, row stride ldx elements.  x_low, x_up [device] float[D].
  * loss [device] double[2 D] or NULL: the objective per channel before the first step and with the returned
- * bounds.  Runs in float64 on `stream`, one kernel, no scratch memory; channels are independent. */
+ * bounds.  A channel whose contracted extremes coincide (a constant channel) is left alone: its factors keep alpha0,
+ * its objective reads 0 and x_low = x_up is returned (Eq. 6 has no scale for it; the caller decides).  Runs in float64 on `stream`, one kernel, no scratch memory; channels are independent. */
 repq_status repq_dual_clip(const float* x, int64_t n, int D, int64_t ldx, int bits, int iters, float lr,
                            float alpha0, float* x_low, float* x_up, double* loss, void* stream);
 

@@ -79,7 +79,9 @@ __global__ void __launch_bounds__(kThreads) dual_clip_kernel(ClipParams P) {
     const double s = sh_s[ch], low = sh_low[ch];
     const double zc = -low / s, z = rint(zc);
     double acc_loss = 0.0, acc_ds = 0.0, acc_dl = 0.0;
-    if (on)
+    // a channel whose bounds coincide (a constant channel, or extremes of 0) has no quantizer to learn: its sums stay
+    // 0, its factors keep their starting value and the contracted extremes are returned as they are
+    if (on && s > 0.0)
       for (int64_t t = lane; t < P.n; t += kLanes) {
         const double x = double(__ldg(col + t * P.ldx));
         const double u = x / s, r = rint(u), pre = r + z;

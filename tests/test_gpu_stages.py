@@ -239,3 +239,21 @@ def test_softmax_log2_at_sweep_sizes_sampled_rows(rows, L, bits):
 ])
 def test_qgemm_at_sweep_sizes_sampled_rows(M, N, K, qbits, out_kind, weights):
     parity.check_qgemm_sampled(M, N, K, qbits, out_kind, weights=weights)
+
+
+def test_dual_clip_leaves_a_constant_channel_alone():
+    import torch
+    from paper_2402_05628_b200 import binding as B
+    dev = torch.device("cuda:0")
+    g = torch.Generator(device=dev).manual_seed(3)
+    x = torch.randn(500, 16, device=dev, generator=g)
+    x[:, 5] = 0.75                      # a constant channel: Eq. 6 has no scale for it
+    x[:, 9] = 0.0
+    lo, hi = torch.empty(16, device=dev), torch.empty(16, device=dev)
+    loss = torch.empty(32, dtype=torch.float64, device=dev)
+    B.repq_dual_clip(x, 4, lo, hi, loss, iters=20, lr=0.01, alpha0=0.0)
+    torch.cuda.synchronize()
+    assert torch.isfinite(lo).all() and torch.isfinite(hi).all() and torch.isfinite(loss).all()
+    assert float(lo[5]) == float(hi[5]) == 0.375 and float(lo[9]) == float(hi[9]) == 0.0       # sigmoid(0) = 1/2 of the extremes
+    assert float(loss[5]) == 0.0 and float(loss[16 + 5]) == 0.0
+    assert (hi[[0, 1, 2]] > lo[[0, 1, 2]]).all()
