@@ -20,7 +20,8 @@
  *    Every `bits` argument or field may carry the flag REPQ_BYTE_CODES (e.g. 4 | REPQ_BYTE_CODES): the
  *    quantizer is unchanged, but its codes are stored one per byte.  That is the operand format of
  *    the 8-bit integer tensor-core instruction, so 4-bit tensors kept this way need no expansion pass
- *    before a GEMM; the packed form is for storage and interchange.
+ *    before a GEMM; the packed form is for storage and interchange.  Weight codes of 6 bits may also be
+ *    stored four to three bytes (REPQ_PACKED6); the GEMM expands packed weight tiles in shared memory.
  *    Code tensors are row-major with a row stride in BYTES; float tensors use strides in ELEMENTS.
  *  - Weights are stored [out features j, in features c] (row j is the paper's column W[:, j]).
  *  - Zero-points are plain integers of any sign (Eq. 6 does not bound them).
@@ -57,6 +58,9 @@ typedef int repq_status;
 #define REPQ_MAX_OUT_GROUPS 4
 
 #define REPQ_BYTE_CODES 0x100       /* OR into a `bits` value: one code per byte whatever the bit width */
+#define REPQ_PACKED6 0x200          /* 6 | REPQ_PACKED6, weight codes only (repq_pack_weights, the weight operand of a
+                                       plain repq_qgemm, repq_block_desc.bits_w): four codes in three bytes, code i of
+                                       a row in bits [6i, 6i + 6) of the row read as a little-endian bit string */
 
 /* Copies the calling thread's last error message (NUL-terminated, truncated to n) and returns its
  * full length. */
@@ -89,7 +93,8 @@ repq_status repq_fold_ln(int D, int N, const float* gamma, const float* beta, co
  * are min(row, 0) and max(row, 0) so that 0 <= z_w <= 2^b - 1; an all-zero row gets s_w = 1.
  * In  [host]: W (float N x K, row-major, dense).
  * Out [host]: codes (N rows of ld_codes_bytes bytes; ld_codes_bytes >= K*bits/8 rounded up, multiple
- *             of 16), s_w (float[N]), z_w (int32[N]), w_row_sum (int32[N]) = sum_c codes[j, c]. */
+ *             of 16; bits_w may carry REPQ_BYTE_CODES, or be 6 | REPQ_PACKED6), s_w (float[N]), z_w (int32[N]),
+ *             w_row_sum (int32[N]) = sum_c codes[j, c]. */
 repq_status repq_pack_weights(int N, int K, int bits_w, const float* W, uint8_t* codes,
                               int64_t ld_codes_bytes, float* s_w, int32_t* z_w, int32_t* w_row_sum);
 
@@ -161,7 +166,7 @@ typedef struct repq_gemm_desc {
   const int32_t* a_row_sum;             /* [device] int32[M], plain GEMM only; NULL = computed here */
   /* weight codes w: [N, K] */
   const uint8_t* w_codes;               /* [device] */
-  int32_t bits_w;
+  int32_t bits_w;                       /* 4, 6 or 8 (| REPQ_BYTE_CODES), or 6 | REPQ_PACKED6 (plain GEMM only) */
   int64_t ldw_bytes, w_stride_outer, w_stride_inner;    /* bytes */
   const float* s_w;                     /* [device] float[N] per output channel; NULL = s_w_scalar */
   const int32_t* z_w;                   /* [device] int32[N]; NULL = z_w_scalar */

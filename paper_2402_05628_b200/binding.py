@@ -22,6 +22,7 @@ REPQ_NORM_LAYERNORM, REPQ_NORM_RMS = 0, 1
 REPQ_OUT_F32, REPQ_OUT_BF16, REPQ_OUT_CODES = 0, 1, 2
 REPQ_MAX_OUT_GROUPS = 4
 REPQ_BYTE_CODES = 0x100
+REPQ_PACKED6 = 0x200          # 6 | REPQ_PACKED6: weight codes, four in three bytes
 
 EXPORTS = (
     "repq_last_error", "repq_abi_version", "repq_scale_zero_from_bounds", "repq_fold_ln",
@@ -207,7 +208,8 @@ def _stream(stream) -> int:
 
 
 def code_row_bytes(n: int, bits: int, align: int = 16) -> int:
-    raw = (n + 1) // 2 if bits == 4 else n          # bits may carry REPQ_BYTE_CODES: then one byte per code
+    # bits may carry REPQ_BYTE_CODES (one byte per code) or be 6 | REPQ_PACKED6 (four codes in three bytes)
+    raw = (n + 1) // 2 if bits == 4 else (n * 3 + 3) // 4 if bits == (6 | REPQ_PACKED6) else n
     return (raw + align - 1) // align * align
 
 

@@ -24,7 +24,7 @@ inline size_t bump(size_t& cur, size_t bytes) {
 repq_status validate(const repq_block_desc& d) {
   REPQ_REQUIRE(d.batch > 0 && d.seq > 0 && d.dim > 0 && d.heads > 0 && d.mlp > 0, REPQ_INVALID_ARG, "block: sizes must be positive");
   REPQ_REQUIRE(d.dim % d.heads == 0, REPQ_INVALID_ARG, "block: dim must be a multiple of heads");
-  REPQ_REQUIRE(bits_ok(d.bits_a) && bits_ok(d.bits_w) && bits_ok(d.bits_p), REPQ_INVALID_ARG, "block: bits must be 4, 6 or 8");
+  REPQ_REQUIRE(bits_ok(d.bits_a) && bits_w_ok(d.bits_w) && bits_ok(d.bits_p), REPQ_INVALID_ARG, "block: bits must be 4, 6 or 8");
   REPQ_REQUIRE(d.dim % 8 == 0 && d.mlp % 8 == 0, REPQ_UNSUPPORTED, "block: dim and mlp must be multiples of 8");
   const int dh = d.dim / d.heads;
   REPQ_REQUIRE(dh % 16 == 0 && dh <= 128, REPQ_UNSUPPORTED, "block: head dim %d must be a multiple of 16, at most 128", dh);

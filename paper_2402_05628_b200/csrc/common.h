@@ -47,8 +47,10 @@ inline bool bits_ok(int b) {
   return (b & ~(0xFF | REPQ_BYTE_CODES)) == 0 && (q == 4 || q == 6 || q == 8);
 }
 inline bool packed4(int b) { return b == 4; }                        // two codes per byte
+inline bool packed6(int b) { return b == (6 | REPQ_PACKED6); }       // four codes in three bytes (weights only)
+inline bool bits_w_ok(int b) { return bits_ok(b) || packed6(b); }
 inline int code_max(int b) { return (1 << quant_bits(b)) - 1; }
-inline int64_t code_row_bytes(int64_t n, int bits) { return packed4(bits) ? (n + 1) / 2 : n; }
+inline int64_t code_row_bytes(int64_t n, int bits) { return packed4(bits) ? (n + 1) / 2 : packed6(bits) ? (n * 3 + 3) / 4 : n; }
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 inline int64_t round_up(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
 

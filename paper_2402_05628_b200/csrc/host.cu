@@ -123,7 +123,7 @@ extern "C" repq_status repq_pack_weights(int N, int K, int bits_w, const float* 
                                          int64_t ld_codes_bytes, float* s_w, int32_t* z_w,
                                          int32_t* w_row_sum) {
   REPQ_REQUIRE(N > 0 && K > 0 && W && codes && s_w && z_w && w_row_sum, REPQ_INVALID_ARG, "pack_weights: bad argument");
-  REPQ_REQUIRE(bits_ok(bits_w), REPQ_INVALID_ARG, "pack_weights: bits must be 4, 6 or 8");
+  REPQ_REQUIRE(bits_w_ok(bits_w), REPQ_INVALID_ARG, "pack_weights: bits must be 4, 6 or 8 (| REPQ_BYTE_CODES) or 6 | REPQ_PACKED6");
   REPQ_REQUIRE(ld_codes_bytes >= code_row_bytes(K, bits_w) && ld_codes_bytes % 16 == 0, REPQ_ALIGNMENT,
                "pack_weights: ld_codes_bytes must cover a row and be a multiple of 16");
   const int qmax = code_max(bits_w);
@@ -151,6 +151,13 @@ extern "C" repq_status repq_pack_weights(int N, int K, int bits_w, const float* 
     memset(out, 0, size_t(ld_codes_bytes));
     if (packed4(bits_w)) {
       for (int c = 0; c < K; ++c) out[c >> 1] |= uint8_t(row[c] << ((c & 1) * 4));
+    } else if (packed6(bits_w)) {
+      for (int c = 0; c < K; ++c) {                 // code c in bits [6c, 6c + 6) of the row
+        const int bit = 6 * c;
+        const uint32_t v = uint32_t(row[c]) << (bit & 7);
+        out[bit >> 3] |= uint8_t(v);
+        if ((bit & 7) > 2) out[(bit >> 3) + 1] |= uint8_t(v >> 8);
+      }
     } else {
       for (int c = 0; c < K; ++c) out[c] = uint8_t(row[c]);
     }

@@ -14,6 +14,20 @@ __global__ void row_sum_kernel(const uint8_t* __restrict__ codes, int bits, int6
   for (int64_t r = warp; r < rows; r += nwarps) {
     const uint8_t* p = codes + r * ld;
     int s = 0;
+    if (bits == 6) {
+      // four codes in three bytes (padding bits of the last group are zero): byte-wise, 24 bits at a time
+      const int64_t nb6 = (n * 3 + 3) / 4;
+      for (int64_t g = lane; g * 3 < nb6; g += 32) {
+        uint32_t f = p[3 * g];
+        if (3 * g + 1 < nb6) f |= uint32_t(p[3 * g + 1]) << 8;
+        if (3 * g + 2 < nb6) f |= uint32_t(p[3 * g + 2]) << 16;
+        s += int((f & 0x3Fu) + ((f >> 6) & 0x3Fu) + ((f >> 12) & 0x3Fu) + (f >> 18));
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+      if (lane == 0) out[r] = s;
+      continue;
+    }
     const bool vec = (reinterpret_cast<uintptr_t>(p) & 15) == 0;
     int64_t b = 0;
     if (vec) {
@@ -77,7 +91,7 @@ __global__ void expand4_kernel(const uint8_t* __restrict__ src, int64_t rows, in
 repq_status validate(const repq_gemm_desc& d) {
   REPQ_REQUIRE(d.M >= 0 && d.N > 0 && d.K > 0, REPQ_INVALID_ARG, "qgemm: M >= 0, N > 0, K > 0 required");
   REPQ_REQUIRE(d.batch_outer > 0 && d.batch_inner > 0, REPQ_INVALID_ARG, "qgemm: batch counts must be positive");
-  REPQ_REQUIRE(bits_ok(d.bits_a) && bits_ok(d.bits_w), REPQ_INVALID_ARG, "qgemm: bits must be 4, 6 or 8");
+  REPQ_REQUIRE(bits_ok(d.bits_a) && bits_w_ok(d.bits_w), REPQ_INVALID_ARG, "qgemm: bits must be 4, 6 or 8");
   if (d.M == 0) return REPQ_OK;
   REPQ_REQUIRE(d.a_codes && d.w_codes && d.out, REPQ_INVALID_ARG, "qgemm: NULL operand or output");
   REPQ_REQUIRE(d.lda_bytes >= code_row_bytes(d.K, d.bits_a) && d.ldw_bytes >= code_row_bytes(d.K, d.bits_w),
@@ -90,6 +104,8 @@ repq_status validate(const repq_gemm_desc& d) {
   if (batched)
     REPQ_REQUIRE(!d.residual && !d.acc_debug && !d.out_row_sum && !d.a_row_sum && !d.w_row_sum, REPQ_UNSUPPORTED,
                  "qgemm: residual / row sums / acc_debug are for plain (unbatched) products");
+  if (packed6(d.bits_w))
+    REPQ_REQUIRE(!batched, REPQ_UNSUPPORTED, "qgemm: REPQ_PACKED6 is for the weights of a plain (unbatched) product");
   const int n_out = d.glu ? d.N / 2 : d.N;        // output columns
   if (d.glu) {
     REPQ_REQUIRE(d.out_groups <= 1, REPQ_UNSUPPORTED, "qgemm: glu takes one output group");
@@ -168,7 +184,7 @@ repq_status launch_row_sum(const uint8_t* codes, int bits, int64_t rows, int64_t
   if (rows == 0) return REPQ_OK;
   const int64_t blocks = (rows + 7) / 8;
   const int grid = int(blocks < 4096 ? blocks : 4096);
-  row_sum_kernel<<<grid, 256, 0, st>>>(codes, packed4(bits) ? 4 : 8, rows, n, ld_bytes, out);
+  row_sum_kernel<<<grid, 256, 0, st>>>(codes, packed4(bits) ? 4 : packed6(bits) ? 6 : 8, rows, n, ld_bytes, out);
   REPQ_CUDA(cudaGetLastError());
   note_launch();
   return REPQ_OK;

@@ -25,6 +25,17 @@ struct MmaOperand {
 // beyond K.  `aligned4` says base and ld allow 32-bit / 16-bit loads at these offsets.
 __device__ __forceinline__ uint32_t load_codes4(const uint8_t* row, int k0, int K, int bits, bool aligned4) {
   if (k0 >= K) return 0u;
+  if (bits == 6) {
+    // four codes in three bytes: the 24 bits at byte 3 k0 / 4 of the row
+    const uint8_t* p = row + (k0 >> 2) * 3;
+    const int left = K - k0;
+    uint32_t f = p[0];
+    if (left > 1) f |= uint32_t(p[1]) << 8;
+    if (left > 2) f |= uint32_t(p[2]) << 16;
+    uint32_t r = (f & 0x3Fu) | ((f & 0xFC0u) << 2) | ((f & 0x3F000u) << 4) | ((f & 0xFC0000u) << 6);
+    if (left < 4) r &= (1u << (8 * left)) - 1u;
+    return r;
+  }
   if (bits == 4) {
     const uint8_t* p = row + (k0 >> 1);
     uint32_t w;
@@ -229,7 +240,7 @@ qgemm_mma_kernel(MmaOperand A, MmaOperand W, int K, int batch_inner, int64_t a_s
 
 repq_status qgemm_mma(const repq_gemm_desc& d, const EpilogueParams& ep, cudaStream_t st) {
   MmaOperand A{d.a_codes, d.lda_bytes, d.M, packed4(d.bits_a) ? 4 : 8};
-  MmaOperand W{d.w_codes, d.ldw_bytes, d.N, packed4(d.bits_w) ? 4 : 8};
+  MmaOperand W{d.w_codes, d.ldw_bytes, d.N, packed4(d.bits_w) ? 4 : packed6(d.bits_w) ? 6 : 8};
   auto al = [](const uint8_t* p, int64_t ld, int64_t so, int64_t si, int bits) {
     const int64_t unit = packed4(bits) ? 2 : 4;
     return aligned(p, size_t(unit)) && ld % unit == 0 && so % unit == 0 && si % unit == 0;

@@ -11,10 +11,10 @@
 //                the main loop of tile i + 1
 //   warps 2..17  epilogue: warp w reads TMEM lanes 32 (w mod 4) .. +31 (one output row per thread) and a
 //                64-column slice of the accumulator columns
-//   packed 4-bit weights: 12 epilogue warps (tiles of at most 192 columns) and 4 converter warps.  The weight tile
-//                arrives packed, two codes per byte, and the converters expand it into the 128-byte-swizzled byte tile
-//                the MMA descriptor expects (there is no 4-bit integer MMA); one more barrier hop between the copy
-//                and the MMA, weights stay packed in HBM
+//   packed weights (4-bit, two codes per byte; 6-bit, four codes in three bytes): 12 epilogue warps (tiles of at most
+//                192 columns) and 4 converter warps.  The weight tile arrives packed and the converters expand it into
+//                the 128-byte-swizzled byte tile the MMA descriptor expects (there is no 4- or 6-bit integer MMA); one
+//                more barrier hop between the copy and the MMA, weights stay packed in HBM
 // The tile width BN (256, 192 or 128) is chosen per problem: rounds of tiles over the SMs times a per-round time
 // with a fixed part.  Packed 4-bit activations are expanded to one code per byte by a separate pass into the
 // workspace (inside the block the producers write byte codes, so that pass does not run there).
@@ -71,12 +71,15 @@ constexpr uint32_t kResBytes = 32 * 128;            // bf16 residual of one warp
 
 // RES: the bf16 residual of a tile comes in by bulk tensor copies, one 32 x 64 box per epilogue warp, asked for one
 // tile ahead (the operand ring gives up a stage for the boxes)
-template <int BN, bool RES, bool W4>
+// WP: 0 = weight tiles arrive as bytes; 4 / 6 = packed (64 / 96 bytes per row of 128 codes), expanded by the converters
+template <int BN, bool RES, int WP>
 struct SharedStorage {
+  static constexpr bool W4 = WP != 0;               // (any packed form)
   // kStages: ring of the bulk copies (activation tile + weight tile as it arrives).  kStagesB: ring of byte weight
   // tiles the MMA reads: the same ring when the weights arrive as bytes; with packed weights a short ring of its own
   // (the hop from converter to MMA is short), which leaves room for a deeper copy ring ahead of the converters.
-  static constexpr int kStages = W4 ? 5 : (RES ? 3 : 4);
+  static constexpr int kStages = WP == 6 ? 4 : WP == 4 ? 5 : (RES ? 3 : 4);
+  static constexpr int kPackedRow = BK * (WP ? WP : 8) / 8;        // bytes of a packed tile row
   static constexpr int kStagesB = W4 ? 2 : kStages;
   static constexpr int kEpi = W4 ? kEpiWarpsW4 : kEpiWarps;
   alignas(1024) uint8_t a[kStages][kABytes];
@@ -85,7 +88,7 @@ struct SharedStorage {
   uint64_t res_full[kEpiWarps];
   alignas(1024) uint8_t epi[kEpi][1024];          // per-warp staging box of the epilogue's bulk stores
   ColTerms cols[kEpi];                            // each epilogue warp stages the terms of its own slice: no barrier
-  alignas(128) uint8_t bp[W4 ? kStages : 1][W4 ? BN * BK / 2 : 128];   // packed weight tiles: rows of 64 bytes, unswizzled
+  alignas(128) uint8_t bp[W4 ? kStages : 1][W4 ? BN * kPackedRow : 128];   // packed weight tiles: unswizzled rows
   alignas(8) uint64_t full[kStages];
   uint64_t empty[kStages];
   uint64_t ready[kStagesB];                         // packed variant: byte weight tile written by the converters
@@ -97,8 +100,9 @@ struct SharedStorage {
   volatile int abort;
 };
 
-static_assert(sizeof(SharedStorage<kMaxBN, false, false>) <= 227 * 1024 && sizeof(SharedStorage<kMaxBNW4, false, true>) <= 227 * 1024 &&
-              sizeof(SharedStorage<192, true, false>) <= 227 * 1024, "shared storage exceeds the 227 KB a CTA may use");
+static_assert(sizeof(SharedStorage<kMaxBN, false, 0>) <= 227 * 1024 && sizeof(SharedStorage<kMaxBNW4, false, 4>) <= 227 * 1024 &&
+              sizeof(SharedStorage<kMaxBNW4, false, 6>) <= 227 * 1024 && sizeof(SharedStorage<192, true, 0>) <= 227 * 1024,
+              "shared storage exceeds the 227 KB a CTA may use");
 
 using namespace tc;
 
@@ -119,7 +123,8 @@ struct TcParams {
   const int32_t* asum;
   const int32_t* wsum;
   int direct_requant;          // codes out, no GELU, no residual: 1/s_o is folded into the column terms
-  int w_packed4;               // weight tiles arrive packed (two codes per byte) and are expanded in shared memory
+  int w_packed4;               // weight tiles arrive packed (4: two codes per byte, 6: four in three bytes) and are
+                               // expanded in shared memory; 0: byte tiles
   int panel;                   // row tiles per panel of the tile order
   EpilogueParams ep;
 };
@@ -363,11 +368,12 @@ __device__ __noinline__ void slow_chunk(const EpilogueParams& ep, const TcParams
 // where asked for: kPairNone, kPairRope (rotary embedding), kPairGlu (gated product; byte codes out)
 enum : int { kPairNone = 0, kPairRope = 1, kPairGlu = 2 };
 
-template <int BN, int OUT, bool RES, int PAIR, bool W4>
+template <int BN, int OUT, bool RES, int PAIR, int WP>
 __global__ void __launch_bounds__(kThreads, 1)
 qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_res, TcParams P) {
-  using Storage = SharedStorage<BN, RES, W4>;
+  using Storage = SharedStorage<BN, RES, WP>;
+  constexpr bool W4 = WP != 0;                           // weights arrive packed
   constexpr int kStages = Storage::kStages;
   constexpr int EW = W4 ? kEpiWarpsW4 : kEpiWarps;       // epilogue warps of this variant
   static_assert(!W4 || BN <= kMaxBNW4, "the packed-weight variant has three column slices");
@@ -423,9 +429,9 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!mbar_wait(smem_u32(&S.empty[stage]), phase ^ 1, abort, 1)) break;
           const uint32_t bar = smem_u32(&S.full[stage]);
-          mbar_expect_tx(bar, kABytes + (W4 ? kBBytes / 2 : kBBytes));
+          mbar_expect_tx(bar, kABytes + (W4 ? uint32_t(BN * Storage::kPackedRow) : kBBytes));
           tma_load_2d(smem_u32(S.a[stage]), &map_a, bar, kb * BK, m0);
-          if constexpr (W4) tma_load_2d(smem_u32(S.bp[stage]), &map_b, bar, kb * (BK / 2), n0);
+          if constexpr (W4) tma_load_2d(smem_u32(S.bp[stage]), &map_b, bar, kb * Storage::kPackedRow, n0);
           else tma_load_2d(smem_u32(S.b[stage]), &map_b, bar, kb * BK, n0);
           ++issued;
           if (++stage == kStages) { stage = 0; phase ^= 1; }
@@ -489,6 +495,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         // the packed tile has landed, and the MMAs that read the byte tile's previous content have completed
         if (!mbar_wait(smem_u32(&S.full[stage]), phase, abort, 7)) { ok = false; break; }
         if (!mbar_wait(smem_u32(&S.bfree[bstage]), bphase ^ 1, abort, 8)) { ok = false; break; }
+        if constexpr (WP == 4) {
         // pieces ct, ct + 128, ...: the row advances by 32 per step, so the row's position inside its group of eight
         // (hence the swizzle) is the thread's own; the pieces of a batch are loaded before any is expanded
         const uint4* src = reinterpret_cast<const uint4*>(S.bp[stage]) + ct;
@@ -516,6 +523,25 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             *reinterpret_cast<uint4*>(d0 + (i0 + u) * 4096) = make_uint4(o[0], o[1], o[2], o[3]);
             *reinterpret_cast<uint4*>(d1 + (i0 + u) * 4096) = make_uint4(o[4], o[5], o[6], o[7]);
           }
+        }
+        } else {
+        // 6-bit codes: a packed row is 96 bytes; output piece p of row n (16 codes) comes from the 12 bytes at 12 p of
+        // that row.  Thread ct takes pieces ct, ct + 128, ...: row (ct >> 3) + 16 per step, piece ct & 7.  The three
+        // words of a warp's 32 pieces fall on 32 different banks (word index 24 n + 3 p).
+        const int n_lo = (ct >> 3) & 7, pc = ct & 7;
+        const uint32_t* src = reinterpret_cast<const uint32_t*>(S.bp[stage]) + (ct >> 3) * 24 + pc * 3;
+        uint8_t* dst = S.b[bstage] + uint32_t(ct >> 6) * 1024u + uint32_t(n_lo) * 128u + (uint32_t(pc ^ n_lo) << 4);
+        constexpr int kSteps = BN * 8 / kConvThreads;                      // 16-row steps per thread
+        auto spread = [](uint32_t f) {      // four 6-bit fields of f[23:0] -> four bytes
+          return (f & 0x3Fu) | ((f & 0xFC0u) << 2) | ((f & 0x3F000u) << 4) | ((f & 0xFC0000u) << 6);
+        };
+#pragma unroll 2
+        for (int i = 0; i < kSteps; ++i) {
+          const uint32_t w0 = src[i * 16 * 24], w1 = src[i * 16 * 24 + 1], w2 = src[i * 16 * 24 + 2];
+          const uint32_t o0 = spread(w0), o1 = spread(__funnelshift_r(w0, w1, 24)), o2 = spread(__funnelshift_r(w1, w2, 16)),
+                         o3 = spread(w2 >> 8);
+          *reinterpret_cast<uint4*>(dst + i * 2048) = make_uint4(o0, o1, o2, o3);
+        }
         }
         fence_async_smem();
         __syncwarp();
@@ -849,17 +875,17 @@ repq_status make_res_map(CUtensorMap* map, const TcParams& P) {
   return REPQ_OK;
 }
 
-template <int BN, int OUT, bool RES, int PAIR, bool W4>
+template <int BN, int OUT, bool RES, int PAIR, int WP>
 repq_status launch_tc_w(const CUtensorMap& map_a, const CUtensorMap& map_b, const TcParams& P, int sms, cudaStream_t st) {
   CUtensorMap map_out, map_res;
   REPQ_TRY(make_out_map(&map_out, P));
   if (RES) REPQ_TRY(make_res_map(&map_res, P));
   else map_res = map_out;                                  // not read
-  const size_t smem = sizeof(SharedStorage<BN, RES, W4>);
-  REPQ_CUDA(cudaFuncSetAttribute(qgemm_tc_kernel<BN, OUT, RES, PAIR, W4>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+  const size_t smem = sizeof(SharedStorage<BN, RES, WP>);
+  REPQ_CUDA(cudaFuncSetAttribute(qgemm_tc_kernel<BN, OUT, RES, PAIR, WP>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
   const int tiles = ((P.M + BM - 1) / BM) * ((P.N + BN - 1) / BN);
   const int grid = tiles < sms ? tiles : sms;
-  REPQ_CUDA(launch_chained(qgemm_tc_kernel<BN, OUT, RES, PAIR, W4>, dim3(grid), dim3(kThreads), smem, st, map_a, map_b, map_out, map_res, P));
+  REPQ_CUDA(launch_chained(qgemm_tc_kernel<BN, OUT, RES, PAIR, WP>, dim3(grid), dim3(kThreads), smem, st, map_a, map_b, map_out, map_res, P));
   note_launch();
   return REPQ_OK;
 }
@@ -867,9 +893,10 @@ repq_status launch_tc_w(const CUtensorMap& map_a, const CUtensorMap& map_b, cons
 template <int BN, int OUT, bool RES, int PAIR = kPairNone>
 repq_status launch_tc_res(const CUtensorMap& map_a, const CUtensorMap& map_b, const TcParams& P, int sms, cudaStream_t st) {
   if constexpr (!RES && BN <= kMaxBNW4) {
-    if (P.w_packed4) return launch_tc_w<BN, OUT, false, PAIR, true>(map_a, map_b, P, sms, st);
+    if (P.w_packed4 == 4) return launch_tc_w<BN, OUT, false, PAIR, 4>(map_a, map_b, P, sms, st);
+    if (P.w_packed4 == 6) return launch_tc_w<BN, OUT, false, PAIR, 6>(map_a, map_b, P, sms, st);
   }
-  return launch_tc_w<BN, OUT, RES, PAIR, false>(map_a, map_b, P, sms, st);
+  return launch_tc_w<BN, OUT, RES, PAIR, 0>(map_a, map_b, P, sms, st);
 }
 
 template <int BN, int OUT>
@@ -961,7 +988,7 @@ repq_status qgemm_tc(const repq_gemm_desc& d, const EpilogueParams& ep, void* ws
     a = w8 + L.off_a; lda = L.ld_a;
   }
   TcParams P{};
-  P.w_packed4 = packed4(d.bits_w);
+  P.w_packed4 = packed4(d.bits_w) ? 4 : packed6(d.bits_w) ? 6 : 0;
   P.M = d.M; P.N = d.N; P.K = d.K;
   P.asum = d.a_row_sum;
   if (!P.asum) {
@@ -989,7 +1016,7 @@ repq_status qgemm_tc(const repq_gemm_desc& d, const EpilogueParams& ep, void* ws
   }
   CUtensorMap map_a, map_b;
   REPQ_TRY(make_map(&map_a, a, d.M, d.K, lda, BM));
-  if (P.w_packed4) REPQ_TRY(make_map(&map_b, d.w_codes, d.N, (int64_t(d.K) + 1) / 2, d.ldw_bytes, bn, BK / 2, false));
+  if (P.w_packed4) REPQ_TRY(make_map(&map_b, d.w_codes, d.N, code_row_bytes(d.K, d.bits_w), d.ldw_bytes, bn, BK * P.w_packed4 / 8, false));
   else REPQ_TRY(make_map(&map_b, d.w_codes, d.N, d.K, d.ldw_bytes, bn));
   if (bn == 256) return launch_tc<256>(map_a, map_b, P, sms, st);
   if (bn == 192) return launch_tc<192>(map_a, map_b, P, sms, st);

@@ -43,8 +43,9 @@ class QuantBlock:
 
     def __init__(self, w, device="cuda:0", out_dtype: Optional[torch.dtype] = None, staged_attention: bool = False,
                  weight_storage: str = "bytes"):
-        """weight_storage: "packed" keeps 4-bit weight codes two per byte in device memory (the GEMM expands the
-        tiles in shared memory); "bytes" keeps one code per byte, the tensor-core operand format."""
+        """weight_storage: "packed" keeps 4-bit weight codes two per byte and 6-bit codes four to three bytes in device
+        memory (the GEMM expands the tiles in shared memory); "bytes" keeps one code per byte, the tensor-core operand
+        format."""
         assert weight_storage in ("packed", "bytes")
         self.weight_storage = weight_storage
         self.staged_attention = bool(staged_attention)
@@ -53,7 +54,11 @@ class QuantBlock:
         dev = torch.device(device)
         self.device = dev
         ba = cfg["bits_a"]
-        bw = self.bits_w = cfg["bits_w"] if weight_storage == "packed" else cfg["bits_w"] | B.REPQ_BYTE_CODES
+        if weight_storage == "packed":
+            bw = cfg["bits_w"] | B.REPQ_PACKED6 if cfg["bits_w"] == 6 else cfg["bits_w"]
+        else:
+            bw = cfg["bits_w"] | B.REPQ_BYTE_CODES
+        self.bits_w = bw
         self.host: Dict[str, object] = {}
 
         def fold(gamma, beta, lo, hi, W, b, tag):

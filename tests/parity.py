@@ -11,6 +11,7 @@ MAX_ABS_TOL = 1e-2         # float outputs: max abs error as a fraction of max |
 
 
 BYTE_CODES = 0x100         # flag of the C ABI: a `bits` value with it set stores one code per byte
+PACKED6 = 0x200            # 6 | PACKED6: weight codes stored four to three bytes
 
 
 def qb(bits: int) -> int:
@@ -35,6 +36,14 @@ def pack_codes(q: np.ndarray, bits: int, ld_bytes: int) -> np.ndarray:
     q = np.asarray(q, dtype=np.uint8)
     rows, n = q.shape
     out = np.zeros((rows, ld_bytes), dtype=np.uint8)
+    if bits == (6 | PACKED6):
+        # code i in bits [6i, 6i + 6) of the row read as a little-endian bit string
+        bits_le = ((q[:, :, None] >> np.arange(6, dtype=np.uint8)[None, None, :]) & 1).reshape(rows, n * 6)
+        pad = (-bits_le.shape[1]) % 8
+        bits_le = np.concatenate([bits_le, np.zeros((rows, pad), dtype=np.uint8)], axis=1)
+        packed = np.packbits(bits_le, axis=1, bitorder="little")
+        out[:, : packed.shape[1]] = packed
+        return out
     if bits == 4:
         if n % 2:
             q = np.concatenate([q, np.zeros((rows, 1), dtype=np.uint8)], axis=1)
@@ -1114,7 +1123,7 @@ def check_softmax_log2_sampled(rows, L, bits, n_sample=64, seed=4):
     return rep
 
 
-def check_qgemm_sampled(M, N, K, qbits, out_kind, n_sample=24, seed=4, weights="bytes"):
+def check_qgemm_sampled(M, N, K, qbits, out_kind, n_sample=24, seed=4, weights="bytes"):  # weights: "bytes" | "packed"
     """repq_qgemm at a sweep size with the operand formats the benchmark times, the oracle on sampled rows."""
     import torch
     from oracle import repq_oracle as orc
@@ -1122,7 +1131,7 @@ def check_qgemm_sampled(M, N, K, qbits, out_kind, n_sample=24, seed=4, weights="
 
     rng = np.random.default_rng(seed)
     bits = qbits | BYTE_CODES
-    bits_w = qbits if weights == "packed" else bits
+    bits_w = (qbits | PACKED6 if qbits == 6 else qbits) if weights == "packed" else bits
     a = rng.integers(0, 1 << qbits, size=(M, K), dtype=np.uint8)
     wq = rng.integers(0, 1 << qbits, size=(N, K), dtype=np.uint8)
     s_a, z_a = np.float32(0.07), int(rng.integers(0, 1 << qbits))

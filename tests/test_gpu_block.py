@@ -92,18 +92,20 @@ def test_calibration_pipeline_matches_oracle(name, batch, overrides):
 
 
 def test_block_with_byte_wide_weight_storage():
-    """4-bit weights kept one code per byte in device memory instead of packed: same block."""
+    """Weights kept one code per byte in device memory or packed (4-bit: two per byte, 6-bit: four to three bytes):
+    the same block output, bit for bit."""
     import numpy as np
     import torch
     from paper_2402_05628_b200.engine import QuantBlock
     from workloads import make_block_inputs
-    w = make_block_inputs("c2_deit_b", batch=3)
-    a, b = QuantBlock(w, weight_storage="packed"), QuantBlock(w, weight_storage="bytes")
-    assert a.qkv.codes.shape[1] * 2 == b.qkv.codes.shape[1]
-    x = torch.from_numpy(np.ascontiguousarray(w.x)).to(a.device).to(a.act_dtype)
-    ya, yb = a.forward(x), b.forward(x)
-    torch.cuda.synchronize()
-    assert torch.equal(ya, yb)
+    for name, ratio in (("c2_deit_b", 2.0), ("c2_deit_b_w6a6", 4.0 / 3.0)):
+        w = make_block_inputs(name, batch=3)
+        a, b = QuantBlock(w, weight_storage="packed"), QuantBlock(w, weight_storage="bytes")
+        assert a.qkv.codes.shape[1] * ratio == b.qkv.codes.shape[1]
+        x = torch.from_numpy(np.ascontiguousarray(w.x)).to(a.device).to(a.act_dtype)
+        ya, yb = a.forward(x), b.forward(x)
+        torch.cuda.synchronize()
+        assert torch.equal(ya, yb)
 
 
 def test_block_with_the_three_separate_attention_stages():

@@ -236,6 +236,7 @@ def test_softmax_log2_at_sweep_sizes_sampled_rows(rows, L, bits):
     (16384, 2304, 768, 4, "codes", "bytes"), (16384, 768, 3072, 8, "bf16", "bytes"), (16384, 12288, 4096, 4, "codes", "bytes"),
     (16384, 4096, 11008, 4, "bf16", "bytes"), (65536, 768, 768, 4, "codes", "bytes"), (2048, 4096, 4096, 8, "codes", "bytes"),
     (16384, 11008, 4096, 4, "codes", "packed"), (8192, 4096, 11008, 4, "bf16", "packed"),
+    (12608, 2304, 768, 6, "codes", "packed"), (8192, 4096, 4096, 6, "bf16", "packed"),
 ])
 def test_qgemm_at_sweep_sizes_sampled_rows(M, N, K, qbits, out_kind, weights):
     parity.check_qgemm_sampled(M, N, K, qbits, out_kind, weights=weights)
@@ -257,3 +258,15 @@ def test_dual_clip_leaves_a_constant_channel_alone():
     assert float(lo[5]) == float(hi[5]) == 0.375 and float(lo[9]) == float(hi[9]) == 0.0       # sigmoid(0) = 1/2 of the extremes
     assert float(loss[5]) == 0.0 and float(loss[16 + 5]) == 0.0
     assert (hi[[0, 1, 2]] > lo[[0, 1, 2]]).all()
+
+
+@pytest.mark.parametrize("M,N,K,out_kind", [
+    (300, 192, 256, "f32"), (389, 576, 384, "codes"), (700, 512, 1000, "bf16"), (130, 72, 100, "f32"), (33, 17, 50, "f32"),
+    (64, 64, 4, "f32"),
+])
+def test_qgemm_six_bit_weights_packed_four_to_three_bytes(M, N, K, out_kind):
+    """Weights stored 6 | REPQ_PACKED6 (tensor-core kernel: expanded in shared memory; small or ragged shapes: the
+    warp-MMA kernel), int32 accumulators bit-exact where they are dumped."""
+    b6 = 6 | parity.BYTE_CODES
+    parity.check_qgemm(M, N, K, b6, 6 | parity.PACKED6, out_kind=out_kind, out_bits=b6, seed=M + K, give_sums=(M % 2 == 0),
+                       want_acc=(out_kind == "f32"))

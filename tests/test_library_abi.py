@@ -118,3 +118,17 @@ def test_rope_table_rotates_like_the_oracle(B):
     assert t[0, :, 0].tolist() == [1.0] * (dh // 2) and t[0, :, 1].tolist() == [0.0] * (dh // 2)
     with pytest.raises(B.RepqError):
         B.repq_rope_table(L, 7, 10000.0)
+
+
+def test_pack_weights_six_bit_layout(B):
+    """6 | REPQ_PACKED6: the same codes as the byte form, four to three bytes, code i in bits [6i, 6i + 6)."""
+    from tests.parity import PACKED6, BYTE_CODES, pack_codes
+    rng = np.random.default_rng(12)
+    W = rng.normal(0, 0.02, (9, 53)).astype(np.float32)
+    c8, s8, z8, sum8 = B.repq_pack_weights(W, 6 | BYTE_CODES)
+    c6, s6, z6, sum6 = B.repq_pack_weights(W, 6 | PACKED6)
+    assert np.array_equal(s8, s6) and np.array_equal(z8, z6) and np.array_equal(sum8, sum6)
+    assert c6.shape[1] == B.code_row_bytes(53, 6 | PACKED6) == 48
+    assert np.array_equal(c6, pack_codes(c8[:, :53], 6 | PACKED6, c6.shape[1]))
+    bits = np.unpackbits(c6, axis=1, bitorder="little")[:, : 53 * 6].reshape(9, 53, 6)
+    assert np.array_equal((bits * (1 << np.arange(6))).sum(axis=2), c8[:, :53])
