@@ -268,7 +268,12 @@ repq_status repq_pv(const repq_pv_desc* d, void* stream);
  * for batch_outer x batch_inner (batch, head) pairs.  q, k, v [device]: codes of one quantizer width, stored one
  * per byte (bits_qkv must carry REPQ_BYTE_CODES); operand (bo, bi) starts at base + bo*stride_outer +
  * bi*stride_inner; Q and K rows 16-byte aligned, V rows 8-byte aligned.  d_h a multiple of 16, at most 128.
- * Output as in repq_pv. */
+ * Output as in repq_pv.
+ * For 4-bit Q / K quantizers with 0 <= z_q <= 15 the score contraction runs on the tensor cores' 8-bit float type
+ * (the operands are integers of at most 15 in magnitude, exactly representable; products and sums are exact in the
+ * float32 accumulator), which saves the integer -> float conversion of every score; the result is bit-identical to
+ * the integer contraction, which the environment variable REPQ_ATTENTION_INT_SCORES=1 (read at every call) selects
+ * instead. */
 typedef struct repq_attention_desc {
   int32_t batch_outer, batch_inner, Lq, Lk, d_h;
   int32_t bits_qkv;

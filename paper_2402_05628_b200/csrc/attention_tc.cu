@@ -29,6 +29,7 @@
 
 #include <cstdlib>
 
+#include "f32x2.cuh"
 #include "kernels.h"
 #include "tc_ptx.cuh"
 
@@ -49,7 +50,6 @@ constexpr uint32_t kKBytes = kKeys * 128;
 constexpr uint32_t kTileBytes = kRows * 128;      // E or O tile of one block (64 keys of bf16 per row)
 constexpr uint32_t kVBlockBytes = kKeys * 128;    // 64 keys x 64 channels of bf16
 constexpr uint32_t kMagicBits = 0x4B400000u;      // float 1.5 * 2^23
-constexpr int kAccCol = 2 * kKeys;                // first tensor-memory column of the P.V accumulators
 
 struct AttnParams {
   const uint8_t* q; const uint8_t* k; const uint8_t* v;
@@ -66,17 +66,26 @@ struct AttnParams {
   void* out; int64_t ldo, o_so, o_si;
   int32_t* out_row_sum;
   int n_pad, tmem_cols, vec_store;
+  int no_f8;                                         // keep integer scores where the 8-bit float form would apply
   int pairs, tiles;                                  // (batch, head) pairs and query tiles of 128 rows: the grid is their product
   int32_t* status;
 };
 
+// Ring depths.  Heads of up to 64 channels run two CTAs per SM (256 tensor-memory columns and about 80 KB of shared
+// memory each), which overlap each other's waits: S and K double-buffered, one stage of operand tiles.  Wider heads
+// have the SM to themselves: four S buffers in tensor memory (4 x 64 columns beside the 2 x 128 of the accumulators),
+// four K tiles and two stages of E / O / V tiles, so that neither the S MMAs' round trip nor the P.V MMAs of the block
+// before stand between a worker warp and its next block.
+template <int NB> struct Rings { static constexpr int kS = NB == 1 ? 2 : 4, kK = NB == 1 ? 2 : 4, kP = NB == 1 ? 1 : 2; };
+
 template <int NB, int kLutBits>
 struct AttnShared {
+  static constexpr int kS = Rings<NB>::kS, kK = Rings<NB>::kK, kP = Rings<NB>::kP;
   alignas(1024) uint8_t q[kQBytes];
-  alignas(1024) uint8_t k[2][kKBytes];
-  alignas(1024) uint8_t e[kTileBytes];
-  alignas(1024) uint8_t o[kTileBytes];
-  alignas(1024) uint8_t v[NB * kVBlockBytes];
+  alignas(1024) uint8_t k[kK][kKBytes];
+  alignas(1024) uint8_t e[kP][kTileBytes];
+  alignas(1024) uint8_t o[kP][kTileBytes];
+  alignas(1024) uint8_t v[kP][NB * kVBlockBytes];
   int row_term[kRows];                              // -z_k qsum[m] + d_h z_q z_k
   int col_term[4][kKeys];                           // -z_q ksum[n], ring of 4 key blocks
   float stat_m[kParts][kRows], stat_z[kParts][kRows];   // pass-1 results of the column parts of every row
@@ -84,9 +93,9 @@ struct AttnShared {
   uint32_t lut[kLutEntries][32];                    // table-driven codes: [code][lane] = E value | O value << 16 (one bank per
                                                     // lane); the last entry repeats the top code (a clamp at 2^bits that
                                                     // rounds up lands there)
-  alignas(8) uint64_t k_full[2];
-  uint64_t k_empty[2];                              // K tile read by its S MMAs (bulk-copy variant)
-  uint64_t s_full[2], s_empty[2], p_full, p_empty;
+  alignas(8) uint64_t k_full[kK];
+  uint64_t k_empty[kK];                             // K tile read by its S MMAs (bulk-copy variant)
+  uint64_t s_full[kS], s_empty[kS], p_full[kP], p_empty[kP];
   uint64_t stats_ready, acc_full, done;
   uint32_t tmem_base;
   volatile int abort;
@@ -104,6 +113,16 @@ __device__ __forceinline__ uint32_t sub_bytes(uint32_t c, uint32_t z4) { return 
 __device__ __forceinline__ uint4 sub_bytes(const uint4& c, uint32_t z4) {
   return make_uint4(sub_bytes(c.x, z4), sub_bytes(c.y, z4), sub_bytes(c.z, z4), sub_bytes(c.w, z4));
 }
+// Bytes in two's complement (within [-127, 127]) -> sign bit and magnitude.
+__device__ __forceinline__ uint32_t sign_magnitude(uint32_t x) { return __vabs4(x) | (x & 0x80808080u); }
+__device__ __forceinline__ uint4 sign_magnitude(const uint4& c) {
+  return make_uint4(sign_magnitude(c.x), sign_magnitude(c.y), sign_magnitude(c.z), sign_magnitude(c.w));
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -112,14 +131,29 @@ __device__ __forceinline__ float ex2(float x) {
 
 // NB: 64-channel blocks of the head; kLutBits: width of the Softmax codes when their operand values come from the
 // per-lane table (4, 6, or 8 where one CTA per SM leaves room for 257 entries), 0: integer arithmetic
-// kCentered: Q and K codes minus their zero points fit a signed byte (quantizers of at most 7 bits); the tiles then
-// hold q - z_q and k - z_k, the S MMAs run signed x signed and their accumulators need no zero-point correction.
-template <int NB, int kLutBits, bool kCentered>
+// kMode: how the scores are formed.
+//   kCorrected  unsigned Q and K tiles, accumulators corrected by the row and column zero-point terms
+//   kCentred    q - z_q fits a signed byte (quantizers of at most 7 bits): the Q tile holds q - z_q, the K tile the raw
+//               codes, the S MMAs run signed x unsigned and their accumulators need no correction
+//   kCentredF8  4-bit quantizers (|q - z_q| <= 15, k <= 15): the same tiles read as 8-bit floats.  A byte below 16 is
+//               the e4m3 number byte * 2^-9 (subnormals and the first binade are linear in the byte), so the raw K codes
+//               are already such numbers and the Q tile stores sign and magnitude of q - z_q.  Products and sums are
+//               multiples of 2^-18 below 2^-3, exact in the float32 accumulator, which therefore holds
+//               2^-18 sum (q - z_q) k as a float: the int -> float conversion of every score is gone (the factor 2^18 is
+//               folded into the score scale on the host, exactly)
+enum : int { kCorrected = 0, kCentred = 1, kCentredF8 = 2 };
+template <int NB, int kLutBits, int kMode>
 __global__ void __launch_bounds__(kThreads, NB == 1 ? 2 : 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
   using Shared = AttnShared<NB, kLutBits>;
   constexpr bool kLut = kLutBits != 0;
+  constexpr bool kCentered = kMode != kCorrected;
+  constexpr bool kF8 = kMode == kCentredF8;
   constexpr int kVItems = NB;                             // 8-channel groups of V per thread and block
+  constexpr int kS = Shared::kS, kK = Shared::kK, kP = Shared::kP;      // ring depths (powers of two)
+  constexpr int kAccCol = kS * kKeys;                     // first tensor-memory column of the P.V accumulators
+  auto ring = [](int i, int depth) { return i & (depth - 1); };
+  auto lap = [](int i, int depth) { return uint32_t(i / depth) & 1u; };       // parity of the slot's use count
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   Shared& S = *reinterpret_cast<Shared*>(smem_raw);
 
@@ -147,14 +181,18 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
   const int pieces = P.dh >> 4;                           // 16-byte pieces of a Q / K row
 
   if (tid == 0) {
-    for (int s = 0; s < 2; ++s) {
+    for (int s = 0; s < kK; ++s) {
       mbar_init(smem_u32(&S.k_full[s]), kCentered ? 1 : kWorkWarps);
       mbar_init(smem_u32(&S.k_empty[s]), 1);
+    }
+    for (int s = 0; s < kS; ++s) {
       mbar_init(smem_u32(&S.s_full[s]), 1);
       mbar_init(smem_u32(&S.s_empty[s]), kWorkWarps);
     }
-    mbar_init(smem_u32(&S.p_full), kWorkWarps);
-    mbar_init(smem_u32(&S.p_empty), 1);
+    for (int s = 0; s < kP; ++s) {
+      mbar_init(smem_u32(&S.p_full[s]), kWorkWarps);
+      mbar_init(smem_u32(&S.p_empty[s]), 1);
+    }
     mbar_init(smem_u32(&S.stats_ready), kWorkWarps);
     mbar_init(smem_u32(&S.acc_full), 1);
     mbar_init(smem_u32(&S.done), 1);
@@ -210,6 +248,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
       if (q0 + qrow < P.Lq && piece < pieces) {
         w = __ldg(reinterpret_cast<const uint4*>(q_base + int64_t(q0 + qrow) * P.ldq) + piece);
         if (kCentered) w = sub_bytes(w, zq4);
+        if (kF8) w = sign_magnitude(w);
       }
       if (piece < 2 * ksteps) *reinterpret_cast<uint4*>(S.q + tile_offset(qrow, piece)) = w;
       s += sum_bytes(w);
@@ -236,34 +275,46 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
     if (lane == 0) {
       // S: D = s32, A = B = unsigned 8-bit, both K-major, N = 64, M = 128
       // (operand formats: 0 = unsigned, 1 = signed bytes)
-      constexpr uint32_t idesc_s = (2u << 4) | (uint32_t(kCentered) << 7) | (0u << 10) | (uint32_t(kKeys >> 3) << 17) |
-                                   (uint32_t(kRows >> 4) << 24);
+      // kCentredF8: D = f32, A = B = e4m3 (format 0)
+      constexpr uint32_t idesc_s = kF8 ? (1u << 4) | (uint32_t(kKeys >> 3) << 17) | (uint32_t(kRows >> 4) << 24)
+                                       : (2u << 4) | (uint32_t(kCentered) << 7) | (0u << 10) | (uint32_t(kKeys >> 3) << 17) |
+                                             (uint32_t(kRows >> 4) << 24);
       // P.V: D = f32, A = B = bf16, A K-major, B MN-major, N = n_pad, M = 128
       const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (uint32_t(P.n_pad >> 3) << 17) |
                                 (uint32_t(kRows >> 4) << 24);
       const uint64_t dq = smem_desc_sw128(smem_u32(S.q));
       bool ok = true;
       auto issue_s = [&](int g) {                          // S of key block g % nb, g counted over both passes
-        const int b = g & 1;
-        const uint32_t ph = uint32_t(g >> 1) & 1u;
-        if (!mbar_wait(smem_u32(&S.k_full[b]), ph, abort, 41, P.status)) return false;
-        if (!mbar_wait(smem_u32(&S.s_empty[b]), ph ^ 1u, abort, 42, P.status)) return false;
+        const int b = ring(g, kS), kb = ring(g, kK);
+        if (!mbar_wait(smem_u32(&S.k_full[kb]), lap(g, kK), abort, 41, P.status)) return false;
+        if (!mbar_wait(smem_u32(&S.s_empty[b]), lap(g, kS) ^ 1u, abort, 42, P.status)) return false;
         tc_fence_after();
-        const uint64_t dk = smem_desc_sw128(smem_u32(S.k[b]));
-        for (int s = 0; s < ksteps; ++s)
-          umma_i8(tmem_base + uint32_t(b * kKeys), dq + uint64_t(2 * s), dk + uint64_t(2 * s), idesc_s, s != 0 ? 1u : 0u);
+        const uint64_t dk = smem_desc_sw128(smem_u32(S.k[kb]));
+        for (int s = 0; s < ksteps; ++s) {
+          if (kF8) umma_f8(tmem_base + uint32_t(b * kKeys), dq + uint64_t(2 * s), dk + uint64_t(2 * s), idesc_s, s != 0 ? 1u : 0u);
+          else umma_i8(tmem_base + uint32_t(b * kKeys), dq + uint64_t(2 * s), dk + uint64_t(2 * s), idesc_s, s != 0 ? 1u : 0u);
+        }
         umma_commit(smem_u32(&S.s_full[b]));
-        if (kCentered) umma_commit(smem_u32(&S.k_empty[b]));      // the K tile may be refilled once these MMAs have read it
+        if (kCentered) umma_commit(smem_u32(&S.k_empty[kb]));     // the K tile may be refilled once these MMAs have read it
         return true;
       };
-      for (int g = 0; g < nb && ok && !*abort; ++g) ok = issue_s(g);
-      if (ok && !*abort) ok = issue_s(nb);
+      // S MMAs run ahead of the workers by as many visits as there are S buffers; the buffer of visit g is free once
+      // visit g - kS has been read, which the workers have done before they hand over the operand tiles of the P.V
+      // MMAs issued next, so this thread never sits in a wait for S while those tiles are ready
+      // (where the workers stage the K tiles themselves, one visit ahead, the S MMAs stay one visit ahead as well)
+      constexpr int kAhead = kCentered ? kS : 2;
+      int next_s = 0;
+      for (; next_s < nb + kAhead - 1 && next_s < 2 * nb && ok && !*abort; ++next_s) ok = issue_s(next_s);
       for (int j = 0; j < nb && ok && !*abort; ++j) {
-        if (j + 1 < nb && !issue_s(nb + j + 1)) { ok = false; break; }
-        if (!mbar_wait(smem_u32(&S.p_full), uint32_t(j) & 1u, abort, 43, P.status)) { ok = false; break; }
+        if (next_s < 2 * nb) {
+          if (!issue_s(next_s)) { ok = false; break; }
+          ++next_s;
+        }
+        const int pb = ring(j, kP);
+        if (!mbar_wait(smem_u32(&S.p_full[pb]), lap(j, kP), abort, 43, P.status)) { ok = false; break; }
         tc_fence_after();
-        const uint64_t de = smem_desc_sw128(smem_u32(S.e)), dd = smem_desc_sw128(smem_u32(S.o));
-        const uint64_t dv = smem_desc_sw128(smem_u32(S.v), kVBlockBytes);
+        const uint64_t de = smem_desc_sw128(smem_u32(S.e[pb])), dd = smem_desc_sw128(smem_u32(S.o[pb]));
+        const uint64_t dv = smem_desc_sw128(smem_u32(S.v[pb]), kVBlockBytes);
         const int keys_here = min(kKeys, k_end - j * kKeys);
         const int steps = (keys_here + 15) >> 4;                       // 16 keys per MMA
         for (int s = 0; s < steps; ++s) {
@@ -271,7 +322,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
           umma_f16(tmem_base + uint32_t(kAccCol), de + uint64_t(2 * s), dv + uint64_t(128 * s), idesc_pv, accumulate);
           umma_f16(tmem_base + uint32_t(kAccCol + P.n_pad), dd + uint64_t(2 * s), dv + uint64_t(128 * s), idesc_pv, accumulate);
         }
-        umma_commit(smem_u32(&S.p_empty));
+        umma_commit(smem_u32(&S.p_empty[pb]));
       }
       if (ok && !*abort) umma_commit(smem_u32(&S.acc_full));
       umma_commit(smem_u32(&S.done));
@@ -282,8 +333,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
     if (kCentered && lane == 0) {
       int issued = 0;
       for (int g = 0; g < 2 * nb && !*abort; ++g) {
-        const int b = g & 1;
-        if (!mbar_wait(smem_u32(&S.k_empty[b]), (uint32_t(g >> 1) & 1u) ^ 1u, abort, 48, P.status)) break;
+        const int b = ring(g, kK);
+        if (!mbar_wait(smem_u32(&S.k_empty[b]), lap(g, kK) ^ 1u, abort, 48, P.status)) break;
         const uint32_t bar = smem_u32(&S.k_full[b]);
         mbar_expect_tx(bar, kKBytes);
         // box: 128 bytes of the head's row (bytes past d_h meet zero bytes of the Q tile), 64 keys (rows past Lk are
@@ -292,7 +343,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
         ++issued;
       }
       // the copies issued last must have landed before this CTA may exit
-      for (int i = issued > 2 ? issued - 2 : 0; i < issued; ++i) mbar_drain(smem_u32(&S.k_full[i & 1]), uint32_t(i >> 1) & 1u);
+      for (int i = issued > kK ? issued - kK : 0; i < issued; ++i) mbar_drain(smem_u32(&S.k_full[ring(i, kK)]), lap(i, kK));
     }
   } else {
     // ---------------------------------------------------------------- tiles, Softmax arithmetic, epilogue
@@ -309,8 +360,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
 #pragma unroll
       for (int p4 = 0; p4 < kCols / 8; ++p4) {
         const uint32_t off = tile_offset(r, part * (kCols / 8) + p4);
-        *reinterpret_cast<uint4*>(S.e + off) = make_uint4(0u, 0u, 0u, 0u);
-        *reinterpret_cast<uint4*>(S.o + off) = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+        for (int pb = 0; pb < kP; ++pb) {
+          *reinterpret_cast<uint4*>(S.e[pb] + off) = make_uint4(0u, 0u, 0u, 0u);
+          *reinterpret_cast<uint4*>(S.o[pb] + off) = make_uint4(0u, 0u, 0u, 0u);
+        }
       }
     }
     const float c = 1.4426950408889634f;
@@ -348,74 +402,89 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
     float m = -CUDART_INF_F, z = 0.f;       // pass 1: running maximum and sum of this thread's columns
     float k0 = 0.f;                         // pass 2: 2 (log2 Z + log2 s), with m the row's final maximum
 
-    // corr = acc - z_k qsum - z_q ksum + d_h z_q z_k of the thread's 16 columns of key block j (buffer g & 1), as
-    // integers.  Frees the buffer as soon as it is read.  Keys the row may not see are dealt with by the callers, in
-    // the blocks that reach past the keys the thread's row sees (`edge`): the values themselves are left as they
-    // come from tensor memory, so that the common path carries no selects or copies.
-    auto read_s = [&](int g, int j, int (&corr)[kCols], bool& edge) -> bool {
-      const int b = g & 1;
-      if (!mbar_wait(smem_u32(&S.s_full[b]), uint32_t(g >> 1) & 1u, abort, 44, P.status)) return false;
+    // The thread's 16 accumulators of visit g: load_s waits for the S MMAs and starts the load into rn, settle_s waits
+    // for the data and frees the buffer.
+    uint32_t rn[kCols];
+    auto load_s = [&](int g) -> bool {
+      const int b = ring(g, kS);
+      if (!mbar_wait(smem_u32(&S.s_full[b]), lap(g, kS), abort, 44, P.status)) return false;
       tc_fence_after();
-      uint32_t r0[16];
       __syncwarp();
-      tmem_ld16(taddr_s + uint32_t(b * kKeys), r0);
-      tmem_ld_wait();
+      tmem_ld16(taddr_s + uint32_t(b * kKeys), rn);
+      return true;
+    };
+    auto settle_s = [&](int g) {
+      tmem_ld_wait(rn);
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&S.s_empty[b]));
-      if (kCentered) {
+      if (lane == 0) mbar_arrive(smem_u32(&S.s_empty[ring(g, kS)]));
+    };
+    // The scores of visit g in units of the score scale, as floats: the accumulator itself (kCentredF8), the converted
+    // accumulator (kCentred), or the converted corr = acc - z_k qsum - z_q ksum + d_h z_q z_k (kCorrected).  Keys the
+    // row may not see are dealt with by the callers, in the blocks that reach past the keys the thread's row sees
+    // (`edge`): the values themselves are left as they come from tensor memory, so that the common path carries no
+    // selects or copies.
+    auto scores = [&](int g, float (&sf)[kCols]) {
+      if (kF8) {
 #pragma unroll
-        for (int e = 0; e < kCols; ++e) corr[e] = int32_t(r0[e]);
+        for (int e = 0; e < kCols; ++e) sf[e] = __uint_as_float(rn[e]);
+      } else if (kCentered) {
+#pragma unroll
+        for (int e = 0; e < kCols; ++e) sf[e] = float(int32_t(rn[e]));
       } else {
         const int* ct = S.col_term[g & 3] + part * kCols;
 #pragma unroll
         for (int e4 = 0; e4 < kCols / 4; ++e4) {
           const int4 c4 = *reinterpret_cast<const int4*>(ct + 4 * e4);
-          corr[4 * e4 + 0] = int32_t(r0[4 * e4 + 0]) + my_row_term + c4.x;
-          corr[4 * e4 + 1] = int32_t(r0[4 * e4 + 1]) + my_row_term + c4.y;
-          corr[4 * e4 + 2] = int32_t(r0[4 * e4 + 2]) + my_row_term + c4.z;
-          corr[4 * e4 + 3] = int32_t(r0[4 * e4 + 3]) + my_row_term + c4.w;
+          sf[4 * e4 + 0] = float(int32_t(rn[4 * e4 + 0]) + my_row_term + c4.x);
+          sf[4 * e4 + 1] = float(int32_t(rn[4 * e4 + 1]) + my_row_term + c4.y);
+          sf[4 * e4 + 2] = float(int32_t(rn[4 * e4 + 2]) + my_row_term + c4.z);
+          sf[4 * e4 + 3] = float(int32_t(rn[4 * e4 + 3]) + my_row_term + c4.w);
         }
       }
-      edge = j * kKeys + part * kCols + kCols > valid;
-      return true;
     };
 
     auto process = [&](int g) -> bool {
       const int j = g < nb ? g : g - nb;
-      int corr[kCols];
-      bool edge;
-      if (!read_s(g, j, corr, edge)) return false;
+      if (!load_s(g)) return false;
+      settle_s(g);
+      float sf[kCols];
+      scores(g, sf);
+      const bool edge = j * kKeys + part * kCols + kCols > valid;
       const int seen = valid - (j * kKeys + part * kCols);       // columns e < seen are keys the row sees
       if (g < nb) {
-        // ---- pass 1: running maximum and sum.  The maximum is taken on the integers (S = scale * float(corr) is
-        // monotonic in corr); a key the row may not see contributes nothing.
-        const float sc = P.scale * c;                             // exponent of 2 per unit of corr
+        // ---- pass 1: running maximum and sum.  The maximum is taken on the unscaled values (S = scale * sf is
+        // monotonic in sf); a key the row may not see contributes nothing.  Exponents and sums on packed pairs.
+        const float sc = P.scale * c;                             // exponent of 2 per unit of sf
         if (__builtin_expect(!edge, 1)) {
-          int bmi = corr[0];
+          float bm = max3(sf[0], sf[1], sf[2]);
 #pragma unroll
-          for (int e = 1; e < kCols; ++e) bmi = max(bmi, corr[e]);
-          const float mn = fmaxf(m, P.scale * float(bmi));
-          const float mnc = mn * c;
-          float acc0 = 0.f, acc1 = 0.f;
+          for (int e = 3; e + 1 < kCols; e += 2) bm = max3(bm, sf[e], sf[e + 1]);
+          bm = fmaxf(bm, sf[kCols - 1]);
+          const float mn = fmaxf(m, P.scale * bm);
+          const f32x2 sc2 = splat2(sc), nm2 = splat2(-(mn * c));
+          f32x2 acc = 0ull;                                       // even columns in the low lane, odd ones in the high lane
 #pragma unroll
           for (int e = 0; e < kCols; e += 2) {
-            acc0 += ex2(fmaf(float(corr[e]), sc, -mnc));
-            acc1 += ex2(fmaf(float(corr[e + 1]), sc, -mnc));
+            float a0, a1;
+            unpack2(fma2(pack2(sf[e], sf[e + 1]), sc2, nm2), a0, a1);
+            acc = add2(acc, pack2(ex2(a0), ex2(a1)));
           }
+          float acc0, acc1;
+          unpack2(acc, acc0, acc1);
           z = z * ex2((m - mn) * c) + (acc0 + acc1);     // m = -inf at first: factor 0
           m = mn;
         } else if (seen > 0) {
-          int bmi = corr[0];
+          float bm = sf[0];
 #pragma unroll
           for (int e = 1; e < kCols; ++e)
-            if (e < seen) bmi = max(bmi, corr[e]);
-          const float mn = fmaxf(m, P.scale * float(bmi));
+            if (e < seen) bm = fmaxf(bm, sf[e]);
+          const float mn = fmaxf(m, P.scale * bm);
           const float mnc = mn * c;
           float acc = 0.f;
 #pragma unroll
           for (int e = 0; e < kCols; ++e)
-            if (e < seen) acc += ex2(fmaf(float(corr[e]), sc, -mnc));
+            if (e < seen) acc += ex2(fmaf(sf[e], sc, -mnc));
           z = z * ex2((m - mn) * c) + acc;
           m = mn;
         }
@@ -449,28 +518,42 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
       // from integer arithmetic for wider ones.  A masked key gets (0, 0).
       const uint32_t lut_addr = smem_u32(&S.lut[0][lane]) - (kMagicBits << 7);
       uint4 ev[kCols / 8], ov[kCols / 8];
-      if (!dead_warp) {
-      uint32_t eo[kCols];
+      // a warp none of whose rows sees a key of its 16 columns (the block past the last key, the blocks beyond the
+      // diagonal under a causal mask) writes zero operands without any arithmetic
+      const bool idle = !dead_warp && !__any_sync(0xffffffffu, seen > 0);
+      if (idle) {
 #pragma unroll
-      for (int e = 0; e < kCols; ++e) {
-        // clamped on both sides whatever the inputs (rows past Lq carry m = -inf, Z = 0): p indexes the table
-        if (kLut) {
-          // table-driven codes: t 2^-bits comes out of one saturating fma (k1 and k0 scaled by 2^-bits, exact, so the
-          // value is t rounded as before and clamped to [0, 1]), the scaling back and the rounding are one more fma;
-          // 2^bits (t within half a code of it) reads the table's copy of the top entry
-          float w;
-          constexpr float kSteps = float(1 << kLutBits), kInvSteps = 1.f / kSteps;      // 2^bits and its reciprocal (exact)
-          asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(w) : "f"(fmaf(float(corr[e]), P.scale, -m)), "f"(k1 * kInvSteps), "f"(k0 * kInvSteps));
-          const uint32_t u = __float_as_uint(fmaf(w, kSteps, magic));
-          asm("ld.shared.u32 %0, [%1];" : "=r"(eo[e]) : "r"(lut_addr + (u << 7)));
-        } else {
-          // wider codes: the same clamp to [0, 2^bits], then the top code by one integer minimum
-          float w;
-          asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(w) : "f"(fmaf(float(corr[e]), P.scale, -m)), "f"(k1 * inv_qs), "f"(k0 * inv_qs));
-          const uint32_t u = min(__float_as_uint(fmaf(w, qs, magic)), u_top);
-          const int kk = int((u - kMagicBits + 1u) >> 1);                       // ceil(p / 2)
-          const uint32_t val = uint32_t(max(127 - kk, 0)) << 7;                 // bf16 bits of 2^-kk (0 below the normal range)
-          eo[e] = (u & 1u) ? val << 16 : val;
+        for (int p4 = 0; p4 < kCols / 8; ++p4) ev[p4] = ov[p4] = make_uint4(0u, 0u, 0u, 0u);
+      }
+      if (!dead_warp && !idle) {
+      uint32_t eo[kCols];
+      // S - m on packed pairs; then t 2^-bits out of one saturating fma each (k1 and k0 scaled by 2^-bits, exact, so the
+      // value is t rounded as before and clamped to [0, 1] whatever the inputs: rows past Lq carry m = -inf, Z = 0), and
+      // the scaling back and the rounding as one more packed fma
+      constexpr float kSteps = kLut ? float(1 << kLutBits) : 0.f;
+      const float steps = kLut ? kSteps : qs, inv_steps = kLut ? 1.f / kSteps : inv_qs;
+      const float k1s = k1 * inv_steps, k0s = k0 * inv_steps;
+      const f32x2 scale2 = splat2(P.scale), nm2 = splat2(-m), steps2 = splat2(steps), magic2 = splat2(magic);
+#pragma unroll
+      for (int e = 0; e < kCols; e += 2) {
+        float x0, x1, w0, w1;
+        unpack2(fma2(pack2(sf[e], sf[e + 1]), scale2, nm2), x0, x1);
+        asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(w0) : "f"(x0), "f"(k1s), "f"(k0s));
+        asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(w1) : "f"(x1), "f"(k1s), "f"(k0s));
+        float uf[2];
+        unpack2(fma2(pack2(w0, w1), steps2, magic2), uf[0], uf[1]);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          if (kLut) {
+            // table-driven codes; 2^bits (t within half a code of it) reads the table's copy of the top entry
+            asm("ld.shared.u32 %0, [%1];" : "=r"(eo[e + h]) : "r"(lut_addr + (__float_as_uint(uf[h]) << 7)));
+          } else {
+            // wider codes: the top code by one integer minimum
+            const uint32_t u = min(__float_as_uint(uf[h]), u_top);
+            const int kk = int((u - kMagicBits + 1u) >> 1);                       // ceil(p / 2)
+            const uint32_t val = uint32_t(max(127 - kk, 0)) << 7;                 // bf16 bits of 2^-kk (0 below the normal range)
+            eo[e + h] = (u & 1u) ? val << 16 : val;
+          }
         }
       }
       if (__builtin_expect(edge, 0)) {
@@ -488,13 +571,14 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
       }
       // one stage of operand tiles: the MMAs of the block before must have read them (the code arithmetic above
       // has overlapped with those MMAs)
-      if (!mbar_wait(smem_u32(&S.p_empty), (uint32_t(j) & 1u) ^ 1u, abort, 46, P.status)) return false;
+      const int pb = ring(j, kP);
+      if (!mbar_wait(smem_u32(&S.p_empty[pb]), lap(j, kP) ^ 1u, abort, 46, P.status)) return false;
       if (!dead_warp) {
 #pragma unroll
         for (int p4 = 0; p4 < kCols / 8; ++p4) {
           const uint32_t off = tile_offset(r, part * (kCols / 8) + p4);
-          *reinterpret_cast<uint4*>(S.e + off) = ev[p4];
-          *reinterpret_cast<uint4*>(S.o + off) = ov[p4];
+          *reinterpret_cast<uint4*>(S.e[pb] + off) = ev[p4];
+          *reinterpret_cast<uint4*>(S.o[pb] + off) = ov[p4];
         }
       }
 #pragma unroll
@@ -525,12 +609,12 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
             }
           }
         }
-        *reinterpret_cast<uint4*>(S.v + v_off[qi]) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+        *reinterpret_cast<uint4*>(S.v[pb] + v_off[qi]) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
       }
       fetch_v(j + 1);
       fence_async_smem();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&S.p_full));
+      if (lane == 0) mbar_arrive(smem_u32(&S.p_full[pb]));
       return true;
     };
 
@@ -538,11 +622,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
     for (int g = 0; g < 2 * nb && !*abort; ++g) {
       if (!kCentered) {
         // tile g & 1 was last read by the S MMAs of g - 2, whose result this thread has already waited for
-        const int ks = store_k(S.k[g & 1]);
+        const int ks = store_k(S.k[ring(g, kK)]);
         if (kq == 0) S.col_term[g & 3][kkey] = -P.zq * ks;
         fence_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&S.k_full[g & 1]));
+        if (lane == 0) mbar_arrive(smem_u32(&S.k_full[ring(g, kK)]));
         kreg = knext;
         k_live = k_live_next;
         // two blocks ahead (global latency is about one block); g + 2 < 2 nb, so the block index needs no division
@@ -632,6 +716,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
   }
 
   // ------------------------------------------------------------------ teardown
+  if (warp < kWorkWarps) tmem_ld_wait();          // an error path may leave a tensor-memory load in flight
   tc_fence_before();
   __syncthreads();
   if (warp == kWorkWarps) {
@@ -656,17 +741,18 @@ repq_status make_k_map(CUtensorMap* map, const AttnParams& P, int batch_outer) {
   return REPQ_OK;
 }
 
-template <int NB, int kLutBits, bool kCentered>
+template <int NB, int kLutBits, int kMode>
 repq_status launch_kernel(const AttnParams& P, int64_t pairs, cudaStream_t st) {
   const size_t smem = sizeof(AttnShared<NB, kLutBits>);
-  REPQ_CUDA(cudaFuncSetAttribute(attention_tc_kernel<NB, kLutBits, kCentered>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+  REPQ_CUDA(cudaFuncSetAttribute(attention_tc_kernel<NB, kLutBits, kMode>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
   AttnParams Q = P;
   Q.pairs = int(pairs);
   Q.tiles = (P.Lq + kRows - 1) / kRows;
+  if (kMode == kCentredF8) Q.scale = P.scale * 262144.f;      // the accumulators hold 2^-18 sum (q - z_q) k
   CUtensorMap map_k{};
-  if (kCentered) REPQ_TRY(make_k_map(&map_k, P, int(pairs / P.batch_inner)));
+  if (kMode != kCorrected) REPQ_TRY(make_k_map(&map_k, P, int(pairs / P.batch_inner)));
   dim3 grid(unsigned(Q.tiles) * unsigned(pairs));
-  REPQ_CUDA(launch_chained(attention_tc_kernel<NB, kLutBits, kCentered>, grid, dim3(kThreads), smem, st, map_k, Q));
+  REPQ_CUDA(launch_chained(attention_tc_kernel<NB, kLutBits, kMode>, grid, dim3(kThreads), smem, st, map_k, Q));
   note_launch();
   return REPQ_OK;
 }
@@ -678,7 +764,10 @@ repq_status launch(const AttnParams& P, int64_t pairs, int qmax_qk, cudaStream_t
   const bool centred = qmax_qk < 128 && P.zq >= 0 && P.zq < 128 && P.zk >= 0 && P.zk < 128 && P.k_so > 0 &&
                        P.ldk < (int64_t(1) << 40) && P.k_so < (int64_t(1) << 40) &&
                        int64_t(P.batch_inner - 1) * P.k_si + P.dh <= P.ldk;
-  return centred ? launch_kernel<NB, kLutBits, true>(P, pairs, st) : launch_kernel<NB, kLutBits, false>(P, pairs, st);
+  // 4-bit quantizers with the zero point of Q inside the code range: the tiles are also valid 8-bit floats
+  const bool f8 = centred && qmax_qk <= 15 && P.zq <= 15 && !P.no_f8;
+  if (f8) return launch_kernel<NB, kLutBits, kCentredF8>(P, pairs, st);
+  return centred ? launch_kernel<NB, kLutBits, kCentred>(P, pairs, st) : launch_kernel<NB, kLutBits, kCorrected>(P, pairs, st);
 }
 
 }  // namespace
@@ -732,13 +821,18 @@ extern "C" repq_status repq_attention(const repq_attention_desc* d, void* stream
   P.out = d->out; P.ldo = d->ldo; P.o_so = d->o_stride_outer; P.o_si = d->o_stride_inner;
   P.out_row_sum = d->out_kind == REPQ_OUT_CODES ? d->out_row_sum : nullptr;
   P.n_pad = (d->d_h + 15) / 16 * 16;
-  P.tmem_cols = 2 * kKeys + 2 * P.n_pad <= 256 ? 256 : 512;
+  P.tmem_cols = d->d_h <= 64 ? 256 : 512;      // 2 x 64 + 2 x 64, or 4 x 64 + 2 x 128 columns
   const int64_t chunk_bytes = d->out_kind == REPQ_OUT_CODES && packed4(d->out_bits) ? 8 : 16 * esz;
   const int64_t al = chunk_bytes < 16 ? chunk_bytes : 16;
   P.vec_store = aligned(d->out, size_t(al)) && (d->ldo * esz) % al == 0 && (d->o_stride_outer * esz) % al == 0 &&
                 (d->o_stride_inner * esz) % al == 0;
   P.status = device_status_word();
   REPQ_REQUIRE(P.status != nullptr, REPQ_CUDA_ERROR, "attention: device status word unavailable");
+  {
+    // read at every call, so that a test can compare the two score forms in one process
+    const char* e = getenv("REPQ_ATTENTION_INT_SCORES");
+    P.no_f8 = e && *e && *e != '0';
+  }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // the per-lane table of the Softmax codes' operand values: 17 / 65 entries everywhere; the 257 entries of 8-bit codes
   // (33 KB) only where the head already limits the SM to one CTA

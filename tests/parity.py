@@ -639,6 +639,19 @@ def check_attention(B_, H, Lq, Lk, dh, bits, bits_p, causal=False, out_kind="f32
             if first is None:
                 first = out.clone()
             assert torch.equal(out, first), "launches differ"
+        if qb(bits) == 4 and 0 <= z_q <= 15:
+            # 4-bit Q / K: the score contraction ran on the 8-bit float type; the integer contraction must give the
+            # same bits
+            import os
+            os.environ["REPQ_ATTENTION_INT_SCORES"] = "1"
+            try:
+                if row_sum is not None:
+                    row_sum.zero_()
+                B.repq_attention(d)
+                torch.cuda.synchronize()
+            finally:
+                del os.environ["REPQ_ATTENTION_INT_SCORES"]
+            assert torch.equal(out, first), "8-bit float scores and integer scores differ"
         assert B.repq_device_status() == 0
         return first, row_sum
 
