@@ -1,28 +1,39 @@
 // Fused attention on integer codes: scores (Eq. 3 with quantized Q and K), Softmax, log-sqrt2 codes (Eq. 15) and
 // P.V with the reparameterized log2 de-quantization (Eqs. 16-17) in one kernel.  Scores and codes never leave the
-// SM.  The code of a score depends on the row's final Softmax sum, so the keys are walked twice:
-//   pass 1   S = Q K^T per block of 64 keys (tcgen05.mma kind::i8 into tensor memory), running row maximum m and
-//            sum Z = sum 2^(c (S - m)) (each thread: one row, 16 of the 64 columns; the four partial results of a row
-//            are merged once, after the pass)
+// SM.  The code of a score depends on the row's final Softmax sum, so the keys are walked twice, a visit being 64 keys
+// (heads of up to 64 channels) or 128 keys (wider heads):
+//   pass 1   S = Q K^T per visit (tcgen05.mma on 8-bit operands into a slot of tensor memory), running row maximum m
+//            and sum Z = sum 2^(c (S - m)) (a thread: one row and a quarter of all columns; the four partial results
+//            of a row are merged once, after the pass)
 //   pass 2   S again, t = 2 (log2 Z + log2 s) - 2 c (S - m), code p = clip(round(t), 0, 2^b - 1), operand values
-//            2^(-ceil(p/2)) split by the parity of p into the tiles E and O (exact bf16 powers of two), V as exact bf16
-//            integers v - z_v, and two tcgen05.mma kind::f16 per 16 keys accumulate E.V and O.V in tensor memory;
-//            O = s s_v (acc_E + sqrt2 acc_O), then the output conversion (Eq. 4 or float)
+//            2^(-ceil(p/2)) split by the parity of p into E and O (exact bf16 powers of two), written back as bf16 pairs
+//            over the very columns of tensor memory the scores came from; V as exact bf16 integers v - z_v in shared
+//            memory; two tcgen05.mma kind::f16 per 16 keys, with the A operand read from tensor memory, accumulate E.V
+//            and O.V; O = s s_v (acc_E + sqrt2 acc_O), then the output conversion (Eq. 4 or float)
 // Float arithmetic on S is the same as in the separate kernels (float(corr) * (alpha s_q s_k); one ex2 per element
 // for Z), so the codes agree with theirs except where the differently ordered sum Z moves a value across a
 // rounding tie.
 //
-// One CTA owns 128 query rows of one (batch, head) pair.  Warps 0..15 (four per tensor-memory lane quarter: a thread
-// has one row and 16 of the 64 columns of a key block): V tiles (and, for quantizers wider than 7 bits, K tiles) from
-// registers (fetched one block ahead) into 128-byte-swizzled shared-memory tiles, the Softmax arithmetic, the E / O
-// tiles, the epilogue.  Warp 16 (one lane): tensor-memory allocation and MMA issue.  Warp 17 (one lane, quantizers of
-// at most 7 bits): K tiles by bulk tensor copies, two blocks ahead.  There the Q tile holds q - z_q as signed bytes and
-// the K tile the raw unsigned codes: S' = sum (q - z_q) k differs from the zero-point-corrected sum by
-// -z_k sum (q - z_q), which is the same for every key of a row and drops out of the Softmax (maximum and values are
-// taken on S' alone), so no correction and no pass over the K bytes is needed.  S is double-buffered in tensor memory (2 x 64 columns),
-// the E / O / V tiles are single (their block's code arithmetic overlaps the MMAs of the block before).  Under a causal mask, key blocks no row of the CTA may see are
-// skipped.  Every mbarrier wait is bounded; when one runs out the kernel records a status code, all roles leave
-// their loops, MMAs in flight are drained, tensor memory is freed and the kernel returns.
+// What bounds the kernel is the tensor-core instruction stream and the hand-shakes around it, not the arithmetic: an
+// MMA instruction of this size takes about 100 cycles whatever its N, the issuing thread waits for each of its
+// barriers in turn, and a worker's visit is a chain of fixed latencies (barrier, tensor-memory load, table look-ups,
+// barrier).  Hence:
+//  - Warps 0..15 are two groups of eight worker warps that take the visits alternately (group g mod 2 takes visit g;
+//    visits are counted over both passes), each with its own slot of tensor memory: while one group waits, the other
+//    computes.  Inside a group a thread has one row (its tensor-memory lane) and half of the visit's columns, handled
+//    in runs of 16 (one tensor-memory load, arithmetic, in pass 2 one tensor-memory store).
+//  - Wide heads use visits of 128 keys (half the instructions per key) and give the P.V MMAs an issuing warp of their
+//    own (warp 18), so that the S MMAs (warp 16) are not held up by the wait for the workers' operands.
+//  - The E / O operands never touch shared memory, whose bandwidth the V tiles, the table look-ups and the MMAs' B
+//    operands already share.
+// A group also builds the V tile of its visits (from registers fetched one of its visits ahead) and, for quantizers
+// wider than 7 bits, the K tiles of its visits.  Warp 17 (one lane, quantizers of at most 7 bits): K tiles by bulk
+// tensor copies.  There the Q tile holds q - z_q as signed bytes and the K tile the raw unsigned codes:
+// S' = sum (q - z_q) k differs from the zero-point-corrected sum by -z_k sum (q - z_q), which is the same for every key
+// of a row and drops out of the Softmax (maximum and values are taken on S' alone), so no correction and no pass over
+// the K bytes is needed.  Under a causal mask, key blocks no row of the CTA may see are skipped.  Every mbarrier wait
+// is bounded; when one runs out the kernel records a status code, all roles leave their loops, MMAs in flight are
+// drained, tensor memory is freed and the kernel returns.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <math_constants.h>
@@ -39,16 +50,18 @@ namespace {
 using namespace tc;
 
 constexpr int kRows = 128;                  // query rows per CTA (MMA M)
-constexpr int kKeys = 64;                   // keys per block
-constexpr int kWorkWarps = 16;                // 4 per tensor-memory lane quarter: a row's 64 columns are split 4 ways
-constexpr int kParts = kWorkWarps / 4;
-constexpr int kCols = kKeys / kParts;         // S columns per thread and key block
+// keys per visit: 64 for heads of up to 64 channels (two CTAs per SM, 256 tensor-memory columns each), 128 for wider
+// heads (one CTA per SM): a tensor-core instruction costs about the same time whether it covers 64 or 128 keys
+template <int NB> struct VisitKeys { static constexpr int value = NB == 1 ? 64 : 128; };
+constexpr int kWorkWarps = 16;                // two groups of eight: 2 per tensor-memory lane quarter and group
+constexpr int kGroupWarps = kWorkWarps / 2;
+constexpr int kGroupThreads = 32 * kGroupWarps;
+constexpr int kParts = kWorkWarps / 4;        // threads that share a row: 2 groups x 2 halves of a block's columns
+constexpr int kCols = 16;                     // S columns per tensor-memory load (a run); a thread takes 2 or 4 runs per visit
 constexpr int kWorkThreads = 32 * kWorkWarps;
-constexpr int kThreads = kWorkThreads + 64;        // + MMA warp + K-copy warp
+// + S-MMA warp + K-copy warp, and for wide heads a P.V-MMA warp of its own (its waits then do not hold up the S MMAs)
+template <int NB> struct Threads { static constexpr int value = kWorkThreads + (NB == 1 ? 64 : 96); };
 constexpr uint32_t kQBytes = kRows * 128;         // Q tile: rows of 128 bytes (the head's codes, zero-padded)
-constexpr uint32_t kKBytes = kKeys * 128;
-constexpr uint32_t kTileBytes = kRows * 128;      // E or O tile of one block (64 keys of bf16 per row)
-constexpr uint32_t kVBlockBytes = kKeys * 128;    // 64 keys x 64 channels of bf16
 constexpr uint32_t kMagicBits = 0x4B400000u;      // float 1.5 * 2^23
 
 struct AttnParams {
@@ -71,23 +84,22 @@ struct AttnParams {
   int32_t* status;
 };
 
-// Ring depths.  Heads of up to 64 channels run two CTAs per SM (256 tensor-memory columns and about 80 KB of shared
-// memory each), which overlap each other's waits: S and K double-buffered, one stage of operand tiles.  Wider heads
-// have the SM to themselves: four S buffers in tensor memory (4 x 64 columns beside the 2 x 128 of the accumulators),
-// four K tiles and two stages of E / O / V tiles, so that neither the S MMAs' round trip nor the P.V MMAs of the block
-// before stand between a worker warp and its next block.
-template <int NB> struct Rings { static constexpr int kS = NB == 1 ? 2 : 4, kK = NB == 1 ? 2 : 4, kP = NB == 1 ? 1 : 2; };
+// Ring depths.  S: one slot of tensor memory per worker group (2 x 64 or 2 x 128 columns beside the accumulators' 2 x 64
+// or 2 x 128).  Heads of up to 64 channels run two CTAs per SM: two K tiles, one V stage.  Wider heads have the SM to
+// themselves: four K tiles, two V stages (one per worker group).
+template <int NB> struct Rings { static constexpr int kS = 2, kK = NB == 1 ? 2 : 4, kP = NB == 1 ? 1 : 2; };
 
 template <int NB, int kLutBits>
 struct AttnShared {
   static constexpr int kS = Rings<NB>::kS, kK = Rings<NB>::kK, kP = Rings<NB>::kP;
+  static constexpr int kKeys = VisitKeys<NB>::value;
+  static constexpr uint32_t kKBytes = kKeys * 128;
+  static constexpr uint32_t kVBlockBytes = kKeys * 128;       // the visit's keys x 64 channels of bf16
   alignas(1024) uint8_t q[kQBytes];
   alignas(1024) uint8_t k[kK][kKBytes];
-  alignas(1024) uint8_t e[kP][kTileBytes];
-  alignas(1024) uint8_t o[kP][kTileBytes];
   alignas(1024) uint8_t v[kP][NB * kVBlockBytes];
   int row_term[kRows];                              // -z_k qsum[m] + d_h z_q z_k
-  int col_term[4][kKeys];                           // -z_q ksum[n], ring of 4 key blocks
+  int col_term[4][kKeys];                           // -z_q ksum[n], ring of 4 visits
   float stat_m[kParts][kRows], stat_z[kParts][kRows];   // pass-1 results of the column parts of every row
   static constexpr int kLutEntries = kLutBits ? (1 << kLutBits) + 1 : 1;
   uint32_t lut[kLutEntries][32];                    // table-driven codes: [code][lane] = E value | O value << 16 (one bank per
@@ -95,8 +107,9 @@ struct AttnShared {
                                                     // rounds up lands there)
   alignas(8) uint64_t k_full[kK];
   uint64_t k_empty[kK];                             // K tile read by its S MMAs (bulk-copy variant)
-  uint64_t s_full[kS], s_empty[kS], p_full[kP], p_empty[kP];
-  uint64_t stats_ready, acc_full, done;
+  uint64_t s_full[kS], s_empty[kS], s_spent[kS], p_full[kP], p_empty[kP];   // s_empty: read in pass 1; s_spent: P.V MMAs of a
+                                                                            // pass-2 visit have read the operands written over S
+  uint64_t stats_ready, acc_full, done, done_pv;
   uint32_t tmem_base;
   volatile int abort;
 };
@@ -143,13 +156,16 @@ __device__ __forceinline__ float ex2(float x) {
 //               folded into the score scale on the host, exactly)
 enum : int { kCorrected = 0, kCentred = 1, kCentredF8 = 2 };
 template <int NB, int kLutBits, int kMode>
-__global__ void __launch_bounds__(kThreads, NB == 1 ? 2 : 1)
+__global__ void __launch_bounds__(Threads<NB>::value, NB == 1 ? 2 : 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
   using Shared = AttnShared<NB, kLutBits>;
+  constexpr int kKeys = Shared::kKeys;
+  constexpr uint32_t kKBytes = Shared::kKBytes, kVBlockBytes = Shared::kVBlockBytes;
+  constexpr bool kSplitIssue = NB != 1;                   // P.V MMAs issued by a warp of their own
+  constexpr int kRuns = kKeys / (2 * kCols);              // runs of 16 columns per thread and visit
   constexpr bool kLut = kLutBits != 0;
   constexpr bool kCentered = kMode != kCorrected;
   constexpr bool kF8 = kMode == kCentredF8;
-  constexpr int kVItems = NB;                             // 8-channel groups of V per thread and block
   constexpr int kS = Shared::kS, kK = Shared::kK, kP = Shared::kP;      // ring depths (powers of two)
   constexpr int kAccCol = kS * kKeys;                     // first tensor-memory column of the P.V accumulators
   auto ring = [](int i, int depth) { return i & (depth - 1); };
@@ -176,26 +192,28 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
   const int shift = P.Lk - P.Lq;
   const int k_end = P.causal ? max(1, min(P.Lk, min(q0 + kRows, P.Lq) + shift)) : P.Lk;
   const int min_valid = P.causal ? max(0, min(P.Lk, q0 + 1 + shift)) : P.Lk;   // fewest keys any row of the CTA sees
-  const int nb = (k_end + kKeys - 1) / kKeys;             // key blocks; every block is visited in both passes
+  const int nb = (k_end + kKeys - 1) / kKeys;             // key blocks of a visit's size; every one is visited in both passes
   const int ksteps = (P.dh + 31) >> 5;                    // S MMAs of K = 32 per key block
   const int pieces = P.dh >> 4;                           // 16-byte pieces of a Q / K row
 
   if (tid == 0) {
     for (int s = 0; s < kK; ++s) {
-      mbar_init(smem_u32(&S.k_full[s]), kCentered ? 1 : kWorkWarps);
+      mbar_init(smem_u32(&S.k_full[s]), kCentered ? 1 : kGroupWarps);
       mbar_init(smem_u32(&S.k_empty[s]), 1);
     }
     for (int s = 0; s < kS; ++s) {
       mbar_init(smem_u32(&S.s_full[s]), 1);
-      mbar_init(smem_u32(&S.s_empty[s]), kWorkWarps);
+      mbar_init(smem_u32(&S.s_empty[s]), kGroupWarps);
+      mbar_init(smem_u32(&S.s_spent[s]), 1);
     }
     for (int s = 0; s < kP; ++s) {
-      mbar_init(smem_u32(&S.p_full[s]), kWorkWarps);
+      mbar_init(smem_u32(&S.p_full[s]), kGroupWarps);
       mbar_init(smem_u32(&S.p_empty[s]), 1);
     }
     mbar_init(smem_u32(&S.stats_ready), kWorkWarps);
     mbar_init(smem_u32(&S.acc_full), 1);
     mbar_init(smem_u32(&S.done), 1);
+    mbar_init(smem_u32(&S.done_pv), 1);
     S.abort = 0;
     if (smem_u32(smem_raw) & 1023u) {                     // the swizzled tiles need this alignment
       atomicCAS(P.status, 0, 49);
@@ -212,32 +230,42 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
   grid_dependency_wait();
   grid_dependency_trigger();
 
-  // ---- K rows: 8 threads per key, one 16-byte piece each; Q rows: 4 threads per row, 2 pieces each
+  // ---- K rows (quantizers wider than 7 bits): a group stages the K tiles of its own visits, 8 threads per key with one
+  // 16-byte piece each, two keys per thread; Q rows: 4 threads per row, 2 pieces each
   const uint8_t* k_base = P.k + bo * P.k_so + bi * P.k_si;
-  const int kkey = (tid >> 3) & (kKeys - 1), kq = tid & 7;
-  uint4 kreg, knext;                            // the thread's piece of the K rows of the next two key blocks
-  bool k_live = false, k_live_next = false;     // whether that piece holds codes (key below Lk, piece below d_h)
-  auto fetch_k = [&](int block, uint4& dst, bool& live) {
-    dst = make_uint4(0u, 0u, 0u, 0u);
-    const int key = block * kKeys + kkey;
-    live = key < P.Lk && kq < pieces;
-    if (live) dst = __ldg(reinterpret_cast<const uint4*>(k_base + int64_t(key) * P.ldk) + kq);
+  const int gt = tid & (kGroupThreads - 1);       // thread in group
+  const int kkey = gt >> 3, kq = gt & 7;          // keys kkey, kkey + 32, ... of a visit
+  constexpr int kKeysPerThread = kKeys / 32;
+  uint4 kreg[kKeysPerThread];                                  // the thread's pieces of the K tile its group stages next
+  auto fetch_k = [&](int block) {
+#pragma unroll
+    for (int u = 0; u < kKeysPerThread; ++u) {
+      kreg[u] = make_uint4(0u, 0u, 0u, 0u);
+      const int key = block * kKeys + kkey + 32 * u;
+      if (key < P.Lk && kq < pieces) kreg[u] = __ldg(reinterpret_cast<const uint4*>(k_base + int64_t(key) * P.ldk) + kq);
+    }
   };
-  const uint32_t zk4 = uint32_t(P.zk) * 0x01010101u, zq4 = uint32_t(P.zq) * 0x01010101u;
-  auto store_k = [&](uint8_t* tile) {            // returns the code sum of the thread's key
-    if (kq < 2 * ksteps) *reinterpret_cast<uint4*>(tile + tile_offset(kkey, kq)) = kreg;
-    int s = sum_bytes(kreg);
-    s += __shfl_xor_sync(0xffffffffu, s, 1);
-    s += __shfl_xor_sync(0xffffffffu, s, 2);
-    s += __shfl_xor_sync(0xffffffffu, s, 4);
-    return s;
+  const uint32_t zq4 = uint32_t(P.zq) * 0x01010101u;
+  // K tile and column terms of visit g from kreg; then the pieces of the group's visit after that are requested
+  auto stage_k = [&](int g) {
+    uint8_t* tile = S.k[ring(g, kK)];
+#pragma unroll
+    for (int u = 0; u < kKeysPerThread; ++u) {
+      if (kq < 2 * ksteps) *reinterpret_cast<uint4*>(tile + tile_offset(kkey + 32 * u, kq)) = kreg[u];
+      int sum = sum_bytes(kreg[u]);
+      sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+      sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+      sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+      if (kq == 0) S.col_term[g & 3][kkey + 32 * u] = -P.zq * sum;
+    }
+    fence_async_smem();
+    __syncwarp();
+    if ((tid & 31) == 0) mbar_arrive(smem_u32(&S.k_full[ring(g, kK)]));
+    if (g + 2 < 2 * nb) fetch_k(g + 2 < nb ? g + 2 : g + 2 - nb);
   };
 
   if (warp < kWorkWarps) {
-    if (!kCentered) {
-      fetch_k(0, kreg, k_live);
-      fetch_k(nb > 1 ? 1 : 0, knext, k_live_next);
-    }
+    if (!kCentered && (tid >> 8) < 2 * nb) fetch_k((tid >> 8) < nb ? (tid >> 8) : (tid >> 8) - nb);   // the group's first visit
     const uint8_t* q_base = P.q + bo * P.q_so + bi * P.q_si;
     const int qrow = (tid >> 2) & (kRows - 1), qh = tid & 3;
     int s = 0;
@@ -270,6 +298,31 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
   const uint32_t tmem_base = S.tmem_base;
   volatile int* abort = &S.abort;
 
+  // P.V: D = f32, A = B = bf16, A from tensor memory, B MN-major, N = n_pad, M = 128
+  const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (uint32_t(P.n_pad >> 3) << 17) |
+                            (uint32_t(kRows >> 4) << 24);
+  // P.V MMAs of block j, from the operands the workers of visit nb + j left: A in tensor memory, in the columns of
+  // S(nb + j) (a row's E values of keys 16 s .. 16 s + 15 in the 8 columns from 16 s, its O values in the next 8),
+  // B = the V tile in shared memory
+  auto issue_pv = [&](int j) {
+    const int pb = ring(j, kP);
+    if (!mbar_wait(smem_u32(&S.p_full[pb]), lap(j, kP), abort, 43, P.status)) return false;
+    tc_fence_after();
+    const uint64_t dv = smem_desc_sw128(smem_u32(S.v[pb]), kVBlockBytes);
+    const int keys_here = min(kKeys, k_end - j * kKeys);
+    const int steps = (keys_here + 15) >> 4;                       // 16 keys per MMA
+    const uint32_t a_base = tmem_base + uint32_t(ring(nb + j, kS) * kKeys);
+    for (int s = 0; s < steps; ++s) {
+      const uint32_t accumulate = (j | s) != 0 ? 1u : 0u;
+      const uint32_t a_e = a_base + uint32_t(16 * s);
+      umma_f16_ts(tmem_base + uint32_t(kAccCol), a_e, dv + uint64_t(128 * s), idesc_pv, accumulate);
+      umma_f16_ts(tmem_base + uint32_t(kAccCol + P.n_pad), a_e + 8u, dv + uint64_t(128 * s), idesc_pv, accumulate);
+    }
+    umma_commit(smem_u32(&S.s_spent[ring(nb + j, kS)]));
+    umma_commit(smem_u32(&S.p_empty[pb]));
+    return true;
+  };
+
   if (warp == kWorkWarps) {
     // ---------------------------------------------------------------- MMA issue
     if (lane == 0) {
@@ -279,15 +332,20 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
       constexpr uint32_t idesc_s = kF8 ? (1u << 4) | (uint32_t(kKeys >> 3) << 17) | (uint32_t(kRows >> 4) << 24)
                                        : (2u << 4) | (uint32_t(kCentered) << 7) | (0u << 10) | (uint32_t(kKeys >> 3) << 17) |
                                              (uint32_t(kRows >> 4) << 24);
-      // P.V: D = f32, A = B = bf16, A K-major, B MN-major, N = n_pad, M = 128
-      const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (uint32_t(P.n_pad >> 3) << 17) |
-                                (uint32_t(kRows >> 4) << 24);
       const uint64_t dq = smem_desc_sw128(smem_u32(S.q));
       bool ok = true;
       auto issue_s = [&](int g) {                          // S of key block g % nb, g counted over both passes
         const int b = ring(g, kS), kb = ring(g, kK);
         if (!mbar_wait(smem_u32(&S.k_full[kb]), lap(g, kK), abort, 41, P.status)) return false;
-        if (!mbar_wait(smem_u32(&S.s_empty[b]), lap(g, kS) ^ 1u, abort, 42, P.status)) return false;
+        // the slot's last user: a pass-1 visit (the workers have read it) or a pass-2 visit (its P.V MMAs have read
+        // the operands the workers wrote over it)
+        const int prev = g - kS;
+        if (prev >= nb) {
+          const int first = nb + ((b - nb) & (kS - 1));         // the slot's first pass-2 visit
+          if (!mbar_wait(smem_u32(&S.s_spent[b]), lap(prev - first, kS), abort, 42, P.status)) return false;
+        } else if (prev >= 0) {
+          if (!mbar_wait(smem_u32(&S.s_empty[b]), lap(prev, kS), abort, 42, P.status)) return false;
+        }
         tc_fence_after();
         const uint64_t dk = smem_desc_sw128(smem_u32(S.k[kb]));
         for (int s = 0; s < ksteps; ++s) {
@@ -298,35 +356,33 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
         if (kCentered) umma_commit(smem_u32(&S.k_empty[kb]));     // the K tile may be refilled once these MMAs have read it
         return true;
       };
-      // S MMAs run ahead of the workers by as many visits as there are S buffers; the buffer of visit g is free once
-      // visit g - kS has been read, which the workers have done before they hand over the operand tiles of the P.V
-      // MMAs issued next, so this thread never sits in a wait for S while those tiles are ready
-      // (where the workers stage the K tiles themselves, one visit ahead, the S MMAs stay one visit ahead as well)
-      constexpr int kAhead = kCentered ? kS : 2;
-      int next_s = 0;
-      for (; next_s < nb + kAhead - 1 && next_s < 2 * nb && ok && !*abort; ++next_s) ok = issue_s(next_s);
-      for (int j = 0; j < nb && ok && !*abort; ++j) {
-        if (next_s < 2 * nb) {
-          if (!issue_s(next_s)) { ok = false; break; }
-          ++next_s;
+      if (kSplitIssue) {
+        // this thread issues the S MMAs only; each waits for its K tile and for its slot
+        for (int g = 0; g < 2 * nb && ok && !*abort; ++g) ok = issue_s(g);
+      } else {
+        // one thread for both: the S MMAs stay one visit ahead of the P.V MMAs
+        int next_s = 0;
+        for (; next_s < nb + 1 && next_s < 2 * nb && ok && !*abort; ++next_s) ok = issue_s(next_s);
+        for (int j = 0; j < nb && ok && !*abort; ++j) {
+          if (next_s < 2 * nb) {
+            if (!issue_s(next_s)) { ok = false; break; }
+            ++next_s;
+          }
+          ok = issue_pv(j);
         }
-        const int pb = ring(j, kP);
-        if (!mbar_wait(smem_u32(&S.p_full[pb]), lap(j, kP), abort, 43, P.status)) { ok = false; break; }
-        tc_fence_after();
-        const uint64_t de = smem_desc_sw128(smem_u32(S.e[pb])), dd = smem_desc_sw128(smem_u32(S.o[pb]));
-        const uint64_t dv = smem_desc_sw128(smem_u32(S.v[pb]), kVBlockBytes);
-        const int keys_here = min(kKeys, k_end - j * kKeys);
-        const int steps = (keys_here + 15) >> 4;                       // 16 keys per MMA
-        for (int s = 0; s < steps; ++s) {
-          const uint32_t accumulate = (j | s) != 0 ? 1u : 0u;
-          umma_f16(tmem_base + uint32_t(kAccCol), de + uint64_t(2 * s), dv + uint64_t(128 * s), idesc_pv, accumulate);
-          umma_f16(tmem_base + uint32_t(kAccCol + P.n_pad), dd + uint64_t(2 * s), dv + uint64_t(128 * s), idesc_pv, accumulate);
-        }
-        umma_commit(smem_u32(&S.p_empty[pb]));
+        if (ok && !*abort) umma_commit(smem_u32(&S.acc_full));
       }
-      if (ok && !*abort) umma_commit(smem_u32(&S.acc_full));
       umma_commit(smem_u32(&S.done));
       mbar_drain(smem_u32(&S.done), 0);
+    }
+  } else if (kSplitIssue && warp == kWorkWarps + 2) {
+    // ---------------------------------------------------------------- P.V MMA issue (wide heads)
+    if (lane == 0) {
+      bool ok = true;
+      for (int j = 0; j < nb && ok && !*abort; ++j) ok = issue_pv(j);
+      if (ok && !*abort) umma_commit(smem_u32(&S.acc_full));
+      umma_commit(smem_u32(&S.done_pv));
+      mbar_drain(smem_u32(&S.done_pv), 0);
     }
   } else if (warp == kWorkWarps + 1) {
     // ---------------------------------------------------------------- K tiles by bulk tensor copies
@@ -347,53 +403,38 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
     }
   } else {
     // ---------------------------------------------------------------- tiles, Softmax arithmetic, epilogue
-    const int quarter = warp & 3, part = warp >> 2;       // lane quarter of tensor memory, column part of the row
+    const int quarter = warp & 3, half = (warp >> 2) & 1, group = warp >> 3;
+    const int part = group * 2 + half;                    // which of the four threads of a row this one is
     const int r = quarter * 32 + lane;                    // the thread's row inside the CTA = its tensor-memory lane
     const int row = q0 + r;
     const int valid = row < P.Lq ? (P.causal ? max(1, min(P.Lk, row + 1 + shift)) : P.Lk) : 0;   // keys the row sees
     const int my_row_term = S.row_term[r];
-    // a warp whose 32 rows all lie past Lq (the tail of the last query tile): its rows of the E / O tiles are
-    // cleared once here and never written again, and it skips the code arithmetic of pass 2; it still stages K
-    // and V and arrives on every barrier
+    // a warp whose 32 rows all lie past Lq (the tail of the last query tile) skips the code arithmetic of pass 2 and
+    // writes zero operands; it still stages K and V and arrives on every barrier
     const bool dead_warp = __all_sync(0xffffffffu, valid == 0);
-    if (dead_warp) {
-#pragma unroll
-      for (int p4 = 0; p4 < kCols / 8; ++p4) {
-        const uint32_t off = tile_offset(r, part * (kCols / 8) + p4);
-#pragma unroll
-        for (int pb = 0; pb < kP; ++pb) {
-          *reinterpret_cast<uint4*>(S.e[pb] + off) = make_uint4(0u, 0u, 0u, 0u);
-          *reinterpret_cast<uint4*>(S.o[pb] + off) = make_uint4(0u, 0u, 0u, 0u);
-        }
-      }
-    }
     const float c = 1.4426950408889634f;
     const float k1 = -2.f * c;
     const float qs = float(P.qmax_p + 1), inv_qs = 1.f / qs;      // 2^bits and its reciprocal (exact)
     const uint32_t u_top = kMagicBits + uint32_t(P.qmax_p);
     const float magic = __uint_as_float(kMagicBits);
-    const uint32_t taddr_s = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(part * kCols);
+    const uint32_t taddr_s = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(half * kRuns * kCols);
 
-    // V items of a block (as in the P.V kernel): 2 NB groups of 8 channels per thread
-    const uint8_t* v_ptr[kVItems];
-    uint32_t v_off[kVItems];
-    int v_key[kVItems];
-#pragma unroll
-    for (int qi = 0; qi < kVItems; ++qi) {
-      const int i = tid + kWorkThreads * qi;
-      const int kr = i / (8 * NB), g8 = i % (8 * NB);
-      v_ptr[qi] = P.v + bo * P.v_so + bi * P.v_si + int64_t(kr) * P.ldv + g8 * 8;
-      v_off[qi] = uint32_t(g8 >> 3) * kVBlockBytes + tile_offset(kr, g8 & 7);
-      v_key[qi] = g8 * 8 < P.dh ? kr : -1;
-    }
-    const int64_t v_step = int64_t(kKeys) * P.ldv;
+    // V items of a visit: the group's 256 threads take the visit's keys x 8 NB groups of 8 channels in kVItems steps;
+    // a thread keeps its channel group and moves down the keys (32 / NB keys per step, a multiple of the swizzle period)
+    constexpr int kVKeyStep = 32 / NB;
+    constexpr int kVItems = kKeys / kVKeyStep;
+    const int v_g8 = gt % (8 * NB), v_key0 = gt / (8 * NB);
+    const bool v_chan_live = v_g8 * 8 < P.dh;
+    const uint8_t* v_ptr = P.v + bo * P.v_so + bi * P.v_si + int64_t(v_key0) * P.ldv + v_g8 * 8;
+    const uint32_t v_off = uint32_t(v_g8 >> 3) * kVBlockBytes + tile_offset(v_key0, v_g8 & 7);
     uint2 vraw[kVItems];
     auto fetch_v = [&](int block) {
 #pragma unroll
       for (int qi = 0; qi < kVItems; ++qi) {
         vraw[qi] = make_uint2(0u, 0u);
-        if (block < nb && v_key[qi] >= 0 && block * kKeys + v_key[qi] < P.Lk)
-          vraw[qi] = __ldg(reinterpret_cast<const uint2*>(v_ptr[qi] + block * v_step));
+        const int key = block * kKeys + v_key0 + qi * kVKeyStep;
+        if (block < nb && v_chan_live && key < P.Lk)
+          vraw[qi] = __ldg(reinterpret_cast<const uint2*>(v_ptr + int64_t(block * kKeys + qi * kVKeyStep) * P.ldv));
       }
     };
     const float vz = __uint_as_float(kMagicBits) + float(P.z_v);
@@ -402,29 +443,29 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
     float m = -CUDART_INF_F, z = 0.f;       // pass 1: running maximum and sum of this thread's columns
     float k0 = 0.f;                         // pass 2: 2 (log2 Z + log2 s), with m the row's final maximum
 
-    // The thread's 16 accumulators of visit g: load_s waits for the S MMAs and starts the load into rn, settle_s waits
-    // for the data and frees the buffer.
-    uint32_t rn[kCols];
-    auto load_s = [&](int g) -> bool {
-      const int b = ring(g, kS);
-      if (!mbar_wait(smem_u32(&S.s_full[b]), lap(g, kS), abort, 44, P.status)) return false;
+    // Start of a visit: the S MMAs of visit g have completed.  (Where the group stages its own K tiles, the tile of its
+    // next visit is written here: with a ring of two it is the tile those MMAs have just finished reading.)
+    auto begin_visit = [&](int g) -> bool {
+      if (!mbar_wait(smem_u32(&S.s_full[ring(g, kS)]), lap(g, kS), abort, 44, P.status)) return false;
       tc_fence_after();
-      __syncwarp();
-      tmem_ld16(taddr_s + uint32_t(b * kKeys), rn);
+      if (!kCentered && g + 2 < 2 * nb) stage_k(g + 2);
       return true;
     };
-    auto settle_s = [&](int g) {
-      tmem_ld_wait(rn);
-      tc_fence_before();
+    // Run h (16 columns) of the thread's scores of visit g in units of the score scale, as floats: the accumulator
+    // itself (kCentredF8), the converted accumulator (kCentred), or the converted corr = acc - z_k qsum - z_q ksum +
+    // d_h z_q z_k (kCorrected).  The buffer is handed back after the second run.  Keys the row may not see are dealt
+    // with by the callers, in the runs that reach past the keys the thread's row sees: the values themselves are left
+    // as they come from tensor memory, so that the common path carries no selects or copies.
+    auto read_run = [&](int g, int h, float (&sf)[kCols]) {
+      uint32_t rn[kCols];
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&S.s_empty[ring(g, kS)]));
-    };
-    // The scores of visit g in units of the score scale, as floats: the accumulator itself (kCentredF8), the converted
-    // accumulator (kCentred), or the converted corr = acc - z_k qsum - z_q ksum + d_h z_q z_k (kCorrected).  Keys the
-    // row may not see are dealt with by the callers, in the blocks that reach past the keys the thread's row sees
-    // (`edge`): the values themselves are left as they come from tensor memory, so that the common path carries no
-    // selects or copies.
-    auto scores = [&](int g, float (&sf)[kCols]) {
+      tmem_ld16(taddr_s + uint32_t(ring(g, kS) * kKeys + h * kCols), rn);
+      tmem_ld_wait();
+      if (h == kRuns - 1 && g < nb) {               // pass 1: the slot is free; pass 2: the operands go back into it
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&S.s_empty[ring(g, kS)]));
+      }
       if (kF8) {
 #pragma unroll
         for (int e = 0; e < kCols; ++e) sf[e] = __uint_as_float(rn[e]);
@@ -432,7 +473,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
 #pragma unroll
         for (int e = 0; e < kCols; ++e) sf[e] = float(int32_t(rn[e]));
       } else {
-        const int* ct = S.col_term[g & 3] + part * kCols;
+        const int* ct = S.col_term[g & 3] + (half * kRuns + h) * kCols;
 #pragma unroll
         for (int e4 = 0; e4 < kCols / 4; ++e4) {
           const int4 c4 = *reinterpret_cast<const int4*>(ct + 4 * e4);
@@ -444,88 +485,59 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
       }
     };
 
-    auto process = [&](int g) -> bool {
-      const int j = g < nb ? g : g - nb;
-      if (!load_s(g)) return false;
-      settle_s(g);
-      float sf[kCols];
-      scores(g, sf);
-      const bool edge = j * kKeys + part * kCols + kCols > valid;
-      const int seen = valid - (j * kKeys + part * kCols);       // columns e < seen are keys the row sees
-      if (g < nb) {
-        // ---- pass 1: running maximum and sum.  The maximum is taken on the unscaled values (S = scale * sf is
-        // monotonic in sf); a key the row may not see contributes nothing.  Exponents and sums on packed pairs.
-        const float sc = P.scale * c;                             // exponent of 2 per unit of sf
-        if (__builtin_expect(!edge, 1)) {
-          float bm = max3(sf[0], sf[1], sf[2]);
+    // ---- pass 1: running maximum and sum of one run.  The maximum is taken on the unscaled values (S = scale * sf is
+    // monotonic in sf); a key the row may not see contributes nothing (`seen`: columns e < seen are keys the row sees).
+    // Exponents and sums on packed pairs.
+    auto stats_run = [&](const float (&sf)[kCols], int seen) {
+      const float sc = P.scale * c;                             // exponent of 2 per unit of sf
+      if (__builtin_expect(seen >= kCols, 1)) {
+        float bm = max3(sf[0], sf[1], sf[2]);
 #pragma unroll
-          for (int e = 3; e + 1 < kCols; e += 2) bm = max3(bm, sf[e], sf[e + 1]);
-          bm = fmaxf(bm, sf[kCols - 1]);
-          const float mn = fmaxf(m, P.scale * bm);
-          const f32x2 sc2 = splat2(sc), nm2 = splat2(-(mn * c));
-          f32x2 acc = 0ull;                                       // even columns in the low lane, odd ones in the high lane
+        for (int e = 3; e + 1 < kCols; e += 2) bm = max3(bm, sf[e], sf[e + 1]);
+        bm = fmaxf(bm, sf[kCols - 1]);
+        const float mn = fmaxf(m, P.scale * bm);
+        const f32x2 sc2 = splat2(sc), nm2 = splat2(-(mn * c));
+        f32x2 acc = 0ull;                                       // even columns in the low lane, odd ones in the high lane
 #pragma unroll
-          for (int e = 0; e < kCols; e += 2) {
-            float a0, a1;
-            unpack2(fma2(pack2(sf[e], sf[e + 1]), sc2, nm2), a0, a1);
-            acc = add2(acc, pack2(ex2(a0), ex2(a1)));
-          }
-          float acc0, acc1;
-          unpack2(acc, acc0, acc1);
-          z = z * ex2((m - mn) * c) + (acc0 + acc1);     // m = -inf at first: factor 0
-          m = mn;
-        } else if (seen > 0) {
-          float bm = sf[0];
-#pragma unroll
-          for (int e = 1; e < kCols; ++e)
-            if (e < seen) bm = fmaxf(bm, sf[e]);
-          const float mn = fmaxf(m, P.scale * bm);
-          const float mnc = mn * c;
-          float acc = 0.f;
-#pragma unroll
-          for (int e = 0; e < kCols; ++e)
-            if (e < seen) acc += ex2(fmaf(sf[e], sc, -mnc));
-          z = z * ex2((m - mn) * c) + acc;
-          m = mn;
+        for (int e = 0; e < kCols; e += 2) {
+          float a0, a1;
+          unpack2(fma2(pack2(sf[e], sf[e + 1]), sc2, nm2), a0, a1);
+          acc = add2(acc, pack2(ex2(a0), ex2(a1)));
         }
-        if (g == nb - 1) {
-          // merge the column parts of every row: m = max, Z = sum of the rescaled partial sums (same order in
-          // every thread of the row, so that all of them hold the same Z)
-          S.stat_m[part][r] = m;
-          S.stat_z[part][r] = z;
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&S.stats_ready));
-          if (!mbar_wait(smem_u32(&S.stats_ready), 0, abort, 45, P.status)) return false;
-          float mn = -CUDART_INF_F;
+        float acc0, acc1;
+        unpack2(acc, acc0, acc1);
+        z = z * ex2((m - mn) * c) + (acc0 + acc1);     // m = -inf at first: factor 0
+        m = mn;
+      } else if (seen > 0) {
+        float bm = sf[0];
 #pragma unroll
-          for (int q = 0; q < kParts; ++q) mn = fmaxf(mn, S.stat_m[q][r]);
-          float zt = 0.f;
+        for (int e = 1; e < kCols; ++e)
+          if (e < seen) bm = fmaxf(bm, sf[e]);
+        const float mn = fmaxf(m, P.scale * bm);
+        const float mnc = mn * c;
+        float acc = 0.f;
 #pragma unroll
-          for (int q = 0; q < kParts; ++q) {
-            const float mq = S.stat_m[q][r];
-            if (mq > -CUDART_INF_F) zt += S.stat_z[q][r] * ex2((mq - mn) * c);
-          }
-          m = mn;
-          k0 = 2.f * (log2f(zt) + P.log2_s);
-          fetch_v(0);
-        }
-        return true;
+        for (int e = 0; e < kCols; ++e)
+          if (e < seen) acc += ex2(fmaf(sf[e], sc, -mnc));
+        z = z * ex2((m - mn) * c) + acc;
+        m = mn;
       }
-      // ---- pass 2: codes, operand tiles, V tile.
-      // Eq. 15: p = clip(round(t), 0, qmax), t = k0 - 2 c (S - m); rounding half to even by the float add of
-      // 1.5 * 2^23, which leaves p in the low mantissa bits u - kMagicBits.  The pair (E, O) of bf16 operand values,
-      // 2^-ceil(p/2) on the side of p's parity and 0 on the other, comes from a per-lane table for 4-bit codes and
-      // from integer arithmetic for wider ones.  A masked key gets (0, 0).
-      const uint32_t lut_addr = smem_u32(&S.lut[0][lane]) - (kMagicBits << 7);
-      uint4 ev[kCols / 8], ov[kCols / 8];
-      // a warp none of whose rows sees a key of its 16 columns (the block past the last key, the blocks beyond the
-      // diagonal under a causal mask) writes zero operands without any arithmetic
-      const bool idle = !dead_warp && !__any_sync(0xffffffffu, seen > 0);
-      if (idle) {
+    };
+
+    // ---- pass 2: codes and operand values of one run.
+    // Eq. 15: p = clip(round(t), 0, qmax), t = k0 - 2 c (S - m); rounding half to even by the float add of
+    // 1.5 * 2^23, which leaves p in the low mantissa bits u - kMagicBits.  The pair (E, O) of bf16 operand values,
+    // 2^-ceil(p/2) on the side of p's parity and 0 on the other, comes from a per-lane table for 4-bit codes and
+    // from integer arithmetic for wider ones.  A masked key gets (0, 0).
+    const uint32_t lut_addr = smem_u32(&S.lut[0][lane]) - (kMagicBits << 7);
+    auto code_run = [&](const float (&sf)[kCols], int seen, uint32_t (&eow)[kCols]) {
+      // a warp none of whose rows sees a key of the run (the block past the last key, the blocks beyond the diagonal
+      // under a causal mask) writes zero operands without any arithmetic
+      if (dead_warp || !__any_sync(0xffffffffu, seen > 0)) {
 #pragma unroll
-        for (int p4 = 0; p4 < kCols / 8; ++p4) ev[p4] = ov[p4] = make_uint4(0u, 0u, 0u, 0u);
+        for (int e = 0; e < kCols; ++e) eow[e] = 0u;
+        return;
       }
-      if (!dead_warp && !idle) {
       uint32_t eo[kCols];
       // S - m on packed pairs; then t 2^-bits out of one saturating fma each (k1 and k0 scaled by 2^-bits, exact, so the
       // value is t rounded as before and clamped to [0, 1] whatever the inputs: rows past Lq carry m = -inf, Z = 0), and
@@ -556,35 +568,79 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
           }
         }
       }
-      if (__builtin_expect(edge, 0)) {
+      if (__builtin_expect(seen < kCols, 0)) {
 #pragma unroll
         for (int e = 0; e < kCols; ++e)
           if (e >= seen) eo[e] = 0u;
       }
+      // E pairs (even key in the low half) in words 0..7, O pairs in words 8..15
 #pragma unroll
-      for (int p4 = 0; p4 < kCols / 8; ++p4) {
-        ev[p4] = make_uint4(__byte_perm(eo[8 * p4 + 0], eo[8 * p4 + 1], 0x5410), __byte_perm(eo[8 * p4 + 2], eo[8 * p4 + 3], 0x5410),
-                            __byte_perm(eo[8 * p4 + 4], eo[8 * p4 + 5], 0x5410), __byte_perm(eo[8 * p4 + 6], eo[8 * p4 + 7], 0x5410));
-        ov[p4] = make_uint4(__byte_perm(eo[8 * p4 + 0], eo[8 * p4 + 1], 0x7632), __byte_perm(eo[8 * p4 + 2], eo[8 * p4 + 3], 0x7632),
-                            __byte_perm(eo[8 * p4 + 4], eo[8 * p4 + 5], 0x7632), __byte_perm(eo[8 * p4 + 6], eo[8 * p4 + 7], 0x7632));
+      for (int e = 0; e < kCols / 2; ++e) {
+        eow[e] = __byte_perm(eo[2 * e], eo[2 * e + 1], 0x5410);
+        eow[kCols / 2 + e] = __byte_perm(eo[2 * e], eo[2 * e + 1], 0x7632);
       }
+    };
+
+    bool ok = true;
+    if (!kCentered && group < 2 * nb) stage_k(group);          // the K tile of the group's first visit
+    // ---- pass 1 over the group's visits
+    for (int g = group; g < nb && !*abort; g += 2) {
+      if (!begin_visit(g)) { ok = false; break; }
+      const int seen = valid - (g * kKeys + half * kRuns * kCols);   // of the thread's columns
+#pragma unroll
+      for (int h = 0; h < kRuns; ++h) {
+        float sf[kCols];
+        read_run(g, h, sf);
+        stats_run(sf, seen - h * kCols);
       }
-      // one stage of operand tiles: the MMAs of the block before must have read them (the code arithmetic above
-      // has overlapped with those MMAs)
+    }
+    // merge the four column parts of every row: m = max, Z = sum of the rescaled partial sums (same order in every
+    // thread of the row, so that all of them hold the same Z)
+    if (ok && !*abort) {
+      S.stat_m[part][r] = m;
+      S.stat_z[part][r] = z;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&S.stats_ready));
+      ok = mbar_wait(smem_u32(&S.stats_ready), 0, abort, 45, P.status);
+    }
+    const int g2 = nb + ((nb ^ group) & 1);                     // the group's first visit of pass 2
+    if (ok && !*abort) {
+      float mn = -CUDART_INF_F;
+#pragma unroll
+      for (int q = 0; q < kParts; ++q) mn = fmaxf(mn, S.stat_m[q][r]);
+      float zt = 0.f;
+#pragma unroll
+      for (int q = 0; q < kParts; ++q) {
+        const float mq = S.stat_m[q][r];
+        if (mq > -CUDART_INF_F) zt += S.stat_z[q][r] * ex2((mq - mn) * c);
+      }
+      m = mn;
+      k0 = 2.f * (log2f(zt) + P.log2_s);
+      fetch_v(g2 - nb);
+    }
+    // ---- pass 2 over the group's visits
+    for (int g = g2; g < 2 * nb && ok && !*abort; g += 2) {
+      const int j = g - nb;
+      if (!begin_visit(g)) { ok = false; break; }
+      const int seen = valid - (j * kKeys + half * kRuns * kCols);
+      // E and O operands of a run: bf16 pairs written back over the run's own 16 columns of S(g) (8 columns of E, then 8
+      // of O), from where the P.V MMAs take their A operand; nothing else reads those columns any more
+#pragma unroll
+      for (int h = 0; h < kRuns; ++h) {
+        float sf[kCols];
+        read_run(g, h, sf);
+        uint32_t eow[kCols];
+        code_run(sf, seen - h * kCols, eow);
+        __syncwarp();
+        tmem_st16(taddr_s + uint32_t(ring(g, kS) * kKeys + h * kCols), eow);
+      }
+      // the stage of the V tile: the MMAs of the block that used it before must have read it
       const int pb = ring(j, kP);
-      if (!mbar_wait(smem_u32(&S.p_empty[pb]), lap(j, kP) ^ 1u, abort, 46, P.status)) return false;
-      if (!dead_warp) {
-#pragma unroll
-        for (int p4 = 0; p4 < kCols / 8; ++p4) {
-          const uint32_t off = tile_offset(r, part * (kCols / 8) + p4);
-          *reinterpret_cast<uint4*>(S.e[pb] + off) = ev[p4];
-          *reinterpret_cast<uint4*>(S.o[pb] + off) = ov[p4];
-        }
-      }
+      if (!mbar_wait(smem_u32(&S.p_empty[pb]), lap(j, kP) ^ 1u, abort, 46, P.status)) { ok = false; break; }
 #pragma unroll
       for (int qi = 0; qi < kVItems; ++qi) {
         uint32_t o4[4] = {0u, 0u, 0u, 0u};
-        if (v_key[qi] >= 0 && j * kKeys + v_key[qi] < P.Lk) {
+        if (v_chan_live && j * kKeys + v_key0 + qi * kVKeyStep < P.Lk) {
           const uint32_t b03 = vraw[qi].x, b47 = vraw[qi].y;
           if (P.v_small) {
             // v - z_v as bf16: for codes below 128, 128 + v is the bit pattern 0x4300 | v and the bf16 subtraction exact
@@ -592,8 +648,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
                                    __byte_perm(b47, 0x43434343u, 0x4140), __byte_perm(b47, 0x43434343u, 0x4342)};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              const __nv_bfloat162 h = __hsub2(*reinterpret_cast<const __nv_bfloat162*>(&w[e]), vz2);
-              o4[e] = *reinterpret_cast<const uint32_t*>(&h);
+              const __nv_bfloat162 hh = __hsub2(*reinterpret_cast<const __nv_bfloat162*>(&w[e]), vz2);
+              o4[e] = *reinterpret_cast<const uint32_t*>(&hh);
             }
           } else {
             float f[8];
@@ -604,37 +660,20 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
             }
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              const __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * e], f[2 * e + 1]);
-              o4[e] = *reinterpret_cast<const uint32_t*>(&h);
+              const __nv_bfloat162 hh = __floats2bfloat162_rn(f[2 * e], f[2 * e + 1]);
+              o4[e] = *reinterpret_cast<const uint32_t*>(&hh);
             }
           }
         }
-        *reinterpret_cast<uint4*>(S.v[pb] + v_off[qi]) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+        *reinterpret_cast<uint4*>(S.v[pb] + v_off + uint32_t(qi * (kVKeyStep / 8)) * 1024u) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
       }
-      fetch_v(j + 1);
+      fetch_v(j + 2);
       fence_async_smem();
+      tmem_st_wait();
+      tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&S.p_full[pb]));
-      return true;
-    };
-
-    bool ok = true;
-    for (int g = 0; g < 2 * nb && !*abort; ++g) {
-      if (!kCentered) {
-        // tile g & 1 was last read by the S MMAs of g - 2, whose result this thread has already waited for
-        const int ks = store_k(S.k[ring(g, kK)]);
-        if (kq == 0) S.col_term[g & 3][kkey] = -P.zq * ks;
-        fence_async_smem();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&S.k_full[ring(g, kK)]));
-        kreg = knext;
-        k_live = k_live_next;
-        // two blocks ahead (global latency is about one block); g + 2 < 2 nb, so the block index needs no division
-        if (g + 2 < 2 * nb) fetch_k(g + 2 < nb ? g + 2 : g + 2 - nb, knext, k_live_next);
-      }
-      if (g > 0 && !process(g - 1)) { ok = false; break; }
     }
-    if (ok && !*abort) ok = process(2 * nb - 1);
 
     // ---------------------------------------------------------------- epilogue: one row per thread, the 16-column
     // chunks of the accumulators dealt to the four warps of a lane quarter
@@ -716,7 +755,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
   }
 
   // ------------------------------------------------------------------ teardown
-  if (warp < kWorkWarps) tmem_ld_wait();          // an error path may leave a tensor-memory load in flight
+  if (warp < kWorkWarps) tmem_st_wait();          // an error path may leave a tensor-memory store in flight
   tc_fence_before();
   __syncthreads();
   if (warp == kWorkWarps) {
@@ -725,14 +764,14 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
   }
 }
 
-// Tensor map of the K codes for the bulk-copy variant: (bytes of a row, keys, batch items); a box is 128 bytes x 64 keys.
-repq_status make_k_map(CUtensorMap* map, const AttnParams& P, int batch_outer) {
+// Tensor map of the K codes for the bulk-copy variant: (bytes of a row, keys, batch items); a box is 128 bytes x the keys of a visit.
+repq_status make_k_map(CUtensorMap* map, const AttnParams& P, int batch_outer, int keys) {
   EncodeTiledFn fn = encode_fn();
   REPQ_REQUIRE(fn != nullptr, REPQ_CUDA_ERROR, "attention: cuTensorMapEncodeTiled is not available");
   const cuuint64_t span = cuuint64_t(P.batch_inner - 1) * cuuint64_t(P.k_si) + cuuint64_t(P.dh);    // bytes the heads cover
   const cuuint64_t dims[3] = {span, cuuint64_t(P.Lk), cuuint64_t(batch_outer)};
   const cuuint64_t strides[2] = {cuuint64_t(P.ldk), cuuint64_t(P.k_so)};
-  const cuuint32_t box[3] = {128, cuuint32_t(kKeys), 1};
+  const cuuint32_t box[3] = {128, cuuint32_t(keys), 1};
   const cuuint32_t estr[3] = {1, 1, 1};
   const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<uint8_t*>(P.k), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -750,9 +789,9 @@ repq_status launch_kernel(const AttnParams& P, int64_t pairs, cudaStream_t st) {
   Q.tiles = (P.Lq + kRows - 1) / kRows;
   if (kMode == kCentredF8) Q.scale = P.scale * 262144.f;      // the accumulators hold 2^-18 sum (q - z_q) k
   CUtensorMap map_k{};
-  if (kMode != kCorrected) REPQ_TRY(make_k_map(&map_k, P, int(pairs / P.batch_inner)));
+  if (kMode != kCorrected) REPQ_TRY(make_k_map(&map_k, P, int(pairs / P.batch_inner), VisitKeys<NB>::value));
   dim3 grid(unsigned(Q.tiles) * unsigned(pairs));
-  REPQ_CUDA(launch_chained(attention_tc_kernel<NB, kLutBits, kMode>, grid, dim3(kThreads), smem, st, map_k, Q));
+  REPQ_CUDA(launch_chained(attention_tc_kernel<NB, kLutBits, kMode>, grid, dim3(Threads<NB>::value), smem, st, map_k, Q));
   note_launch();
   return REPQ_OK;
 }
