@@ -6,6 +6,7 @@
 #include <cstdint>
 
 #include "../../include/repq.h"
+#include "f32x2.cuh"
 
 namespace repq {
 
@@ -85,6 +86,26 @@ __device__ __forceinline__ float gelu_erf(float v) {
   float h;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(h) : "f"(fmaf(-t, q, -1.f)));
   return v * (v < 0.f ? h : 1.f - h);
+}
+
+// The same on two values at once (packed float pairs where the operation exists in that form): every lane goes through
+// the operations of gelu_erf in the same order, so the results are the same bits.
+__device__ __forceinline__ void gelu_erf_pair(float& v0, float& v1) {
+  float a0, a1;
+  unpack2(mul2(pack2(v0, v1), splat2(0.70710678118654752f)), a0, a1);       // |v| c = |v c|
+  const f32x2 t = pack2(fminf(fabsf(a0), 4.f), fminf(fabsf(a1), 4.f));
+  f32x2 q = splat2(-1.002269491e-04f);
+  q = fma2(q, t, splat2(4.616116930e-04f));
+  q = fma2(q, t, splat2(2.302142326e-03f));
+  q = fma2(q, t, splat2(-2.945240214e-02f));
+  q = fma2(q, t, splat2(1.489636004e-01f));
+  q = fma2(q, t, splat2(9.183286428e-01f));
+  q = fma2(q, t, splat2(1.627913713e+00f));
+  float e0, e1, h0, h1;
+  unpack2(fma2(t, q, splat2(1.f)), e0, e1);                                  // fma(-t, q, -1) = -fma(t, q, 1)
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(h0) : "f"(-e0));
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(h1) : "f"(-e1));
+  unpack2(mul2(pack2(v0, v1), pack2(v0 < 0.f ? h0 : 1.f - h0, v1 < 0.f ? h1 : 1.f - h1)), v0, v1);
 }
 
 // acc -> corrected integer -> float value before the output conversion.

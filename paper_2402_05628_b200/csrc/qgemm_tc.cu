@@ -118,6 +118,45 @@ constexpr uint32_t idesc_for(int bn) {
   return (2u << 4) | (0u << 7) | (0u << 10) | (uint32_t(bn >> 3) << 17) | (uint32_t(BM >> 4) << 24);
 }
 
+// Order of the output tiles.  The row tiles are cut into panels of P.panel; a panel is walked column tile by column
+// tile with its row tiles innermost.  The CTAs that run at the same time then share a panel of activations small
+// enough to stay in L2 while the weight tiles stream past it (with long K the activations of all row tiles do not
+// fit, and walking every row tile per column tile read them from DRAM once per wave of CTAs).
+// Every role of the CTA needs the origin of every tile it visits, and a division by a run-time number is a chain of
+// some 25 dependent instructions that all epilogue warps would walk through at the same moment; the divisors are
+// fixed per launch, so the host supplies their reciprocals (n / d = umulhi(n, ceil(2^32 / d)) while n d < 2^32).
+struct FastDiv { uint32_t d, mul; };                            // mul == 0: plain division
+inline FastDiv fast_div(uint32_t d, uint64_t n_max) {
+  FastDiv f{d, 0u};
+  if (d > 1 && n_max * d < (uint64_t(1) << 32)) f.mul = uint32_t((uint64_t(1) << 32) / d) + 1u;
+  return f;
+}
+__device__ __forceinline__ uint32_t div_by(uint32_t n, const FastDiv& f) { return f.mul ? __umulhi(n, f.mul) : n / f.d; }
+struct TileOrder {
+  int full;                    // tiles inside whole panels
+  int panel, last_rows;        // row tiles of a whole panel and of the last, shorter one
+  int m_tiles;
+  FastDiv by_panel_tiles;      // panel * n_tiles
+  FastDiv by_panel, by_last_rows;
+};
+struct TileOrigin { int m0, n0; };
+__device__ __forceinline__ TileOrigin tile_origin(int tile, const TileOrder& T, int bn) {
+  uint32_t rows = uint32_t(T.panel), first = 0, t = uint32_t(tile);
+  uint32_t col;
+  if (tile >= T.full) {                                          // the last, shorter panel
+    t = uint32_t(tile - T.full);
+    rows = uint32_t(T.last_rows);
+    first = uint32_t(T.m_tiles) - rows;
+    col = div_by(t, T.by_last_rows);
+  } else {
+    const uint32_t p = div_by(t, T.by_panel_tiles);
+    first = p * uint32_t(T.panel);
+    t -= p * T.by_panel_tiles.d;
+    col = div_by(t, T.by_panel);
+  }
+  return TileOrigin{int(first + (t - col * rows)) * BM, int(col) * bn};
+}
+
 struct TcParams {
   int M, N, K;
   const int32_t* asum;
@@ -125,30 +164,11 @@ struct TcParams {
   int direct_requant;          // codes out, no GELU, no residual: 1/s_o is folded into the column terms
   int w_packed4;               // weight tiles arrive packed (4: two codes per byte, 6: four in three bytes) and are
                                // expanded in shared memory; 0: byte tiles
-  int panel;                   // row tiles per panel of the tile order
+  TileOrder order;             // panels of row tiles (see TileOrder)
   EpilogueParams ep;
 };
 
 enum : int { kOutF32 = 0, kOutBf16 = 1, kOutC4 = 2, kOutC8 = 3 };   // compile-time output kinds of the fast path
-
-// Order of the output tiles.  The row tiles are cut into panels of P.panel; a panel is walked column tile by column
-// tile with its row tiles innermost.  The CTAs that run at the same time then share a panel of activations small
-// enough to stay in L2 while the weight tiles stream past it (with long K the activations of all row tiles do not
-// fit, and walking every row tile per column tile read them from DRAM once per wave of CTAs).
-struct TileOrigin { int m0, n0; };
-__device__ __forceinline__ TileOrigin tile_origin(int tile, int m_tiles, int n_tiles, int panel, int bn) {
-  const int full = (m_tiles / panel) * panel * n_tiles;       // tiles inside whole panels
-  int rows = panel, first = 0, t = tile;
-  if (tile >= full) {                                          // the last, shorter panel
-    t = tile - full;
-    rows = m_tiles - (m_tiles / panel) * panel;
-    first = m_tiles - rows;
-  } else {
-    first = (tile / (panel * n_tiles)) * panel;
-    t = tile % (panel * n_tiles);
-  }
-  return TileOrigin{(first + t % rows) * BM, (t / rows) * bn};
-}
 
 // Output quantizer of one 16-column chunk (Eq. 4 with the chunk's column group).
 struct ChunkQuant {
@@ -250,12 +270,16 @@ __device__ __forceinline__ void emit_chunk(const CUtensorMap* map_out, uint32_t 
       // saturating fma whose unclamped result is exact, u = magic + 2^bits w.  The low byte of u is the code,
       // except that 2^bits stands for the top code 2^bits - 1; that bit is subtracted after packing.
       uint32_t w[4];
-      if (direct) {
+      // (the adds and multiply-adds around the saturating one on packed pairs: same operations, same bits)
+      const f32x2 magic2 = splat2(magic), qs2 = splat2(q.qs), mult2 = splat2(q.mult);
 #pragma unroll
-        for (int e = 0; e < kChunk; ++e) u[e] = __float_as_uint(fmaf(fma_sat(v[e] + magic, q.inv_qs, q.csat), q.qs, magic));
-      } else {
-#pragma unroll
-        for (int e = 0; e < kChunk; ++e) u[e] = __float_as_uint(fmaf(fma_sat(fmaf(v[e], q.mult, magic), q.inv_qs, q.csat), q.qs, magic));
+      for (int e = 0; e < kChunk; e += 2) {
+        float r0, r1, u0, u1;
+        const f32x2 v2 = pack2(v[e], v[e + 1]);
+        unpack2(direct ? add2(v2, magic2) : fma2(v2, mult2, magic2), r0, r1);
+        unpack2(fma2(pack2(fma_sat(r0, q.inv_qs, q.csat), fma_sat(r1, q.inv_qs, q.csat)), qs2, magic2), u0, u1);
+        u[e] = __float_as_uint(u0);
+        u[e + 1] = __float_as_uint(u1);
       }
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
@@ -268,10 +292,16 @@ __device__ __forceinline__ void emit_chunk(const CUtensorMap* map_out, uint32_t 
       if (c & 1) box_end(map_out, buf, lane, col0 - kChunk, row0);
       return;
     }
+    {
+      const f32x2 magic2 = splat2(magic), mult2 = splat2(q.mult);
 #pragma unroll
-    for (int e = 0; e < kChunk; ++e) {
-      const float t = fminf(fmaxf(v[e] * q.mult, q.lo), q.hi);
-      u[e] = __float_as_uint(t + magic);             // magic_bits + round_half_even(t)
+      for (int e = 0; e < kChunk; e += 2) {
+        float t0, t1, u0, u1;
+        unpack2(mul2(pack2(v[e], v[e + 1]), mult2), t0, t1);
+        unpack2(add2(pack2(fminf(fmaxf(t0, q.lo), q.hi), fminf(fmaxf(t1, q.lo), q.hi)), magic2), u0, u1);   // magic_bits + round_half_even(t)
+        u[e] = __float_as_uint(u0);
+        u[e + 1] = __float_as_uint(u1);
+      }
     }
     if constexpr (OUT == kOutC4) {
       uint32_t w[2];
@@ -424,7 +454,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       uint32_t stage = 0, phase = 0;
       long long issued = 0;
       for (int tile = blockIdx.x; tile < tiles && !*abort; tile += gridDim.x) {
-        const TileOrigin o = tile_origin(tile, m_tiles, n_tiles, P.panel, BN);
+        const TileOrigin o = tile_origin(tile, P.order, BN);
         const int m0 = o.m0, n0 = o.n0;
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!mbar_wait(smem_u32(&S.empty[stage]), phase ^ 1, abort, 1)) break;
@@ -573,7 +603,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     float nx_sw[2] = {0.f, 0.f}, nx_bs[2] = {0.f, 0.f};
     auto fetch_terms = [&](int t) {
       if (t >= tiles || !slice_on) return;
-      const TileOrigin o = tile_origin(t, m_tiles, n_tiles, P.panel, BN);
+      const TileOrigin o = tile_origin(t, P.order, BN);
       const int tm0 = o.m0, tn0 = o.n0;
       // plain loads from clamped indices: nothing here may consume a loaded value (a select on it would hold the
       // warp until the load returns); rows and columns outside the matrix are dealt with where the values are used
@@ -594,7 +624,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     bool res_pending = false;
     auto fetch_residual = [&](int t) {
       if (!RES || t >= tiles || !slice_on) return;
-      const TileOrigin o = tile_origin(t, m_tiles, n_tiles, P.panel, BN);
+      const TileOrigin o = tile_origin(t, P.order, BN);
       const int tm0 = o.m0, tn0 = o.n0;
       if (lane == 0) {
         mbar_expect_tx(res_bar, kResBytes);
@@ -607,7 +637,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     int it = 0;
     for (int tile = blockIdx.x; tile < tiles && !*abort; tile += gridDim.x, ++it) {
       const uint32_t acc = it & 1, acc_phase = (it >> 1) & 1;
-      const TileOrigin o = tile_origin(tile, m_tiles, n_tiles, P.panel, BN);
+      const TileOrigin o = tile_origin(tile, P.order, BN);
       const int m0 = o.m0, n0 = o.n0;
       const int64_t m = int64_t(m0) + quarter * 32 + lane;
       const bool row_ok = m < P.M;
@@ -677,14 +707,14 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             const int4 kw = *reinterpret_cast<const int4*>(&C.kw[c * kChunk + 4 * q4]);
             const float4 sc = *reinterpret_cast<const float4*>(&C.sc[c * kChunk + 4 * q4]);
             const float4 bi = *reinterpret_cast<const float4*>(&C.bi[c * kChunk + 4 * q4]);
-            v[4 * q4 + 0] = fmaf(sc.x, float(int32_t(r[4 * q4 + 0]) + nz.x * asum_c + kw.x), bi.x);
-            v[4 * q4 + 1] = fmaf(sc.y, float(int32_t(r[4 * q4 + 1]) + nz.y * asum_c + kw.y), bi.y);
-            v[4 * q4 + 2] = fmaf(sc.z, float(int32_t(r[4 * q4 + 2]) + nz.z * asum_c + kw.z), bi.z);
-            v[4 * q4 + 3] = fmaf(sc.w, float(int32_t(r[4 * q4 + 3]) + nz.w * asum_c + kw.w), bi.w);
+            const float f0 = float(int32_t(r[4 * q4 + 0]) + nz.x * asum_c + kw.x), f1 = float(int32_t(r[4 * q4 + 1]) + nz.y * asum_c + kw.y);
+            const float f2 = float(int32_t(r[4 * q4 + 2]) + nz.z * asum_c + kw.z), f3 = float(int32_t(r[4 * q4 + 3]) + nz.w * asum_c + kw.w);
+            unpack2(fma2(pack2(sc.x, sc.y), pack2(f0, f1), pack2(bi.x, bi.y)), v[4 * q4 + 0], v[4 * q4 + 1]);
+            unpack2(fma2(pack2(sc.z, sc.w), pack2(f2, f3), pack2(bi.z, bi.w)), v[4 * q4 + 2], v[4 * q4 + 3]);
           }
           if (ep.gelu) {
 #pragma unroll
-            for (int e = 0; e < kChunk; ++e) v[e] = gelu_erf(v[e]);
+            for (int e = 0; e < kChunk; e += 2) gelu_erf_pair(v[e], v[e + 1]);
           }
           if (res32 && row_ok) {
             // float32 residual: read where it is used (16 columns = four 16-byte loads of this thread's row)
@@ -709,10 +739,9 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
               }
               const uint32_t ws[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
-              for (int k = 0; k < 4; ++k) {
-                v[i * 8 + 2 * k] += __uint_as_float(ws[k] << 16);
-                v[i * 8 + 2 * k + 1] += __uint_as_float(ws[k] & 0xffff0000u);
-              }
+              for (int k = 0; k < 4; ++k)
+                unpack2(add2(pack2(v[i * 8 + 2 * k], v[i * 8 + 2 * k + 1]), pack2(__uint_as_float(ws[k] << 16), __uint_as_float(ws[k] & 0xffff0000u))),
+                        v[i * 8 + 2 * k], v[i * 8 + 2 * k + 1]);
             }
           }
           if (PAIR == kPairRope && rope_row != nullptr && col0 < ep.rope_cols) {       // warp-uniform: range edges fall on chunk edges
@@ -1009,10 +1038,19 @@ repq_status qgemm_tc(const repq_gemm_desc& d, const EpilogueParams& ep, void* ws
   const int bn = pick_bn(d.M, d.N, sms, P.w_packed4 != 0);
   {
     // panels of activations of about 40 MB (a third of the L2 capacity), at least 8 row tiles
-    const int m_tiles = (d.M + BM - 1) / BM;
+    const int m_tiles = (d.M + BM - 1) / BM, n_tiles = (d.N + bn - 1) / bn;
     const int64_t fit = (int64_t(40) << 20) / (int64_t(BM) * d.K);
-    P.panel = int(fit < 8 ? 8 : fit);
-    if (P.panel > m_tiles) P.panel = m_tiles;
+    int panel = int(fit < 8 ? 8 : fit);
+    if (panel > m_tiles) panel = m_tiles;
+    TileOrder& T = P.order;
+    T.panel = panel;
+    T.m_tiles = m_tiles;
+    T.last_rows = m_tiles - (m_tiles / panel) * panel;
+    T.full = (m_tiles / panel) * panel * n_tiles;
+    const uint64_t tiles = uint64_t(m_tiles) * uint64_t(n_tiles);
+    T.by_panel_tiles = fast_div(uint32_t(panel) * uint32_t(n_tiles), tiles);
+    T.by_panel = fast_div(uint32_t(panel), tiles);
+    T.by_last_rows = fast_div(uint32_t(T.last_rows > 0 ? T.last_rows : 1), tiles);
   }
   CUtensorMap map_a, map_b;
   REPQ_TRY(make_map(&map_a, a, d.M, d.K, lda, BM));
