@@ -68,25 +68,82 @@ __device__ __forceinline__ uint32_t push_pair_u8(int e0, int e1, uint32_t c) {
   return d;
 }
 
-// Sum over the TPR threads of a group, for kRows values at once.
-template <int TPR, int kRows, typename V>
-__device__ __forceinline__ void group_reduce(V (&v)[kRows], V* red, int group_first_warp) {
+// Sum over the TPR threads of a group, for kRows values at once.  Inside a warp: xor shuffles (two rows travel as one
+// packed pair per add; integers take the warp-wide reduction instruction).  Across the warps of a group: lane 0 of
+// every warp leaves its partial sums in shared memory, and after the barrier the first TPR / 32 lanes of every warp pick
+// up one warp's partials each and finish with log2(TPR / 32) more shuffle steps (instead of every thread adding up all
+// partials itself).
+template <int TPR, int kRows>
+__device__ __forceinline__ void group_reduce(float (&v)[kRows], float* red, int group_first_warp) {
   constexpr int kShfl = TPR < 32 ? TPR : 32;
+  if constexpr (kRows == 2) {
+    f32x2 p = pack2(v[0], v[1]);
 #pragma unroll
-  for (int o = kShfl / 2; o > 0; o >>= 1)
+    for (int o = kShfl / 2; o > 0; o >>= 1) {
+      float a, b;
+      unpack2(p, a, b);
+      p = add2(p, pack2(__shfl_xor_sync(0xffffffffu, a, o), __shfl_xor_sync(0xffffffffu, b, o)));
+    }
+    unpack2(p, v[0], v[1]);
+  } else {
 #pragma unroll
-    for (int r = 0; r < kRows; ++r) v[r] += __shfl_xor_sync(0xffffffffu, v[r], o);
+    for (int o = kShfl / 2; o > 0; o >>= 1)
+#pragma unroll
+      for (int r = 0; r < kRows; ++r) v[r] += __shfl_xor_sync(0xffffffffu, v[r], o);
+  }
   if constexpr (TPR > 32) {
-    if ((threadIdx.x & 31) == 0)
+    constexpr int kWarps = TPR / 32;
+    const int lane = threadIdx.x & 31;
+    if (lane == 0)
 #pragma unroll
       for (int r = 0; r < kRows; ++r) red[(threadIdx.x >> 5) * kRows + r] = v[r];
     __syncthreads();
+    // lane l < kWarps takes the partials of warp l of its group; the other lanes repeat them (l mod kWarps), so that
+    // the xor steps below leave the full sum in every lane
+    const float* src = red + (group_first_warp + (lane & (kWarps - 1))) * kRows;
+    if constexpr (kRows == 2) {
+      const float2 t = *reinterpret_cast<const float2*>(src);
+      f32x2 p = pack2(t.x, t.y);
+#pragma unroll
+      for (int o = kWarps / 2; o > 0; o >>= 1) {
+        float a, b;
+        unpack2(p, a, b);
+        p = add2(p, pack2(__shfl_xor_sync(0xffffffffu, a, o), __shfl_xor_sync(0xffffffffu, b, o)));
+      }
+      unpack2(p, v[0], v[1]);
+    } else {
+#pragma unroll
+      for (int r = 0; r < kRows; ++r) v[r] = src[r];
+#pragma unroll
+      for (int o = kWarps / 2; o > 0; o >>= 1)
+#pragma unroll
+        for (int r = 0; r < kRows; ++r) v[r] += __shfl_xor_sync(0xffffffffu, v[r], o);
+    }
+  }
+}
+template <int TPR, int kRows>
+__device__ __forceinline__ void group_reduce(int (&v)[kRows], int* red, int group_first_warp) {
+  if constexpr (TPR >= 32) {
+#pragma unroll
+    for (int r = 0; r < kRows; ++r) v[r] = __reduce_add_sync(0xffffffffu, v[r]);
+  } else {
+#pragma unroll
+    for (int o = TPR / 2; o > 0; o >>= 1)
+#pragma unroll
+      for (int r = 0; r < kRows; ++r) v[r] += __shfl_xor_sync(0xffffffffu, v[r], o);
+  }
+  if constexpr (TPR > 32) {
+    constexpr int kWarps = TPR / 32;
+    const int lane = threadIdx.x & 31;
+    if (lane == 0)
+#pragma unroll
+      for (int r = 0; r < kRows; ++r) red[(threadIdx.x >> 5) * kRows + r] = v[r];
+    __syncthreads();
+    const int* src = red + (group_first_warp + (lane & (kWarps - 1))) * kRows;
 #pragma unroll
     for (int r = 0; r < kRows; ++r) {
-      V acc = V(0);
-#pragma unroll
-      for (int w = 0; w < TPR / 32; ++w) acc += red[(group_first_warp + w) * kRows + r];
-      v[r] = acc;
+      // every group of kWarps consecutive lanes holds all partials: the warp-wide sum counts each 32 / kWarps times
+      v[r] = __reduce_add_sync(0xffffffffu, src[r]) / (32 / kWarps);
     }
   }
 }
@@ -107,9 +164,9 @@ ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
   // next reduction is that barrier; the mean-free form without row sums has the variance reduction alone (one
   // barrier per iteration), so red_b alternates between two halves by iteration parity: the write of iteration
   // k + 2 follows the barrier of iteration k + 1, which every thread reaches after its reads of iteration k.
-  __shared__ float red_a[kBlock / 32 * kRows];
-  __shared__ float red_b[2][kBlock / 32 * kRows];
-  __shared__ int red_c[kBlock / 32 * kRows];
+  __shared__ __align__(8) float red_a[kBlock / 32 * kRows];
+  __shared__ __align__(8) float red_b[2][kBlock / 32 * kRows];
+  __shared__ __align__(8) int red_c[kBlock / 32 * kRows];
 
   float* s_g = s_gb;
   float* s_b = s_gb + D;
@@ -184,7 +241,7 @@ ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
 
     float mu[kRows];
     if (!rms) {
-      group_reduce<TPR, kRows, float>(sum, red_a, group_first_warp);
+      group_reduce<TPR, kRows>(sum, red_a, group_first_warp);
 #pragma unroll
       for (int r = 0; r < kRows; ++r) mu[r] = sum[r] * inv_d;
     } else {
@@ -211,7 +268,7 @@ ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
       unpack2(acc, lo, hi);
       ss[r] = lo + hi;
     }
-    group_reduce<TPR, kRows, float>(ss, red_b[parity], group_first_warp);
+    group_reduce<TPR, kRows>(ss, red_b[parity], group_first_warp);
     f32x2 rstd[kRows];
 #pragma unroll
     for (int r = 0; r < kRows; ++r) rstd[r] = splat2(rsqrtf(ss[r] * inv_d + eps));
@@ -278,7 +335,7 @@ ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
       }
     }
     if (row_sum != nullptr) {
-      group_reduce<TPR, kRows, int>(csum, red_c, group_first_warp);
+      group_reduce<TPR, kRows>(csum, red_c, group_first_warp);
       if (tig == 0) {
 #pragma unroll
         for (int r = 0; r < kRows; ++r)
