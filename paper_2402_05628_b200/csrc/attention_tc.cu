@@ -230,6 +230,20 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
   grid_dependency_wait();
   grid_dependency_trigger();
 
+  // The first K tiles are asked for before the Q tile is staged (their barriers must be visible first), so that the
+  // copies' latency and the Q loads' run side by side.
+  int k_issued = 0;
+  if (kCentered) {
+    __syncthreads();
+    if (warp == kWorkWarps + 1 && lane == 0) {
+      for (; k_issued < kK && k_issued < 2 * nb; ++k_issued) {
+        const uint32_t bar = smem_u32(&S.k_full[k_issued]);
+        mbar_expect_tx(bar, kKBytes);
+        tma_load_3d(smem_u32(S.k[k_issued]), &map_k, bar, bi * int(P.k_si), (k_issued < nb ? k_issued : k_issued - nb) * kKeys, bo);
+      }
+    }
+  }
+
   // ---- K rows (quantizers wider than 7 bits): a group stages the K tiles of its own visits, 8 threads per key with one
   // 16-byte piece each, two keys per thread; Q rows: 4 threads per row, 2 pieces each
   const uint8_t* k_base = P.k + bo * P.k_so + bi * P.k_si;
@@ -387,8 +401,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_k, AttnParams P) {
   } else if (warp == kWorkWarps + 1) {
     // ---------------------------------------------------------------- K tiles by bulk tensor copies
     if (kCentered && lane == 0) {
-      int issued = 0;
-      for (int g = 0; g < 2 * nb && !*abort; ++g) {
+      int issued = k_issued;
+      for (int g = k_issued; g < 2 * nb && !*abort; ++g) {
         const int b = ring(g, kK);
         if (!mbar_wait(smem_u32(&S.k_empty[b]), lap(g, kK) ^ 1u, abort, 48, P.status)) break;
         const uint32_t bar = smem_u32(&S.k_full[b]);
