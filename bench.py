@@ -39,21 +39,22 @@ HEADLINE = "c4_llama7b"
 OTHER_WORKLOADS = ("c1_vit_s", "c2_deit_b", "c2_deit_b_w6a6", "c3_vit_l", "c4_llama7b_arch")
 INT8_OVER_BF16 = 2.0          # nominal dense int8 : bf16 tensor throughput on B200
 L2_BYTES = 126 << 20
-# Own model of the fused attention kernel's arithmetic, kept as a side figure: about 8 thread instructions per score
-# in the statistics pass (int -> float, scale, max, subtract, ex2, add) and 15 in the code pass.
+# Own model of the fused attention kernel's arithmetic, kept as a side figure from the first version of the kernel: about
+# 8 thread instructions per score in the statistics pass (int -> float, scale, max, subtract, ex2, add) and 15 in the code
+# pass.  (The present kernel needs about half of that and is not bound by it.)
 ATTENTION_INSTR_PER_SCORE = 23
 
 # DRAM traffic of one launch of a stage kernel, from one ncu capture of the same bench command (summaries under
 # profiles/).  A figure is reported only while the kernel's sources still hash to what was captured.
 NCU_TRAFFIC = {   # (workload, batch, stage): (DRAM bytes read + written per launch, kernel sources, their sha1 when captured)
-    ("c4_llama7b", 4, "attention"): (140183808, ["attention_tc.cu", "tc_ptx.cuh"], "25f127db9567"),
-    ("c4_llama7b", 4, "qkv"): (188480000, ["qgemm_tc.cu", "tc_ptx.cuh", "epilogue.cuh"], "56d623be4aa8"),
-    ("c4_llama7b", 4, "proj"): (209939712, ["qgemm_tc.cu", "tc_ptx.cuh", "epilogue.cuh"], "56d623be4aa8"),
-    ("c4_llama7b", 4, "fc1"): (170638080, ["qgemm_tc.cu", "tc_ptx.cuh", "epilogue.cuh"], "56d623be4aa8"),
-    ("c4_llama7b", 4, "fc2"): (569528064, ["qgemm_tc.cu", "tc_ptx.cuh", "epilogue.cuh"], "56d623be4aa8"),
-    ("c4_llama7b", 4, "ln1"): (71457792, ["ln_quant.cu", "f32x2.cuh"], "8927f8809457"),
-    ("c4_llama7b", 4, "ln2"): (71122432, ["ln_quant.cu", "f32x2.cuh"], "8927f8809457"),
-    ("c2_deit_b", 64, "attention"): (29162496, ["attention_tc.cu", "tc_ptx.cuh"], "25f127db9567"),
+    ("c4_llama7b", 4, "attention"): (138199296, ["attention_tc.cu", "tc_ptx.cuh"], "47dd87935b26"),
+    ("c4_llama7b", 4, "qkv"): (191884544, ["qgemm_tc.cu", "tc_ptx.cuh", "epilogue.cuh"], "35028e88a4f9"),
+    ("c4_llama7b", 4, "proj"): (214569984, ["qgemm_tc.cu", "tc_ptx.cuh", "epilogue.cuh"], "35028e88a4f9"),
+    ("c4_llama7b", 4, "fc1"): (175095040, ["qgemm_tc.cu", "tc_ptx.cuh", "epilogue.cuh"], "35028e88a4f9"),
+    ("c4_llama7b", 4, "fc2"): (572544256, ["qgemm_tc.cu", "tc_ptx.cuh", "epilogue.cuh"], "35028e88a4f9"),
+    ("c4_llama7b", 4, "ln1"): (72495360, ["ln_quant.cu", "f32x2.cuh"], "c6afda1fcbd9"),
+    ("c4_llama7b", 4, "ln2"): (71312128, ["ln_quant.cu", "f32x2.cuh"], "c6afda1fcbd9"),
+    ("c2_deit_b", 64, "attention"): (29160192, ["attention_tc.cu", "tc_ptx.cuh"], "47dd87935b26"),
 }
 
 
@@ -505,7 +506,8 @@ def main():
                     help="run only the single-kernel sweep points of this kernel and print them (profiling aid)")
     ap.add_argument("--sweep-dim", type=int, default=None, help="with --sweep-only: only this D (ln), L (softmax) or N (gemm)")
     ap.add_argument("--weights", default="bytes", choices=["packed", "bytes"],
-                    help="4-bit weight codes in device memory: two per byte (expanded in shared memory by the GEMM) or one per byte")
+                    help="weight codes in device memory: packed (4-bit two per byte, 6-bit four to three bytes; expanded in shared memory "
+                         "by the GEMM) or one per byte")
     ap.add_argument("--staged-attention", action="store_true",
                     help="run scores, Softmax codes and P.V as three kernels instead of the fused attention kernel")
     args = ap.parse_args()
