@@ -16,7 +16,8 @@ def _built():
 @pytest.mark.parametrize("rows,D,bits,bf16", [
     (197, 384, 4, False), (1000, 768, 4, True), (515, 768, 6, True), (333, 1024, 4, True),
     (130, 4096, 4, True), (67, 8192, 8, True), (9, 16384, 4, False), (1, 8, 4, False), (77, 200, 8, True),
-    (4099, 768, 4, False),
+    (4099, 768, 4, False), (5003, 1024, 4 | parity.BYTE_CODES, True), (2500, 2048, 6, True), (3001, 4096, 8, True),
+    (1201, 8192, 4, True), (333, 1024, 4, False),
 ])
 def test_ln_quant_matches_channelwise_oracle(rows, D, bits, bf16):
     rep = parity.check_ln_quant(rows, D, bits, bf16, seed=rows + D)
@@ -24,7 +25,7 @@ def test_ln_quant_matches_channelwise_oracle(rows, D, bits, bf16):
     assert rep["mismatch"] <= max(2, 2e-4 * rep["total"]), rep
 
 
-@pytest.mark.parametrize("D", [4096, 8192, 768])
+@pytest.mark.parametrize("D", [4096, 8192, 768, 1024, 2048])
 def test_ln_quant_mean_free_without_row_sums_repeated(D):
     """Mean-free normalisation without row sums runs one reduction per row (one barrier per iteration of a thread
     group wider than a warp): repeated launches over many rows per block agree with the oracle and one another."""
