@@ -73,6 +73,14 @@ __device__ __forceinline__ uint32_t push_pair_u8(int e0, int e1, uint32_t c) {
 // every warp leaves its partial sums in shared memory, and after the barrier the first TPR / 32 lanes of every warp pick
 // up one warp's partials each and finish with log2(TPR / 32) more shuffle steps (instead of every thread adding up all
 // partials itself).
+// Barrier of one thread group: the whole block where a group is the block, else a named barrier of the group's own (the
+// groups of a block then no longer wait for one another).
+template <int TPR>
+__device__ __forceinline__ void group_sync(int group_first_warp) {
+  if constexpr (TPR >= 256) __syncthreads();
+  else asm volatile("bar.sync %0, %1;" ::"r"(1 + group_first_warp / (TPR / 32)), "n"(TPR) : "memory");
+}
+
 template <int TPR, int kRows>
 __device__ __forceinline__ void group_reduce(float (&v)[kRows], float* red, int group_first_warp) {
   constexpr int kShfl = TPR < 32 ? TPR : 32;
@@ -97,7 +105,7 @@ __device__ __forceinline__ void group_reduce(float (&v)[kRows], float* red, int 
     if (lane == 0)
 #pragma unroll
       for (int r = 0; r < kRows; ++r) red[(threadIdx.x >> 5) * kRows + r] = v[r];
-    __syncthreads();
+    group_sync<TPR>(group_first_warp);
     // lane l < kWarps takes the partials of warp l of its group; the other lanes repeat them (l mod kWarps), so that
     // the xor steps below leave the full sum in every lane
     const float* src = red + (group_first_warp + (lane & (kWarps - 1))) * kRows;
@@ -138,7 +146,7 @@ __device__ __forceinline__ void group_reduce(int (&v)[kRows], int* red, int grou
     if (lane == 0)
 #pragma unroll
       for (int r = 0; r < kRows; ++r) red[(threadIdx.x >> 5) * kRows + r] = v[r];
-    __syncthreads();
+    group_sync<TPR>(group_first_warp);
     const int* src = red + (group_first_warp + (lane & (kWarps - 1))) * kRows;
 #pragma unroll
     for (int r = 0; r < kRows; ++r) {
