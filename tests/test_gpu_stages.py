@@ -136,6 +136,11 @@ def test_scores_from_byte_codes_match_oracle(Bn, H, Lq, Lk, dh, bits, causal):
     (2, 2, 64, 64, 32, 6, 6, False), (1, 1, 1, 130, 16, 8, 8, False), (1, 2, 100, 260, 48, 4, 4, True),
     (1, 1, 70, 70, 96, 8, 4, True), (1, 2, 700, 700, 64, 4, 4, True), (1, 2, 150, 150, 128, 6, 6, False),
     (1, 2, 300, 300, 64, 4, 6, True),
+    # wide heads (visits of 128 keys, two issuing warps): one visit, a visit with a single key, odd and even numbers of
+    # visits, every score form and code width, head sizes that do not fill the tile, keys beyond the queries under a mask
+    (1, 2, 128, 128, 128, 4, 8, False), (1, 1, 129, 129, 128, 4, 4, True), (1, 2, 260, 1000, 128, 4, 8, True),
+    (1, 1, 200, 700, 128, 8, 8, False), (1, 2, 140, 385, 80, 4, 6, False), (1, 1, 257, 640, 112, 6, 8, True),
+    (2, 1, 33, 1030, 96, 4, 4, True),
 ])
 def test_fused_attention_matches_oracle(Bn, H, Lq, Lk, dh, bits, bp, causal):
     parity.check_attention(Bn, H, Lq, Lk, dh, bits, bp, causal, seed=Lq + dh)
