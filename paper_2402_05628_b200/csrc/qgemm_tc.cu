@@ -183,9 +183,12 @@ struct ChunkQuant {
 __device__ __forceinline__ ChunkQuant chunk_quant(const EpilogueParams& ep, const TcParams& P, int col0) {
   const int gw = ep.group_width;
   const int group = (col0 >= gw) + (col0 >= 2 * gw) + (col0 >= 3 * gw);
-  const int zo = ep.out_zero[group];
+  // (selects, not run-time indexing: an indexed kernel parameter makes every thread keep a copy of the parameters in
+  // local memory)
+  const int zo = group == 0 ? ep.out_zero[0] : group == 1 ? ep.out_zero[1] : group == 2 ? ep.out_zero[2] : ep.out_zero[3];
+  const float inv = group == 0 ? ep.inv_out_scale[0] : group == 1 ? ep.inv_out_scale[1] : group == 2 ? ep.inv_out_scale[2] : ep.inv_out_scale[3];
   ChunkQuant q;
-  q.mult = P.direct_requant ? 1.f : ep.inv_out_scale[group];
+  q.mult = P.direct_requant ? 1.f : inv;
   q.lo = float(-zo);
   q.hi = float(ep.qmax - zo);
   q.pack_k = (kMagicBits - uint32_t(zo)) * 0x11111111u;
@@ -401,7 +404,7 @@ enum : int { kPairNone = 0, kPairRope = 1, kPairGlu = 2 };
 template <int BN, int OUT, bool RES, int PAIR, int WP>
 __global__ void __launch_bounds__(kThreads, 1)
 qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_res, TcParams P) {
+                const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_res, const __grid_constant__ TcParams P) {
   using Storage = SharedStorage<BN, RES, WP>;
   constexpr bool W4 = WP != 0;                           // weights arrive packed
   constexpr int kStages = Storage::kStages;
@@ -646,11 +649,18 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       const bool any_row = m0 + quarter * 32 < P.M;          // warp-uniform: at least one valid row
       const bool fast = fast_ok && slice_on && n0 + cl0 + kSliceCols <= P.N && any_row;
       // bf16 residual of the slice: requested now, needed only after the main loop of the tile
-      uint4 res[kSliceCols / 8];
-      if (!RES && fast && res16 && row_ok) {
-        const uint4* rp = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(ep.residual) + m * ep.ld_residual + n0 + cl0);
+      // (the pieces of two chunks at a time: those of the first two chunks here, those of the next two while the first two
+      // are worked on; every index into the register arrays is a compile-time one)
+      constexpr int kPairPieces = 2 * (kChunk / 8);
+      uint4 res[kPairPieces], res_next[kPairPieces];
+      // (float outputs: that is where a residual stream is added; a code output with a residual loads the pieces where
+      // they are used)
+      constexpr bool kResRegs = !RES && (OUT == kOutF32 || OUT == kOutBf16);
+      const bool res_regs = kResRegs && fast && res16 && row_ok;
+      const uint4* res_ptr = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(ep.residual) + m * ep.ld_residual + n0 + cl0);
+      if (res_regs) {
 #pragma unroll
-        for (int i = 0; i < kSliceCols / 8; ++i) res[i] = __ldg(rp + i);
+        for (int i = 0; i < kPairPieces; ++i) res[i] = __ldg(res_ptr + i);
       }
       // corr = acc - z_w (asum - K z_a) - z_a wsum; this tile's inputs were fetched during the previous tile
       const int32_t asum_c = row_ok ? nx_asum - kza : 0;
@@ -664,7 +674,8 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
           float sc = in ? ep.scale_a * (ep.s_w ? nx_sw[h] : ep.s_w_scalar) : 0.f, bi = in && ep.bias ? nx_bs[h] : 0.f;
           if (direct) {
             const int gw = ep.group_width;
-            const float inv = ep.inv_out_scale[(j >= gw) + (j >= 2 * gw) + (j >= 3 * gw)];
+            const int gi = (j >= gw) + (j >= 2 * gw) + (j >= 3 * gw);
+            const float inv = gi == 0 ? ep.inv_out_scale[0] : gi == 1 ? ep.inv_out_scale[1] : gi == 2 ? ep.inv_out_scale[2] : ep.inv_out_scale[3];
             sc *= inv;
             bi *= inv;
           }
@@ -693,8 +704,17 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         res_pending = false;
       }
       if (fast) {
+        // (two chunks per trip: unrolled further, the 16 values of four chunks in flight spill at 96 registers)
+        static_assert(kSliceChunks % 2 == 0, "the chunk loop takes two chunks per trip");
+#pragma unroll 1
+        for (int cp = 0; cp < kSliceChunks; cp += 2) {
+          if (res_regs && cp + 2 < kSliceChunks) {
 #pragma unroll
-        for (int c = 0; c < kSliceChunks; ++c) {
+            for (int i = 0; i < kPairPieces; ++i) res_next[i] = __ldg(res_ptr + (cp + 2) * (kChunk / 8) + i);
+          }
+#pragma unroll
+        for (int cu = 0; cu < 2; ++cu) {
+          const int c = cp + cu;
           const int cl = cl0 + c * kChunk;                     // column inside the tile
           const int col0 = n0 + cl;
           uint32_t r[kChunk];
@@ -735,7 +755,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w4.x), "=r"(w4.y), "=r"(w4.z), "=r"(w4.w)
                              : "r"(res_buf + uint32_t(lane) * 128u + ((piece ^ uint32_t(lane & 7)) << 4)));
               } else {
-                w4 = res[c * (kChunk / 8) + i];
+                w4 = kResRegs ? res[cu * (kChunk / 8) + i] : __ldg(res_ptr + c * (kChunk / 8) + i);
               }
               const uint32_t ws[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
@@ -782,6 +802,9 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             }
           }
           emit_chunk<OUT>(&map_out, smem_u32(S.epi[ew]), lane, q, v, c, col0, m0 + quarter * 32, code_sum, direct, sat);
+        }
+#pragma unroll
+          for (int i = 0; i < kPairPieces; ++i) res[i] = res_next[i];
         }
       } else if (slice_on && any_row && n0 + cl0 < P.N) {
 #pragma unroll 1
