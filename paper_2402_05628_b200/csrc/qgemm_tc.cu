@@ -649,10 +649,11 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       const bool any_row = m0 + quarter * 32 < P.M;          // warp-uniform: at least one valid row
       const bool fast = fast_ok && slice_on && n0 + cl0 + kSliceCols <= P.N && any_row;
       // bf16 residual of the slice: requested now, needed only after the main loop of the tile
-      // (the pieces of two chunks at a time: those of the first two chunks here, those of the next two while the first two
-      // are worked on; every index into the register arrays is a compile-time one)
+      // (the pieces of two chunks at a time, in one set of registers: those of the first two chunks are requested here,
+      // those of the next two as soon as the first two have been added, a chunk's store and the next chunk's accumulator
+      // load ahead of their use; every index into the register array is a compile-time one)
       constexpr int kPairPieces = 2 * (kChunk / 8);
-      uint4 res[kPairPieces], res_next[kPairPieces];
+      uint4 res[kPairPieces];
       // (float outputs: that is where a residual stream is added; a code output with a residual loads the pieces where
       // they are used)
       constexpr bool kResRegs = !RES && (OUT == kOutF32 || OUT == kOutBf16);
@@ -708,10 +709,6 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         static_assert(kSliceChunks % 2 == 0, "the chunk loop takes two chunks per trip");
 #pragma unroll 1
         for (int cp = 0; cp < kSliceChunks; cp += 2) {
-          if (res_regs && cp + 2 < kSliceChunks) {
-#pragma unroll
-            for (int i = 0; i < kPairPieces; ++i) res_next[i] = __ldg(res_ptr + (cp + 2) * (kChunk / 8) + i);
-          }
 #pragma unroll
         for (int cu = 0; cu < 2; ++cu) {
           const int c = cp + cu;
@@ -764,6 +761,10 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                         v[i * 8 + 2 * k], v[i * 8 + 2 * k + 1]);
             }
           }
+          if (cu == 1 && res_regs && cp + 2 < kSliceChunks) {      // both chunks of the pair have taken their pieces
+#pragma unroll
+            for (int i = 0; i < kPairPieces; ++i) res[i] = __ldg(res_ptr + (cp + 2) * (kChunk / 8) + i);
+          }
           if (PAIR == kPairRope && rope_row != nullptr && col0 < ep.rope_cols) {       // warp-uniform: range edges fall on chunk edges
             int hx = rope_hb + c * kChunk;
             while (hx >= ep.rope_dim) hx -= ep.rope_dim;
@@ -803,8 +804,6 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
           }
           emit_chunk<OUT>(&map_out, smem_u32(S.epi[ew]), lane, q, v, c, col0, m0 + quarter * 32, code_sum, direct, sat);
         }
-#pragma unroll
-          for (int i = 0; i < kPairPieces; ++i) res[i] = res_next[i];
         }
       } else if (slice_on && any_row && n0 + cl0 < P.N) {
 #pragma unroll 1
