@@ -52,8 +52,8 @@ NCU_TRAFFIC = {   # (workload, batch, stage): (DRAM bytes read + written per lau
     ("c4_llama7b", 4, "proj"): (198638080, ["qgemm_tc.cu", "tc_ptx.cuh", "epilogue.cuh"], "b27c09ffa1f7"),
     ("c4_llama7b", 4, "fc1"): (150345216, ["qgemm_tc.cu", "tc_ptx.cuh", "epilogue.cuh"], "b27c09ffa1f7"),
     ("c4_llama7b", 4, "fc2"): (607551232, ["qgemm_tc.cu", "tc_ptx.cuh", "epilogue.cuh"], "b27c09ffa1f7"),
-    ("c4_llama7b", 4, "ln1"): (71301120, ["ln_quant.cu", "f32x2.cuh"], "baca6d8b8047"),
-    ("c4_llama7b", 4, "ln2"): (71044096, ["ln_quant.cu", "f32x2.cuh"], "baca6d8b8047"),
+    ("c4_llama7b", 4, "ln1"): (71826432, ["ln_quant.cu", "f32x2.cuh"], "1eacf83c9513"),
+    ("c4_llama7b", 4, "ln2"): (71635712, ["ln_quant.cu", "f32x2.cuh"], "1eacf83c9513"),
     ("c2_deit_b", 64, "attention"): (29160192, ["attention_tc.cu", "tc_ptx.cuh"], "47dd87935b26"),
 }
 

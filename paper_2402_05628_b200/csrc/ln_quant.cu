@@ -6,7 +6,9 @@
 // and centred variance are two register passes with shuffle reductions.  Each group works on one or two rows
 // at a time, and the rows of its next iteration are requested before the current ones are reduced, so that
 // loads stay in flight all the time.
-// The per-channel factors gamma~/s~ and beta~/s~ are staged once per CTA in shared memory.
+// The per-channel factors gamma~/s~ and beta~/s~ are staged once per CTA in shared memory (halves of the 8-element
+// chunks apart, so that a warp's 16-byte reads are free of bank conflicts), or, for rows of 3080 to 4096 bf16 elements,
+// kept in the registers of the thread that owns their columns.
 //
 // The float work runs on packed pairs (two elements per add / mul / fma issue slot).  Rounding is done by the
 // float adder: t + 1.5 * 2^23 leaves rint(t) (half to even, on t itself, as Eq. 4 has it) in the low mantissa
@@ -27,6 +29,14 @@ constexpr int kMaxVPT = 4;  // chunks per thread: 1..4, chosen per row length
 // except where four chunks per thread would cost a resident block (measured: 16 x 3 / 32 x 3 / 256 x 4 threads x
 // chunks run best with two rows, 32 x 4 / 128 x 4 with one).
 __host__ __device__ constexpr int rows_in_flight(int vpt, int tpr) { return vpt >= 4 && tpr < 256 ? 1 : 2; }
+
+// Where a thread's slice of gamma~/s~ and beta~/s~ stays in registers for the whole kernel instead of being read from
+// shared memory for every pair of rows: two chunks per thread at most (32 registers) in groups of at least 128 threads,
+// bf16 input (two resident blocks of 256 threads at 108 registers; measured at D = 4096: 670 -> 595 us for 262144 rows,
+// three blocks with spills or one row at a time were slower).
+__host__ __device__ constexpr bool factors_in_registers(int vpt, int tpr, int elem_bytes) {
+  return vpt <= 2 && tpr >= 128 && elem_bytes == 2;
+}
 
 // A chunk of 8 elements as it is loaded (kept in this form while the rows before it are processed), and
 // its expansion into 4 packed float pairs.
@@ -84,7 +94,22 @@ __device__ __forceinline__ void group_sync(int group_first_warp) {
 template <int TPR, int kRows>
 __device__ __forceinline__ void group_reduce(float (&v)[kRows], float* red, int group_first_warp) {
   constexpr int kShfl = TPR < 32 ? TPR : 32;
-  if constexpr (kRows == 2) {
+  const bool odd = threadIdx.x & 1;
+  if constexpr (kRows == 2 && kShfl >= 4) {
+    // neighbouring lanes split the two rows between them (one shuffle for both rows), every further step then moves one
+    // value per lane, and a last exchange hands each lane the other row's total: kShfl's log + 1 shuffles instead of
+    // twice the log.  All lanes of a parity add the same pairs at every step, so they end with the same bits.
+    float t = (odd ? v[1] : v[0]) + __shfl_xor_sync(0xffffffffu, odd ? v[0] : v[1], 1);
+#pragma unroll
+    for (int o = kShfl / 2; o > 1; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+    if constexpr (TPR <= 32) {
+      const float u = __shfl_xor_sync(0xffffffffu, t, 1);
+      v[0] = odd ? u : t;
+      v[1] = odd ? t : u;
+    } else {
+      v[0] = t;      // even lanes: row 0, odd lanes: row 1 (lanes 0 and 1 leave them in shared memory)
+    }
+  } else if constexpr (kRows == 2) {
     f32x2 p = pack2(v[0], v[1]);
 #pragma unroll
     for (int o = kShfl / 2; o > 0; o >>= 1) {
@@ -102,24 +127,25 @@ __device__ __forceinline__ void group_reduce(float (&v)[kRows], float* red, int 
   if constexpr (TPR > 32) {
     constexpr int kWarps = TPR / 32;
     const int lane = threadIdx.x & 31;
-    if (lane == 0)
-#pragma unroll
-      for (int r = 0; r < kRows; ++r) red[(threadIdx.x >> 5) * kRows + r] = v[r];
-    group_sync<TPR>(group_first_warp);
-    // lane l < kWarps takes the partials of warp l of its group; the other lanes repeat them (l mod kWarps), so that
-    // the xor steps below leave the full sum in every lane
-    const float* src = red + (group_first_warp + (lane & (kWarps - 1))) * kRows;
     if constexpr (kRows == 2) {
-      const float2 t = *reinterpret_cast<const float2*>(src);
-      f32x2 p = pack2(t.x, t.y);
+      // lanes 0 and 1 hold the warp's sums of rows 0 and 1.  After the barrier lane l takes row (l mod 2) of warp
+      // (l / 2 mod kWarps): xor steps over the warp index, then one exchange between neighbours.
+      if (lane < 2) red[(threadIdx.x >> 5) * 2 + lane] = v[0];
+      group_sync<TPR>(group_first_warp);
+      float t = red[(group_first_warp + ((lane >> 1) & (kWarps - 1))) * 2 + (lane & 1)];
 #pragma unroll
-      for (int o = kWarps / 2; o > 0; o >>= 1) {
-        float a, b;
-        unpack2(p, a, b);
-        p = add2(p, pack2(__shfl_xor_sync(0xffffffffu, a, o), __shfl_xor_sync(0xffffffffu, b, o)));
-      }
-      unpack2(p, v[0], v[1]);
+      for (int o = kWarps; o > 1; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+      const float u = __shfl_xor_sync(0xffffffffu, t, 1);
+      v[0] = odd ? u : t;
+      v[1] = odd ? t : u;
     } else {
+      if (lane == 0)
+#pragma unroll
+        for (int r = 0; r < kRows; ++r) red[(threadIdx.x >> 5) * kRows + r] = v[r];
+      group_sync<TPR>(group_first_warp);
+      // lane l < kWarps takes the partials of warp l of its group; the other lanes repeat them (l mod kWarps), so that
+      // the xor steps below leave the full sum in every lane
+      const float* src = red + (group_first_warp + (lane & (kWarps - 1))) * kRows;
 #pragma unroll
       for (int r = 0; r < kRows; ++r) v[r] = src[r];
 #pragma unroll
@@ -157,7 +183,8 @@ __device__ __forceinline__ void group_reduce(int (&v)[kRows], int* red, int grou
 }
 
 template <typename T, int TPR, int kVPT, bool kPack4, bool kFull>
-__global__ void __launch_bounds__((TPR > 256 ? TPR : 256), (kVPT <= 2 && TPR == 256 ? 3 : 0))
+__global__ void __launch_bounds__((TPR > 256 ? TPR : 256),
+                                  (kVPT <= 2 && TPR == 256 ? (factors_in_registers(kVPT, TPR, sizeof(T)) ? 2 : 3) : 0))
 ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
                 const float* __restrict__ gamma_t, const float* __restrict__ beta_t, float eps, int rms,
                 float inv_s, int z, int qmax, uint8_t* __restrict__ codes, int64_t ldc,
@@ -166,7 +193,8 @@ ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
   constexpr int kBlock = TPR > 256 ? TPR : 256;
   constexpr int kGroups = kBlock / TPR;
   constexpr int kRowsPerBlock = kGroups * kRows;
-  extern __shared__ __align__(16) float s_gb[];          // g[D] then b[D]: gamma~/s~ and beta~/s~
+  constexpr bool kRegFactors = factors_in_registers(kVPT, TPR, sizeof(T));
+  extern __shared__ __align__(16) float s_gb[];          // g[D] then b[D]: gamma~/s~ and beta~/s~ (unless in registers)
   // One array per reduction of a row.  A slot may be overwritten only after every thread of the block has passed
   // a barrier that follows its reads of the slot.  With two or three reductions per iteration the barrier of the
   // next reduction is that barrier; the mean-free form without row sums has the variance reduction alone (one
@@ -183,11 +211,39 @@ ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
   // is clamped and converted, so that adding z cannot wrap (a whole-kernel decision, taken here once).
   const float root_d = sqrtf(float(D));
   bool wide = false;
-  for (int i = threadIdx.x; i < D; i += kBlock) {
-    const float gi = __ldg(gamma_t + i) * inv_s, bi = __ldg(beta_t + i) * inv_s;
-    s_g[i] = gi;
-    s_b[i] = bi;
-    wide = wide || !(fabsf(gi) * root_d + fabsf(bi) < 4.0e6f);
+  f32x2 g_reg[kRegFactors ? kVPT : 1][kChunk / 2], b_reg[kRegFactors ? kVPT : 1][kChunk / 2];
+  if constexpr (kRegFactors) {
+    // every thread works on the same columns of every row: its factors are loaded once
+#pragma unroll
+    for (int i = 0; i < kVPT; ++i) {
+      const int c = threadIdx.x % TPR + i * TPR;
+      const bool on = kFull || c < D / kChunk;
+      float gi[kChunk], bi[kChunk];
+#pragma unroll
+      for (int e = 0; e < kChunk; ++e) {
+        gi[e] = on ? __ldg(gamma_t + c * kChunk + e) * inv_s : 0.f;
+        bi[e] = on ? __ldg(beta_t + c * kChunk + e) * inv_s : 0.f;
+      }
+#pragma unroll
+      for (int e = 0; e < kChunk; ++e) wide = wide || !(fabsf(gi[e]) * root_d + fabsf(bi[e]) < 4.0e6f);
+#pragma unroll
+      for (int e = 0; e < kChunk / 2; ++e) {
+        g_reg[i][e] = pack2(gi[2 * e], gi[2 * e + 1]);
+        b_reg[i][e] = pack2(bi[2 * e], bi[2 * e + 1]);
+      }
+    }
+  } else {
+    // layout: the first halves (4 floats) of all chunks, then the second halves, so that the 16-byte reads of
+    // neighbouring lanes are neighbours in shared memory (chunk by chunk they would sit 32 bytes apart: two-way
+    // bank conflicts)
+    const int half_stride = D / 2;
+    for (int i = threadIdx.x; i < D; i += kBlock) {
+      const float gi = __ldg(gamma_t + i) * inv_s, bi = __ldg(beta_t + i) * inv_s;
+      const int at = ((i >> 2) & 1) * half_stride + (i >> 3) * 4 + (i & 3);
+      s_g[at] = gi;
+      s_b[at] = bi;
+      wide = wide || !(fabsf(gi) * root_d + fabsf(bi) < 4.0e6f);
+    }
   }
   const bool guard = __syncthreads_or(wide) != 0;
   // gamma~ and beta~ are parameters; x and the outputs belong to the chain of kernels
@@ -295,11 +351,14 @@ ln_quant_kernel(const T* __restrict__ x, int64_t rows, int D, int64_t ldx,
       const int c = tig + i * TPR;
       if (kFull || c < nchunks) {
         f32x2 g[kChunk / 2], b[kChunk / 2];
-        {
-          const float4 g0 = *reinterpret_cast<const float4*>(s_g + c * kChunk);
-          const float4 g1 = *reinterpret_cast<const float4*>(s_g + c * kChunk + 4);
-          const float4 b0 = *reinterpret_cast<const float4*>(s_b + c * kChunk);
-          const float4 b1 = *reinterpret_cast<const float4*>(s_b + c * kChunk + 4);
+        if constexpr (kRegFactors) {
+#pragma unroll
+          for (int e = 0; e < kChunk / 2; ++e) { g[e] = g_reg[i][e]; b[e] = b_reg[i][e]; }
+        } else {
+          const float4 g0 = *reinterpret_cast<const float4*>(s_g + c * 4);
+          const float4 g1 = *reinterpret_cast<const float4*>(s_g + D / 2 + c * 4);
+          const float4 b0 = *reinterpret_cast<const float4*>(s_b + c * 4);
+          const float4 b1 = *reinterpret_cast<const float4*>(s_b + D / 2 + c * 4);
           g[0] = pack2(g0.x, g0.y); g[1] = pack2(g0.z, g0.w); g[2] = pack2(g1.x, g1.y); g[3] = pack2(g1.z, g1.w);
           b[0] = pack2(b0.x, b0.y); b[1] = pack2(b0.z, b0.w); b[2] = pack2(b1.x, b1.y); b[3] = pack2(b1.z, b1.w);
         }
@@ -362,7 +421,7 @@ repq_status launch(const T* x, int64_t rows, int D, int64_t ldx, const float* g,
   const int64_t need = (rows + kRowsPerBlock - 1) / kRowsPerBlock;
   const float inv_s = 1.f / s_t;
   const int qmax = code_max(bits);
-  const size_t smem = size_t(D) * 2 * sizeof(float);
+  const size_t smem = factors_in_registers(kVPT, TPR, sizeof(T)) ? 0 : size_t(D) * 2 * sizeof(float);
   const bool full = D == TPR * kVPT * kChunk;   // the row fills the group exactly: no chunk is predicated
   auto kern = packed4(bits) ? (full ? ln_quant_kernel<T, TPR, kVPT, true, true> : ln_quant_kernel<T, TPR, kVPT, true, false>)
                             : (full ? ln_quant_kernel<T, TPR, kVPT, false, true> : ln_quant_kernel<T, TPR, kVPT, false, false>);
