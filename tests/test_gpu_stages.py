@@ -18,6 +18,8 @@ def _built():
     (130, 4096, 4, True), (67, 8192, 8, True), (9, 16384, 4, False), (1, 8, 4, False), (77, 200, 8, True),
     (4099, 768, 4, False), (5003, 1024, 4 | parity.BYTE_CODES, True), (2500, 2048, 6, True), (3001, 4096, 8, True),
     (1201, 8192, 4, True), (333, 1024, 4, False),
+    # rows that do not fill their thread group: factors in registers (3200, 4088), factors in shared memory (1000, 1096)
+    (257, 3200, 4, True), (99, 4088, 8, True), (301, 1000, 4, True), (150, 1096, 6, True),
 ])
 def test_ln_quant_matches_channelwise_oracle(rows, D, bits, bf16):
     rep = parity.check_ln_quant(rows, D, bits, bf16, seed=rows + D)
