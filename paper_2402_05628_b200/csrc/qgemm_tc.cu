@@ -877,7 +877,14 @@ TcLayout tc_layout(const repq_gemm_desc& d) {
 // Tile width: rounds of tiles over the SMs times the time of one round, which has a part that does not depend on the
 // width (per-tile waits, staging and bulk-store latencies of the epilogue warps) and a part proportional to it
 // (measured: about 160 columns' worth of fixed time for K = 768).
-int pick_bn(int M, int N, int sms, bool w_packed4) {
+// Whether a launch takes its bf16 residual through bulk-copied boxes (tiles of at most 192 columns, short K).
+bool residual_boxes(const TcParams& P) {
+  const EpilogueParams& ep = P.ep;
+  return (ep.out_kind == REPQ_OUT_F32 || ep.out_kind == REPQ_OUT_BF16) && ep.residual != nullptr && ep.residual_bf16 &&
+         ep.acc_debug == nullptr && P.K <= 1536 && !P.w_packed4;
+}
+
+int pick_bn(int M, int N, int sms, bool w_packed4, bool res_boxes) {
   const int m_tiles = (M + BM - 1) / BM;
   int best = 256;
   long best_cost = -1;
@@ -885,7 +892,10 @@ int pick_bn(int M, int N, int sms, bool w_packed4) {
     if (w_packed4 && bn > kMaxBNW4) continue;
     const long tiles = long(m_tiles) * ((N + bn - 1) / bn);
     const long rounds = (tiles + sms - 1) / sms;
-    const long cost = rounds * (bn + 160);
+    // a round costs its width plus a fixed part; where the epilogue adds a bf16 residual at short K it sets the pace
+    // alone, and a 256-column tile (residual by row-per-lane loads) takes 1.7 x the time of a narrower one whose
+    // residual box was copied in a tile ahead (measured at 18464 x 1024 x 1024: 39.6 us with 256 columns, 33.9 with 192)
+    const long cost = res_boxes ? rounds * (bn == 256 ? 95 : 55) : rounds * (bn + 160);
     if (best_cost < 0 || cost < best_cost) { best = bn; best_cost = cost; }
   }
   return best;
@@ -956,7 +966,7 @@ repq_status launch_tc_out(const CUtensorMap& map_a, const CUtensorMap& map_b, co
   // Taken for short K, where the epilogue sets the pace (measured at 12608 x 768: K = 768 24 us against 27 us with
   // row-per-lane residual loads; K = 3072 46 us against 39 us, the main loop missing its fourth stage).
   if constexpr (BN <= 192 && (OUT == kOutF32 || OUT == kOutBf16)) {
-    if (P.ep.residual != nullptr && P.ep.residual_bf16 && P.ep.acc_debug == nullptr && P.K <= 1536 && !P.w_packed4)
+    if (residual_boxes(P))
       return launch_tc_res<BN, OUT, true>(map_a, map_b, P, sms, st);
   }
   return launch_tc_res<BN, OUT, false>(map_a, map_b, P, sms, st);
@@ -1057,7 +1067,7 @@ repq_status qgemm_tc(const repq_gemm_desc& d, const EpilogueParams& ep, void* ws
   P.direct_requant = d.out_kind == REPQ_OUT_CODES && !d.gelu && !d.residual && !d.glu;
   REPQ_REQUIRE(device_status_word() != nullptr, REPQ_CUDA_ERROR, "qgemm: device status word unavailable");
   const int sms = sm_count();
-  const int bn = pick_bn(d.M, d.N, sms, P.w_packed4 != 0);
+  const int bn = pick_bn(d.M, d.N, sms, P.w_packed4 != 0, residual_boxes(P));
   {
     // panels of activations of about 40 MB (a third of the L2 capacity), at least 8 row tiles
     const int m_tiles = (d.M + BM - 1) / BM, n_tiles = (d.N + bn - 1) / bn;
