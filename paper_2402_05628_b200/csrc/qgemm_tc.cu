@@ -1069,9 +1069,12 @@ repq_status qgemm_tc(const repq_gemm_desc& d, const EpilogueParams& ep, void* ws
   const int sms = sm_count();
   const int bn = pick_bn(d.M, d.N, sms, P.w_packed4 != 0, residual_boxes(P));
   {
-    // panels of activations of about 40 MB (a third of the L2 capacity), at least 8 row tiles
+    // panels of activations: all row tiles while the activations take at most 40 MB (a third of the L2 capacity),
+    // else about 24 MB (measured at 8192 x 4096 x 11008 with residual: 248 us with 40 MB panels, 240-242 with
+    // 12..30 MB: the weight tiles and the residual / output rows stream through the same L2), at least 8 row tiles
     const int m_tiles = (d.M + BM - 1) / BM, n_tiles = (d.N + bn - 1) / bn;
-    const int64_t fit = (int64_t(40) << 20) / (int64_t(BM) * d.K);
+    const int64_t a_bytes = int64_t(d.M) * d.K;
+    const int64_t fit = (int64_t(a_bytes <= (int64_t(40) << 20) ? 40 : 24) << 20) / (int64_t(BM) * d.K);
     int panel = int(fit < 8 ? 8 : fit);
     if (panel > m_tiles) panel = m_tiles;
     TileOrder& T = P.order;
