@@ -69,8 +69,9 @@ struct alignas(16) ColTerms {                          // per output column of a
 
 constexpr uint32_t kResBytes = 32 * 128;            // bf16 residual of one warp and tile: 32 rows x 64 columns
 
-// RES: the bf16 residual of a tile comes in by bulk tensor copies, one 32 x 64 box per epilogue warp, asked for one
-// tile ahead (the operand ring gives up a stage for the boxes)
+// RES (bf16 output with a bf16 residual, tiles of at most 192 columns): the residual of a tile comes in by bulk tensor
+// copies, one 32 x 64 box per epilogue warp, asked for one tile ahead; the output values are written over the residual
+// values they were computed from and the box leaves by one bulk tensor store (no staging buffer beside it)
 // WP: 0 = weight tiles arrive as bytes; 4 / 6 = packed (64 / 96 bytes per row of 128 codes), expanded by the converters
 template <int BN, bool RES, int WP>
 struct SharedStorage {
@@ -78,15 +79,15 @@ struct SharedStorage {
   // kStages: ring of the bulk copies (activation tile + weight tile as it arrives).  kStagesB: ring of byte weight
   // tiles the MMA reads: the same ring when the weights arrive as bytes; with packed weights a short ring of its own
   // (the hop from converter to MMA is short), which leaves room for a deeper copy ring ahead of the converters.
-  static constexpr int kStages = WP == 6 ? 4 : WP == 4 ? 5 : (RES ? 3 : 4);
+  static constexpr int kStages = WP == 6 ? 4 : WP == 4 ? 5 : 4;
   static constexpr int kPackedRow = BK * (WP ? WP : 8) / 8;        // bytes of a packed tile row
   static constexpr int kStagesB = W4 ? 2 : kStages;
   static constexpr int kEpi = W4 ? kEpiWarpsW4 : kEpiWarps;
   alignas(1024) uint8_t a[kStages][kABytes];
   alignas(1024) uint8_t b[kStagesB][BN * BK];
-  alignas(1024) uint8_t res[RES ? kEpiWarps * kResBytes : 1024];
+  alignas(1024) uint8_t res[RES ? (BN / kSliceCols) * 4 * kResBytes : 1024];   // one box per active epilogue warp
   uint64_t res_full[kEpiWarps];
-  alignas(1024) uint8_t epi[kEpi][1024];          // per-warp staging box of the epilogue's bulk stores
+  alignas(1024) uint8_t epi[RES ? 1 : kEpi][1024]; // per-warp staging box of the epilogue's bulk stores (RES: the residual box itself)
   ColTerms cols[kEpi];                            // each epilogue warp stages the terms of its own slice: no barrier
   alignas(128) uint8_t bp[W4 ? kStages : 1][W4 ? BN * kPackedRow : 128];   // packed weight tiles: unswizzled rows
   alignas(8) uint64_t full[kStages];
@@ -630,6 +631,8 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       const TileOrigin o = tile_origin(t, P.order, BN);
       const int tm0 = o.m0, tn0 = o.n0;
       if (lane == 0) {
+        // the box's last content may still be on its way out (the bulk store of the previous tile reads it)
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
         mbar_expect_tx(res_bar, kResBytes);
         tma_load_2d(res_buf, &map_res, res_bar, tn0 + cl0, tm0 + quarter * 32);
       }
@@ -802,7 +805,31 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
               continue;
             }
           }
-          emit_chunk<OUT>(&map_out, smem_u32(S.epi[ew]), lane, q, v, c, col0, m0 + quarter * 32, code_sum, direct, sat);
+          if constexpr (RES && OUT == kOutBf16) {
+            // in place: the 16 output values take the two 16-byte pieces their residual values came from
+            uint32_t w[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+              const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * k], v[2 * k + 1]);
+              w[k] = *reinterpret_cast<const uint32_t*>(&h);
+            }
+#pragma unroll
+            for (int i = 0; i < kChunk / 8; ++i) {
+              const uint32_t piece = uint32_t(c * (kChunk / 8) + i);
+              sts128(res_buf + uint32_t(lane) * 128u + ((piece ^ uint32_t(lane & 7)) << 4), w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+            }
+            if (c == kSliceChunks - 1) {
+              asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+              __syncwarp();
+              if (lane == 0) {
+                tma_store_2d(&map_out, res_buf, n0 + cl0, m0 + quarter * 32);
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+              }
+            }
+            continue;
+          }
+          if constexpr (!(RES && OUT == kOutBf16))
+            emit_chunk<OUT>(&map_out, smem_u32(S.epi[ew]), lane, q, v, c, col0, m0 + quarter * 32, code_sum, direct, sat);
         }
         }
       } else if (slice_on && any_row && n0 + cl0 < P.N) {
@@ -880,11 +907,14 @@ TcLayout tc_layout(const repq_gemm_desc& d) {
 // Whether a launch takes its bf16 residual through bulk-copied boxes (tiles of at most 192 columns, short K).
 bool residual_boxes(const TcParams& P) {
   const EpilogueParams& ep = P.ep;
-  return (ep.out_kind == REPQ_OUT_F32 || ep.out_kind == REPQ_OUT_BF16) && ep.residual != nullptr && ep.residual_bf16 &&
-         ep.acc_debug == nullptr && P.K <= 1536 && !P.w_packed4;
+  // (up to K = 3072: beyond, the main loop sets the pace, and its time per k-block does not shrink with the tile width
+  // (the operand copies in flight, four stages, against the L2 latency), so that 256-column tiles win: measured at
+  // 8192 x 4096 x 4096 101 us with 256 columns against 111 with 192, at 18464 x 1024 x 4096 67 against 79)
+  return ep.out_kind == REPQ_OUT_BF16 && ep.residual != nullptr && ep.residual_bf16 && ep.acc_debug == nullptr &&
+         ep.glu == 0 && P.K <= 3072 && !P.w_packed4;
 }
 
-int pick_bn(int M, int N, int sms, bool w_packed4, bool res_boxes) {
+int pick_bn(int M, int N, int K, int sms, bool w_packed4, bool res_boxes) {
   const int m_tiles = (M + BM - 1) / BM;
   int best = 256;
   long best_cost = -1;
@@ -892,10 +922,12 @@ int pick_bn(int M, int N, int sms, bool w_packed4, bool res_boxes) {
     if (w_packed4 && bn > kMaxBNW4) continue;
     const long tiles = long(m_tiles) * ((N + bn - 1) / bn);
     const long rounds = (tiles + sms - 1) / sms;
-    // a round costs its width plus a fixed part; where the epilogue adds a bf16 residual at short K it sets the pace
-    // alone, and a 256-column tile (residual by row-per-lane loads) takes 1.7 x the time of a narrower one whose
-    // residual box was copied in a tile ahead (measured at 18464 x 1024 x 1024: 39.6 us with 256 columns, 33.9 with 192)
-    const long cost = res_boxes ? rounds * (bn == 256 ? 95 : 55) : rounds * (bn + 160);
+    // a round costs its width plus a fixed part; where the epilogue adds a bf16 residual at short K, a round is the longer
+    // of the main loop (0.34 us per k-block) and the epilogue, and the epilogue of a 256-column tile (residual by
+    // row-per-lane loads) takes 1.7 x the time of a narrower one whose residual box was copied in a tile ahead (measured
+    // at 18464 x 1024 x 1024: 39.6 us with 256 columns, 33.9 with 192)
+    const long main_loop = 34L * ((K + BK - 1) / BK), epilogue = bn == 256 ? 950 : 550;
+    const long cost = res_boxes ? rounds * (main_loop > epilogue ? main_loop : epilogue) : rounds * (bn + 160);
     if (best_cost < 0 || cost < best_cost) { best = bn; best_cost = cost; }
   }
   return best;
@@ -921,27 +953,32 @@ repq_status make_out_map(CUtensorMap* map, const TcParams& P) {
   return REPQ_OK;
 }
 
-// Tensor map of a bf16 residual for the epilogue warps' boxes: 32 rows x 64 columns, 128-byte swizzle.
-repq_status make_res_map(CUtensorMap* map, const TcParams& P) {
+// Tensor map of a bf16 matrix (the residual, the output) for the epilogue warps' boxes: 32 rows x 64 columns, 128-byte
+// swizzle.
+repq_status make_box_map(CUtensorMap* map, const TcParams& P, const void* base, int64_t ld) {
   EncodeTiledFn fn = encode_fn();
   REPQ_REQUIRE(fn != nullptr, REPQ_CUDA_ERROR, "qgemm: cuTensorMapEncodeTiled is not available");
   const cuuint64_t dims[2] = {cuuint64_t(P.N), cuuint64_t(P.M)};
-  const cuuint64_t strides[1] = {cuuint64_t(P.ep.ld_residual) * 2};
+  const cuuint64_t strides[1] = {cuuint64_t(ld) * 2};
   const cuuint32_t box[2] = {kSliceCols, 32};
   const cuuint32_t estr[2] = {1, 1};
-  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(P.ep.residual), dims, strides, box, estr,
+  const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  REPQ_REQUIRE(r == CUDA_SUCCESS, REPQ_CUDA_ERROR, "qgemm: residual tensor map failed with code %d", int(r));
+  REPQ_REQUIRE(r == CUDA_SUCCESS, REPQ_CUDA_ERROR, "qgemm: box tensor map failed with code %d", int(r));
   return REPQ_OK;
 }
 
 template <int BN, int OUT, bool RES, int PAIR, int WP>
 repq_status launch_tc_w(const CUtensorMap& map_a, const CUtensorMap& map_b, const TcParams& P, int sms, cudaStream_t st) {
   CUtensorMap map_out, map_res;
-  REPQ_TRY(make_out_map(&map_out, P));
-  if (RES) REPQ_TRY(make_res_map(&map_res, P));
-  else map_res = map_out;                                  // not read
+  if (RES) {
+    REPQ_TRY(make_box_map(&map_res, P, P.ep.residual, P.ep.ld_residual));
+    REPQ_TRY(make_box_map(&map_out, P, P.ep.out, P.ep.ldo));
+  } else {
+    REPQ_TRY(make_out_map(&map_out, P));
+    map_res = map_out;                                     // not read
+  }
   const size_t smem = sizeof(SharedStorage<BN, RES, WP>);
   REPQ_CUDA(cudaFuncSetAttribute(qgemm_tc_kernel<BN, OUT, RES, PAIR, WP>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
   const int tiles = ((P.M + BM - 1) / BM) * ((P.N + BN - 1) / BN);
@@ -962,10 +999,9 @@ repq_status launch_tc_res(const CUtensorMap& map_a, const CUtensorMap& map_b, co
 
 template <int BN, int OUT>
 repq_status launch_tc_out(const CUtensorMap& map_a, const CUtensorMap& map_b, const TcParams& P, int sms, cudaStream_t st) {
-  // float outputs with a bf16 residual on tiles of at most 192 columns: the residual boxes fit beside three stages.
-  // Taken for short K, where the epilogue sets the pace (measured at 12608 x 768: K = 768 24 us against 27 us with
-  // row-per-lane residual loads; K = 3072 46 us against 39 us, the main loop missing its fourth stage).
-  if constexpr (BN <= 192 && (OUT == kOutF32 || OUT == kOutBf16)) {
+  // bf16 outputs with a bf16 residual on tiles of at most 192 columns: the residual boxes, which also carry the output,
+  // fit beside the four stages
+  if constexpr (BN <= 192 && OUT == kOutBf16) {
     if (residual_boxes(P))
       return launch_tc_res<BN, OUT, true>(map_a, map_b, P, sms, st);
   }
@@ -1067,7 +1103,7 @@ repq_status qgemm_tc(const repq_gemm_desc& d, const EpilogueParams& ep, void* ws
   P.direct_requant = d.out_kind == REPQ_OUT_CODES && !d.gelu && !d.residual && !d.glu;
   REPQ_REQUIRE(device_status_word() != nullptr, REPQ_CUDA_ERROR, "qgemm: device status word unavailable");
   const int sms = sm_count();
-  const int bn = pick_bn(d.M, d.N, sms, P.w_packed4 != 0, residual_boxes(P));
+  const int bn = pick_bn(d.M, d.N, d.K, sms, P.w_packed4 != 0, residual_boxes(P));
   {
     // panels of activations: all row tiles while the activations take at most 40 MB (a third of the L2 capacity),
     // else about 24 MB (measured at 8192 x 4096 x 11008 with residual: 248 us with 40 MB panels, 240-242 with
